@@ -1,0 +1,212 @@
+/*
+ * phyai.h - C ABI of the B200 (sm_100a) flow-matching action-expert denoising library.
+ *
+ * One policy request returns one H-action chunk (paper, Sec. "Task Formulation", Eq. 1:
+ * a_{t:t+H-1} = pi_theta(x_t)); for flow policies pi_theta refines an action latent over
+ * several steps.  This library is that refinement loop alone: for k = 0..n-1 the action-expert
+ * transformer is evaluated on the suffix tokens (optional robot-state token + H noisy action
+ * tokens, conditioned on the time t_k) attending to themselves and to a frozen per-layer
+ * prefix KV cache, followed by the Euler update x <- x + dt * v(x, t_k), dt = -1/n, t from 1
+ * towards 0 (Sec. "Optimization Methods", graph-replay paragraph: the prefix stays fixed over
+ * the ten Euler steps, its KV tensors are retained, the sinusoidal timestep table and each
+ * layer's AdaRMS modulation table are built before denoising, the full loop is captured in one
+ * CUDA graph).  The per-layer operators are those of the kernel-fusion paragraph: (Ada)RMSNorm,
+ * one GEMM for Q,K,V, attention of the few suffix queries over the long prefix (operator-selection
+ * paragraph), residual add, one GEMM for MLP gate and up with GeGLU fused, down projection.
+ *
+ * Conventions
+ *   - All matrices are row-major [in, out]; activations are row vectors (y = x W + b).
+ *   - "device" pointers are CUDA device memory owned by the caller; "host" pointers are ordinary
+ *     host memory.  The library never frees caller memory and keeps no caller pointer after the
+ *     work it enqueued has finished.
+ *   - Every call returns a phyai_status_t; nothing throws or aborts across the ABI.
+ *     phyai_last_error() gives a thread-local description of the last failure.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Not thread-safe per handle; one call in flight per handle; handles are independent.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point fails.
+ */
+#ifndef PHYAI_H_
+#define PHYAI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct phyai_expert phyai_expert_t; /* opaque: packed weights, tables, workspace, graphs */
+
+typedef enum {
+  PHYAI_OK = 0,
+  PHYAI_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, size out of the configured range        */
+  PHYAI_ERR_UNSUPPORTED = 2, /* a shape or mode the kernels do not cover                          */
+  PHYAI_ERR_OOM = 3,         /* device or host allocation failed                                   */
+  PHYAI_ERR_CUDA = 4,        /* a CUDA runtime call failed (message in phyai_last_error)           */
+  PHYAI_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported by phyai_poll_status) */
+} phyai_status_t;
+
+/* Storage precision of weights and prefix KV. */
+typedef enum {
+  PHYAI_F32 = 0,       /* everything float32; arithmetic in true fp32 (no TF32)                       */
+  PHYAI_BF16 = 1,      /* weights and prefix KV bfloat16; bf16 tensor-core operands, fp32 accumulate   */
+  PHYAI_W8E4M3_A16 = 2 /* the seven large per-layer matrices as e4m3 bytes with one fp32 scale per
+                          output channel (offline round-to-nearest, quantization paragraph); all other
+                          tensors and the prefix KV bfloat16; activations bf16                        */
+} phyai_dtype_t;
+
+/* How the time t_k conditions the expert. */
+typedef enum {
+  PHYAI_COND_PI0_CONCAT = 0, /* action token = swish([x Wa + ba ; tau] W1 + b1) W2 + b2; plain RMSNorm */
+  PHYAI_COND_PI05_ADARMS = 1 /* action token = x Wa + ba; c = swish(swish(tau W1+b1) W2+b2); every norm
+                                site has a dense D -> 3D (scale | shift | gate): n = rms(h)(1+scale)+shift,
+                                gate multiplies the sub-layer output before the residual add            */
+} phyai_cond_t;
+
+/* Kernel family (debug / verification aid). */
+typedef enum {
+  PHYAI_ENGINE_AUTO = 0,  /* fp32 storage -> CUDA-core path; bf16 / e4m3 -> tcgen05 tensor path */
+  PHYAI_ENGINE_SIMT = 1   /* force the CUDA-core fp32-arithmetic path for any storage type       */
+} phyai_engine_t;
+
+typedef struct {
+  uint32_t struct_size;      /* = sizeof(phyai_expert_config_t), for ABI growth                        */
+  uint32_t n_layers, width, mlp_dim, n_q_heads, n_kv_heads, head_dim;
+  uint32_t state_dim, action_dim, horizon;
+  uint32_t has_state_token;  /* 1: suffix = state token + H action tokens; 0: H action tokens          */
+  uint32_t max_prefix_len;   /* largest prefix_len of one request                                      */
+  uint32_t max_batch;        /* largest batch of phyai_denoise_batched                                 */
+  uint32_t cond;             /* phyai_cond_t                                                           */
+  uint32_t dtype;            /* phyai_dtype_t                                                          */
+  float rms_eps;             /* inside the square root                                                 */
+  float rope_theta;          /* 0 = no rotary embedding; suffix token i sits at position prefix_len+i  */
+  float time_min_period, time_max_period; /* sinusoid periods, geometric over width/2 channels         */
+  uint32_t gelu_exact;       /* 0 = tanh form, 1 = erf form                                            */
+  uint32_t suffix_block_causal; /* 0 = suffix fully bidirectional; 1 = state token sees only itself    */
+  uint32_t engine;           /* phyai_engine_t                                                         */
+} phyai_expert_config_t;
+
+/*
+ * Weights: device pointers, caller-owned, storage per `dtype` (float32 / bfloat16; for
+ * PHYAI_W8E4M3_A16 the seven per-layer matrices are uint8 e4m3 codes and `scales` is set).
+ * Per-layer members are HOST arrays of n_layers DEVICE pointers.  Members a mode does not
+ * have are NULL.  phyai_expert_create copies / repacks everything, so the caller may free its
+ * copies once the create call's stream work is complete (create synchronises before returning).
+ *
+ *   state_w [Ds,D], state_b [D]                      (has_state_token only)
+ *   action_in_w [A,D], action_in_b [D]
+ *   time_mlp1_w [2D,D] (pi0: rows 0..D-1 multiply the action embedding, rows D..2D-1 multiply tau)
+ *               [D,D]  (pi0.5), time_mlp1_b [D], time_mlp2_w [D,D], time_mlp2_b [D]
+ *   action_out_w [D,A], action_out_b [A]
+ *   final_norm: gamma [D] (gain is 1+gamma)  |  pi0.5: W_mod [D,3D], final_norm_b [3D]
+ *   wq [D,Hq*dh] wk [D,Hkv*dh] wv [D,Hkv*dh] wo [Hq*dh,D] wgate [D,F] wup [D,F] wdown [F,D]  (no biases)
+ *   norm1 / norm2: gamma [D]  |  pi0.5: W_mod [D,3D] with norm1_b / norm2_b [3D]
+ *   scales[m][l] -> float[out] for m = 0..6 (q,k,v,o,gate,up,down)
+ */
+typedef struct {
+  const void *state_w, *state_b, *action_in_w, *action_in_b;
+  const void *time_mlp1_w, *time_mlp1_b, *time_mlp2_w, *time_mlp2_b;
+  const void *action_out_w, *action_out_b, *final_norm, *final_norm_b;
+  const void *const *wq, *const *wk, *const *wv, *const *wo, *const *wgate, *const *wup, *const *wdown;
+  const void *const *norm1, *const *norm1_b, *const *norm2, *const *norm2_b;
+  const float *const *scales[7];
+} phyai_weights_t;
+
+/*
+ * Create an expert (Sec. "Architecture": the model runner owns buffers, caches and graphs; the
+ * modelling code is stateless).  Allocates packed weights, the rotary table and a workspace
+ * sized from max_batch and max_prefix_len, repacks the weights on `stream` and synchronises it.
+ * On failure *out is NULL.  Errors: INVALID_ARG (NULL, zero sizes, n_q_heads not a multiple of
+ * n_kv_heads, odd head_dim/width), UNSUPPORTED (shape outside the tensor path's tiling:
+ * width, mlp_dim, n_q_heads*head_dim must be multiples of 128 there), OOM, CUDA.
+ */
+phyai_status_t phyai_expert_create(const phyai_expert_config_t *cfg, const phyai_weights_t *weights,
+                                   void *stream, phyai_expert_t **out);
+
+/* Free everything the handle owns (synchronises the device first). NULL is ignored. */
+void phyai_expert_destroy(phyai_expert_t *h);
+
+/* Bytes of a prefix-KV buffer holding `total_prefix_tokens` tokens, layout below. 0 on bad input. */
+size_t phyai_prefix_kv_bytes(const phyai_expert_config_t *cfg, uint64_t total_prefix_tokens);
+
+/*
+ * Denoise one action chunk (graph-replay paragraph: ten Euler steps over a fixed prefix).
+ *
+ *   prefix_kv   device, layout [n_layers][2 (K,V)][kv_tokens][n_kv_heads][head_dim], head_dim
+ *               contiguous, float32 for PHYAI_F32 else bfloat16, 16-byte aligned; K is used as
+ *               given (already rotated by the producer).  kv_tokens is the token capacity of the
+ *               buffer (>= prefix_len); rows >= prefix_len are never read.
+ *   prefix_len  0 <= prefix_len <= min(kv_tokens, max_prefix_len); 0 = suffix-only attention.
+ *   state       device float32 [state_dim] (NULL iff has_state_token == 0)
+ *   noise       device float32 [horizon, action_dim]: x at t = 1
+ *   n_steps     >= 1; dt = -1/n_steps, t_k = 1 - k/n_steps
+ *   out_actions device float32 [horizon, action_dim]: x at t = 0; may alias `noise`
+ *
+ * Only enqueues work on `stream` and returns; results are valid once the stream has been
+ * synchronised.  The first call with a new n_steps builds that step count's tables (time
+ * embedding, per-step bias or modulation) and, unless disabled, captures the loop as a CUDA
+ * graph; it is slower and should be kept out of timed regions.  Errors: INVALID_ARG.
+ */
+phyai_status_t phyai_denoise(phyai_expert_t *h, const void *prefix_kv, uint64_t kv_tokens, uint32_t prefix_len,
+                             const float *state, const float *noise, uint32_t n_steps, float *out_actions,
+                             void *stream);
+
+/*
+ * Batched variant for many concurrent rollouts (Sec. "Parallel Execution": requests are
+ * independent and exchange no state).  Request b uses rows cu_prefix_lens[b] ..
+ * cu_prefix_lens[b+1]-1 of the packed prefix KV (same layout, requests concatenated along the
+ * token axis, no padding rows), its own state and noise.
+ *
+ *   batch           1 <= batch <= max_batch
+ *   prefix_kv       device, [n_layers][2][kv_tokens][n_kv_heads][head_dim]
+ *   cu_prefix_lens  device int32 [batch+1], non-decreasing, cu[0] >= 0, cu[batch] <= kv_tokens,
+ *                   every difference <= max_prefix_len (checked on the device: a violation sets
+ *                   the status word to INVALID_ARG and the call writes nothing)
+ *   states          device float32 [batch, state_dim] or NULL
+ *   noise, out      device float32 [batch, horizon, action_dim]
+ */
+phyai_status_t phyai_denoise_batched(phyai_expert_t *h, uint32_t batch, const void *prefix_kv, uint64_t kv_tokens,
+                                     const int32_t *cu_prefix_lens, const float *states, const float *noise,
+                                     uint32_t n_steps, float *out_actions, void *stream);
+
+/*
+ * Host-buffer variants: all tensor arguments (cu_prefix_lens included) are HOST pointers
+ * (pinned memory makes the copies asynchronous).  The call copies them into handle-owned
+ * device staging buffers on `stream`, runs the same kernels, and copies the actions back to
+ * `out_actions` (host).  The result is valid after the stream is synchronised.  The KV staging
+ * buffer holds max_batch * max_prefix_len tokens; kv_tokens beyond that -> INVALID_ARG.
+ */
+phyai_status_t phyai_denoise_host(phyai_expert_t *h, const void *prefix_kv, uint64_t kv_tokens, uint32_t prefix_len,
+                                  const float *state, const float *noise, uint32_t n_steps, float *out_actions,
+                                  void *stream);
+phyai_status_t phyai_denoise_batched_host(phyai_expert_t *h, uint32_t batch, const void *prefix_kv,
+                                          uint64_t kv_tokens, const int32_t *cu_prefix_lens, const float *states,
+                                          const float *noise, uint32_t n_steps, float *out_actions, void *stream);
+
+/*
+ * After the stream has been synchronised: read and clear the handle's device status word.
+ * PHYAI_OK, PHYAI_ERR_TIMEOUT (a bounded wait inside a kernel expired; results are invalid) or
+ * PHYAI_ERR_INVALID_ARG (device-side validation of cu_prefix_lens failed).  Synchronises the
+ * device copy of one word; do not call during stream capture.
+ */
+phyai_status_t phyai_poll_status(phyai_expert_t *h);
+
+/* Options. key "use_graph": 0 launches the kernels directly, 1 (default) replays a captured CUDA
+ * graph per (batch, n_steps).  key "wait_limit": iteration bound of device-side waits (testing).
+ * Unknown key -> INVALID_ARG. */
+phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t value);
+
+/* Number of kernel launches (graph nodes) one denoise call with this batch / n_steps issues;
+ * 0 if unknown.  Reporting aid for benchmarks. */
+uint64_t phyai_launches_per_call(phyai_expert_t *h, uint32_t batch, uint32_t n_steps);
+
+/* Thread-local, NUL-terminated description of the last error on this thread ("" if none). */
+const char *phyai_last_error(void);
+
+/* Library version string. */
+const char *phyai_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PHYAI_H_ */

@@ -1,0 +1,244 @@
+"""Thin ctypes binding of the C-ABI library (``include/phyai.h``): argument marshalling only.
+
+Every step of the denoising loop runs inside the CUDA library; PyTorch is used here for device
+memory and streams.  There is no CPU fallback: loading fails loudly when ``libphyai.so`` has not
+been built, and every compute call fails without a CUDA device.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libphyai.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(6)
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "OOM", 4: "CUDA", 5: "TIMEOUT"}
+DTYPES = {"f32": 0, "bf16": 1, "w8e4m3": 2}
+CONDS = {"pi0": 0, "pi05": 1}
+ENGINES = {"auto": 0, "simt": 1}
+BIG = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
+
+#: every symbol the header declares
+EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes", "phyai_denoise",
+           "phyai_denoise_batched", "phyai_denoise_host", "phyai_denoise_batched_host", "phyai_poll_status",
+           "phyai_set_option", "phyai_launches_per_call", "phyai_last_error", "phyai_version")
+
+
+class PhyaiError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"phyai status {STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class ConfigStruct(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in
+                ("struct_size", "n_layers", "width", "mlp_dim", "n_q_heads", "n_kv_heads", "head_dim", "state_dim",
+                 "action_dim", "horizon", "has_state_token", "max_prefix_len", "max_batch", "cond", "dtype")] + \
+               [(n, C.c_float) for n in ("rms_eps", "rope_theta", "time_min_period", "time_max_period")] + \
+               [(n, C.c_uint32) for n in ("gelu_exact", "suffix_block_causal", "engine")]
+
+
+_VP = C.c_void_p
+_VPP = C.POINTER(C.c_void_p)
+
+
+class WeightsStruct(C.Structure):
+    _fields_ = [(n, _VP) for n in
+                ("state_w", "state_b", "action_in_w", "action_in_b", "time_mlp1_w", "time_mlp1_b", "time_mlp2_w",
+                 "time_mlp2_b", "action_out_w", "action_out_b", "final_norm", "final_norm_b")] + \
+               [(n, _VPP) for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown",
+                                    "norm1", "norm1_b", "norm2", "norm2_b")] + \
+               [("scales", _VPP * 7)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Load ``libphyai.so`` (built by ``paper_2608_03682_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_03682_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    lib.phyai_last_error.restype = C.c_char_p
+    lib.phyai_version.restype = C.c_char_p
+    lib.phyai_prefix_kv_bytes.restype = C.c_size_t
+    lib.phyai_prefix_kv_bytes.argtypes = [C.POINTER(ConfigStruct), C.c_uint64]
+    lib.phyai_expert_create.argtypes = [C.POINTER(ConfigStruct), C.POINTER(WeightsStruct), _VP, C.POINTER(_VP)]
+    lib.phyai_expert_destroy.argtypes = [_VP]
+    lib.phyai_expert_destroy.restype = None
+    single = [_VP, _VP, C.c_uint64, C.c_uint32, _VP, _VP, C.c_uint32, _VP, _VP]
+    batched = [_VP, C.c_uint32, _VP, C.c_uint64, _VP, _VP, _VP, C.c_uint32, _VP, _VP]
+    lib.phyai_denoise.argtypes = single
+    lib.phyai_denoise_host.argtypes = single
+    lib.phyai_denoise_batched.argtypes = batched
+    lib.phyai_denoise_batched_host.argtypes = batched
+    lib.phyai_poll_status.argtypes = [_VP]
+    lib.phyai_set_option.argtypes = [_VP, C.c_char_p, C.c_int64]
+    lib.phyai_launches_per_call.argtypes = [_VP, C.c_uint32, C.c_uint32]
+    lib.phyai_launches_per_call.restype = C.c_uint64
+    _lib = lib
+    return lib
+
+
+def _check(status: int):
+    if status != OK:
+        raise PhyaiError(status, load_library().phyai_last_error().decode())
+
+
+def make_config_struct(cfg, engine: str = "auto") -> ConfigStruct:
+    s = ConfigStruct()
+    s.struct_size = C.sizeof(ConfigStruct)
+    for n in ("n_layers", "width", "mlp_dim", "n_q_heads", "n_kv_heads", "head_dim", "state_dim", "action_dim",
+              "horizon", "max_prefix_len", "max_batch"):
+        setattr(s, n, int(getattr(cfg, n)))
+    s.has_state_token = int(bool(cfg.has_state_token))
+    s.cond = CONDS[cfg.cond]
+    s.dtype = DTYPES[cfg.dtype]
+    s.rms_eps, s.rope_theta = cfg.rms_eps, cfg.rope_theta
+    s.time_min_period, s.time_max_period = cfg.time_min_period, cfg.time_max_period
+    s.gelu_exact = int(bool(cfg.gelu_exact))
+    s.suffix_block_causal = int(bool(cfg.suffix_block_causal))
+    s.engine = ENGINES[engine]
+    return s
+
+
+def prefix_kv_bytes(cfg, tokens: int) -> int:
+    s = make_config_struct(cfg)
+    return int(load_library().phyai_prefix_kv_bytes(C.byref(s), tokens))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+class Expert:
+    """One action expert on the current CUDA device.  ``weights``: name -> CUDA tensor (per-layer
+    names suffixed ``.{layer}``); for the e4m3 mode the seven big matrices are ``(codes, scales)``."""
+
+    def __init__(self, cfg, weights: Dict[str, object], engine: str = "auto", stream=None):
+        self.lib = load_library()
+        self.cfg = cfg
+        self._handle = _VP()
+        cs = make_config_struct(cfg, engine)
+        ws = WeightsStruct()
+        keep = []
+        L = cfg.n_layers
+
+        def dev(t):
+            if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+                raise ValueError("weights must be contiguous CUDA tensors")
+            keep.append(t)
+            return t.data_ptr()
+
+        for n in ("state_w", "state_b", "action_in_w", "action_in_b", "time_mlp1_w", "time_mlp1_b", "time_mlp2_w",
+                  "time_mlp2_b", "action_out_w", "action_out_b", "final_norm", "final_norm_b"):
+            if n in weights:
+                setattr(ws, n, dev(weights[n]))
+        scale_arrays = {m: (C.c_void_p * L)() for m in BIG}
+        for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown", "norm1", "norm1_b", "norm2", "norm2_b"):
+            if f"{n}.0" not in weights:
+                continue
+            arr = (C.c_void_p * L)()
+            for l in range(L):
+                w = weights[f"{n}.{l}"]
+                if isinstance(w, tuple):
+                    arr[l] = dev(w[0])
+                    scale_arrays[n][l] = dev(w[1])
+                else:
+                    arr[l] = dev(w)
+            keep.append(arr)
+            setattr(ws, n, C.cast(arr, _VPP))
+        if cfg.dtype == "w8e4m3":
+            for i, m in enumerate(BIG):
+                keep.append(scale_arrays[m])
+                ws.scales[i] = C.cast(scale_arrays[m], _VPP)
+        _check(self.lib.phyai_expert_create(C.byref(cs), C.byref(ws), _stream_ptr(stream), C.byref(self._handle)))
+        del keep  # create has repacked everything and synchronised
+
+    # ------------------------------------------------------------------------------------------
+    def close(self):
+        if getattr(self, "_handle", None) is not None and self._handle.value:
+            self.lib.phyai_expert_destroy(self._handle)
+            self._handle = _VP()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    # ------------------------------------------------------------------------------------------
+    def denoise(self, prefix_kv: torch.Tensor, prefix_len: int, state: Optional[torch.Tensor], noise: torch.Tensor,
+                n_steps: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """phyai_denoise: device tensors; ``prefix_kv`` [L,2,T,Hkv,dh]; returns ``out`` [H,A] (enqueued only)."""
+        if out is None:
+            out = torch.empty_like(noise)
+        kv_tokens = 0 if prefix_kv is None else int(prefix_kv.shape[2])
+        _check(self.lib.phyai_denoise(self._handle, _ptr(prefix_kv), kv_tokens, int(prefix_len), _ptr(state),
+                                      _ptr(noise), int(n_steps), _ptr(out), _stream_ptr(stream)))
+        return out
+
+    def denoise_batched(self, prefix_kv: torch.Tensor, cu_prefix_lens: torch.Tensor, states: Optional[torch.Tensor],
+                        noise: torch.Tensor, n_steps: int, out: Optional[torch.Tensor] = None,
+                        stream=None) -> torch.Tensor:
+        """phyai_denoise_batched: packed ``prefix_kv`` [L,2,T_total,Hkv,dh], device int32 ``cu_prefix_lens`` [B+1]."""
+        if out is None:
+            out = torch.empty_like(noise)
+        batch = int(noise.shape[0])
+        _check(self.lib.phyai_denoise_batched(self._handle, batch, _ptr(prefix_kv), int(prefix_kv.shape[2]),
+                                              _ptr(cu_prefix_lens), _ptr(states), _ptr(noise), int(n_steps), _ptr(out),
+                                              _stream_ptr(stream)))
+        return out
+
+    def denoise_host(self, prefix_kv: torch.Tensor, prefix_len: int, state, noise, n_steps: int, out: torch.Tensor,
+                     stream=None) -> torch.Tensor:
+        """phyai_denoise_host: all tensors are (ideally pinned) host tensors."""
+        _check(self.lib.phyai_denoise_host(self._handle, _ptr(prefix_kv), int(prefix_kv.shape[2]), int(prefix_len),
+                                           _ptr(state), _ptr(noise), int(n_steps), _ptr(out), _stream_ptr(stream)))
+        return out
+
+    def denoise_batched_host(self, prefix_kv, cu_prefix_lens, states, noise, n_steps: int, out, stream=None):
+        batch = int(noise.shape[0])
+        _check(self.lib.phyai_denoise_batched_host(self._handle, batch, _ptr(prefix_kv), int(prefix_kv.shape[2]),
+                                                   _ptr(cu_prefix_lens), _ptr(states), _ptr(noise), int(n_steps),
+                                                   _ptr(out), _stream_ptr(stream)))
+        return out
+
+    def poll_status(self) -> int:
+        """Read-and-clear the device status word (call after synchronising); returns the status code."""
+        return int(self.lib.phyai_poll_status(self._handle))
+
+    def set_option(self, key: str, value: int):
+        _check(self.lib.phyai_set_option(self._handle, key.encode(), int(value)))
+
+    def launches_per_call(self, batch: int, n_steps: int) -> int:
+        return int(self.lib.phyai_launches_per_call(self._handle, batch, n_steps))
+
+
+def weights_to_device(weights: Dict[str, object], device="cuda") -> Dict[str, object]:
+    """Copy a generated weight dictionary to the device (tuples element-wise)."""
+    out = {}
+    for k, v in weights.items():
+        out[k] = tuple(t.to(device).contiguous() for t in v) if isinstance(v, tuple) else v.to(device).contiguous()
+    return out

@@ -1,0 +1,725 @@
+// Host side of the C ABI: handle lifetime, weight repacking, per-step-count tables, the launch
+// sequence of one denoising loop, CUDA-graph capture and replay.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <utility>
+#include <vector>
+
+#include "../../include/phyai.h"
+#include "kernels.h"
+
+using namespace phyai;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+phyai_status_t fail(phyai_status_t code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+#define CU(call)                                                                                       \
+  do {                                                                                                 \
+    cudaError_t e_ = (call);                                                                           \
+    if (e_ != cudaSuccess)                                                                             \
+      return fail(e_ == cudaErrorMemoryAllocation ? PHYAI_ERR_OOM : PHYAI_ERR_CUDA, "%s failed: %s", #call, \
+                  cudaGetErrorString(e_));                                                             \
+  } while (0)
+
+struct Tables {             // per n_steps
+  float* tau = nullptr;     // [n][D]
+  float* tb = nullptr;      // pi0:  [n][D]  time bias of the folded action MLP
+  float* cvec = nullptr;    // pi05: [n][D]
+  float* mod = nullptr;     // pi05: [n][sites][3D]  (1+scale | shift | gate)
+};
+
+inline int kind_of(uint32_t dtype) { return dtype == PHYAI_F32 ? 0 : 1; }
+
+}  // namespace
+
+struct phyai_expert {
+  phyai_expert_config_t cfg{};
+  Dims d{};
+  bool tc = false;       // tensor-core engine
+  bool ada = false;
+  int sites = 0;
+  int Mpad = 0;
+  std::vector<void*> allocs;
+
+  // small tensors (fp32)
+  float *state_w = nullptr, *state_b = nullptr;
+  float *Wc = nullptr;        // pi0: folded [A][D];  pi05: Wa [A][D]
+  float *bcfold = nullptr;    // pi0: ba W1[0:D] + b1   pi05: ba
+  float *W1tau = nullptr;     // pi0: W1[D:2D] fp32 [D][D]; pi05: W1 [D][D]
+  float *b1 = nullptr, *W2f = nullptr, *b2 = nullptr;  // W2f: fp32 [D][D] (SIMT pi0 / pi05 table)
+  __nv_bfloat16* W2p = nullptr;                        // TC pi0: packed
+  float *Wout = nullptr, *bout = nullptr;
+  float* gains = nullptr;      // plain: [sites][D] = 1 + gamma
+  void* wmod = nullptr;        // ada: [sites][D][3D] in source storage
+  float* bmod = nullptr;       // ada: [sites][3D]
+  int wmod_kind = 0;
+
+  // big matrices
+  std::vector<float*> f_qkv, f_o, f_g, f_u, f_d;                 // SIMT fp32 row-major
+  std::vector<__nv_bfloat16*> p_qkv, p_o, p_g, p_u, p_d;         // TC packed
+  std::vector<float*> s_qkv, s_o, s_g, s_u, s_d;                 // TC per-channel scales (or null)
+
+  float2* rope = nullptr;
+
+  // workspace
+  float *h = nullptr, *qkv = nullptr, *state_tok = nullptr;
+  float *xn_f = nullptr, *attn_f = nullptr, *m_f = nullptr, *u_f = nullptr;
+  __nv_bfloat16 *xn_t = nullptr, *attn_t = nullptr, *m_t = nullptr, *u_t = nullptr;
+
+  Request* rq = nullptr;
+  int* cu_internal = nullptr;
+  int* status = nullptr;
+
+  std::map<int, Tables> tables;
+  std::map<std::pair<int, int>, cudaGraphExec_t> graphs;
+  std::map<std::pair<int, int>, uint64_t> launch_counts;
+  cudaStream_t cap_stream = nullptr;
+
+  // host-variant staging (allocated on first use)
+  void* stg_kv = nullptr; size_t stg_kv_bytes = 0;
+  float *stg_states = nullptr, *stg_noise = nullptr, *stg_out = nullptr;
+  int* stg_cu = nullptr;
+
+  int use_graph = 1;
+  unsigned wait_limit = 1u << 22;
+  uint64_t counting = 0;  // launches counted by the last enqueue
+
+  template <typename T>
+  phyai_status_t alloc(T** p, size_t count, bool zero = false) {
+    void* q = nullptr;
+    const size_t bytes = count * sizeof(T) > 0 ? count * sizeof(T) : 16;
+    cudaError_t e = cudaMalloc(&q, bytes);
+    if (e != cudaSuccess) return fail(PHYAI_ERR_OOM, "cudaMalloc(%zu bytes) failed: %s", bytes, cudaGetErrorString(e));
+    allocs.push_back(q);
+    if (zero) {
+      e = cudaMemset(q, 0, bytes);
+      if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "cudaMemset failed: %s", cudaGetErrorString(e));
+    }
+    *p = reinterpret_cast<T*>(q);
+    return PHYAI_OK;
+  }
+};
+
+#define ST(call)                         \
+  do {                                   \
+    phyai_status_t s_ = (call);          \
+    if (s_ != PHYAI_OK) return s_;       \
+  } while (0)
+
+namespace {
+
+size_t kv_elem_bytes(uint32_t dtype) { return dtype == PHYAI_F32 ? 4 : 2; }
+
+phyai_status_t check_config(const phyai_expert_config_t* c) {
+  if (!c) return fail(PHYAI_ERR_INVALID_ARG, "config is NULL");
+  if (c->struct_size != sizeof(phyai_expert_config_t))
+    return fail(PHYAI_ERR_INVALID_ARG, "config.struct_size %u != %zu", c->struct_size, sizeof(phyai_expert_config_t));
+  if (!c->n_layers || !c->width || !c->mlp_dim || !c->n_q_heads || !c->n_kv_heads || !c->head_dim || !c->action_dim ||
+      !c->horizon || !c->max_batch)
+    return fail(PHYAI_ERR_INVALID_ARG, "a size in the config is zero");
+  if (c->has_state_token > 1 || (c->has_state_token && !c->state_dim))
+    return fail(PHYAI_ERR_INVALID_ARG, "has_state_token / state_dim inconsistent");
+  if (c->n_q_heads % c->n_kv_heads) return fail(PHYAI_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
+  if ((c->head_dim & 1) || (c->width & 1)) return fail(PHYAI_ERR_INVALID_ARG, "head_dim and width must be even");
+  if (c->cond > PHYAI_COND_PI05_ADARMS || c->dtype > PHYAI_W8E4M3_A16 || c->engine > PHYAI_ENGINE_SIMT)
+    return fail(PHYAI_ERR_INVALID_ARG, "unknown cond / dtype / engine value");
+  if (!(c->rms_eps >= 0.f) || !(c->rope_theta >= 0.f) || !(c->time_min_period > 0.f) || !(c->time_max_period > 0.f))
+    return fail(PHYAI_ERR_INVALID_ARG, "rms_eps / rope_theta / time periods out of range");
+  if (c->head_dim > 256) return fail(PHYAI_ERR_UNSUPPORTED, "head_dim > 256 is not covered");
+  if ((uint64_t)c->max_batch * (c->horizon + c->has_state_token) > (1u << 22))
+    return fail(PHYAI_ERR_UNSUPPORTED, "max_batch * suffix_len too large");
+  return PHYAI_OK;
+}
+
+bool tc_shape_ok(const phyai_expert_config_t* c) {
+  const uint32_t nq = c->n_q_heads * c->head_dim, nqkv = (c->n_q_heads + 2 * c->n_kv_heads) * c->head_dim;
+  return c->width % 128 == 0 && c->mlp_dim % 128 == 0 && nq % 128 == 0 && nqkv % 128 == 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// tables for one n_steps (time grid, sinusoid, pi0 time bias / pi0.5 modulation)
+// ---------------------------------------------------------------------------------------------
+phyai_status_t build_tables(phyai_expert* h, int n, cudaStream_t st, Tables** out) {
+  auto it = h->tables.find(n);
+  if (it != h->tables.end()) {
+    *out = &it->second;
+    return PHYAI_OK;
+  }
+  if (h->tables.size() >= 16) return fail(PHYAI_ERR_UNSUPPORTED, "more than 16 distinct n_steps on one handle");
+  const int D = h->d.D;
+  Tables t;
+  ST(h->alloc(&t.tau, (size_t)n * D));
+  launch_sinusoid(t.tau, n, D, (double)h->cfg.time_min_period, (double)h->cfg.time_max_period, st);
+  if (!h->ada) {
+    ST(h->alloc(&t.tb, (size_t)n * D));
+    // tb_k = tau_k W1[D:2D] + (b1 + ba W1[0:D])
+    launch_rows_gemm(t.tau, D, h->W1tau, 0, 0, D, D, h->bcfold, nullptr, 0, t.tb, D, n, st);
+  } else {
+    float* hid = nullptr;
+    ST(h->alloc(&hid, (size_t)n * D));
+    ST(h->alloc(&t.cvec, (size_t)n * D));
+    ST(h->alloc(&t.mod, (size_t)n * h->sites * 3 * D));
+    launch_rows_gemm(t.tau, D, h->W1tau, 0, 0, D, D, h->b1, nullptr, 1, hid, D, n, st);
+    launch_rows_gemm(hid, D, h->W2f, 0, 0, D, D, h->b2, nullptr, 1, t.cvec, D, n, st);
+    const size_t wsite = (size_t)D * 3 * D * (h->wmod_kind == 0 ? 4 : 2);
+    for (int s = 0; s < h->sites; ++s)
+      launch_rows_gemm(t.cvec, D, reinterpret_cast<const uint8_t*>(h->wmod) + s * wsite, h->wmod_kind, 0, 3 * D, D,
+                       h->bmod + (size_t)s * 3 * D, nullptr, 0, t.mod + (size_t)s * 3 * D, h->sites * 3 * D, n, st);
+    launch_mod_finish(t.mod, n * h->sites, D, st);
+  }
+  CU(cudaGetLastError());
+  auto ins = h->tables.emplace(n, t);
+  *out = &ins.first->second;
+  return PHYAI_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// the loop: launches of one denoise call (x <- noise; n x [embed, L layers, head + Euler])
+// ---------------------------------------------------------------------------------------------
+int pick_nt(int M) { return M <= 64 ? 64 : (M <= 1024 ? 128 : 256); }
+
+int pick_splits(int n_tiles, int tok_tiles, int KC) {
+  int want = 148 / (n_tiles * tok_tiles);
+  int s = 1;
+  while (s * 2 <= want && s * 2 <= KC) s *= 2;
+  return s;
+}
+
+phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, cudaStream_t st) {
+  const Dims& d = h->d;
+  const int M = batch * d.S, D = d.D;
+  const int nt = pick_nt(M);
+  const int tok_tiles = (M + nt - 1) / nt;
+  const float dt = -1.0f / (float)n;
+  uint64_t cnt = 0;
+  auto site = [&](int k, int s, const float** gain, const float** shift, const float** gate) {
+    if (h->ada) {
+      const float* base = t.mod + ((size_t)k * h->sites + s) * 3 * D;
+      *gain = base, *shift = base + D, *gate = base + 2 * D;
+    } else {
+      *gain = h->gains + (size_t)s * D, *shift = nullptr, *gate = nullptr;
+    }
+  };
+  auto tc_gemm = [&](TcGemm g) -> phyai_status_t {
+    g.rows_pad = h->Mpad, g.M = g.M ? g.M : M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact;
+    cudaError_t e = launch_tc_gemm(h->status, g, nt, st);
+    if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tensor GEMM launch failed: %s", cudaGetErrorString(e));
+    ++cnt;
+    return PHYAI_OK;
+  };
+  auto simt_gemm = [&](SimtGemm g) {
+    if (!g.rows_in) g.rows_in = g.rows_out = 1 << 30, g.row_off = 0;
+    g.gelu_exact = d.gelu_exact;
+    launch_simt_gemm(h->status, g, st);
+    ++cnt;
+  };
+
+  launch_begin(h->rq, h->status, h->state_w, h->state_b, h->state_tok, d, batch, st);
+  ++cnt;
+  for (int k = 0; k < n; ++k) {
+    // ---- suffix embedding ----
+    if (!h->ada) {
+      launch_embed_pi0(h->rq, h->status, h->Wc, t.tb + (size_t)k * D, h->state_tok, h->h, h->u_f, h->u_t, h->Mpad, d,
+                       batch, st);
+      ++cnt;
+      const int rows = batch * d.H;
+      if (h->tc) {
+        TcGemm g{};
+        g.W = h->W2p, g.X = h->u_t, g.M = rows, g.N = D, g.K = D, g.epi = TC_BIAS_ROWMAP, g.bias = h->b2;
+        g.out_f32 = h->h, g.ldo = D, g.rows_in = d.H, g.rows_out = d.S, g.row_off = d.ns, g.splits = 1;
+        // token tiling of the action rows alone
+        g.rows_pad = h->Mpad, g.wait_limit = h->wait_limit;
+        cudaError_t e = launch_tc_gemm(h->status, g, pick_nt(rows), st);
+        if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tensor GEMM launch failed: %s", cudaGetErrorString(e));
+        ++cnt;
+      } else {
+        SimtGemm g{};
+        g.A = h->u_f, g.lda = D, g.B = h->W2f, g.M = rows, g.N = D, g.K = D, g.epi = EPI_STORE, g.bias = h->b2;
+        g.out = h->h, g.ldo = D, g.rows_in = d.H, g.rows_out = d.S, g.row_off = d.ns;
+        simt_gemm(g);
+      }
+    } else {
+      launch_embed_pi05(h->rq, h->status, h->Wc, h->bcfold, h->state_tok, h->h, d, batch, st);
+      ++cnt;
+    }
+    // ---- transformer layers ----
+    for (int l = 0; l < d.L; ++l) {
+      const float *gain, *shift, *gate;
+      site(k, 2 * l, &gain, &shift, &gate);
+      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st);
+      ++cnt;
+      if (h->tc) {
+        TcGemm g{};
+        g.W = h->p_qkv[l], g.X = h->xn_t, g.N = d.Nqkv, g.K = D, g.epi = TC_STORE, g.scale = h->s_qkv[l];
+        g.out_f32 = h->qkv, g.ldo = d.Nqkv, g.splits = 1;
+        ST(tc_gemm(g));
+      } else {
+        SimtGemm g{};
+        g.A = h->xn_f, g.lda = D, g.B = h->f_qkv[l], g.M = M, g.N = d.Nqkv, g.K = D, g.epi = EPI_STORE;
+        g.out = h->qkv, g.ldo = d.Nqkv;
+        simt_gemm(g);
+      }
+      launch_attention_simt(h->rq, h->status, h->qkv, h->rope, l, h->cfg.dtype != PHYAI_F32, h->attn_f, h->attn_t,
+                            h->Mpad, d, batch, st);
+      ++cnt;
+      if (h->tc) {
+        TcGemm g{};
+        g.W = h->p_o[l], g.X = h->attn_t, g.N = D, g.K = d.Nq, g.epi = TC_RESID, g.scale = h->s_o[l], g.gate = gate;
+        g.out_f32 = h->h, g.ldo = D, g.splits = pick_splits(D / 128, tok_tiles, d.Nq / 64);
+        ST(tc_gemm(g));
+      } else {
+        SimtGemm g{};
+        g.A = h->attn_f, g.lda = d.Nq, g.B = h->f_o[l], g.M = M, g.N = D, g.K = d.Nq, g.epi = EPI_RESID, g.gate = gate;
+        g.out = h->h, g.ldo = D;
+        simt_gemm(g);
+      }
+      site(k, 2 * l + 1, &gain, &shift, &gate);
+      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st);
+      ++cnt;
+      if (h->tc) {
+        TcGemm g{};
+        g.W = h->p_g[l], g.W2 = h->p_u[l], g.X = h->xn_t, g.N = d.F, g.K = D, g.epi = TC_GEGLU;
+        g.scale = h->s_g[l], g.scale2 = h->s_u[l], g.out_tiled = h->m_t, g.splits = 1;
+        ST(tc_gemm(g));
+        TcGemm g2{};
+        g2.W = h->p_d[l], g2.X = h->m_t, g2.N = D, g2.K = d.F, g2.epi = TC_RESID, g2.scale = h->s_d[l], g2.gate = gate;
+        g2.out_f32 = h->h, g2.ldo = D, g2.splits = pick_splits(D / 128, tok_tiles, d.F / 64);
+        ST(tc_gemm(g2));
+      } else {
+        SimtGemm g{};
+        g.A = h->xn_f, g.lda = D, g.B = h->f_g[l], g.B2 = h->f_u[l], g.M = M, g.N = d.F, g.K = D, g.epi = EPI_GEGLU;
+        g.out = h->m_f, g.ldo = d.F;
+        simt_gemm(g);
+        SimtGemm g2{};
+        g2.A = h->m_f, g2.lda = d.F, g2.B = h->f_d[l], g2.M = M, g2.N = D, g2.K = d.F, g2.epi = EPI_RESID, g2.gate = gate;
+        g2.out = h->h, g2.ldo = D;
+        simt_gemm(g2);
+      }
+    }
+    // ---- final norm, velocity head, Euler update ----
+    const float *gain, *shift, *gate;
+    site(k, 2 * d.L, &gain, &shift, &gate);
+    launch_final(h->rq, h->status, h->h, gain, shift, h->Wout, h->bout, dt, d, batch, st);
+    ++cnt;
+  }
+  h->counting = cnt;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return PHYAI_OK;
+}
+
+phyai_status_t run(phyai_expert* h, const Request& r, int n, cudaStream_t st) {
+  Tables* t = nullptr;
+  ST(build_tables(h, n, st, &t));
+  launch_set_request(h->rq, r, h->cu_internal, st);
+  if (r.cu_lens != nullptr) launch_validate(h->rq, h->status, (int)h->cfg.max_prefix_len, st);
+  const auto key = std::make_pair(r.batch, n);
+  if (!h->use_graph) {
+    ST(enqueue_loop(h, r.batch, n, *t, st));
+    h->launch_counts[key] = h->counting;
+    return PHYAI_OK;
+  }
+  auto it = h->graphs.find(key);
+  if (it == h->graphs.end()) {
+    if (h->graphs.size() >= 64) return fail(PHYAI_ERR_UNSUPPORTED, "more than 64 captured (batch, n_steps) graphs");
+    // tables were enqueued on `st`; the capture stream must not run ahead of them on first replay,
+    // which holds because the graph is launched on `st` below.
+    cudaGraph_t graph = nullptr;
+    CU(cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal));
+    phyai_status_t s = enqueue_loop(h, r.batch, n, *t, h->cap_stream);
+    cudaError_t e = cudaStreamEndCapture(h->cap_stream, &graph);
+    if (s != PHYAI_OK) {
+      if (graph) cudaGraphDestroy(graph);
+      return s;
+    }
+    if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "graph capture failed: %s", cudaGetErrorString(e));
+    cudaGraphExec_t exec = nullptr;
+    e = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "graph instantiate failed: %s", cudaGetErrorString(e));
+    it = h->graphs.emplace(key, exec).first;
+    h->launch_counts[key] = h->counting;
+  }
+  CU(cudaGraphLaunch(it->second, st));
+  return PHYAI_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+phyai_status_t check_call(phyai_expert* h, const void* kv, uint64_t kv_tokens, const float* noise, uint32_t n_steps,
+                          const float* out, const float* states) {
+  if (!h) return fail(PHYAI_ERR_INVALID_ARG, "handle is NULL");
+  if (!noise || !out) return fail(PHYAI_ERR_INVALID_ARG, "noise / out_actions is NULL");
+  if (n_steps == 0 || n_steps > 1000) return fail(PHYAI_ERR_INVALID_ARG, "n_steps must be in 1..1000");
+  if (kv_tokens > 0 && !kv) return fail(PHYAI_ERR_INVALID_ARG, "prefix_kv is NULL with kv_tokens > 0");
+  if (kv && !aligned16(kv)) return fail(PHYAI_ERR_INVALID_ARG, "prefix_kv must be 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(noise) & 3u) || (reinterpret_cast<uintptr_t>(out) & 3u))
+    return fail(PHYAI_ERR_INVALID_ARG, "noise / out_actions must be 4-byte aligned");
+  if (h->cfg.has_state_token && !states) return fail(PHYAI_ERR_INVALID_ARG, "state is NULL but the expert has a state token");
+  return PHYAI_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+const char* phyai_last_error(void) { return g_err; }
+const char* phyai_version(void) { return "phyai-b200 0.1 (sm_100a)"; }
+
+size_t phyai_prefix_kv_bytes(const phyai_expert_config_t* c, uint64_t tokens) {
+  if (!c || !c->n_layers || !c->n_kv_heads || !c->head_dim) return 0;
+  return (size_t)c->n_layers * 2 * tokens * c->n_kv_heads * c->head_dim * kv_elem_bytes(c->dtype);
+}
+
+phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai_weights_t* w, void* stream,
+                                   phyai_expert_t** out) {
+  if (!out) return fail(PHYAI_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  ST(check_config(cfg));
+  if (!w) return fail(PHYAI_ERR_INVALID_ARG, "weights is NULL");
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0)
+    return fail(PHYAI_ERR_CUDA, "no CUDA device: this library has no CPU fallback");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+  const bool ada = cfg->cond == PHYAI_COND_PI05_ADARMS;
+  const bool tc = cfg->dtype != PHYAI_F32 && cfg->engine != PHYAI_ENGINE_SIMT;
+  if (tc && !tc_shape_ok(cfg))
+    return fail(PHYAI_ERR_UNSUPPORTED, "tensor path needs width, mlp_dim, q and qkv widths to be multiples of 128");
+  // required pointers
+  const bool need_state = cfg->has_state_token != 0;
+  if (!w->action_in_w || !w->action_in_b || !w->time_mlp1_w || !w->time_mlp1_b || !w->time_mlp2_w || !w->time_mlp2_b ||
+      !w->action_out_w || !w->action_out_b || !w->final_norm || (ada && !w->final_norm_b) ||
+      (need_state && (!w->state_w || !w->state_b)) || !w->wq || !w->wk || !w->wv || !w->wo || !w->wgate || !w->wup ||
+      !w->wdown || !w->norm1 || !w->norm2 || (ada && (!w->norm1_b || !w->norm2_b)))
+    return fail(PHYAI_ERR_INVALID_ARG, "a required weight pointer is NULL");
+  for (uint32_t l = 0; l < cfg->n_layers; ++l)
+    if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->wgate[l] || !w->wup[l] || !w->wdown[l] || !w->norm1[l] ||
+        !w->norm2[l] || (ada && (!w->norm1_b[l] || !w->norm2_b[l])))
+      return fail(PHYAI_ERR_INVALID_ARG, "a per-layer weight pointer is NULL (layer %u)", l);
+  const bool w8 = cfg->dtype == PHYAI_W8E4M3_A16;
+  if (w8)
+    for (int m = 0; m < 7; ++m) {
+      if (!w->scales[m]) return fail(PHYAI_ERR_INVALID_ARG, "scales[%d] is NULL", m);
+      for (uint32_t l = 0; l < cfg->n_layers; ++l)
+        if (!w->scales[m][l]) return fail(PHYAI_ERR_INVALID_ARG, "scales[%d][%u] is NULL", m, l);
+    }
+
+  phyai_expert* h = new (std::nothrow) phyai_expert();
+  if (!h) return fail(PHYAI_ERR_OOM, "host allocation failed");
+  h->cfg = *cfg;
+  h->tc = tc, h->ada = ada;
+  Dims& d = h->d;
+  d.L = cfg->n_layers, d.D = cfg->width, d.F = cfg->mlp_dim, d.Hq = cfg->n_q_heads, d.Hkv = cfg->n_kv_heads;
+  d.dh = cfg->head_dim, d.Ds = cfg->state_dim, d.A = cfg->action_dim, d.H = cfg->horizon, d.ns = cfg->has_state_token;
+  d.S = d.H + d.ns, d.Nq = d.Hq * d.dh, d.Nqkv = (d.Hq + 2 * d.Hkv) * d.dh;
+  d.eps = cfg->rms_eps, d.gelu_exact = cfg->gelu_exact, d.block_causal = cfg->suffix_block_causal;
+  h->sites = 2 * d.L + 1;
+  h->Mpad = (int)(((size_t)cfg->max_batch * d.S + 255) / 256 * 256);
+  const int D = d.D, L = d.L, kind = kind_of(cfg->dtype);     // storage of non-quantised tensors
+  const int big_kind = w8 ? 2 : kind;                         // storage of the seven big matrices
+  const size_t Mp = h->Mpad;
+
+  auto body = [&]() -> phyai_status_t {
+    if (tc) CU(tc_gemm_setup());
+    CU(cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking));
+    ST(h->alloc(&h->status, 1, true));
+    ST(h->alloc(&h->cu_internal, 2, true));
+    ST(h->alloc(&h->rq, 1, true));
+    // ---- small tensors -> fp32 ----
+    if (need_state) {
+      ST(h->alloc(&h->state_w, (size_t)d.Ds * D));
+      ST(h->alloc(&h->state_b, D));
+      launch_to_f32(w->state_w, kind, h->state_w, (size_t)d.Ds * D, st);
+      launch_to_f32(w->state_b, kind, h->state_b, D, st);
+    }
+    ST(h->alloc(&h->Wout, (size_t)D * d.A));
+    ST(h->alloc(&h->bout, d.A));
+    launch_to_f32(w->action_out_w, kind, h->Wout, (size_t)D * d.A, st);
+    launch_to_f32(w->action_out_b, kind, h->bout, d.A, st);
+    ST(h->alloc(&h->b1, D));
+    ST(h->alloc(&h->b2, D));
+    launch_to_f32(w->time_mlp1_b, kind, h->b1, D, st);
+    launch_to_f32(w->time_mlp2_b, kind, h->b2, D, st);
+    ST(h->alloc(&h->Wc, (size_t)d.A * D));
+    ST(h->alloc(&h->bcfold, D));
+    ST(h->alloc(&h->W1tau, (size_t)D * D));
+    float *Wa = nullptr, *ba = nullptr;
+    ST(h->alloc(&Wa, (size_t)d.A * D));
+    ST(h->alloc(&ba, D));
+    launch_to_f32(w->action_in_w, kind, Wa, (size_t)d.A * D, st);
+    launch_to_f32(w->action_in_b, kind, ba, D, st);
+    const size_t esz = kind == 0 ? 4 : 2;
+    if (!ada) {
+      // fold the action projection into the first MLP layer: Wc = Wa W1[0:D], bcfold = ba W1[0:D] + b1
+      launch_rows_gemm(Wa, D, w->time_mlp1_w, kind, 0, D, D, nullptr, nullptr, 0, h->Wc, D, d.A, st);
+      launch_rows_gemm(ba, D, w->time_mlp1_w, kind, 0, D, D, h->b1, nullptr, 0, h->bcfold, D, 1, st);
+      launch_to_f32(reinterpret_cast<const uint8_t*>(w->time_mlp1_w) + (size_t)D * D * esz, kind, h->W1tau,
+                    (size_t)D * D, st);
+      if (tc) {
+        ST(h->alloc(&h->W2p, (size_t)D * D));
+        launch_pack_tiled(w->time_mlp2_w, kind, h->W2p, D, D, 0, st);
+      } else {
+        ST(h->alloc(&h->W2f, (size_t)D * D));
+        launch_to_f32(w->time_mlp2_w, kind, h->W2f, (size_t)D * D, st);
+      }
+    } else {
+      CU(cudaMemcpyAsync(h->Wc, Wa, (size_t)d.A * D * 4, cudaMemcpyDeviceToDevice, st));
+      CU(cudaMemcpyAsync(h->bcfold, ba, (size_t)D * 4, cudaMemcpyDeviceToDevice, st));
+      launch_to_f32(w->time_mlp1_w, kind, h->W1tau, (size_t)D * D, st);
+      ST(h->alloc(&h->W2f, (size_t)D * D));
+      launch_to_f32(w->time_mlp2_w, kind, h->W2f, (size_t)D * D, st);
+    }
+    // ---- norm parameters ----
+    if (!ada) {
+      ST(h->alloc(&h->gains, (size_t)h->sites * D));
+      float* tmp = nullptr;
+      ST(h->alloc(&tmp, D));
+      for (int s = 0; s < h->sites; ++s) {
+        const void* src = s == 2 * L ? w->final_norm : (s & 1 ? w->norm2[s / 2] : w->norm1[s / 2]);
+        launch_to_f32(src, kind, tmp, D, st);
+        launch_one_plus(tmp, h->gains + (size_t)s * D, D, st);
+      }
+    } else {
+      h->wmod_kind = kind;
+      const size_t wsite = (size_t)D * 3 * D * esz;
+      uint8_t* wm = nullptr;
+      ST(h->alloc(&wm, wsite * h->sites));
+      h->wmod = wm;
+      ST(h->alloc(&h->bmod, (size_t)h->sites * 3 * D));
+      for (int s = 0; s < h->sites; ++s) {
+        const void* src = s == 2 * L ? w->final_norm : (s & 1 ? w->norm2[s / 2] : w->norm1[s / 2]);
+        const void* bsrc = s == 2 * L ? w->final_norm_b : (s & 1 ? w->norm2_b[s / 2] : w->norm1_b[s / 2]);
+        CU(cudaMemcpyAsync(wm + s * wsite, src, wsite, cudaMemcpyDeviceToDevice, st));
+        launch_to_f32(bsrc, kind, h->bmod + (size_t)s * 3 * D, (size_t)3 * D, st);
+      }
+    }
+    // ---- the seven big matrices per layer ----
+    const int Nq = d.Nq, Nkv = d.Hkv * d.dh, Nqkv = d.Nqkv, F = d.F;
+    for (int l = 0; l < L; ++l) {
+      const float* sq = w8 ? w->scales[0][l] : nullptr; const float* sk = w8 ? w->scales[1][l] : nullptr;
+      const float* sv = w8 ? w->scales[2][l] : nullptr; const float* so = w8 ? w->scales[3][l] : nullptr;
+      const float* sg = w8 ? w->scales[4][l] : nullptr; const float* su = w8 ? w->scales[5][l] : nullptr;
+      const float* sd = w8 ? w->scales[6][l] : nullptr;
+      if (tc) {
+        __nv_bfloat16 *pq, *po, *pg, *pu, *pd;
+        ST(h->alloc(&pq, (size_t)D * Nqkv)); ST(h->alloc(&po, (size_t)Nq * D));
+        ST(h->alloc(&pg, (size_t)D * F)); ST(h->alloc(&pu, (size_t)D * F)); ST(h->alloc(&pd, (size_t)F * D));
+        launch_pack_tiled(w->wq[l], big_kind, pq, D, Nq, 0, st);
+        launch_pack_tiled(w->wk[l], big_kind, pq, D, Nkv, Nq, st);
+        launch_pack_tiled(w->wv[l], big_kind, pq, D, Nkv, Nq + Nkv, st);
+        launch_pack_tiled(w->wo[l], big_kind, po, Nq, D, 0, st);
+        launch_pack_tiled(w->wgate[l], big_kind, pg, D, F, 0, st);
+        launch_pack_tiled(w->wup[l], big_kind, pu, D, F, 0, st);
+        launch_pack_tiled(w->wdown[l], big_kind, pd, F, D, 0, st);
+        h->p_qkv.push_back(pq), h->p_o.push_back(po), h->p_g.push_back(pg), h->p_u.push_back(pu), h->p_d.push_back(pd);
+        float *cq = nullptr, *co = nullptr, *cg = nullptr, *cu = nullptr, *cd = nullptr;
+        if (w8) {
+          ST(h->alloc(&cq, Nqkv)); ST(h->alloc(&co, D)); ST(h->alloc(&cg, F)); ST(h->alloc(&cu, F)); ST(h->alloc(&cd, D));
+          CU(cudaMemcpyAsync(cq, sq, (size_t)Nq * 4, cudaMemcpyDeviceToDevice, st));
+          CU(cudaMemcpyAsync(cq + Nq, sk, (size_t)Nkv * 4, cudaMemcpyDeviceToDevice, st));
+          CU(cudaMemcpyAsync(cq + Nq + Nkv, sv, (size_t)Nkv * 4, cudaMemcpyDeviceToDevice, st));
+          CU(cudaMemcpyAsync(co, so, (size_t)D * 4, cudaMemcpyDeviceToDevice, st));
+          CU(cudaMemcpyAsync(cg, sg, (size_t)F * 4, cudaMemcpyDeviceToDevice, st));
+          CU(cudaMemcpyAsync(cu, su, (size_t)F * 4, cudaMemcpyDeviceToDevice, st));
+          CU(cudaMemcpyAsync(cd, sd, (size_t)D * 4, cudaMemcpyDeviceToDevice, st));
+        }
+        h->s_qkv.push_back(cq), h->s_o.push_back(co), h->s_g.push_back(cg), h->s_u.push_back(cu), h->s_d.push_back(cd);
+      } else {
+        float *fq, *fo, *fg, *fu, *fd;
+        ST(h->alloc(&fq, (size_t)D * Nqkv)); ST(h->alloc(&fo, (size_t)Nq * D));
+        ST(h->alloc(&fg, (size_t)D * F)); ST(h->alloc(&fu, (size_t)D * F)); ST(h->alloc(&fd, (size_t)F * D));
+        launch_copy_cols(w->wq[l], big_kind, sq, fq, D, Nq, Nqkv, 0, st);
+        launch_copy_cols(w->wk[l], big_kind, sk, fq, D, Nkv, Nqkv, Nq, st);
+        launch_copy_cols(w->wv[l], big_kind, sv, fq, D, Nkv, Nqkv, Nq + Nkv, st);
+        launch_copy_cols(w->wo[l], big_kind, so, fo, Nq, D, D, 0, st);
+        launch_copy_cols(w->wgate[l], big_kind, sg, fg, D, F, F, 0, st);
+        launch_copy_cols(w->wup[l], big_kind, su, fu, D, F, F, 0, st);
+        launch_copy_cols(w->wdown[l], big_kind, sd, fd, F, D, D, 0, st);
+        h->f_qkv.push_back(fq), h->f_o.push_back(fo), h->f_g.push_back(fg), h->f_u.push_back(fu), h->f_d.push_back(fd);
+      }
+    }
+    // ---- rotary table ----
+    if (cfg->rope_theta > 0.f) {
+      const int npos = (int)cfg->max_prefix_len + d.S;
+      ST(h->alloc(&h->rope, (size_t)npos * (d.dh / 2)));
+      launch_rope_table(h->rope, npos, d.dh, (double)cfg->rope_theta, st);
+    }
+    // ---- workspace (zeroed: padding rows of the tiled buffers stay finite) ----
+    ST(h->alloc(&h->h, Mp * D, true));
+    ST(h->alloc(&h->qkv, Mp * Nqkv, true));
+    ST(h->alloc(&h->state_tok, (size_t)cfg->max_batch * D, true));
+    if (tc) {
+      ST(h->alloc(&h->xn_t, Mp * D, true));
+      ST(h->alloc(&h->attn_t, Mp * Nq, true));
+      ST(h->alloc(&h->m_t, Mp * F, true));
+      if (!ada) ST(h->alloc(&h->u_t, Mp * D, true));
+    } else {
+      ST(h->alloc(&h->xn_f, Mp * D, true));
+      ST(h->alloc(&h->attn_f, Mp * Nq, true));
+      ST(h->alloc(&h->m_f, Mp * F, true));
+      if (!ada) ST(h->alloc(&h->u_f, Mp * D, true));
+    }
+    CU(cudaGetLastError());
+    CU(cudaStreamSynchronize(st));
+    CU(cudaDeviceSynchronize());  // the zero-fills above ran on the default stream
+    return PHYAI_OK;
+  };
+  phyai_status_t s = body();
+  if (s != PHYAI_OK) {
+    char keep[sizeof(g_err)];
+    memcpy(keep, g_err, sizeof(keep));
+    phyai_expert_destroy(h);
+    memcpy(g_err, keep, sizeof(keep));
+    return s;
+  }
+  *out = h;
+  return PHYAI_OK;
+}
+
+void phyai_expert_destroy(phyai_expert_t* h) {
+  if (!h) return;
+  cudaDeviceSynchronize();
+  for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+  if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
+  for (void* p : h->allocs) cudaFree(p);
+  delete h;
+}
+
+phyai_status_t phyai_denoise(phyai_expert_t* h, const void* prefix_kv, uint64_t kv_tokens, uint32_t prefix_len,
+                             const float* state, const float* noise, uint32_t n_steps, float* out, void* stream) {
+  ST(check_call(h, prefix_kv, kv_tokens, noise, n_steps, out, state));
+  if (prefix_len > h->cfg.max_prefix_len || prefix_len > kv_tokens)
+    return fail(PHYAI_ERR_INVALID_ARG, "prefix_len %u exceeds max_prefix_len %u or kv_tokens %llu", prefix_len,
+                h->cfg.max_prefix_len, (unsigned long long)kv_tokens);
+  Request r{};
+  r.prefix_kv = prefix_kv, r.kv_tokens = kv_tokens, r.cu_lens = nullptr, r.states = state, r.noise = noise, r.x = out;
+  r.batch = 1, r.single_len = (int)prefix_len;
+  return run(h, r, (int)n_steps, reinterpret_cast<cudaStream_t>(stream));
+}
+
+phyai_status_t phyai_denoise_batched(phyai_expert_t* h, uint32_t batch, const void* prefix_kv, uint64_t kv_tokens,
+                                     const int32_t* cu, const float* states, const float* noise, uint32_t n_steps,
+                                     float* out, void* stream) {
+  ST(check_call(h, prefix_kv, kv_tokens, noise, n_steps, out, states));
+  if (batch == 0 || batch > h->cfg.max_batch)
+    return fail(PHYAI_ERR_INVALID_ARG, "batch %u outside 1..max_batch (%u)", batch, h->cfg.max_batch);
+  if (!cu) return fail(PHYAI_ERR_INVALID_ARG, "cu_prefix_lens is NULL");
+  if (kv_tokens > (uint64_t)INT32_MAX) return fail(PHYAI_ERR_INVALID_ARG, "kv_tokens exceeds int32 range");
+  Request r{};
+  r.prefix_kv = prefix_kv, r.kv_tokens = kv_tokens, r.cu_lens = cu, r.states = states, r.noise = noise, r.x = out;
+  r.batch = (int)batch, r.single_len = 0;
+  return run(h, r, (int)n_steps, reinterpret_cast<cudaStream_t>(stream));
+}
+
+static phyai_status_t ensure_staging(phyai_expert* h) {
+  if (h->stg_noise) return PHYAI_OK;
+  const size_t B = h->cfg.max_batch;
+  h->stg_kv_bytes = phyai_prefix_kv_bytes(&h->cfg, (uint64_t)B * h->cfg.max_prefix_len);
+  uint8_t* kv = nullptr;
+  ST(h->alloc(&kv, h->stg_kv_bytes));
+  h->stg_kv = kv;
+  ST(h->alloc(&h->stg_states, B * (h->d.Ds ? h->d.Ds : 1)));
+  ST(h->alloc(&h->stg_out, B * h->d.H * h->d.A));
+  ST(h->alloc(&h->stg_cu, B + 1));
+  ST(h->alloc(&h->stg_noise, B * h->d.H * h->d.A));
+  return PHYAI_OK;
+}
+
+phyai_status_t phyai_denoise_batched_host(phyai_expert_t* h, uint32_t batch, const void* prefix_kv, uint64_t kv_tokens,
+                                          const int32_t* cu, const float* states, const float* noise, uint32_t n_steps,
+                                          float* out, void* stream) {
+  ST(check_call(h, prefix_kv, kv_tokens, noise, n_steps, out, states));
+  if (batch == 0 || batch > h->cfg.max_batch)
+    return fail(PHYAI_ERR_INVALID_ARG, "batch %u outside 1..max_batch (%u)", batch, h->cfg.max_batch);
+  if (!cu) return fail(PHYAI_ERR_INVALID_ARG, "cu_prefix_lens is NULL");
+  if (kv_tokens > (uint64_t)h->cfg.max_batch * h->cfg.max_prefix_len)
+    return fail(PHYAI_ERR_INVALID_ARG, "kv_tokens exceeds the staging capacity max_batch * max_prefix_len");
+  ST(ensure_staging(h));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const size_t kvb = phyai_prefix_kv_bytes(&h->cfg, kv_tokens), ha = (size_t)batch * h->d.H * h->d.A * 4;
+  if (kvb) CU(cudaMemcpyAsync(h->stg_kv, prefix_kv, kvb, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(h->stg_cu, cu, (size_t)(batch + 1) * 4, cudaMemcpyHostToDevice, st));
+  if (states) CU(cudaMemcpyAsync(h->stg_states, states, (size_t)batch * h->d.Ds * 4, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(h->stg_noise, noise, ha, cudaMemcpyHostToDevice, st));
+  Request r{};
+  r.prefix_kv = h->stg_kv, r.kv_tokens = kv_tokens, r.cu_lens = h->stg_cu, r.states = states ? h->stg_states : nullptr;
+  r.noise = h->stg_noise, r.x = h->stg_out, r.batch = (int)batch, r.single_len = 0;
+  ST(run(h, r, (int)n_steps, st));
+  CU(cudaMemcpyAsync(out, h->stg_out, ha, cudaMemcpyDeviceToHost, st));
+  return PHYAI_OK;
+}
+
+phyai_status_t phyai_denoise_host(phyai_expert_t* h, const void* prefix_kv, uint64_t kv_tokens, uint32_t prefix_len,
+                                  const float* state, const float* noise, uint32_t n_steps, float* out, void* stream) {
+  if (!h) return fail(PHYAI_ERR_INVALID_ARG, "handle is NULL");
+  if (prefix_len > h->cfg.max_prefix_len || prefix_len > kv_tokens)
+    return fail(PHYAI_ERR_INVALID_ARG, "prefix_len %u exceeds max_prefix_len %u or kv_tokens %llu", prefix_len,
+                h->cfg.max_prefix_len, (unsigned long long)kv_tokens);
+  ST(check_call(h, prefix_kv, kv_tokens, noise, n_steps, out, state));
+  ST(ensure_staging(h));
+  if (kv_tokens > (uint64_t)h->cfg.max_batch * h->cfg.max_prefix_len)
+    return fail(PHYAI_ERR_INVALID_ARG, "kv_tokens exceeds the staging capacity max_batch * max_prefix_len");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const size_t kvb = phyai_prefix_kv_bytes(&h->cfg, kv_tokens), ha = (size_t)h->d.H * h->d.A * 4;
+  if (kvb) CU(cudaMemcpyAsync(h->stg_kv, prefix_kv, kvb, cudaMemcpyHostToDevice, st));
+  if (state) CU(cudaMemcpyAsync(h->stg_states, state, (size_t)h->d.Ds * 4, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(h->stg_noise, noise, ha, cudaMemcpyHostToDevice, st));
+  Request r{};
+  r.prefix_kv = h->stg_kv, r.kv_tokens = kv_tokens, r.cu_lens = nullptr, r.states = state ? h->stg_states : nullptr;
+  r.noise = h->stg_noise, r.x = h->stg_out, r.batch = 1, r.single_len = (int)prefix_len;
+  ST(run(h, r, (int)n_steps, st));
+  CU(cudaMemcpyAsync(out, h->stg_out, ha, cudaMemcpyDeviceToHost, st));
+  return PHYAI_OK;
+}
+
+phyai_status_t phyai_poll_status(phyai_expert_t* h) {
+  if (!h) return fail(PHYAI_ERR_INVALID_ARG, "handle is NULL");
+  int v = 0;
+  CU(cudaMemcpy(&v, h->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (v != 0) {
+    CU(cudaMemset(h->status, 0, sizeof(int)));
+    if (v == ST_TIMEOUT) return fail(PHYAI_ERR_TIMEOUT, "a bounded device-side wait expired; results are invalid");
+    return fail(PHYAI_ERR_INVALID_ARG, "device-side validation of cu_prefix_lens failed; nothing was written");
+  }
+  return PHYAI_OK;
+}
+
+phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t value) {
+  if (!h || !key) return fail(PHYAI_ERR_INVALID_ARG, "handle or key is NULL");
+  if (!strcmp(key, "use_graph")) {
+    h->use_graph = value != 0;
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "wait_limit")) {
+    if (value < 1 || value > (int64_t)0x7fffffff) return fail(PHYAI_ERR_INVALID_ARG, "wait_limit out of range");
+    h->wait_limit = (unsigned)value;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);  // the limit is baked into captured launches
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  return fail(PHYAI_ERR_INVALID_ARG, "unknown option '%s'", key);
+}
+
+uint64_t phyai_launches_per_call(phyai_expert_t* h, uint32_t batch, uint32_t n_steps) {
+  if (!h) return 0;
+  auto it = h->launch_counts.find(std::make_pair((int)batch, (int)n_steps));
+  return it == h->launch_counts.end() ? 0 : it->second + 1 /* request-block kernel */;
+}
+
+}  // extern "C"

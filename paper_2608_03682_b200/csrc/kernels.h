@@ -1,0 +1,97 @@
+// Host-callable launchers of every kernel family.  Each launcher only enqueues on `st`.
+#pragma once
+
+#include "common.cuh"
+
+namespace phyai {
+
+struct Dims {
+  int L, D, F, Hq, Hkv, dh, Ds, A, H, ns, S, Nqkv, Nq;
+  float eps;
+  int gelu_exact, block_causal;
+};
+
+// ---- request block ---------------------------------------------------------------------------
+void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st);
+void launch_validate(const Request* rq, int* status, int max_prefix, cudaStream_t st);
+
+// ---- one-off table / packing kernels (CUDA cores, fp64 accumulation where cheap) ---------------
+// src_kind: 0 = float32, 1 = bfloat16, 2 = e4m3 byte codes
+void launch_to_f32(const void* src, int src_kind, float* dst, size_t n, cudaStream_t st);
+// dst[r][col_off + c] = src[r][c] * (scale ? scale[c] : 1)
+void launch_copy_cols(const void* src, int src_kind, const float* scale, float* dst, int rows, int cols, int ld_dst,
+                      int col_off, cudaStream_t st);
+// [in=K][out=N] source -> 128x64 blocks of the 128-byte-swizzled K-major bf16 image, out channel
+// n stored at packed row n_off + n of a matrix with KC = K/64 column chunks.
+void launch_pack_tiled(const void* src, int src_kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st);
+// Y[r][n] = act( sum_d X[r][d] * W[(w_row_off + d)][n] + bias[n] + add[n] ), r < R
+void launch_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K, const float* bias,
+                      const float* add, int act_swish, float* Y, int ldy, int R, cudaStream_t st);
+void launch_sinusoid(float* tau, int n_steps, int D, double min_period, double max_period, cudaStream_t st);
+void launch_rope_table(float2* tab, int n_pos, int dh, double theta, cudaStream_t st);
+// gains[d] = 1 + gamma[d]
+void launch_one_plus(const float* gamma, float* out, int n, cudaStream_t st);
+// mod rows [R][3D] (scale|shift|gate) -> in place (1+scale|shift|gate)
+void launch_mod_finish(float* mod, int R, int D, cudaStream_t st);
+
+// ---- per-call / per-step small kernels ---------------------------------------------------------
+void launch_begin(const Request* rq, const int* status, const float* Ws, const float* bs, float* state_tok,
+                  const Dims& d, int batch, cudaStream_t st);
+// pi0: u[r][n] = swish(x[r] . Wc[:,n] + tb[n]) for the B*H action rows (+ state rows of h)
+void launch_embed_pi0(const Request* rq, const int* status, const float* Wc, const float* tb, const float* state_tok,
+                      float* h, float* u_f32, __nv_bfloat16* u_tiled, int rows_pad, const Dims& d, int batch,
+                      cudaStream_t st);
+// pi0.5: h[b*S+ns+i][n] = x . Wa[:,n] + ba[n] (+ state rows)
+void launch_embed_pi05(const Request* rq, const int* status, const float* Wa, const float* ba, const float* state_tok,
+                       float* h, const Dims& d, int batch, cudaStream_t st);
+// n = h * rsqrt(mean h^2 + eps) * gain + shift  -> fp32 row-major or tiled bf16
+void launch_rmsnorm(const int* status, const float* h, const float* gain, const float* shift, float* out_f32,
+                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st);
+// final norm -> out-proj -> Euler update x += dt * (v + bout)
+void launch_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
+                  const float* Wout, const float* bout, float dt, const Dims& d, int batch, cudaStream_t st);
+
+// ---- CUDA-core GEMM (fp32 FMA) -----------------------------------------------------------------
+enum : int { EPI_STORE = 0, EPI_SWISH = 1, EPI_RESID = 2, EPI_GEGLU = 3 };
+struct SimtGemm {
+  const float* A; int lda;        // [M][K] row-major
+  const float* B; const float* B2;  // [K][N] row-major (B2: "up" matrix of GeGLU)
+  int M, N, K;
+  int epi;
+  const float* bias;              // [N] or null (STORE / SWISH)
+  const float* gate;              // [N] or null (RESID)
+  float* out; int ldo;
+  int rows_in, rows_out, row_off; // output row = (m / rows_in) * rows_out + row_off + m % rows_in
+  int gelu_exact;
+};
+void launch_simt_gemm(const int* status, const SimtGemm& g, cudaStream_t st);
+
+// ---- CUDA-core attention -----------------------------------------------------------------------
+void launch_attention_simt(const Request* rq, const int* status, const float* qkv, const float2* rope, int layer,
+                           int kv_is_bf16, float* out_f32, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
+                           int batch, cudaStream_t st);
+
+// ---- tcgen05 GEMM ------------------------------------------------------------------------------
+enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3 };
+struct TcGemm {
+  const __nv_bfloat16* W;   // packed blocks [N/128][KC][128x64]
+  const __nv_bfloat16* W2;  // second matrix (GeGLU "up"), same packing, or null
+  const __nv_bfloat16* X;   // tiled activations [KC][rows_pad][64]
+  int rows_pad, M, N, K;
+  int epi;
+  const float* scale;  // per-out-channel dequant scale or null
+  const float* scale2;
+  const float* bias;   // TC_BIAS_ROWMAP
+  const float* gate;   // TC_RESID (null = 1)
+  float* out_f32; int ldo;          // TC_STORE / TC_RESID / TC_BIAS_ROWMAP
+  __nv_bfloat16* out_tiled;         // TC_GEGLU: [N/64][rows_pad][64]
+  int rows_in, rows_out, row_off;   // TC_BIAS_ROWMAP row remap
+  int gelu_exact;
+  int splits;                       // split-K factor (TC_RESID only)
+  unsigned wait_limit;
+};
+// Returns cudaSuccess or the launch error; `nt` is the token-tile width (64, 128 or 256).
+cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st);
+cudaError_t tc_gemm_setup();  // one-time attribute setup (dynamic shared memory opt-in)
+
+}  // namespace phyai

@@ -1,0 +1,548 @@
+// CUDA-core kernels: request block, tables, packing, embedding, norms, the Euler head, a generic
+// fp32 GEMM and a generic fp32 attention.  They serve the fp32 configuration end to end (true
+// fp32 FMA, no TF32) and provide the small memory-bound steps of the tensor-core path.
+#include <cuda_fp8.h>
+
+#include "kernels.h"
+
+namespace phyai {
+
+// =============================================================================================
+// request block
+// =============================================================================================
+__global__ void k_set_request(Request* dst, Request src, int* cu_internal) {
+  if (threadIdx.x == 0) {
+    if (src.cu_lens == nullptr) {  // single-request entry point: build cu = {0, prefix_len}
+      cu_internal[0] = 0;
+      cu_internal[1] = src.single_len;
+      src.cu_lens = cu_internal;
+    }
+    *dst = src;
+  }
+}
+void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st) {
+  k_set_request<<<1, 32, 0, st>>>(dst, src, cu_internal);
+}
+
+// cu_prefix_lens must be non-decreasing, start >= 0, end <= kv_tokens, differences <= max_prefix.
+__global__ void k_validate(const Request* rq, int* status, int max_prefix) {
+  const int B = rq->batch;
+  const int* cu = rq->cu_lens;
+  bool bad = false;
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    const int lo = cu[b], hi = cu[b + 1];
+    if (lo < 0 || hi < lo || hi - lo > max_prefix || (uint64_t)hi > rq->kv_tokens) bad = true;
+  }
+  if (bad) atomicExch(status, ST_INVALID_ARG);
+}
+void launch_validate(const Request* rq, int* status, int max_prefix, cudaStream_t st) {
+  k_validate<<<1, 256, 0, st>>>(rq, status, max_prefix);
+}
+
+// =============================================================================================
+// storage decoding
+// =============================================================================================
+__device__ __forceinline__ float load_src(const void* src, int kind, size_t i) {
+  if (kind == 0) return reinterpret_cast<const float*>(src)[i];
+  if (kind == 1) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(src)[i]);
+  const __half_raw hr = __nv_cvt_fp8_to_halfraw(reinterpret_cast<const __nv_fp8_storage_t*>(src)[i], __NV_E4M3);
+  return __half2float(__half(hr));
+}
+
+__global__ void k_to_f32(const void* src, int kind, float* dst, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = load_src(src, kind, i);
+}
+void launch_to_f32(const void* src, int kind, float* dst, size_t n, cudaStream_t st) {
+  if (n == 0) return;
+  const int blocks = (int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096);
+  k_to_f32<<<blocks, 256, 0, st>>>(src, kind, dst, n);
+}
+
+__global__ void k_copy_cols(const void* src, int kind, const float* scale, float* dst, int rows, int cols, int ld_dst,
+                            int col_off) {
+  const size_t n = (size_t)rows * cols;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / cols), c = (int)(i % cols);
+    float v = load_src(src, kind, i);
+    if (scale) v *= scale[c];
+    dst[(size_t)r * ld_dst + col_off + c] = v;
+  }
+}
+void launch_copy_cols(const void* src, int kind, const float* scale, float* dst, int rows, int cols, int ld_dst,
+                      int col_off, cudaStream_t st) {
+  const size_t n = (size_t)rows * cols;
+  const int blocks = (int)((n + 255) / 256 < 8192 ? (n + 255) / 256 : 8192);
+  k_copy_cols<<<blocks, 256, 0, st>>>(src, kind, scale, dst, rows, cols, ld_dst, col_off);
+}
+
+// Weight [K][N] -> packed out-channel-major swizzled blocks.  One thread per 16-byte chunk
+// (8 consecutive k of one out channel): reads are strided by N (one-off cost at create).
+__global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off) {
+  const int KC = K >> 6;
+  const size_t chunks = (size_t)N * (K >> 3);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
+    const int n = (int)(i % N);         // consecutive threads -> consecutive n: coalesced source reads
+    const int k8 = (int)(i / N);        // chunk index along K
+    const int k0 = k8 << 3;
+    const int np = n_off + n;
+    const int kc = k0 >> 6, c = (k0 & 63) >> 3;
+    const size_t base = (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 64 + (size_t)((c ^ (np & 7)) << 3);
+    __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __float2bfloat16_rn(load_src(src, kind, (size_t)(k0 + j) * N + n));
+    *reinterpret_cast<uint4*>(dst + base) = *reinterpret_cast<const uint4*>(v);
+  }
+}
+void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st) {
+  const size_t chunks = (size_t)N * (K >> 3);
+  const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
+  k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off);
+}
+
+// =============================================================================================
+// tables
+// =============================================================================================
+__global__ void k_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K,
+                            const float* bias, const float* add, int act_swish, float* Y, int ldy) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = blockIdx.y;
+  if (n >= N) return;
+  double acc = 0.0;
+  const float* x = X + (size_t)r * ldx;
+  for (int d = 0; d < K; ++d) acc += (double)x[d] * (double)load_src(W, w_kind, (size_t)(w_row_off + d) * N + n);
+  if (bias) acc += (double)bias[n];
+  if (add) acc += (double)add[n];
+  if (act_swish) acc = acc / (1.0 + exp(-acc));
+  Y[(size_t)r * ldy + n] = (float)acc;
+}
+void launch_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K, const float* bias,
+                      const float* add, int act_swish, float* Y, int ldy, int R, cudaStream_t st) {
+  dim3 grid((N + 127) / 128, R);
+  k_rows_gemm<<<grid, 128, 0, st>>>(X, ldx, W, w_kind, w_row_off, N, K, bias, add, act_swish, Y, ldy);
+}
+
+// tau[k][j] = sin(2 pi t_k / period_j), tau[k][D/2 + j] = cos(...), t_k = 1 - k/n, in fp64.
+__global__ void k_sinusoid(float* tau, int n_steps, int D, double pmin, double pmax) {
+  const int half = D / 2;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_steps * half) return;
+  const int k = idx / half, j = idx % half;
+  const double t = 1.0 - (double)k / (double)n_steps;
+  const double frac = half > 1 ? (double)j / (double)(half - 1) : 0.0;
+  const double period = pmin * pow(pmax / pmin, frac);
+  const double arg = 6.283185307179586476925286766559 * t / period;
+  tau[(size_t)k * D + j] = (float)sin(arg);
+  tau[(size_t)k * D + half + j] = (float)cos(arg);
+}
+void launch_sinusoid(float* tau, int n_steps, int D, double pmin, double pmax, cudaStream_t st) {
+  const int n = n_steps * (D / 2);
+  k_sinusoid<<<(n + 127) / 128, 128, 0, st>>>(tau, n_steps, D, pmin, pmax);
+}
+
+__global__ void k_rope_table(float2* tab, int n_pos, int dh, double theta) {
+  const int half = dh / 2;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_pos * half) return;
+  const int pos = idx / half, j = idx % half;
+  const double phi = (double)pos * pow(theta, -2.0 * (double)j / (double)dh);
+  tab[idx] = make_float2((float)cos(phi), (float)sin(phi));
+}
+void launch_rope_table(float2* tab, int n_pos, int dh, double theta, cudaStream_t st) {
+  const int n = n_pos * (dh / 2);
+  k_rope_table<<<(n + 127) / 128, 128, 0, st>>>(tab, n_pos, dh, theta);
+}
+
+__global__ void k_one_plus(const float* g, float* out, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = 1.0f + g[i];
+}
+void launch_one_plus(const float* gamma, float* out, int n, cudaStream_t st) {
+  k_one_plus<<<(n + 255) / 256, 256, 0, st>>>(gamma, out, n);
+}
+
+__global__ void k_mod_finish(float* mod, int R, int D) {
+  const size_t n = (size_t)R * D;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t r = i / D, d = i % D;
+    mod[r * 3 * D + d] += 1.0f;
+  }
+}
+void launch_mod_finish(float* mod, int R, int D, cudaStream_t st) {
+  k_mod_finish<<<256, 256, 0, st>>>(mod, R, D);
+}
+
+// =============================================================================================
+// per-call prologue: x <- noise, state-token rows
+// =============================================================================================
+__global__ void k_begin(const Request* rq, const int* status, const float* Ws, const float* bs, float* state_tok,
+                        int Ds, int D, int HA, int batch, int ns) {
+  if (status_set(status)) return;
+  const Request r = *rq;
+  const size_t total = (size_t)batch * HA;
+  const size_t tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, nth = (size_t)gridDim.x * blockDim.x;
+  if (r.x != r.noise)
+    for (size_t i = tid; i < total; i += nth) r.x[i] = r.noise[i];
+  if (ns) {
+    const size_t tot2 = (size_t)batch * D;
+    for (size_t i = tid; i < tot2; i += nth) {
+      const int b = (int)(i / D), n = (int)(i % D);
+      float acc = 0.f;
+      for (int s = 0; s < Ds; ++s) acc = fmaf(r.states[(size_t)b * Ds + s], Ws[(size_t)s * D + n], acc);
+      state_tok[i] = acc + bs[n];
+    }
+  }
+}
+void launch_begin(const Request* rq, const int* status, const float* Ws, const float* bs, float* state_tok,
+                  const Dims& d, int batch, cudaStream_t st) {
+  const size_t work = (size_t)batch * (d.H * d.A > d.D ? d.H * d.A : d.D);
+  const int blocks = (int)((work + 255) / 256 < 1024 ? (work + 255) / 256 : 1024);
+  k_begin<<<blocks, 256, 0, st>>>(rq, status, Ws, bs, state_tok, d.Ds, d.D, d.H * d.A, batch, d.ns);
+}
+
+// =============================================================================================
+// suffix embedding
+// =============================================================================================
+// pi0 (time concatenated into the action MLP): with the first MLP layer folded into the action
+// projection, u = swish(x Wc + tb_k) where Wc = Wa W1[0:D] and tb_k = tau_k W1[D:2D] + b1 + ba W1[0:D].
+template <class Writer>
+__global__ void k_embed_pi0(const Request* rq, const int* status, const float* Wc, const float* tb,
+                            const float* state_tok, float* h, Writer u, int A, int H, int D, int S, int ns) {
+  if (status_set(status)) return;
+  extern __shared__ float xs[];
+  const int r = blockIdx.x;  // action row b*H + i
+  const int b = r / H, i = r % H;
+  const float* x = rq->x + (size_t)r * A;
+  for (int a = threadIdx.x; a < A; a += blockDim.x) xs[a] = x[a];
+  __syncthreads();
+  for (int n = threadIdx.x; n < D; n += blockDim.x) {
+    float acc = 0.f;
+    for (int a = 0; a < A; ++a) acc = fmaf(xs[a], Wc[(size_t)a * D + n], acc);
+    u.store(r, n, swish_precise(acc + tb[n]));
+    if (ns && i == 0) h[(size_t)(b * S) * D + n] = state_tok[(size_t)b * D + n];
+  }
+}
+void launch_embed_pi0(const Request* rq, const int* status, const float* Wc, const float* tb, const float* state_tok,
+                      float* h, float* u_f32, __nv_bfloat16* u_tiled, int rows_pad, const Dims& d, int batch,
+                      cudaStream_t st) {
+  const int rows = batch * d.H;
+  if (u_tiled)
+    k_embed_pi0<<<rows, 256, d.A * sizeof(float), st>>>(rq, status, Wc, tb, state_tok, h, TiledBf16{u_tiled, rows_pad},
+                                                        d.A, d.H, d.D, d.S, d.ns);
+  else
+    k_embed_pi0<<<rows, 256, d.A * sizeof(float), st>>>(rq, status, Wc, tb, state_tok, h, RowMajorF32{u_f32, d.D}, d.A,
+                                                        d.H, d.D, d.S, d.ns);
+}
+
+__global__ void k_embed_pi05(const Request* rq, const int* status, const float* Wa, const float* ba,
+                             const float* state_tok, float* h, int A, int H, int D, int S, int ns) {
+  if (status_set(status)) return;
+  extern __shared__ float xs[];
+  const int r = blockIdx.x;
+  const int b = r / H, i = r % H;
+  const float* x = rq->x + (size_t)r * A;
+  for (int a = threadIdx.x; a < A; a += blockDim.x) xs[a] = x[a];
+  __syncthreads();
+  float* hrow = h + (size_t)(b * S + ns + i) * D;
+  for (int n = threadIdx.x; n < D; n += blockDim.x) {
+    float acc = 0.f;
+    for (int a = 0; a < A; ++a) acc = fmaf(xs[a], Wa[(size_t)a * D + n], acc);
+    hrow[n] = acc + ba[n];
+    if (ns && i == 0) h[(size_t)(b * S) * D + n] = state_tok[(size_t)b * D + n];
+  }
+}
+void launch_embed_pi05(const Request* rq, const int* status, const float* Wa, const float* ba, const float* state_tok,
+                       float* h, const Dims& d, int batch, cudaStream_t st) {
+  k_embed_pi05<<<batch * d.H, 256, d.A * sizeof(float), st>>>(rq, status, Wa, ba, state_tok, h, d.A, d.H, d.D, d.S,
+                                                              d.ns);
+}
+
+// =============================================================================================
+// (Ada)RMSNorm: one warp per row
+// =============================================================================================
+template <class Writer>
+__global__ void k_rmsnorm(const int* status, const float* h, const float* gain, const float* shift, Writer out, int M,
+                          int D, float eps) {
+  if (status_set(status)) return;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const float* x = h + (size_t)row * D;
+  float ss = 0.f;
+  for (int d = lane; d < D; d += 32) ss = fmaf(x[d], x[d], ss);
+  ss = warp_sum(ss);
+  const float r = 1.0f / sqrtf(ss / (float)D + eps);
+  for (int d = lane; d < D; d += 32) {
+    float v = x[d] * r * gain[d];
+    if (shift) v += shift[d];
+    out.store(row, d, v);
+  }
+}
+void launch_rmsnorm(const int* status, const float* h, const float* gain, const float* shift, float* out_f32,
+                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st) {
+  const int blocks = (M + 3) / 4;
+  if (out_tiled)
+    k_rmsnorm<<<blocks, 128, 0, st>>>(status, h, gain, shift, TiledBf16{out_tiled, rows_pad}, M, D, eps);
+  else
+    k_rmsnorm<<<blocks, 128, 0, st>>>(status, h, gain, shift, RowMajorF32{out_f32, D}, M, D, eps);
+}
+
+// =============================================================================================
+// final norm -> out-projection -> Euler update (epilogue): x += dt * (n . Wout + bout)
+// =============================================================================================
+__global__ void k_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
+                        const float* Wout, const float* bout, float dt, int A, int H, int D, int S, int ns, float eps) {
+  if (status_set(status)) return;
+  extern __shared__ float nrm[];  // D floats + 1
+  __shared__ float red[32];
+  const int r = blockIdx.x;  // action row
+  const int b = r / H, i = r % H;
+  const float* x = h + (size_t)(b * S + ns + i) * D;
+  float ss = 0.f;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) ss = fmaf(x[d], x[d], ss);
+  ss = warp_sum(ss);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  if (lane == 0) red[warp] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < nw; ++w) tot += red[w];
+  const float rr = 1.0f / sqrtf(tot / (float)D + eps);
+  for (int d = threadIdx.x; d < D; d += blockDim.x) {
+    float v = x[d] * rr * gain[d];
+    if (shift) v += shift[d];
+    nrm[d] = v;
+  }
+  __syncthreads();
+  float* xo = rq->x + (size_t)r * A;
+  for (int a = warp; a < A; a += nw) {
+    float acc = 0.f;
+    for (int d = lane; d < D; d += 32) acc = fmaf(nrm[d], Wout[(size_t)d * A + a], acc);
+    acc = warp_sum(acc);
+    if (lane == 0) xo[a] = xo[a] + dt * (acc + bout[a]);
+  }
+}
+void launch_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
+                  const float* Wout, const float* bout, float dt, const Dims& d, int batch, cudaStream_t st) {
+  k_final<<<batch * d.H, 256, d.D * sizeof(float), st>>>(rq, status, h, gain, shift, Wout, bout, dt, d.A, d.H, d.D, d.S,
+                                                         d.ns, d.eps);
+}
+
+// =============================================================================================
+// generic fp32 GEMM, 64x64x16 tiles, 256 threads, 4x4 outputs per thread
+// =============================================================================================
+template <bool DUAL>
+__global__ void __launch_bounds__(256) k_simt_gemm(const int* status, SimtGemm g) {
+  if (status_set(status)) return;
+  __shared__ float As[16][64 + 1];
+  __shared__ float Bs[16][64];
+  __shared__ float Bs2[DUAL ? 16 : 1][64];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  float acc[4][4] = {}, acc2[4][4] = {};
+  for (int k0 = 0; k0 < g.K; k0 += 16) {
+    for (int i = threadIdx.x; i < 64 * 16; i += 256) {
+      const int m = i >> 4, k = i & 15;
+      As[k][m] = (m0 + m < g.M && k0 + k < g.K) ? g.A[(size_t)(m0 + m) * g.lda + k0 + k] : 0.f;
+    }
+    for (int i = threadIdx.x; i < 16 * 64; i += 256) {
+      const int k = i >> 6, n = i & 63;
+      const bool ok = (k0 + k < g.K && n0 + n < g.N);
+      Bs[k][n] = ok ? g.B[(size_t)(k0 + k) * g.N + n0 + n] : 0.f;
+      if (DUAL) Bs2[k][n] = ok ? g.B2[(size_t)(k0 + k) * g.N + n0 + n] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      float a[4], b[4], b2[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[k][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        b[j] = Bs[k][tx * 4 + j];
+        if (DUAL) b2[j] = Bs2[k][tx * 4 + j];
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+          if (DUAL) acc2[i][j] = fmaf(a[i], b2[j], acc2[i][j]);
+        }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= g.M) continue;
+    const int orow = (m / g.rows_in) * g.rows_out + g.row_off + m % g.rows_in;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= g.N) continue;
+      float* o = g.out + (size_t)orow * g.ldo + n;
+      float v = acc[i][j];
+      if (g.epi == EPI_STORE) {
+        *o = v + (g.bias ? g.bias[n] : 0.f);
+      } else if (g.epi == EPI_SWISH) {
+        *o = swish_precise(v + (g.bias ? g.bias[n] : 0.f));
+      } else if (g.epi == EPI_RESID) {
+        *o = *o + (g.gate ? g.gate[n] * v : v);
+      } else {
+        *o = gelu_f(v, g.gelu_exact) * acc2[i][j];
+      }
+    }
+  }
+}
+void launch_simt_gemm(const int* status, const SimtGemm& g, cudaStream_t st) {
+  dim3 grid((g.N + 63) / 64, (g.M + 63) / 64);
+  if (g.epi == EPI_GEGLU)
+    k_simt_gemm<true><<<grid, 256, 0, st>>>(status, g);
+  else
+    k_simt_gemm<false><<<grid, 256, 0, st>>>(status, g);
+}
+
+// =============================================================================================
+// generic fp32 attention: one block (4 warps) per (suffix row, query head); every warp walks a
+// strided share of the keys with an online softmax; the four partial states merge in shared memory.
+// =============================================================================================
+template <typename KV, class Writer>
+__global__ void __launch_bounds__(128) k_attention_simt(const Request* rq, const int* status, const float* qkv,
+                                                        const float2* rope, int layer, Writer out, Dims d) {
+  if (status_set(status)) return;
+  constexpr int MAXR = 8;  // head_dim <= 256
+  extern __shared__ float sm[];
+  float* qs = sm;                 // [dh] rotated, pre-scaled query
+  float* part = sm + d.dh;        // [4][dh + 2] partial (acc, m, l)
+  const int row = blockIdx.x;     // b*S + i
+  const int a = blockIdx.y;       // query head
+  const int b = row / d.S, i = row % d.S;
+  const int hk = a / (d.Hq / d.Hkv);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const Request r = *rq;
+  const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
+  const int half = d.dh >> 1;
+  const float scale = rsqrtf((float)d.dh);
+  const bool use_rope = rope != nullptr;
+
+  // query, rotated at position P + i
+  const float* qrow = qkv + (size_t)row * d.Nqkv + a * d.dh;
+  for (int t = threadIdx.x; t < d.dh; t += blockDim.x) {
+    float v = qrow[t];
+    if (use_rope) {
+      const int j = t < half ? t : t - half;
+      const float2 cs = rope[(size_t)(P + i) * half + j];
+      const float other = qrow[t < half ? t + half : t - half];
+      v = t < half ? v * cs.x - other * cs.y : v * cs.x + other * cs.y;
+    }
+    qs[t] = v * scale;
+  }
+  __syncthreads();
+
+  const KV* Kp = reinterpret_cast<const KV*>(r.prefix_kv) + ((size_t)(layer * 2 + 0) * r.kv_tokens + p0) * d.Hkv * d.dh +
+                 (size_t)hk * d.dh;
+  const KV* Vp = reinterpret_cast<const KV*>(r.prefix_kv) + ((size_t)(layer * 2 + 1) * r.kv_tokens + p0) * d.Hkv * d.dh +
+                 (size_t)hk * d.dh;
+  const size_t kv_stride = (size_t)d.Hkv * d.dh;
+
+  float m = -INFINITY, l = 0.f, acc[MAXR];
+#pragma unroll
+  for (int t = 0; t < MAXR; ++t) acc[t] = 0.f;
+
+  const int nkeys = P + d.S;
+  for (int j = warp; j < nkeys; j += 4) {
+    float dot = 0.f;
+    float vreg[MAXR];
+    if (j < P) {
+      const KV* k = Kp + (size_t)j * kv_stride;
+      const KV* v = Vp + (size_t)j * kv_stride;
+#pragma unroll
+      for (int t = 0; t < MAXR; ++t) {
+        const int dd = lane + 32 * t;
+        if (dd < d.dh) {
+          dot = fmaf(qs[dd], to_float<KV>(k[dd]), dot);
+          vreg[t] = to_float<KV>(v[dd]);
+        } else {
+          vreg[t] = 0.f;
+        }
+      }
+    } else {
+      const int js = j - P;
+      if (d.block_causal && d.ns && i == 0 && js != 0) continue;  // state token sees only itself (warp-uniform)
+      const float* krow = qkv + (size_t)(b * d.S + js) * d.Nqkv + d.Nq + hk * d.dh;
+      const float* vrow = krow + d.Hkv * d.dh;
+#pragma unroll
+      for (int t = 0; t < MAXR; ++t) {
+        const int dd = lane + 32 * t;
+        if (dd < d.dh) {
+          float kvv = krow[dd];
+          if (use_rope) {
+            const int jj = dd < half ? dd : dd - half;
+            const float2 cs = rope[(size_t)(P + js) * half + jj];
+            const float other = krow[dd < half ? dd + half : dd - half];
+            kvv = dd < half ? kvv * cs.x - other * cs.y : kvv * cs.x + other * cs.y;
+          }
+          dot = fmaf(qs[dd], kvv, dot);
+          vreg[t] = vrow[dd];
+        } else {
+          vreg[t] = 0.f;
+        }
+      }
+    }
+    dot = warp_sum(dot);
+    const float mn = fmaxf(m, dot);
+    const float corr = __expf(m - mn), p = __expf(dot - mn);
+    l = l * corr + p;
+#pragma unroll
+    for (int t = 0; t < MAXR; ++t) acc[t] = acc[t] * corr + p * vreg[t];
+    m = mn;
+  }
+  float* mine = part + warp * (d.dh + 2);
+#pragma unroll
+  for (int t = 0; t < MAXR; ++t) {
+    const int dd = lane + 32 * t;
+    if (dd < d.dh) mine[dd] = acc[t];
+  }
+  if (lane == 0) {
+    mine[d.dh] = m;
+    mine[d.dh + 1] = l;
+  }
+  __syncthreads();
+  float mm = -INFINITY;
+  for (int w = 0; w < 4; ++w) mm = fmaxf(mm, part[w * (d.dh + 2) + d.dh]);
+  float ll = 0.f;
+  float wgt[4];
+  for (int w = 0; w < 4; ++w) {
+    const float mw = part[w * (d.dh + 2) + d.dh];
+    wgt[w] = (mw == -INFINITY) ? 0.f : __expf(mw - mm);
+    ll += wgt[w] * part[w * (d.dh + 2) + d.dh + 1];
+  }
+  const float inv = 1.0f / ll;
+  for (int t = threadIdx.x; t < d.dh; t += blockDim.x) {
+    float o = 0.f;
+    for (int w = 0; w < 4; ++w) o += wgt[w] * part[w * (d.dh + 2) + t];
+    out.store(row, a * d.dh + t, o * inv);
+  }
+}
+
+void launch_attention_simt(const Request* rq, const int* status, const float* qkv, const float2* rope, int layer,
+                           int kv_is_bf16, float* out_f32, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
+                           int batch, cudaStream_t st) {
+  dim3 grid(batch * d.S, d.Hq);
+  const size_t smem = (size_t)(d.dh + 4 * (d.dh + 2)) * sizeof(float);
+  if (kv_is_bf16) {
+    if (out_tiled)
+      k_attention_simt<__nv_bfloat16><<<grid, 128, smem, st>>>(rq, status, qkv, rope, layer,
+                                                               TiledBf16{out_tiled, rows_pad}, d);
+    else
+      k_attention_simt<__nv_bfloat16><<<grid, 128, smem, st>>>(rq, status, qkv, rope, layer,
+                                                               RowMajorF32{out_f32, d.Nq}, d);
+  } else {
+    if (out_tiled)
+      k_attention_simt<float><<<grid, 128, smem, st>>>(rq, status, qkv, rope, layer, TiledBf16{out_tiled, rows_pad}, d);
+    else
+      k_attention_simt<float><<<grid, 128, smem, st>>>(rq, status, qkv, rope, layer, RowMajorF32{out_f32, d.Nq}, d);
+  }
+}
+
+}  // namespace phyai

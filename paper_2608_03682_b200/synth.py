@@ -52,6 +52,12 @@ class ExpertConfig:
     gelu_exact: bool = False
     suffix_block_causal: bool = False
 
+    def __post_init__(self):
+        # The C ABI carries these four as float32; store the float32-representable value so that
+        # every consumer of the configuration sees exactly the same number.
+        for name in ("rms_eps", "rope_theta", "time_min_period", "time_max_period"):
+            object.__setattr__(self, name, float(np.float32(getattr(self, name))))
+
     @property
     def suffix_len(self) -> int:
         return self.horizon + (1 if self.has_state_token else 0)

@@ -1,0 +1,37 @@
+"""Shared helpers of the GPU parity tests: run the CUDA library and the oracle on the same inputs."""
+import numpy as np
+import torch
+
+from oracle import expert_oracle as O
+from paper_2608_03682_b200 import binding, synth
+
+BAR = {"f32": 1e-4, "bf16": 2e-2, "w8e4m3": 2e-2}   # max relative error on the final action chunk
+
+
+def gpu_single(cfg, W, kv, P, state, noise, n_steps, engine="auto", use_graph=True, expert=None):
+    """One request through phyai_denoise; returns the [H,A] result as float64 numpy."""
+    ex = expert or binding.Expert(cfg, binding.weights_to_device(W), engine=engine)
+    try:
+        if not use_graph:
+            ex.set_option("use_graph", 0)
+        out = ex.denoise(kv.cuda(), P, None if state is None else state.cuda(), noise.cuda(), n_steps)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        return out.double().cpu().numpy()
+    finally:
+        if expert is None:
+            ex.close()
+
+
+def small_bf16_config(cond="pi0", **kw):
+    """A reduced expert whose dimensions still satisfy the tensor path's tiling (multiples of 128)
+    and span several tiles: 3 layers, width 256, MLP 512, 2 query heads of 128."""
+    base = dict(n_layers=3, width=256, mlp_dim=512, n_q_heads=2, n_kv_heads=1, head_dim=128, state_dim=6,
+                action_dim=5, horizon=13, has_state_token=(cond == "pi0"), max_prefix_len=200, max_batch=1,
+                cond=cond, dtype="bf16")
+    base.update(kw)
+    return synth.ExpertConfig(**base)
+
+
+def rel_err(got, ref):
+    return O.max_rel_err(got, ref)

@@ -346,7 +346,7 @@ def test_blocks_switched_off_leave_embedding_then_head_pi0():
         W[f"wdown.{l}"] = np.zeros_like(W[f"wdown.{l}"])
     t, D = 1.0, cfg.width
     half = D // 2
-    period = 4e-3 * (4.0 / 4e-3) ** (np.arange(half) / (half - 1))
+    period = cfg.time_min_period * (cfg.time_max_period / cfg.time_min_period) ** (np.arange(half) / (half - 1))
     tau = np.concatenate([np.sin(2 * math.pi * t / period), np.cos(2 * math.pi * t / period)])
     rows = []
     for i in range(cfg.horizon):
