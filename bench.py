@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the action-expert denoising loop on B200.
+
+One "step" = one whole action chunk: one call of the hot path (embedding, all layers, head and
+Euler update for every integration step) over one batch of synthetic input.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2|C3|C4|C5b1|...] [--impl reference]
+
+Prints ONE JSON line.  ``value`` is measured with the inputs resident in device memory and CUDA
+events on the launching stream; ``e2e`` goes through the host-buffer entry point (pinned host
+inputs, host<->device copies inside the timed region).  ``--impl reference`` times the float64 CPU
+oracle on the host cores instead.  Under torchrun every rank runs an independent replica (the
+path shards by request, no collective); rank 0 reports the maximum time over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_03682_b200 import synth  # noqa: E402
+
+METRIC = "ms per action chunk (batch 1, 10 steps)"
+METRIC_BATCHED = "chunks/sec at batch %d"
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+
+
+# ------------------------------------------------------------------------------------------------
+# workloads
+# ------------------------------------------------------------------------------------------------
+def workload(name: str):
+    """(cfg, cfg_id, batch, prefix lengths, n_steps)"""
+    if name == "C1":
+        return synth.tiny_config(), 1, 1, [64], 4
+    if name == "C2":
+        return synth.pi0_config(), 2, 1, [816], 10
+    if name == "C3":
+        return synth.pi05_config(), 3, 1, [968], 10
+    if name == "C4":
+        lens = synth.make_ragged_lengths(4, 64, 600, 968)
+        return synth.pi0_config(max_batch=64), 4, 64, [int(x) for x in lens], 10
+    if name.startswith("C5b"):
+        b = int(name[3:])
+        return synth.pi0_config(max_batch=b, dtype="w8e4m3", max_prefix_len=816), 5, b, [816] * b, 10
+    raise SystemExit(f"unknown workload {name}")
+
+
+def algorithmic_cost(cfg, lens, n_steps):
+    """Bytes that must cross HBM and FLOPs per chunk: every big weight once per Euler step, each
+    request's prefix KV once per layer per step; activations and tables are cache resident."""
+    D, F, L, S = cfg.width, cfg.mlp_dim, cfg.n_layers, cfg.suffix_len
+    wbytes = 1 if cfg.dtype == "w8e4m3" else (4 if cfg.dtype == "f32" else 2)
+    ebytes = 4 if cfg.dtype == "f32" else 2
+    nqkv = cfg.q_dim + 2 * cfg.kv_dim
+    per_layer_params = D * nqkv + cfg.q_dim * D + 2 * D * F + F * D
+    embed_params = D * D + (cfg.action_dim * D) + D * cfg.action_dim if cfg.cond == "pi0" else 2 * cfg.action_dim * D
+    B = len(lens)
+    kv_bytes = sum(lens) * L * 2 * cfg.kv_dim * ebytes
+    bytes_step = L * per_layer_params * wbytes + embed_params * ebytes + kv_bytes
+    lin_flops = 2 * B * S * L * per_layer_params + (2 * B * cfg.horizon * D * D if cfg.cond == "pi0" else 0)
+    attn_flops = sum(4 * S * (p + S) * cfg.n_q_heads * cfg.head_dim for p in lens) * L
+    return bytes_step * n_steps, (lin_flops + attn_flops) * n_steps
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS, bf16_tflops_sustained=1400.0,
+                source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])), mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        # samples under load: the upper half of the observed clocks (idle samples precede the run)
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# oracle timing (CPU baseline and the reference arm)
+# ------------------------------------------------------------------------------------------------
+def time_oracle(cfg, cfg_id, lens, n_steps, budget_s: float, repeats: int = 1, warm: int = 0):
+    """Times the float64 oracle as it stands on a bounded sample: one request, ``sample_steps`` of
+    the ``n_steps`` Euler steps (all steps cost the same), scaled to a whole batch of chunks."""
+    from oracle import expert_oracle as O
+
+    W = O.Weights(synth.make_weights(cfg, cfg_id))
+    P = lens[0]
+    kv = O.to_f64(synth.make_prefix_kv(cfg, cfg_id, P, 0))
+    state = synth.make_state(cfg, cfg_id, 0) if cfg.has_state_token else None
+    st = None if state is None else O.to_f64(state)
+    x = O.to_f64(synth.make_noise(cfg, cfg_id, 0))
+    t0 = time.perf_counter()
+    O.velocity(cfg, W, kv, P, st, x, 1.0)
+    one = time.perf_counter() - t0
+    per_call = budget_s / max(1, repeats + warm)
+    sample_steps = int(max(1, min(n_steps, per_call // max(one, 1e-9))))
+    times = []
+    for i in range(warm + repeats):
+        t0 = time.perf_counter()
+        xx = x
+        for k in range(sample_steps):
+            xx = xx + (-1.0 / n_steps) * O.velocity(cfg, W, kv, P, st, xx, 1.0 - k / n_steps)
+        if i >= warm:
+            times.append(time.perf_counter() - t0)
+    scale = (n_steps / sample_steps) * len(lens)
+    ms_per_batch = float(np.mean(times)) * 1e3 * scale
+    sample = (f"1 of {len(lens)} request(s) (prefix {P}), {sample_steps} of {n_steps} Euler steps, "
+              f"scaled x{scale:g}; {repeats} timed repeat(s)")
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count()
+    return ms_per_batch, sample, cores
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--impl", default="phyai", choices=["phyai", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
+    args = ap.parse_args()
+    K, Wm = args.steps, max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg, cfg_id, batch, lens, n_steps = workload(args.workload)
+    batched = batch > 1
+    metric = (METRIC_BATCHED % batch) if batched else METRIC
+    unit = "chunks/s" if batched else "ms"
+    config = {"workload": f"{args.workload}: {cfg.cond}-shaped expert, {cfg.dtype}, batch {batch}, "
+                          f"prefix {min(lens)}..{max(lens)}, {cfg.suffix_len} suffix tokens, {n_steps} Euler steps",
+              "batch": batch, "n_steps": n_steps, "replicas": world,
+              "l2": "inputs larger than L2 (weights streamed per step exceed 126 MB); no flush"}
+
+    # -------------------------------------------------------------------------- reference arm
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        ms, sample, cores = time_oracle(cfg, cfg_id, lens, n_steps, budget_s=120.0, repeats=K, warm=min(Wm, 1))
+        value = batch / (ms / 1e3) if batched else ms
+        line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": K,
+                "warmup": Wm, "ms_per_step": ms, "higher_is_better": batched, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f64", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
+                "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    # -------------------------------------------------------------------------- CUDA arm
+    import torch
+
+    from paper_2608_03682_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    W = synth.make_weights(cfg, cfg_id)
+    ex = binding.Expert(cfg, binding.weights_to_device(W))
+    if args.no_graph:
+        ex.set_option("use_graph", 0)
+    del W
+    kvs = [synth.make_prefix_kv(cfg, cfg_id, p, b) for b, p in enumerate(lens)]
+    kv_h, cu = synth.pack_prefix_kv(kvs)
+    del kvs
+    states_h = torch.stack([synth.make_state(cfg, cfg_id, b) for b in range(batch)]) if cfg.has_state_token else None
+    noise_h = torch.stack([synth.make_noise(cfg, cfg_id, b) for b in range(batch)])
+    cu_h = torch.from_numpy(cu)
+    kv_d, noise_d, cu_d = kv_h.cuda(), noise_h.cuda(), cu_h.cuda()
+    states_d = None if states_h is None else states_h.cuda()
+    out_d = torch.empty_like(noise_d)
+    stream = torch.cuda.current_stream()
+
+    def call_device():
+        if batched:
+            ex.denoise_batched(kv_d, cu_d, states_d, noise_d, n_steps, out=out_d, stream=stream)
+        else:
+            ex.denoise(kv_d, lens[0], None if states_d is None else states_d[0], noise_d[0], n_steps, out=out_d[0],
+                       stream=stream)
+
+    pin = lambda t: None if t is None else t.pin_memory()
+    kv_p, noise_p, states_p, cu_p = pin(kv_h), pin(noise_h), pin(states_h), pin(cu_h)
+    out_p = torch.empty_like(noise_h).pin_memory()
+
+    def call_host():
+        if batched:
+            ex.denoise_batched_host(kv_p, cu_p, states_p, noise_p, n_steps, out_p, stream=stream)
+        else:
+            ex.denoise_host(kv_p, lens[0], None if states_p is None else states_p[0], noise_p[0], n_steps, out_p[0],
+                            stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(iters):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(Wm):
+        call_device()
+    torch.cuda.synchronize()
+    status = ex.poll_status()
+    if status != 0:
+        raise SystemExit(f"device status {status} after warm-up")
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    total_ms = timed(call_device, K)
+    clocks = sampler.stop() if sampler else None
+    ms_per_step = total_ms / K
+
+    for _ in range(3):
+        call_host()
+    e2e_ms = timed(call_host, K) / K
+    status = ex.poll_status()
+    if status != 0:
+        raise SystemExit(f"device status {status} after the timed region")
+    result_ok = bool(torch.isfinite(out_d).all().item()) and bool(torch.isfinite(out_p).all().item())
+
+    launches = ex.launches_per_call(batch, n_steps)
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    alg_bytes, alg_flops = algorithmic_cost(cfg, lens, n_steps)
+    secs = ms_per_step / 1e3
+    hbm_bound = not batched or batch < 8
+    if hbm_bound:
+        achieved = alg_bytes / secs / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "kernel": "whole captured loop (one graph launch = one chunk)",
+                    "peak_source": f"{peaks['source']} copy bandwidth", "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
+                    "algorithmic_bytes_per_launch": alg_bytes}
+    else:
+        achieved = alg_flops / secs / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "kernel": "whole captured loop (one graph launch = one batch of chunks)",
+                    "peak_source": f"{peaks['source']} sustained bf16 GEMM",
+                    "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS, "algorithmic_flops_per_launch": alg_flops}
+
+    value = world * batch / secs if batched else ms_per_step
+    e2e_value = world * batch / (e2e_ms / 1e3) if batched else e2e_ms
+    h2d = kv_h.numel() * kv_h.element_size() + noise_h.numel() * 4 + (0 if states_h is None else states_h.numel() * 4)
+    if batched:
+        h2d += cu_h.numel() * 4
+    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms_per_step, "higher_is_better": batched, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if cfg.dtype != "f32" else "f32", "data": "synthetic", "config": config,
+            "chunks_per_s": world * batch / secs, "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": int(h2d),
+                    "d2h_bytes_per_step": int(noise_h.numel() * 4), "ms_per_step": e2e_ms},
+            "gpu_launches": int(launches * K), "launches_per_step": int(launches), "finite": result_ok,
+            "roofline": roofline}
+
+    if not args.no_cpu_baseline and world == 1:
+        ms, sample, cores = time_oracle(cfg, cfg_id, lens, n_steps, budget_s=15.0, repeats=1)
+        line["cpu_baseline"] = {"value": batch / (ms / 1e3) if batched else ms, "unit": unit, "cores": cores,
+                                "kind": "oracle", "sample": sample}
+    print(json.dumps(line))
+    ex.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
