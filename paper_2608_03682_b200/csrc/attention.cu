@@ -1,0 +1,398 @@
+// Suffix -> (prefix U suffix) attention on tensor cores (operator-selection paragraph of the paper:
+// a ~50-token query against a longer prefix with head dimension 256).
+//
+// Few queries, long shared KV: one CTA takes the (<= 64) suffix rows of HPC query heads that share a
+// kv head and a contiguous slice of that request's keys.  K/V rows are staged into shared memory by
+// the bulk-copy engine, one 1-D copy per row into rows padded by 16 bytes (bank-conflict-free
+// ldmatrix without a swizzle), double buffered.  Q K^T and P V run on mma.sync m16n8k16 (bf16 in,
+// fp32 out); the softmax is the online form in fp32 with quad shuffles for the row max / sum.
+// The suffix's own K/V (fp32 from the QKV GEMM) are rotated and appended as the last tile.
+// When the key range is split over several CTAs each writes an unnormalised partial (O, m, l) and a
+// merge kernel combines them.
+#include <mma.h>
+
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace phyai {
+namespace {
+
+constexpr int KT = 64;      // keys per tile
+constexpr int QROWS = 64;   // query rows per head (suffix length <= 64)
+constexpr float LOG2E = 1.4426950408889634f;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+struct AttnArgs {
+  const Request* rq;
+  int* status;
+  const float* qkv;      // [rows][Nqkv] fp32 (q | k | v), un-rotated
+  const float2* rope;    // [pos][dh/2] (cos, sin) or null
+  int layer;
+  __nv_bfloat16* out;    // tiled bf16 [Nq/64][rows_pad][64]
+  int rows_pad;
+  int num_splits;
+  float* part_o;         // [b][head][split][64][DH] unnormalised
+  float* part_ml;        // [b][head][split][64][2]  (max in log2 units, sum)
+  Dims d;
+  unsigned wait_limit;
+};
+
+// DH: head_dim; HPC: query heads per CTA (4 warps each).
+template <int DH, int HPC>
+__global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
+  constexpr int LDS = DH + 8;                 // padded row stride in elements (+16 bytes)
+  constexpr int ROWB = DH * 2;                // bytes per K/V row
+  constexpr int NTHREADS = HPC * 128;
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem_raw);          // [HPC*64][LDS]
+  __nv_bfloat16* Ks = Qs + (size_t)HPC * QROWS * LDS;                       // [2][KT][LDS]
+  __nv_bfloat16* Vs = Ks + (size_t)2 * KT * LDS;                            // [2][KT][LDS]
+  __shared__ __align__(8) uint64_t bar_full[2];
+  __shared__ int abort_flag, skip_flag;
+
+  const Dims& d = a.d;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int split = blockIdx.x, hgrp = blockIdx.y, b = blockIdx.z;
+  const int head0 = hgrp * HPC;
+  const int hk = head0 / (d.Hq / d.Hkv);
+  const int S = d.S;
+
+  if (tid == 0) {
+    skip_flag = status_set(a.status);
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar_full[0]), 1);
+    mbar_init(smem_u32(&bar_full[1]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (skip_flag) return;
+  const WaitCtx wc{a.status, &abort_flag, a.wait_limit};
+
+  const Request r = *a.rq;
+  const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
+  const int Tp = (P + KT - 1) / KT;          // prefix tiles; tile index Tp is the suffix tile
+  const int T = Tp + 1;
+  const int t_begin = (int)(((long long)T * split) / a.num_splits);
+  const int t_end = (int)(((long long)T * (split + 1)) / a.num_splits);
+
+  const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(r.prefix_kv) +
+                            ((size_t)(a.layer * 2 + 0) * r.kv_tokens + p0) * d.Hkv * DH + (size_t)hk * DH;
+  const __nv_bfloat16* Vg = reinterpret_cast<const __nv_bfloat16*>(r.prefix_kv) +
+                            ((size_t)(a.layer * 2 + 1) * r.kv_tokens + p0) * d.Hkv * DH + (size_t)hk * DH;
+  const size_t kv_stride = (size_t)d.Hkv * DH;
+  const int half = DH / 2;
+
+  // ---- Q: rotate, scale by dh^-1/2, round to bf16, into shared memory -----------------------------
+  const float qscale = rsqrtf((float)DH);
+  for (int idx = tid; idx < HPC * QROWS * half; idx += NTHREADS) {
+    const int hl = idx / (QROWS * half), rem = idx % (QROWS * half);
+    const int i = rem / half, j = rem % half;
+    float lo = 0.f, hi = 0.f;
+    if (i < S) {
+      const float* q = a.qkv + (size_t)(b * S + i) * d.Nqkv + (size_t)(head0 + hl) * DH;
+      lo = q[j], hi = q[j + half];
+      if (a.rope) {
+        const float2 cs = a.rope[(size_t)(P + i) * half + j];
+        const float l2 = lo * cs.x - hi * cs.y, h2 = hi * cs.x + lo * cs.y;
+        lo = l2, hi = h2;
+      }
+      lo *= qscale, hi *= qscale;
+    }
+    __nv_bfloat16* dst = Qs + ((size_t)hl * QROWS + i) * LDS;
+    dst[j] = __float2bfloat16_rn(lo);
+    dst[j + half] = __float2bfloat16_rn(hi);
+  }
+
+  // ---- per-warp state -----------------------------------------------------------------------------
+  const int hl = warp >> 2, rb = warp & 3;             // local head, 16-row block
+  const int g = lane >> 2, qd = lane & 3;              // row within 8, column pair
+  const int row0 = rb * 16 + g, row1 = row0 + 8;       // this thread's two query rows
+  float o[DH / 8][4];
+#pragma unroll
+  for (int n = 0; n < DH / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+  const uint32_t q_base = smem_u32(Qs + ((size_t)hl * QROWS + rb * 16 + (lane & 15)) * LDS + (lane >> 4) * 8);
+
+  // copies of the first tile: the expected byte count is posted before any copy can complete
+  if (t_begin < t_end && t_begin < Tp && tid == 0)
+    mbar_expect_tx(smem_u32(&bar_full[0]), (uint32_t)min(KT, P - t_begin * KT) * ROWB * 2);
+  __syncthreads();  // Q visible; expect_tx posted
+  if (t_begin < t_end && t_begin < Tp && tid < min(KT, P - t_begin * KT)) {
+    const size_t gofs = (size_t)(t_begin * KT + tid) * kv_stride;
+    bulk_g2s(smem_u32(Ks + (size_t)tid * LDS), Kg + gofs, ROWB, smem_u32(&bar_full[0]));
+    bulk_g2s(smem_u32(Vs + (size_t)tid * LDS), Vg + gofs, ROWB, smem_u32(&bar_full[0]));
+  }
+
+  uint32_t phase_bits = 0u;  // bit b = parity to wait for on buffer b
+  for (int t = t_begin; t < t_end; ++t) {
+    const int buf = (t - t_begin) & 1;
+    const int nb = buf ^ 1;
+    __nv_bfloat16* Kb = Ks + (size_t)buf * KT * LDS;
+    __nv_bfloat16* Vb = Vs + (size_t)buf * KT * LDS;
+    int valid;  // keys of this tile that exist
+    // -- prefetch the next prefix tile into the other buffer (it was released by the barrier that
+    //    ended the previous iteration)
+    if (t + 1 < t_end && t + 1 < Tp) {
+      if (tid == 0) mbar_expect_tx(smem_u32(&bar_full[nb]), (uint32_t)min(KT, P - (t + 1) * KT) * ROWB * 2);
+    }
+    if (t < Tp) {
+      valid = min(KT, P - t * KT);
+      if (valid < KT) {  // ragged last prefix tile: rows that are not copied must be finite
+        for (int idx = tid; idx < (KT - valid) * (DH / 8); idx += NTHREADS) {
+          const int rr = valid + idx / (DH / 8), c = (idx % (DH / 8)) * 8;
+          *reinterpret_cast<uint4*>(Kb + (size_t)rr * LDS + c) = make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(Vb + (size_t)rr * LDS + c) = make_uint4(0, 0, 0, 0);
+        }
+      }
+    } else {
+      // -- suffix tile: rotate this request's own keys, round K and V to bf16
+      valid = S;
+      for (int idx = tid; idx < KT * half; idx += NTHREADS) {
+        const int js = idx / half, j = idx % half;
+        float klo = 0.f, khi = 0.f, vlo = 0.f, vhi = 0.f;
+        if (js < S) {
+          const float* kr = a.qkv + (size_t)(b * S + js) * d.Nqkv + d.Nq + (size_t)hk * DH;
+          const float* vr = kr + d.Hkv * DH;
+          klo = kr[j], khi = kr[j + half], vlo = vr[j], vhi = vr[j + half];
+          if (a.rope) {
+            const float2 cs = a.rope[(size_t)(P + js) * half + j];
+            const float l2 = klo * cs.x - khi * cs.y, h2 = khi * cs.x + klo * cs.y;
+            klo = l2, khi = h2;
+          }
+        }
+        Kb[(size_t)js * LDS + j] = __float2bfloat16_rn(klo);
+        Kb[(size_t)js * LDS + j + half] = __float2bfloat16_rn(khi);
+        Vb[(size_t)js * LDS + j] = __float2bfloat16_rn(vlo);
+        Vb[(size_t)js * LDS + j + half] = __float2bfloat16_rn(vhi);
+      }
+    }
+    __syncthreads();  // zero-fill / suffix tile visible; next tile's expect_tx posted
+    if (t + 1 < t_end && t + 1 < Tp && tid < min(KT, P - (t + 1) * KT) && !abort_flag) {
+      const size_t gofs = (size_t)((t + 1) * KT + tid) * kv_stride;
+      bulk_g2s(smem_u32(Ks + ((size_t)nb * KT + tid) * LDS), Kg + gofs, ROWB, smem_u32(&bar_full[nb]));
+      bulk_g2s(smem_u32(Vs + ((size_t)nb * KT + tid) * LDS), Vg + gofs, ROWB, smem_u32(&bar_full[nb]));
+    }
+    bool ok = true;
+    if (t < Tp) {
+      ok = mbar_wait(smem_u32(&bar_full[buf]), (phase_bits >> buf) & 1u, wc);
+      phase_bits ^= 1u << buf;
+    }
+    if (ok) {
+      // ---------------- S = Q K^T (16 rows x 64 keys per warp) ---------------------------------
+      float s[KT / 8][4];
+#pragma unroll
+      for (int n = 0; n < KT / 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+      const uint32_t k_base = smem_u32(Kb + (size_t)((lane & 7) + (lane >> 4) * 8) * LDS + ((lane >> 3) & 1) * 8);
+#pragma unroll 4
+      for (int kk = 0; kk < DH / 16; ++kk) {
+        uint32_t af[4];
+        ldsm_x4(q_base + kk * 32, af[0], af[1], af[2], af[3]);
+#pragma unroll
+        for (int np = 0; np < KT / 16; ++np) {
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(k_base + (uint32_t)(np * 16 * LDS * 2) + kk * 32, b0, b1, b2, b3);
+          mma_bf16(s[2 * np], af, b0, b1);
+          mma_bf16(s[2 * np + 1], af, b2, b3);
+        }
+      }
+      // ---------------- mask + online softmax (log2 domain) ----------------------------------------
+      const bool suffix_tile = t >= Tp;
+      const bool causal = suffix_tile && d.block_causal && d.ns;
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int n = 0; n < KT / 8; ++n) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int key = n * 8 + qd * 2 + (e & 1);
+          const int row = (e < 2) ? row0 : row1;
+          bool vis = key < valid;
+          if (causal && row == 0 && key != 0) vis = false;  // state token sees only itself
+          s[n][e] = vis ? s[n][e] * LOG2E : -INFINITY;
+        }
+        mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
+        mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+      const float c0 = (mn0 == -INFINITY) ? 1.f : exp2f(m0 - mn0);
+      const float c1 = (mn1 == -INFINITY) ? 1.f : exp2f(m1 - mn1);
+      const float sub0 = (mn0 == -INFINITY) ? 0.f : mn0, sub1 = (mn1 == -INFINITY) ? 0.f : mn1;
+      m0 = mn0, m1 = mn1;
+      float rs0 = 0.f, rs1 = 0.f;
+      uint32_t pf[KT / 16][4];
+#pragma unroll
+      for (int n = 0; n < KT / 8; ++n) {
+        const float p0 = exp2f(s[n][0] - sub0), p1 = exp2f(s[n][1] - sub0);
+        const float p2 = exp2f(s[n][2] - sub1), p3 = exp2f(s[n][3] - sub1);
+        rs0 += p0 + p1, rs1 += p2 + p3;
+        pf[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
+        pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+      }
+      l0 = l0 * c0 + rs0, l1 = l1 * c1 + rs1;
+#pragma unroll
+      for (int n = 0; n < DH / 8; ++n) {
+        o[n][0] *= c0, o[n][1] *= c0, o[n][2] *= c1, o[n][3] *= c1;
+      }
+      // ---------------- O += P V ----------------------------------------------------------------------
+      const uint32_t v_base = smem_u32(Vb + (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * LDS + (lane >> 4) * 8);
+#pragma unroll
+      for (int kj = 0; kj < KT / 16; ++kj) {
+#pragma unroll
+        for (int np = 0; np < DH / 16; ++np) {
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(v_base + (uint32_t)(kj * 16 * LDS * 2) + np * 32, b0, b1, b2, b3);
+          mma_bf16(o[2 * np], pf[kj], b0, b1);
+          mma_bf16(o[2 * np + 1], pf[kj], b2, b3);
+        }
+      }
+    }
+    __syncthreads();  // everyone is done with `buf` before it is refilled
+  }
+
+  // ---- finish: quad-reduce the row sums, write output or partial ----------------------------------------
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  if (abort_flag) return;
+  const int head = head0 + hl;
+  if (a.num_splits == 1) {
+    const float i0 = 1.0f / l0, i1 = 1.0f / l1;
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n) {
+      const int col = head * DH + n * 8 + qd * 2;
+      if (row0 < S)
+        *reinterpret_cast<uint32_t*>(a.out + tiled_index(b * S + row0, col, a.rows_pad)) =
+            pack_bf16(o[n][0] * i0, o[n][1] * i0);
+      if (row1 < S)
+        *reinterpret_cast<uint32_t*>(a.out + tiled_index(b * S + row1, col, a.rows_pad)) =
+            pack_bf16(o[n][2] * i1, o[n][3] * i1);
+    }
+  } else {
+    const size_t slab = ((size_t)(b * d.Hq + head) * a.num_splits + split) * QROWS;
+    float* po = a.part_o + slab * DH;
+    float* pm = a.part_ml + slab * 2;
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n) {
+      const int col = n * 8 + qd * 2;
+      if (row0 < S) *reinterpret_cast<float2*>(po + (size_t)row0 * DH + col) = make_float2(o[n][0], o[n][1]);
+      if (row1 < S) *reinterpret_cast<float2*>(po + (size_t)row1 * DH + col) = make_float2(o[n][2], o[n][3]);
+    }
+    if (qd == 0) {
+      if (row0 < S) pm[row0 * 2] = m0, pm[row0 * 2 + 1] = l0;
+      if (row1 < S) pm[row1 * 2] = m1, pm[row1 * 2 + 1] = l1;
+    }
+  }
+}
+
+// Combine the per-split partials: out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s.
+template <int DH>
+__global__ void k_attn_merge(const int* status, const float* part_o, const float* part_ml, __nv_bfloat16* out,
+                             int rows_pad, int num_splits, int S, int Hq) {
+  if (status_set(status)) return;
+  const int row = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
+  const size_t slab0 = ((size_t)(b * Hq + head) * num_splits) * QROWS;
+  float mm = -INFINITY;
+  for (int s = 0; s < num_splits; ++s) mm = fmaxf(mm, part_ml[(slab0 + (size_t)s * QROWS + row) * 2]);
+  float ll = 0.f;
+  for (int s = 0; s < num_splits; ++s) {
+    const float* ml = part_ml + (slab0 + (size_t)s * QROWS + row) * 2;
+    if (ml[0] != -INFINITY) ll += exp2f(ml[0] - mm) * ml[1];
+  }
+  const float inv = 1.0f / ll;
+  for (int c = threadIdx.x * 2; c < DH; c += blockDim.x * 2) {
+    float a0 = 0.f, a1 = 0.f;
+    for (int s = 0; s < num_splits; ++s) {
+      const float ms = part_ml[(slab0 + (size_t)s * QROWS + row) * 2];
+      if (ms == -INFINITY) continue;
+      const float w = exp2f(ms - mm);
+      const float2 v = *reinterpret_cast<const float2*>(part_o + (slab0 + (size_t)s * QROWS + row) * DH + c);
+      a0 = fmaf(w, v.x, a0), a1 = fmaf(w, v.y, a1);
+    }
+    *reinterpret_cast<uint32_t*>(out + tiled_index(b * S + row, head * DH + c, rows_pad)) =
+        pack_bf16(a0 * inv, a1 * inv);
+  }
+}
+
+template <int DH, int HPC>
+constexpr size_t attn_smem() {
+  return (size_t)(HPC * QROWS + 4 * KT) * (DH + 8) * 2;
+}
+
+template <int DH, int HPC>
+cudaError_t launch_attn(const AttnArgs& a, int batch, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_attn_mma<DH, HPC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)attn_smem<DH, HPC>());
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid(a.num_splits, a.d.Hq / HPC, batch);
+  k_attn_mma<DH, HPC><<<grid, HPC * 128, attn_smem<DH, HPC>(), st>>>(a);
+  if (a.num_splits > 1) {
+    dim3 g2(a.d.S, a.d.Hq, batch);
+    k_attn_merge<DH><<<g2, 128, 0, st>>>(a.status, a.part_o, a.part_ml, a.out, a.rows_pad, a.num_splits, a.d.S, a.d.Hq);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool attention_mma_supported(const Dims& d) {
+  return (d.dh == 64 || d.dh == 128 || d.dh == 256) && d.S <= QROWS;
+}
+
+int attention_pick_splits(const Dims& d, int batch, int max_prefix) {
+  const int ctas = batch * d.Hq;
+  int want = (2 * 148 + ctas - 1) / ctas;
+  const int tiles = (max_prefix + KT - 1) / KT + 1;
+  if (want > tiles) want = tiles;
+  if (want > 16) want = 16;
+  return want < 1 ? 1 : want;
+}
+
+size_t attention_scratch_floats(const Dims& d, int batch, int splits) {
+  return splits > 1 ? (size_t)batch * d.Hq * splits * QROWS * (d.dh + 2) : 0;
+}
+
+cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qkv, const float2* rope, int layer,
+                                 __nv_bfloat16* out_tiled, int rows_pad, int num_splits, float* scratch, const Dims& d,
+                                 int batch, unsigned wait_limit, cudaStream_t st) {
+  AttnArgs a;
+  a.rq = rq, a.status = status, a.qkv = qkv, a.rope = rope, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
+  a.num_splits = num_splits, a.d = d, a.wait_limit = wait_limit;
+  a.part_o = scratch;
+  a.part_ml = scratch ? scratch + (size_t)batch * d.Hq * num_splits * QROWS * d.dh : nullptr;
+  const int G = d.Hq / d.Hkv;
+  const bool two = (G % 2 == 0) && (batch * d.Hq * num_splits >= 2 * 296);
+  if (d.dh == 256) return two ? launch_attn<256, 2>(a, batch, st) : launch_attn<256, 1>(a, batch, st);
+  if (d.dh == 128) return two ? launch_attn<128, 2>(a, batch, st) : launch_attn<128, 1>(a, batch, st);
+  return two ? launch_attn<64, 2>(a, batch, st) : launch_attn<64, 1>(a, batch, st);
+}
+
+}  // namespace phyai

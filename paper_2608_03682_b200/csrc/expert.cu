@@ -78,6 +78,9 @@ struct phyai_expert {
   float *xn_f = nullptr, *attn_f = nullptr, *m_f = nullptr, *u_f = nullptr;
   __nv_bfloat16 *xn_t = nullptr, *attn_t = nullptr, *m_t = nullptr, *u_t = nullptr;
 
+  float* attn_scratch = nullptr;  // split-KV partials of the tensor-core attention
+  bool attn_mma = false;
+
   Request* rq = nullptr;
   int* cu_internal = nullptr;
   int* status = nullptr;
@@ -271,9 +274,17 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         g.out = h->qkv, g.ldo = d.Nqkv;
         simt_gemm(g);
       }
-      launch_attention_simt(h->rq, h->status, h->qkv, h->rope, l, h->cfg.dtype != PHYAI_F32, h->attn_f, h->attn_t,
-                            h->Mpad, d, batch, st);
-      ++cnt;
+      if (h->attn_mma) {
+        const int splits = attention_pick_splits(d, batch, (int)h->cfg.max_prefix_len);
+        cudaError_t e = launch_attention_mma(h->rq, h->status, h->qkv, h->rope, l, h->attn_t, h->Mpad, splits,
+                                             h->attn_scratch, d, batch, h->wait_limit, st);
+        if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
+        cnt += splits > 1 ? 2 : 1;
+      } else {
+        launch_attention_simt(h->rq, h->status, h->qkv, h->rope, l, h->cfg.dtype != PHYAI_F32, h->attn_f, h->attn_t,
+                              h->Mpad, d, batch, st);
+        ++cnt;
+      }
       if (h->tc) {
         TcGemm g{};
         g.W = h->p_o[l], g.X = h->attn_t, g.N = D, g.K = d.Nq, g.epi = TC_RESID, g.scale = h->s_o[l], g.gate = gate;
@@ -565,6 +576,15 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
     ST(h->alloc(&h->qkv, Mp * Nqkv, true));
     ST(h->alloc(&h->state_tok, (size_t)cfg->max_batch * D, true));
     if (tc) {
+      h->attn_mma = attention_mma_supported(d);
+      if (h->attn_mma) {
+        size_t need = 0;
+        for (int bb = 1; bb <= (int)cfg->max_batch; ++bb) {
+          const size_t n = attention_scratch_floats(d, bb, attention_pick_splits(d, bb, (int)cfg->max_prefix_len));
+          need = n > need ? n : need;
+        }
+        if (need) ST(h->alloc(&h->attn_scratch, need, true));
+      }
       ST(h->alloc(&h->xn_t, Mp * D, true));
       ST(h->alloc(&h->attn_t, Mp * Nq, true));
       ST(h->alloc(&h->m_t, Mp * F, true));

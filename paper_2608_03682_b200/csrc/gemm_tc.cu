@@ -17,53 +17,10 @@
 // Every wait is bounded: on expiry the CTA raises the status word, stops issuing copies, and
 // drains to its normal exit (TMEM is always released).
 #include "kernels.h"
+#include "ptx.cuh"
 
 namespace phyai {
 namespace {
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-
-struct WaitCtx {
-  int* status;
-  volatile int* abort_flag;  // shared memory, CTA-wide
-  uint32_t limit;
-};
-// Bounded wait.  Returns false (and records ST_TIMEOUT) when the limit expires or the CTA has
-// already given up; callers then skip their side effects but keep walking their loops.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& c) {
-  if (*c.abort_flag) return false;
-  for (uint32_t it = 0; it < c.limit; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if (it > 128) __nanosleep(32);
-  }
-  *c.abort_flag = 1;
-  atomicExch(c.status, ST_TIMEOUT);
-  return false;
-}
-
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
 
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols)

@@ -71,6 +71,14 @@ void launch_attention_simt(const Request* rq, const int* status, const float* qk
                            int kv_is_bf16, float* out_f32, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
                            int batch, cudaStream_t st);
 
+// ---- tensor-core attention (mma.sync, bulk-copy staged K/V) ------------------------------------------
+bool attention_mma_supported(const Dims& d);
+int attention_pick_splits(const Dims& d, int batch, int max_prefix);
+size_t attention_scratch_floats(const Dims& d, int batch, int splits);  // split-KV partials (O, m, l)
+cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qkv, const float2* rope, int layer,
+                                 __nv_bfloat16* out_tiled, int rows_pad, int num_splits, float* scratch, const Dims& d,
+                                 int batch, unsigned wait_limit, cudaStream_t st);
+
 // ---- tcgen05 GEMM ------------------------------------------------------------------------------
 enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3 };
 struct TcGemm {

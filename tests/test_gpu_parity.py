@@ -70,3 +70,69 @@ def test_pi_shaped_bf16_batch1_matches_oracle(name):
     err = rel_err(got, ref)
     print(f"{name}: max rel err {err:.3e}, ||ref||inf {np.abs(ref).max():.3f}")
     assert err <= BAR["bf16"], err
+
+
+# ------------------------------------------------------------------------------------------ batched, ragged
+def _batched_case(cfg, cfg_id, lens, n_steps, check, engine="auto", std=0.05):
+    W = synth.make_weights(cfg, cfg_id, std=std)
+    kvs = [synth.make_prefix_kv(cfg, cfg_id, int(p), b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    B = len(lens)
+    states = torch.stack([synth.make_state(cfg, cfg_id, b) for b in range(B)]) if cfg.has_state_token else None
+    noise = torch.stack([synth.make_noise(cfg, cfg_id, b) for b in range(B)])
+    with binding.Expert(cfg, binding.weights_to_device(W), engine=engine) as ex:
+        out = ex.denoise_batched(packed.cuda(), torch.from_numpy(cu).cuda(), None if states is None else states.cuda(),
+                                 noise.cuda(), n_steps)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        out = out.double().cpu().numpy()
+        singles = {}
+        for b in check:
+            singles[b] = ex.denoise(kvs[b].cuda(), int(lens[b]), None if states is None else states[b].cuda(),
+                                    noise[b].cuda(), n_steps).double().cpu().numpy()
+        torch.cuda.synchronize()
+    bar = BAR["f32"] if (cfg.dtype == "f32" or engine == "simt") else BAR["bf16"]
+    Wf = O.Weights(W)
+    for b in check:
+        ref = O.denoise(cfg, Wf, kvs[b], int(lens[b]), None if states is None else states[b], noise[b], n_steps)
+        assert rel_err(out[b], ref) <= bar, (b, rel_err(out[b], ref))
+        # the batched call and the single-request call agree far inside the bar (split-K order differs)
+        assert rel_err(out[b], singles[b]) <= bar / 4, (b, rel_err(out[b], singles[b]))
+    assert np.isfinite(out).all()
+
+
+@pytest.mark.parametrize("cond", ["pi0", "pi05"])
+def test_small_bf16_ragged_batch_matches_oracle_per_request(cond):
+    cfg = small_bf16_config(cond, max_batch=5)
+    _batched_case(cfg, 13, [200, 0, 63, 64, 129], 3, check=[0, 1, 2, 3, 4])
+
+
+def test_small_bf16_large_batch_uses_wide_tiles_and_unsplit_attention():
+    cfg = small_bf16_config("pi0", max_batch=300, max_prefix_len=96)
+    lens = synth.make_ragged_lengths(14, 300, 10, 96)
+    order = np.argsort(lens)
+    _batched_case(cfg, 14, lens, 2, check=[0, 299, int(order[0]), int(order[-1])])
+
+
+def test_fp32_ragged_batch_matches_oracle_per_request():
+    cfg = synth.ExpertConfig(n_layers=2, width=64, mlp_dim=96, n_q_heads=2, n_kv_heads=2, head_dim=16, state_dim=3,
+                             action_dim=4, horizon=6, has_state_token=True, max_prefix_len=30, max_batch=4,
+                             cond="pi0", dtype="f32")
+    _batched_case(cfg, 15, [30, 0, 7, 19], 3, check=[0, 1, 2, 3], std=0.1)
+
+
+def test_bad_cu_prefix_lens_is_reported_and_nothing_is_written():
+    cfg = small_bf16_config("pi0", max_batch=2)
+    W = synth.make_weights(cfg, 13, std=0.05)
+    kv = synth.make_prefix_kv(cfg, 13, 50).cuda()
+    noise = torch.stack([synth.make_noise(cfg, 13, b) for b in range(2)]).cuda()
+    states = torch.stack([synth.make_state(cfg, 13, b) for b in range(2)]).cuda()
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        out = torch.full_like(noise, 7.0)
+        ex.denoise_batched(kv, torch.tensor([0, 40, 30], dtype=torch.int32).cuda(), states, noise, 2, out=out)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == binding.ERR_INVALID_ARG
+        assert bool((out == 7.0).all())
+        ex.denoise_batched(kv, torch.tensor([0, 20, 50], dtype=torch.int32).cuda(), states, noise, 2, out=out)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0 and bool(torch.isfinite(out).all())
