@@ -200,6 +200,46 @@ phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t valu
  * 0 if unknown.  Reporting aid for benchmarks. */
 uint64_t phyai_launches_per_call(phyai_expert_t *h, uint32_t batch, uint32_t n_steps);
 
+/*
+ * Stand-alone operator: suffix -> (prefix U suffix) attention of one layer (operator-selection
+ * paragraph: a ~50-token query against a longer prefix, head dimension 256), the kernel the
+ * denoising loop uses, callable on its own.
+ *
+ *   desc            shapes; head_dim in {64,128,256}, suffix_len <= 64; num_splits 0 lets the
+ *                   library choose how many CTAs share one request's key range (1..16 to fix it)
+ *   qkv             device float32 [batch*suffix_len][(Hq + 2 Hkv) * head_dim] = (q | k | v) rows of
+ *                   the suffix tokens, NOT yet rotated
+ *   prefix_kv       device bfloat16 [n_layers][2][kv_tokens][Hkv][head_dim]; planes of `layer` are read
+ *   cu_prefix_lens  device int32 [batch+1]
+ *   rope_cos_sin    device float32 [positions][head_dim/2][2] = (cos, sin) of position * theta^(-2j/dh)
+ *                   for every position < max prefix_len + suffix_len, or NULL for no rotation;
+ *                   suffix token i of a request sits at position prefix_len + i
+ *   out             device bfloat16 (as uint16) row-major [batch*suffix_len][Hq*head_dim]
+ *   status_word     device int32, zeroed by the caller; stays 0 on success, becomes
+ *                   PHYAI_ERR_TIMEOUT if a bounded wait inside the kernel expired
+ *
+ * Split-KV partial results need scratch memory: this entry point takes it from the stream-ordered
+ * allocator (cudaMallocAsync / cudaFreeAsync on `stream`).  Only enqueues work.  Errors: INVALID_ARG,
+ * UNSUPPORTED, OOM, CUDA; message in phyai_op_last_error().
+ */
+typedef struct {
+  uint32_t struct_size;
+  uint32_t n_q_heads, n_kv_heads, head_dim, suffix_len;
+  uint32_t n_layers, layer;
+  uint32_t state_token_block_causal; /* 1: suffix row 0 sees, of the suffix keys, only key 0 */
+  uint32_t num_splits;
+} phyai_attention_desc_t;
+
+phyai_status_t phyai_suffix_attention(const phyai_attention_desc_t *desc, uint32_t batch, const float *qkv,
+                                      const void *prefix_kv, uint64_t kv_tokens, const int32_t *cu_prefix_lens,
+                                      const float *rope_cos_sin, uint16_t *out, int32_t *status_word, void *stream);
+
+/* Scratch bytes phyai_suffix_attention uses for this shape and batch (upper bound when num_splits is 0). */
+size_t phyai_suffix_attention_scratch_bytes(const phyai_attention_desc_t *desc, uint32_t batch);
+
+/* Thread-local description of the last error of an operator entry point. */
+const char *phyai_op_last_error(void);
+
 /* Thread-local, NUL-terminated description of the last error on this thread ("" if none). */
 const char *phyai_last_error(void);
 

@@ -26,7 +26,8 @@ BIG = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
 #: every symbol the header declares
 EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes", "phyai_denoise",
            "phyai_denoise_batched", "phyai_denoise_host", "phyai_denoise_batched_host", "phyai_poll_status",
-           "phyai_set_option", "phyai_launches_per_call", "phyai_last_error", "phyai_version")
+           "phyai_set_option", "phyai_launches_per_call", "phyai_last_error", "phyai_version",
+           "phyai_suffix_attention", "phyai_suffix_attention_scratch_bytes", "phyai_op_last_error")
 
 
 class PhyaiError(RuntimeError):
@@ -45,6 +46,11 @@ class ConfigStruct(C.Structure):
 
 _VP = C.c_void_p
 _VPP = C.POINTER(C.c_void_p)
+
+
+class AttentionDesc(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("struct_size", "n_q_heads", "n_kv_heads", "head_dim", "suffix_len",
+                                          "n_layers", "layer", "state_token_block_causal", "num_splits")]
 
 
 class WeightsStruct(C.Structure):
@@ -85,6 +91,11 @@ def load_library() -> C.CDLL:
     lib.phyai_set_option.argtypes = [_VP, C.c_char_p, C.c_int64]
     lib.phyai_launches_per_call.argtypes = [_VP, C.c_uint32, C.c_uint32]
     lib.phyai_launches_per_call.restype = C.c_uint64
+    lib.phyai_op_last_error.restype = C.c_char_p
+    lib.phyai_suffix_attention_scratch_bytes.restype = C.c_size_t
+    lib.phyai_suffix_attention_scratch_bytes.argtypes = [C.POINTER(AttentionDesc), C.c_uint32]
+    lib.phyai_suffix_attention.argtypes = [C.POINTER(AttentionDesc), C.c_uint32, _VP, _VP, C.c_uint64, _VP, _VP, _VP,
+                                           _VP, _VP]
     _lib = lib
     return lib
 
@@ -242,3 +253,26 @@ def weights_to_device(weights: Dict[str, object], device="cuda") -> Dict[str, ob
     for k, v in weights.items():
         out[k] = tuple(t.to(device).contiguous() for t in v) if isinstance(v, tuple) else v.to(device).contiguous()
     return out
+
+
+def attention_desc(n_q_heads, n_kv_heads, head_dim, suffix_len, n_layers, layer, block_causal=False, num_splits=0):
+    d = AttentionDesc()
+    d.struct_size = C.sizeof(AttentionDesc)
+    d.n_q_heads, d.n_kv_heads, d.head_dim, d.suffix_len = n_q_heads, n_kv_heads, head_dim, suffix_len
+    d.n_layers, d.layer, d.state_token_block_causal, d.num_splits = n_layers, layer, int(block_causal), num_splits
+    return d
+
+
+def suffix_attention(desc: AttentionDesc, qkv: torch.Tensor, prefix_kv: torch.Tensor, cu_prefix_lens: torch.Tensor,
+                     rope_cos_sin: Optional[torch.Tensor], entry: str = "phyai_suffix_attention", stream=None):
+    """Stand-alone attention operator; returns (out bf16 [rows, Hq*dh], status_word int32 tensor)."""
+    lib = load_library()
+    batch = int(cu_prefix_lens.numel()) - 1
+    rows = batch * desc.suffix_len
+    out = torch.empty(rows, desc.n_q_heads * desc.head_dim, dtype=torch.bfloat16, device=qkv.device)
+    status = torch.zeros(1, dtype=torch.int32, device=qkv.device)
+    st = getattr(lib, entry)(C.byref(desc), batch, _ptr(qkv), _ptr(prefix_kv), int(prefix_kv.shape[2]),
+                             _ptr(cu_prefix_lens), _ptr(rope_cos_sin), _ptr(out), _ptr(status), _stream_ptr(stream))
+    if st != OK:
+        raise PhyaiError(st, lib.phyai_op_last_error().decode())
+    return out, status

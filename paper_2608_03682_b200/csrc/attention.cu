@@ -9,8 +9,9 @@
 // The suffix's own K/V (fp32 from the QKV GEMM) are rotated and appended as the last tile.
 // When the key range is split over several CTAs each writes an unnormalised partial (O, m, l) and a
 // merge kernel combines them.
-#include <mma.h>
+#include <cstdio>
 
+#include "../../include/phyai.h"
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -42,13 +43,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Output element index: tiled bf16 when rows_pad > 0, else row-major with leading dimension ld.
+__device__ __forceinline__ size_t out_index(int row, int col, int rows_pad, int ld) {
+  return rows_pad > 0 ? tiled_index(row, col, rows_pad) : (size_t)row * ld + col;
+}
+
 struct AttnArgs {
   const Request* rq;
   int* status;
   const float* qkv;      // [rows][Nqkv] fp32 (q | k | v), un-rotated
   const float2* rope;    // [pos][dh/2] (cos, sin) or null
   int layer;
-  __nv_bfloat16* out;    // tiled bf16 [Nq/64][rows_pad][64]
+  __nv_bfloat16* out;    // tiled bf16 [Nq/64][rows_pad][64], or row-major [rows][Nq] when rows_pad <= 0
   int rows_pad;
   int num_splits;
   float* part_o;         // [b][head][split][64][DH] unnormalised
@@ -286,10 +292,10 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
     for (int n = 0; n < DH / 8; ++n) {
       const int col = head * DH + n * 8 + qd * 2;
       if (row0 < S)
-        *reinterpret_cast<uint32_t*>(a.out + tiled_index(b * S + row0, col, a.rows_pad)) =
+        *reinterpret_cast<uint32_t*>(a.out + out_index(b * S + row0, col, a.rows_pad, d.Nq)) =
             pack_bf16(o[n][0] * i0, o[n][1] * i0);
       if (row1 < S)
-        *reinterpret_cast<uint32_t*>(a.out + tiled_index(b * S + row1, col, a.rows_pad)) =
+        *reinterpret_cast<uint32_t*>(a.out + out_index(b * S + row1, col, a.rows_pad, d.Nq)) =
             pack_bf16(o[n][2] * i1, o[n][3] * i1);
     }
   } else {
@@ -333,7 +339,7 @@ __global__ void k_attn_merge(const int* status, const float* part_o, const float
       const float2 v = *reinterpret_cast<const float2*>(part_o + (slab0 + (size_t)s * QROWS + row) * DH + c);
       a0 = fmaf(w, v.x, a0), a1 = fmaf(w, v.y, a1);
     }
-    *reinterpret_cast<uint32_t*>(out + tiled_index(b * S + row, head * DH + c, rows_pad)) =
+    *reinterpret_cast<uint32_t*>(out + out_index(b * S + row, head * DH + c, rows_pad, Hq * DH)) =
         pack_bf16(a0 * inv, a1 * inv);
   }
 }
@@ -396,3 +402,97 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
 }
 
 }  // namespace phyai
+
+// =============================================================================================
+// Stand-alone operator entry point
+// =============================================================================================
+namespace phyai {
+namespace {
+
+thread_local char g_op_err[256] = "";
+
+// Shared body of the operator entry points: fills the request block at the head of `scratch`,
+// then launches the attention (and merge) kernels with the split-KV partials placed after it.
+phyai_status_t attention_op(const phyai_attention_desc_t* desc, uint32_t batch, const float* qkv, const void* prefix_kv,
+                            uint64_t kv_tokens, const int32_t* cu, const float* rope, uint16_t* out, int32_t* status_word,
+                            void* scratch, size_t scratch_bytes, cudaStream_t st) {
+  auto bad = [](const char* m) {
+    snprintf(g_op_err, sizeof(g_op_err), "%s", m);
+    return PHYAI_ERR_INVALID_ARG;
+  };
+  if (!desc || desc->struct_size != sizeof(phyai_attention_desc_t)) return bad("desc is NULL or has a wrong struct_size");
+  if (!qkv || !cu || !out || !status_word || !batch) return bad("qkv / cu_prefix_lens / out / status_word is NULL or batch is 0");
+  if (kv_tokens && !prefix_kv) return bad("prefix_kv is NULL with kv_tokens > 0");
+  if ((reinterpret_cast<uintptr_t>(prefix_kv) & 15u) || (reinterpret_cast<uintptr_t>(out) & 3u))
+    return bad("prefix_kv must be 16-byte aligned and out 4-byte aligned");
+  if (!desc->n_q_heads || !desc->n_kv_heads || desc->n_q_heads % desc->n_kv_heads || desc->layer >= desc->n_layers)
+    return bad("head counts or layer index out of range");
+  if (kv_tokens > (uint64_t)INT32_MAX || batch > (1u << 16)) return bad("kv_tokens or batch too large");
+  Dims d{};
+  d.L = (int)desc->n_layers, d.Hq = (int)desc->n_q_heads, d.Hkv = (int)desc->n_kv_heads, d.dh = (int)desc->head_dim;
+  d.S = (int)desc->suffix_len, d.H = d.S, d.Nq = d.Hq * d.dh, d.Nqkv = (d.Hq + 2 * d.Hkv) * d.dh;
+  d.block_causal = desc->state_token_block_causal ? 1 : 0, d.ns = d.block_causal;
+  if (!attention_mma_supported(d)) {
+    snprintf(g_op_err, sizeof(g_op_err), "head_dim must be 64, 128 or 256 and suffix_len <= 64");
+    return PHYAI_ERR_UNSUPPORTED;
+  }
+  int splits = (int)desc->num_splits;
+  if (splits == 0) splits = attention_pick_splits(d, (int)batch, (int)(kv_tokens < 4096 ? kv_tokens : 4096));
+  if (splits < 1 || splits > 16) return bad("num_splits must be 0 (choose) or 1..16");
+  const size_t need = 256 + attention_scratch_floats(d, (int)batch, splits) * sizeof(float);
+  if (need > scratch_bytes) {
+    snprintf(g_op_err, sizeof(g_op_err), "needs %zu bytes of scratch, only %zu available", need, scratch_bytes);
+    return PHYAI_ERR_INVALID_ARG;
+  }
+  Request r{};
+  r.prefix_kv = prefix_kv, r.kv_tokens = kv_tokens, r.cu_lens = cu, r.batch = (int)batch;
+  Request* rq = reinterpret_cast<Request*>(scratch);
+  launch_set_request(rq, r, nullptr, st);
+  float* partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(scratch) + 256);
+  cudaError_t e = launch_attention_mma(rq, status_word, qkv, reinterpret_cast<const float2*>(rope), (int)desc->layer,
+                                       reinterpret_cast<__nv_bfloat16*>(out), 0, splits, splits > 1 ? partials : nullptr,
+                                       d, (int)batch, 1u << 22, st);
+  if (e != cudaSuccess) {
+    snprintf(g_op_err, sizeof(g_op_err), "attention launch failed: %s", cudaGetErrorString(e));
+    return PHYAI_ERR_CUDA;
+  }
+  return PHYAI_OK;
+}
+
+}  // namespace
+}  // namespace phyai
+
+extern "C" {
+
+const char* phyai_op_last_error(void) { return phyai::g_op_err; }
+
+size_t phyai_suffix_attention_scratch_bytes(const phyai_attention_desc_t* desc, uint32_t batch) {
+  if (!desc || !batch) return 0;
+  phyai::Dims d{};
+  d.Hq = (int)desc->n_q_heads, d.Hkv = (int)desc->n_kv_heads, d.dh = (int)desc->head_dim, d.S = (int)desc->suffix_len;
+  const int splits = desc->num_splits ? (int)desc->num_splits : 16;
+  return 256 + phyai::attention_scratch_floats(d, (int)batch, splits) * sizeof(float);
+}
+
+phyai_status_t phyai_suffix_attention(const phyai_attention_desc_t* desc, uint32_t batch, const float* qkv,
+                                      const void* prefix_kv, uint64_t kv_tokens, const int32_t* cu_prefix_lens,
+                                      const float* rope_cos_sin, uint16_t* out, int32_t* status_word, void* stream) {
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const size_t bytes = phyai_suffix_attention_scratch_bytes(desc, batch);
+  if (!bytes) {
+    snprintf(phyai::g_op_err, sizeof(phyai::g_op_err), "desc is NULL or batch is 0");
+    return PHYAI_ERR_INVALID_ARG;
+  }
+  void* scratch = nullptr;
+  cudaError_t e = cudaMallocAsync(&scratch, bytes, st);
+  if (e != cudaSuccess) {
+    snprintf(phyai::g_op_err, sizeof(phyai::g_op_err), "cudaMallocAsync(%zu) failed: %s", bytes, cudaGetErrorString(e));
+    return PHYAI_ERR_OOM;
+  }
+  phyai_status_t s = phyai::attention_op(desc, batch, qkv, prefix_kv, kv_tokens, cu_prefix_lens, rope_cos_sin, out,
+                                         status_word, scratch, bytes, st);
+  cudaFreeAsync(scratch, st);  // stream-ordered: released after the kernels above have run
+  return s;
+}
+
+}  // extern "C"
