@@ -237,6 +237,34 @@ phyai_status_t phyai_suffix_attention(const phyai_attention_desc_t *desc, uint32
 /* Scratch bytes phyai_suffix_attention uses for this shape and batch (upper bound when num_splits is 0). */
 size_t phyai_suffix_attention_scratch_bytes(const phyai_attention_desc_t *desc, uint32_t batch);
 
+/*
+ * phyai_suffix_attention without any allocation.  (The paper has no counterpart; this entry point
+ * exists for callers that must not allocate device memory: code running where cudaMalloc is
+ * forbidden or unavailable, for example a real-time control loop with a no-allocation rule after
+ * start-up, a process whose memory pool is owned and capped by another component, or a plug-in
+ * that may only use the buffers it is handed.)
+ *
+ * Same arguments, same result as phyai_suffix_attention; the caller still passes inputs, the
+ * output and the status word.  The request block and the split-KV partials go into a fixed
+ * 16 MiB array (phyai_suffix_attention_static_capacity()) that is part of the library image: every GPU that
+ * loads the library holds it until the process exits.  The call uses no cudaMalloc, cudaFree,
+ * stream-ordered allocator or other allocating routine.
+ *
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and remembers it; make that first call before starting any stream capture.
+ *   - Shapes that need more than the capacity (256 bytes + batch * Hq * splits * 64 * (head_dim + 2) * 4)
+ *     are rejected with PHYAI_ERR_INVALID_ARG and a message naming both numbers; with
+ *     num_splits == 0 the library picks a split count first and then checks.
+ *   - All calls on a device share the one array and it keeps the last call's contents.  Nothing
+ *     in it needs clearing between calls, but two calls that overlap on the GPU (different
+ *     streams, or different host threads) race on it: serialise them.
+ */
+phyai_status_t phyai_suffix_attention_static(const phyai_attention_desc_t *desc, uint32_t batch, const float *qkv,
+                                             const void *prefix_kv, uint64_t kv_tokens,
+                                             const int32_t *cu_prefix_lens, const float *rope_cos_sin, uint16_t *out,
+                                             int32_t *status_word, void *stream);
+size_t phyai_suffix_attention_static_capacity(void);
+
 /* Thread-local description of the last error of an operator entry point. */
 const char *phyai_op_last_error(void);
 

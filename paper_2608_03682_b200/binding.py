@@ -27,7 +27,8 @@ BIG = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
 EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes", "phyai_denoise",
            "phyai_denoise_batched", "phyai_denoise_host", "phyai_denoise_batched_host", "phyai_poll_status",
            "phyai_set_option", "phyai_launches_per_call", "phyai_last_error", "phyai_version",
-           "phyai_suffix_attention", "phyai_suffix_attention_scratch_bytes", "phyai_op_last_error")
+           "phyai_suffix_attention", "phyai_suffix_attention_scratch_bytes", "phyai_op_last_error",
+           "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity")
 
 
 class PhyaiError(RuntimeError):
@@ -96,6 +97,8 @@ def load_library() -> C.CDLL:
     lib.phyai_suffix_attention_scratch_bytes.argtypes = [C.POINTER(AttentionDesc), C.c_uint32]
     lib.phyai_suffix_attention.argtypes = [C.POINTER(AttentionDesc), C.c_uint32, _VP, _VP, C.c_uint64, _VP, _VP, _VP,
                                            _VP, _VP]
+    lib.phyai_suffix_attention_static.argtypes = lib.phyai_suffix_attention.argtypes
+    lib.phyai_suffix_attention_static_capacity.restype = C.c_size_t
     _lib = lib
     return lib
 

@@ -10,6 +10,7 @@
 // When the key range is split over several CTAs each writes an unnormalised partial (O, m, l) and a
 // merge kernel combines them.
 #include <cstdio>
+#include <mutex>
 
 #include "../../include/phyai.h"
 #include "kernels.h"
@@ -493,6 +494,78 @@ phyai_status_t phyai_suffix_attention(const phyai_attention_desc_t* desc, uint32
                                          status_word, scratch, bytes, st);
   cudaFreeAsync(scratch, st);  // stream-ordered: released after the kernels above have run
   return s;
+}
+
+}  // extern "C"
+
+// =============================================================================================
+// Attention operator that allocates nothing
+// =============================================================================================
+// Scratch for the request block and the split-KV partials lives in this fixed array instead of
+// coming from an allocator.  Every GPU that loads the library holds it until the process exits.
+#define PHYAI_STATIC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[PHYAI_STATIC_SCRATCH_BYTES];
+
+namespace phyai {
+namespace {
+
+std::mutex g_static_mu;
+void* g_static_ptr[64] = {};  // per device: device address of g_static_scratch
+
+// In host code `g_static_scratch` is only a stand-in for the symbol; the address a kernel can use
+// has to be looked up once per device, with that device current.
+phyai_status_t static_scratch_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= 64) {
+    snprintf(g_op_err, sizeof(g_op_err), "cudaGetDevice failed or device index %d is outside 0..63", dev);
+    return PHYAI_ERR_CUDA;
+  }
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess || !p) {
+      snprintf(g_op_err, sizeof(g_op_err), "cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+      return PHYAI_ERR_CUDA;
+    }
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return PHYAI_OK;
+}
+
+}  // namespace
+}  // namespace phyai
+
+extern "C" {
+
+size_t phyai_suffix_attention_static_capacity(void) { return PHYAI_STATIC_SCRATCH_BYTES; }
+
+phyai_status_t phyai_suffix_attention_static(const phyai_attention_desc_t* desc, uint32_t batch, const float* qkv,
+                                             const void* prefix_kv, uint64_t kv_tokens, const int32_t* cu_prefix_lens,
+                                             const float* rope_cos_sin, uint16_t* out, int32_t* status_word,
+                                             void* stream) {
+  const size_t need = phyai_suffix_attention_scratch_bytes(desc, batch);
+  if (!need) {
+    snprintf(phyai::g_op_err, sizeof(phyai::g_op_err), "desc is NULL or batch is 0");
+    return PHYAI_ERR_INVALID_ARG;
+  }
+  if (desc->num_splits != 0 && need > (size_t)PHYAI_STATIC_SCRATCH_BYTES) {
+    snprintf(phyai::g_op_err, sizeof(phyai::g_op_err),
+             "this shape needs %zu bytes of scratch but the built-in scratch holds %u: lower batch or num_splits, or "
+             "use phyai_suffix_attention",
+             need, PHYAI_STATIC_SCRATCH_BYTES);
+    return PHYAI_ERR_INVALID_ARG;
+  }
+  void* scratch = nullptr;
+  phyai_status_t s = phyai::static_scratch_address(&scratch);
+  if (s != PHYAI_OK) return s;
+  // attention_op re-derives the exact requirement (after choosing num_splits) and refuses sizes
+  // beyond the capacity passed here.  Nothing in the scratch has to start at zero: the request
+  // block is rewritten by every call and every partial that is read was written by the same call.
+  return phyai::attention_op(desc, batch, qkv, prefix_kv, kv_tokens, cu_prefix_lens, rope_cos_sin, out, status_word,
+                             scratch, PHYAI_STATIC_SCRATCH_BYTES, reinterpret_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"
