@@ -2,9 +2,11 @@
 // a ~50-token query against a longer prefix with head dimension 256).
 //
 // Few queries, long shared KV: one CTA takes the (<= 64) suffix rows of HPC query heads that share a
-// kv head and a contiguous slice of that request's keys.  K/V rows are staged into shared memory by
-// the bulk-copy engine, one 1-D copy per row into rows padded by 16 bytes (bank-conflict-free
-// ldmatrix without a swizzle), double buffered.  Q K^T and P V run on mma.sync m16n8k16 (bf16 in,
+// kv head and a contiguous slice of that request's keys.  K/V tiles are staged into shared memory
+// with 16-byte asynchronous copies issued by all threads into XOR-swizzled rows (bank-conflict-free
+// ldmatrix), double buffered.  (Per-row bulk copies were measured first: one warp's bulk copies
+// complete one at a time, which made 128 small copies per tile the bottleneck.)  Q K^T and P V run on
+// mma.sync m16n8k16 (bf16 in,
 // fp32 out); the softmax is the online form in fp32 with quad shuffles for the row max / sum.
 // The suffix's own K/V (fp32 from the QKV GEMM) are rotated and appended as the last tile.
 // When the key range is split over several CTAs each writes an unnormalised partial (O, m, l) and a
@@ -64,18 +66,30 @@ struct AttnArgs {
   unsigned wait_limit;
 };
 
+// Shared-memory tiles are rows of DH bf16 with no padding; the 16-byte chunk c of row r sits at
+// chunk position c ^ (r & 7), which makes every ldmatrix (8 rows x 16 bytes) bank-conflict free.
+__device__ __forceinline__ uint32_t swz(int row, int chunk, int rowb) {
+  return (uint32_t)row * rowb + (uint32_t)((chunk ^ (row & 7)) << 4);
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 // DH: head_dim; HPC: query heads per CTA (4 warps each).
 template <int DH, int HPC>
 __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
-  constexpr int LDS = DH + 8;                 // padded row stride in elements (+16 bytes)
-  constexpr int ROWB = DH * 2;                // bytes per K/V row
+  constexpr int ROWB = DH * 2;                // bytes per row
+  constexpr int CH = DH / 8;                  // 16-byte chunks per row
   constexpr int NTHREADS = HPC * 128;
-  extern __shared__ __align__(16) uint8_t smem_raw[];
-  __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem_raw);          // [HPC*64][LDS]
-  __nv_bfloat16* Ks = Qs + (size_t)HPC * QROWS * LDS;                       // [2][KT][LDS]
-  __nv_bfloat16* Vs = Ks + (size_t)2 * KT * LDS;                            // [2][KT][LDS]
-  __shared__ __align__(8) uint64_t bar_full[2];
-  __shared__ int abort_flag, skip_flag;
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  const uint32_t Qs = smem_u32(smem_raw);                         // [HPC*64] rows
+  const uint32_t Ks = Qs + (uint32_t)HPC * QROWS * ROWB;          // [2][KT] rows
+  const uint32_t Vs = Ks + 2u * KT * ROWB;                        // [2][KT] rows
 
   const Dims& d = a.d;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -83,17 +97,7 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
   const int head0 = hgrp * HPC;
   const int hk = head0 / (d.Hq / d.Hkv);
   const int S = d.S;
-
-  if (tid == 0) {
-    skip_flag = status_set(a.status);
-    abort_flag = 0;
-    mbar_init(smem_u32(&bar_full[0]), 1);
-    mbar_init(smem_u32(&bar_full[1]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-  if (skip_flag) return;
-  const WaitCtx wc{a.status, &abort_flag, a.wait_limit};
+  if (status_set(a.status)) return;   // no block-wide waits depend on other blocks: a plain early exit is safe
 
   const Request r = *a.rq;
   const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
@@ -102,123 +106,122 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
   const int t_begin = (int)(((long long)T * split) / a.num_splits);
   const int t_end = (int)(((long long)T * (split + 1)) / a.num_splits);
 
-  const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(r.prefix_kv) +
-                            ((size_t)(a.layer * 2 + 0) * r.kv_tokens + p0) * d.Hkv * DH + (size_t)hk * DH;
-  const __nv_bfloat16* Vg = reinterpret_cast<const __nv_bfloat16*>(r.prefix_kv) +
-                            ((size_t)(a.layer * 2 + 1) * r.kv_tokens + p0) * d.Hkv * DH + (size_t)hk * DH;
-  const size_t kv_stride = (size_t)d.Hkv * DH;
-  const int half = DH / 2;
+  const uint8_t* Kg = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
+                      (((size_t)(a.layer * 2 + 0) * r.kv_tokens + p0) * d.Hkv + hk) * ROWB;
+  const uint8_t* Vg = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
+                      (((size_t)(a.layer * 2 + 1) * r.kv_tokens + p0) * d.Hkv + hk) * ROWB;
+  const size_t kv_stride = (size_t)d.Hkv * ROWB;  // bytes between consecutive tokens
+  constexpr int half = DH / 2;
 
-  // ---- Q: rotate, scale by dh^-1/2, round to bf16, into shared memory -----------------------------
+  // K/V tile t -> buffer buf with 16-byte asynchronous copies; rows past the prefix are zero-filled
+  auto load_tile = [&](int t, int buf) {
+    const int rows = min(KT, P - t * KT);
+    const uint32_t kb = Ks + (uint32_t)buf * KT * ROWB, vb = Vs + (uint32_t)buf * KT * ROWB;
+    for (int idx = tid; idx < KT * CH; idx += NTHREADS) {
+      const int row = idx / CH, c = idx % CH;
+      const bool ok = row < rows;
+      const size_t g = (size_t)(t * KT + (ok ? row : 0)) * kv_stride + (size_t)c * 16;
+      const uint32_t o = swz(row, c, ROWB);
+      cp_async16(kb + o, Kg + g, ok ? 16u : 0u);
+      cp_async16(vb + o, Vg + g, ok ? 16u : 0u);
+    }
+  };
+  if (t_begin < t_end && t_begin < Tp) load_tile(t_begin, 0);
+  cp_async_commit();
+
+  // ---- Q: rotate, scale by dh^-1/2, round to bf16, into shared memory (4 column pairs per thread)
   const float qscale = rsqrtf((float)DH);
-  for (int idx = tid; idx < HPC * QROWS * half; idx += NTHREADS) {
-    const int hl = idx / (QROWS * half), rem = idx % (QROWS * half);
-    const int i = rem / half, j = rem % half;
-    float lo = 0.f, hi = 0.f;
+  for (int idx = tid; idx < HPC * QROWS * (half / 4); idx += NTHREADS) {
+    const int hl = idx / (QROWS * (half / 4)), rem = idx % (QROWS * (half / 4));
+    const int i = rem / (half / 4), j = (rem % (half / 4)) * 4;
+    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
     if (i < S) {
       const float* q = a.qkv + (size_t)(b * S + i) * d.Nqkv + (size_t)(head0 + hl) * DH;
-      lo = q[j], hi = q[j + half];
+      lo = *reinterpret_cast<const float4*>(q + j);
+      hi = *reinterpret_cast<const float4*>(q + j + half);
       if (a.rope) {
-        const float2 cs = a.rope[(size_t)(P + i) * half + j];
-        const float l2 = lo * cs.x - hi * cs.y, h2 = hi * cs.x + lo * cs.y;
-        lo = l2, hi = h2;
+        const float4 cs0 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j);
+        const float4 cs1 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j + 2);
+        const float4 l2 = make_float4(lo.x * cs0.x - hi.x * cs0.y, lo.y * cs0.z - hi.y * cs0.w,
+                                      lo.z * cs1.x - hi.z * cs1.y, lo.w * cs1.z - hi.w * cs1.w);
+        hi = make_float4(hi.x * cs0.x + lo.x * cs0.y, hi.y * cs0.z + lo.y * cs0.w, hi.z * cs1.x + lo.z * cs1.y,
+                         hi.w * cs1.z + lo.w * cs1.w);
+        lo = l2;
       }
-      lo *= qscale, hi *= qscale;
     }
-    __nv_bfloat16* dst = Qs + ((size_t)hl * QROWS + i) * LDS;
-    dst[j] = __float2bfloat16_rn(lo);
-    dst[j + half] = __float2bfloat16_rn(hi);
+    const int row = hl * QROWS + i;
+    const uint2 plo = make_uint2(pack_bf16(lo.x * qscale, lo.y * qscale), pack_bf16(lo.z * qscale, lo.w * qscale));
+    const uint2 phi = make_uint2(pack_bf16(hi.x * qscale, hi.y * qscale), pack_bf16(hi.z * qscale, hi.w * qscale));
+    asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Qs + swz(row, j >> 3, ROWB) + (j & 7) * 2), "r"(plo.x), "r"(plo.y) : "memory");
+    asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Qs + swz(row, (j + half) >> 3, ROWB) + (j & 7) * 2), "r"(phi.x), "r"(phi.y) : "memory");
   }
 
   // ---- per-warp state -----------------------------------------------------------------------------
   const int hl = warp >> 2, rb = warp & 3;             // local head, 16-row block
   const int g = lane >> 2, qd = lane & 3;              // row within 8, column pair
   const int row0 = rb * 16 + g, row1 = row0 + 8;       // this thread's two query rows
+  const int sw = lane & 7;                             // swizzle term of every ldmatrix row this lane addresses
   float o[DH / 8][4];
 #pragma unroll
   for (int n = 0; n < DH / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  const uint32_t q_row = Qs + (uint32_t)(hl * QROWS + rb * 16 + (lane & 15)) * ROWB;
+  const int q_c0 = lane >> 4;
 
-  const uint32_t q_base = smem_u32(Qs + ((size_t)hl * QROWS + rb * 16 + (lane & 15)) * LDS + (lane >> 4) * 8);
-
-  // copies of the first tile: the expected byte count is posted before any copy can complete
-  if (t_begin < t_end && t_begin < Tp && tid == 0)
-    mbar_expect_tx(smem_u32(&bar_full[0]), (uint32_t)min(KT, P - t_begin * KT) * ROWB * 2);
-  __syncthreads();  // Q visible; expect_tx posted
-  if (t_begin < t_end && t_begin < Tp && tid < min(KT, P - t_begin * KT)) {
-    const size_t gofs = (size_t)(t_begin * KT + tid) * kv_stride;
-    bulk_g2s(smem_u32(Ks + (size_t)tid * LDS), Kg + gofs, ROWB, smem_u32(&bar_full[0]));
-    bulk_g2s(smem_u32(Vs + (size_t)tid * LDS), Vg + gofs, ROWB, smem_u32(&bar_full[0]));
-  }
-
-  uint32_t phase_bits = 0u;  // bit b = parity to wait for on buffer b
   for (int t = t_begin; t < t_end; ++t) {
     const int buf = (t - t_begin) & 1;
-    const int nb = buf ^ 1;
-    __nv_bfloat16* Kb = Ks + (size_t)buf * KT * LDS;
-    __nv_bfloat16* Vb = Vs + (size_t)buf * KT * LDS;
+    const uint32_t Kb = Ks + (uint32_t)buf * KT * ROWB, Vb = Vs + (uint32_t)buf * KT * ROWB;
     int valid;  // keys of this tile that exist
-    // -- prefetch the next prefix tile into the other buffer (it was released by the barrier that
-    //    ended the previous iteration)
-    if (t + 1 < t_end && t + 1 < Tp) {
-      if (tid == 0) mbar_expect_tx(smem_u32(&bar_full[nb]), (uint32_t)min(KT, P - (t + 1) * KT) * ROWB * 2);
-    }
+    if (t + 1 < t_end && t + 1 < Tp) load_tile(t + 1, buf ^ 1);   // the other buffer was released by the
+    cp_async_commit();                                            // barrier that ended the previous iteration
     if (t < Tp) {
       valid = min(KT, P - t * KT);
-      if (valid < KT) {  // ragged last prefix tile: rows that are not copied must be finite
-        for (int idx = tid; idx < (KT - valid) * (DH / 8); idx += NTHREADS) {
-          const int rr = valid + idx / (DH / 8), c = (idx % (DH / 8)) * 8;
-          *reinterpret_cast<uint4*>(Kb + (size_t)rr * LDS + c) = make_uint4(0, 0, 0, 0);
-          *reinterpret_cast<uint4*>(Vb + (size_t)rr * LDS + c) = make_uint4(0, 0, 0, 0);
-        }
-      }
     } else {
       // -- suffix tile: rotate this request's own keys, round K and V to bf16
       valid = S;
-      for (int idx = tid; idx < KT * half; idx += NTHREADS) {
-        const int js = idx / half, j = idx % half;
-        float klo = 0.f, khi = 0.f, vlo = 0.f, vhi = 0.f;
+      for (int idx = tid; idx < KT * (half / 4); idx += NTHREADS) {
+        const int js = idx / (half / 4), j = (idx % (half / 4)) * 4;
+        float4 klo = make_float4(0.f, 0.f, 0.f, 0.f), khi = klo, vlo = klo, vhi = klo;
         if (js < S) {
           const float* kr = a.qkv + (size_t)(b * S + js) * d.Nqkv + d.Nq + (size_t)hk * DH;
           const float* vr = kr + d.Hkv * DH;
-          klo = kr[j], khi = kr[j + half], vlo = vr[j], vhi = vr[j + half];
+          klo = *reinterpret_cast<const float4*>(kr + j), khi = *reinterpret_cast<const float4*>(kr + j + half);
+          vlo = *reinterpret_cast<const float4*>(vr + j), vhi = *reinterpret_cast<const float4*>(vr + j + half);
           if (a.rope) {
-            const float2 cs = a.rope[(size_t)(P + js) * half + j];
-            const float l2 = klo * cs.x - khi * cs.y, h2 = khi * cs.x + klo * cs.y;
-            klo = l2, khi = h2;
+            const float4 cs0 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + js) * half + j);
+            const float4 cs1 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + js) * half + j + 2);
+            const float4 l2 = make_float4(klo.x * cs0.x - khi.x * cs0.y, klo.y * cs0.z - khi.y * cs0.w,
+                                          klo.z * cs1.x - khi.z * cs1.y, klo.w * cs1.z - khi.w * cs1.w);
+            khi = make_float4(khi.x * cs0.x + klo.x * cs0.y, khi.y * cs0.z + klo.y * cs0.w,
+                              khi.z * cs1.x + klo.z * cs1.y, khi.w * cs1.z + klo.w * cs1.w);
+            klo = l2;
           }
         }
-        Kb[(size_t)js * LDS + j] = __float2bfloat16_rn(klo);
-        Kb[(size_t)js * LDS + j + half] = __float2bfloat16_rn(khi);
-        Vb[(size_t)js * LDS + j] = __float2bfloat16_rn(vlo);
-        Vb[(size_t)js * LDS + j + half] = __float2bfloat16_rn(vhi);
+        const uint32_t olo = swz(js, j >> 3, ROWB) + (j & 7) * 2, ohi = swz(js, (j + half) >> 3, ROWB) + (j & 7) * 2;
+        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Kb + olo), "r"(pack_bf16(klo.x, klo.y)), "r"(pack_bf16(klo.z, klo.w)) : "memory");
+        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Kb + ohi), "r"(pack_bf16(khi.x, khi.y)), "r"(pack_bf16(khi.z, khi.w)) : "memory");
+        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Vb + olo), "r"(pack_bf16(vlo.x, vlo.y)), "r"(pack_bf16(vlo.z, vlo.w)) : "memory");
+        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Vb + ohi), "r"(pack_bf16(vhi.x, vhi.y)), "r"(pack_bf16(vhi.z, vhi.w)) : "memory");
       }
     }
-    __syncthreads();  // zero-fill / suffix tile visible; next tile's expect_tx posted
-    if (t + 1 < t_end && t + 1 < Tp && tid < min(KT, P - (t + 1) * KT) && !abort_flag) {
-      const size_t gofs = (size_t)((t + 1) * KT + tid) * kv_stride;
-      bulk_g2s(smem_u32(Ks + ((size_t)nb * KT + tid) * LDS), Kg + gofs, ROWB, smem_u32(&bar_full[nb]));
-      bulk_g2s(smem_u32(Vs + ((size_t)nb * KT + tid) * LDS), Vg + gofs, ROWB, smem_u32(&bar_full[nb]));
-    }
-    bool ok = true;
-    if (t < Tp) {
-      ok = mbar_wait(smem_u32(&bar_full[buf]), (phase_bits >> buf) & 1u, wc);
-      phase_bits ^= 1u << buf;
-    }
-    if (ok) {
+    cp_async_wait<1>();   // everything but the prefetch just issued has landed
+    __syncthreads();      // tile t (copied or built above) and Q visible to all warps
+    {
       // ---------------- S = Q K^T (16 rows x 64 keys per warp) ---------------------------------
       float s[KT / 8][4];
 #pragma unroll
       for (int n = 0; n < KT / 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
-      const uint32_t k_base = smem_u32(Kb + (size_t)((lane & 7) + (lane >> 4) * 8) * LDS + ((lane >> 3) & 1) * 8);
+      const uint32_t k_row = Kb + (uint32_t)((lane & 7) + (lane >> 4) * 8) * ROWB;
+      const int k_c0 = (lane >> 3) & 1;
 #pragma unroll 4
       for (int kk = 0; kk < DH / 16; ++kk) {
         uint32_t af[4];
-        ldsm_x4(q_base + kk * 32, af[0], af[1], af[2], af[3]);
+        ldsm_x4(q_row + (uint32_t)(((kk * 2 + q_c0) ^ sw) << 4), af[0], af[1], af[2], af[3]);
+        const uint32_t kofs = (uint32_t)(((kk * 2 + k_c0) ^ sw) << 4);
 #pragma unroll
         for (int np = 0; np < KT / 16; ++np) {
           uint32_t b0, b1, b2, b3;
-          ldsm_x4(k_base + (uint32_t)(np * 16 * LDS * 2) + kk * 32, b0, b1, b2, b3);
+          ldsm_x4(k_row + (uint32_t)(np * 16 * ROWB) + kofs, b0, b1, b2, b3);
           mma_bf16(s[2 * np], af, b0, b1);
           mma_bf16(s[2 * np + 1], af, b2, b3);
         }
@@ -265,13 +268,14 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
         o[n][0] *= c0, o[n][1] *= c0, o[n][2] *= c1, o[n][3] *= c1;
       }
       // ---------------- O += P V ----------------------------------------------------------------------
-      const uint32_t v_base = smem_u32(Vb + (size_t)((lane & 7) + ((lane >> 3) & 1) * 8) * LDS + (lane >> 4) * 8);
+      const uint32_t v_row = Vb + (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB;
+      const int v_c0 = lane >> 4;
 #pragma unroll
       for (int kj = 0; kj < KT / 16; ++kj) {
 #pragma unroll
         for (int np = 0; np < DH / 16; ++np) {
           uint32_t b0, b1, b2, b3;
-          ldsm_x4_t(v_base + (uint32_t)(kj * 16 * LDS * 2) + np * 32, b0, b1, b2, b3);
+          ldsm_x4_t(v_row + (uint32_t)(kj * 16 * ROWB) + (uint32_t)(((np * 2 + v_c0) ^ sw) << 4), b0, b1, b2, b3);
           mma_bf16(o[2 * np], pf[kj], b0, b1);
           mma_bf16(o[2 * np + 1], pf[kj], b2, b3);
         }
@@ -279,13 +283,13 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
     }
     __syncthreads();  // everyone is done with `buf` before it is refilled
   }
+  cp_async_wait<0>();
 
   // ---- finish: quad-reduce the row sums, write output or partial ----------------------------------------
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
   l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-  if (abort_flag) return;
   const int head = head0 + hl;
   if (a.num_splits == 1) {
     const float i0 = 1.0f / l0, i1 = 1.0f / l1;
@@ -347,7 +351,7 @@ __global__ void k_attn_merge(const int* status, const float* part_o, const float
 
 template <int DH, int HPC>
 constexpr size_t attn_smem() {
-  return (size_t)(HPC * QROWS + 4 * KT) * (DH + 8) * 2;
+  return (size_t)(HPC * QROWS + 4 * KT) * DH * 2;
 }
 
 template <int DH, int HPC>
@@ -396,7 +400,7 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
   a.part_o = scratch;
   a.part_ml = scratch ? scratch + (size_t)batch * d.Hq * num_splits * QROWS * d.dh : nullptr;
   const int G = d.Hq / d.Hkv;
-  const bool two = (G % 2 == 0) && (batch * d.Hq * num_splits >= 2 * 296);
+  const bool two = (G % 2 == 0) && (batch * d.Hq * num_splits >= 2 * 148);
   if (d.dh == 256) return two ? launch_attn<256, 2>(a, batch, st) : launch_attn<256, 1>(a, batch, st);
   if (d.dh == 128) return two ? launch_attn<128, 2>(a, batch, st) : launch_attn<128, 1>(a, batch, st);
   return two ? launch_attn<64, 2>(a, batch, st) : launch_attn<64, 1>(a, batch, st);

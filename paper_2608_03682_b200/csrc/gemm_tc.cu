@@ -12,8 +12,10 @@
 //   B: activations kept in the tiled bf16 layout, so an NT x 64 tile is one contiguous block.
 // Every load is therefore a 1-D bulk copy (16-byte aligned, size a multiple of 16): no tensor map.
 //
-// Warp roles (192 threads): warp 0 = copy producer, warp 1 = TMEM owner + MMA issuer,
-// warps 2..5 = epilogue (TMEM lane quarter = warp % 4).
+// Warp roles (288 threads): warps 0..3 = copy producers (stage i is loaded by warp i % 4: one
+// warp's bulk copies complete one at a time, about 0.5 us each whatever their size, so several
+// issuing warps are needed to keep more than ~30 GB/s per SM in flight), warp 4 = TMEM owner +
+// MMA issuer, warps 5..8 = epilogue (TMEM lane quarter = warp % 4).
 // Every wait is bounded: on expiry the CTA raises the status word, stops issuing copies, and
 // drains to its normal exit (TMEM is always released).
 #include "kernels.h"
@@ -77,7 +79,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
 constexpr int A_BYTES = 128 * 128;  // one weight block: 128 out channels x 64 k (bf16)
 
 template <int NT, bool DUAL, int STAGES>
-__global__ void __launch_bounds__(192, 1) k_gemm_tc(int* status, const TcGemm g) {
+__global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g) {
   constexpr int B_BYTES = NT * 128;
   constexpr int STAGE_BYTES = A_BYTES * (DUAL ? 2 : 1) + B_BYTES;
   constexpr int COLS = DUAL ? 2 * NT : NT;
@@ -116,7 +118,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tc(int* status, const TcGemm g)
     mbar_init(smem_u32(&bar_accum), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == 4) {
     tmem_alloc(smem_u32(&tmem_slot), COLS);
     tc_fence_before();
   }
@@ -125,15 +127,16 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tc(int* status, const TcGemm g)
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
   const WaitCtx wc{status, &abort_flag, g.wait_limit};
 
-  if (warp == 0) {
-    // ---------------- producer: one lane streams weight blocks and activation tiles ----------
-    if (lane == 0) {
+  constexpr int NPROD = STAGES < 4 ? STAGES : 4;
+  if (warp < 4) {
+    // ---------------- producers: warp w streams the stages i = w, w + NPROD, ... ---------------------
+    if (lane == 0 && warp < NPROD) {
       const uint8_t* wsrc = reinterpret_cast<const uint8_t*>(g.W) + ((size_t)nt_idx * KC + kc_begin) * A_BYTES;
       const uint8_t* wsrc2 =
           DUAL ? reinterpret_cast<const uint8_t*>(g.W2) + ((size_t)nt_idx * KC + kc_begin) * A_BYTES : nullptr;
       const uint8_t* xsrc =
           reinterpret_cast<const uint8_t*>(g.X) + ((size_t)kc_begin * g.rows_pad + (size_t)tt * NT) * 128;
-      for (int i = 0; i < nk; ++i) {
+      for (int i = warp; i < nk; i += NPROD) {
         const int s = i % STAGES;
         const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
         if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc)) break;  // stop issuing copies once aborted
@@ -145,7 +148,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tc(int* status, const TcGemm g)
         bulk_g2s(dst + A_BYTES * (DUAL ? 2 : 1), xsrc + (size_t)i * g.rows_pad * 128, B_BYTES, full);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 4) {
     // ---------------- MMA issuer ---------------------------------------------------------------
     if (lane == 0) {
       for (int i = 0; i < nk; ++i) {
@@ -226,7 +229,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tc(int* status, const TcGemm g)
     // give any bulk copy still in flight time to land before shared memory is released
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
   }
-  if (warp == 1) {
+  if (warp == 4) {
     tc_fence_after();
     tmem_dealloc(tmem_base, COLS);
   }
@@ -240,7 +243,7 @@ constexpr size_t smem_bytes() {
 template <int NT, bool DUAL, int STAGES>
 cudaError_t launch_one(int* status, const TcGemm& g, cudaStream_t st) {
   dim3 grid(g.N / 128, (g.M + NT - 1) / NT, g.splits > 0 ? g.splits : 1);
-  k_gemm_tc<NT, DUAL, STAGES><<<grid, 192, smem_bytes<NT, DUAL, STAGES>(), st>>>(status, g);
+  k_gemm_tc<NT, DUAL, STAGES><<<grid, 288, smem_bytes<NT, DUAL, STAGES>(), st>>>(status, g);
   return cudaGetLastError();
 }
 
