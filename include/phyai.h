@@ -192,9 +192,22 @@ phyai_status_t phyai_denoise_batched_host(phyai_expert_t *h, uint32_t batch, con
 phyai_status_t phyai_poll_status(phyai_expert_t *h);
 
 /* Options. key "use_graph": 0 launches the kernels directly, 1 (default) replays a captured CUDA
- * graph per (batch, n_steps).  key "wait_limit": iteration bound of device-side waits (testing).
- * Unknown key -> INVALID_ARG. */
+ * graph per (batch, n_steps).  key "use_persistent": 1 (default) runs calls with batch * suffix_len
+ * <= 64 tokens as one persistent cooperative kernel (the whole n-step loop, no kernel boundaries),
+ * 0 uses the per-operator kernels for every batch.  key "wait_limit": iteration bound of
+ * device-side waits (testing).  Unknown key -> INVALID_ARG. */
 phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t value);
+
+/*
+ * Tracing aid (the paper times phases with GPU-side profiler scopes; Sec. "Results", measurement
+ * protocol).  With option "trace" = step * 1000 + layer the persistent kernel records, for that
+ * step and layer, two device-global-timer stamps (ns) per CTA and phase: inputs ready, role done.
+ * After the stream is synchronised phyai_read_trace copies them to `out` (HOST memory,
+ * capacity >= 148 * 11 * 2 entries) as [cta][phase][2]; unused slots are 0.  Phases in order: norm1,
+ * qkv, attention, merge, o-proj, norm2, gate/up, down, embed, embed-gemm, final.  "trace" = -1 turns it off.
+ */
+phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_ctas,
+                                uint32_t *n_phases);
 
 /* Number of kernel launches (graph nodes) one denoise call with this batch / n_steps issues;
  * 0 if unknown.  Reporting aid for benchmarks. */

@@ -28,7 +28,7 @@ EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes
            "phyai_denoise_batched", "phyai_denoise_host", "phyai_denoise_batched_host", "phyai_poll_status",
            "phyai_set_option", "phyai_launches_per_call", "phyai_last_error", "phyai_version",
            "phyai_suffix_attention", "phyai_suffix_attention_scratch_bytes", "phyai_op_last_error",
-           "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity")
+           "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity", "phyai_read_trace")
 
 
 class PhyaiError(RuntimeError):
@@ -92,6 +92,7 @@ def load_library() -> C.CDLL:
     lib.phyai_set_option.argtypes = [_VP, C.c_char_p, C.c_int64]
     lib.phyai_launches_per_call.argtypes = [_VP, C.c_uint32, C.c_uint32]
     lib.phyai_launches_per_call.restype = C.c_uint64
+    lib.phyai_read_trace.argtypes = [_VP, _VP, C.c_size_t, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
     lib.phyai_op_last_error.restype = C.c_char_p
     lib.phyai_suffix_attention_scratch_bytes.restype = C.c_size_t
     lib.phyai_suffix_attention_scratch_bytes.argtypes = [C.POINTER(AttentionDesc), C.c_uint32]
@@ -245,6 +246,14 @@ class Expert:
 
     def set_option(self, key: str, value: int):
         _check(self.lib.phyai_set_option(self._handle, key.encode(), int(value)))
+
+    def read_trace(self) -> np.ndarray:
+        """Per-CTA, per-phase (inputs-ready, done) device timestamps in ns: array [ctas, phases, 2]."""
+        buf = np.zeros(148 * 11 * 2, dtype=np.uint64)
+        n_ctas, n_ph = C.c_uint32(), C.c_uint32()
+        _check(self.lib.phyai_read_trace(self._handle, buf.ctypes.data_as(_VP), buf.size, C.byref(n_ctas),
+                                         C.byref(n_ph)))
+        return buf.reshape(n_ctas.value, n_ph.value, 2)
 
     def launches_per_call(self, batch: int, n_steps: int) -> int:
         return int(self.lib.phyai_launches_per_call(self._handle, batch, n_steps))

@@ -17,308 +17,10 @@
 #include "../../include/phyai.h"
 #include "kernels.h"
 #include "ptx.cuh"
+#include "attention.cuh"
 
 namespace phyai {
 namespace {
-
-constexpr int KT = 64;      // keys per tile
-constexpr int QROWS = 64;   // query rows per head (suffix length <= 64)
-constexpr float LOG2E = 1.4426950408889634f;
-
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// Output element index: tiled bf16 when rows_pad > 0, else row-major with leading dimension ld.
-__device__ __forceinline__ size_t out_index(int row, int col, int rows_pad, int ld) {
-  return rows_pad > 0 ? tiled_index(row, col, rows_pad) : (size_t)row * ld + col;
-}
-
-struct AttnArgs {
-  const Request* rq;
-  int* status;
-  const float* qkv;      // [rows][Nqkv] fp32 (q | k | v), un-rotated
-  const float2* rope;    // [pos][dh/2] (cos, sin) or null
-  int layer;
-  __nv_bfloat16* out;    // tiled bf16 [Nq/64][rows_pad][64], or row-major [rows][Nq] when rows_pad <= 0
-  int rows_pad;
-  int num_splits;
-  float* part_o;         // [b][head][split][64][DH] unnormalised
-  float* part_ml;        // [b][head][split][64][2]  (max in log2 units, sum)
-  Dims d;
-  unsigned wait_limit;
-};
-
-// Shared-memory tiles are rows of DH bf16 with no padding; the 16-byte chunk c of row r sits at
-// chunk position c ^ (r & 7), which makes every ldmatrix (8 rows x 16 bytes) bank-conflict free.
-__device__ __forceinline__ uint32_t swz(int row, int chunk, int rowb) {
-  return (uint32_t)row * rowb + (uint32_t)((chunk ^ (row & 7)) << 4);
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-// DH: head_dim; HPC: query heads per CTA (4 warps each).
-template <int DH, int HPC>
-__global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
-  constexpr int ROWB = DH * 2;                // bytes per row
-  constexpr int CH = DH / 8;                  // 16-byte chunks per row
-  constexpr int NTHREADS = HPC * 128;
-  extern __shared__ __align__(128) uint8_t smem_raw[];
-  const uint32_t Qs = smem_u32(smem_raw);                         // [HPC*64] rows
-  const uint32_t Ks = Qs + (uint32_t)HPC * QROWS * ROWB;          // [2][KT] rows
-  const uint32_t Vs = Ks + 2u * KT * ROWB;                        // [2][KT] rows
-
-  const Dims& d = a.d;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int split = blockIdx.x, hgrp = blockIdx.y, b = blockIdx.z;
-  const int head0 = hgrp * HPC;
-  const int hk = head0 / (d.Hq / d.Hkv);
-  const int S = d.S;
-  if (status_set(a.status)) return;   // no block-wide waits depend on other blocks: a plain early exit is safe
-
-  const Request r = *a.rq;
-  const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
-  const int Tp = (P + KT - 1) / KT;          // prefix tiles; tile index Tp is the suffix tile
-  const int T = Tp + 1;
-  const int t_begin = (int)(((long long)T * split) / a.num_splits);
-  const int t_end = (int)(((long long)T * (split + 1)) / a.num_splits);
-
-  const uint8_t* Kg = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
-                      (((size_t)(a.layer * 2 + 0) * r.kv_tokens + p0) * d.Hkv + hk) * ROWB;
-  const uint8_t* Vg = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
-                      (((size_t)(a.layer * 2 + 1) * r.kv_tokens + p0) * d.Hkv + hk) * ROWB;
-  const size_t kv_stride = (size_t)d.Hkv * ROWB;  // bytes between consecutive tokens
-  constexpr int half = DH / 2;
-
-  // K/V tile t -> buffer buf with 16-byte asynchronous copies; rows past the prefix are zero-filled
-  auto load_tile = [&](int t, int buf) {
-    const int rows = min(KT, P - t * KT);
-    const uint32_t kb = Ks + (uint32_t)buf * KT * ROWB, vb = Vs + (uint32_t)buf * KT * ROWB;
-    for (int idx = tid; idx < KT * CH; idx += NTHREADS) {
-      const int row = idx / CH, c = idx % CH;
-      const bool ok = row < rows;
-      const size_t g = (size_t)(t * KT + (ok ? row : 0)) * kv_stride + (size_t)c * 16;
-      const uint32_t o = swz(row, c, ROWB);
-      cp_async16(kb + o, Kg + g, ok ? 16u : 0u);
-      cp_async16(vb + o, Vg + g, ok ? 16u : 0u);
-    }
-  };
-  if (t_begin < t_end && t_begin < Tp) load_tile(t_begin, 0);
-  cp_async_commit();
-
-  // ---- Q: rotate, scale by dh^-1/2, round to bf16, into shared memory (4 column pairs per thread)
-  const float qscale = rsqrtf((float)DH);
-  for (int idx = tid; idx < HPC * QROWS * (half / 4); idx += NTHREADS) {
-    const int hl = idx / (QROWS * (half / 4)), rem = idx % (QROWS * (half / 4));
-    const int i = rem / (half / 4), j = (rem % (half / 4)) * 4;
-    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-    if (i < S) {
-      const float* q = a.qkv + (size_t)(b * S + i) * d.Nqkv + (size_t)(head0 + hl) * DH;
-      lo = *reinterpret_cast<const float4*>(q + j);
-      hi = *reinterpret_cast<const float4*>(q + j + half);
-      if (a.rope) {
-        const float4 cs0 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j);
-        const float4 cs1 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j + 2);
-        const float4 l2 = make_float4(lo.x * cs0.x - hi.x * cs0.y, lo.y * cs0.z - hi.y * cs0.w,
-                                      lo.z * cs1.x - hi.z * cs1.y, lo.w * cs1.z - hi.w * cs1.w);
-        hi = make_float4(hi.x * cs0.x + lo.x * cs0.y, hi.y * cs0.z + lo.y * cs0.w, hi.z * cs1.x + lo.z * cs1.y,
-                         hi.w * cs1.z + lo.w * cs1.w);
-        lo = l2;
-      }
-    }
-    const int row = hl * QROWS + i;
-    const uint2 plo = make_uint2(pack_bf16(lo.x * qscale, lo.y * qscale), pack_bf16(lo.z * qscale, lo.w * qscale));
-    const uint2 phi = make_uint2(pack_bf16(hi.x * qscale, hi.y * qscale), pack_bf16(hi.z * qscale, hi.w * qscale));
-    asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Qs + swz(row, j >> 3, ROWB) + (j & 7) * 2), "r"(plo.x), "r"(plo.y) : "memory");
-    asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Qs + swz(row, (j + half) >> 3, ROWB) + (j & 7) * 2), "r"(phi.x), "r"(phi.y) : "memory");
-  }
-
-  // ---- per-warp state -----------------------------------------------------------------------------
-  const int hl = warp >> 2, rb = warp & 3;             // local head, 16-row block
-  const int g = lane >> 2, qd = lane & 3;              // row within 8, column pair
-  const int row0 = rb * 16 + g, row1 = row0 + 8;       // this thread's two query rows
-  const int sw = lane & 7;                             // swizzle term of every ldmatrix row this lane addresses
-  float o[DH / 8][4];
-#pragma unroll
-  for (int n = 0; n < DH / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-  const uint32_t q_row = Qs + (uint32_t)(hl * QROWS + rb * 16 + (lane & 15)) * ROWB;
-  const int q_c0 = lane >> 4;
-
-  for (int t = t_begin; t < t_end; ++t) {
-    const int buf = (t - t_begin) & 1;
-    const uint32_t Kb = Ks + (uint32_t)buf * KT * ROWB, Vb = Vs + (uint32_t)buf * KT * ROWB;
-    int valid;  // keys of this tile that exist
-    if (t + 1 < t_end && t + 1 < Tp) load_tile(t + 1, buf ^ 1);   // the other buffer was released by the
-    cp_async_commit();                                            // barrier that ended the previous iteration
-    if (t < Tp) {
-      valid = min(KT, P - t * KT);
-    } else {
-      // -- suffix tile: rotate this request's own keys, round K and V to bf16
-      valid = S;
-      for (int idx = tid; idx < KT * (half / 4); idx += NTHREADS) {
-        const int js = idx / (half / 4), j = (idx % (half / 4)) * 4;
-        float4 klo = make_float4(0.f, 0.f, 0.f, 0.f), khi = klo, vlo = klo, vhi = klo;
-        if (js < S) {
-          const float* kr = a.qkv + (size_t)(b * S + js) * d.Nqkv + d.Nq + (size_t)hk * DH;
-          const float* vr = kr + d.Hkv * DH;
-          klo = *reinterpret_cast<const float4*>(kr + j), khi = *reinterpret_cast<const float4*>(kr + j + half);
-          vlo = *reinterpret_cast<const float4*>(vr + j), vhi = *reinterpret_cast<const float4*>(vr + j + half);
-          if (a.rope) {
-            const float4 cs0 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + js) * half + j);
-            const float4 cs1 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + js) * half + j + 2);
-            const float4 l2 = make_float4(klo.x * cs0.x - khi.x * cs0.y, klo.y * cs0.z - khi.y * cs0.w,
-                                          klo.z * cs1.x - khi.z * cs1.y, klo.w * cs1.z - khi.w * cs1.w);
-            khi = make_float4(khi.x * cs0.x + klo.x * cs0.y, khi.y * cs0.z + klo.y * cs0.w,
-                              khi.z * cs1.x + klo.z * cs1.y, khi.w * cs1.z + klo.w * cs1.w);
-            klo = l2;
-          }
-        }
-        const uint32_t olo = swz(js, j >> 3, ROWB) + (j & 7) * 2, ohi = swz(js, (j + half) >> 3, ROWB) + (j & 7) * 2;
-        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Kb + olo), "r"(pack_bf16(klo.x, klo.y)), "r"(pack_bf16(klo.z, klo.w)) : "memory");
-        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Kb + ohi), "r"(pack_bf16(khi.x, khi.y)), "r"(pack_bf16(khi.z, khi.w)) : "memory");
-        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Vb + olo), "r"(pack_bf16(vlo.x, vlo.y)), "r"(pack_bf16(vlo.z, vlo.w)) : "memory");
-        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Vb + ohi), "r"(pack_bf16(vhi.x, vhi.y)), "r"(pack_bf16(vhi.z, vhi.w)) : "memory");
-      }
-    }
-    cp_async_wait<1>();   // everything but the prefetch just issued has landed
-    __syncthreads();      // tile t (copied or built above) and Q visible to all warps
-    {
-      // ---------------- S = Q K^T (16 rows x 64 keys per warp) ---------------------------------
-      float s[KT / 8][4];
-#pragma unroll
-      for (int n = 0; n < KT / 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
-      const uint32_t k_row = Kb + (uint32_t)((lane & 7) + (lane >> 4) * 8) * ROWB;
-      const int k_c0 = (lane >> 3) & 1;
-#pragma unroll 4
-      for (int kk = 0; kk < DH / 16; ++kk) {
-        uint32_t af[4];
-        ldsm_x4(q_row + (uint32_t)(((kk * 2 + q_c0) ^ sw) << 4), af[0], af[1], af[2], af[3]);
-        const uint32_t kofs = (uint32_t)(((kk * 2 + k_c0) ^ sw) << 4);
-#pragma unroll
-        for (int np = 0; np < KT / 16; ++np) {
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(k_row + (uint32_t)(np * 16 * ROWB) + kofs, b0, b1, b2, b3);
-          mma_bf16(s[2 * np], af, b0, b1);
-          mma_bf16(s[2 * np + 1], af, b2, b3);
-        }
-      }
-      // ---------------- mask + online softmax (log2 domain) ----------------------------------------
-      const bool suffix_tile = t >= Tp;
-      const bool causal = suffix_tile && d.block_causal && d.ns;
-      float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-      for (int n = 0; n < KT / 8; ++n) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int key = n * 8 + qd * 2 + (e & 1);
-          const int row = (e < 2) ? row0 : row1;
-          bool vis = key < valid;
-          if (causal && row == 0 && key != 0) vis = false;  // state token sees only itself
-          s[n][e] = vis ? s[n][e] * LOG2E : -INFINITY;
-        }
-        mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
-        mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
-      }
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-      const float c0 = (mn0 == -INFINITY) ? 1.f : exp2f(m0 - mn0);
-      const float c1 = (mn1 == -INFINITY) ? 1.f : exp2f(m1 - mn1);
-      const float sub0 = (mn0 == -INFINITY) ? 0.f : mn0, sub1 = (mn1 == -INFINITY) ? 0.f : mn1;
-      m0 = mn0, m1 = mn1;
-      float rs0 = 0.f, rs1 = 0.f;
-      uint32_t pf[KT / 16][4];
-#pragma unroll
-      for (int n = 0; n < KT / 8; ++n) {
-        const float p0 = exp2f(s[n][0] - sub0), p1 = exp2f(s[n][1] - sub0);
-        const float p2 = exp2f(s[n][2] - sub1), p3 = exp2f(s[n][3] - sub1);
-        rs0 += p0 + p1, rs1 += p2 + p3;
-        pf[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
-        pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
-      }
-      l0 = l0 * c0 + rs0, l1 = l1 * c1 + rs1;
-#pragma unroll
-      for (int n = 0; n < DH / 8; ++n) {
-        o[n][0] *= c0, o[n][1] *= c0, o[n][2] *= c1, o[n][3] *= c1;
-      }
-      // ---------------- O += P V ----------------------------------------------------------------------
-      const uint32_t v_row = Vb + (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB;
-      const int v_c0 = lane >> 4;
-#pragma unroll
-      for (int kj = 0; kj < KT / 16; ++kj) {
-#pragma unroll
-        for (int np = 0; np < DH / 16; ++np) {
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4_t(v_row + (uint32_t)(kj * 16 * ROWB) + (uint32_t)(((np * 2 + v_c0) ^ sw) << 4), b0, b1, b2, b3);
-          mma_bf16(o[2 * np], pf[kj], b0, b1);
-          mma_bf16(o[2 * np + 1], pf[kj], b2, b3);
-        }
-      }
-    }
-    __syncthreads();  // everyone is done with `buf` before it is refilled
-  }
-  cp_async_wait<0>();
-
-  // ---- finish: quad-reduce the row sums, write output or partial ----------------------------------------
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-  const int head = head0 + hl;
-  if (a.num_splits == 1) {
-    const float i0 = 1.0f / l0, i1 = 1.0f / l1;
-#pragma unroll
-    for (int n = 0; n < DH / 8; ++n) {
-      const int col = head * DH + n * 8 + qd * 2;
-      if (row0 < S)
-        *reinterpret_cast<uint32_t*>(a.out + out_index(b * S + row0, col, a.rows_pad, d.Nq)) =
-            pack_bf16(o[n][0] * i0, o[n][1] * i0);
-      if (row1 < S)
-        *reinterpret_cast<uint32_t*>(a.out + out_index(b * S + row1, col, a.rows_pad, d.Nq)) =
-            pack_bf16(o[n][2] * i1, o[n][3] * i1);
-    }
-  } else {
-    const size_t slab = ((size_t)(b * d.Hq + head) * a.num_splits + split) * QROWS;
-    float* po = a.part_o + slab * DH;
-    float* pm = a.part_ml + slab * 2;
-#pragma unroll
-    for (int n = 0; n < DH / 8; ++n) {
-      const int col = n * 8 + qd * 2;
-      if (row0 < S) *reinterpret_cast<float2*>(po + (size_t)row0 * DH + col) = make_float2(o[n][0], o[n][1]);
-      if (row1 < S) *reinterpret_cast<float2*>(po + (size_t)row1 * DH + col) = make_float2(o[n][2], o[n][3]);
-    }
-    if (qd == 0) {
-      if (row0 < S) pm[row0 * 2] = m0, pm[row0 * 2 + 1] = l0;
-      if (row1 < S) pm[row1 * 2] = m1, pm[row1 * 2 + 1] = l1;
-    }
-  }
-}
 
 // Combine the per-split partials: out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s.
 template <int DH>

@@ -10,6 +10,7 @@
 
 #include "../../include/phyai.h"
 #include "kernels.h"
+#include "mega.h"
 
 using namespace phyai;
 
@@ -80,6 +81,21 @@ struct phyai_expert {
 
   float* attn_scratch = nullptr;  // split-KV partials of the tensor-core attention
   bool attn_mma = false;
+
+  // persistent loop kernel (batch * suffix_len <= 64)
+  bool mega_ok = false;
+  int use_mega = 1;
+  int n_sm = 0;
+  __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
+  float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
+  __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
+  float* mega_scratch = nullptr;
+  float* mega_slab = nullptr;
+  unsigned* mega_counters = nullptr;
+  unsigned long long* mega_trace = nullptr;   // [148][MP_COUNT][2] when tracing is on
+  int trace_step = 0, trace_layer = 0;
+  struct MegaBatch { MegaCtaPlan* plans = nullptr; int n_cta[MP_COUNT]; int splits = 1; };
+  std::map<int, MegaBatch> mega_batches;
 
   Request* rq = nullptr;
   int* cu_internal = nullptr;
@@ -200,8 +216,55 @@ int pick_splits(int n_tiles, int tok_tiles, int KC) {
   return s;
 }
 
+// Per-batch role plan of the persistent kernel (built outside any stream capture: it allocates).
+phyai_status_t mega_prepare(phyai_expert* h, int batch) {
+  const Dims& d = h->d;
+  const int ncta = h->n_sm < 148 ? h->n_sm : 148;
+  if (h->mega_batches.find(batch) == h->mega_batches.end()) {
+    phyai_expert::MegaBatch mb;
+    mb.splits = mega_attention_splits(d, batch, (int)h->cfg.max_prefix_len, ncta);
+    std::vector<MegaCtaPlan> plans(ncta);
+    if (!mega_plan(d, batch, h->ada ? 1 : 0, mb.splits, ncta, plans.data(), mb.n_cta))
+      return fail(PHYAI_ERR_UNSUPPORTED, "persistent kernel cannot plan this shape");
+    ST(h->alloc(&mb.plans, (size_t)ncta));
+    CU(cudaMemcpy(mb.plans, plans.data(), sizeof(MegaCtaPlan) * ncta, cudaMemcpyHostToDevice));
+    h->mega_batches.emplace(batch, mb);
+  }
+  return PHYAI_OK;
+}
+
+// Small batches: the whole loop as one persistent cooperative kernel.
+phyai_status_t enqueue_mega(phyai_expert* h, int batch, int n, const Tables& t, cudaStream_t st) {
+  const Dims& d = h->d;
+  const int ncta = h->n_sm < 148 ? h->n_sm : 148;
+  const phyai_expert::MegaBatch& mb = h->mega_batches.at(batch);
+  MegaParams p{};
+  p.d = d, p.batch = batch, p.M = batch * d.S, p.n_steps = n, p.ada = h->ada ? 1 : 0, p.sites = h->sites;
+  p.attn_splits = mb.splits, p.hpc = 2, p.dt = -1.0f / (float)n, p.wait_limit = h->wait_limit;
+  p.rq = h->rq, p.status = h->status, p.counters = h->mega_counters, p.plans = mb.plans;
+  for (int i = 0; i < MP_COUNT; ++i) p.n_cta[i] = mb.n_cta[i];
+  p.w_qkv = h->p_qkv[0], p.w_o = h->p_o[0], p.w_gu = h->p_gu_all, p.w_d = h->p_d[0], p.w_embed = h->W2p;
+  p.stride_qkv = (size_t)d.D * d.Nqkv * 2, p.stride_o = (size_t)d.Nq * d.D * 2;
+  p.stride_gu = (size_t)d.D * 2 * d.F * 2, p.stride_d = (size_t)d.F * d.D * 2;
+  p.s_qkv = h->s_qkv_all, p.s_o = h->s_o_all, p.s_g = h->s_g_all, p.s_u = h->s_u_all, p.s_d = h->s_d_all;
+  p.Wc = h->Wc, p.bcfold = h->bcfold, p.b2 = h->b2, p.state_tok = h->state_tok, p.Wout = h->Wout, p.bout = h->bout;
+  p.gains = h->gains, p.mod = t.mod, p.tb = t.tb, p.rope = h->rope;
+  p.h = h->h, p.qkv = h->qkv, p.xn64 = h->xn64, p.attn64 = h->attn64, p.m64 = h->m64, p.u64 = h->u64;
+  p.attn_scratch = h->mega_scratch;
+  p.slab = h->mega_slab, p.o_splits = (d.Nq / 64 + 7) / 8, p.d_splits = (d.F / 64 + 7) / 8;
+  p.trace = h->mega_trace, p.trace_step = h->trace_step < n ? h->trace_step : n - 1;
+  p.trace_layer = h->trace_layer < d.L ? h->trace_layer : d.L - 1;
+  launch_begin(h->rq, h->status, h->state_w, h->state_b, h->state_tok, d, batch, st);
+  CU(cudaMemsetAsync(h->mega_counters, 0, sizeof(unsigned) * MP_COUNT, st));
+  cudaError_t e = launch_mega(p, ncta, st);
+  if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "persistent kernel launch failed: %s", cudaGetErrorString(e));
+  h->counting = 2;
+  return PHYAI_OK;
+}
+
 phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, cudaStream_t st) {
   const Dims& d = h->d;
+  if (h->mega_ok && h->use_mega && mega_supported(d, batch)) return enqueue_mega(h, batch, n, t, st);
   const int M = batch * d.S, D = d.D;
   const int nt = pick_nt(M);
   const int tok_tiles = (M + nt - 1) / nt;
@@ -334,6 +397,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
 phyai_status_t run(phyai_expert* h, const Request& r, int n, cudaStream_t st) {
   Tables* t = nullptr;
   ST(build_tables(h, n, st, &t));
+  if (h->mega_ok && h->use_mega && mega_supported(h->d, r.batch)) ST(mega_prepare(h, r.batch));
   launch_set_request(h->rq, r, h->cu_internal, st);
   if (r.cu_lens != nullptr) launch_validate(h->rq, h->status, (int)h->cfg.max_prefix_len, st);
   const auto key = std::make_pair(r.batch, n);
@@ -522,15 +586,32 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
     }
     // ---- the seven big matrices per layer ----
     const int Nq = d.Nq, Nkv = d.Hkv * d.dh, Nqkv = d.Nqkv, F = d.F;
+    __nv_bfloat16 *pq_all = nullptr, *po_all = nullptr, *pg_all = nullptr, *pu_all = nullptr, *pd_all = nullptr;
+    if (tc) {   // one allocation per matrix kind, layers at a fixed stride (the persistent kernel indexes by layer)
+      ST(h->alloc(&pq_all, (size_t)L * D * Nqkv)); ST(h->alloc(&po_all, (size_t)L * Nq * D));
+      ST(h->alloc(&pg_all, (size_t)L * D * F)); ST(h->alloc(&pu_all, (size_t)L * D * F));
+      ST(h->alloc(&pd_all, (size_t)L * F * D));
+      h->mega_ok = mega_supported(d, 1);
+      if (h->mega_ok) ST(h->alloc(&h->p_gu_all, (size_t)L * D * 2 * F));
+      if (w8) {
+        ST(h->alloc(&h->s_qkv_all, (size_t)L * Nqkv)); ST(h->alloc(&h->s_o_all, (size_t)L * D));
+        ST(h->alloc(&h->s_g_all, (size_t)L * F)); ST(h->alloc(&h->s_u_all, (size_t)L * F));
+        ST(h->alloc(&h->s_d_all, (size_t)L * D));
+      }
+    }
     for (int l = 0; l < L; ++l) {
       const float* sq = w8 ? w->scales[0][l] : nullptr; const float* sk = w8 ? w->scales[1][l] : nullptr;
       const float* sv = w8 ? w->scales[2][l] : nullptr; const float* so = w8 ? w->scales[3][l] : nullptr;
       const float* sg = w8 ? w->scales[4][l] : nullptr; const float* su = w8 ? w->scales[5][l] : nullptr;
       const float* sd = w8 ? w->scales[6][l] : nullptr;
       if (tc) {
-        __nv_bfloat16 *pq, *po, *pg, *pu, *pd;
-        ST(h->alloc(&pq, (size_t)D * Nqkv)); ST(h->alloc(&po, (size_t)Nq * D));
-        ST(h->alloc(&pg, (size_t)D * F)); ST(h->alloc(&pu, (size_t)D * F)); ST(h->alloc(&pd, (size_t)F * D));
+        __nv_bfloat16 *pq = pq_all + (size_t)l * D * Nqkv, *po = po_all + (size_t)l * Nq * D;
+        __nv_bfloat16 *pg = pg_all + (size_t)l * D * F, *pu = pu_all + (size_t)l * D * F, *pd = pd_all + (size_t)l * F * D;
+        if (h->mega_ok) {
+          __nv_bfloat16* pgu = h->p_gu_all + (size_t)l * D * 2 * F;
+          launch_pack_tiled(w->wgate[l], big_kind, pgu, D, F, 0, st, 64, 0);
+          launch_pack_tiled(w->wup[l], big_kind, pgu, D, F, 0, st, 64, 1);
+        }
         launch_pack_tiled(w->wq[l], big_kind, pq, D, Nq, 0, st);
         launch_pack_tiled(w->wk[l], big_kind, pq, D, Nkv, Nq, st);
         launch_pack_tiled(w->wv[l], big_kind, pq, D, Nkv, Nq + Nkv, st);
@@ -541,7 +622,8 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         h->p_qkv.push_back(pq), h->p_o.push_back(po), h->p_g.push_back(pg), h->p_u.push_back(pu), h->p_d.push_back(pd);
         float *cq = nullptr, *co = nullptr, *cg = nullptr, *cu = nullptr, *cd = nullptr;
         if (w8) {
-          ST(h->alloc(&cq, Nqkv)); ST(h->alloc(&co, D)); ST(h->alloc(&cg, F)); ST(h->alloc(&cu, F)); ST(h->alloc(&cd, D));
+          cq = h->s_qkv_all + (size_t)l * Nqkv, co = h->s_o_all + (size_t)l * D, cg = h->s_g_all + (size_t)l * F;
+          cu = h->s_u_all + (size_t)l * F, cd = h->s_d_all + (size_t)l * D;
           CU(cudaMemcpyAsync(cq, sq, (size_t)Nq * 4, cudaMemcpyDeviceToDevice, st));
           CU(cudaMemcpyAsync(cq + Nq, sk, (size_t)Nkv * 4, cudaMemcpyDeviceToDevice, st));
           CU(cudaMemcpyAsync(cq + Nq + Nkv, sv, (size_t)Nkv * 4, cudaMemcpyDeviceToDevice, st));
@@ -584,6 +666,26 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
           need = n > need ? n : need;
         }
         if (need) ST(h->alloc(&h->attn_scratch, need, true));
+      }
+      if (h->mega_ok) {
+        CU(cudaDeviceGetAttribute(&h->n_sm, cudaDevAttrMultiProcessorCount, 0));
+        int dev = 0;
+        CU(cudaGetDevice(&dev));
+        CU(cudaDeviceGetAttribute(&h->n_sm, cudaDevAttrMultiProcessorCount, dev));
+        int coop = 0;
+        CU(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+        if (!coop || h->n_sm < 8) h->mega_ok = false;
+      }
+      if (h->mega_ok) {
+        CU(mega_setup(d.dh));
+        ST(h->alloc(&h->xn64, (size_t)64 * D, true));
+        ST(h->alloc(&h->attn64, (size_t)64 * Nq, true));
+        ST(h->alloc(&h->m64, (size_t)64 * F, true));
+        ST(h->alloc(&h->u64, (size_t)64 * D, true));
+        ST(h->alloc(&h->mega_scratch, mega_scratch_floats(d, 64 / d.S > 0 ? 64 / d.S : 1, 16), true));
+        ST(h->alloc(&h->mega_counters, (size_t)MP_COUNT, true));
+        const int so = (d.Nq / 64 + 7) / 8, sd = (d.F / 64 + 7) / 8;
+        ST(h->alloc(&h->mega_slab, (size_t)(so > sd ? so : sd) * 64 * D, true));
       }
       ST(h->alloc(&h->xn_t, Mp * D, true));
       ST(h->alloc(&h->attn_t, Mp * Nq, true));
@@ -726,6 +828,25 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     h->use_graph = value != 0;
     return PHYAI_OK;
   }
+  if (!strcmp(key, "trace")) {   // value = step * 1000 + layer to trace; negative = off
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    if (value < 0) {
+      h->mega_trace = nullptr;
+      return PHYAI_OK;
+    }
+    if (!h->mega_ok) return fail(PHYAI_ERR_UNSUPPORTED, "tracing needs the persistent kernel");
+    unsigned long long* buf = nullptr;
+    ST(h->alloc(&buf, (size_t)148 * MP_COUNT * 2, true));
+    h->mega_trace = buf, h->trace_step = (int)(value / 1000), h->trace_layer = (int)(value % 1000);
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_persistent")) {
+    h->use_mega = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
   if (!strcmp(key, "wait_limit")) {
     if (value < 1 || value > (int64_t)0x7fffffff) return fail(PHYAI_ERR_INVALID_ARG, "wait_limit out of range");
     h->wait_limit = (unsigned)value;
@@ -734,6 +855,17 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     return PHYAI_OK;
   }
   return fail(PHYAI_ERR_INVALID_ARG, "unknown option '%s'", key);
+}
+
+phyai_status_t phyai_read_trace(phyai_expert_t* h, uint64_t* out, size_t capacity, uint32_t* n_ctas,
+                                uint32_t* n_phases) {
+  if (!h || !out || !n_ctas || !n_phases) return fail(PHYAI_ERR_INVALID_ARG, "NULL argument");
+  if (!h->mega_trace) return fail(PHYAI_ERR_INVALID_ARG, "tracing is off (phyai_set_option(h, \"trace\", ...))");
+  const size_t n = (size_t)148 * MP_COUNT * 2;
+  if (capacity < n) return fail(PHYAI_ERR_INVALID_ARG, "capacity %zu < %zu entries", capacity, n);
+  CU(cudaMemcpy(out, h->mega_trace, n * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+  *n_ctas = 148, *n_phases = MP_COUNT;
+  return PHYAI_OK;
 }
 
 uint64_t phyai_launches_per_call(phyai_expert_t* h, uint32_t batch, uint32_t n_steps) {

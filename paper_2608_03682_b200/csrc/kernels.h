@@ -23,7 +23,10 @@ void launch_copy_cols(const void* src, int src_kind, const float* scale, float* 
                       int col_off, cudaStream_t st);
 // [in=K][out=N] source -> 128x64 blocks of the 128-byte-swizzled K-major bf16 image, out channel
 // n stored at packed row n_off + n of a matrix with KC = K/64 column chunks.
-void launch_pack_tiled(const void* src, int src_kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st);
+// With il_group > 0 the channels of two matrices are interleaved in groups of il_group rows
+// (il_second selects the second matrix): packed row = (n / g) * 2g + n % g + (second ? g : 0).
+void launch_pack_tiled(const void* src, int src_kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st,
+                       int il_group = 0, int il_second = 0);
 // Y[r][n] = act( sum_d X[r][d] * W[(w_row_off + d)][n] + bias[n] + add[n] ), r < R
 void launch_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K, const float* bias,
                       const float* add, int act_swish, float* Y, int ldy, int R, cudaStream_t st);

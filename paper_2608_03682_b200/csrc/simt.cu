@@ -78,14 +78,16 @@ void launch_copy_cols(const void* src, int kind, const float* scale, float* dst,
 
 // Weight [K][N] -> packed out-channel-major swizzled blocks.  One thread per 16-byte chunk
 // (8 consecutive k of one out channel): reads are strided by N (one-off cost at create).
-__global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off) {
+__global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, int il_group,
+                             int il_second) {
   const int KC = K >> 6;
   const size_t chunks = (size_t)N * (K >> 3);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
     const int n = (int)(i % N);         // consecutive threads -> consecutive n: coalesced source reads
     const int k8 = (int)(i / N);        // chunk index along K
     const int k0 = k8 << 3;
-    const int np = n_off + n;
+    // optional interleave: groups of il_group channels of two matrices alternate in the packed rows
+    const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0) : n_off + n;
     const int kc = k0 >> 6, c = (k0 & 63) >> 3;
     const size_t base = (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 64 + (size_t)((c ^ (np & 7)) << 3);
     __align__(16) __nv_bfloat16 v[8];
@@ -94,10 +96,11 @@ __global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int 
     *reinterpret_cast<uint4*>(dst + base) = *reinterpret_cast<const uint4*>(v);
   }
 }
-void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st) {
+void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st,
+                       int il_group, int il_second) {
   const size_t chunks = (size_t)N * (K >> 3);
   const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
-  k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off);
+  k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off, il_group, il_second);
 }
 
 // =============================================================================================
