@@ -201,9 +201,10 @@ phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t valu
 /*
  * Tracing aid (the paper times phases with GPU-side profiler scopes; Sec. "Results", measurement
  * protocol).  With option "trace" = step * 1000 + layer the persistent kernel records, for that
- * step and layer, two device-global-timer stamps (ns) per CTA and phase: inputs ready, role done.
- * After the stream is synchronised phyai_read_trace copies them to `out` (HOST memory,
- * capacity >= 148 * 11 * 2 entries) as [cta][phase][2]; unused slots are 0.  Phases in order: norm1,
+ * step and layer, four device-global-timer stamps (ns) per CTA and phase: inputs ready (for a
+ * GEMM role: accumulator complete), role done, and for GEMM roles first activations in shared memory and
+ * last MMA issued.  After the stream is synchronised phyai_read_trace copies them to `out` (HOST
+ * memory, capacity >= 148 * 11 * 4 entries) as [cta][phase][4]; unused slots are 0.  Phases in order: norm1,
  * qkv, attention, merge, o-proj, norm2, gate/up, down, embed, embed-gemm, final.  "trace" = -1 turns it off.
  */
 phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_ctas,

@@ -248,12 +248,12 @@ class Expert:
         _check(self.lib.phyai_set_option(self._handle, key.encode(), int(value)))
 
     def read_trace(self) -> np.ndarray:
-        """Per-CTA, per-phase (inputs-ready, done) device timestamps in ns: array [ctas, phases, 2]."""
-        buf = np.zeros(148 * 11 * 2, dtype=np.uint64)
+        """Per-CTA, per-phase device timestamps in ns: array [ctas, phases, 4]."""
+        buf = np.zeros(148 * 11 * 4, dtype=np.uint64)
         n_ctas, n_ph = C.c_uint32(), C.c_uint32()
         _check(self.lib.phyai_read_trace(self._handle, buf.ctypes.data_as(_VP), buf.size, C.byref(n_ctas),
                                          C.byref(n_ph)))
-        return buf.reshape(n_ctas.value, n_ph.value, 2)
+        return buf.reshape(n_ctas.value, n_ph.value, 4)
 
     def launches_per_call(self, batch: int, n_steps: int) -> int:
         return int(self.lib.phyai_launches_per_call(self._handle, batch, n_steps))

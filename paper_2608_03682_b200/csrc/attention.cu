@@ -96,7 +96,7 @@ size_t attention_scratch_floats(const Dims& d, int batch, int splits) {
 cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qkv, const float2* rope, int layer,
                                  __nv_bfloat16* out_tiled, int rows_pad, int num_splits, float* scratch, const Dims& d,
                                  int batch, unsigned wait_limit, cudaStream_t st) {
-  AttnArgs a;
+  AttnArgs a{};
   a.rq = rq, a.status = status, a.qkv = qkv, a.rope = rope, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
   a.num_splits = num_splits, a.d = d, a.wait_limit = wait_limit;
   a.part_o = scratch;

@@ -42,6 +42,7 @@ struct AttnArgs {
   const Request* rq;
   int* status;
   const float* qkv;      // [rows][Nqkv] fp32 (q | k | v), un-rotated
+  const __nv_bfloat16 *qr, *kr, *vr;  // or: rotated, scaled bf16 q [b][Hq][S][dh], k / v [b][Hkv][S][dh] (null = use qkv)
   const float2* rope;    // [pos][dh/2] (cos, sin) or null
   int layer;
   __nv_bfloat16* out;    // tiled bf16 [Nq/64][rows_pad][64], or row-major [rows][Nq] when rows_pad <= 0
@@ -75,16 +76,18 @@ __device__ __forceinline__ void group_sync() {
 // One attention role: the suffix rows of HPC query heads (head group `hgrp`) of request `b` against
 // key tiles [T*split/num_splits, T*(split+1)/num_splits).  Executed by HPC*128 threads (`tid` is the
 // thread's index within that group) that synchronise on named barrier BAR.  DH: head_dim; NBUF: K/V
-// buffers (2 = prefetch the next tile during compute).  Shared memory at `smem_base` (128-byte
-// aligned): (HPC*64 + 2*NBUF*64) rows of DH bf16.
-template <int DH, int HPC, int NBUF, int BAR>
+// buffers (2 = prefetch the next tile during compute); KTT: keys per tile.  Shared memory at
+// `smem_base` (128-byte aligned): (HPC*64 + 2*NBUF*KTT) rows of DH bf16.  When a.qr is set, q / k / v of
+// the suffix are read as bf16, already rotated and scaled (written by the QKV epilogue of the
+// persistent kernel); otherwise they are taken from the fp32 QKV output and rotated here.
+template <int DH, int HPC, int NBUF, int BAR, int KTT>
 __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp, int b, uint32_t smem_base, int tid) {
   constexpr int ROWB = DH * 2;                // bytes per row
   constexpr int CH = DH / 8;                  // 16-byte chunks per row
   constexpr int NTHREADS = HPC * 128;
   const uint32_t Qs = smem_base;                                  // [HPC*64] rows
-  const uint32_t Ks = Qs + (uint32_t)HPC * QROWS * ROWB;          // [NBUF][KT] rows
-  const uint32_t Vs = Ks + (uint32_t)NBUF * KT * ROWB;            // [NBUF][KT] rows
+  const uint32_t Ks = Qs + (uint32_t)HPC * QROWS * ROWB;          // [NBUF][KTT] rows
+  const uint32_t Vs = Ks + (uint32_t)NBUF * KTT * ROWB;            // [NBUF][KTT] rows
 
   const Dims& d = a.d;
   const int warp = tid >> 5, lane = tid & 31;
@@ -94,8 +97,8 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
 
   const Request r = *a.rq;
   const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
-  const int Tp = (P + KT - 1) / KT;          // prefix tiles; tile index Tp is the suffix tile
-  const int T = Tp + 1;
+  const int Tp = (P + KTT - 1) / KTT;          // prefix tiles, followed by the suffix tiles
+  const int T = Tp + (S + KTT - 1) / KTT;
   const int t_begin = (int)(((long long)T * split) / a.num_splits);
   const int t_end = (int)(((long long)T * (split + 1)) / a.num_splits);
 
@@ -108,12 +111,12 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
 
   // K/V tile t -> buffer buf with 16-byte asynchronous copies; rows past the prefix are zero-filled
   auto load_tile = [&](int t, int buf) {
-    const int rows = min(KT, P - t * KT);
-    const uint32_t kb = Ks + (uint32_t)buf * KT * ROWB, vb = Vs + (uint32_t)buf * KT * ROWB;
-    for (int idx = tid; idx < KT * CH; idx += NTHREADS) {
+    const int rows = min(KTT, P - t * KTT);
+    const uint32_t kb = Ks + (uint32_t)buf * KTT * ROWB, vb = Vs + (uint32_t)buf * KTT * ROWB;
+    for (int idx = tid; idx < KTT * CH; idx += NTHREADS) {
       const int row = idx / CH, c = idx % CH;
       const bool ok = row < rows;
-      const size_t g = (size_t)(t * KT + (ok ? row : 0)) * kv_stride + (size_t)c * 16;
+      const size_t g = (size_t)(t * KTT + (ok ? row : 0)) * kv_stride + (size_t)c * 16;
       const uint32_t o = swz(row, c, ROWB);
       cp_async16(kb + o, Kg + g, ok ? 16u : 0u);
       cp_async16(vb + o, Vg + g, ok ? 16u : 0u);
@@ -122,8 +125,21 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
   if (t_begin < t_end && t_begin < Tp) load_tile(t_begin, 0);
   cp_async_commit();
 
+  if (a.qr) {
+    // ---- Q rows are ready-made bf16: straight asynchronous copies (rows past the suffix are zero-filled)
+    for (int idx = tid; idx < HPC * QROWS * CH; idx += NTHREADS) {
+      const int hl = idx / (QROWS * CH), rem = idx % (QROWS * CH);
+      const int i = rem / CH, c = rem % CH;
+      const bool ok = i < S;
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(a.qr) +
+                           ((size_t)((b * d.Hq + head0 + hl) * S + (ok ? i : 0)) * CH + c) * 16;
+      cp_async16(Qs + swz(hl * QROWS + i, c, ROWB), src, ok ? 16u : 0u);
+    }
+    cp_async_commit();
+  }
   // ---- Q: rotate, scale by dh^-1/2, round to bf16, into shared memory (4 column pairs per thread)
   const float qscale = rsqrtf((float)DH);
+  if (!a.qr)
 #pragma unroll 4
   for (int idx = tid; idx < HPC * QROWS * (half / 4); idx += NTHREADS) {
     const int hl = idx / (QROWS * (half / 4)), rem = idx % (QROWS * (half / 4));
@@ -164,20 +180,35 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
 
   for (int t = t_begin; t < t_end; ++t) {
     const int buf = NBUF == 2 ? ((t - t_begin) & 1) : 0;
-    const uint32_t Kb = Ks + (uint32_t)buf * KT * ROWB, Vb = Vs + (uint32_t)buf * KT * ROWB;
+    const uint32_t Kb = Ks + (uint32_t)buf * KTT * ROWB, Vb = Vs + (uint32_t)buf * KTT * ROWB;
     int valid;  // keys of this tile that exist
     if (NBUF == 2) {
       if (t + 1 < t_end && t + 1 < Tp) load_tile(t + 1, buf ^ 1);   // the other buffer was released by the
       cp_async_commit();                                            // barrier that ended the previous iteration
     }
     if (t < Tp) {
-      valid = min(KT, P - t * KT);
+      valid = min(KTT, P - t * KTT);
+    } else if (a.qr) {
+      // -- suffix tile from the ready-made bf16 keys / values
+      const int j0 = (t - Tp) * KTT;
+      valid = min(KTT, S - j0);
+      const uint8_t* ksrc = reinterpret_cast<const uint8_t*>(a.kr) + (size_t)((b * d.Hkv + hk) * S + j0) * ROWB;
+      const uint8_t* vsrc = reinterpret_cast<const uint8_t*>(a.vr) + (size_t)((b * d.Hkv + hk) * S + j0) * ROWB;
+      for (int idx = tid; idx < KTT * CH; idx += NTHREADS) {
+        const int row = idx / CH, c = idx % CH;
+        const bool ok = row < valid;
+        const size_t g = (size_t)(ok ? row : 0) * ROWB + (size_t)c * 16;
+        cp_async16(Kb + swz(row, c, ROWB), ksrc + g, ok ? 16u : 0u);
+        cp_async16(Vb + swz(row, c, ROWB), vsrc + g, ok ? 16u : 0u);
+      }
+      cp_async_commit();
     } else {
       // -- suffix tile: rotate this request's own keys, round K and V to bf16
-      valid = S;
+      const int j0 = (t - Tp) * KTT;
+      valid = min(KTT, S - j0);
 #pragma unroll 2
-      for (int idx = tid; idx < KT * (half / 4); idx += NTHREADS) {
-        const int js = idx / (half / 4), j = (idx % (half / 4)) * 4;
+      for (int idx = tid; idx < KTT * (half / 4); idx += NTHREADS) {
+        const int lr = idx / (half / 4), js = j0 + lr, j = (idx % (half / 4)) * 4;
         float4 klo = make_float4(0.f, 0.f, 0.f, 0.f), khi = klo, vlo = klo, vhi = klo;
         if (js < S) {
           const float* kr = a.qkv + (size_t)(b * S + js) * d.Nqkv + d.Nq + (size_t)hk * DH;
@@ -194,21 +225,21 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
             klo = l2;
           }
         }
-        const uint32_t olo = swz(js, j >> 3, ROWB) + (j & 7) * 2, ohi = swz(js, (j + half) >> 3, ROWB) + (j & 7) * 2;
+        const uint32_t olo = swz(lr, j >> 3, ROWB) + (j & 7) * 2, ohi = swz(lr, (j + half) >> 3, ROWB) + (j & 7) * 2;
         asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Kb + olo), "r"(pack_bf16(klo.x, klo.y)), "r"(pack_bf16(klo.z, klo.w)) : "memory");
         asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Kb + ohi), "r"(pack_bf16(khi.x, khi.y)), "r"(pack_bf16(khi.z, khi.w)) : "memory");
         asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Vb + olo), "r"(pack_bf16(vlo.x, vlo.y)), "r"(pack_bf16(vlo.z, vlo.w)) : "memory");
         asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(Vb + ohi), "r"(pack_bf16(vhi.x, vhi.y)), "r"(pack_bf16(vhi.z, vhi.w)) : "memory");
       }
     }
-    if (NBUF == 2) cp_async_wait<1>();   // everything but the prefetch just issued has landed
+    if (NBUF == 2 && !(a.qr && t >= Tp)) cp_async_wait<1>();   // everything but the prefetch just issued has landed
     else cp_async_wait<0>();
     group_sync<BAR, NTHREADS>();         // tile t (copied or built above) and Q visible to all warps
     {
-      // ---------------- S = Q K^T (16 rows x 64 keys per warp) ---------------------------------
-      float s[KT / 8][4];
+      // ---------------- S = Q K^T (16 rows x KTT keys per warp) ---------------------------------
+      float s[KTT / 8][4];
 #pragma unroll
-      for (int n = 0; n < KT / 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+      for (int n = 0; n < KTT / 8; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
       const uint32_t k_row = Kb + (uint32_t)((lane & 7) + (lane >> 4) * 8) * ROWB;
       const int k_c0 = (lane >> 3) & 1;
 #pragma unroll 4
@@ -217,7 +248,7 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
         ldsm_x4(q_row + (uint32_t)(((kk * 2 + q_c0) ^ sw) << 4), af[0], af[1], af[2], af[3]);
         const uint32_t kofs = (uint32_t)(((kk * 2 + k_c0) ^ sw) << 4);
 #pragma unroll
-        for (int np = 0; np < KT / 16; ++np) {
+        for (int np = 0; np < KTT / 16; ++np) {
           uint32_t b0, b1, b2, b3;
           ldsm_x4(k_row + (uint32_t)(np * 16 * ROWB) + kofs, b0, b1, b2, b3);
           mma_bf16(s[2 * np], af, b0, b1);
@@ -229,13 +260,13 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       const bool causal = suffix_tile && d.block_causal && d.ns;
       float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-      for (int n = 0; n < KT / 8; ++n) {
+      for (int n = 0; n < KTT / 8; ++n) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int key = n * 8 + qd * 2 + (e & 1);
           const int row = (e < 2) ? row0 : row1;
           bool vis = key < valid;
-          if (causal && row == 0 && key != 0) vis = false;  // state token sees only itself
+          if (causal && row == 0 && (t - Tp) * KTT + key != 0) vis = false;  // state token sees only itself
           s[n][e] = vis ? s[n][e] * LOG2E : -INFINITY;
         }
         mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
@@ -251,9 +282,9 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       const float sub0 = (mn0 == -INFINITY) ? 0.f : mn0, sub1 = (mn1 == -INFINITY) ? 0.f : mn1;
       m0 = mn0, m1 = mn1;
       float rs0 = 0.f, rs1 = 0.f;
-      uint32_t pf[KT / 16][4];
+      uint32_t pf[KTT / 16][4];
 #pragma unroll
-      for (int n = 0; n < KT / 8; ++n) {
+      for (int n = 0; n < KTT / 8; ++n) {
         const float p0 = exp2f(s[n][0] - sub0), p1 = exp2f(s[n][1] - sub0);
         const float p2 = exp2f(s[n][2] - sub1), p3 = exp2f(s[n][3] - sub1);
         rs0 += p0 + p1, rs1 += p2 + p3;
@@ -269,7 +300,7 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       const uint32_t v_row = Vb + (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB;
       const int v_c0 = lane >> 4;
 #pragma unroll
-      for (int kj = 0; kj < KT / 16; ++kj) {
+      for (int kj = 0; kj < KTT / 16; ++kj) {
 #pragma unroll
         for (int np = 0; np < DH / 16; ++np) {
           uint32_t b0, b1, b2, b3;
@@ -327,7 +358,7 @@ template <int DH, int HPC>
 __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   if (status_set(a.status)) return;   // no wait in this kernel depends on another block: a plain exit is safe
-  attn_role<DH, HPC, 2, 0>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
+  attn_role<DH, HPC, 2, 0, KT>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
 }
 
 }  // namespace

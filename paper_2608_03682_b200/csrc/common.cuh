@@ -48,6 +48,23 @@ __host__ __device__ __forceinline__ size_t tiled_index(int row, int col, int row
   return ((size_t)kc * rows_pad + row) * 64 + (size_t)chunk * 8 + (within & 7);
 }
 
+// Row order of the packed fused-QKV weight matrix.  Inside every q / k head the dh channels are
+// arranged so that each 128-row tile holds 64 channels of the first half of the head followed by
+// their 64 rotary partners (channel + dh/2): a GEMM epilogue then finds both members of a rotary pair
+// in one accumulator tile, 64 rows apart.  The v region and heads of <= 128 channels keep their order.
+__host__ __device__ __forceinline__ int qkv_channel_to_packed(int c, int dh) {
+  if (dh <= 128) return c;
+  const int hb = c - c % dh, w = c % dh, half = dh >> 1;
+  const int t = (w % half) >> 6, r = (w & 63) + (w >= half ? 64 : 0);
+  return hb + t * 128 + r;
+}
+__host__ __device__ __forceinline__ int qkv_packed_to_channel(int n, int dh) {
+  if (dh <= 128) return n;
+  const int hb = n - n % dh, w = n % dh, half = dh >> 1;
+  const int t = w >> 7, r = w & 127;
+  return hb + (r < 64 ? t * 64 + r : half + t * 64 + (r - 64));
+}
+
 struct RowMajorF32 {
   float* p;
   int ld;

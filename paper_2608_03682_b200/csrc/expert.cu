@@ -89,6 +89,7 @@ struct phyai_expert {
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
+  __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
   float* mega_scratch = nullptr;
   float* mega_slab = nullptr;
   unsigned* mega_counters = nullptr;
@@ -250,6 +251,7 @@ phyai_status_t enqueue_mega(phyai_expert* h, int batch, int n, const Tables& t, 
   p.Wc = h->Wc, p.bcfold = h->bcfold, p.b2 = h->b2, p.state_tok = h->state_tok, p.Wout = h->Wout, p.bout = h->bout;
   p.gains = h->gains, p.mod = t.mod, p.tb = t.tb, p.rope = h->rope;
   p.h = h->h, p.qkv = h->qkv, p.xn64 = h->xn64, p.attn64 = h->attn64, p.m64 = h->m64, p.u64 = h->u64;
+  p.qr = h->qr64, p.kr = h->kr64, p.vr = h->vr64;
   p.attn_scratch = h->mega_scratch;
   p.slab = h->mega_slab, p.o_splits = (d.Nq / 64 + 7) / 8, p.d_splits = (d.F / 64 + 7) / 8;
   p.trace = h->mega_trace, p.trace_step = h->trace_step < n ? h->trace_step : n - 1;
@@ -329,6 +331,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       if (h->tc) {
         TcGemm g{};
         g.W = h->p_qkv[l], g.X = h->xn_t, g.N = d.Nqkv, g.K = D, g.epi = TC_STORE, g.scale = h->s_qkv[l];
+        g.perm_dh = d.dh, g.perm_end = d.Nq + d.Hkv * d.dh;
         g.out_f32 = h->qkv, g.ldo = d.Nqkv, g.splits = 1;
         ST(tc_gemm(g));
       } else {
@@ -612,8 +615,8 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
           launch_pack_tiled(w->wgate[l], big_kind, pgu, D, F, 0, st, 64, 0);
           launch_pack_tiled(w->wup[l], big_kind, pgu, D, F, 0, st, 64, 1);
         }
-        launch_pack_tiled(w->wq[l], big_kind, pq, D, Nq, 0, st);
-        launch_pack_tiled(w->wk[l], big_kind, pq, D, Nkv, Nq, st);
+        launch_pack_tiled(w->wq[l], big_kind, pq, D, Nq, 0, st, 0, 0, d.dh);
+        launch_pack_tiled(w->wk[l], big_kind, pq, D, Nkv, Nq, st, 0, 0, d.dh);
         launch_pack_tiled(w->wv[l], big_kind, pq, D, Nkv, Nq + Nkv, st);
         launch_pack_tiled(w->wo[l], big_kind, po, Nq, D, 0, st);
         launch_pack_tiled(w->wgate[l], big_kind, pg, D, F, 0, st);
@@ -624,8 +627,8 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         if (w8) {
           cq = h->s_qkv_all + (size_t)l * Nqkv, co = h->s_o_all + (size_t)l * D, cg = h->s_g_all + (size_t)l * F;
           cu = h->s_u_all + (size_t)l * F, cd = h->s_d_all + (size_t)l * D;
-          CU(cudaMemcpyAsync(cq, sq, (size_t)Nq * 4, cudaMemcpyDeviceToDevice, st));
-          CU(cudaMemcpyAsync(cq + Nq, sk, (size_t)Nkv * 4, cudaMemcpyDeviceToDevice, st));
+          launch_permute_scales(sq, cq, Nq, 0, d.dh, st);
+          launch_permute_scales(sk, cq, Nkv, Nq, d.dh, st);
           CU(cudaMemcpyAsync(cq + Nq + Nkv, sv, (size_t)Nkv * 4, cudaMemcpyDeviceToDevice, st));
           CU(cudaMemcpyAsync(co, so, (size_t)D * 4, cudaMemcpyDeviceToDevice, st));
           CU(cudaMemcpyAsync(cg, sg, (size_t)F * 4, cudaMemcpyDeviceToDevice, st));
@@ -682,6 +685,9 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         ST(h->alloc(&h->attn64, (size_t)64 * Nq, true));
         ST(h->alloc(&h->m64, (size_t)64 * F, true));
         ST(h->alloc(&h->u64, (size_t)64 * D, true));
+        ST(h->alloc(&h->qr64, (size_t)64 * Nq, true));
+        ST(h->alloc(&h->kr64, (size_t)64 * Nkv, true));
+        ST(h->alloc(&h->vr64, (size_t)64 * Nkv, true));
         ST(h->alloc(&h->mega_scratch, mega_scratch_floats(d, 64 / d.S > 0 ? 64 / d.S : 1, 16), true));
         ST(h->alloc(&h->mega_counters, (size_t)MP_COUNT, true));
         const int so = (d.Nq / 64 + 7) / 8, sd = (d.F / 64 + 7) / 8;
@@ -837,7 +843,7 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     }
     if (!h->mega_ok) return fail(PHYAI_ERR_UNSUPPORTED, "tracing needs the persistent kernel");
     unsigned long long* buf = nullptr;
-    ST(h->alloc(&buf, (size_t)148 * MP_COUNT * 2, true));
+    ST(h->alloc(&buf, (size_t)148 * MP_COUNT * 4, true));
     h->mega_trace = buf, h->trace_step = (int)(value / 1000), h->trace_layer = (int)(value % 1000);
     return PHYAI_OK;
   }
@@ -861,7 +867,7 @@ phyai_status_t phyai_read_trace(phyai_expert_t* h, uint64_t* out, size_t capacit
                                 uint32_t* n_phases) {
   if (!h || !out || !n_ctas || !n_phases) return fail(PHYAI_ERR_INVALID_ARG, "NULL argument");
   if (!h->mega_trace) return fail(PHYAI_ERR_INVALID_ARG, "tracing is off (phyai_set_option(h, \"trace\", ...))");
-  const size_t n = (size_t)148 * MP_COUNT * 2;
+  const size_t n = (size_t)148 * MP_COUNT * 4;
   if (capacity < n) return fail(PHYAI_ERR_INVALID_ARG, "capacity %zu < %zu entries", capacity, n);
   CU(cudaMemcpy(out, h->mega_trace, n * sizeof(uint64_t), cudaMemcpyDeviceToHost));
   *n_ctas = 148, *n_phases = MP_COUNT;

@@ -98,28 +98,31 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
       }
     }
   } else if (warp == 4) {
-    // ---------------- MMA issuer ---------------------------------------------------------------
-    if (lane == 0) {
-      for (int i = 0; i < nk; ++i) {
-        const int s = i % STAGES;
-        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        const bool ok = mbar_wait(smem_u32(&bar_full[s]), ph, wc);
-        tc_fence_after();
+    // ---------------- MMA issuer (whole warp in the loop, one elected lane issues) ---------------------
+    for (int i = 0; i < nk; ++i) {
+      const int s = i % STAGES;
+      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+      const bool ok = mbar_wait(smem_u32(&bar_full[s]), ph, wc);
+      tc_fence_after();
+      const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
+      const uint64_t da = make_desc(a0);
+      const uint64_t da2 = make_desc(a0 + A_BYTES);
+      const uint64_t db = make_desc(a0 + A_BYTES * (DUAL ? 2 : 1));
+      if (elect_one()) {
         if (ok) {
-          const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
-          const uint64_t da = make_desc(a0);
-          const uint64_t db = make_desc(a0 + A_BYTES * (DUAL ? 2 : 1));
 #pragma unroll
           for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
             const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
             umma_bf16(tmem_base, da + 2 * k, db + 2 * k, IDESC, acc);
-            if (DUAL) umma_bf16(tmem_base + NT, make_desc(a0 + A_BYTES) + 2 * k, db + 2 * k, IDESC, acc);
+            if (DUAL) umma_bf16(tmem_base + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
           }
         }
         umma_commit(smem_u32(&bar_empty[s]));  // frees the stage when the MMAs above have read it
       }
-      umma_commit(smem_u32(&bar_accum));
+      __syncwarp();
     }
+    if (elect_one()) umma_commit(smem_u32(&bar_accum));
+    __syncwarp();
   } else {
     // ---------------- epilogue: TMEM -> registers -> global --------------------------------------
     const int q = warp & 3;
@@ -127,6 +130,7 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
     const bool ok = mbar_wait(smem_u32(&bar_accum), 0, wc);
     tc_fence_after();
     const float sc = g.scale ? g.scale[n] : 1.0f;
+    const int n_out = (g.perm_dh && n < g.perm_end) ? qkv_packed_to_channel(n, g.perm_dh) : n;  // output column
     const int tok_base = tt * NT;
     if (ok) {
       if (!DUAL) {
@@ -142,7 +146,7 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
             if (tok < g.M) {
               const float val = v[j] * sc;
               if (g.epi == TC_STORE) {
-                g.out_f32[(size_t)tok * g.ldo + n] = val;
+                g.out_f32[(size_t)tok * g.ldo + n_out] = val;
               } else if (g.epi == TC_RESID) {
                 atomicAdd(&g.out_f32[(size_t)tok * g.ldo + n], gt * val);
               } else {

@@ -25,8 +25,11 @@ void launch_copy_cols(const void* src, int src_kind, const float* scale, float* 
 // n stored at packed row n_off + n of a matrix with KC = K/64 column chunks.
 // With il_group > 0 the channels of two matrices are interleaved in groups of il_group rows
 // (il_second selects the second matrix): packed row = (n / g) * 2g + n % g + (second ? g : 0).
+// With perm_dh > 0 the channels follow the rotary-pair row order of the fused QKV matrix
+// (qkv_channel_to_packed).
 void launch_pack_tiled(const void* src, int src_kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st,
-                       int il_group = 0, int il_second = 0);
+                       int il_group = 0, int il_second = 0, int perm_dh = 0);
+void launch_permute_scales(const float* src, float* dst, int N, int n_off, int perm_dh, cudaStream_t st);
 // Y[r][n] = act( sum_d X[r][d] * W[(w_row_off + d)][n] + bias[n] + add[n] ), r < R
 void launch_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K, const float* bias,
                       const float* add, int act_swish, float* Y, int ldy, int R, cudaStream_t st);
@@ -99,6 +102,7 @@ struct TcGemm {
   int rows_in, rows_out, row_off;   // TC_BIAS_ROWMAP row remap
   int gelu_exact;
   int splits;                       // split-K factor (TC_RESID only)
+  int perm_dh, perm_end;            // TC_STORE: packed rows < perm_end map to channels by qkv_packed_to_channel
   unsigned wait_limit;
 };
 // Returns cudaSuccess or the launch error; `nt` is the token-tile width (64, 128 or 256).

@@ -12,11 +12,14 @@
 // flowing while the CTA waits for activations.
 //
 // Warp roles (512 threads): warps 0-7 workers (epilogues, attention, norms, head; 224 registers via
-// setmaxnreg), warp 8 tcgen05 MMA issuer + TMEM owner, warps 9-11 activation producers, warps 12-15
+// setmaxnreg), warp 8 tcgen05 MMA issuer + TMEM owner, warps 9-10 activation producers, warps 11-15
 // weight producers (32 registers).
 //
-// Shared memory: 5 x 16 KB weight ring + 128 KB "region A" (the activations of the current GEMM role,
-// or the attention tiles, or the GeGLU exchange buffer; its users take turns in program order).
+// Shared memory: 9 x 16 KB weight ring (a CTA's next GEMM role is prefetched in full) + 64 KB
+// "region A": two 32 KB slots through which the activations of the current GEMM role stream in chunks
+// of four 64-wide k-chunks; the same 64 KB serve the attention role (Q tile + one K/V tile of 32 keys),
+// the rotary / GeGLU exchange of the epilogues and the velocity head.  Its users take turns in program
+// order.
 #include "mega.h"
 
 #include <algorithm>
@@ -29,10 +32,14 @@
 namespace phyai {
 namespace {
 
-constexpr int RING = 5;                 // weight ring slots
+constexpr int RING = 9;                 // weight ring slots
 constexpr int UNIT = 16384;             // one weight block: 128 rows x 64 k, bf16
 constexpr int ACT_TILE = 8192;          // one activation tile: 64 tokens x 64 k, bf16
-constexpr int REGION_A = 131072;
+constexpr int ACT_SLOT = 4 * ACT_TILE;   // activations stream through two slots of four k-chunks
+constexpr int REGION_A = 2 * ACT_SLOT;
+constexpr int KTA = 32;                 // keys per attention tile inside the persistent kernel
+constexpr int NPROD_W = 5;              // weight producer warps (11..15)
+constexpr int BAR_ATTN = 2;             // named barrier of the four attention warps
 constexpr int NWORK = 256;              // worker threads
 constexpr int BAR_WORK = 1;             // named barrier of the 8 worker warps
 constexpr int MAX_D = 2048;
@@ -64,23 +71,35 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// GELU for the GeGLU epilogue: tanh form written as z * sigmoid(2u) (one exp, one fast divide), erf form as is.
+__device__ __forceinline__ float gelu_fast(float z, int exact) {
+  if (exact) return gelu_erf_f(z);
+  const float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
+  return __fdividef(z, 1.0f + __expf(-2.0f * u));
+}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Trace stamp of worker thread 0: which = 0 (inputs ready) or 1 (role done).
+// Trace stamp: which = 0 (worker: inputs ready / accumulator complete), 1 (worker: role done),
+// 2 (MMA issuer: first activation chunk in shared memory), 3 (MMA issuer: last MMA issued).
 __device__ __forceinline__ void stamp(const MegaParams& p, int phase, int step, int layer, int which, int wt) {
   if (p.trace && wt == 0 && step == p.trace_step && (layer == p.trace_layer || phase >= MP_EMBED))
-    p.trace[((size_t)blockIdx.x * MP_COUNT + phase) * 2 + which] = global_ns();
+    p.trace[((size_t)blockIdx.x * MP_COUNT + phase) * 4 + which] = global_ns();
 }
 
 struct Shared {
   uint64_t w_full[RING], w_empty[RING];
-  uint64_t act_full, act_empty, acc_full, acc_empty;
+  uint64_t act_full[2], chunk_free[2];   // per activation slot
+  uint64_t act_empty, acc_full, acc_empty;
   uint32_t tmem_slot;
   int abort_flag;
   int bcast;
+  int tok_pos[64];   // rotary position of every suffix token: prefix_len of its request + index
+  int tok_q[64];     // b * Hq * S + i   (row offset of the token in the rotated q buffer, before the head term)
+  int tok_kv[64];    // b * Hkv * S + i
+  int arow_out[64];  // residual-stream row of action row r: (r / H) * S + ns + r % H
   float red[16];
   float xs[64];
   alignas(16) float row[MAX_D];   // float4 accesses
@@ -282,7 +301,10 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
       mbar_init(smem_u32(&sh.w_full[s]), 1);
       mbar_init(smem_u32(&sh.w_empty[s]), 1);
     }
-    mbar_init(smem_u32(&sh.act_full), 3);
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(smem_u32(&sh.act_full[k]), 1);
+      mbar_init(smem_u32(&sh.chunk_free[k]), 1);
+    }
     mbar_init(smem_u32(&sh.act_empty), 1);
     mbar_init(smem_u32(&sh.acc_full), 1);
     mbar_init(smem_u32(&sh.acc_empty), 1);
@@ -303,20 +325,20 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
 
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 32;");
-    if (warp >= 12) {
-      // ============ weight producers: unit u of the CTA's stream is loaded by warp 12 + (u & 3) ============
+    if (warp >= 11) {
+      // ============ weight producers: unit u of the CTA's stream is loaded by warp 11 + u % 5 ================
       if (lane == 0) {
         ProgIter it(p, pl);
         Item im;
         unsigned u = 0;
-        const unsigned me = (unsigned)(warp - 12);
+        const unsigned me = (unsigned)(warp - 11);
         bool alive = true;
         while (alive && it.next(im)) {
           if (!im.gemm) continue;
           const uint8_t* src =
               weight_base(p, im.phase, im.layer) + ((size_t)im.role.tile * phase_kc(p, im.phase) + im.role.kc_begin) * UNIT;
           for (int j = 0; j < im.role.kc_count; ++j, ++u) {
-            if ((u & 3u) != me) continue;
+            if (u % NPROD_W != me) continue;
             const unsigned s = u % RING, ph = (u / RING) & 1u;
             if (!mbar_wait(smem_u32(&sh.w_empty[s]), ph ^ 1u, wc)) {
               alive = false;
@@ -329,11 +351,13 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
         }
       }
     } else if (warp >= 9) {
-      // ============ activation producers: each loads a third of the role's k-chunks into region A ===========
+      // ============ activation producers: warp 9 feeds slot 0, warp 10 slot 1; a role's k-chunks stream
+      //              through the two slots in groups of four ==============================================
       if (lane == 0) {
         ProgIter it(p, pl);
         Item im;
         unsigned a_idx = 0;
+        unsigned uses = 0;           // how many chunk groups this slot has received so far
         const int me = warp - 9;
         while (it.next(im)) {
           const unsigned a = a_idx++;
@@ -344,39 +368,65 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
           gemm_dep(p, im.phase, im.step, im.layer, dep, target);
           const bool ok = wait_count(p.counters + dep, target, wc);
           fence_async_proxy();
-          const int j0 = im.role.kc_count * me / 3, j1 = im.role.kc_count * (me + 1) / 3;
-          const uint32_t bytes = ok ? (uint32_t)(j1 - j0) * ACT_TILE : 0u;
-          const uint32_t full = smem_u32(&sh.act_full);
-          mbar_expect_tx(full, bytes);
-          if (bytes)
-            bulk_g2s(regA + (uint32_t)j0 * ACT_TILE, act_base(p, im.phase) + (size_t)(im.role.kc_begin + j0) * ACT_TILE,
-                     bytes, full);
+          const int groups = (im.role.kc_count + 3) / 4;
+          for (int gidx = me; gidx < groups; gidx += 2, ++uses) {
+            // within a role the slot is reused every other group: wait until the MMAs of its previous
+            // occupant have finished reading it
+            if (gidx >= 2) mbar_wait(smem_u32(&sh.chunk_free[me]), (uses - 1) & 1u, wc);
+            const int j0 = gidx * 4, n = min(4, im.role.kc_count - j0);
+            const uint32_t bytes = ok ? (uint32_t)n * ACT_TILE : 0u;
+            const uint32_t full = smem_u32(&sh.act_full[me]);
+            mbar_expect_tx(full, bytes);
+            if (bytes)
+              bulk_g2s(regA + (uint32_t)me * ACT_SLOT, act_base(p, im.phase) + (size_t)(im.role.kc_begin + j0) * ACT_TILE,
+                       bytes, full);
+          }
         }
       }
     } else if (warp == 8) {
-      // ============ MMA issuer =====================================================================================
-      if (lane == 0) {
+      // ============ MMA issuer: the whole warp walks the program, one elected lane issues ==========================
+      {
         ProgIter it(p, pl);
         Item im;
         unsigned u = 0, g = 0;
+        unsigned uses0 = 0u, uses1 = 0u;   // chunk groups consumed from each slot
         while (it.next(im)) {
           if (!im.gemm) continue;
-          bool ok = mbar_wait(smem_u32(&sh.act_full), g & 1u, wc);
-          if (g > 0) ok = mbar_wait(smem_u32(&sh.acc_empty), (g - 1) & 1u, wc) && ok;  // epilogue drained TMEM
-          tc_fence_after();
-          for (int j = 0; j < im.role.kc_count; ++j, ++u) {
-            const unsigned s = u % RING, ph = (u / RING) & 1u;
-            const bool okw = mbar_wait(smem_u32(&sh.w_full[s]), ph, wc);
+          bool ok = true;
+          if (g > 0) ok = mbar_wait(smem_u32(&sh.acc_empty), (g - 1) & 1u, wc);  // epilogue drained TMEM
+          const int groups = (im.role.kc_count + 3) / 4;
+          for (int gidx = 0; gidx < groups; ++gidx) {
+            const int sl = gidx & 1;
+            ok = mbar_wait(smem_u32(&sh.act_full[sl]), (sl ? uses1 : uses0) & 1u, wc) && ok;
+            if (sl) ++uses1; else ++uses0;
+            if (gidx == 0 && lane == 0) stamp(p, im.phase, im.step, im.layer, 2, 0);
             tc_fence_after();
-            if (ok && okw) {
+            const int j0 = gidx * 4, n = min(4, im.role.kc_count - j0);
+            bool okw = true;
+            for (int j = 0; j < n; ++j) okw = mbar_wait(smem_u32(&sh.w_full[(u + j) % RING]), ((u + j) / RING) & 1u, wc) && okw;
+            tc_fence_after();
+            for (int j = 0; j < n; ++j) {   // warp-uniform loop; one elected lane issues
+              const unsigned s = (u + j) % RING;
               const uint64_t da = make_desc(ring + s * UNIT);
-              const uint64_t db = make_desc(regA + (uint32_t)j * ACT_TILE);
-#pragma unroll
-              for (int k = 0; k < 4; ++k) umma_bf16(tmem_base, da + 2 * k, db + 2 * k, IDESC64, (j > 0 || k > 0) ? 1u : 0u);
+              const uint64_t db = make_desc(regA + (uint32_t)sl * ACT_SLOT + (uint32_t)j * ACT_TILE);
+              const uint32_t first = (j0 + j > 0) ? 1u : 0u;
+              if (elect_one()) {
+                if (ok && okw) {
+                  umma_bf16(tmem_base, da, db, IDESC64, first);
+                  umma_bf16(tmem_base, da + 2, db + 2, IDESC64, 1u);
+                  umma_bf16(tmem_base, da + 4, db + 4, IDESC64, 1u);
+                  umma_bf16(tmem_base, da + 6, db + 6, IDESC64, 1u);
+                }
+                umma_commit(smem_u32(&sh.w_empty[s]));
+                if (j == n - 1) umma_commit(smem_u32(&sh.chunk_free[sl]));   // the slot may be refilled
+              }
+              __syncwarp();
             }
-            umma_commit(smem_u32(&sh.w_empty[s]));
+            u += n;
           }
-          umma_commit(smem_u32(&sh.acc_full));
+          if (lane == 0) stamp(p, im.phase, im.step, im.layer, 3, 0);
+          if (elect_one()) umma_commit(smem_u32(&sh.acc_full));
+          __syncwarp();
           ++g;
         }
       }
@@ -387,6 +437,14 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
     const int wt = tid;                       // 0..255
     const int q = warp & 3, hf = warp >> 2;   // TMEM lane quarter, token-column half
     const Request rq = *p.rq;
+    if (wt < 64) {   // per-token index tables: no integer division in the epilogue loops
+      const int b = wt / d.S, i = wt % d.S;
+      sh.tok_pos[wt] = wt < p.M ? rq.cu_lens[b + 1] - rq.cu_lens[b] + i : 0;
+      sh.tok_q[wt] = b * d.Hq * d.S + i;
+      sh.tok_kv[wt] = b * d.Hkv * d.S + i;
+      sh.arow_out[wt] = (wt / d.H) * d.S + d.ns + wt % d.H;
+    }
+    work_sync();
     unsigned a_idx = 0, g_idx = 0;
     const int D = d.D, S = d.S, H = d.H;
     const int embed_last = p.ada ? MP_EMBED : MP_EMBED_GEMM;
@@ -408,11 +466,46 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
       const int tok0 = hf * 32;
       if (ok) {
         if (phase == MP_QKV) {
+          // rows 0..63 hold 64 channels of the first half of a head, rows 64..127 their rotary partners
+          // (v tiles: plain order).  Exchange through shared memory, rotate, scale q, round to bf16.
           const int n = r.tile * 128 + ch;
           const float sc = p.s_qkv ? p.s_qkv[(size_t)layer * d.Nqkv + n] : 1.0f;
+          const int Nk_end = d.Nq + d.Hkv * DH;
+          const bool is_v = n >= Nk_end, is_q = n < d.Nq;
+          const int c = is_v ? n : qkv_packed_to_channel(n, DH);     // channel in (q | k | v)
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (tok0 + j < p.M) p.qkv[(size_t)(tok0 + j) * d.Nqkv + n] = v[j] * sc;
+          for (int j = 0; j < 32; ++j) regA_f[(tok0 + j) * 128 + ch] = v[j] * sc;
+          work_sync();
+          constexpr int half = DH / 2;
+          const int cin = is_q ? c % DH : (is_v ? (c - Nk_end) % DH : (c - d.Nq) % DH);   // channel within the head
+          const int head = is_q ? c / DH : (is_v ? (c - Nk_end) / DH : (c - d.Nq) / DH);
+          const int jrot = cin % half;
+          const bool lower = cin < half;
+          const float qs = is_q ? rsqrtf((float)DH) : 1.0f;
+          const int partner = ch ^ 64;
+          // two batches of 16 tokens: all table loads of a batch are issued before they are used
+#pragma unroll
+          for (int j0 = 0; j0 < 32; j0 += 16) {
+            float2 cs[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int tok = tok0 + j0 + j;
+              cs[j] = make_float2(1.f, 0.f);
+              if (tok < p.M && !is_v && p.rope) cs[j] = p.rope[(size_t)sh.tok_pos[tok] * half + jrot];
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int tok = tok0 + j0 + j;
+              if (tok < p.M) {
+                const float other = regA_f[tok * 128 + partner];
+                const float x = v[j0 + j] * sc;
+                const float y = lower ? x * cs[j].x - other * cs[j].y : x * cs[j].x + other * cs[j].y;
+                __nv_bfloat16* dst = is_q ? p.qr + (size_t)(sh.tok_q[tok] + head * S) * DH
+                                          : (is_v ? p.vr : p.kr) + (size_t)(sh.tok_kv[tok] + head * S) * DH;
+                dst[cin] = __float2bfloat16_rn(y * qs);
+              }
+            }
+          }
         } else if (phase == MP_O || phase == MP_DOWN) {
           const int n = r.tile * 128 + ch;
           const float* sp = phase == MP_O ? p.s_o : p.s_d;
@@ -428,7 +521,7 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const int tok = tok0 + j;
-            if (tok < p.batch * H) p.h[(size_t)((tok / H) * S + d.ns + tok % H) * D + n] = v[j] + bs;
+            if (tok < p.batch * H) p.h[(size_t)sh.arow_out[tok] * D + n] = v[j] + bs;
           }
         } else {  // MP_GATEUP: rows 0..63 gate, rows 64..127 up of the same 64 channels
           const int c64 = ch & 63;
@@ -439,19 +532,28 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
             for (int j = 0; j < 32; ++j) regA_f[(tok0 + j) * 64 + c64] = v[j] * su;
           }
           work_sync();
+          // the 64 x 64 bf16 result is exactly k-chunk `tile` of the down projection's input: build its
+          // swizzled 8 KB image in shared memory, then copy it out with 16-byte stores
+          __nv_bfloat16* img = reinterpret_cast<__nv_bfloat16*>(regA_f + 64 * 64);
           if (q < 2) {
             const float sg = p.s_g ? p.s_g[(size_t)layer * d.F + f] : 1.0f;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int tok = tok0 + j;
-              if (tok < p.M) {
-                const float m = gelu_f(v[j] * sg, d.gelu_exact) * regA_f[tok * 64 + c64];
-                p.m64[tiled_index(tok, f, 64)] = __float2bfloat16_rn(m);
-              }
+              const float m = gelu_fast(v[j] * sg, d.gelu_exact) * regA_f[tok * 64 + c64];
+              img[tok * 64 + (((c64 >> 3) ^ (tok & 7)) << 3) + (c64 & 7)] = __float2bfloat16_rn(m);
             }
           }
+          work_sync();
+          uint4* gdst = reinterpret_cast<uint4*>(p.m64 + (size_t)r.tile * 64 * 64);
+          const uint4* gsrc = reinterpret_cast<const uint4*>(img);
+          for (int idx = wt; idx < 64 * 8; idx += NWORK)
+            if ((idx >> 3) < p.M) gdst[idx] = gsrc[idx];
         }
       } else if (phase == MP_GATEUP) {
+        work_sync();
+        work_sync();
+      } else if (phase == MP_QKV) {
         work_sync();
       }
       signal_phase(p, phase, wt);
@@ -472,16 +574,28 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
           const int b = r / H, i = r % H;
           if (wt < d.A) sh.xs[wt] = rq.x[(size_t)r * d.A + wt];
           work_sync();
-          for (int n = wt; n < D; n += NWORK) {
-            float acc = 0.f;
+          for (int n = wt * 4; n < D; n += NWORK * 4) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
-            for (int a = 0; a < d.A; ++a) acc = fmaf(sh.xs[a], p.Wc[(size_t)a * D + n], acc);
-            if (p.ada) {
-              p.h[(size_t)(b * S + d.ns + i) * D + n] = acc + p.bcfold[n];
-            } else {
-              p.u64[tiled_index(r, n, 64)] = __float2bfloat16_rn(swish_precise(acc + p.tb[(size_t)step * D + n]));
+            for (int a = 0; a < d.A; ++a) {
+              const float4 w4 = *reinterpret_cast<const float4*>(p.Wc + (size_t)a * D + n);
+              const float xa = sh.xs[a];
+              acc.x = fmaf(xa, w4.x, acc.x), acc.y = fmaf(xa, w4.y, acc.y);
+              acc.z = fmaf(xa, w4.z, acc.z), acc.w = fmaf(xa, w4.w, acc.w);
             }
-            if (d.ns && i == 0) p.h[(size_t)(b * S) * D + n] = p.state_tok[(size_t)b * D + n];
+            if (p.ada) {
+              const float4 bb = *reinterpret_cast<const float4*>(p.bcfold + n);
+              *reinterpret_cast<float4*>(p.h + (size_t)(b * S + d.ns + i) * D + n) =
+                  make_float4(acc.x + bb.x, acc.y + bb.y, acc.z + bb.z, acc.w + bb.w);
+            } else {
+              const float4 tb = *reinterpret_cast<const float4*>(p.tb + (size_t)step * D + n);
+              *reinterpret_cast<uint2*>(p.u64 + tiled_index(r, n, 64)) =
+                  make_uint2(pack_bf16(swish_precise(acc.x + tb.x), swish_precise(acc.y + tb.y)),
+                             pack_bf16(swish_precise(acc.z + tb.z), swish_precise(acc.w + tb.w)));
+            }
+            if (d.ns && i == 0)
+              *reinterpret_cast<float4*>(p.h + (size_t)(b * S) * D + n) =
+                  *reinterpret_cast<const float4*>(p.state_tok + (size_t)b * D + n);
           }
           work_sync();
         }
@@ -513,16 +627,16 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
           if (wt == 0 && a_idx > 0) mbar_wait(smem_u32(&sh.act_empty), (a_idx - 1) & 1u, wc);
           const bool go = await_phase(p, sh, MP_QKV, (unsigned)(inst + 1) * (unsigned)p.n_cta[MP_QKV], wc, wt);
           stamp(p, MP_ATTN, step, layer, 0, wt);
-          AttnArgs a;
-          a.rq = p.rq, a.status = p.status, a.qkv = p.qkv, a.rope = p.rope, a.layer = layer, a.out = p.attn64;
+          AttnArgs a{};
+          a.rq = p.rq, a.status = p.status, a.qkv = nullptr, a.rope = nullptr, a.layer = layer, a.out = p.attn64;
+          a.qr = p.qr, a.kr = p.kr, a.vr = p.vr;
           a.rows_pad = 64, a.num_splits = p.attn_splits, a.part_o = p.attn_scratch;
           a.part_ml = p.attn_scratch + (size_t)p.batch * d.Hq * p.attn_splits * QROWS * DH;
           a.d = d, a.wait_limit = p.wait_limit;
-          const int HG = d.Hq / 2;
-          if (go) {
+          if (go && warp < 4) {   // one head per role, four warps; the other four workers wait at the barrier below
             for (int id = pl.attn_begin; id < pl.attn_end; ++id) {
-              const int split = id % p.attn_splits, hg = (id / p.attn_splits) % HG, b = id / (p.attn_splits * HG);
-              attn_role<DH, 2, 1, BAR_WORK>(a, split, hg, b, regA, wt);
+              const int split = id % p.attn_splits, head = (id / p.attn_splits) % d.Hq, b = id / (p.attn_splits * d.Hq);
+              attn_role<DH, 1, 1, BAR_ATTN, KTA>(a, split, head, b, regA, wt);
             }
           }
           signal_phase(p, MP_ATTN, wt);
@@ -650,7 +764,6 @@ constexpr size_t MEGA_SMEM = 1024 + (size_t)RING * UNIT + REGION_A;
 bool mega_supported(const Dims& d, int batch) {
   if (batch * d.S > 64 || d.S > 64) return false;
   if (d.dh != 128 && d.dh != 256) return false;
-  if (d.Hq % 2 || (d.Hq / d.Hkv) % 2) return false;   // two query heads of one kv head per attention role
   if (d.D % 128 || d.F % 64 || d.Nq % 128 || d.Nqkv % 128) return false;
   if (d.D > MAX_D || d.D / 64 > 16 || d.A > 64) return false;  // full-K roles hold <= 16 k-chunks in region A
   return true;
@@ -661,9 +774,9 @@ size_t mega_scratch_floats(const Dims& d, int batch, int splits) {
 }
 
 int mega_attention_splits(const Dims& d, int batch, int max_prefix, int ncta) {
-  const int groups = batch * (d.Hq / 2);
+  const int groups = batch * d.Hq;
   int want = ncta / groups;
-  const int tiles = (max_prefix + KT - 1) / KT + 1;
+  const int tiles = (max_prefix + KTA - 1) / KTA + (d.S + KTA - 1) / KTA;
   want = std::min(want, std::min(tiles, 16));
   return std::max(want, 1);
 }
@@ -729,7 +842,7 @@ bool mega_plan(const Dims& d, int batch, int ada, int attn_splits, int ncta, Meg
   spread(rowsA, [](MegaCtaPlan& pl, int b, int e) { pl.embed_begin = b, pl.embed_end = e; }, n_cta[MP_EMBED]);
   spread(rowsA, [](MegaCtaPlan& pl, int b, int e) { pl.final_begin = b, pl.final_end = e; }, n_cta[MP_FINAL]);
   // attention roles over all CTAs, least loaded first
-  const int n_attn = batch * (d.Hq / 2) * attn_splits;
+  const int n_attn = batch * d.Hq * attn_splits;
   spread(n_attn, [](MegaCtaPlan& pl, int b, int e) { pl.attn_begin = b, pl.attn_end = e; }, n_cta[MP_ATTN]);
   if (attn_splits > 1) {
     const int n_merge = batch * d.Hq * d.S;

@@ -51,11 +51,12 @@ struct MegaParams {
   // activations (tiled bf16 with rows_pad = 64 so that consecutive k-chunks are contiguous)
   float *h, *qkv;
   __nv_bfloat16 *xn64, *attn64, *m64, *u64;
+  __nv_bfloat16 *qr, *kr, *vr;   // rotated (q also scaled) bf16 q [b][Hq][S][dh], k / v [b][Hkv][S][dh]
   float* attn_scratch;
   float* slab;                   // [max(o_splits, d_splits)][64][D] split-K partial sums of O / down
   int o_splits, d_splits;
-  // optional trace: [gridDim.x][MP_COUNT][2] globaltimer stamps (ns) of (inputs ready, role done) for
-  // the traced (step, layer); null = off
+  // optional trace: [gridDim.x][MP_COUNT][4] globaltimer stamps (ns) for the traced (step, layer):
+  // worker inputs ready, worker role done, MMA issuer first activations, MMA issuer last MMA; null = off
   unsigned long long* trace;
   int trace_step, trace_layer;
 };

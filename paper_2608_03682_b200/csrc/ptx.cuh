@@ -34,6 +34,7 @@ struct WaitCtx {
 // Bounded wait.  Returns false (and records ST_TIMEOUT) when the limit expires or the CTA has
 // already given up; callers then skip their side effects but keep walking their loops.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& c) {
+  if (mbar_test(bar, parity)) return true;   // fast path: already complete
   if (*c.abort_flag) return false;
   for (uint32_t it = 0; it < c.limit; ++it) {
     if (mbar_test(bar, parity)) return true;

@@ -79,7 +79,7 @@ void launch_copy_cols(const void* src, int kind, const float* scale, float* dst,
 // Weight [K][N] -> packed out-channel-major swizzled blocks.  One thread per 16-byte chunk
 // (8 consecutive k of one out channel): reads are strided by N (one-off cost at create).
 __global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, int il_group,
-                             int il_second) {
+                             int il_second, int perm_dh) {
   const int KC = K >> 6;
   const size_t chunks = (size_t)N * (K >> 3);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
@@ -87,7 +87,8 @@ __global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int 
     const int k8 = (int)(i / N);        // chunk index along K
     const int k0 = k8 << 3;
     // optional interleave: groups of il_group channels of two matrices alternate in the packed rows
-    const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0) : n_off + n;
+    const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
+                            : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
     const int kc = k0 >> 6, c = (k0 & 63) >> 3;
     const size_t base = (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 64 + (size_t)((c ^ (np & 7)) << 3);
     __align__(16) __nv_bfloat16 v[8];
@@ -97,10 +98,19 @@ __global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int 
   }
 }
 void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st,
-                       int il_group, int il_second) {
+                       int il_group, int il_second, int perm_dh) {
   const size_t chunks = (size_t)N * (K >> 3);
   const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
-  k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off, il_group, il_second);
+  k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off, il_group, il_second, perm_dh);
+}
+
+// dst[n_off + packed(c)] = src[c]: per-channel scales in the packed row order of the fused QKV matrix
+__global__ void k_permute_scales(const float* src, float* dst, int N, int n_off, int perm_dh) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < N) dst[n_off + (perm_dh ? qkv_channel_to_packed(c, perm_dh) : c)] = src[c];
+}
+void launch_permute_scales(const float* src, float* dst, int N, int n_off, int perm_dh, cudaStream_t st) {
+  k_permute_scales<<<(N + 255) / 256, 256, 0, st>>>(src, dst, N, n_off, perm_dh);
 }
 
 // =============================================================================================
