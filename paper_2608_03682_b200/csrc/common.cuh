@@ -92,6 +92,13 @@ __device__ __forceinline__ float gelu_tanh_f(float z) {
 __device__ __forceinline__ float gelu_erf_f(float z) { return 0.5f * z * (1.0f + erff(z * 0.7071067811865476f)); }
 __device__ __forceinline__ float gelu_f(float z, int exact) { return exact ? gelu_erf_f(z) : gelu_tanh_f(z); }
 
+// GELU for the GeGLU epilogues: tanh form written as z * sigmoid(2u) (one exp, one fast divide), erf form as is.
+__device__ __forceinline__ float gelu_fast(float z, int exact) {
+  if (exact) return gelu_erf_f(z);
+  const float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
+  return __fdividef(z, 1.0f + __expf(-2.0f * u));
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

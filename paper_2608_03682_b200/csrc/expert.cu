@@ -354,7 +354,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       if (h->tc) {
         TcGemm g{};
         g.W = h->p_o[l], g.X = h->attn_t, g.N = D, g.K = d.Nq, g.epi = TC_RESID, g.scale = h->s_o[l], g.gate = gate;
-        g.out_f32 = h->h, g.ldo = D, g.splits = pick_splits(D / 128, tok_tiles, d.Nq / 64);
+        g.out_f32 = h->h, g.ldo = D, g.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.Nq / 64);
         ST(tc_gemm(g));
       } else {
         SimtGemm g{};
@@ -372,7 +372,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         ST(tc_gemm(g));
         TcGemm g2{};
         g2.W = h->p_d[l], g2.X = h->m_t, g2.N = D, g2.K = d.F, g2.epi = TC_RESID, g2.scale = h->s_d[l], g2.gate = gate;
-        g2.out_f32 = h->h, g2.ldo = D, g2.splits = pick_splits(D / 128, tok_tiles, d.F / 64);
+        g2.out_f32 = h->h, g2.ldo = D, g2.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.F / 64);
         ST(tc_gemm(g2));
       } else {
         SimtGemm g{};

@@ -12,10 +12,15 @@
 //   B: activations kept in the tiled bf16 layout, so an NT x 64 tile is one contiguous block.
 // Every load is therefore a 1-D bulk copy (16-byte aligned, size a multiple of 16): no tensor map.
 //
-// Warp roles (288 threads): warps 0..3 = copy producers (stage i is loaded by warp i % 4: one
-// warp's bulk copies complete one at a time, about 0.5 us each whatever their size, so several
-// issuing warps are needed to keep more than ~30 GB/s per SM in flight), warp 4 = TMEM owner +
-// MMA issuer, warps 5..8 = epilogue (TMEM lane quarter = warp % 4).
+// A CTA computes NA (1 or 2) 128-channel tiles against one NT-token tile: with NA = 2 and NT = 256 a
+// k-step moves 64 KB for 8 MMAs of 128 clocks, i.e. 64 bytes per clock, which is what one SM's L2 port
+// delivers (~126 GB/s measured); a single 128 x 256 tile would need 96 bytes per clock.
+//
+// Warp roles (544 threads): warps 0..7 = copy producers (the copies of all stages are dealt round
+// robin to the eight warps: one warp's bulk copies complete one at a time, about 0.5 us each whatever
+// their size, so many issuing warps are needed to keep the SM's L2 port busy), warp 8 = TMEM owner +
+// MMA issuer (whole warp in the loop, one elected lane issues), warps 9..16 = epilogue (TMEM lane
+// quarter = warp % 4, token-column half = (warp - 9) / 4).
 // Every wait is bounded: on expiry the CTA raises the status word, stops issuing copies, and
 // drains to its normal exit (TMEM is always released).
 #include "kernels.h"
@@ -26,12 +31,20 @@ namespace phyai {
 namespace {
 
 constexpr int A_BYTES = 128 * 128;  // one weight block: 128 out channels x 64 k (bf16)
+constexpr int NPROD = 8;
+constexpr int NEPI = 256;           // epilogue threads
+constexpr int BAR_EPI = 1;
 
-template <int NT, bool DUAL, int STAGES>
-__global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g) {
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync %0, %1;" ::"n"(BAR_EPI), "n"(NEPI) : "memory"); }
+
+template <int NT, int NA, int STAGES>
+__global__ void __launch_bounds__(544, 1) k_gemm_tc(int* status, const TcGemm g) {
   constexpr int B_BYTES = NT * 128;
-  constexpr int STAGE_BYTES = A_BYTES * (DUAL ? 2 : 1) + B_BYTES;
-  constexpr int COLS = DUAL ? 2 * NT : NT;
+  constexpr int NB = NT > 128 ? NT / 128 : 1;          // the activation tile is copied in pieces of <= 16 KB
+  constexpr int B_PIECE = B_BYTES / NB;
+  constexpr int NCOPY = NA + NB;
+  constexpr int STAGE_BYTES = A_BYTES * NA + B_BYTES;
+  constexpr int COLS = NA * NT;
   // instruction descriptor: D fp32 (bit 4), A bf16 (bit 7), B bf16 (bit 10), both K-major,
   // N >> 3 at bit 17, M >> 4 at bit 24.
   constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((128u >> 4) << 24);
@@ -46,6 +59,7 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt_idx = blockIdx.x, tt = blockIdx.y;
+  const bool geglu = g.epi == TC_GEGLU;
   const int KC = g.K >> 6;
   const int kc_begin = (int)(((long long)KC * blockIdx.z) / gridDim.z);
   const int kc_end = (int)(((long long)KC * (blockIdx.z + 1)) / gridDim.z);
@@ -59,16 +73,17 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
   if (skip_flag) return;
 
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tiles_ptr = smem_raw + (tiles - smem_u32(smem_raw));
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_full[s]), NCOPY);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
     mbar_init(smem_u32(&bar_accum), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 4) {
-    tmem_alloc(smem_u32(&tmem_slot), COLS);
+  if (warp == 8) {
+    tmem_alloc(smem_u32(&tmem_slot), COLS < 32 ? 32 : COLS);
     tc_fence_before();
   }
   __syncthreads();
@@ -76,28 +91,38 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
   const WaitCtx wc{status, &abort_flag, g.wait_limit};
 
-  constexpr int NPROD = STAGES < 4 ? STAGES : 4;
-  if (warp < 4) {
-    // ---------------- producers: warp w streams the stages i = w, w + NPROD, ... ---------------------
-    if (lane == 0 && warp < NPROD) {
-      const uint8_t* wsrc = reinterpret_cast<const uint8_t*>(g.W) + ((size_t)nt_idx * KC + kc_begin) * A_BYTES;
-      const uint8_t* wsrc2 =
-          DUAL ? reinterpret_cast<const uint8_t*>(g.W2) + ((size_t)nt_idx * KC + kc_begin) * A_BYTES : nullptr;
+  // weight tile of accumulator a: GeGLU pairs the gate and up tiles of the same channels, otherwise
+  // a CTA owns NA consecutive tiles
+  auto wtile = [&](int a) -> const uint8_t* {
+    const __nv_bfloat16* base = (geglu && a == 1) ? g.W2 : g.W;
+    const int tile = geglu ? nt_idx : nt_idx * NA + a;
+    return reinterpret_cast<const uint8_t*>(base) + ((size_t)tile * KC + kc_begin) * A_BYTES;
+  };
+
+  if (warp < NPROD) {
+    // ---------------- producers: copy number id = stage * NCOPY + piece goes to warp id % 8 --------------
+    if (lane == 0) {
       const uint8_t* xsrc =
           reinterpret_cast<const uint8_t*>(g.X) + ((size_t)kc_begin * g.rows_pad + (size_t)tt * NT) * 128;
-      for (int i = warp; i < nk; i += NPROD) {
+      for (int id = warp; id < nk * NCOPY; id += NPROD) {
+        const int i = id / NCOPY, c = id % NCOPY;
         const int s = i % STAGES;
         const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
         if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc)) break;  // stop issuing copies once aborted
         const uint32_t full = smem_u32(&bar_full[s]);
         const uint32_t dst = tiles + (uint32_t)s * STAGE_BYTES;
-        mbar_expect_tx(full, STAGE_BYTES);
-        bulk_g2s(dst, wsrc + (size_t)i * A_BYTES, A_BYTES, full);
-        if (DUAL) bulk_g2s(dst + A_BYTES, wsrc2 + (size_t)i * A_BYTES, A_BYTES, full);
-        bulk_g2s(dst + A_BYTES * (DUAL ? 2 : 1), xsrc + (size_t)i * g.rows_pad * 128, B_BYTES, full);
+        if (c < NA) {
+          mbar_expect_tx(full, A_BYTES);
+          bulk_g2s(dst + c * A_BYTES, wtile(c) + (size_t)i * A_BYTES, A_BYTES, full);
+        } else {
+          const int pc = c - NA;
+          mbar_expect_tx(full, B_PIECE);
+          bulk_g2s(dst + NA * A_BYTES + pc * B_PIECE, xsrc + (size_t)i * g.rows_pad * 128 + (size_t)pc * B_PIECE, B_PIECE,
+                   full);
+        }
       }
     }
-  } else if (warp == 4) {
+  } else if (warp == 8) {
     // ---------------- MMA issuer (whole warp in the loop, one elected lane issues) ---------------------
     for (int i = 0; i < nk; ++i) {
       const int s = i % STAGES;
@@ -107,14 +132,14 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
       const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
       const uint64_t da = make_desc(a0);
       const uint64_t da2 = make_desc(a0 + A_BYTES);
-      const uint64_t db = make_desc(a0 + A_BYTES * (DUAL ? 2 : 1));
+      const uint64_t db = make_desc(a0 + A_BYTES * NA);
       if (elect_one()) {
         if (ok) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
             const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
             umma_bf16(tmem_base, da + 2 * k, db + 2 * k, IDESC, acc);
-            if (DUAL) umma_bf16(tmem_base + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
+            if (NA == 2) umma_bf16(tmem_base + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
           }
         }
         umma_commit(smem_u32(&bar_empty[s]));  // frees the stage when the MMAs above have read it
@@ -125,21 +150,27 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
     __syncwarp();
   } else {
     // ---------------- epilogue: TMEM -> registers -> global --------------------------------------
-    const int q = warp & 3;
-    const int n = nt_idx * 128 + q * 32 + lane;  // this thread's output channel
+    const int ew = warp - 9;                      // 0..7
+    const int q = warp & 3, hf = ew >> 2;         // TMEM lane quarter, token-column half
+    const int et = ew * 32 + lane;                // 0..255
+    const int ch = q * 32 + lane;                 // row of the 128-row tile
     const bool ok = mbar_wait(smem_u32(&bar_accum), 0, wc);
     tc_fence_after();
-    const float sc = g.scale ? g.scale[n] : 1.0f;
-    const int n_out = (g.perm_dh && n < g.perm_end) ? qkv_packed_to_channel(n, g.perm_dh) : n;  // output column
     const int tok_base = tt * NT;
-    if (ok) {
-      if (!DUAL) {
+    constexpr int HALF = NT / 2;
+    const int c_begin = hf * HALF;
+    if (ok && !geglu) {
+#pragma unroll
+      for (int a = 0; a < NA; ++a) {
+        const int n = (nt_idx * NA + a) * 128 + ch;   // packed output channel
+        const float sc = g.scale ? g.scale[n] : 1.0f;
+        const int n_out = (g.perm_dh && n < g.perm_end) ? qkv_packed_to_channel(n, g.perm_dh) : n;
         const float gt = (g.epi == TC_RESID && g.gate) ? g.gate[n] : 1.0f;
         const float bs = (g.epi == TC_BIAS_ROWMAP && g.bias) ? g.bias[n] : 0.0f;
-        for (int c0 = 0; c0 < NT; c0 += 16) {
+        for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;  // warp-uniform
           float v[16];
-          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NT + c0), v);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int tok = tok_base + c0 + j;
@@ -148,7 +179,9 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
               if (g.epi == TC_STORE) {
                 g.out_f32[(size_t)tok * g.ldo + n_out] = val;
               } else if (g.epi == TC_RESID) {
-                atomicAdd(&g.out_f32[(size_t)tok * g.ldo + n], gt * val);
+                float* o = &g.out_f32[(size_t)tok * g.ldo + n];
+                if (gridDim.z == 1) *o = *o + gt * val;   // the element has a single owner: plain update
+                else atomicAdd(o, gt * val);
               } else {
                 const int orow = (tok / g.rows_in) * g.rows_out + g.row_off + tok % g.rows_in;
                 g.out_f32[(size_t)orow * g.ldo + n] = val + bs;
@@ -156,21 +189,37 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
             }
           }
         }
-      } else {
-        const float sc2 = g.scale2 ? g.scale2[n] : 1.0f;
-        for (int c0 = 0; c0 < NT; c0 += 16) {
+      }
+    }
+    if (geglu) {
+      // accumulator 0 = gate, 1 = up of channels nt_idx*128 .. +127.  The bf16 result is built in shared
+      // memory as the swizzled image of two k-chunks of the down projection's input (the stages are
+      // free: every MMA has completed), then copied out with 16-byte stores.
+      __nv_bfloat16* img = reinterpret_cast<__nv_bfloat16*>(tiles_ptr);   // [2][NT][64]
+      if (ok) {
+        const int n = nt_idx * 128 + ch;
+        const float sg = g.scale ? g.scale[n] : 1.0f, su = g.scale2 ? g.scale2[n] : 1.0f;
+        const int kc_sel = ch >> 6, c64 = ch & 63;
+        for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;
           float vg[16], vu[16];
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, vg);
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(NT + c0), vu);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const int tok = tok_base + c0 + j;
-            if (tok < g.M) {
-              const float val = gelu_f(vg[j] * sc, g.gelu_exact) * (vu[j] * sc2);
-              g.out_tiled[tiled_index(tok, n, g.rows_pad)] = __float2bfloat16_rn(val);
-            }
+            const int t = c0 + j;   // token within the tile
+            const float val = gelu_fast(vg[j] * sg, g.gelu_exact) * (vu[j] * su);
+            img[((size_t)kc_sel * NT + t) * 64 + (((c64 >> 3) ^ (t & 7)) << 3) + (c64 & 7)] = __float2bfloat16_rn(val);
           }
+        }
+      }
+      epi_sync();
+      if (ok) {
+        const int rows = min(NT, g.M - tok_base);
+        for (int kc_sel = 0; kc_sel < 2; ++kc_sel) {
+          uint4* dst = reinterpret_cast<uint4*>(g.out_tiled + ((size_t)(nt_idx * 2 + kc_sel) * g.rows_pad + tok_base) * 64);
+          const uint4* src = reinterpret_cast<const uint4*>(img + (size_t)kc_sel * NT * 64);
+          for (int idx = et; idx < rows * 8; idx += NEPI) dst[idx] = src[idx];
         }
       }
     }
@@ -182,48 +231,51 @@ __global__ void __launch_bounds__(288, 1) k_gemm_tc(int* status, const TcGemm g)
     // give any bulk copy still in flight time to land before shared memory is released
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, COLS);
+    tmem_dealloc(tmem_base, COLS < 32 ? 32 : COLS);
   }
 }
 
-template <int NT, bool DUAL, int STAGES>
+template <int NT, int NA, int STAGES>
 constexpr size_t smem_bytes() {
-  return (size_t)STAGES * (A_BYTES * (DUAL ? 2 : 1) + NT * 128) + 1024;
+  return (size_t)STAGES * (A_BYTES * NA + NT * 128) + 1024;
 }
 
-template <int NT, bool DUAL, int STAGES>
+template <int NT, int NA, int STAGES>
 cudaError_t launch_one(int* status, const TcGemm& g, cudaStream_t st) {
-  dim3 grid(g.N / 128, (g.M + NT - 1) / NT, g.splits > 0 ? g.splits : 1);
-  k_gemm_tc<NT, DUAL, STAGES><<<grid, 288, smem_bytes<NT, DUAL, STAGES>(), st>>>(status, g);
+  dim3 grid(g.N / 128 / (g.epi == TC_GEGLU ? 1 : NA), (g.M + NT - 1) / NT, g.splits > 0 ? g.splits : 1);
+  k_gemm_tc<NT, NA, STAGES><<<grid, 544, smem_bytes<NT, NA, STAGES>(), st>>>(status, g);
   return cudaGetLastError();
 }
 
-template <int NT, bool DUAL, int STAGES>
+template <int NT, int NA, int STAGES>
 cudaError_t setup_one() {
-  return cudaFuncSetAttribute(k_gemm_tc<NT, DUAL, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)smem_bytes<NT, DUAL, STAGES>());
+  return cudaFuncSetAttribute(k_gemm_tc<NT, NA, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)smem_bytes<NT, NA, STAGES>());
 }
 
 }  // namespace
 
 cudaError_t tc_gemm_setup() {
   cudaError_t e;
-  if ((e = setup_one<64, false, 6>()) != cudaSuccess) return e;
-  if ((e = setup_one<64, true, 4>()) != cudaSuccess) return e;
-  if ((e = setup_one<128, false, 5>()) != cudaSuccess) return e;
-  if ((e = setup_one<128, true, 4>()) != cudaSuccess) return e;
-  if ((e = setup_one<256, false, 4>()) != cudaSuccess) return e;
-  if ((e = setup_one<256, true, 3>()) != cudaSuccess) return e;
+  if ((e = setup_one<64, 1, 6>()) != cudaSuccess) return e;
+  if ((e = setup_one<64, 2, 4>()) != cudaSuccess) return e;
+  if ((e = setup_one<128, 1, 5>()) != cudaSuccess) return e;
+  if ((e = setup_one<128, 2, 4>()) != cudaSuccess) return e;
+  if ((e = setup_one<256, 1, 4>()) != cudaSuccess) return e;
+  if ((e = setup_one<256, 2, 3>()) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
+// GeGLU always pairs the gate and up tiles (NA = 2).  Other epilogues take two consecutive channel
+// tiles per CTA when the token tile is 256 wide and the channel count allows it (halves the
+// activation traffic per MMA), else one.
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st) {
-  const bool dual = g.epi == TC_GEGLU;
-  if (nt == 64) return dual ? launch_one<64, true, 4>(status, g, st) : launch_one<64, false, 6>(status, g, st);
-  if (nt == 128) return dual ? launch_one<128, true, 4>(status, g, st) : launch_one<128, false, 5>(status, g, st);
-  return dual ? launch_one<256, true, 3>(status, g, st) : launch_one<256, false, 4>(status, g, st);
+  const bool two = g.epi == TC_GEGLU || (nt == 256 && g.N % 256 == 0);
+  if (nt == 64) return two ? launch_one<64, 2, 4>(status, g, st) : launch_one<64, 1, 6>(status, g, st);
+  if (nt == 128) return two ? launch_one<128, 2, 4>(status, g, st) : launch_one<128, 1, 5>(status, g, st);
+  return two ? launch_one<256, 2, 3>(status, g, st) : launch_one<256, 1, 4>(status, g, st);
 }
 
 }  // namespace phyai
