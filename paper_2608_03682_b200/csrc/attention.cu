@@ -51,22 +51,22 @@ __global__ void k_attn_merge(const int* status, const float* part_o, const float
   }
 }
 
-template <int DH, int HPC>
+template <int DH, int HPC, int KTT>
 constexpr size_t attn_smem() {
-  return (size_t)(HPC * QROWS + 4 * KT) * DH * 2;
+  return (size_t)(HPC * QROWS + 4 * KTT) * DH * 2;
 }
 
-template <int DH, int HPC>
+template <int DH, int HPC, int KTT>
 cudaError_t launch_attn(const AttnArgs& a, int batch, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_attn_mma<DH, HPC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)attn_smem<DH, HPC>());
+    cudaError_t e = cudaFuncSetAttribute(k_attn_mma<DH, HPC, KTT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)attn_smem<DH, HPC, KTT>());
     if (e != cudaSuccess) return e;
     configured = true;
   }
   dim3 grid(a.num_splits, a.d.Hq / HPC, batch);
-  k_attn_mma<DH, HPC><<<grid, HPC * 128, attn_smem<DH, HPC>(), st>>>(a);
+  k_attn_mma<DH, HPC, KTT><<<grid, HPC * 128, attn_smem<DH, HPC, KTT>(), st>>>(a);
   if (a.num_splits > 1) {
     dim3 g2(a.d.S, a.d.Hq, batch);
     k_attn_merge<DH><<<g2, 128, 0, st>>>(a.status, a.part_o, a.part_ml, a.out, a.rows_pad, a.num_splits, a.d.S, a.d.Hq);
@@ -103,9 +103,10 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
   a.part_ml = scratch ? scratch + (size_t)batch * d.Hq * num_splits * QROWS * d.dh : nullptr;
   const int G = d.Hq / d.Hkv;
   const bool two = (G % 2 == 0) && (batch * d.Hq * num_splits >= 2 * 148);
-  if (d.dh == 256) return two ? launch_attn<256, 2>(a, batch, st) : launch_attn<256, 1>(a, batch, st);
-  if (d.dh == 128) return two ? launch_attn<128, 2>(a, batch, st) : launch_attn<128, 1>(a, batch, st);
-  return two ? launch_attn<64, 2>(a, batch, st) : launch_attn<64, 1>(a, batch, st);
+  // (one head per CTA with 32-key tiles, two CTAs per SM, was measured no faster than two heads per CTA)
+  if (d.dh == 256) return two ? launch_attn<256, 2, 64>(a, batch, st) : launch_attn<256, 1, 64>(a, batch, st);
+  if (d.dh == 128) return two ? launch_attn<128, 2, 64>(a, batch, st) : launch_attn<128, 1, 64>(a, batch, st);
+  return two ? launch_attn<64, 2, 64>(a, batch, st) : launch_attn<64, 1, 64>(a, batch, st);
 }
 
 }  // namespace phyai

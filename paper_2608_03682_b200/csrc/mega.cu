@@ -379,44 +379,62 @@ __global__ void __launch_bounds__(512, 1) k_mega(const __grid_constant__ MegaPar
       }
     } else if (warp == 8) {
       // ============ MMA issuer: the whole warp walks the program, one elected lane issues ==========================
+      // A single warp issues roughly one instruction every few clocks, so the per-k-chunk body is kept
+      // minimal: ring slot, parity and descriptors advance incrementally (no division), the weights of a
+      // whole 4-chunk group are awaited up front, and the 16 MMAs of a group are issued back to back.
       {
         ProgIter it(p, pl);
         Item im;
-        unsigned u = 0, g = 0;
-        unsigned uses0 = 0u, uses1 = 0u;   // chunk groups consumed from each slot
+        unsigned g = 0;
+        unsigned uses0 = 0u, uses1 = 0u;   // chunk groups consumed from each activation slot
+        unsigned ws = 0u, wph = 0u;        // weight ring slot and parity of the next unit
+        const uint64_t da0 = make_desc(ring);
+        const uint64_t db0 = make_desc(regA);
         while (it.next(im)) {
           if (!im.gemm) continue;
           bool ok = true;
           if (g > 0) ok = mbar_wait(smem_u32(&sh.acc_empty), (g - 1) & 1u, wc);  // epilogue drained TMEM
-          const int groups = (im.role.kc_count + 3) / 4;
+          const int groups = (im.role.kc_count + 3) >> 2;
+          uint32_t accum = 0u;
           for (int gidx = 0; gidx < groups; ++gidx) {
             const int sl = gidx & 1;
             ok = mbar_wait(smem_u32(&sh.act_full[sl]), (sl ? uses1 : uses0) & 1u, wc) && ok;
             if (sl) ++uses1; else ++uses0;
             if (gidx == 0 && lane == 0) stamp(p, im.phase, im.step, im.layer, 2, 0);
-            tc_fence_after();
-            const int j0 = gidx * 4, n = min(4, im.role.kc_count - j0);
-            bool okw = true;
-            for (int j = 0; j < n; ++j) okw = mbar_wait(smem_u32(&sh.w_full[(u + j) % RING]), ((u + j) / RING) & 1u, wc) && okw;
-            tc_fence_after();
-            for (int j = 0; j < n; ++j) {   // warp-uniform loop; one elected lane issues
-              const unsigned s = (u + j) % RING;
-              const uint64_t da = make_desc(ring + s * UNIT);
-              const uint64_t db = make_desc(regA + (uint32_t)sl * ACT_SLOT + (uint32_t)j * ACT_TILE);
-              const uint32_t first = (j0 + j > 0) ? 1u : 0u;
-              if (elect_one()) {
-                if (ok && okw) {
-                  umma_bf16(tmem_base, da, db, IDESC64, first);
-                  umma_bf16(tmem_base, da + 2, db + 2, IDESC64, 1u);
-                  umma_bf16(tmem_base, da + 4, db + 4, IDESC64, 1u);
-                  umma_bf16(tmem_base, da + 6, db + 6, IDESC64, 1u);
-                }
-                umma_commit(smem_u32(&sh.w_empty[s]));
-                if (j == n - 1) umma_commit(smem_u32(&sh.chunk_free[sl]));   // the slot may be refilled
+            const int n = min(4, im.role.kc_count - gidx * 4);
+            {   // all weight units of the group
+              unsigned s2 = ws, ph2 = wph;
+              for (int j = 0; j < n; ++j) {
+                ok = mbar_wait(smem_u32(&sh.w_full[s2]), ph2, wc) && ok;
+                if (++s2 == RING) s2 = 0, ph2 ^= 1u;
               }
-              __syncwarp();
             }
-            u += n;
+            tc_fence_after();
+            const uint64_t db = db0 + (uint64_t)((sl * ACT_SLOT) >> 4);
+            // a vote makes the condition provably warp-uniform, which keeps the descriptors below in
+            // uniform registers (a branch on a value the compiler cannot prove uniform costs ~2x per MMA)
+            if (__all_sync(0xffffffffu, ok)) {
+              for (int j = 0; j < n; ++j) {
+                const uint64_t da = da0 + (uint64_t)((ws * UNIT) >> 4);
+                const uint64_t dbj = db + (uint64_t)((j * ACT_TILE) >> 4);
+                if (elect_one()) {
+                  umma_bf16(tmem_base, da, dbj, IDESC64, accum);
+                  umma_bf16(tmem_base, da + 2, dbj + 2, IDESC64, 1u);
+                  umma_bf16(tmem_base, da + 4, dbj + 4, IDESC64, 1u);
+                  umma_bf16(tmem_base, da + 6, dbj + 6, IDESC64, 1u);
+                  umma_commit(smem_u32(&sh.w_empty[ws]));
+                }
+                accum = 1u;
+                if (++ws == RING) ws = 0, wph ^= 1u;
+              }
+            } else {
+              for (int j = 0; j < n; ++j) {   // aborted: keep the ring protocol moving without issuing MMAs
+                if (elect_one()) umma_commit(smem_u32(&sh.w_empty[ws]));
+                if (++ws == RING) ws = 0, wph ^= 1u;
+              }
+            }
+            if (elect_one()) umma_commit(smem_u32(&sh.chunk_free[sl]));   // the slot may be refilled
+            __syncwarp();
           }
           if (lane == 0) stamp(p, im.phase, im.step, im.layer, 3, 0);
           if (elect_one()) umma_commit(smem_u32(&sh.acc_full));
