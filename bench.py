@@ -33,6 +33,9 @@ from paper_2608_03682_b200 import synth  # noqa: E402
 METRIC = "ms per action chunk (batch 1, 10 steps)"
 METRIC_BATCHED = "chunks/sec at batch %d"
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (bench.py cannot run ncu itself)
+NCU_TRAFFIC = {"C2": (6.433488e9 + 69.605376e6, "profiles/persistent_kernel_c2_batch1.md")}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 
 
@@ -256,11 +259,12 @@ def main():
             ex.denoise_host(kv_p, lens[0], None if states_p is None else states_p[0], noise_p[0], n_steps, out_p[0],
                             stream=stream)
 
+    from paper_2608_03682_b200 import replicas
+
     def barrier():
         torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier()
+        torch.cuda.synchronize()
 
     def timed(fn, iters):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -270,12 +274,7 @@ def main():
             fn()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return replicas.max_over_ranks(e0.elapsed_time(e1), device="cuda")
 
     for _ in range(Wm):
         call_device()
@@ -307,11 +306,14 @@ def main():
     alg_bytes, alg_flops = algorithmic_cost(cfg, lens, n_steps)
     secs = ms_per_step / 1e3
     hbm_bound = not batched or batch < 8
+    persistent = batch * cfg.suffix_len <= 64 and cfg.dtype != "f32"
+    traffic = NCU_TRAFFIC.get(args.workload, (None, None))
     if hbm_bound:
         achieved = alg_bytes / secs / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                    "kernel": "whole captured loop (one graph launch = one chunk)",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": traffic[0], "traffic_source": traffic[1],
+                    "kernel": ("k_mega: persistent kernel, one launch = one chunk (all Euler steps and layers)"
+                               if persistent else "whole captured loop (one graph launch = one chunk)"),
                     "peak_source": f"{peaks['source']} copy bandwidth", "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
                     "algorithmic_bytes_per_launch": alg_bytes}
     else:

@@ -1,0 +1,51 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times, on sampled
+requests the oracle can compute one by one: the ragged batch-64 workload and the e4m3-weight sweep."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import expert_oracle as O
+from paper_2608_03682_b200 import binding, synth
+from tests.helpers import BAR, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_batched(cfg, cfg_id, W, lens, n_steps, check):
+    kvs = [synth.make_prefix_kv(cfg, cfg_id, int(p), b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    B = len(lens)
+    states = torch.stack([synth.make_state(cfg, cfg_id, b) for b in range(B)])
+    noise = torch.stack([synth.make_noise(cfg, cfg_id, b) for b in range(B)])
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        out = ex.denoise_batched(packed.cuda(), torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), n_steps)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        out = out.double().cpu().numpy()
+    assert np.isfinite(out).all()
+    Wf = O.Weights(W)
+    errs = {}
+    for b in check:
+        ref = O.denoise(cfg, Wf, kvs[b], int(lens[b]), states[b], noise[b], n_steps)
+        errs[b] = rel_err(out[b], ref)
+    return errs
+
+
+def test_batch64_ragged_rollout_matches_oracle_on_sampled_requests():
+    cfg = synth.pi0_config(max_batch=64)
+    lens = synth.make_ragged_lengths(4, 64, 600, 968)
+    order = np.argsort(lens)
+    check = sorted({0, 63, int(order[0]), int(order[-1])})
+    errs = _run_batched(cfg, 4, synth.make_weights(cfg, 4), lens, 10, check)
+    print("C4 max rel err per sampled request:", {b: f"{e:.2e}" for b, e in errs.items()})
+    assert max(errs.values()) <= BAR["bf16"], errs
+
+
+@pytest.mark.parametrize("batch", [1, 8])
+def test_e4m3_weight_expert_matches_oracle(batch):
+    cfg = synth.pi0_config(max_batch=batch, dtype="w8e4m3", max_prefix_len=816)
+    W = synth.make_weights(cfg, 5)
+    check = [0] if batch == 1 else [0, batch - 1]
+    errs = _run_batched(cfg, 5, W, [816] * batch, 10, check)
+    print(f"C5 batch {batch} max rel err:", {b: f"{e:.2e}" for b, e in errs.items()})
+    assert max(errs.values()) <= BAR["w8e4m3"], errs
