@@ -291,9 +291,44 @@ __global__ void k_rmsnorm(const int* status, const float* h, const float* gain, 
     out.store(row, d, v);
   }
 }
+// Vectorised variant for the tensor path: D a multiple of 128, tiled bf16 output, one warp per row,
+// float4 loads and 8-byte stores.
+__global__ void k_rmsnorm_tiled4(const int* status, const float* h, const float* gain, const float* shift,
+                                 __nv_bfloat16* out, int rows_pad, int M, int D, float eps) {
+  if (status_set(status)) return;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const float* x = h + (size_t)row * D;
+  float ss = 0.f;
+  for (int d = lane * 4; d < D; d += 128) {
+    const float4 v = *reinterpret_cast<const float4*>(x + d);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = warp_sum(ss);
+  const float r = 1.0f / sqrtf(ss / (float)D + eps);
+  for (int d = lane * 4; d < D; d += 128) {
+    const float4 v = *reinterpret_cast<const float4*>(x + d);
+    const float4 g = *reinterpret_cast<const float4*>(gain + d);
+    float4 o = make_float4(v.x * r * g.x, v.y * r * g.y, v.z * r * g.z, v.w * r * g.w);
+    if (shift) {
+      const float4 s4 = *reinterpret_cast<const float4*>(shift + d);
+      o.x += s4.x, o.y += s4.y, o.z += s4.z, o.w += s4.w;
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(out + tiled_index(row, d, rows_pad)) = pk;
+  }
+}
+
 void launch_rmsnorm(const int* status, const float* h, const float* gain, const float* shift, float* out_f32,
                     __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st) {
   const int blocks = (M + 3) / 4;
+  if (out_tiled && D % 128 == 0) {
+    k_rmsnorm_tiled4<<<blocks, 128, 0, st>>>(status, h, gain, shift, out_tiled, rows_pad, M, D, eps);
+    return;
+  }
   if (out_tiled)
     k_rmsnorm<<<blocks, 128, 0, st>>>(status, h, gain, shift, TiledBf16{out_tiled, rows_pad}, M, D, eps);
   else
@@ -303,41 +338,56 @@ void launch_rmsnorm(const int* status, const float* h, const float* gain, const 
 // =============================================================================================
 // final norm -> out-projection -> Euler update (epilogue): x += dt * (n . Wout + bout)
 // =============================================================================================
-__global__ void k_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
-                        const float* Wout, const float* bout, float dt, int A, int H, int D, int S, int ns, float eps) {
+// One block normalises FR action rows into shared memory, then thread (a, row) walks D once: every
+// element of Wout is read once per block and used for all its rows.
+constexpr int FR = 8;
+__global__ void __launch_bounds__(256) k_final(const Request* rq, const int* status, const float* h, const float* gain,
+                                               const float* shift, const float* Wout, const float* bout, float dt, int A,
+                                               int H, int D, int S, int ns, float eps, int rows_total) {
   if (status_set(status)) return;
-  extern __shared__ float nrm[];  // D floats + 1
-  __shared__ float red[32];
-  const int r = blockIdx.x;  // action row
-  const int b = r / H, i = r % H;
-  const float* x = h + (size_t)(b * S + ns + i) * D;
-  float ss = 0.f;
-  for (int d = threadIdx.x; d < D; d += blockDim.x) ss = fmaf(x[d], x[d], ss);
-  ss = warp_sum(ss);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-  if (lane == 0) red[warp] = ss;
-  __syncthreads();
-  float tot = 0.f;
-  for (int w = 0; w < nw; ++w) tot += red[w];
-  const float rr = 1.0f / sqrtf(tot / (float)D + eps);
-  for (int d = threadIdx.x; d < D; d += blockDim.x) {
-    float v = x[d] * rr * gain[d];
-    if (shift) v += shift[d];
-    nrm[d] = v;
+  extern __shared__ float nrm[];  // FR x D
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r0 = blockIdx.x * FR;
+  // one warp per row: norm
+  {
+    const int r = r0 + warp;
+    if (r < rows_total) {
+      const int b = r / H, i = r % H;
+      const float* x = h + (size_t)(b * S + ns + i) * D;
+      float ss = 0.f;
+      for (int d = lane; d < D; d += 32) ss = fmaf(x[d], x[d], ss);
+      ss = warp_sum(ss);
+      const float rr = 1.0f / sqrtf(ss / (float)D + eps);
+      for (int d = lane; d < D; d += 32) {
+        float v = x[d] * rr * gain[d];
+        if (shift) v += shift[d];
+        nrm[warp * D + d] = v;
+      }
+    }
   }
   __syncthreads();
+  // outputs: warp w owns row r0 + w; lanes own action channels a = lane, lane + 32, ...
+  const int r = r0 + warp;
+  if (r >= rows_total) return;
   float* xo = rq->x + (size_t)r * A;
-  for (int a = warp; a < A; a += nw) {
+  const float* n = nrm + warp * D;
+  for (int a = lane; a < A; a += 32) {
     float acc = 0.f;
-    for (int d = lane; d < D; d += 32) acc = fmaf(nrm[d], Wout[(size_t)d * A + a], acc);
-    acc = warp_sum(acc);
-    if (lane == 0) xo[a] = xo[a] + dt * (acc + bout[a]);
+#pragma unroll 8
+    for (int d = 0; d < D; ++d) acc = fmaf(n[d], Wout[(size_t)d * A + a], acc);
+    xo[a] = xo[a] + dt * (acc + bout[a]);
   }
 }
 void launch_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
                   const float* Wout, const float* bout, float dt, const Dims& d, int batch, cudaStream_t st) {
-  k_final<<<batch * d.H, 256, d.D * sizeof(float), st>>>(rq, status, h, gain, shift, Wout, bout, dt, d.A, d.H, d.D, d.S,
-                                                         d.ns, d.eps);
+  const int rows = batch * d.H;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(k_final, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    configured = true;
+  }
+  k_final<<<(rows + FR - 1) / FR, 256, (size_t)FR * d.D * sizeof(float), st>>>(rq, status, h, gain, shift, Wout, bout, dt,
+                                                                               d.A, d.H, d.D, d.S, d.ns, d.eps, rows);
 }
 
 // =============================================================================================
