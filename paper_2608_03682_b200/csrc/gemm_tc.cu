@@ -16,11 +16,12 @@
 // k-step moves 64 KB for 8 MMAs of 128 clocks, i.e. 64 bytes per clock, which is what one SM's L2 port
 // delivers (~126 GB/s measured); a single 128 x 256 tile would need 96 bytes per clock.
 //
-// Warp roles (544 threads): warps 0..7 = copy producers (the copies of all stages are dealt round
+// Warp roles (800 threads): warps 0..7 = copy producers (the copies of all stages are dealt round
 // robin to the eight warps: one warp's bulk copies complete one at a time, about 0.5 us each whatever
 // their size, so many issuing warps are needed to keep the SM's L2 port busy), warp 8 = TMEM owner +
-// MMA issuer (whole warp in the loop, one elected lane issues), warps 9..16 = epilogue (TMEM lane
-// quarter = warp % 4, token-column half = (warp - 9) / 4).
+// MMA issuer (whole warp in the loop, one elected lane issues), warps 9..24 = epilogue (TMEM lane
+// quarter = warp % 4, token-column quarter = (warp - 9) / 4).  The epilogue of a 256 x 256 tile is not
+// overlapped with a next tile (TMEM is full), so it gets 16 warps and batches its global loads.
 // Every wait is bounded: on expiry the CTA raises the status word, stops issuing copies, and
 // drains to its normal exit (TMEM is always released).
 #include "kernels.h"
@@ -32,13 +33,13 @@ namespace {
 
 constexpr int A_BYTES = 128 * 128;  // one weight block: 128 out channels x 64 k (bf16)
 constexpr int NPROD = 8;
-constexpr int NEPI = 256;           // epilogue threads
+constexpr int NEPI = 512;           // epilogue threads (16 warps)
 constexpr int BAR_EPI = 1;
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync %0, %1;" ::"n"(BAR_EPI), "n"(NEPI) : "memory"); }
 
 template <int NT, int NA, int STAGES>
-__global__ void __launch_bounds__(544, 1) k_gemm_tc(int* status, const TcGemm g) {
+__global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g) {
   constexpr int B_BYTES = NT * 128;
   constexpr int NB = NT > 128 ? NT / 128 : 1;          // the activation tile is copied in pieces of <= 16 KB
   constexpr int B_PIECE = B_BYTES / NB;
@@ -150,14 +151,14 @@ __global__ void __launch_bounds__(544, 1) k_gemm_tc(int* status, const TcGemm g)
     __syncwarp();
   } else {
     // ---------------- epilogue: TMEM -> registers -> global --------------------------------------
-    const int ew = warp - 9;                      // 0..7
-    const int q = warp & 3, hf = ew >> 2;         // TMEM lane quarter, token-column half
-    const int et = ew * 32 + lane;                // 0..255
+    const int ew = warp - 9;                      // 0..15
+    const int q = warp & 3, hf = ew >> 2;         // TMEM lane quarter, token-column quarter
+    const int et = ew * 32 + lane;                // 0..511
     const int ch = q * 32 + lane;                 // row of the 128-row tile
     const bool ok = mbar_wait(smem_u32(&bar_accum), 0, wc);
     tc_fence_after();
     const int tok_base = tt * NT;
-    constexpr int HALF = NT / 2;
+    constexpr int HALF = NT / 4;   // token columns per epilogue warp
     const int c_begin = hf * HALF;
     if (ok && !geglu) {
 #pragma unroll
@@ -171,6 +172,21 @@ __global__ void __launch_bounds__(544, 1) k_gemm_tc(int* status, const TcGemm g)
           if (tok_base + c0 >= g.M) break;  // warp-uniform
           float v[16];
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NT + c0), v);
+          if (g.epi == TC_RESID && gridDim.z == 1) {
+            // single owner per element: plain read-modify-write, with the 16 loads issued before any is used
+            float old[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int tok = tok_base + c0 + j;
+              old[j] = tok < g.M ? g.out_f32[(size_t)tok * g.ldo + n] : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int tok = tok_base + c0 + j;
+              if (tok < g.M) g.out_f32[(size_t)tok * g.ldo + n] = old[j] + gt * (v[j] * sc);
+            }
+            continue;
+          }
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int tok = tok_base + c0 + j;
@@ -179,9 +195,7 @@ __global__ void __launch_bounds__(544, 1) k_gemm_tc(int* status, const TcGemm g)
               if (g.epi == TC_STORE) {
                 g.out_f32[(size_t)tok * g.ldo + n_out] = val;
               } else if (g.epi == TC_RESID) {
-                float* o = &g.out_f32[(size_t)tok * g.ldo + n];
-                if (gridDim.z == 1) *o = *o + gt * val;   // the element has a single owner: plain update
-                else atomicAdd(o, gt * val);
+                atomicAdd(&g.out_f32[(size_t)tok * g.ldo + n], gt * val);
               } else {
                 const int orow = (tok / g.rows_in) * g.rows_out + g.row_off + tok % g.rows_in;
                 g.out_f32[(size_t)orow * g.ldo + n] = val + bs;
@@ -245,7 +259,7 @@ constexpr size_t smem_bytes() {
 template <int NT, int NA, int STAGES>
 cudaError_t launch_one(int* status, const TcGemm& g, cudaStream_t st) {
   dim3 grid(g.N / 128 / (g.epi == TC_GEGLU ? 1 : NA), (g.M + NT - 1) / NT, g.splits > 0 ? g.splits : 1);
-  k_gemm_tc<NT, NA, STAGES><<<grid, 544, smem_bytes<NT, NA, STAGES>(), st>>>(status, g);
+  k_gemm_tc<NT, NA, STAGES><<<grid, 800, smem_bytes<NT, NA, STAGES>(), st>>>(status, g);
   return cudaGetLastError();
 }
 
