@@ -194,7 +194,8 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
 /* Options. key "use_graph": 0 launches the kernels directly, 1 (default) replays a captured CUDA
  * graph per (batch, n_steps).  key "use_persistent": 1 (default) runs calls with batch * suffix_len
  * <= 64 tokens as one persistent cooperative kernel (the whole n-step loop, no kernel boundaries),
- * 0 uses the per-operator kernels for every batch.  key "wait_limit": iteration bound of
+ * 0 uses the per-operator kernels for every batch.  key "use_tc_attention": 1 (default) lets large
+ * batches use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "wait_limit": iteration bound of
  * device-side waits (testing).  Unknown key -> INVALID_ARG. */
 phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t value);
 

@@ -85,6 +85,7 @@ struct phyai_expert {
   // persistent loop kernel (batch * suffix_len <= 64)
   bool mega_ok = false;
   int use_mega = 1;
+  int use_tc_attention = 1;
   int n_sm = 0;
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
@@ -340,7 +341,12 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         g.out = h->qkv, g.ldo = d.Nqkv;
         simt_gemm(g);
       }
-      if (h->attn_mma) {
+      if (h->attn_mma && h->use_tc_attention && attention_tc_supported(d) && batch * (d.Hq / 2) >= 100) {
+        cudaError_t e = launch_attention_tc(h->rq, h->status, h->qkv, h->rope, l, h->attn_t, h->Mpad, d, batch,
+                                            h->wait_limit, st);
+        if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
+        ++cnt;
+      } else if (h->attn_mma) {
         const int splits = attention_pick_splits(d, batch, (int)h->cfg.max_prefix_len);
         cudaError_t e = launch_attention_mma(h->rq, h->status, h->qkv, h->rope, l, h->attn_t, h->Mpad, splits,
                                              h->attn_scratch, d, batch, h->wait_limit, st);
@@ -845,6 +851,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     unsigned long long* buf = nullptr;
     ST(h->alloc(&buf, (size_t)148 * MP_COUNT * 4, true));
     h->mega_trace = buf, h->trace_step = (int)(value / 1000), h->trace_layer = (int)(value % 1000);
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_tc_attention")) {
+    h->use_tc_attention = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
     return PHYAI_OK;
   }
   if (!strcmp(key, "use_persistent")) {

@@ -85,6 +85,12 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
                                  __nv_bfloat16* out_tiled, int rows_pad, int num_splits, float* scratch, const Dims& d,
                                  int batch, unsigned wait_limit, cudaStream_t st);
 
+// ---- tcgen05 attention (large batches: two heads per CTA, whole key range, no split) ------------------
+bool attention_tc_supported(const Dims& d);
+cudaError_t launch_attention_tc(const Request* rq, int* status, const float* qkv, const float2* rope, int layer,
+                                __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
+                                cudaStream_t st);
+
 // ---- tcgen05 GEMM ------------------------------------------------------------------------------
 enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3 };
 struct TcGemm {

@@ -168,3 +168,31 @@ def test_persistent_kernel_and_per_operator_kernels_agree(cond):
         for b in range(4):
             for mode in (1, 0):
                 assert rel_err(outs[mode][b], refs[b]) <= BAR["bf16"], (mode, b, rel_err(outs[mode][b], refs[b]))
+
+
+def test_large_batch_tcgen05_attention_matches_oracle_and_the_mma_sync_kernel():
+    """head_dim 256 and >= 100 head-pair CTAs select the tcgen05 attention kernel; ragged prefixes with
+    empty, sub-tile, exact-tile and multi-tile lengths."""
+    cfg = small_bf16_config("pi0", head_dim=256, max_batch=104, max_prefix_len=200)
+    lens = synth.make_ragged_lengths(17, 104, 0, 200)
+    lens[:6] = [0, 1, 63, 64, 65, 200]
+    W = synth.make_weights(cfg, 17, std=0.05)
+    kvs = [synth.make_prefix_kv(cfg, 17, int(p), b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    states = torch.stack([synth.make_state(cfg, 17, b) for b in range(104)])
+    noise = torch.stack([synth.make_noise(cfg, 17, b) for b in range(104)])
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        args = (packed.cuda(), torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), 2)
+        tc = ex.denoise_batched(*args).double().cpu().numpy()
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        ex.set_option("use_tc_attention", 0)
+        legacy = ex.denoise_batched(*args).double().cpu().numpy()
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+    assert np.isfinite(tc).all()
+    Wf = O.Weights(W)
+    for b in (0, 1, 2, 3, 4, 5, 50, 103):
+        ref = O.denoise(cfg, Wf, kvs[b], int(lens[b]), states[b], noise[b], 2)
+        assert rel_err(tc[b], ref) <= BAR["bf16"], (b, rel_err(tc[b], ref))
+        assert rel_err(legacy[b], ref) <= BAR["bf16"], (b, rel_err(legacy[b], ref))
