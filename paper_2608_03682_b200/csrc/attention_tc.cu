@@ -2,17 +2,19 @@
 //
 // One CTA takes the suffix rows of two query heads that share a kv head (2 x 64 padded rows = the 128
 // rows of one MMA) and walks all key tiles of its request:
-//   S = Q K^T      tcgen05.mma, M = 128, N = 64 keys, K = head_dim, fp32 accumulator in TMEM
+//   S = Q K^T      tcgen05.mma, M = 128, N = 64 keys, K = head_dim, fp32 accumulator in TMEM (two buffers)
 //   softmax        one thread per row reads its S row from TMEM (no shuffles), online max / sum in the
 //                  log2 domain, writes P (bf16) to shared memory as the next MMA's A operand
 //   O += P V       tcgen05.mma, M = 128, N = head_dim, K = 64 keys, accumulator stays in TMEM; V is used
 //                  as an MN-major B operand, so K and V tiles share one shared-memory layout and loader
-// K/V tiles (64 keys) are double buffered and staged with 16-byte cp.async into the 128-byte-swizzled
-// block layout the MMA descriptors expect.  The O accumulator is rescaled only when a row's running
+// K/V tiles (64 keys) and P are double buffered; K and V are staged by separate warps with 16-byte cp.async
+// into the 128-byte-swizzled block layout the MMA descriptors expect, one tile ahead of their consumer.
+// The suffix keys are tile 0 (built from the fp32 q/k/v by every thread while the first prefix tile is in
+// flight); the prefix tiles follow.  The O accumulator is rescaled only when a row's running
 // maximum grows by more than 2^8 (otherwise the old maximum is kept, which is exact algebra and costs
 // nothing), so the TMEM round trip of the correction is rare.
 //
-// Warps: 0-3 load K/V (and build Q and the suffix tile), 4 issues the MMAs (whole warp in the loop, one
+// Warps: 0-1 load K, 2-3 load V, 4 issues the MMAs (whole warp in the loop, one
 // elected lane issues), 5-8 softmax / correction / output (TMEM lane quarter = warp % 4).
 // All waits are bounded; on expiry the CTA raises the status word and drains.
 #include "attention.cuh"
@@ -22,8 +24,8 @@ namespace phyai {
 namespace {
 
 constexpr int KTC = 64;          // keys per tile
-constexpr int BAR_LOAD = 1;      // named barrier of the 4 loader warps
-constexpr int BAR_SOFT = 2;      // named barrier of the 4 softmax warps
+constexpr int BAR_LOAD = 1;      // named barrier of the 2 K loader warps
+constexpr int BAR_SOFT = 2;      // named barrier of the 4 softmax warps (3 = the V loader warps)
 constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units
 
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
@@ -37,6 +39,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ float ex2_fast(float x) {   // 2^x, x <= a few units; -inf -> 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -54,18 +61,18 @@ __device__ __forceinline__ uint64_t make_desc_mn(uint32_t saddr, uint32_t lbo, u
 
 template <int DH>
 __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
-  constexpr int NB = DH / 64;                 // 64-element blocks along head_dim
-  constexpr int Q_BYTES = 128 * DH * 2;       // NB blocks of [128 rows x 128 B]
-  constexpr int KV_BYTES = KTC * DH * 2;      // NB blocks of [64 keys x 128 B]
+  constexpr int Q_BYTES = 128 * DH * 2;       // DH/64 blocks of [128 rows x 128 B]
+  constexpr int KV_BYTES = KTC * DH * 2;      // DH/64 blocks of [64 keys x 128 B]
   constexpr int KV_BLOCK = KTC * 128;
   constexpr int P_BYTES = 128 * KTC * 2;      // one block [128 rows x 64 keys]
-  constexpr int COLS = 512;                   // S at columns [0, 64), O at [64, 64 + DH)
+  constexpr int COLS = 512;                   // S (two buffers) at columns [0, 128), O at [128, 128 + DH)
+  constexpr int half = DH / 2;
   constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KTC >> 3) << 17) | ((128u >> 4) << 24);
   constexpr uint32_t IDESC_PV =
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((128u >> 4) << 24);
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t kv_full[2], kv_free[2], s_full, s_free, p_full, pv_done;
+  __shared__ __align__(8) uint64_t k_full[2], v_full[2], p_full[2], pv_done[2], s_full[2], s_free[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, skip_flag;
 
@@ -84,13 +91,13 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     skip_flag = status_set(a.status) ? 1 : 0;
     abort_flag = 0;
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&kv_full[i]), 1);
-      mbar_init(smem_u32(&kv_free[i]), 1);
+      mbar_init(smem_u32(&k_full[i]), 1);
+      mbar_init(smem_u32(&v_full[i]), 1);
+      mbar_init(smem_u32(&p_full[i]), 1);
+      mbar_init(smem_u32(&pv_done[i]), 1);
+      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&s_free[i]), 1);
     }
-    mbar_init(smem_u32(&s_full), 1);
-    mbar_init(smem_u32(&s_free), 1);
-    mbar_init(smem_u32(&p_full), 1);
-    mbar_init(smem_u32(&pv_done), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -99,144 +106,158 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     tmem_alloc(smem_u32(&tmem_slot), COLS);
     tc_fence_before();
   }
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + KTC;
   const WaitCtx wc{a.status, &abort_flag, a.wait_limit};
 
   const Request r = *a.rq;
   const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
   const int Tp = (P + KTC - 1) / KTC;
-  const int T = Tp + 1;                       // the suffix (<= 64 keys) is the last tile
-  constexpr int half = DH / 2;
+  // Tile 0 is the suffix (this request's own <= 64 keys, built below while the first prefix tile is in
+  // flight); tile t >= 1 is prefix keys [(t-1) * 64, t * 64).  Softmax does not care about the order.
+  const int T = Tp + 1;
+
+  // ---- loader state (warps 0-3): warps 0-1 stream K tiles, warps 2-3 stream V tiles -----------------
+  const bool is_v = warp >= 2;
+  const int lt2 = tid & 63;                  // thread within its stream
+  const int lc = lt2 & 31, r0 = lt2 >> 5;    // 16-byte chunk column; rows r0, r0 + 2, ...
+  const size_t kv_stride = (size_t)d.Hkv * DH * 2;
+  const uint8_t* G = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
+                     (((size_t)(a.layer * 2 + (is_v ? 1 : 0)) * r.kv_tokens + p0) * d.Hkv + hk) * (DH * 2) + (size_t)lc * 16;
+  const uint32_t tile_base = (is_v ? Vs : Ks) + (uint32_t)(lc >> 3) * KV_BLOCK;
+  auto issue = [&](int t) {                  // t >= 1
+    const uint32_t tb = tile_base + (uint32_t)(t & 1) * KV_BYTES;
+    const int rows = min(KTC, P - (t - 1) * KTC);
+    const uint8_t* g0 = G + (size_t)(t - 1) * KTC * kv_stride;
+#pragma unroll 8
+    for (int row = r0; row < KTC; row += 2) {
+      const bool ok = row < rows;            // rows past the prefix are zero-filled
+      cp_async16(tb + (uint32_t)row * 128 + (uint32_t)(((lc & 7) ^ (row & 7)) << 4), g0 + (size_t)(ok ? row : 0) * kv_stride,
+                 ok ? 16u : 0u);
+    }
+    cp_async_commit();
+  };
+  if (warp < 4 && T > 1) issue(1);
+
+  // ---- every thread: Q (rotated, scaled) and the suffix K (rotated) / V tile, rounded to bf16 -------
+  // Items [0, 128 * J4) are Q (row, 4-column group), the next 64 * J4 the suffix K tile, the last 64 * J4
+  // the suffix V tile.  Each thread first issues the loads of four items (always from valid addresses, so
+  // nothing is predicated), then rotates and stores them: the global-load latency is paid once per four.
+  {
+    constexpr int J4 = half / 4;              // float4 pairs per row
+    constexpr int NQ = 128 * J4, NK = KTC * J4, NALL = NQ + 2 * NK;
+    const float qscale = rsqrtf((float)DH);
+    const bool rot_any = a.rope != nullptr;
+    const float* kv_src = a.qkv + d.Nq + (size_t)hk * DH;
+    for (int base0 = tid; base0 < NALL; base0 += 288 * 4) {
+      float4 lo[4], hi[4], cs0[4], cs1[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int idx = min(base0 + u * 288, NALL - 1);
+        const int isq = idx < NQ, k = idx - NQ, isv = k >= NK;
+        const int row = isq ? idx / J4 : (k - isv * NK) / J4, j = (idx % J4) * 4;
+        const int i = min(isq ? (row & 63) : row, S - 1);
+        const float* src = a.qkv + (size_t)(b * S + i) * d.Nqkv +
+                           (isq ? (size_t)(head0 + (row >> 6)) * DH : (size_t)(d.Nq + hk * DH + isv * d.Hkv * DH));
+        lo[u] = __ldg(reinterpret_cast<const float4*>(src + j));
+        hi[u] = __ldg(reinterpret_cast<const float4*>(src + j + half));
+        if (rot_any) {
+          cs0[u] = __ldg(reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j));
+          cs1[u] = __ldg(reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j + 2));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int idx = base0 + u * 288;
+        if (idx >= NALL) break;
+        const int isq = idx < NQ, k = idx - NQ, isv = k >= NK;
+        const int row = isq ? idx / J4 : (k - isv * NK) / J4, j = (idx % J4) * 4;
+        float4 l4 = lo[u], h4 = hi[u];
+        if (rot_any && !isv) {
+          const float4 c0 = cs0[u], c1 = cs1[u];
+          const float4 l2 = make_float4(l4.x * c0.x - h4.x * c0.y, l4.y * c0.z - h4.y * c0.w, l4.z * c1.x - h4.z * c1.y,
+                                        l4.w * c1.z - h4.w * c1.w);
+          h4 = make_float4(h4.x * c0.x + l4.x * c0.y, h4.y * c0.z + l4.y * c0.w, h4.z * c1.x + l4.z * c1.y,
+                           h4.w * c1.z + l4.w * c1.w);
+          l4 = l2;
+        }
+        const float sc = (isq ? (row & 63) : row) < S ? (isq ? qscale : 1.0f) : 0.0f;   // padding rows are zero
+        const uint32_t tile = isq ? Qs : (isv ? Vs : Ks), blk = isq ? 128 * 128 : KV_BLOCK;
+        auto put = [&](int col, float4 v) {       // 4 consecutive columns of `row`
+          const uint32_t addr = tile + (uint32_t)(col >> 6) * blk + (uint32_t)row * 128 +
+                                (uint32_t)((((col & 63) >> 3) ^ (row & 7)) << 4) + (uint32_t)(col & 7) * 2;
+          asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(addr), "r"(pack_bf16(v.x * sc, v.y * sc)),
+                       "r"(pack_bf16(v.z * sc, v.w * sc)));
+        };
+        put(j, l4);
+        put(j + half, h4);
+      }
+    }
+  }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * KTC;
+  if (tid == 0) {                             // tile 0 is in place
+    mbar_arrive_local(smem_u32(&k_full[0]));
+    mbar_arrive_local(smem_u32(&v_full[0]));
+  }
 
   if (warp < 4) {
     // =========================== loaders ==========================================================
-    const int lt = tid;   // 0..127
-    const uint8_t* Kg = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
-                        (((size_t)(a.layer * 2 + 0) * r.kv_tokens + p0) * d.Hkv + hk) * (DH * 2);
-    const uint8_t* Vg = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
-                        (((size_t)(a.layer * 2 + 1) * r.kv_tokens + p0) * d.Hkv + hk) * (DH * 2);
-    const size_t kv_stride = (size_t)d.Hkv * DH * 2;
-    // ---- Q: rotate, scale, round to bf16 into the [block][row][128 B] swizzled image ----
-    const float qscale = rsqrtf((float)DH);
-    for (int idx = lt; idx < 128 * (half / 4); idx += 128) {
-      const int row = idx / (half / 4), j = (idx % (half / 4)) * 4;   // row = head_local * 64 + i
-      const int hl = row >> 6, i = row & 63;
-      float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-      if (i < S) {
-        const float* q = a.qkv + (size_t)(b * S + i) * d.Nqkv + (size_t)(head0 + hl) * DH;
-        lo = *reinterpret_cast<const float4*>(q + j);
-        hi = *reinterpret_cast<const float4*>(q + j + half);
-        if (a.rope) {
-          const float4 cs0 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j);
-          const float4 cs1 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j + 2);
-          const float4 l2 = make_float4(lo.x * cs0.x - hi.x * cs0.y, lo.y * cs0.z - hi.y * cs0.w,
-                                        lo.z * cs1.x - hi.z * cs1.y, lo.w * cs1.z - hi.w * cs1.w);
-          hi = make_float4(hi.x * cs0.x + lo.x * cs0.y, hi.y * cs0.z + lo.y * cs0.w, hi.z * cs1.x + lo.z * cs1.y,
-                           hi.w * cs1.z + lo.w * cs1.w);
-          lo = l2;
-        }
-      }
-      auto put = [&](int col, float4 v) {   // 4 consecutive columns of `row`
-        const int blk = col >> 6, c = (col & 63) >> 3;
-        const uint32_t addr = Qs + (uint32_t)blk * (128 * 128) + (uint32_t)row * 128 + (uint32_t)((c ^ (row & 7)) << 4) +
-                              (uint32_t)(col & 7) * 2;
-        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(addr), "r"(pack_bf16(v.x * qscale, v.y * qscale)),
-                     "r"(pack_bf16(v.z * qscale, v.w * qscale))
-                     : "memory");
-      };
-      put(j, lo);
-      put(j + half, hi);
-    }
-    for (int t = 0; t < T; ++t) {
-      const int buf = t & 1;
-      const uint32_t ph = (uint32_t)(t >> 1) & 1u;
-      if (t >= 2) mbar_wait(smem_u32(&kv_free[buf]), ph ^ 1u, wc);   // PV of tile t-2 has read this buffer
-      const uint32_t kb = Ks + (uint32_t)buf * KV_BYTES, vb = Vs + (uint32_t)buf * KV_BYTES;
-      if (t < Tp) {
-        const int rows = min(KTC, P - t * KTC);
-        for (int idx = lt; idx < KTC * (DH / 8); idx += 128) {
-          const int row = idx / (DH / 8), c = idx % (DH / 8);
-          const bool ok = row < rows;
-          const size_t g = (size_t)(t * KTC + (ok ? row : 0)) * kv_stride + (size_t)c * 16;
-          const uint32_t o = (uint32_t)(c >> 3) * KV_BLOCK + (uint32_t)row * 128 + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
-          cp_async16(kb + o, Kg + g, ok ? 16u : 0u);
-          cp_async16(vb + o, Vg + g, ok ? 16u : 0u);
-        }
-        cp_async_commit();
-        cp_async_wait<0>();
-      } else {
-        // suffix tile: rotate this request's own keys, round K and V to bf16
-        for (int idx = lt; idx < KTC * (half / 4); idx += 128) {
-          const int js = idx / (half / 4), j = (idx % (half / 4)) * 4;
-          float4 klo = make_float4(0.f, 0.f, 0.f, 0.f), khi = klo, vlo = klo, vhi = klo;
-          if (js < S) {
-            const float* kr = a.qkv + (size_t)(b * S + js) * d.Nqkv + d.Nq + (size_t)hk * DH;
-            const float* vr = kr + d.Hkv * DH;
-            klo = *reinterpret_cast<const float4*>(kr + j), khi = *reinterpret_cast<const float4*>(kr + j + half);
-            vlo = *reinterpret_cast<const float4*>(vr + j), vhi = *reinterpret_cast<const float4*>(vr + j + half);
-            if (a.rope) {
-              const float4 cs0 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + js) * half + j);
-              const float4 cs1 = *reinterpret_cast<const float4*>(a.rope + (size_t)(P + js) * half + j + 2);
-              const float4 l2 = make_float4(klo.x * cs0.x - khi.x * cs0.y, klo.y * cs0.z - khi.y * cs0.w,
-                                            klo.z * cs1.x - khi.z * cs1.y, klo.w * cs1.z - khi.w * cs1.w);
-              khi = make_float4(khi.x * cs0.x + klo.x * cs0.y, khi.y * cs0.z + klo.y * cs0.w,
-                                khi.z * cs1.x + klo.z * cs1.y, khi.w * cs1.z + klo.w * cs1.w);
-              klo = l2;
-            }
-          }
-          auto put = [&](uint32_t tb, int col, float4 v) {
-            const uint32_t addr = tb + (uint32_t)(col >> 6) * KV_BLOCK + (uint32_t)js * 128 +
-                                  (uint32_t)((((col & 63) >> 3) ^ (js & 7)) << 4) + (uint32_t)(col & 7) * 2;
-            asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(addr), "r"(pack_bf16(v.x, v.y)), "r"(pack_bf16(v.z, v.w))
-                         : "memory");
-          };
-          put(kb, j, klo), put(kb, j + half, khi), put(vb, j, vlo), put(vb, j + half, vhi);
-        }
-      }
-      fence_async_smem();                  // these generic-proxy writes are read by the tensor core
-      group_sync<BAR_LOAD, 128>();
-      if (lt == 0) mbar_arrive_local(smem_u32(&kv_full[buf]));
+    // K buffer (t & 1) is free again once the logits of tile t exist (s_full), V buffer once P V of tile t has
+    // completed (pv_done).  Tile t + 1 is published only after that wait: its consumer could not start
+    // earlier anyway, and it keeps the waited barrier from running a whole phase ahead of the parity wait.
+    uint64_t* full = is_v ? v_full : k_full;
+    for (int t = 0; t + 1 < T; ++t) {
+      if (is_v) mbar_wait(smem_u32(&pv_done[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
+      else mbar_wait(smem_u32(&s_full[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
+      cp_async_wait<0>();                    // tile t + 1 (issued one iteration ago) has landed
+      fence_async_smem();                    // generic-proxy writes, read next by the tensor core
+      if (is_v) group_sync<BAR_LOAD + 2, 64>(); else group_sync<BAR_LOAD, 64>();
+      if (lt2 == 0) mbar_arrive_local(smem_u32(&full[(t + 1) & 1]));
+      if (t + 2 < T) issue(t + 2);
     }
   } else if (warp == 4) {
     // =========================== MMA issuer ========================================================
-    for (int t = 0; t < T; ++t) {
+    // Order: S(0), S(1); then for every tile t: P(t) V(t), S(t+2).  With two S buffers in TMEM the logits are
+    // always ready one tile before the softmax warps want them.
+    auto issue_s = [&](int t) {
       const int buf = t & 1;
-      const uint32_t ph = (uint32_t)(t >> 1) & 1u;
-      bool ok = mbar_wait(smem_u32(&kv_full[buf]), ph, wc);
-      if (t > 0) ok = mbar_wait(smem_u32(&s_free), (uint32_t)(t - 1) & 1u, wc) && ok;   // softmax has read S of t-1
+      bool ok = mbar_wait(smem_u32(&k_full[buf]), (uint32_t)(t >> 1) & 1u, wc);
+      if (t >= 2) ok = mbar_wait(smem_u32(&s_free[buf]), (uint32_t)((t >> 1) - 1) & 1u, wc) && ok;   // S(t-2) has been read
       tc_fence_after();
-      const uint32_t kb = Ks + (uint32_t)buf * KV_BYTES, vb = Vs + (uint32_t)buf * KV_BYTES;
-      const bool go = __all_sync(0xffffffffu, ok);
-      // ---- S = Q K^T ----
-      if (go) {
+      const uint32_t kb = Ks + (uint32_t)buf * KV_BYTES;
+      if (__all_sync(0xffffffffu, ok)) {
 #pragma unroll
         for (int kk = 0; kk < DH / 16; ++kk) {
           const uint64_t da = make_desc(Qs + (uint32_t)(kk >> 2) * (128 * 128) + (uint32_t)(kk & 3) * 32);
           const uint64_t db = make_desc(kb + (uint32_t)(kk >> 2) * KV_BLOCK + (uint32_t)(kk & 3) * 32);
-          if (elect_one()) umma_bf16(tmem_s, da, db, IDESC_S, kk > 0 ? 1u : 0u);
+          if (elect_one()) umma_bf16(tmem_s + (uint32_t)buf * KTC, da, db, IDESC_S, kk > 0 ? 1u : 0u);
         }
       }
-      if (elect_one()) umma_commit(smem_u32(&s_full));
+      if (elect_one()) umma_commit(smem_u32(&s_full[buf]));
       __syncwarp();
-      // ---- O += P V ----
-      ok = mbar_wait(smem_u32(&p_full), (uint32_t)t & 1u, wc);
+    };
+    issue_s(0);
+    if (T > 1) issue_s(1);
+    for (int t = 0; t < T; ++t) {
+      const int buf = t & 1;
+      const uint32_t vb = Vs + (uint32_t)buf * KV_BYTES, pb = Ps + (uint32_t)buf * P_BYTES;
+      bool ok = mbar_wait(smem_u32(&v_full[buf]), (uint32_t)(t >> 1) & 1u, wc);
+      ok = mbar_wait(smem_u32(&p_full[buf]), (uint32_t)(t >> 1) & 1u, wc) && ok;
       tc_fence_after();
-      if (__all_sync(0xffffffffu, ok) && go) {
+      if (__all_sync(0xffffffffu, ok)) {
 #pragma unroll
         for (int kj = 0; kj < KTC / 16; ++kj) {
-          const uint64_t da = make_desc(Ps + (uint32_t)kj * 32);
+          const uint64_t da = make_desc(pb + (uint32_t)kj * 32);
           const uint64_t db = make_desc_mn(vb + (uint32_t)kj * (16 * 128), KV_BLOCK, 1024);
           if (elect_one()) umma_bf16(tmem_o, da, db, IDESC_PV, (t > 0 || kj > 0) ? 1u : 0u);
         }
       }
-      if (elect_one()) {
-        umma_commit(smem_u32(&kv_free[buf]));
-        umma_commit(smem_u32(&pv_done));
-      }
+      if (elect_one()) umma_commit(smem_u32(&pv_done[buf]));
       __syncwarp();
+      if (t + 2 < T) issue_s(t + 2);
     }
   } else {
     // =========================== softmax / correction / output =====================================
@@ -245,52 +266,57 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     const int row = q * 32 + lane;            // accumulator row = TMEM lane
     const int hl = row >> 6, i = row & 63;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    float m = -INFINITY, l = 0.f;
+    float m = -INFINITY, l = 0.f;             // running maximum (log2 units) and sum
     const bool causal_row = d.block_causal && d.ns && i == 0;
     for (int t = 0; t < T; ++t) {
-      const bool ok = mbar_wait(smem_u32(&s_full), (uint32_t)t & 1u, wc);
+      mbar_wait(smem_u32(&s_full[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
       tc_fence_after();
-      const int valid = t < Tp ? min(KTC, P - t * KTC) : S;
+      const int valid = t == 0 ? S : min(KTC, P - (t - 1) * KTC);
       float s[KTC];
 #pragma unroll
-      for (int c = 0; c < KTC; c += 16) tmem_ld16(tmem_s + lane_addr + (uint32_t)c, s + c);
+      for (int c = 0; c < KTC; c += 16) tmem_ld16(tmem_s + (uint32_t)(t & 1) * KTC + lane_addr + (uint32_t)c, s + c);
       tc_fence_before();
       group_sync<BAR_SOFT, 128>();
-      if (st == 0) mbar_arrive_local(smem_u32(&s_free));     // S may be overwritten by the next tile
-      float mx = -INFINITY;
+      if (st == 0) mbar_arrive_local(smem_u32(&s_free[t & 1]));     // this S buffer may be overwritten
+      if (valid < KTC) {
 #pragma unroll
-      for (int c = 0; c < KTC; ++c) {
-        bool vis = c < valid;
-        if (causal_row && t >= Tp && c != 0) vis = false;   // state token sees, of the suffix, only itself
-        s[c] = vis ? s[c] * LOG2E : -INFINITY;
-        mx = fmaxf(mx, s[c]);
+        for (int c = 0; c < KTC; ++c) s[c] = c < valid ? s[c] : -INFINITY;
       }
+      if (causal_row && t == 0) {             // the state token sees, of the suffix, only itself
+#pragma unroll
+        for (int c = 1; c < KTC; ++c) s[c] = -INFINITY;
+      }
+      float mx = s[0];
+#pragma unroll
+      for (int c = 1; c < KTC; ++c) mx = fmaxf(mx, s[c]);
+      mx *= LOG2E;
       // running maximum: keep the old one unless the new exceeds it by more than the threshold
       float m_new = m;
       if (mx > m + RESCALE_THRESHOLD || m == -INFINITY) m_new = fmaxf(m, mx);
       const bool rescale = m_new != m && m != -INFINITY;
       const float corr = rescale ? exp2f(m - m_new) : 1.0f;
-      const float sub = m_new == -INFINITY ? 0.f : m_new;
+      const float nsub = m_new == -INFINITY ? 0.f : -m_new;
       float rs = 0.f;
-      // the previous tile's P V must have finished before P is overwritten (and before O is touched)
-      bool okp = true;
-      if (t > 0) okp = mbar_wait(smem_u32(&pv_done), (uint32_t)(t - 1) & 1u, wc);
-      tc_fence_after();
+      // P buffer (t & 1) was last read by P V of tile t - 2
+      if (t >= 2) mbar_wait(smem_u32(&pv_done[t & 1]), (uint32_t)((t >> 1) - 1) & 1u, wc);
+      uint8_t* prow = Ps_ptr + (size_t)(t & 1) * P_BYTES + (size_t)row * 128;
 #pragma unroll
       for (int c8 = 0; c8 < KTC / 8; ++c8) {
         uint32_t w[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float p0 = exp2f(s[c8 * 8 + 2 * e] - sub), p1 = exp2f(s[c8 * 8 + 2 * e + 1] - sub);
-          rs += p0 + p1;
-          w[e] = pack_bf16(p0, p1);
+          const float e0 = ex2_fast(fmaf(s[c8 * 8 + 2 * e], LOG2E, nsub)), e1 = ex2_fast(fmaf(s[c8 * 8 + 2 * e + 1], LOG2E, nsub));
+          rs += e0 + e1;
+          w[e] = pack_bf16(e0, e1);
         }
-        *reinterpret_cast<uint4*>(Ps_ptr + (size_t)row * 128 + (size_t)((c8 ^ (row & 7)) << 4)) =
-            make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(prow + (size_t)((c8 ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
       l = l * corr + rs;
       m = m_new;
       if (__any_sync(0xffffffffu, rescale)) {     // rare: rescale this warp's 32 accumulator rows
+        // every P V issued so far must have completed before O is touched
+        mbar_wait(smem_u32(&pv_done[(t - 1) & 1]), (uint32_t)((t - 1) >> 1) & 1u, wc);
+        tc_fence_after();
 #pragma unroll 1
         for (int c = 0; c < DH; c += 16) {
           float o[16];
@@ -304,12 +330,11 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       tc_fence_before();
       fence_async_smem();
       group_sync<BAR_SOFT, 128>();
-      if (st == 0) mbar_arrive_local(smem_u32(&p_full));
-      (void)ok;
-      (void)okp;
+      if (st == 0) mbar_arrive_local(smem_u32(&p_full[t & 1]));
     }
     // ---- output: O / l -> bf16 ----
-    const bool okf = __all_sync(0xffffffffu, mbar_wait(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, wc));
+    const bool okf =
+        __all_sync(0xffffffffu, mbar_wait(smem_u32(&pv_done[(T - 1) & 1]), (uint32_t)((T - 1) >> 1) & 1u, wc));
     tc_fence_after();
     {
       const bool wr = okf && i < S;             // the TMEM loads stay warp-uniform; only the stores are predicated
@@ -341,7 +366,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
 
 template <int DH>
 constexpr size_t attn_tc_smem() {
-  return 1024 + (size_t)128 * DH * 2 + 4 * (size_t)KTC * DH * 2 + (size_t)128 * KTC * 2;
+  return 1024 + (size_t)128 * DH * 2 + 4 * (size_t)KTC * DH * 2 + 2 * (size_t)128 * KTC * 2;
 }
 
 }  // namespace
