@@ -195,7 +195,10 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
  * graph per (batch, n_steps).  key "use_persistent": 1 (default) runs calls with batch * suffix_len
  * <= 64 tokens as one persistent cooperative kernel (the whole n-step loop, no kernel boundaries),
  * 0 uses the per-operator kernels for every batch.  key "use_tc_attention": 1 (default) lets large
- * batches use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "wait_limit": iteration bound of
+ * batches use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "use_pair_gemm": 1 runs the
+ * GEMMs of batches above 1024 tokens on CTA pairs (tcgen05 cta_group::2, persistent, overlapped epilogue), 0
+ * (default) keeps the single-CTA kernel, which measured faster on the batch-64 shapes.
+ * key "wait_limit": iteration bound of
  * device-side waits (testing).  Unknown key -> INVALID_ARG. */
 phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t value);
 

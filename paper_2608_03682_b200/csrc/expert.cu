@@ -86,6 +86,7 @@ struct phyai_expert {
   bool mega_ok = false;
   int use_mega = 1;
   int use_tc_attention = 1;
+  int use_pair_gemm = 0;   // measured slower than the single-CTA kernel on the batch-64 shapes: opt-in
   int n_sm = 0;
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
@@ -283,7 +284,11 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
   };
   auto tc_gemm = [&](TcGemm g) -> phyai_status_t {
     g.rows_pad = h->Mpad, g.M = g.M ? g.M : M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact;
-    cudaError_t e = launch_tc_gemm(h->status, g, nt, st);
+    cudaError_t e;
+    TcGemm gp = g;
+    gp.splits = 1;   // the CTA-pair kernel never splits K
+    if (h->use_pair_gemm && nt == 256 && g.M == M && tc_gemm_pair_supported(gp)) e = launch_tc_gemm_pair(h->status, gp, h->n_sm, st);
+    else e = launch_tc_gemm(h->status, g, nt, st);
     if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tensor GEMM launch failed: %s", cudaGetErrorString(e));
     ++cnt;
     return PHYAI_OK;
@@ -521,6 +526,12 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
 
   auto body = [&]() -> phyai_status_t {
     if (tc) CU(tc_gemm_setup());
+    if (tc) CU(tc_gemm_pair_setup());
+    {
+      int dev = 0;
+      CU(cudaGetDevice(&dev));
+      CU(cudaDeviceGetAttribute(&h->n_sm, cudaDevAttrMultiProcessorCount, dev));
+    }
     CU(cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking));
     ST(h->alloc(&h->status, 1, true));
     ST(h->alloc(&h->cu_internal, 2, true));
@@ -855,6 +866,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   }
   if (!strcmp(key, "use_tc_attention")) {
     h->use_tc_attention = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_pair_gemm")) {
+    h->use_pair_gemm = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

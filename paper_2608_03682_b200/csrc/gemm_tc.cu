@@ -46,6 +46,9 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   constexpr int NCOPY = NA + NB;
   constexpr int STAGE_BYTES = A_BYTES * NA + B_BYTES;
   constexpr int COLS = NA * NT;
+  // A producer warp's consecutive copies are NPROD / NCOPY k-steps apart; its parity wait on "stage free" is only
+  // meaningful while that step does not exceed the ring depth.
+  static_assert((NPROD + NCOPY - 1) / NCOPY <= STAGES, "producer stride exceeds the stage ring");
   // instruction descriptor: D fp32 (bit 4), A bf16 (bit 7), B bf16 (bit 10), both K-major,
   // N >> 3 at bit 17, M >> 4 at bit 24.
   constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((128u >> 4) << 24);

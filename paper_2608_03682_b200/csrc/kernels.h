@@ -114,5 +114,10 @@ struct TcGemm {
 // Returns cudaSuccess or the launch error; `nt` is the token-tile width (64, 128 or 256).
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st);
 cudaError_t tc_gemm_setup();  // one-time attribute setup (dynamic shared memory opt-in)
+// Large-batch variant on CTA pairs (256-token x 256-channel tiles, persistent, overlapped epilogue).
+// Covers TC_STORE, TC_RESID and TC_GEGLU without split-K; rows_pad must be a multiple of 256.
+bool tc_gemm_pair_supported(const TcGemm& g);
+cudaError_t launch_tc_gemm_pair(int* status, const TcGemm& g, int n_sm, cudaStream_t st);
+cudaError_t tc_gemm_pair_setup();
 
 }  // namespace phyai
