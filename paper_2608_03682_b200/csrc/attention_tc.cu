@@ -9,8 +9,8 @@
 //                  as an MN-major B operand, so K and V tiles share one shared-memory layout and loader
 // K/V tiles (64 keys) and P are double buffered; K and V are staged by separate warps with 16-byte cp.async
 // into the 128-byte-swizzled block layout the MMA descriptors expect, one tile ahead of their consumer.
-// The suffix keys are tile 0 (built from the fp32 q/k/v by every thread while the first prefix tile is in
-// flight); the prefix tiles follow.  The O accumulator is rescaled only when a row's running
+// The suffix keys are tile 0; the prefix tiles follow.  Q and the suffix K / V arrive as bf16, already
+// rotated (q also scaled), from the QKV projection's epilogue, so the prologue is plain 16-byte copies.  The O accumulator is rescaled only when a row's running
 // maximum grows by more than 2^8 (otherwise the old maximum is kept, which is exact algebra and costs
 // nothing), so the TMEM round trip of the correction is rare.
 //
@@ -135,62 +135,33 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     }
     cp_async_commit();
   };
-  if (warp < 4 && T > 1) issue(1);
-
-  // ---- every thread: Q (rotated, scaled) and the suffix K (rotated) / V tile, rounded to bf16 -------
-  // Items [0, 128 * J4) are Q (row, 4-column group), the next 64 * J4 the suffix K tile, the last 64 * J4
-  // the suffix V tile.  Each thread first issues the loads of four items (always from valid addresses, so
-  // nothing is predicated), then rotates and stores them: the global-load latency is paid once per four.
+  // ---- every thread: Q and the suffix K / V tile (tile 0), already rotated / scaled bf16, as 16-byte copies ----
   {
-    constexpr int J4 = half / 4;              // float4 pairs per row
-    constexpr int NQ = 128 * J4, NK = KTC * J4, NALL = NQ + 2 * NK;
-    const float qscale = rsqrtf((float)DH);
-    const bool rot_any = a.rope != nullptr;
-    const float* kv_src = a.qkv + d.Nq + (size_t)hk * DH;
-    for (int base0 = tid; base0 < NALL; base0 += 288 * 4) {
-      float4 lo[4], hi[4], cs0[4], cs1[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int idx = min(base0 + u * 288, NALL - 1);
-        const int isq = idx < NQ, k = idx - NQ, isv = k >= NK;
-        const int row = isq ? idx / J4 : (k - isv * NK) / J4, j = (idx % J4) * 4;
-        const int i = min(isq ? (row & 63) : row, S - 1);
-        const float* src = a.qkv + (size_t)(b * S + i) * d.Nqkv +
-                           (isq ? (size_t)(head0 + (row >> 6)) * DH : (size_t)(d.Nq + hk * DH + isv * d.Hkv * DH));
-        lo[u] = __ldg(reinterpret_cast<const float4*>(src + j));
-        hi[u] = __ldg(reinterpret_cast<const float4*>(src + j + half));
-        if (rot_any) {
-          cs0[u] = __ldg(reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j));
-          cs1[u] = __ldg(reinterpret_cast<const float4*>(a.rope + (size_t)(P + i) * half + j + 2));
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int idx = base0 + u * 288;
-        if (idx >= NALL) break;
-        const int isq = idx < NQ, k = idx - NQ, isv = k >= NK;
-        const int row = isq ? idx / J4 : (k - isv * NK) / J4, j = (idx % J4) * 4;
-        float4 l4 = lo[u], h4 = hi[u];
-        if (rot_any && !isv) {
-          const float4 c0 = cs0[u], c1 = cs1[u];
-          const float4 l2 = make_float4(l4.x * c0.x - h4.x * c0.y, l4.y * c0.z - h4.y * c0.w, l4.z * c1.x - h4.z * c1.y,
-                                        l4.w * c1.z - h4.w * c1.w);
-          h4 = make_float4(h4.x * c0.x + l4.x * c0.y, h4.y * c0.z + l4.y * c0.w, h4.z * c1.x + l4.z * c1.y,
-                           h4.w * c1.z + l4.w * c1.w);
-          l4 = l2;
-        }
-        const float sc = (isq ? (row & 63) : row) < S ? (isq ? qscale : 1.0f) : 0.0f;   // padding rows are zero
-        const uint32_t tile = isq ? Qs : (isv ? Vs : Ks), blk = isq ? 128 * 128 : KV_BLOCK;
-        auto put = [&](int col, float4 v) {       // 4 consecutive columns of `row`
-          const uint32_t addr = tile + (uint32_t)(col >> 6) * blk + (uint32_t)row * 128 +
-                                (uint32_t)((((col & 63) >> 3) ^ (row & 7)) << 4) + (uint32_t)(col & 7) * 2;
-          asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(addr), "r"(pack_bf16(v.x * sc, v.y * sc)),
-                       "r"(pack_bf16(v.z * sc, v.w * sc)));
-        };
-        put(j, l4);
-        put(j + half, h4);
-      }
+    const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(a.qr) + ((size_t)(b * d.Hq + head0) * S) * (DH * 2);
+    for (int idx = tid; idx < 128 * (DH / 8); idx += 288) {
+      const int row = idx / (DH / 8), c = idx % (DH / 8);        // row = head_local * 64 + i
+      const int hl = row >> 6, i = row & 63;
+      const bool ok = i < S;                                      // padding rows are zero-filled
+      cp_async16(Qs + (uint32_t)(c >> 3) * (128 * 128) + (uint32_t)row * 128 + (uint32_t)(((c & 7) ^ (row & 7)) << 4),
+                 qsrc + ((size_t)hl * S + (ok ? i : 0)) * (DH * 2) + (size_t)c * 16, ok ? 16u : 0u);
     }
+    const size_t kvoff = ((size_t)(b * d.Hkv + hk) * S) * (DH * 2);
+    const uint8_t* ksrc = reinterpret_cast<const uint8_t*>(a.kr) + kvoff;
+    const uint8_t* vsrc = reinterpret_cast<const uint8_t*>(a.vr) + kvoff;
+    for (int idx = tid; idx < 2 * KTC * (DH / 8); idx += 288) {
+      const int isv = idx >= KTC * (DH / 8), k = idx - isv * KTC * (DH / 8);
+      const int js = k / (DH / 8), c = k % (DH / 8);
+      const bool ok = js < S;
+      cp_async16((isv ? Vs : Ks) + (uint32_t)(c >> 3) * KV_BLOCK + (uint32_t)js * 128 + (uint32_t)(((c & 7) ^ (js & 7)) << 4),
+                 (isv ? vsrc : ksrc) + (size_t)(ok ? js : 0) * (DH * 2) + (size_t)c * 16, ok ? 16u : 0u);
+    }
+    cp_async_commit();
+  }
+  if (warp < 4 && T > 1) {
+    issue(1);                // first prefix tile: stays in flight past the barrier below
+    cp_async_wait<1>();
+  } else {
+    cp_async_wait<0>();
   }
   fence_async_smem();
   tc_fence_before();
@@ -375,9 +346,9 @@ bool attention_tc_supported(const Dims& d) {
   return d.dh == 256 && d.S <= 64 && d.Hq % 2 == 0 && (d.Hq / d.Hkv) % 2 == 0;
 }
 
-cudaError_t launch_attention_tc(const Request* rq, int* status, const float* qkv, const float2* rope, int layer,
-                                __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
-                                cudaStream_t st) {
+cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
+                                const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
+                                int batch, unsigned wait_limit, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(k_attn_tc<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -386,7 +357,7 @@ cudaError_t launch_attention_tc(const Request* rq, int* status, const float* qkv
     configured = true;
   }
   AttnArgs a{};
-  a.rq = rq, a.status = status, a.qkv = qkv, a.rope = rope, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
+  a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
   a.num_splits = 1, a.d = d, a.wait_limit = wait_limit;
   dim3 grid(d.Hq / 2, batch);
   k_attn_tc<256><<<grid, 288, attn_tc_smem<256>(), st>>>(a);

@@ -92,6 +92,7 @@ struct phyai_expert {
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
   __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
+  __nv_bfloat16 *qr_big = nullptr, *kr_big = nullptr, *vr_big = nullptr;   // rotated bf16 q / k / v of large batches
   float* mega_scratch = nullptr;
   float* mega_slab = nullptr;
   unsigned* mega_counters = nullptr;
@@ -334,11 +335,18 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       site(k, 2 * l, &gain, &shift, &gate);
       launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st);
       ++cnt;
+      const bool attn_tc = h->attn_mma && h->use_tc_attention && h->qr_big && attention_tc_supported(d) &&
+                           batch * (d.Hq / 2) >= 100;
       if (h->tc) {
         TcGemm g{};
         g.W = h->p_qkv[l], g.X = h->xn_t, g.N = d.Nqkv, g.K = D, g.epi = TC_STORE, g.scale = h->s_qkv[l];
         g.perm_dh = d.dh, g.perm_end = d.Nq + d.Hkv * d.dh;
         g.out_f32 = h->qkv, g.ldo = d.Nqkv, g.splits = 1;
+        if (attn_tc) {
+          // the tcgen05 attention kernel takes its operands rotated, scaled and rounded from this epilogue
+          g.epi = TC_QKV_ROT, g.rq = h->rq, g.rope = h->rope, g.qr = h->qr_big, g.kr = h->kr_big, g.vr = h->vr_big;
+          g.S = d.S, g.Hq = d.Hq, g.Hkv = d.Hkv, g.dh = d.dh;
+        }
         ST(tc_gemm(g));
       } else {
         SimtGemm g{};
@@ -346,9 +354,9 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         g.out = h->qkv, g.ldo = d.Nqkv;
         simt_gemm(g);
       }
-      if (h->attn_mma && h->use_tc_attention && attention_tc_supported(d) && batch * (d.Hq / 2) >= 100) {
-        cudaError_t e = launch_attention_tc(h->rq, h->status, h->qkv, h->rope, l, h->attn_t, h->Mpad, d, batch,
-                                            h->wait_limit, st);
+      if (attn_tc) {
+        cudaError_t e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn_t, h->Mpad, d,
+                                            batch, h->wait_limit, st);
         if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
         ++cnt;
       } else if (h->attn_mma) {
@@ -676,6 +684,11 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
     // ---- workspace (zeroed: padding rows of the tiled buffers stay finite) ----
     ST(h->alloc(&h->h, Mp * D, true));
     ST(h->alloc(&h->qkv, Mp * Nqkv, true));
+    if (tc && attention_tc_supported(d) && (int)cfg->max_batch * (d.Hq / 2) >= 100) {
+      ST(h->alloc(&h->qr_big, Mp * d.Nq, true));
+      ST(h->alloc(&h->kr_big, Mp * (size_t)(d.Hkv * d.dh), true));
+      ST(h->alloc(&h->vr_big, Mp * (size_t)(d.Hkv * d.dh), true));
+    }
     ST(h->alloc(&h->state_tok, (size_t)cfg->max_batch * D, true));
     if (tc) {
       h->attn_mma = attention_mma_supported(d);

@@ -60,6 +60,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int skip_flag;
+  __shared__ int2 tok_tab[NT];   // TC_QKV_ROT: per token of the tile (position, request * 64 + suffix row)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt_idx = blockIdx.x, tt = blockIdx.y;
@@ -158,12 +159,25 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     const int q = warp & 3, hf = ew >> 2;         // TMEM lane quarter, token-column quarter
     const int et = ew * 32 + lane;                // 0..511
     const int ch = q * 32 + lane;                 // row of the 128-row tile
+    const int tok_base = tt * NT;
+    if (g.epi == TC_QKV_ROT) {
+      // while the main loop runs: where each token of the tile sits (request, suffix row, rotary position)
+      for (int idx = et; idx < NT; idx += NEPI) {
+        const int tok = tok_base + idx;
+        int2 e = make_int2(0, 0);
+        if (tok < g.M) {
+          const int b = tok / g.S, i = tok - b * g.S;
+          const int* cu = g.rq->cu_lens;
+          e = make_int2(cu[b + 1] - cu[b] + i, b * 64 + i);
+        }
+        tok_tab[idx] = e;
+      }
+    }
     const bool ok = mbar_wait(smem_u32(&bar_accum), 0, wc);
     tc_fence_after();
-    const int tok_base = tt * NT;
     constexpr int HALF = NT / 4;   // token columns per epilogue warp
     const int c_begin = hf * HALF;
-    if (ok && !geglu) {
+    if (ok && !geglu && g.epi != TC_QKV_ROT) {
 #pragma unroll
       for (int a = 0; a < NA; ++a) {
         const int n = (nt_idx * NA + a) * 128 + ch;   // packed output channel
@@ -206,6 +220,91 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
             }
           }
         }
+      }
+    }
+    if (g.epi == TC_QKV_ROT) {
+      // Each accumulator is one 128-row tile of the packed q|k|v matrix: 64 channels of the first half of a head
+      // followed by their rotary partners (or 128 v channels).  The tile is transposed through shared memory
+      // (the stages are free: every MMA has completed) as fp32 [token][128 + 4]; then one thread takes 8
+      // channels and their partners of one token, rotates, and writes two 16-byte bf16 runs.
+      constexpr int PITCH = 132;
+      float* stage = reinterpret_cast<float*>(tiles_ptr);
+      const int half = g.dh >> 1;
+      const int rows = min(NT, g.M - tok_base);
+      const int Nq = g.Hq * g.dh, Nk = g.Hkv * g.dh;
+      const float qscale = rsqrtf((float)g.dh);
+#pragma unroll 1
+      for (int a = 0; a < NA; ++a) {
+        const int n0 = (nt_idx * NA + a) * 128;       // first packed row of this accumulator
+        if (ok) {
+          const float sc = g.scale ? g.scale[n0 + ch] : 1.0f;
+          for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
+            if (tok_base + c0 >= g.M) break;          // warp-uniform
+            float v[16];
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NT + c0), v);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * PITCH + ch] = v[j] * sc;
+          }
+        }
+        epi_sync();
+        if (ok) {
+          if (n0 < Nq + Nk) {
+            const bool isq = n0 < Nq;
+            const int nn = isq ? n0 : n0 - Nq;
+            const int head = nn / g.dh, t = (nn - head * g.dh) >> 7;   // 64-channel slice of the head's first half
+            __nv_bfloat16* base = isq ? g.qr : g.kr;
+            const int H = isq ? g.Hq : g.Hkv;
+            const float osc = isq ? qscale : 1.0f;
+            for (int it = et; it < rows * 8; it += NEPI) {
+              const int tl = it >> 3, j0 = (it & 7) * 8;
+              const int2 e = tok_tab[tl];
+              const float* sp = stage + (size_t)tl * PITCH + j0;
+              float lo[8], hi[8];
+              *reinterpret_cast<float4*>(lo) = *reinterpret_cast<const float4*>(sp);
+              *reinterpret_cast<float4*>(lo + 4) = *reinterpret_cast<const float4*>(sp + 4);
+              *reinterpret_cast<float4*>(hi) = *reinterpret_cast<const float4*>(sp + 64);
+              *reinterpret_cast<float4*>(hi + 4) = *reinterpret_cast<const float4*>(sp + 68);
+              if (g.rope) {
+                const float4* cs = reinterpret_cast<const float4*>(g.rope + (size_t)e.x * half + t * 64 + j0);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                  const float4 c = __ldg(cs + u);    // (cos, sin) of channels 2u and 2u + 1
+                  const float l0 = lo[2 * u], h0 = hi[2 * u], l1 = lo[2 * u + 1], h1 = hi[2 * u + 1];
+                  lo[2 * u] = l0 * c.x - h0 * c.y, hi[2 * u] = h0 * c.x + l0 * c.y;
+                  lo[2 * u + 1] = l1 * c.z - h1 * c.w, hi[2 * u + 1] = h1 * c.z + l1 * c.w;
+                }
+              }
+              const int b = e.y >> 6, i = e.y & 63;
+              __nv_bfloat16* dst = base + ((size_t)(b * H + head) * g.S + i) * g.dh + t * 64 + j0;
+              auto pk = [&](const float* x) {
+                __nv_bfloat162 p0 = __floats2bfloat162_rn(x[0] * osc, x[1] * osc), p1 = __floats2bfloat162_rn(x[2] * osc, x[3] * osc);
+                __nv_bfloat162 p2 = __floats2bfloat162_rn(x[4] * osc, x[5] * osc), p3 = __floats2bfloat162_rn(x[6] * osc, x[7] * osc);
+                return make_uint4(*reinterpret_cast<uint32_t*>(&p0), *reinterpret_cast<uint32_t*>(&p1),
+                                  *reinterpret_cast<uint32_t*>(&p2), *reinterpret_cast<uint32_t*>(&p3));
+              };
+              *reinterpret_cast<uint4*>(dst) = pk(lo);
+              *reinterpret_cast<uint4*>(dst + half) = pk(hi);
+            }
+          } else {
+            const int nn = n0 - Nq - Nk;
+            const int head = nn / g.dh, coff = nn - head * g.dh;       // 128 consecutive v channels
+            for (int it = et; it < rows * 16; it += NEPI) {
+              const int tl = it >> 4, j0 = (it & 15) * 8;
+              const int2 e = tok_tab[tl];
+              const float* sp = stage + (size_t)tl * PITCH + j0;
+              float x[8];
+              *reinterpret_cast<float4*>(x) = *reinterpret_cast<const float4*>(sp);
+              *reinterpret_cast<float4*>(x + 4) = *reinterpret_cast<const float4*>(sp + 4);
+              const int b = e.y >> 6, i = e.y & 63;
+              __nv_bfloat162 p0 = __floats2bfloat162_rn(x[0], x[1]), p1 = __floats2bfloat162_rn(x[2], x[3]);
+              __nv_bfloat162 p2 = __floats2bfloat162_rn(x[4], x[5]), p3 = __floats2bfloat162_rn(x[6], x[7]);
+              *reinterpret_cast<uint4*>(g.vr + ((size_t)(b * g.Hkv + head) * g.S + i) * g.dh + coff + j0) =
+                  make_uint4(*reinterpret_cast<uint32_t*>(&p0), *reinterpret_cast<uint32_t*>(&p1),
+                             *reinterpret_cast<uint32_t*>(&p2), *reinterpret_cast<uint32_t*>(&p3));
+            }
+          }
+        }
+        epi_sync();
       }
     }
     if (geglu) {

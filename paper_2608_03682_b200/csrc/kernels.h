@@ -87,12 +87,12 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
 
 // ---- tcgen05 attention (large batches: two heads per CTA, whole key range, no split) ------------------
 bool attention_tc_supported(const Dims& d);
-cudaError_t launch_attention_tc(const Request* rq, int* status, const float* qkv, const float2* rope, int layer,
-                                __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
-                                cudaStream_t st);
+cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
+                                const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
+                                int batch, unsigned wait_limit, cudaStream_t st);
 
 // ---- tcgen05 GEMM ------------------------------------------------------------------------------
-enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3 };
+enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3, TC_QKV_ROT = 4 };
 struct TcGemm {
   const __nv_bfloat16* W;   // packed blocks [N/128][KC][128x64]
   const __nv_bfloat16* W2;  // second matrix (GeGLU "up"), same packing, or null
@@ -109,6 +109,14 @@ struct TcGemm {
   int gelu_exact;
   int splits;                       // split-K factor (TC_RESID only)
   int perm_dh, perm_end;            // TC_STORE: packed rows < perm_end map to channels by qkv_packed_to_channel
+  // TC_QKV_ROT: the fused q|k|v projection (rows packed by qkv_channel_to_packed) leaves the kernel as the
+  // attention kernel's operands: q rotated and scaled by 1/sqrt(dh), k rotated, v as is, all bf16,
+  // q [b][Hq][S][dh], k and v [b][Hkv][S][dh]; token t is suffix row t % S of request t / S at position
+  // prefix_len(request) + t % S.
+  const Request* rq;
+  const float2* rope;               // [pos][dh/2] (cos, sin) or null (no rotation)
+  __nv_bfloat16 *qr, *kr, *vr;
+  int S, Hq, Hkv, dh;
   unsigned wait_limit;
 };
 // Returns cudaSuccess or the launch error; `nt` is the token-tile width (64, 128 or 256).
