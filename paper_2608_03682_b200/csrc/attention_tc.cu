@@ -24,6 +24,7 @@ namespace phyai {
 namespace {
 
 constexpr int KTC = 64;          // keys per tile
+constexpr int NKV = 3;           // K and V tile buffers each
 constexpr int BAR_LOAD = 1;      // named barrier of the 2 K loader warps
 constexpr int BAR_SOFT = 2;      // named barrier of the 4 softmax warps (3 = the V loader warps)
 constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units
@@ -35,6 +36,23 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
       "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
       "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
       "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16u(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+      "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]^T: the A operand (128 rows, K = 16 bf16 = 8 columns) is read from tensor memory.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -61,18 +79,16 @@ __device__ __forceinline__ uint64_t make_desc_mn(uint32_t saddr, uint32_t lbo, u
 
 template <int DH>
 __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
-  constexpr int Q_BYTES = 128 * DH * 2;       // DH/64 blocks of [128 rows x 128 B]
   constexpr int KV_BYTES = KTC * DH * 2;      // DH/64 blocks of [64 keys x 128 B]
   constexpr int KV_BLOCK = KTC * 128;
-  constexpr int P_BYTES = 128 * KTC * 2;      // one block [128 rows x 64 keys]
-  constexpr int COLS = 512;                   // S (two buffers) at columns [0, 128), O at [128, 128 + DH)
+  constexpr int COLS = 512;                   // S / P (two buffers) at columns [0, 128), O at [128, 384), Q at [384, 512)
   constexpr int half = DH / 2;
   constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KTC >> 3) << 17) | ((128u >> 4) << 24);
   constexpr uint32_t IDESC_PV =
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((128u >> 4) << 24);
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full[2], v_full[2], p_full[2], pv_done[2], s_full[2], s_free[2];
+  __shared__ __align__(8) uint64_t k_full[NKV], v_full[NKV], p_full[2], pv_done[2], s_full[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, skip_flag;
 
@@ -84,19 +100,19 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
   const int S = d.S;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t Qs = base, Ks = Qs + Q_BYTES, Vs = Ks + 2 * KV_BYTES, Ps = Vs + 2 * KV_BYTES;
-  uint8_t* Ps_ptr = smem_raw + (Ps - smem_u32(smem_raw));
+  const uint32_t Ks = base, Vs = Ks + NKV * KV_BYTES;
 
   if (tid == 0) {
     skip_flag = status_set(a.status) ? 1 : 0;
     abort_flag = 0;
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < NKV; ++i) {
       mbar_init(smem_u32(&k_full[i]), 1);
       mbar_init(smem_u32(&v_full[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&p_full[i]), 1);
       mbar_init(smem_u32(&pv_done[i]), 1);
       mbar_init(smem_u32(&s_full[i]), 1);
-      mbar_init(smem_u32(&s_free[i]), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -107,6 +123,10 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     tc_fence_before();
   }
   const WaitCtx wc{a.status, &abort_flag, a.wait_limit};
+  __syncthreads();                             // the TMEM base address is published
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * KTC, tmem_q = tmem_base + 2 * KTC + DH;
 
   const Request r = *a.rq;
   const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
@@ -124,7 +144,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
                      (((size_t)(a.layer * 2 + (is_v ? 1 : 0)) * r.kv_tokens + p0) * d.Hkv + hk) * (DH * 2) + (size_t)lc * 16;
   const uint32_t tile_base = (is_v ? Vs : Ks) + (uint32_t)(lc >> 3) * KV_BLOCK;
   auto issue = [&](int t) {                  // t >= 1
-    const uint32_t tb = tile_base + (uint32_t)(t & 1) * KV_BYTES;
+    const uint32_t tb = tile_base + (uint32_t)(t % NKV) * KV_BYTES;
     const int rows = min(KTC, P - (t - 1) * KTC);
     const uint8_t* g0 = G + (size_t)(t - 1) * KTC * kv_stride;
 #pragma unroll 8
@@ -135,40 +155,47 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     }
     cp_async_commit();
   };
-  // ---- every thread: Q and the suffix K / V tile (tile 0), already rotated / scaled bf16, as 16-byte copies ----
+  // ---- prologue: the suffix K / V tile (tile 0) as 16-byte copies by every thread; Q (already rotated, scaled
+  // bf16) goes from global memory straight into tensor memory, one row per softmax thread, where it serves as
+  // the A operand of every S = Q K^T (two bf16 per 32-bit column, in memory order) ----
   {
-    const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(a.qr) + ((size_t)(b * d.Hq + head0) * S) * (DH * 2);
-    for (int idx = tid; idx < 128 * (DH / 8); idx += 288) {
-      const int row = idx / (DH / 8), c = idx % (DH / 8);        // row = head_local * 64 + i
-      const int hl = row >> 6, i = row & 63;
-      const bool ok = i < S;                                      // padding rows are zero-filled
-      cp_async16(Qs + (uint32_t)(c >> 3) * (128 * 128) + (uint32_t)row * 128 + (uint32_t)(((c & 7) ^ (row & 7)) << 4),
-                 qsrc + ((size_t)hl * S + (ok ? i : 0)) * (DH * 2) + (size_t)c * 16, ok ? 16u : 0u);
-    }
     const size_t kvoff = ((size_t)(b * d.Hkv + hk) * S) * (DH * 2);
     const uint8_t* ksrc = reinterpret_cast<const uint8_t*>(a.kr) + kvoff;
     const uint8_t* vsrc = reinterpret_cast<const uint8_t*>(a.vr) + kvoff;
     for (int idx = tid; idx < 2 * KTC * (DH / 8); idx += 288) {
       const int isv = idx >= KTC * (DH / 8), k = idx - isv * KTC * (DH / 8);
       const int js = k / (DH / 8), c = k % (DH / 8);
-      const bool ok = js < S;
+      const bool ok = js < S;                                     // padding rows are zero-filled
       cp_async16((isv ? Vs : Ks) + (uint32_t)(c >> 3) * KV_BLOCK + (uint32_t)js * 128 + (uint32_t)(((c & 7) ^ (js & 7)) << 4),
                  (isv ? vsrc : ksrc) + (size_t)(ok ? js : 0) * (DH * 2) + (size_t)c * 16, ok ? 16u : 0u);
     }
     cp_async_commit();
   }
-  if (warp < 4 && T > 1) {
-    issue(1);                // first prefix tile: stays in flight past the barrier below
-    cp_async_wait<1>();
+  if (warp < 4) {
+    // the first prefix tiles stay in flight past the barrier below
+    if (T > 1) issue(1);
+    if (T > 2) issue(2);
+    if (T > 2) cp_async_wait<2>(); else if (T > 1) cp_async_wait<1>(); else cp_async_wait<0>();
   } else {
+    if (warp >= 5) {
+      const int row = (warp & 3) * 32 + lane, hl = row >> 6, i = row & 63;
+      const uint4* qsrc = reinterpret_cast<const uint4*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S + (i < S ? i : 0)) * DH);
+      const uint32_t qdst = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
+#pragma unroll 2
+      for (int c = 0; c < DH / 2; c += 16) {                      // 16 columns = 32 bf16 = 4 x 16 bytes
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = i < S ? __ldg(qsrc + (c >> 2) + u) : make_uint4(0u, 0u, 0u, 0u);
+        tmem_st16u(qdst + (uint32_t)c, reinterpret_cast<const uint32_t*>(v));
+      }
+      tmem_st_wait();
+    }
     cp_async_wait<0>();
   }
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * KTC;
   if (tid == 0) {                             // tile 0 is in place
     mbar_arrive_local(smem_u32(&k_full[0]));
     mbar_arrive_local(smem_u32(&v_full[0]));
@@ -176,35 +203,34 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
 
   if (warp < 4) {
     // =========================== loaders ==========================================================
-    // K buffer (t & 1) is free again once the logits of tile t exist (s_full), V buffer once P V of tile t has
+    // K buffer (t % 3) is free again once the logits of tile t exist (s_full), V buffer once P V of tile t has
     // completed (pv_done).  Tile t + 1 is published only after that wait: its consumer could not start
     // earlier anyway, and it keeps the waited barrier from running a whole phase ahead of the parity wait.
     uint64_t* full = is_v ? v_full : k_full;
     for (int t = 0; t + 1 < T; ++t) {
       if (is_v) mbar_wait(smem_u32(&pv_done[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
       else mbar_wait(smem_u32(&s_full[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
-      cp_async_wait<0>();                    // tile t + 1 (issued one iteration ago) has landed
+      if (t + 2 < T) cp_async_wait<1>(); else cp_async_wait<0>();   // tile t + 1 has landed (t + 2 may be in flight)
       fence_async_smem();                    // generic-proxy writes, read next by the tensor core
       if (is_v) group_sync<BAR_LOAD + 2, 64>(); else group_sync<BAR_LOAD, 64>();
-      if (lt2 == 0) mbar_arrive_local(smem_u32(&full[(t + 1) & 1]));
-      if (t + 2 < T) issue(t + 2);
+      if (lt2 == 0) mbar_arrive_local(smem_u32(&full[(t + 1) % NKV]));
+      if (t + 3 < T) issue(t + 3);           // into the buffer tile t has just released
     }
   } else if (warp == 4) {
     // =========================== MMA issuer ========================================================
     // Order: S(0), S(1); then for every tile t: P(t) V(t), S(t+2).  With two S buffers in TMEM the logits are
     // always ready one tile before the softmax warps want them.
     auto issue_s = [&](int t) {
-      const int buf = t & 1;
-      bool ok = mbar_wait(smem_u32(&k_full[buf]), (uint32_t)(t >> 1) & 1u, wc);
-      if (t >= 2) ok = mbar_wait(smem_u32(&s_free[buf]), (uint32_t)((t >> 1) - 1) & 1u, wc) && ok;   // S(t-2) has been read
+      const int buf = t & 1, kbuf = t % NKV;
+      // (S buffer `buf` last held P of tile t - 2, whose P V was issued before this: the tensor pipe runs in order)
+      const bool ok = mbar_wait(smem_u32(&k_full[kbuf]), (uint32_t)(t / NKV) & 1u, wc);
       tc_fence_after();
-      const uint32_t kb = Ks + (uint32_t)buf * KV_BYTES;
+      const uint32_t kb = Ks + (uint32_t)kbuf * KV_BYTES;
       if (__all_sync(0xffffffffu, ok)) {
 #pragma unroll
         for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint64_t da = make_desc(Qs + (uint32_t)(kk >> 2) * (128 * 128) + (uint32_t)(kk & 3) * 32);
           const uint64_t db = make_desc(kb + (uint32_t)(kk >> 2) * KV_BLOCK + (uint32_t)(kk & 3) * 32);
-          if (elect_one()) umma_bf16(tmem_s + (uint32_t)buf * KTC, da, db, IDESC_S, kk > 0 ? 1u : 0u);
+          if (elect_one()) umma_bf16_ts(tmem_s + (uint32_t)buf * KTC, tmem_q + (uint32_t)kk * 8, db, IDESC_S, kk > 0 ? 1u : 0u);
         }
       }
       if (elect_one()) umma_commit(smem_u32(&s_full[buf]));
@@ -213,17 +239,18 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     issue_s(0);
     if (T > 1) issue_s(1);
     for (int t = 0; t < T; ++t) {
-      const int buf = t & 1;
-      const uint32_t vb = Vs + (uint32_t)buf * KV_BYTES, pb = Ps + (uint32_t)buf * P_BYTES;
-      bool ok = mbar_wait(smem_u32(&v_full[buf]), (uint32_t)(t >> 1) & 1u, wc);
+      const int buf = t & 1, vbuf = t % NKV;
+      const uint32_t vb = Vs + (uint32_t)vbuf * KV_BYTES;
+      bool ok = mbar_wait(smem_u32(&v_full[vbuf]), (uint32_t)(t / NKV) & 1u, wc);
       ok = mbar_wait(smem_u32(&p_full[buf]), (uint32_t)(t >> 1) & 1u, wc) && ok;
       tc_fence_after();
       if (__all_sync(0xffffffffu, ok)) {
 #pragma unroll
         for (int kj = 0; kj < KTC / 16; ++kj) {
-          const uint64_t da = make_desc(pb + (uint32_t)kj * 32);
+          // A = P of this tile: bf16 pairs in the first 32 columns of S buffer `buf`
           const uint64_t db = make_desc_mn(vb + (uint32_t)kj * (16 * 128), KV_BLOCK, 1024);
-          if (elect_one()) umma_bf16(tmem_o, da, db, IDESC_PV, (t > 0 || kj > 0) ? 1u : 0u);
+          if (elect_one())
+            umma_bf16_ts(tmem_o, tmem_s + (uint32_t)buf * KTC + (uint32_t)kj * 8, db, IDESC_PV, (t > 0 || kj > 0) ? 1u : 0u);
         }
       }
       if (elect_one()) umma_commit(smem_u32(&pv_done[buf]));
@@ -246,9 +273,6 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       float s[KTC];
 #pragma unroll
       for (int c = 0; c < KTC; c += 16) tmem_ld16(tmem_s + (uint32_t)(t & 1) * KTC + lane_addr + (uint32_t)c, s + c);
-      tc_fence_before();
-      group_sync<BAR_SOFT, 128>();
-      if (st == 0) mbar_arrive_local(smem_u32(&s_free[t & 1]));     // this S buffer may be overwritten
       if (valid < KTC) {
 #pragma unroll
         for (int c = 0; c < KTC; ++c) s[c] = c < valid ? s[c] : -INFINITY;
@@ -268,19 +292,19 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       const float corr = rescale ? exp2f(m - m_new) : 1.0f;
       const float nsub = m_new == -INFINITY ? 0.f : -m_new;
       float rs = 0.f;
-      // P buffer (t & 1) was last read by P V of tile t - 2
-      if (t >= 2) mbar_wait(smem_u32(&pv_done[t & 1]), (uint32_t)((t >> 1) - 1) & 1u, wc);
-      uint8_t* prow = Ps_ptr + (size_t)(t & 1) * P_BYTES + (size_t)row * 128;
+      // P overwrites this thread's own row of the S buffer it has just read (bf16 pairs, first 32 columns):
+      // it is the A operand of P V, read from tensor memory
+      const uint32_t pdst = tmem_s + (uint32_t)(t & 1) * KTC + lane_addr;
 #pragma unroll
-      for (int c8 = 0; c8 < KTC / 8; ++c8) {
-        uint32_t w[4];
+      for (int c16 = 0; c16 < KTC / 32; ++c16) {
+        uint32_t w[16];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float e0 = ex2_fast(fmaf(s[c8 * 8 + 2 * e], LOG2E, nsub)), e1 = ex2_fast(fmaf(s[c8 * 8 + 2 * e + 1], LOG2E, nsub));
+        for (int e = 0; e < 16; ++e) {
+          const float e0 = ex2_fast(fmaf(s[c16 * 32 + 2 * e], LOG2E, nsub)), e1 = ex2_fast(fmaf(s[c16 * 32 + 2 * e + 1], LOG2E, nsub));
           rs += e0 + e1;
           w[e] = pack_bf16(e0, e1);
         }
-        *reinterpret_cast<uint4*>(prow + (size_t)((c8 ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        tmem_st16u(pdst + (uint32_t)c16 * 16, w);
       }
       l = l * corr + rs;
       m = m_new;
@@ -298,8 +322,8 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
         }
         tmem_st_wait();
       }
+      tmem_st_wait();
       tc_fence_before();
-      fence_async_smem();
       group_sync<BAR_SOFT, 128>();
       if (st == 0) mbar_arrive_local(smem_u32(&p_full[t & 1]));
     }
@@ -337,7 +361,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
 
 template <int DH>
 constexpr size_t attn_tc_smem() {
-  return 1024 + (size_t)128 * DH * 2 + 4 * (size_t)KTC * DH * 2 + 2 * (size_t)128 * KTC * 2;
+  return 1024 + 2 * (size_t)NKV * KTC * DH * 2;
 }
 
 }  // namespace
