@@ -55,6 +55,23 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, u
       "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// 64 consecutive columns of this warp's 32 lanes: four loads issued back to back, one wait.
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float* v) {
+  uint32_t r[64];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[16 * k + 0]), "=r"(r[16 * k + 1]), "=r"(r[16 * k + 2]), "=r"(r[16 * k + 3]), "=r"(r[16 * k + 4]),
+          "=r"(r[16 * k + 5]), "=r"(r[16 * k + 6]), "=r"(r[16 * k + 7]), "=r"(r[16 * k + 8]), "=r"(r[16 * k + 9]),
+          "=r"(r[16 * k + 10]), "=r"(r[16 * k + 11]), "=r"(r[16 * k + 12]), "=r"(r[16 * k + 13]), "=r"(r[16 * k + 14]),
+          "=r"(r[16 * k + 15])
+        : "r"(taddr + 16u * k)
+        : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ float ex2_fast(float x) {   // 2^x, x <= a few units; -inf -> 0
@@ -181,12 +198,13 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       const int row = (warp & 3) * 32 + lane, hl = row >> 6, i = row & 63;
       const uint4* qsrc = reinterpret_cast<const uint4*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S + (i < S ? i : 0)) * DH);
       const uint32_t qdst = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
-#pragma unroll 2
-      for (int c = 0; c < DH / 2; c += 16) {                      // 16 columns = 32 bf16 = 4 x 16 bytes
-        uint4 v[4];
+#pragma unroll 1
+      for (int c = 0; c < DH / 2; c += 64) {                      // 64 columns = 128 bf16 = 16 x 16 bytes per round,
+        uint4 v[16];                                              // all loads of a round in flight together
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = i < S ? __ldg(qsrc + (c >> 2) + u) : make_uint4(0u, 0u, 0u, 0u);
-        tmem_st16u(qdst + (uint32_t)c, reinterpret_cast<const uint32_t*>(v));
+        for (int u = 0; u < 16; ++u) v[u] = i < S ? __ldg(qsrc + (c >> 2) + u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) tmem_st16u(qdst + (uint32_t)(c + 16 * u), reinterpret_cast<const uint32_t*>(v + 4 * u));
       }
       tmem_st_wait();
     }
@@ -271,8 +289,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       tc_fence_after();
       const int valid = t == 0 ? S : min(KTC, P - (t - 1) * KTC);
       float s[KTC];
-#pragma unroll
-      for (int c = 0; c < KTC; c += 16) tmem_ld16(tmem_s + (uint32_t)(t & 1) * KTC + lane_addr + (uint32_t)c, s + c);
+      tmem_ld64(tmem_s + (uint32_t)(t & 1) * KTC + lane_addr, s);
       if (valid < KTC) {
 #pragma unroll
         for (int c = 0; c < KTC; ++c) s[c] = c < valid ? s[c] : -INFINITY;
@@ -336,16 +353,14 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       const float inv = 1.0f / l;
       const int orow = b * S + (i < S ? i : 0), head = head0 + hl;
 #pragma unroll 1
-      for (int c = 0; c < DH; c += 16) {
-        float o[16];
-        tmem_ld16(tmem_o + lane_addr + (uint32_t)c, o);
-        const uint4 lo = make_uint4(pack_bf16(o[0] * inv, o[1] * inv), pack_bf16(o[2] * inv, o[3] * inv),
-                                    pack_bf16(o[4] * inv, o[5] * inv), pack_bf16(o[6] * inv, o[7] * inv));
-        const uint4 hi = make_uint4(pack_bf16(o[8] * inv, o[9] * inv), pack_bf16(o[10] * inv, o[11] * inv),
-                                    pack_bf16(o[12] * inv, o[13] * inv), pack_bf16(o[14] * inv, o[15] * inv));
-        if (wr) {
-          *reinterpret_cast<uint4*>(a.out + out_index(orow, head * DH + c, a.rows_pad, d.Nq)) = lo;
-          *reinterpret_cast<uint4*>(a.out + out_index(orow, head * DH + c + 8, a.rows_pad, d.Nq)) = hi;
+      for (int c = 0; c < DH; c += 64) {
+        float o[64];
+        tmem_ld64(tmem_o + lane_addr + (uint32_t)c, o);         // four loads in flight, one wait
+#pragma unroll
+        for (int e = 0; e < 64; e += 8) {
+          const uint4 w = make_uint4(pack_bf16(o[e] * inv, o[e + 1] * inv), pack_bf16(o[e + 2] * inv, o[e + 3] * inv),
+                                     pack_bf16(o[e + 4] * inv, o[e + 5] * inv), pack_bf16(o[e + 6] * inv, o[e + 7] * inv));
+          if (wr) *reinterpret_cast<uint4*>(a.out + out_index(orow, head * DH + c + e, a.rows_pad, d.Nq)) = w;
         }
       }
     }
