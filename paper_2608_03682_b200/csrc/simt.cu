@@ -322,9 +322,52 @@ __global__ void k_rmsnorm_tiled4(const int* status, const float* h, const float*
   }
 }
 
+// Same, with the whole row held in registers (D = NV * 128): every load of the row is in flight at once and the
+// row is read once.
+template <int NV>
+__global__ void k_rmsnorm_tiled_reg(const int* status, const float* h, const float* gain, const float* shift,
+                                    __nv_bfloat16* out, int rows_pad, int M, float eps) {
+  if (status_set(status)) return;
+  constexpr int D = NV * 128;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const float* x = h + (size_t)row * D;
+  float4 v[NV];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) v[k] = *reinterpret_cast<const float4*>(x + k * 128 + lane * 4);
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+  ss = warp_sum(ss);
+  const float r = 1.0f / sqrtf(ss / (float)D + eps);
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int d = k * 128 + lane * 4;
+    const float4 g = __ldg(reinterpret_cast<const float4*>(gain + d));
+    float4 o = make_float4(v[k].x * r * g.x, v[k].y * r * g.y, v[k].z * r * g.z, v[k].w * r * g.w);
+    if (shift) {
+      const float4 s4 = __ldg(reinterpret_cast<const float4*>(shift + d));
+      o.x += s4.x, o.y += s4.y, o.z += s4.z, o.w += s4.w;
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(out + tiled_index(row, d, rows_pad)) = pk;
+  }
+}
+
 void launch_rmsnorm(const int* status, const float* h, const float* gain, const float* shift, float* out_f32,
                     __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st) {
   const int blocks = (M + 3) / 4;
+  if (out_tiled && D == 1024) {
+    k_rmsnorm_tiled_reg<8><<<blocks, 128, 0, st>>>(status, h, gain, shift, out_tiled, rows_pad, M, eps);
+    return;
+  }
+  if (out_tiled && D == 2048) {
+    k_rmsnorm_tiled_reg<16><<<blocks, 128, 0, st>>>(status, h, gain, shift, out_tiled, rows_pad, M, eps);
+    return;
+  }
   if (out_tiled && D % 128 == 0) {
     k_rmsnorm_tiled4<<<blocks, 128, 0, st>>>(status, h, gain, shift, out_tiled, rows_pad, M, D, eps);
     return;
@@ -372,9 +415,18 @@ __global__ void __launch_bounds__(256) k_final(const Request* rq, const int* sta
   float* xo = rq->x + (size_t)r * A;
   const float* n = nrm + warp * D;
   for (int a = lane; a < A; a += 32) {
-    float acc = 0.f;
-#pragma unroll 8
-    for (int d = 0; d < D; ++d) acc = fmaf(n[d], Wout[(size_t)d * A + a], acc);
+    // four partial sums over d mod 4 (independent dependency chains), combined in a fixed order
+    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+    int d = 0;
+#pragma unroll 4
+    for (; d + 4 <= D; d += 4) {
+      acc0 = fmaf(n[d], __ldg(Wout + (size_t)d * A + a), acc0);
+      acc1 = fmaf(n[d + 1], __ldg(Wout + (size_t)(d + 1) * A + a), acc1);
+      acc2 = fmaf(n[d + 2], __ldg(Wout + (size_t)(d + 2) * A + a), acc2);
+      acc3 = fmaf(n[d + 3], __ldg(Wout + (size_t)(d + 3) * A + a), acc3);
+    }
+    for (; d < D; ++d) acc0 = fmaf(n[d], __ldg(Wout + (size_t)d * A + a), acc0);
+    const float acc = (acc0 + acc1) + (acc2 + acc3);
     xo[a] = xo[a] + dt * (acc + bout[a]);
   }
 }
