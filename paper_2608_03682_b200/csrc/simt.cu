@@ -381,53 +381,77 @@ void launch_rmsnorm(const int* status, const float* h, const float* gain, const 
 // =============================================================================================
 // final norm -> out-projection -> Euler update (epilogue): x += dt * (n . Wout + bout)
 // =============================================================================================
-// One block normalises FR action rows into shared memory, then thread (a, row) walks D once: every
-// element of Wout is read once per block and used for all its rows.
-constexpr int FR = 8;
+// One block normalises FR action rows into shared memory (one warp per two rows).  The contraction over D is
+// then split over the 8 warps: warp w takes D/8 consecutive d for all FR rows, lane = action channel, so an
+// element of Wout is loaded once per block and used for FR rows, and the normalised rows are read as
+// float4.  The 8 partial sums are combined in a fixed order.
+constexpr int FR = 16;
 __global__ void __launch_bounds__(256) k_final(const Request* rq, const int* status, const float* h, const float* gain,
                                                const float* shift, const float* Wout, const float* bout, float dt, int A,
                                                int H, int D, int S, int ns, float eps, int rows_total) {
   if (status_set(status)) return;
-  extern __shared__ float nrm[];  // FR x D
+  extern __shared__ float nrm[];            // FR x D, then 8 x FR x 32 partial sums
+  float* part = nrm + (size_t)FR * D;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r0 = blockIdx.x * FR;
-  // one warp per row: norm
-  {
-    const int r = r0 + warp;
+  for (int rr = warp; rr < FR; rr += 8) {
+    const int r = r0 + rr;
     if (r < rows_total) {
       const int b = r / H, i = r % H;
       const float* x = h + (size_t)(b * S + ns + i) * D;
       float ss = 0.f;
       for (int d = lane; d < D; d += 32) ss = fmaf(x[d], x[d], ss);
       ss = warp_sum(ss);
-      const float rr = 1.0f / sqrtf(ss / (float)D + eps);
+      const float rs = 1.0f / sqrtf(ss / (float)D + eps);
       for (int d = lane; d < D; d += 32) {
-        float v = x[d] * rr * gain[d];
+        float v = x[d] * rs * gain[d];
         if (shift) v += shift[d];
-        nrm[warp * D + d] = v;
+        nrm[rr * D + d] = v;
       }
+    } else {
+      for (int d = lane; d < D; d += 32) nrm[rr * D + d] = 0.f;
     }
   }
   __syncthreads();
-  // outputs: warp w owns row r0 + w; lanes own action channels a = lane, lane + 32, ...
-  const int r = r0 + warp;
-  if (r >= rows_total) return;
-  float* xo = rq->x + (size_t)r * A;
-  const float* n = nrm + warp * D;
-  for (int a = lane; a < A; a += 32) {
-    // four partial sums over d mod 4 (independent dependency chains), combined in a fixed order
-    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-    int d = 0;
-#pragma unroll 4
-    for (; d + 4 <= D; d += 4) {
-      acc0 = fmaf(n[d], __ldg(Wout + (size_t)d * A + a), acc0);
-      acc1 = fmaf(n[d + 1], __ldg(Wout + (size_t)(d + 1) * A + a), acc1);
-      acc2 = fmaf(n[d + 2], __ldg(Wout + (size_t)(d + 2) * A + a), acc2);
-      acc3 = fmaf(n[d + 3], __ldg(Wout + (size_t)(d + 3) * A + a), acc3);
+  const bool vec = (D & 31) == 0;           // float4 reads of the rows need 8 equal, 4-aligned ranges
+  const int dper = vec ? D / 8 : (D + 7) / 8;
+  for (int a0 = 0; a0 < A; a0 += 32) {
+    const int a = a0 + lane;
+    float acc[FR];
+#pragma unroll
+    for (int rr = 0; rr < FR; ++rr) acc[rr] = 0.f;
+    if (a < A && !vec) {
+      for (int d = warp * dper; d < min(D, (warp + 1) * dper); ++d) {
+        const float w0 = __ldg(Wout + (size_t)d * A + a);
+#pragma unroll
+        for (int rr = 0; rr < FR; ++rr) acc[rr] = fmaf(nrm[rr * D + d], w0, acc[rr]);
+      }
     }
-    for (; d < D; ++d) acc0 = fmaf(n[d], __ldg(Wout + (size_t)d * A + a), acc0);
-    const float acc = (acc0 + acc1) + (acc2 + acc3);
-    xo[a] = xo[a] + dt * (acc + bout[a]);
+    if (a < A && vec) {
+      for (int d = warp * dper; d < (warp + 1) * dper; d += 4) {
+        const float w0 = __ldg(Wout + (size_t)d * A + a), w1 = __ldg(Wout + (size_t)(d + 1) * A + a);
+        const float w2 = __ldg(Wout + (size_t)(d + 2) * A + a), w3 = __ldg(Wout + (size_t)(d + 3) * A + a);
+#pragma unroll
+        for (int rr = 0; rr < FR; ++rr) {
+          const float4 n4 = *reinterpret_cast<const float4*>(nrm + rr * D + d);
+          acc[rr] = fmaf(n4.x, w0, fmaf(n4.y, w1, fmaf(n4.z, w2, fmaf(n4.w, w3, acc[rr]))));
+        }
+      }
+    }
+#pragma unroll
+    for (int rr = 0; rr < FR; ++rr) part[(warp * FR + rr) * 32 + lane] = acc[rr];
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < FR * 32; idx += 256) {
+      const int rr = idx >> 5, al = idx & 31, r = r0 + rr, aa = a0 + al;
+      if (r < rows_total && aa < A) {
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += part[(w * FR + rr) * 32 + al];
+        float* xo = rq->x + (size_t)r * A;
+        xo[aa] = xo[aa] + dt * (v + bout[aa]);
+      }
+    }
+    __syncthreads();
   }
 }
 void launch_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
@@ -438,7 +462,7 @@ void launch_final(const Request* rq, const int* status, const float* h, const fl
     cudaFuncSetAttribute(k_final, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
     configured = true;
   }
-  k_final<<<(rows + FR - 1) / FR, 256, (size_t)FR * d.D * sizeof(float), st>>>(rq, status, h, gain, shift, Wout, bout, dt,
+  k_final<<<(rows + FR - 1) / FR, 256, ((size_t)FR * d.D + 8 * FR * 32) * sizeof(float), st>>>(rq, status, h, gain, shift, Wout, bout, dt,
                                                                                d.A, d.H, d.D, d.S, d.ns, d.eps, rows);
 }
 
