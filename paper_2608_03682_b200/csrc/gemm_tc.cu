@@ -177,7 +177,8 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     tc_fence_after();
     constexpr int HALF = NT / 4;   // token columns per epilogue warp
     const int c_begin = hf * HALF;
-    if (ok && !geglu && g.epi != TC_QKV_ROT) {
+    const bool resid_red = g.epi == TC_RESID && gridDim.z > 1;   // split-K: vector reductions, see below
+    if (ok && !geglu && g.epi != TC_QKV_ROT && !resid_red) {
 #pragma unroll
       for (int a = 0; a < NA; ++a) {
         const int n = (nt_idx * NA + a) * 128 + ch;   // packed output channel
@@ -220,6 +221,39 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
             }
           }
         }
+      }
+    }
+    if (resid_red) {
+      // Split-K residual: every k-range adds its partial tile to h.  The tile is transposed through shared memory
+      // (fp32 [token][128 + 4]) so that one thread adds 4 consecutive channels of one token with a single
+      // 16-byte reduction: a quarter of the reduction operations of per-element atomics, in whole 128-byte lines.
+      constexpr int PITCH = 132;
+      float* stage = reinterpret_cast<float*>(tiles_ptr);
+      const int rows = min(NT, g.M - tok_base);
+#pragma unroll 1
+      for (int a = 0; a < NA; ++a) {
+        const int n0 = (nt_idx * NA + a) * 128;
+        if (ok) {
+          const float sc = (g.scale ? g.scale[n0 + ch] : 1.0f) * (g.gate ? g.gate[n0 + ch] : 1.0f);
+          for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
+            if (tok_base + c0 >= g.M) break;          // warp-uniform
+            float v[16];
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NT + c0), v);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * PITCH + ch] = v[j] * sc;
+          }
+        }
+        epi_sync();
+        if (ok) {
+          for (int it = et; it < rows * 32; it += NEPI) {
+            const int tl = it >> 5, j0 = (it & 31) * 4;
+            const float4 x = *reinterpret_cast<const float4*>(stage + (size_t)tl * PITCH + j0);
+            float* dst = g.out_f32 + (size_t)(tok_base + tl) * g.ldo + n0 + j0;
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w)
+                         : "memory");
+          }
+        }
+        epi_sync();
       }
     }
     if (g.epi == TC_QKV_ROT) {
