@@ -95,8 +95,13 @@ __device__ __forceinline__ float gelu_f(float z, int exact) { return exact ? gel
 // GELU for the GeGLU epilogues: tanh form written as z * sigmoid(2u) (one exp, one fast divide), erf form as is.
 __device__ __forceinline__ float gelu_fast(float z, int exact) {
   if (exact) return gelu_erf_f(z);
-  const float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
-  return __fdividef(z, 1.0f + __expf(-2.0f * u));
+  // 0.5 z (1 + tanh(u)), u = sqrt(2/pi) (z + 0.044715 z^3), with the hardware tanh (absolute error ~5e-4 of a
+  // factor in [0, 2]: far inside the bf16 rounding of the result)
+  const float u = z * fmaf(0.7978845608028654f * 0.044715f, z * z, 0.7978845608028654f);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  const float hz = 0.5f * z;
+  return fmaf(hz, t, hz);
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
