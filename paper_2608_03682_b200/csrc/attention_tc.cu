@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((128u >> 4) << 24);
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full[NKV], v_full[NKV], p_full[2], pv_done[2], s_full[2];
+  __shared__ __align__(8) uint64_t k_full[NKV], v_full[NKV], p_full[2], pv_done[2], s_full[2], q_full;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, skip_flag;
 
@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       mbar_init(smem_u32(&k_full[i]), 1);
       mbar_init(smem_u32(&v_full[i]), 1);
     }
+    mbar_init(smem_u32(&q_full), 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&p_full[i]), 1);
       mbar_init(smem_u32(&pv_done[i]), 1);
@@ -155,59 +156,34 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     }
     cp_async_commit();
   };
-  // ---- prologue: the suffix K / V tile (tile 0) as 16-byte copies by every thread; Q (already rotated, scaled
-  // bf16) goes from global memory straight into tensor memory, one row per softmax thread, where it serves as
-  // the A operand of every S = Q K^T (two bf16 per 32-bit column, in memory order) ----
-  {
-    const size_t kvoff = ((size_t)(b * d.Hkv + hk) * S) * (DH * 2);
-    const uint8_t* ksrc = reinterpret_cast<const uint8_t*>(a.kr) + kvoff;
-    const uint8_t* vsrc = reinterpret_cast<const uint8_t*>(a.vr) + kvoff;
-    for (int idx = tid; idx < 2 * KTC * (DH / 8); idx += 288) {
-      const int isv = idx >= KTC * (DH / 8), k = idx - isv * KTC * (DH / 8);
-      const int js = k / (DH / 8), c = k % (DH / 8);
-      const bool ok = js < S;                                     // padding rows are zero-filled
-      cp_async16((isv ? Vs : Ks) + (uint32_t)(c >> 3) * KV_BLOCK + (uint32_t)js * 128 + (uint32_t)(((c & 7) ^ (js & 7)) << 4),
-                 (isv ? vsrc : ksrc) + (size_t)(ok ? js : 0) * (DH * 2) + (size_t)c * 16, ok ? 16u : 0u);
-    }
-    cp_async_commit();
-  }
-  if (warp < 4) {
-    // the first prefix tiles stay in flight past the barrier below
-    if (T > 1) issue(1);
-    if (T > 2) issue(2);
-    if (T > 2) cp_async_wait<2>(); else if (T > 1) cp_async_wait<1>(); else cp_async_wait<0>();
-  } else {
-    if (warp >= 5) {
-      const int row = (warp & 3) * 32 + lane, hl = row >> 6, i = row & 63;
-      const uint4* qsrc = reinterpret_cast<const uint4*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S + (i < S ? i : 0)) * DH);
-      const uint32_t qdst = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < DH / 2; c += 64) {                      // 64 columns = 128 bf16 = 16 x 16 bytes per round,
-        uint4 v[16];                                              // all loads of a round in flight together
-#pragma unroll
-        for (int u = 0; u < 16; ++u) v[u] = i < S ? __ldg(qsrc + (c >> 2) + u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) tmem_st16u(qdst + (uint32_t)(c + 16 * u), reinterpret_cast<const uint32_t*>(v + 4 * u));
-      }
-      tmem_st_wait();
-    }
-    cp_async_wait<0>();
-  }
-  fence_async_smem();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  if (tid == 0) {                             // tile 0 is in place
-    mbar_arrive_local(smem_u32(&k_full[0]));
-    mbar_arrive_local(smem_u32(&v_full[0]));
-  }
-
+  // ---- no CTA-wide prologue barrier: each stream publishes its own first tile, so S(0) starts as soon as Q and
+  // the suffix keys are in place while the suffix values and the first prefix tiles are still in flight ----
   if (warp < 4) {
     // =========================== loaders ==========================================================
     // K buffer (t % 3) is free again once the logits of tile t exist (s_full), V buffer once P V of tile t has
     // completed (pv_done).  Tile t + 1 is published only after that wait: its consumer could not start
     // earlier anyway, and it keeps the waited barrier from running a whole phase ahead of the parity wait.
     uint64_t* full = is_v ? v_full : k_full;
+    {
+      // tile 0 = this request's own keys / values (rotated bf16 from the QKV epilogue); rows >= S are zero-filled
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(is_v ? a.vr : a.kr) + ((size_t)(b * d.Hkv + hk) * S) * (DH * 2) +
+                           (size_t)lc * 16;
+#pragma unroll 8
+      for (int row = r0; row < KTC; row += 2) {
+        const bool ok = row < S;
+        cp_async16(tile_base + (uint32_t)row * 128 + (uint32_t)(((lc & 7) ^ (row & 7)) << 4),
+                   src + (size_t)(ok ? row : 0) * (DH * 2), ok ? 16u : 0u);
+      }
+      cp_async_commit();
+      // The prefix tiles are requested only after tile 0 has landed: every CTA of the grid starts at the same time,
+      // and requests issued together share the SM's ingest bandwidth, which would delay the data needed first.
+      cp_async_wait<0>();
+      fence_async_smem();
+      if (is_v) group_sync<BAR_LOAD + 2, 64>(); else group_sync<BAR_LOAD, 64>();
+      if (lt2 == 0) mbar_arrive_local(smem_u32(&full[0]));
+      if (T > 1) issue(1);
+      if (T > 2) issue(2);
+    }
     for (int t = 0; t + 1 < T; ++t) {
       if (is_v) mbar_wait(smem_u32(&pv_done[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
       else mbar_wait(smem_u32(&s_full[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
@@ -237,6 +213,10 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       if (elect_one()) umma_commit(smem_u32(&s_full[buf]));
       __syncwarp();
     };
+    {
+      mbar_wait(smem_u32(&q_full), 0u, wc);    // Q is in tensor memory
+      tc_fence_after();
+    }
     issue_s(0);
     if (T > 1) issue_s(1);
     for (int t = 0; t < T; ++t) {
@@ -266,6 +246,24 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     const int hl = row >> 6, i = row & 63;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     float m = -INFINITY, l = 0.f;             // running maximum (log2 units) and sum
+    {
+      // Q (already rotated, scaled bf16) goes from global memory straight into tensor memory, one row per thread,
+      // where it is the A operand of every S = Q K^T (two bf16 per 32-bit column, in memory order)
+      const uint4* qsrc = reinterpret_cast<const uint4*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S + (i < S ? i : 0)) * DH);
+      const uint32_t qdst = tmem_q + lane_addr;
+#pragma unroll 1
+      for (int c = 0; c < DH / 2; c += 64) {                      // 64 columns = 128 bf16 = 16 x 16 bytes per round,
+        uint4 v[16];                                              // all loads of a round in flight together
+#pragma unroll
+        for (int u = 0; u < 16; ++u) v[u] = i < S ? __ldg(qsrc + (c >> 2) + u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) tmem_st16u(qdst + (uint32_t)(c + 16 * u), reinterpret_cast<const uint32_t*>(v + 4 * u));
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      group_sync<BAR_SOFT, 128>();
+      if (st == 0) mbar_arrive_local(smem_u32(&q_full));
+    }
     const bool causal_row = d.block_causal && d.ns && i == 0;
     for (int t = 0; t < T; ++t) {
       mbar_wait(smem_u32(&s_full[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
