@@ -213,6 +213,26 @@ phyai_status_t build_tables(phyai_expert* h, int n, cudaStream_t st, Tables** ou
 // ---------------------------------------------------------------------------------------------
 int pick_nt(int M) { return M <= 64 ? 64 : (M <= 1024 ? 128 : 256); }
 
+// Token-tile width and split-K factor of a residual GEMM (N = width, large token counts): the pair that minimises
+// waves x (k-chunks per CTA x clocks per k-chunk + epilogue).  Clocks per k-chunk follow the measured SM ingest of
+// ~39 bytes per clock: 64 KB per k-chunk at 256 tokens, 56 KB at 192.
+void pick_resid_tiling(int M, int Mpad, int N, int KC, int n_sm, int* nt_out, int* splits_out) {
+  const int nts[2] = {256, 192};
+  double best = 1e30;
+  *nt_out = 256, *splits_out = 1;
+  for (int nt : nts) {
+    const int tok_tiles = (M + nt - 1) / nt;
+    if (tok_tiles * nt > Mpad || N % 256) continue;
+    for (int s = 1; s <= 4 && s <= KC; s *= 2) {
+      const int ctas = tok_tiles * (N / 256) * s;
+      const int waves = (ctas + n_sm - 1) / n_sm;
+      const double per_kc = nt == 256 ? 1640.0 : 1436.0, epi = (s > 1 ? 9000.0 : 11000.0) * nt / 256.0 + 4000.0;
+      const double cost = waves * ((double)((KC + s - 1) / s) * per_kc + epi);
+      if (cost < best) best = cost, *nt_out = nt, *splits_out = s;
+    }
+  }
+}
+
 int pick_splits(int n_tiles, int tok_tiles, int KC) {
   int want = 148 / (n_tiles * tok_tiles);
   int s = 1;
@@ -289,7 +309,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     TcGemm gp = g;
     gp.splits = 1;   // the CTA-pair kernel never splits K
     if (h->use_pair_gemm && nt == 256 && g.M == M && tc_gemm_pair_supported(gp)) e = launch_tc_gemm_pair(h->status, gp, h->n_sm, st);
-    else e = launch_tc_gemm(h->status, g, nt, st);
+    else e = launch_tc_gemm(h->status, g, g.nt_override ? g.nt_override : nt, st);
     if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tensor GEMM launch failed: %s", cudaGetErrorString(e));
     ++cnt;
     return PHYAI_OK;
@@ -374,6 +394,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         TcGemm g{};
         g.W = h->p_o[l], g.X = h->attn_t, g.N = D, g.K = d.Nq, g.epi = TC_RESID, g.scale = h->s_o[l], g.gate = gate;
         g.out_f32 = h->h, g.ldo = D, g.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.Nq / 64);
+        if (nt == 256 && D % 256 == 0) pick_resid_tiling(M, h->Mpad, D, d.Nq / 64, h->n_sm, &g.nt_override, &g.splits);
         ST(tc_gemm(g));
       } else {
         SimtGemm g{};
@@ -392,6 +413,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         TcGemm g2{};
         g2.W = h->p_d[l], g2.X = h->m_t, g2.N = D, g2.K = d.F, g2.epi = TC_RESID, g2.scale = h->s_d[l], g2.gate = gate;
         g2.out_f32 = h->h, g2.ldo = D, g2.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.F / 64);
+        if (nt == 256 && D % 256 == 0) pick_resid_tiling(M, h->Mpad, D, d.F / 64, h->n_sm, &g2.nt_override, &g2.splits);
         ST(tc_gemm(g2));
       } else {
         SimtGemm g{};

@@ -46,6 +46,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   constexpr int NCOPY = NA + NB;
   constexpr int STAGE_BYTES = A_BYTES * NA + B_BYTES;
   constexpr int COLS = NA * NT;
+  constexpr int ALLOC_COLS = COLS <= 32 ? 32 : COLS <= 64 ? 64 : COLS <= 128 ? 128 : COLS <= 256 ? 256 : 512;   // power of two
   // A producer warp's consecutive copies are NPROD / NCOPY k-steps apart; its parity wait on "stage free" is only
   // meaningful while that step does not exceed the ring depth.
   static_assert((NPROD + NCOPY - 1) / NCOPY <= STAGES, "producer stride exceeds the stage ring");
@@ -88,7 +89,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 8) {
-    tmem_alloc(smem_u32(&tmem_slot), COLS < 32 ? 32 : COLS);
+    tmem_alloc(smem_u32(&tmem_slot), ALLOC_COLS);
     tc_fence_before();
   }
   __syncthreads();
@@ -383,7 +384,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   }
   if (warp == 8) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, COLS < 32 ? 32 : COLS);
+    tmem_dealloc(tmem_base, ALLOC_COLS);
   }
 }
 
@@ -415,6 +416,7 @@ cudaError_t tc_gemm_setup() {
   if ((e = setup_one<128, 2, 4>()) != cudaSuccess) return e;
   if ((e = setup_one<256, 1, 4>()) != cudaSuccess) return e;
   if ((e = setup_one<256, 2, 3>()) != cudaSuccess) return e;
+  if ((e = setup_one<192, 2, 4>()) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
@@ -422,9 +424,11 @@ cudaError_t tc_gemm_setup() {
 // tiles per CTA when the token tile is 256 wide and the channel count allows it (halves the
 // activation traffic per MMA), else one.
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st) {
-  const bool two = g.epi == TC_GEGLU || (nt == 256 && g.N % 256 == 0);
+  const bool two = g.epi == TC_GEGLU || (nt >= 192 && g.N % 256 == 0);
   if (nt == 64) return two ? launch_one<64, 2, 4>(status, g, st) : launch_one<64, 1, 6>(status, g, st);
   if (nt == 128) return two ? launch_one<128, 2, 4>(status, g, st) : launch_one<128, 1, 5>(status, g, st);
+  // 192-token tiles (two channel tiles per CTA only): for token counts where they fill the SMs better
+  if (nt == 192 && g.epi != TC_GEGLU && g.N % 256 == 0) return launch_one<192, 2, 4>(status, g, st);
   return two ? launch_one<256, 2, 3>(status, g, st) : launch_one<256, 1, 4>(status, g, st);
 }
 

@@ -108,6 +108,7 @@ struct TcGemm {
   int rows_in, rows_out, row_off;   // TC_BIAS_ROWMAP row remap
   int gelu_exact;
   int splits;                       // split-K factor (TC_RESID only)
+  int nt_override;                  // host side: token-tile width chosen for this GEMM (0 = the caller's default)
   int perm_dh, perm_end;            // TC_STORE: packed rows < perm_end map to channels by qkv_packed_to_channel
   // TC_QKV_ROT: the fused q|k|v projection (rows packed by qkv_channel_to_packed) leaves the kernel as the
   // attention kernel's operands: q rotated and scaled by 1/sqrt(dh), k rotated, v as is, all bf16,
