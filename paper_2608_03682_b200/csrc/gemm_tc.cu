@@ -290,9 +290,25 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
             __nv_bfloat16* base = isq ? g.qr : g.kr;
             const int H = isq ? g.Hq : g.Hkv;
             const float osc = isq ? qscale : 1.0f;
+            // the rotary table rows of the next item are requested before this item is processed
+            float4 cs_next[4];
+            int2 e_next = make_int2(0, 0);
+            auto fetch = [&](int it2) {
+              e_next = tok_tab[it2 >> 3];
+              if (g.rope) {
+                const float4* cs = reinterpret_cast<const float4*>(g.rope + (size_t)e_next.x * half + t * 64 + (it2 & 7) * 8);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) cs_next[u] = __ldg(cs + u);
+              }
+            };
+            if (et < rows * 8) fetch(et);
             for (int it = et; it < rows * 8; it += NEPI) {
               const int tl = it >> 3, j0 = (it & 7) * 8;
-              const int2 e = tok_tab[tl];
+              const int2 e = e_next;
+              float4 csc[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) csc[u] = cs_next[u];
+              if (it + NEPI < rows * 8) fetch(it + NEPI);
               const float* sp = stage + (size_t)tl * PITCH + j0;
               float lo[8], hi[8];
               *reinterpret_cast<float4*>(lo) = *reinterpret_cast<const float4*>(sp);
@@ -300,10 +316,9 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
               *reinterpret_cast<float4*>(hi) = *reinterpret_cast<const float4*>(sp + 64);
               *reinterpret_cast<float4*>(hi + 4) = *reinterpret_cast<const float4*>(sp + 68);
               if (g.rope) {
-                const float4* cs = reinterpret_cast<const float4*>(g.rope + (size_t)e.x * half + t * 64 + j0);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                  const float4 c = __ldg(cs + u);    // (cos, sin) of channels 2u and 2u + 1
+                  const float4 c = csc[u];           // (cos, sin) of channels 2u and 2u + 1
                   const float l0 = lo[2 * u], h0 = hi[2 * u], l1 = lo[2 * u + 1], h1 = hi[2 * u + 1];
                   lo[2 * u] = l0 * c.x - h0 * c.y, hi[2 * u] = h0 * c.x + l0 * c.y;
                   lo[2 * u + 1] = l1 * c.z - h1 * c.w, hi[2 * u + 1] = h1 * c.z + l1 * c.w;
@@ -424,7 +439,10 @@ cudaError_t tc_gemm_setup() {
 // tiles per CTA when the token tile is 256 wide and the channel count allows it (halves the
 // activation traffic per MMA), else one.
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st) {
-  const bool two = g.epi == TC_GEGLU || (nt >= 192 && g.N % 256 == 0);
+  bool two = g.epi == TC_GEGLU || (nt >= 192 && g.N % 256 == 0);
+  // a plain store epilogue cannot split K: when two-tile CTAs would leave more than half of the SMs idle, take one
+  // channel tile per CTA instead
+  if (g.epi == TC_BIAS_ROWMAP && nt == 256 && (g.N / 256) * ((g.M + 255) / 256) <= 74) two = false;
   if (nt == 64) return two ? launch_one<64, 2, 4>(status, g, st) : launch_one<64, 1, 6>(status, g, st);
   if (nt == 128) return two ? launch_one<128, 2, 4>(status, g, st) : launch_one<128, 1, 5>(status, g, st);
   // 192-token tiles (two channel tiles per CTA only): for token counts where they fill the SMs better

@@ -235,10 +235,60 @@ __global__ void k_embed_pi0(const Request* rq, const int* status, const float* W
     if (ns && i == 0) h[(size_t)(b * S) * D + n] = state_tok[(size_t)b * D + n];
   }
 }
+// Tiled-bf16 variant for large batches: one block takes ER action rows, a thread four consecutive output channels
+// of all of them, so an element of Wc is fetched once per ER rows and the results leave as 8-byte stores.
+constexpr int ER = 16;
+__global__ void __launch_bounds__(256) k_embed_pi0_rows(const Request* rq, const int* status, const float* Wc,
+                                                        const float* tb, const float* state_tok, float* h,
+                                                        __nv_bfloat16* u, int rows_pad, int A, int H, int D, int S, int ns,
+                                                        int rows_total) {
+  if (status_set(status)) return;
+  extern __shared__ float xs[];            // ER x A
+  const int r0 = blockIdx.x * ER;
+  for (int idx = threadIdx.x; idx < ER * A; idx += blockDim.x) {
+    const int r = r0 + idx / A;
+    xs[idx] = r < rows_total ? rq->x[(size_t)r * A + idx % A] : 0.f;
+  }
+  __syncthreads();
+  for (int n = threadIdx.x * 4; n < D; n += blockDim.x * 4) {
+    float4 acc[ER];
+#pragma unroll
+    for (int e = 0; e < ER; ++e) acc[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int a = 0; a < A; ++a) {
+      const float4 w = __ldg(reinterpret_cast<const float4*>(Wc + (size_t)a * D + n));
+#pragma unroll
+      for (int e = 0; e < ER; ++e) {
+        const float x = xs[e * A + a];
+        acc[e].x = fmaf(x, w.x, acc[e].x), acc[e].y = fmaf(x, w.y, acc[e].y);
+        acc[e].z = fmaf(x, w.z, acc[e].z), acc[e].w = fmaf(x, w.w, acc[e].w);
+      }
+    }
+    const float4 t4 = __ldg(reinterpret_cast<const float4*>(tb + n));
+#pragma unroll
+    for (int e = 0; e < ER; ++e) {
+      const int r = r0 + e;
+      if (r >= rows_total) break;
+      __nv_bfloat162 lo = __floats2bfloat162_rn(swish_precise(acc[e].x + t4.x), swish_precise(acc[e].y + t4.y));
+      __nv_bfloat162 hi = __floats2bfloat162_rn(swish_precise(acc[e].z + t4.z), swish_precise(acc[e].w + t4.w));
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(u + tiled_index(r, n, rows_pad)) = pk;
+      if (ns && r % H == 0)
+        *reinterpret_cast<float4*>(h + (size_t)((r / H) * S) * D + n) =
+            __ldg(reinterpret_cast<const float4*>(state_tok + (size_t)(r / H) * D + n));
+    }
+  }
+}
+
 void launch_embed_pi0(const Request* rq, const int* status, const float* Wc, const float* tb, const float* state_tok,
                       float* h, float* u_f32, __nv_bfloat16* u_tiled, int rows_pad, const Dims& d, int batch,
                       cudaStream_t st) {
   const int rows = batch * d.H;
+  if (u_tiled && d.D % 4 == 0 && rows >= 4 * ER) {
+    k_embed_pi0_rows<<<(rows + ER - 1) / ER, 256, (size_t)ER * d.A * sizeof(float), st>>>(
+        rq, status, Wc, tb, state_tok, h, u_tiled, rows_pad, d.A, d.H, d.D, d.S, d.ns, rows);
+    return;
+  }
   if (u_tiled)
     k_embed_pi0<<<rows, 256, d.A * sizeof(float), st>>>(rq, status, Wc, tb, state_tok, h, TiledBf16{u_tiled, rows_pad},
                                                         d.A, d.H, d.D, d.S, d.ns);
