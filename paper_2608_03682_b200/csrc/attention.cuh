@@ -52,6 +52,7 @@ struct AttnArgs {
   float* part_ml;        // [b][head][split][64][2]  (max in log2 units, sum)
   Dims d;
   unsigned wait_limit;
+  const int* order;      // optional: request index of each grid row (batch entries)
 };
 
 // Shared-memory tiles are rows of DH bf16 with no padding; the 16-byte chunk c of row r sits at

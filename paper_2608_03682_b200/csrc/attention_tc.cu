@@ -94,7 +94,8 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
 
   const Dims& d = a.d;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int hp = blockIdx.x, b = blockIdx.y;
+  const int hp = blockIdx.x;
+  const int b = a.order ? a.order[blockIdx.y] : (int)blockIdx.y;   // longest requests first
   const int head0 = hp * 2;
   const int hk = head0 / (d.Hq / d.Hkv);
   const int S = d.S;
@@ -368,7 +369,7 @@ bool attention_tc_supported(const Dims& d) {
 
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, unsigned wait_limit, cudaStream_t st) {
+                                int batch, const int* order, unsigned wait_limit, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(k_attn_tc<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -378,7 +379,7 @@ cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloa
   }
   AttnArgs a{};
   a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
-  a.num_splits = 1, a.d = d, a.wait_limit = wait_limit;
+  a.num_splits = 1, a.d = d, a.wait_limit = wait_limit, a.order = order;
   dim3 grid(d.Hq / 2, batch);
   k_attn_tc<256><<<grid, 288, attn_tc_smem<256>(), st>>>(a);
   return cudaGetLastError();

@@ -103,6 +103,7 @@ struct phyai_expert {
 
   Request* rq = nullptr;
   int* cu_internal = nullptr;
+  int* order = nullptr;        // requests by descending prefix length, rewritten by every batched call
   int* status = nullptr;
 
   std::map<int, Tables> tables;
@@ -376,7 +377,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       }
       if (attn_tc) {
         cudaError_t e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn_t, h->Mpad, d,
-                                            batch, h->wait_limit, st);
+                                            batch, h->order, h->wait_limit, st);
         if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
         ++cnt;
       } else if (h->attn_mma) {
@@ -443,7 +444,7 @@ phyai_status_t run(phyai_expert* h, const Request& r, int n, cudaStream_t st) {
   ST(build_tables(h, n, st, &t));
   if (h->mega_ok && h->use_mega && mega_supported(h->d, r.batch)) ST(mega_prepare(h, r.batch));
   launch_set_request(h->rq, r, h->cu_internal, st);
-  if (r.cu_lens != nullptr) launch_validate(h->rq, h->status, (int)h->cfg.max_prefix_len, st);
+  if (r.cu_lens != nullptr) launch_validate(h->rq, h->status, (int)h->cfg.max_prefix_len, h->order, st);
   const auto key = std::make_pair(r.batch, n);
   if (!h->use_graph) {
     ST(enqueue_loop(h, r.batch, n, *t, st));
@@ -565,6 +566,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
     CU(cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking));
     ST(h->alloc(&h->status, 1, true));
     ST(h->alloc(&h->cu_internal, 2, true));
+    ST(h->alloc(&h->order, (size_t)cfg->max_batch, true));
     ST(h->alloc(&h->rq, 1, true));
     // ---- small tensors -> fp32 ----
     if (need_state) {

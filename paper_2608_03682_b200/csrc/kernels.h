@@ -13,7 +13,7 @@ struct Dims {
 
 // ---- request block ---------------------------------------------------------------------------
 void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st);
-void launch_validate(const Request* rq, int* status, int max_prefix, cudaStream_t st);
+void launch_validate(const Request* rq, int* status, int max_prefix, int* order, cudaStream_t st);
 
 // ---- one-off table / packing kernels (CUDA cores, fp64 accumulation where cheap) ---------------
 // src_kind: 0 = float32, 1 = bfloat16, 2 = e4m3 byte codes
@@ -89,7 +89,7 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
 bool attention_tc_supported(const Dims& d);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, unsigned wait_limit, cudaStream_t st);
+                                int batch, const int* order, unsigned wait_limit, cudaStream_t st);
 
 // ---- tcgen05 GEMM ------------------------------------------------------------------------------
 enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3, TC_QKV_ROT = 4 };

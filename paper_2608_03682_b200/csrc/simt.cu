@@ -25,18 +25,29 @@ void launch_set_request(Request* dst, const Request& src, int* cu_internal, cuda
 }
 
 // cu_prefix_lens must be non-decreasing, start >= 0, end <= kv_tokens, differences <= max_prefix.
-__global__ void k_validate(const Request* rq, int* status, int max_prefix) {
+// Also writes `order`: the requests sorted by descending prefix length (ties by index).  Kernels whose CTAs
+// take one request each walk the batch in this order, so the longest requests start first and the grid's tail is short.
+__global__ void k_validate(const Request* rq, int* status, int max_prefix, int* order) {
   const int B = rq->batch;
   const int* cu = rq->cu_lens;
   bool bad = false;
   for (int b = threadIdx.x; b < B; b += blockDim.x) {
     const int lo = cu[b], hi = cu[b + 1];
     if (lo < 0 || hi < lo || hi - lo > max_prefix || (uint64_t)hi > rq->kv_tokens) bad = true;
+    if (order) {
+      const int len = hi - lo;
+      int rank = 0;
+      for (int c = 0; c < B; ++c) {
+        const int lc = cu[c + 1] - cu[c];
+        rank += (lc > len || (lc == len && c < b)) ? 1 : 0;
+      }
+      order[rank] = b;
+    }
   }
   if (bad) atomicExch(status, ST_INVALID_ARG);
 }
-void launch_validate(const Request* rq, int* status, int max_prefix, cudaStream_t st) {
-  k_validate<<<1, 256, 0, st>>>(rq, status, max_prefix);
+void launch_validate(const Request* rq, int* status, int max_prefix, int* order, cudaStream_t st) {
+  k_validate<<<1, 256, 0, st>>>(rq, status, max_prefix, order);
 }
 
 // =============================================================================================
