@@ -26,6 +26,7 @@ namespace {
 template <int DH>
 __global__ void k_attn_merge(const int* status, const float* part_o, const float* part_ml, __nv_bfloat16* out,
                              int rows_pad, int num_splits, int S, int Hq) {
+  pdl_enter();
   if (status_set(status)) return;
   const int row = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
   const size_t slab0 = ((size_t)(b * Hq + head) * num_splits) * QROWS;
@@ -66,12 +67,13 @@ cudaError_t launch_attn(const AttnArgs& a, int batch, cudaStream_t st) {
     configured = true;
   }
   dim3 grid(a.num_splits, a.d.Hq / HPC, batch);
-  k_attn_mma<DH, HPC, KTT><<<grid, HPC * 128, attn_smem<DH, HPC, KTT>(), st>>>(a);
-  if (a.num_splits > 1) {
+  cudaError_t e = launch_pdl(k_attn_mma<DH, HPC, KTT>, grid, dim3(HPC * 128), attn_smem<DH, HPC, KTT>(), st, a);
+  if (e == cudaSuccess && a.num_splits > 1) {
     dim3 g2(a.d.S, a.d.Hq, batch);
-    k_attn_merge<DH><<<g2, 128, 0, st>>>(a.status, a.part_o, a.part_ml, a.out, a.rows_pad, a.num_splits, a.d.S, a.d.Hq);
+    e = launch_pdl(k_attn_merge<DH>, g2, dim3(128), 0, st, a.status, a.part_o, a.part_ml, a.out, a.rows_pad, a.num_splits,
+                   a.d.S, a.d.Hq);
   }
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace

@@ -358,6 +358,7 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
 template <int DH, int HPC, int KTT>
 __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
+  pdl_enter();
   if (status_set(a.status)) return;   // no wait in this kernel depends on another block: a plain exit is safe
   attn_role<DH, HPC, 2, 0, KTT>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
 }

@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t Ks = base, Vs = Ks + NKV * KV_BYTES;
 
+  pdl_enter();
   if (tid == 0) {
     skip_flag = status_set(a.status) ? 1 : 0;
     abort_flag = 0;
@@ -381,8 +382,7 @@ cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloa
   a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
   a.num_splits = 1, a.d = d, a.wait_limit = wait_limit, a.order = order;
   dim3 grid(d.Hq / 2, batch);
-  k_attn_tc<256><<<grid, 288, attn_tc_smem<256>(), st>>>(a);
-  return cudaGetLastError();
+  return launch_pdl(k_attn_tc<256>, grid, dim3(288), attn_tc_smem<256>(), st, a);
 }
 
 }  // namespace phyai

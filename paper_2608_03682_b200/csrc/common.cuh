@@ -19,6 +19,18 @@ __device__ __forceinline__ bool status_set(const int* status) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  Kernels of the per-operator loop are launched with the "programmatic stream
+// serialization" attribute: the next kernel's CTAs may be scheduled (and run their set-up) while this kernel
+// drains.  Every such kernel calls pdl_enter() before its first global-memory access: it lets its own dependents
+// start early and then waits until the kernels it depends on have completed and their writes are visible.  In a
+// launch without the attribute both instructions are no-ops.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
 // Request block: written by a tiny kernel right before each denoise call, read by every kernel
 // of the loop.  Keeping the per-request pointers and lengths here (not in kernel arguments) lets
 // one captured CUDA graph serve every request of the same (batch, n_steps).

@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   const int kc_end = (int)(((long long)KC * (blockIdx.z + 1)) / gridDim.z);
   const int nk = kc_end - kc_begin;
 
+  pdl_enter();
   if (threadIdx.x == 0) {
     skip_flag = status_set(status) || nk <= 0;
     abort_flag = 0;
@@ -411,8 +412,7 @@ constexpr size_t smem_bytes() {
 template <int NT, int NA, int STAGES>
 cudaError_t launch_one(int* status, const TcGemm& g, cudaStream_t st) {
   dim3 grid(g.N / 128 / (g.epi == TC_GEGLU ? 1 : NA), (g.M + NT - 1) / NT, g.splits > 0 ? g.splits : 1);
-  k_gemm_tc<NT, NA, STAGES><<<grid, 800, smem_bytes<NT, NA, STAGES>(), st>>>(status, g);
-  return cudaGetLastError();
+  return launch_pdl(k_gemm_tc<NT, NA, STAGES>, grid, dim3(800), smem_bytes<NT, NA, STAGES>(), st, status, g);
 }
 
 template <int NT, int NA, int STAGES>

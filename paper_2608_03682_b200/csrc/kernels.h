@@ -3,7 +3,22 @@
 
 #include "common.cuh"
 
+#include <utility>
+
 namespace phyai {
+
+// Launch with programmatic stream serialization (see pdl_enter in common.cuh): only for kernels that call
+// pdl_enter() before touching global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at, cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 
 struct Dims {
   int L, D, F, Hq, Hkv, dh, Ds, A, H, ns, S, Nqkv, Nq;

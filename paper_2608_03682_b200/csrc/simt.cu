@@ -253,6 +253,7 @@ __global__ void __launch_bounds__(256) k_embed_pi0_rows(const Request* rq, const
                                                         const float* tb, const float* state_tok, float* h,
                                                         __nv_bfloat16* u, int rows_pad, int A, int H, int D, int S, int ns,
                                                         int rows_total) {
+  pdl_enter();
   if (status_set(status)) return;
   extern __shared__ float xs[];            // ER x A
   const int r0 = blockIdx.x * ER;
@@ -296,8 +297,8 @@ void launch_embed_pi0(const Request* rq, const int* status, const float* Wc, con
                       cudaStream_t st) {
   const int rows = batch * d.H;
   if (u_tiled && d.D % 4 == 0 && rows >= 4 * ER) {
-    k_embed_pi0_rows<<<(rows + ER - 1) / ER, 256, (size_t)ER * d.A * sizeof(float), st>>>(
-        rq, status, Wc, tb, state_tok, h, u_tiled, rows_pad, d.A, d.H, d.D, d.S, d.ns, rows);
+    launch_pdl(k_embed_pi0_rows, dim3((rows + ER - 1) / ER), dim3(256), (size_t)ER * d.A * sizeof(float), st, rq, status,
+               Wc, tb, state_tok, h, u_tiled, rows_pad, d.A, d.H, d.D, d.S, d.ns, rows);
     return;
   }
   if (u_tiled)
@@ -356,6 +357,7 @@ __global__ void k_rmsnorm(const int* status, const float* h, const float* gain, 
 // float4 loads and 8-byte stores.
 __global__ void k_rmsnorm_tiled4(const int* status, const float* h, const float* gain, const float* shift,
                                  __nv_bfloat16* out, int rows_pad, int M, int D, float eps) {
+  pdl_enter();
   if (status_set(status)) return;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -388,6 +390,7 @@ __global__ void k_rmsnorm_tiled4(const int* status, const float* h, const float*
 template <int NV>
 __global__ void k_rmsnorm_tiled_reg(const int* status, const float* h, const float* gain, const float* shift,
                                     __nv_bfloat16* out, int rows_pad, int M, float eps) {
+  pdl_enter();
   if (status_set(status)) return;
   constexpr int D = NV * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -422,15 +425,15 @@ void launch_rmsnorm(const int* status, const float* h, const float* gain, const 
                     __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st) {
   const int blocks = (M + 3) / 4;
   if (out_tiled && D == 1024) {
-    k_rmsnorm_tiled_reg<8><<<blocks, 128, 0, st>>>(status, h, gain, shift, out_tiled, rows_pad, M, eps);
+    launch_pdl(k_rmsnorm_tiled_reg<8>, dim3(blocks), dim3(128), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps);
     return;
   }
   if (out_tiled && D == 2048) {
-    k_rmsnorm_tiled_reg<16><<<blocks, 128, 0, st>>>(status, h, gain, shift, out_tiled, rows_pad, M, eps);
+    launch_pdl(k_rmsnorm_tiled_reg<16>, dim3(blocks), dim3(128), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps);
     return;
   }
   if (out_tiled && D % 128 == 0) {
-    k_rmsnorm_tiled4<<<blocks, 128, 0, st>>>(status, h, gain, shift, out_tiled, rows_pad, M, D, eps);
+    launch_pdl(k_rmsnorm_tiled4, dim3(blocks), dim3(128), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, D, eps);
     return;
   }
   if (out_tiled)
@@ -450,6 +453,7 @@ constexpr int FR = 16;
 __global__ void __launch_bounds__(256) k_final(const Request* rq, const int* status, const float* h, const float* gain,
                                                const float* shift, const float* Wout, const float* bout, float dt, int A,
                                                int H, int D, int S, int ns, float eps, int rows_total) {
+  pdl_enter();
   if (status_set(status)) return;
   extern __shared__ float nrm[];            // FR x D, then 8 x FR x 32 partial sums
   float* part = nrm + (size_t)FR * D;
@@ -523,8 +527,8 @@ void launch_final(const Request* rq, const int* status, const float* h, const fl
     cudaFuncSetAttribute(k_final, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
     configured = true;
   }
-  k_final<<<(rows + FR - 1) / FR, 256, ((size_t)FR * d.D + 8 * FR * 32) * sizeof(float), st>>>(rq, status, h, gain, shift, Wout, bout, dt,
-                                                                               d.A, d.H, d.D, d.S, d.ns, d.eps, rows);
+  launch_pdl(k_final, dim3((rows + FR - 1) / FR), dim3(256), ((size_t)FR * d.D + 8 * FR * 32) * sizeof(float), st, rq, status,
+             h, gain, shift, Wout, bout, dt, d.A, d.H, d.D, d.S, d.ns, d.eps, rows);
 }
 
 // =============================================================================================
