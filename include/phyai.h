@@ -192,10 +192,13 @@ phyai_status_t phyai_denoise_batched_host(phyai_expert_t *h, uint32_t batch, con
 phyai_status_t phyai_poll_status(phyai_expert_t *h);
 
 /* Options. key "use_graph": 0 launches the kernels directly, 1 (default) replays a captured CUDA
- * graph per (batch, n_steps).  key "use_persistent": 1 (default) runs calls with batch * suffix_len
- * <= 64 tokens as one persistent cooperative kernel (the whole n-step loop, no kernel boundaries),
- * 0 uses the per-operator kernels for every batch.  key "use_tc_attention": 1 (default) lets large
- * batches use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "use_pair_gemm": 1 runs the
+ * graph per (batch, n_steps).  key "use_persistent": 1 runs calls with batch * suffix_len <= 64
+ * tokens as one persistent cooperative kernel (the whole n-step loop, no kernel boundaries; bit-reproducible run
+ * to run), 0 (default) uses the per-operator kernels, captured as one CUDA graph, for every batch: with
+ * programmatic dependent launch they measured faster than the persistent kernel.  key "use_tc_attention": 1 (default) lets large
+ * batches use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "use_cluster_attention": 1 (default) lets calls with few
+ * requests merge their key-split attention partials through distributed shared memory (clusters of 8 CTAs), 0
+ * keeps the split kernel + merge kernel.  key "use_pair_gemm": 1 runs the
  * GEMMs of batches above 1024 tokens on CTA pairs (tcgen05 cta_group::2, persistent, overlapped epilogue), 0
  * (default) keeps the single-CTA kernel, which measured faster on the batch-64 shapes.
  * key "wait_limit": iteration bound of

@@ -76,7 +76,46 @@ cudaError_t launch_attn(const AttnArgs& a, int batch, cudaStream_t st) {
   return e;
 }
 
+template <int DH, int KTT>
+constexpr size_t attn_cluster_smem() {   // Q / K / V buffers + the receive area of the push merge
+  return attn_smem<DH, 1, KTT>() + (size_t)8 * 8 * (DH + 4) * 4 + 512;
+}
+
+template <int DH, int KTT>
+cudaError_t launch_attn_cluster(const AttnArgs& a, int batch, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_attn_cluster<DH, KTT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)attn_cluster_smem<DH, KTT>());
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(8, a.d.Hq, batch), cfg.blockDim = dim3(128), cfg.dynamicSmemBytes = attn_cluster_smem<DH, KTT>(), cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 8, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at, cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, k_attn_cluster<DH, KTT>, a);
+}
+
 }  // namespace
+
+// Key-split attention whose partials are merged through distributed shared memory (clusters of 8 CTAs).
+cudaError_t launch_attention_cluster(const Request* rq, int* status, const float* qkv, const float2* rope,
+                                     const __nv_bfloat16* qr, const __nv_bfloat16* kr, const __nv_bfloat16* vr, int layer,
+                                     __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
+                                     cudaStream_t st) {
+  AttnArgs a{};
+  a.rq = rq, a.status = status, a.qkv = qkv, a.rope = rope, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
+  a.qr = qr, a.kr = kr, a.vr = vr;   // when set: rotated bf16 operands instead of the fp32 QKV output
+  a.num_splits = 8, a.d = d, a.wait_limit = wait_limit;
+  if (d.dh == 256) return launch_attn_cluster<256, 64>(a, batch, st);
+  if (d.dh == 128) return launch_attn_cluster<128, 64>(a, batch, st);
+  return launch_attn_cluster<64, 64>(a, batch, st);
+}
 
 bool attention_mma_supported(const Dims& d) {
   return (d.dh == 64 || d.dh == 128 || d.dh == 256) && d.S <= QROWS;

@@ -81,7 +81,11 @@ __device__ __forceinline__ void group_sync() {
 // `smem_base` (128-byte aligned): (HPC*64 + 2*NBUF*KTT) rows of DH bf16.  When a.qr is set, q / k / v of
 // the suffix are read as bf16, already rotated and scaled (written by the QKV epilogue of the
 // persistent kernel); otherwise they are taken from the fp32 QKV output and rotated here.
-template <int DH, int HPC, int NBUF, int BAR, int KTT>
+// CLUSTER (HPC = 1): the num_splits = 8 key ranges of a head are the 8 CTAs of a thread-block cluster; each pushes
+// the rows of its partial (O, max, sum) into the shared memory of the CTA that owns them (distributed shared
+// memory stores) and, after one cluster barrier, merges its own 8 of the 64 rows: no partials in global memory, no
+// merge kernel.  Needs 8 * 8 * (DH + 4) * 4 + 512 bytes of shared memory beyond the Q / K / V buffers.
+template <int DH, int HPC, int NBUF, int BAR, int KTT, bool CLUSTER = false>
 __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp, int b, uint32_t smem_base, int tid) {
   constexpr int ROWB = DH * 2;                // bytes per row
   constexpr int CH = DH / 8;                  // 16-byte chunks per row
@@ -325,7 +329,68 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
   l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
   const int head = head0 + hl;
-  if (a.num_splits == 1) {
+  if constexpr (CLUSTER) {
+    // Push merge: CTA `rank` of the cluster owns rows [8 * rank, 8 * rank + 8).  Every CTA stores its partial rows
+    // (and their max / sum) straight into the owners' shared memory (remote stores, fire and forget), into a
+    // receive area beyond the Q / K / V buffers, which the owner may still be using.  After one cluster barrier
+    // each CTA merges its 8 rows from its own shared memory.
+    constexpr int PP = DH + 4;                       // row pitch in floats
+    const uint32_t recv = smem_base + (uint32_t)(HPC * QROWS + 2 * NBUF * KTT) * ROWB;   // [8 sources][8 rows][PP]
+    const uint32_t recv_ml = recv + 8u * 8u * PP * 4u;                                   // [8 sources][8 rows][2]
+    {
+      uint32_t d0, d1, m0a, m1a;
+      const uint32_t o0 = (uint32_t)((split * 8 + (row0 & 7)) * PP) * 4, o1 = (uint32_t)((split * 8 + (row1 & 7)) * PP) * 4;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(d0) : "r"(recv + o0), "r"(row0 >> 3));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(d1) : "r"(recv + o1), "r"(row1 >> 3));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(m0a) : "r"(recv_ml + (uint32_t)(split * 8 + (row0 & 7)) * 8), "r"(row0 >> 3));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(m1a) : "r"(recv_ml + (uint32_t)(split * 8 + (row1 & 7)) * 8), "r"(row1 >> 3));
+#pragma unroll
+      for (int n = 0; n < DH / 8; ++n) {
+        const uint32_t col = (uint32_t)(n * 8 + qd * 2) * 4;
+        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d0 + col), "f"(o[n][0]), "f"(o[n][1]) : "memory");
+        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d1 + col), "f"(o[n][2]), "f"(o[n][3]) : "memory");
+      }
+      if (qd == 0) {
+        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m0a), "f"(m0), "f"(l0) : "memory");
+        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m1a), "f"(m1), "f"(l1) : "memory");
+      }
+    }
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    constexpr int CPT = DH / 16;                                  // columns per thread: 16 threads cover a row
+    const int rl = tid >> 4, r = split * 8 + rl, c0 = (tid & 15) * CPT;
+    if (r < S) {
+      float ms[8], ls[8], mm = -INFINITY;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(ms[s]), "=f"(ls[s]) : "r"(recv_ml + (uint32_t)(s * 8 + rl) * 8) : "memory");
+        mm = fmaxf(mm, ms[s]);
+      }
+      float acc[CPT], ll = 0.f;
+#pragma unroll
+      for (int e = 0; e < CPT; ++e) acc[e] = 0.f;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        if (ms[s] == -INFINITY) continue;
+        const float w = exp2f(ms[s] - mm);
+        ll = fmaf(w, ls[s], ll);
+#pragma unroll
+        for (int u = 0; u < CPT / 4; ++u) {
+          float4 v;
+          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                       : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                       : "r"(recv + (uint32_t)((s * 8 + rl) * PP + c0 + 4 * u) * 4)
+                       : "memory");
+          acc[4 * u] = fmaf(w, v.x, acc[4 * u]), acc[4 * u + 1] = fmaf(w, v.y, acc[4 * u + 1]);
+          acc[4 * u + 2] = fmaf(w, v.z, acc[4 * u + 2]), acc[4 * u + 3] = fmaf(w, v.w, acc[4 * u + 3]);
+        }
+      }
+      const float inv = 1.0f / ll;
+#pragma unroll
+      for (int u = 0; u < CPT / 4; ++u)     // 4 consecutive columns = 8 bytes, inside one 16-byte chunk of the tiled layout
+        *reinterpret_cast<uint2*>(a.out + out_index(b * S + r, head * DH + c0 + 4 * u, a.rows_pad, d.Nq)) =
+            make_uint2(pack_bf16(acc[4 * u] * inv, acc[4 * u + 1] * inv), pack_bf16(acc[4 * u + 2] * inv, acc[4 * u + 3] * inv));
+    }
+  } else if (a.num_splits == 1) {
     const float i0 = 1.0f / l0, i1 = 1.0f / l1;
 #pragma unroll
     for (int n = 0; n < DH / 8; ++n) {
@@ -361,6 +426,15 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
   pdl_enter();
   if (status_set(a.status)) return;   // no wait in this kernel depends on another block: a plain exit is safe
   attn_role<DH, HPC, 2, 0, KTT>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
+}
+
+// Cluster variant: grid (8, heads, requests), cluster (8, 1, 1); see attn_role.
+template <int DH, int KTT>
+__global__ void __launch_bounds__(128, 1) k_attn_cluster(const AttnArgs a) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  pdl_enter();
+  if (status_set(a.status)) return;   // the word is only written by kernels that completed before this one started
+  attn_role<DH, 1, 2, 0, KTT, true>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
 }
 
 }  // namespace

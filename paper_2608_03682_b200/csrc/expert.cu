@@ -84,8 +84,9 @@ struct phyai_expert {
 
   // persistent loop kernel (batch * suffix_len <= 64)
   bool mega_ok = false;
-  int use_mega = 1;
+  int use_mega = 0;   // the captured per-operator loop measured faster (10.0 vs 12.6 ms on the pi0-shaped expert): opt-in
   int use_tc_attention = 1;
+  int use_cluster_attention = 1;
   int use_pair_gemm = 0;   // measured slower than the single-CTA kernel on the batch-64 shapes: opt-in
   int n_sm = 0;
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
@@ -103,6 +104,8 @@ struct phyai_expert {
 
   Request* rq = nullptr;
   int* cu_internal = nullptr;
+  int slab_splits = 8;         // most k-ranges a residual GEMM is split into when its partials go to slabs
+  float* slab = nullptr;       // [MAX_SLABS][64][width] split-K partials of the residual GEMMs (one token tile)
   int* order = nullptr;        // requests by descending prefix length, rewritten by every batched call
   int* status = nullptr;
 
@@ -212,6 +215,11 @@ phyai_status_t build_tables(phyai_expert* h, int n, cudaStream_t st, Tables** ou
 // ---------------------------------------------------------------------------------------------
 // the loop: launches of one denoise call (x <- noise; n x [embed, L layers, head + Euler])
 // ---------------------------------------------------------------------------------------------
+// The tcgen05 attention kernel walks all keys of a request in one CTA per pair of query heads (no key split, no
+// merge pass): from this many CTAs on it beats the split mma.sync kernel + merge.
+constexpr int ATTN_TC_MIN_CTAS = 8;
+constexpr int MAX_SLABS = 16;
+
 int pick_nt(int M) { return M <= 64 ? 64 : (M <= 1024 ? 128 : 256); }
 
 // Token-tile width and split-K factor of a residual GEMM (N = width, large token counts): the pair that minimises
@@ -304,8 +312,20 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       *gain = h->gains + (size_t)s * D, *shift = nullptr, *gate = nullptr;
     }
   };
+  // Split-K partial sums of the residual GEMMs at one token tile go to slabs that the next reader of h (a norm or
+  // the velocity head) adds in a fixed order: no atomics, so a request gives the same bits every time.
+  int pending_slabs = 0;
+  auto take_slabs = [&]() {
+    SlabSum sl{h->slab, pending_slabs, (size_t)M * D};
+    pending_slabs = 0;
+    return sl;
+  };
   auto tc_gemm = [&](TcGemm g) -> phyai_status_t {
     g.rows_pad = h->Mpad, g.M = g.M ? g.M : M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact;
+    if (g.epi == TC_RESID && g.splits > 1 && nt == 64 && h->slab && D <= 2048) {
+      if (g.splits > h->slab_splits) g.splits = h->slab_splits;
+      g.slab = h->slab, pending_slabs = g.splits;
+    }
     cudaError_t e;
     TcGemm gp = g;
     gp.splits = 1;   // the CTA-pair kernel never splits K
@@ -354,17 +374,19 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     for (int l = 0; l < d.L; ++l) {
       const float *gain, *shift, *gate;
       site(k, 2 * l, &gain, &shift, &gate);
-      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st);
+      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs());
       ++cnt;
       const bool attn_tc = h->attn_mma && h->use_tc_attention && h->qr_big && attention_tc_supported(d) &&
-                           batch * (d.Hq / 2) >= 100;
+                           batch * (d.Hq / 2) >= ATTN_TC_MIN_CTAS;
+      const bool attn_cluster = !attn_tc && h->attn_mma && h->use_cluster_attention && batch * d.Hq * 8 <= 2 * h->n_sm;
+      const bool attn_rot = h->qr_big && (attn_tc || attn_cluster);   // q / k / v leave the QKV epilogue rotated, bf16
       if (h->tc) {
         TcGemm g{};
         g.W = h->p_qkv[l], g.X = h->xn_t, g.N = d.Nqkv, g.K = D, g.epi = TC_STORE, g.scale = h->s_qkv[l];
         g.perm_dh = d.dh, g.perm_end = d.Nq + d.Hkv * d.dh;
         g.out_f32 = h->qkv, g.ldo = d.Nqkv, g.splits = 1;
-        if (attn_tc) {
-          // the tcgen05 attention kernel takes its operands rotated, scaled and rounded from this epilogue
+        if (attn_rot) {
+          // these attention kernels take their operands rotated, scaled and rounded from this epilogue
           g.epi = TC_QKV_ROT, g.rq = h->rq, g.rope = h->rope, g.qr = h->qr_big, g.kr = h->kr_big, g.vr = h->vr_big;
           g.S = d.S, g.Hq = d.Hq, g.Hkv = d.Hkv, g.dh = d.dh;
         }
@@ -378,6 +400,12 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       if (attn_tc) {
         cudaError_t e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn_t, h->Mpad, d,
                                             batch, h->order, h->wait_limit, st);
+        if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
+        ++cnt;
+      } else if (attn_cluster) {
+        // few requests: 8 key ranges per head in a cluster of 8 CTAs, merged through distributed shared memory
+        cudaError_t e = launch_attention_cluster(h->rq, h->status, h->qkv, h->rope, attn_rot ? h->qr_big : nullptr, h->kr_big,
+                                                 h->vr_big, l, h->attn_t, h->Mpad, d, batch, h->wait_limit, st);
         if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
         ++cnt;
       } else if (h->attn_mma) {
@@ -404,12 +432,16 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         simt_gemm(g);
       }
       site(k, 2 * l + 1, &gain, &shift, &gate);
-      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st);
+      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs());
       ++cnt;
       if (h->tc) {
         TcGemm g{};
         g.W = h->p_g[l], g.W2 = h->p_u[l], g.X = h->xn_t, g.N = d.F, g.K = D, g.epi = TC_GEGLU;
         g.scale = h->s_g[l], g.scale2 = h->s_u[l], g.out_tiled = h->m_t, g.splits = 1;
+        if (nt == 64 && h->p_gu_all) {
+          // a single token tile: interleaved gate / up tiles put the weight stream on twice as many SMs
+          g.W = h->p_gu_all + (size_t)l * D * 2 * d.F, g.W2 = nullptr, g.N = 2 * d.F, g.epi = TC_GEGLU_IL;
+        }
         ST(tc_gemm(g));
         TcGemm g2{};
         g2.W = h->p_d[l], g2.X = h->m_t, g2.N = D, g2.K = d.F, g2.epi = TC_RESID, g2.scale = h->s_d[l], g2.gate = gate;
@@ -430,6 +462,10 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     // ---- final norm, velocity head, Euler update ----
     const float *gain, *shift, *gate;
     site(k, 2 * d.L, &gain, &shift, &gate);
+    if (pending_slabs) {
+      launch_add_slabs(h->status, h->h, M, D, st, take_slabs());
+      ++cnt;
+    }
     launch_final(h->rq, h->status, h->h, gain, shift, h->Wout, h->bout, dt, d, batch, st);
     ++cnt;
   }
@@ -566,6 +602,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
     CU(cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking));
     ST(h->alloc(&h->status, 1, true));
     ST(h->alloc(&h->cu_internal, 2, true));
+    if (tc) ST(h->alloc(&h->slab, (size_t)MAX_SLABS * 64 * D, true));
     ST(h->alloc(&h->order, (size_t)cfg->max_batch, true));
     ST(h->alloc(&h->rq, 1, true));
     // ---- small tensors -> fp32 ----
@@ -708,7 +745,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
     // ---- workspace (zeroed: padding rows of the tiled buffers stay finite) ----
     ST(h->alloc(&h->h, Mp * D, true));
     ST(h->alloc(&h->qkv, Mp * Nqkv, true));
-    if (tc && attention_tc_supported(d) && (int)cfg->max_batch * (d.Hq / 2) >= 100) {
+    if (tc && (d.dh == 128 || d.dh == 256)) {   // rotated bf16 q / k / v for the tcgen05 and cluster attention kernels
       ST(h->alloc(&h->qr_big, Mp * d.Nq, true));
       ST(h->alloc(&h->kr_big, Mp * (size_t)(d.Hkv * d.dh), true));
       ST(h->alloc(&h->vr_big, Mp * (size_t)(d.Hkv * d.dh), true));
@@ -903,6 +940,19 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   }
   if (!strcmp(key, "use_tc_attention")) {
     h->use_tc_attention = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "slab_splits")) {
+    if (value < 1 || value > MAX_SLABS) return fail(PHYAI_ERR_INVALID_ARG, "slab_splits out of range");
+    h->slab_splits = (int)value;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_cluster_attention")) {
+    h->use_cluster_attention = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

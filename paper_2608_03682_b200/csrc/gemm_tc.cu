@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     constexpr int HALF = NT / 4;   // token columns per epilogue warp
     const int c_begin = hf * HALF;
     const bool resid_red = g.epi == TC_RESID && gridDim.z > 1;   // split-K: vector reductions, see below
-    if (ok && !geglu && g.epi != TC_QKV_ROT && !resid_red) {
+    if (ok && !geglu && g.epi != TC_QKV_ROT && g.epi != TC_GEGLU_IL && !resid_red) {
 #pragma unroll
       for (int a = 0; a < NA; ++a) {
         const int n = (nt_idx * NA + a) * 128 + ch;   // packed output channel
@@ -225,6 +225,47 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         }
       }
     }
+    if (g.epi == TC_GEGLU_IL) {
+      // One 128-row tile = 64 gate channels (rows 0..63) and the matching 64 up channels (rows 64..127): twice as
+      // many CTAs stream the gate / up weights as with separate 128-row gate and up tiles, which is what matters
+      // when there is a single token tile.  The up half goes through shared memory to the gate half, which writes
+      // the bf16 result as the swizzled image of k-chunk `tile` of the down projection's input.
+      float* stage = reinterpret_cast<float*>(tiles_ptr);                                  // [NT][64] up values
+      __nv_bfloat16* img = reinterpret_cast<__nv_bfloat16*>(stage + (size_t)NT * 64);      // [NT][64] bf16, swizzled
+      const int c64 = ch & 63, f = nt_idx * 64 + c64;
+      if (ok && q >= 2) {
+        const float su = g.scale2 ? g.scale2[f] : 1.0f;
+        for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
+          if (tok_base + c0 >= g.M) break;
+          float v[16];
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * 64 + c64] = v[j] * su;
+        }
+      }
+      epi_sync();
+      if (ok && q < 2) {
+        const float sg = g.scale ? g.scale[f] : 1.0f;
+        for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
+          if (tok_base + c0 >= g.M) break;
+          float v[16];
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int t = c0 + j;
+            const float m = gelu_fast(v[j] * sg, g.gelu_exact) * stage[(size_t)t * 64 + c64];
+            img[(size_t)t * 64 + (((c64 >> 3) ^ (t & 7)) << 3) + (c64 & 7)] = __float2bfloat16_rn(m);
+          }
+        }
+      }
+      epi_sync();
+      if (ok) {
+        const int rows = min(NT, g.M - tok_base);
+        uint4* dst = reinterpret_cast<uint4*>(g.out_tiled + ((size_t)nt_idx * g.rows_pad + tok_base) * 64);
+        const uint4* src = reinterpret_cast<const uint4*>(img);
+        for (int idx = et; idx < rows * 8; idx += NEPI) dst[idx] = src[idx];
+      }
+    }
     if (resid_red) {
       // Split-K residual: every k-range adds its partial tile to h.  The tile is transposed through shared memory
       // (fp32 [token][128 + 4]) so that one thread adds 4 consecutive channels of one token with a single
@@ -250,6 +291,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
           for (int it = et; it < rows * 32; it += NEPI) {
             const int tl = it >> 5, j0 = (it & 31) * 4;
             const float4 x = *reinterpret_cast<const float4*>(stage + (size_t)tl * PITCH + j0);
+            if (g.slab) {   // deterministic variant: plain stores of this k-range's partial
+              *reinterpret_cast<float4*>(g.slab + ((size_t)blockIdx.z * g.M + tok_base + tl) * g.ldo + n0 + j0) = x;
+              continue;
+            }
             float* dst = g.out_f32 + (size_t)(tok_base + tl) * g.ldo + n0 + j0;
             asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w)
                          : "memory");
@@ -439,7 +484,7 @@ cudaError_t tc_gemm_setup() {
 // tiles per CTA when the token tile is 256 wide and the channel count allows it (halves the
 // activation traffic per MMA), else one.
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st) {
-  bool two = g.epi == TC_GEGLU || (nt >= 192 && g.N % 256 == 0);
+  bool two = g.epi == TC_GEGLU || (nt >= 192 && g.N % 256 == 0 && g.epi != TC_GEGLU_IL);
   // a plain store epilogue cannot split K: when two-tile CTAs would leave more than half of the SMs idle, take one
   // channel tile per CTA instead
   if (g.epi == TC_BIAS_ROWMAP && nt == 256 && (g.N / 256) * ((g.M + 255) / 256) <= 74) two = false;

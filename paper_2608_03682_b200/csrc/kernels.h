@@ -66,11 +66,22 @@ void launch_embed_pi0(const Request* rq, const int* status, const float* Wc, con
 void launch_embed_pi05(const Request* rq, const int* status, const float* Wa, const float* ba, const float* state_tok,
                        float* h, const Dims& d, int batch, cudaStream_t st);
 // n = h * rsqrt(mean h^2 + eps) * gain + shift  -> fp32 row-major or tiled bf16
-void launch_rmsnorm(const int* status, const float* h, const float* gain, const float* shift, float* out_f32,
-                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st);
+// Pending split-K partial sums of the residual stream: n slabs of [M][D] floats, `stride` floats apart.  The kernel
+// that reads h next adds them to each row in slab order (a fixed order: results are reproducible run to run) and,
+// for the norms, writes the row back.
+struct SlabSum {
+  const float* slab;
+  int n;
+  size_t stride;
+};
+void launch_rmsnorm(const int* status, float* h, const float* gain, const float* shift, float* out_f32,
+                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st,
+                    SlabSum slabs = SlabSum{nullptr, 0, 0});
 // final norm -> out-proj -> Euler update x += dt * (v + bout)
 void launch_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
                   const float* Wout, const float* bout, float dt, const Dims& d, int batch, cudaStream_t st);
+// h[row] += pending slabs (no-op when there are none)
+void launch_add_slabs(const int* status, float* h, int M, int D, cudaStream_t st, SlabSum slabs);
 
 // ---- CUDA-core GEMM (fp32 FMA) -----------------------------------------------------------------
 enum : int { EPI_STORE = 0, EPI_SWISH = 1, EPI_RESID = 2, EPI_GEGLU = 3 };
@@ -102,12 +113,16 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
 
 // ---- tcgen05 attention (large batches: two heads per CTA, whole key range, no split) ------------------
 bool attention_tc_supported(const Dims& d);
+cudaError_t launch_attention_cluster(const Request* rq, int* status, const float* qkv, const float2* rope,
+                                     const __nv_bfloat16* qr, const __nv_bfloat16* kr, const __nv_bfloat16* vr, int layer,
+                                     __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
+                                     cudaStream_t st);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
                                 int batch, const int* order, unsigned wait_limit, cudaStream_t st);
 
 // ---- tcgen05 GEMM ------------------------------------------------------------------------------
-enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3, TC_QKV_ROT = 4 };
+enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3, TC_QKV_ROT = 4, TC_GEGLU_IL = 5 };
 struct TcGemm {
   const __nv_bfloat16* W;   // packed blocks [N/128][KC][128x64]
   const __nv_bfloat16* W2;  // second matrix (GeGLU "up"), same packing, or null
@@ -119,10 +134,13 @@ struct TcGemm {
   const float* bias;   // TC_BIAS_ROWMAP
   const float* gate;   // TC_RESID (null = 1)
   float* out_f32; int ldo;          // TC_STORE / TC_RESID / TC_BIAS_ROWMAP
-  __nv_bfloat16* out_tiled;         // TC_GEGLU: [N/64][rows_pad][64]
+  __nv_bfloat16* out_tiled;         // TC_GEGLU: [N/64][rows_pad][64]; TC_GEGLU_IL: W holds gate and up interleaved in groups
+                                    // of 64 channels (N = 2 x mlp_dim packed rows), one 64-channel k-chunk of output per tile
   int rows_in, rows_out, row_off;   // TC_BIAS_ROWMAP row remap
   int gelu_exact;
   int splits;                       // split-K factor (TC_RESID only)
+  float* slab;                      // TC_RESID with splits > 1: when set, k-range z stores its partial tile to
+                                    // slab[z][M][ldo] (summed by the next reader of h) instead of reducing into out_f32
   int nt_override;                  // host side: token-tile width chosen for this GEMM (0 = the caller's default)
   int perm_dh, perm_end;            // TC_STORE: packed rows < perm_end map to channels by qkv_packed_to_channel
   // TC_QKV_ROT: the fused q|k|v projection (rows packed by qkv_channel_to_packed) leaves the kernel as the

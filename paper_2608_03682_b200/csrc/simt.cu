@@ -355,17 +355,24 @@ __global__ void k_rmsnorm(const int* status, const float* h, const float* gain, 
 }
 // Vectorised variant for the tensor path: D a multiple of 128, tiled bf16 output, one warp per row,
 // float4 loads and 8-byte stores.
-__global__ void k_rmsnorm_tiled4(const int* status, const float* h, const float* gain, const float* shift,
-                                 __nv_bfloat16* out, int rows_pad, int M, int D, float eps) {
+__global__ void k_rmsnorm_tiled4(const int* status, float* h, const float* gain, const float* shift,
+                                 __nv_bfloat16* out, int rows_pad, int M, int D, float eps, SlabSum sl) {
   pdl_enter();
   if (status_set(status)) return;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
-  const float* x = h + (size_t)row * D;
+  float* x = h + (size_t)row * D;
   float ss = 0.f;
   for (int d = lane * 4; d < D; d += 128) {
-    const float4 v = *reinterpret_cast<const float4*>(x + d);
+    float4 v = *reinterpret_cast<const float4*>(x + d);
+    if (sl.n) {   // add the pending split-K partials in slab order and keep the sum (re-read below by this thread)
+      for (int s = 0; s < sl.n; ++s) {
+        const float4 p = *reinterpret_cast<const float4*>(sl.slab + (size_t)s * sl.stride + (size_t)row * D + d);
+        v.x += p.x, v.y += p.y, v.z += p.z, v.w += p.w;
+      }
+      *reinterpret_cast<float4*>(x + d) = v;
+    }
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = warp_sum(ss);
@@ -388,18 +395,30 @@ __global__ void k_rmsnorm_tiled4(const int* status, const float* h, const float*
 // Same, with the whole row held in registers (D = NV * 128): every load of the row is in flight at once and the
 // row is read once.
 template <int NV>
-__global__ void k_rmsnorm_tiled_reg(const int* status, const float* h, const float* gain, const float* shift,
-                                    __nv_bfloat16* out, int rows_pad, int M, float eps) {
+__global__ void k_rmsnorm_tiled_reg(const int* status, float* h, const float* gain, const float* shift,
+                                    __nv_bfloat16* out, int rows_pad, int M, float eps, SlabSum sl) {
   pdl_enter();
   if (status_set(status)) return;
   constexpr int D = NV * 128;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
-  const float* x = h + (size_t)row * D;
+  float* x = h + (size_t)row * D;
   float4 v[NV];
 #pragma unroll
   for (int k = 0; k < NV; ++k) v[k] = *reinterpret_cast<const float4*>(x + k * 128 + lane * 4);
+  if (sl.n) {   // add the pending split-K partials in slab order and write the row back
+    for (int s = 0; s < sl.n; ++s) {
+      const float* p = sl.slab + (size_t)s * sl.stride + (size_t)row * D + lane * 4;
+#pragma unroll
+      for (int k = 0; k < NV; ++k) {
+        const float4 q = __ldg(reinterpret_cast<const float4*>(p + k * 128));
+        v[k].x += q.x, v[k].y += q.y, v[k].z += q.z, v[k].w += q.w;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < NV; ++k) *reinterpret_cast<float4*>(x + k * 128 + lane * 4) = v[k];
+  }
   float ss = 0.f;
 #pragma unroll
   for (int k = 0; k < NV; ++k) ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
@@ -421,19 +440,68 @@ __global__ void k_rmsnorm_tiled_reg(const int* status, const float* h, const flo
   }
 }
 
-void launch_rmsnorm(const int* status, const float* h, const float* gain, const float* shift, float* out_f32,
-                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st) {
-  const int blocks = (M + 3) / 4;
+// Row update with pending split-K partials: h[row] += slab_0[row] + slab_1[row] + ... (that order), optionally
+// followed by the norm into the tiled bf16 layout.  One block per row, one float4 per thread (D / 4 threads): the
+// slab loads of a thread are independent, so they are all in flight together.
+__global__ void __launch_bounds__(512) k_add_slabs_norm(const int* status, float* h, const float* gain, const float* shift,
+                                                        __nv_bfloat16* out, int rows_pad, int D, float eps, SlabSum sl) {
+  pdl_enter();
+  if (status_set(status)) return;
+  __shared__ float red[16];
+  const int row = blockIdx.x, t = threadIdx.x, d = t * 4;
+  float* x = h + (size_t)row * D + d;
+  float4 v = *reinterpret_cast<const float4*>(x);
+  const float* p = sl.slab + (size_t)row * D + d;
+#pragma unroll 8
+  for (int s = 0; s < sl.n; ++s) {
+    const float4 q = __ldg(reinterpret_cast<const float4*>(p + (size_t)s * sl.stride));
+    v.x += q.x, v.y += q.y, v.z += q.z, v.w += q.w;
+  }
+  *reinterpret_cast<float4*>(x) = v;
+  if (!out) return;
+  float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
+  if ((t & 31) == 0) red[t >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];   // same order in every thread
+  const float r = 1.0f / sqrtf(tot / (float)D + eps);
+  const float4 g = __ldg(reinterpret_cast<const float4*>(gain + d));
+  float4 o = make_float4(v.x * r * g.x, v.y * r * g.y, v.z * r * g.z, v.w * r * g.w);
+  if (shift) {
+    const float4 s4 = __ldg(reinterpret_cast<const float4*>(shift + d));
+    o.x += s4.x, o.y += s4.y, o.z += s4.z, o.w += s4.w;
+  }
+  __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+  uint2 pk;
+  pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(out + tiled_index(row, d, rows_pad)) = pk;
+}
+// h += pending slabs, nothing else (before the velocity head)
+void launch_add_slabs(const int* status, float* h, int M, int D, cudaStream_t st, SlabSum sl) {
+  if (!sl.n) return;
+  launch_pdl(k_add_slabs_norm, dim3(M), dim3(D / 4), 0, st, status, h, (const float*)nullptr, (const float*)nullptr,
+             (__nv_bfloat16*)nullptr, 0, D, 0.0f, sl);
+}
+
+void launch_rmsnorm(const int* status, float* h, const float* gain, const float* shift, float* out_f32,
+                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st, SlabSum sl) {
+  if (sl.n && out_tiled && D % 128 == 0 && D <= 2048) {
+    launch_pdl(k_add_slabs_norm, dim3(M), dim3(D / 4), 0, st, status, h, gain, shift, out_tiled, rows_pad, D, eps, sl);
+    return;
+  }
+  // with pending slabs a row costs several times more reads: one warp per block spreads the rows over more SMs
+  const int wpb = sl.n ? 1 : 4;
+  const int blocks = (M + wpb - 1) / wpb;
   if (out_tiled && D == 1024) {
-    launch_pdl(k_rmsnorm_tiled_reg<8>, dim3(blocks), dim3(128), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps);
+    launch_pdl(k_rmsnorm_tiled_reg<8>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl);
     return;
   }
   if (out_tiled && D == 2048) {
-    launch_pdl(k_rmsnorm_tiled_reg<16>, dim3(blocks), dim3(128), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps);
+    launch_pdl(k_rmsnorm_tiled_reg<16>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl);
     return;
   }
   if (out_tiled && D % 128 == 0) {
-    launch_pdl(k_rmsnorm_tiled4, dim3(blocks), dim3(128), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, D, eps);
+    launch_pdl(k_rmsnorm_tiled4, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, D, eps, sl);
     return;
   }
   if (out_tiled)
