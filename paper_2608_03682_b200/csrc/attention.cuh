@@ -129,6 +129,20 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
   };
   if (t_begin < t_end && t_begin < Tp) load_tile(t_begin, 0);
   cp_async_commit();
+  bool early2 = false;   // second key tile requested before the dependency wait (cluster variant)
+  if constexpr (CLUSTER && NBUF == 2) {
+    if (t_begin + 1 < t_end && t_begin + 1 < Tp) load_tile(t_begin + 1, 1), early2 = true;
+    cp_async_commit();
+  }
+  if constexpr (CLUSTER) {
+    // Programmatic dependent launch: the request block and the prefix K/V were complete before this grid could
+    // start, so the first key tile is already on its way; q / k / v of the suffix come from the kernel before.
+    pdl_wait();
+    if (status_set(a.status)) {   // same answer in every CTA of the cluster (all earlier kernels have completed)
+      cp_async_wait<0>();
+      return;
+    }
+  }
 
   if (a.qr) {
     // ---- Q rows are ready-made bf16: straight asynchronous copies (rows past the suffix are zero-filled)
@@ -188,7 +202,7 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
     const uint32_t Kb = Ks + (uint32_t)buf * KTT * ROWB, Vb = Vs + (uint32_t)buf * KTT * ROWB;
     int valid;  // keys of this tile that exist
     if (NBUF == 2) {
-      if (t + 1 < t_end && t + 1 < Tp) load_tile(t + 1, buf ^ 1);   // the other buffer was released by the
+      if (t + 1 < t_end && t + 1 < Tp && !(early2 && t == t_begin)) load_tile(t + 1, buf ^ 1);   // the other buffer was released by the
       cp_async_commit();                                            // barrier that ended the previous iteration
     }
     if (t < Tp) {
@@ -432,8 +446,7 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
 template <int DH, int KTT>
 __global__ void __launch_bounds__(128, 1) k_attn_cluster(const AttnArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  pdl_enter();
-  if (status_set(a.status)) return;   // the word is only written by kernels that completed before this one started
+  pdl_launch_dependents();            // (the dependency wait and the status check are inside the role)
   attn_role<DH, 1, 2, 0, KTT, true>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
 }
 

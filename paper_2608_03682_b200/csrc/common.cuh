@@ -25,6 +25,8 @@ __device__ __forceinline__ bool status_set(const int* status) {
 // start early and then waits until the kernels it depends on have completed and their writes are visible.  In a
 // launch without the attribute both instructions are no-ops.
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_enter() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");

@@ -71,17 +71,14 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   const int kc_end = (int)(((long long)KC * (blockIdx.z + 1)) / gridDim.z);
   const int nk = kc_end - kc_begin;
 
-  pdl_enter();
-  if (threadIdx.x == 0) {
-    skip_flag = status_set(status) || nk <= 0;
-    abort_flag = 0;
-  }
-  __syncthreads();
-  if (skip_flag) return;
-
+  // Programmatic dependent launch: this grid may start while the kernel before it is still running.  Everything up
+  // to pdl_wait() touches only shared / tensor memory and the weights (constants): barriers, TMEM, and the weight
+  // halves of the first STAGES stages are in flight before the activations this GEMM depends on exist.
+  pdl_launch_dependents();
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles_ptr = smem_raw + (tiles - smem_u32(smem_raw));
   if (threadIdx.x == 0) {
+    abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bar_full[s]), NCOPY);
       mbar_init(smem_u32(&bar_empty[s]), 1);
@@ -105,6 +102,36 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     const int tile = geglu ? nt_idx : nt_idx * NA + a;
     return reinterpret_cast<const uint8_t*>(base) + ((size_t)tile * KC + kc_begin) * A_BYTES;
   };
+  const int n_early = nk < STAGES ? (nk > 0 ? nk : 0) : STAGES;   // stages whose weight copies are issued before the wait
+  if (warp < NPROD && lane == 0) {
+    for (int id = warp; id < n_early * NCOPY; id += NPROD) {
+      const int i = id / NCOPY, c = id % NCOPY;
+      if (c >= NA) continue;
+      const uint32_t full = smem_u32(&bar_full[i]);
+      mbar_expect_tx(full, A_BYTES);
+      bulk_g2s(tiles + (uint32_t)i * STAGE_BYTES + c * A_BYTES, wtile(c) + (size_t)i * A_BYTES, A_BYTES, full);
+    }
+  }
+  pdl_wait();
+  if (threadIdx.x == 0) skip_flag = status_set(status) || nk <= 0;
+  __syncthreads();
+  if (skip_flag) {
+    // the weight copies already issued must land before this CTA's shared memory is released: complete their
+    // barriers with empty arrivals in place of the activation copies, then wait for them
+    if (warp < NPROD && lane == 0) {
+      for (int id = warp; id < n_early * NCOPY; id += NPROD)
+        if (id % NCOPY >= NA) mbar_expect_tx(smem_u32(&bar_full[id / NCOPY]), 0);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+      for (int i = 0; i < n_early; ++i) mbar_wait(smem_u32(&bar_full[i]), 0u, wc);
+    __syncthreads();
+    if (warp == 8) {
+      tc_fence_after();
+      tmem_dealloc(tmem_base, ALLOC_COLS);
+    }
+    return;
+  }
 
   if (warp < NPROD) {
     // ---------------- producers: copy number id = stage * NCOPY + piece goes to warp id % 8 --------------
@@ -113,6 +140,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
           reinterpret_cast<const uint8_t*>(g.X) + ((size_t)kc_begin * g.rows_pad + (size_t)tt * NT) * 128;
       for (int id = warp; id < nk * NCOPY; id += NPROD) {
         const int i = id / NCOPY, c = id % NCOPY;
+        if (i < n_early && c < NA) continue;                          // issued before the dependency wait
         const int s = i % STAGES;
         const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
         if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc)) break;  // stop issuing copies once aborted
