@@ -35,7 +35,7 @@ METRIC_BATCHED = "chunks/sec at batch %d"
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (bench.py cannot run ncu itself)
-NCU_TRAFFIC = {"C2": (6.433488e9 + 69.605376e6, "profiles/persistent_kernel_c2_batch1.md")}
+NCU_TRAFFIC = {"C2": (6.407961e9 + 0.188113e9, "profiles/per_operator_loop_c2_batch1.md")}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 
 
@@ -306,14 +306,12 @@ def main():
     alg_bytes, alg_flops = algorithmic_cost(cfg, lens, n_steps)
     secs = ms_per_step / 1e3
     hbm_bound = not batched or batch < 8
-    persistent = batch * cfg.suffix_len <= 64 and cfg.dtype != "f32"
     traffic = NCU_TRAFFIC.get(args.workload, (None, None))
     if hbm_bound:
         achieved = alg_bytes / secs / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "traffic": traffic[0], "traffic_source": traffic[1],
-                    "kernel": ("k_mega: persistent kernel, one launch = one chunk (all Euler steps and layers)"
-                               if persistent else "whole captured loop (one graph launch = one chunk)"),
+                    "kernel": "whole captured loop (one graph launch = one chunk: all Euler steps and layers)",
                     "peak_source": f"{peaks['source']} copy bandwidth", "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
                     "algorithmic_bytes_per_launch": alg_bytes}
     else:
