@@ -241,7 +241,8 @@ __global__ void k_embed_pi0(const Request* rq, const int* status, const float* W
   __syncthreads();
   for (int n = threadIdx.x; n < D; n += blockDim.x) {
     float acc = 0.f;
-    for (int a = 0; a < A; ++a) acc = fmaf(xs[a], Wc[(size_t)a * D + n], acc);
+#pragma unroll 8
+    for (int a = 0; a < A; ++a) acc = fmaf(xs[a], __ldg(Wc + (size_t)a * D + n), acc);   // loads of 8 rows in flight
     u.store(r, n, swish_precise(acc + tb[n]));
     if (ns && i == 0) h[(size_t)(b * S) * D + n] = state_tok[(size_t)b * D + n];
   }
@@ -517,7 +518,7 @@ void launch_rmsnorm(const int* status, float* h, const float* gain, const float*
 // then split over the 8 warps: warp w takes D/8 consecutive d for all FR rows, lane = action channel, so an
 // element of Wout is loaded once per block and used for FR rows, and the normalised rows are read as
 // float4.  The 8 partial sums are combined in a fixed order.
-constexpr int FR = 16;
+template <int FR>
 __global__ void __launch_bounds__(256) k_final(const Request* rq, const int* status, const float* h, const float* gain,
                                                const float* shift, const float* Wout, const float* bout, float dt, int A,
                                                int H, int D, int S, int ns, float eps, int rows_total) {
@@ -592,11 +593,17 @@ void launch_final(const Request* rq, const int* status, const float* h, const fl
   const int rows = batch * d.H;
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(k_final, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    cudaFuncSetAttribute(k_final<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    cudaFuncSetAttribute(k_final<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
     configured = true;
   }
-  launch_pdl(k_final, dim3((rows + FR - 1) / FR), dim3(256), ((size_t)FR * d.D + 8 * FR * 32) * sizeof(float), st, rq, status,
-             h, gain, shift, Wout, bout, dt, d.A, d.H, d.D, d.S, d.ns, d.eps, rows);
+  // few rows (one request): two rows per block so that the work spreads over more SMs
+  if (rows <= 256)
+    launch_pdl(k_final<2>, dim3((rows + 1) / 2), dim3(256), ((size_t)2 * d.D + 8 * 2 * 32) * sizeof(float), st, rq, status, h,
+               gain, shift, Wout, bout, dt, d.A, d.H, d.D, d.S, d.ns, d.eps, rows);
+  else
+    launch_pdl(k_final<16>, dim3((rows + 15) / 16), dim3(256), ((size_t)16 * d.D + 8 * 16 * 32) * sizeof(float), st, rq,
+               status, h, gain, shift, Wout, bout, dt, d.A, d.H, d.D, d.S, d.ns, d.eps, rows);
 }
 
 // =============================================================================================
