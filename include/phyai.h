@@ -201,6 +201,8 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
  * keeps the split kernel + merge kernel.  key "use_pair_gemm": 1 runs the
  * GEMMs of batches above 1024 tokens on CTA pairs (tcgen05 cta_group::2, persistent, overlapped epilogue), 0
  * (default) keeps the single-CTA kernel, which measured faster on the batch-64 shapes.
+ * key "slab_splits": 1..16 (default 8), the most k-ranges a residual projection of a single-token-tile call is split into
+ * (its partial sums are written as slabs and added in slab order by the next kernel: bit-reproducible).
  * key "wait_limit": iteration bound of
  * device-side waits (testing).  Unknown key -> INVALID_ARG. */
 phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t value);

@@ -58,6 +58,25 @@ def test_small_bf16_expert_matches_oracle(cond, engine):
         assert rel_err(got, ref) <= bar, (P, rel_err(got, ref))
 
 
+@pytest.mark.parametrize("head_dim,n_q,n_kv", [(64, 4, 2), (256, 2, 1)])
+def test_small_bf16_other_head_sizes_through_every_batch1_path(head_dim, n_q, n_kv):
+    """head_dim 64 takes the fp32 QKV output (no rotary epilogue) into the cluster-merged attention, head_dim 256 the
+    rotated bf16 operands; each also through the split attention + merge kernels and the persistent kernel where it
+    covers the shape.  Prefix lengths: empty, shorter than one key tile, several tiles."""
+    cfg = small_bf16_config("pi0", head_dim=head_dim, n_q_heads=n_q, n_kv_heads=n_kv, max_prefix_len=700)
+    W = synth.make_weights(cfg, 18, std=0.05)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        for P in (0, 41, 700):
+            kv, state, noise = _inputs(cfg, 18, P)
+            ref = O.denoise(cfg, W, kv, P, state, noise, 3)
+            for opts in ({"use_cluster_attention": 1, "use_persistent": 0}, {"use_cluster_attention": 0},
+                         {"use_persistent": 1}):
+                for k, v in opts.items():
+                    ex.set_option(k, v)
+                got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
+                assert rel_err(got, ref) <= BAR["bf16"], (P, opts, rel_err(got, ref))
+
+
 # ------------------------------------------------------------------------------------------ C2 / C3
 @pytest.mark.parametrize("name", ["C2", "C3"])
 def test_pi_shaped_bf16_batch1_matches_oracle(name):
