@@ -1,21 +1,25 @@
-// Suffix -> (prefix U suffix) attention on the tcgen05 tensor cores, for large batches.
+// Suffix -> (prefix U suffix) attention on the tcgen05 tensor cores, for calls with two or more requests.
 //
 // One CTA takes the suffix rows of two query heads that share a kv head (2 x 64 padded rows = the 128
 // rows of one MMA) and walks all key tiles of its request:
-//   S = Q K^T      tcgen05.mma, M = 128, N = 64 keys, K = head_dim, fp32 accumulator in TMEM (two buffers)
-//   softmax        one thread per row reads its S row from TMEM (no shuffles), online max / sum in the
-//                  log2 domain, writes P (bf16) to shared memory as the next MMA's A operand
-//   O += P V       tcgen05.mma, M = 128, N = head_dim, K = 64 keys, accumulator stays in TMEM; V is used
-//                  as an MN-major B operand, so K and V tiles share one shared-memory layout and loader
-// K/V tiles (64 keys) and P are double buffered; K and V are staged by separate warps with 16-byte cp.async
-// into the 128-byte-swizzled block layout the MMA descriptors expect, one tile ahead of their consumer.
-// The suffix keys are tile 0; the prefix tiles follow.  Q and the suffix K / V arrive as bf16, already
-// rotated (q also scaled), from the QKV projection's epilogue, so the prologue is plain 16-byte copies.  The O accumulator is rescaled only when a row's running
-// maximum grows by more than 2^8 (otherwise the old maximum is kept, which is exact algebra and costs
-// nothing), so the TMEM round trip of the correction is rare.
+//   S = Q K^T      tcgen05.mma, M = 128, N = 64 keys, K = head_dim; Q sits in tensor memory (A operand), K in
+//                  shared memory; fp32 accumulator in TMEM, two buffers
+//   softmax        one thread per row reads its S row from TMEM (no shuffles), online max / sum in the log2
+//                  domain, writes P (bf16 pairs) over the first half of the S buffer it has just read
+//   O += P V       tcgen05.mma, M = 128, N = head_dim, K = 64 keys; P is the tensor-memory A operand, V an
+//                  MN-major B operand in shared memory (K and V tiles share one layout and loader code);
+//                  the accumulator stays in TMEM
+// TMEM columns: S / P buffers [0, 128), O [128, 384), Q [384, 512).  The tensor pipe executes one thread's MMAs
+// in issue order, which is what lets P alias S: S(t + 2) is issued after P(t) V(t).
+// K and V tiles (64 keys) stream through two three-deep rings, each filled by its own pair of warps with 16-byte
+// cp.async into the 128-byte-swizzled block layout the MMA descriptors expect.  The suffix keys are tile 0; the
+// prefix tiles follow.  Q and the suffix K / V arrive as bf16, already rotated (q also scaled), from the QKV
+// projection's epilogue.  The O accumulator is rescaled only when a row's running maximum grows by more than 2^8
+// (otherwise the old maximum is kept, which is exact algebra and costs nothing), so the TMEM round trip of the
+// correction is rare.
 //
-// Warps: 0-1 load K, 2-3 load V, 4 issues the MMAs (whole warp in the loop, one
-// elected lane issues), 5-8 softmax / correction / output (TMEM lane quarter = warp % 4).
+// Warps: 0-1 load K, 2-3 load V, 4 issues the MMAs (whole warp in the loop, one elected lane issues), 5-8 Q into
+// TMEM, softmax / correction / output (TMEM lane quarter = warp % 4).
 // All waits are bounded; on expiry the CTA raises the status word and drains.
 #include "attention.cuh"
 #include "tc.cuh"

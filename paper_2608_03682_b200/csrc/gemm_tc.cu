@@ -12,9 +12,10 @@
 //   B: activations kept in the tiled bf16 layout, so an NT x 64 tile is one contiguous block.
 // Every load is therefore a 1-D bulk copy (16-byte aligned, size a multiple of 16): no tensor map.
 //
-// A CTA computes NA (1 or 2) 128-channel tiles against one NT-token tile: with NA = 2 and NT = 256 a
-// k-step moves 64 KB for 8 MMAs of 128 clocks, i.e. 64 bytes per clock, which is what one SM's L2 port
-// delivers (~126 GB/s measured); a single 128 x 256 tile would need 96 bytes per clock.
+// A CTA computes NA (1 or 2) 128-channel tiles against one NT-token tile (NT = 64, 128, 192 or 256): with NA = 2
+// and NT = 256 a k-step moves 64 KB for 8 MMAs of 128 clocks, i.e. 64 bytes per clock.  One SM alone ingests that
+// (~126 GB/s measured); with all SMs streaming the measured rate is 38-40 bytes per clock per SM, which makes the
+// main loop crossbar-bound at ~1600 clocks per k-step.  A single 128 x 256 tile would need 96 bytes per clock.
 //
 // Warp roles (800 threads): warps 0..7 = copy producers (the copies of all stages are dealt round
 // robin to the eight warps: one warp's bulk copies complete one at a time, about 0.5 us each whatever
@@ -22,6 +23,11 @@
 // MMA issuer (whole warp in the loop, one elected lane issues), warps 9..24 = epilogue (TMEM lane
 // quarter = warp % 4, token-column quarter = (warp - 9) / 4).  The epilogue of a 256 x 256 tile is not
 // overlapped with a next tile (TMEM is full), so it gets 16 warps and batches its global loads.
+// Epilogues: plain store, gated residual (read-modify-write; split-K: 16-byte vector reductions, or slabs that the
+// next kernel sums in a fixed order), GeGLU (paired gate / up tiles, or interleaved 64 + 64 tiles), bias + row remap,
+// and the rotary epilogue of the fused QKV projection (rotated, scaled bf16 q / k / v in the attention layout).
+// The kernel is launched with programmatic stream serialization: barriers, TMEM and the weight halves of the first
+// STAGES stages are set up before griddepcontrol.wait, i.e. while the kernel producing the activations still runs.
 // Every wait is bounded: on expiry the CTA raises the status word, stops issuing copies, and
 // drains to its normal exit (TMEM is always released).
 #include "kernels.h"
