@@ -358,15 +358,17 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(d1) : "r"(recv + o1), "r"(row1 >> 3));
       asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(m0a) : "r"(recv_ml + (uint32_t)(split * 8 + (row0 & 7)) * 8), "r"(row0 >> 3));
       asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(m1a) : "r"(recv_ml + (uint32_t)(split * 8 + (row1 & 7)) * 8), "r"(row1 >> 3));
+      // (remote stores are the slow part of the merge: rows past the suffix are not sent, nobody reads them)
+      const bool send0 = row0 < S, send1 = row1 < S;
 #pragma unroll
       for (int n = 0; n < DH / 8; ++n) {
         const uint32_t col = (uint32_t)(n * 8 + qd * 2) * 4;
-        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d0 + col), "f"(o[n][0]), "f"(o[n][1]) : "memory");
-        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d1 + col), "f"(o[n][2]), "f"(o[n][3]) : "memory");
+        if (send0) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d0 + col), "f"(o[n][0]), "f"(o[n][1]) : "memory");
+        if (send1) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d1 + col), "f"(o[n][2]), "f"(o[n][3]) : "memory");
       }
       if (qd == 0) {
-        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m0a), "f"(m0), "f"(l0) : "memory");
-        asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m1a), "f"(m1), "f"(l1) : "memory");
+        if (send0) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m0a), "f"(m0), "f"(l0) : "memory");
+        if (send1) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m1a), "f"(m1), "f"(l1) : "memory");
       }
     }
     asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
