@@ -81,12 +81,13 @@ __device__ __forceinline__ void group_sync() {
 // `smem_base` (128-byte aligned): (HPC*64 + 2*NBUF*KTT) rows of DH bf16.  When a.qr is set, q / k / v of
 // the suffix are read as bf16, already rotated and scaled (written by the QKV epilogue of the
 // persistent kernel); otherwise they are taken from the fp32 QKV output and rotated here.
-// CLUSTER (HPC = 1): the num_splits = 8 key ranges of a head are the 8 CTAs of a thread-block cluster; each pushes
-// the rows of its partial (O, max, sum) into the shared memory of the CTA that owns them (distributed shared
-// memory stores) and, after one cluster barrier, merges its own 8 of the 64 rows: no partials in global memory, no
-// merge kernel.  Needs 8 * 8 * (DH + 4) * 4 + 512 bytes of shared memory beyond the Q / K / V buffers.
+// CLUSTER (HPC = 1): the num_splits = 8 key ranges of a head are the 8 CTAs of a thread-block cluster; each sends
+// the rows of its partial (O, max, sum) into the shared memory of the CTA that owns them (bulk copies over
+// distributed shared memory, counted on the owner's mbarrier) and every CTA merges its own 8 of the 64 rows: no
+// partials in global memory, no merge kernel.  Needs 8 * 8 * (DH + 4) * 4 + 512 bytes of shared memory beyond the Q / K / V buffers.
 template <int DH, int HPC, int NBUF, int BAR, int KTT, bool CLUSTER = false>
-__device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp, int b, uint32_t smem_base, int tid) {
+__device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp, int b, uint32_t smem_base, int tid,
+                                          uint32_t mrg_bar = 0, volatile int* abort_flag = nullptr) {
   constexpr int ROWB = DH * 2;                // bytes per row
   constexpr int CH = DH / 8;                  // 16-byte chunks per row
   constexpr int NTHREADS = HPC * 128;
@@ -344,34 +345,46 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
   l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
   const int head = head0 + hl;
   if constexpr (CLUSTER) {
-    // Push merge: CTA `rank` of the cluster owns rows [8 * rank, 8 * rank + 8).  Every CTA stores its partial rows
-    // (and their max / sum) straight into the owners' shared memory (remote stores, fire and forget), into a
-    // receive area beyond the Q / K / V buffers, which the owner may still be using.  After one cluster barrier
-    // each CTA merges its 8 rows from its own shared memory.
+    // Push merge: CTA `rank` of the cluster owns rows [8 * rank, 8 * rank + 8).  Every CTA sends the owners their
+    // rows of its partial (and their max / sum), into a receive area beyond the Q / K / V buffers, which the owner
+    // may still be using; each CTA then merges its 8 rows from its own shared memory.
     constexpr int PP = DH + 4;                       // row pitch in floats
+    constexpr uint32_t OWN_BYTES = 8u * PP * 4u;     // one owner's 8 rows of a partial
     const uint32_t recv = smem_base + (uint32_t)(HPC * QROWS + 2 * NBUF * KTT) * ROWB;   // [8 sources][8 rows][PP]
-    const uint32_t recv_ml = recv + 8u * 8u * PP * 4u;                                   // [8 sources][8 rows][2]
-    {
-      uint32_t d0, d1, m0a, m1a;
-      const uint32_t o0 = (uint32_t)((split * 8 + (row0 & 7)) * PP) * 4, o1 = (uint32_t)((split * 8 + (row1 & 7)) * PP) * 4;
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(d0) : "r"(recv + o0), "r"(row0 >> 3));
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(d1) : "r"(recv + o1), "r"(row1 >> 3));
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(m0a) : "r"(recv_ml + (uint32_t)(split * 8 + (row0 & 7)) * 8), "r"(row0 >> 3));
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(m1a) : "r"(recv_ml + (uint32_t)(split * 8 + (row1 & 7)) * 8), "r"(row1 >> 3));
-      // (remote stores are the slow part of the merge: rows past the suffix are not sent, nobody reads them)
-      const bool send0 = row0 < S, send1 = row1 < S;
+    const uint32_t recv_ml = recv + 8u * OWN_BYTES;                                       // [8 sources][8 rows][2]
+    // The partial is first written to this CTA's own shared memory (over the K / V buffers, which every thread has
+    // finished with: the tile loop ends with a barrier), grouped by owner, then sent with one bulk copy per owner
+    // (distributed shared memory, completion counted on the owner's mbarrier): remote stores from the threads
+    // themselves measured ~3 us for the 64 KB.
+    const uint32_t stg = Ks, stg_ml = Ks + 8u * OWN_BYTES;
 #pragma unroll
-      for (int n = 0; n < DH / 8; ++n) {
-        const uint32_t col = (uint32_t)(n * 8 + qd * 2) * 4;
-        if (send0) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d0 + col), "f"(o[n][0]), "f"(o[n][1]) : "memory");
-        if (send1) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(d1 + col), "f"(o[n][2]), "f"(o[n][3]) : "memory");
-      }
-      if (qd == 0) {
-        if (send0) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m0a), "f"(m0), "f"(l0) : "memory");
-        if (send1) asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(m1a), "f"(m1), "f"(l1) : "memory");
-      }
+    for (int n = 0; n < DH / 8; ++n) {
+      const uint32_t col = (uint32_t)(n * 8 + qd * 2) * 4;
+      asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(stg + (uint32_t)(row0 * PP) * 4 + col), "f"(o[n][0]), "f"(o[n][1]) : "memory");
+      asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(stg + (uint32_t)(row1 * PP) * 4 + col), "f"(o[n][2]), "f"(o[n][3]) : "memory");
     }
-    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (qd == 0) {
+      asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(stg_ml + (uint32_t)row0 * 8), "f"(m0), "f"(l0) : "memory");
+      asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(stg_ml + (uint32_t)row1 * 8), "f"(m1), "f"(l1) : "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the bulk-copy engine
+    group_sync<BAR, NTHREADS>();
+    if (tid < 16) {
+      const uint32_t owner = (uint32_t)tid & 7u, ml = (uint32_t)tid >> 3;
+      const uint32_t src = ml ? stg_ml + owner * 64u : stg + owner * OWN_BYTES;
+      const uint32_t bytes = ml ? 64u : OWN_BYTES;
+      const uint32_t dst_local = ml ? recv_ml + (uint32_t)split * 64u : recv + (uint32_t)split * OWN_BYTES;
+      uint32_t dst, bar;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(dst_local), "r"(owner));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(mrg_bar), "r"(owner));
+      asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                   "r"(src), "r"(bytes), "r"(bar)
+                   : "memory");
+    }
+    {
+      const WaitCtx wc{a.status, abort_flag, a.wait_limit};
+      mbar_wait(mrg_bar, 0u, wc);     // all eight partials of my rows have landed in `recv`
+    }
     constexpr int CPT = DH / 16;                                  // columns per thread: 16 threads cover a row
     const int rl = tid >> 4, r = split * 8 + rl, c0 = (tid & 15) * CPT;
     if (r < S) {
@@ -406,6 +419,9 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
         *reinterpret_cast<uint2*>(a.out + out_index(b * S + r, head * DH + c0 + 4 * u, a.rows_pad, d.Nq)) =
             make_uint2(pack_bf16(acc[4 * u] * inv, acc[4 * u + 1] * inv), pack_bf16(acc[4 * u + 2] * inv, acc[4 * u + 3] * inv));
     }
+    // every CTA has received everything by now, i.e. every outgoing copy has finished reading its source: only
+    // then may a CTA leave and release its shared memory
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   } else if (a.num_splits == 1) {
     const float i0 = 1.0f / l0, i1 = 1.0f / l1;
 #pragma unroll
@@ -448,8 +464,19 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
 template <int DH, int KTT>
 __global__ void __launch_bounds__(128, 1) k_attn_cluster(const AttnArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t mrg_bar;
+  __shared__ int abort_flag;
   pdl_launch_dependents();            // (the dependency wait and the status check are inside the role)
-  attn_role<DH, 1, 2, 0, KTT, true>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&mrg_bar), 1);
+    mbar_expect_tx(smem_u32(&mrg_bar), 8u * (8u * (DH + 4) * 4u + 64u));   // eight sources: 8 rows of O and of (max, sum)
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // every CTA's merge barrier exists before any peer can send to it (this runs before the dependency wait)
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  attn_role<DH, 1, 2, 0, KTT, true>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x,
+                                    smem_u32(&mrg_bar), &abort_flag);
 }
 
 }  // namespace
