@@ -174,17 +174,19 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       const uint64_t da = make_desc(a0);
       const uint64_t da2 = make_desc(a0 + A_BYTES);
       const uint64_t db = make_desc(a0 + A_BYTES * NA);
-      if (elect_one()) {
-        if (ok) {
+      // control flow and descriptors stay warp-uniform; only the tcgen05 instructions themselves are predicated on
+      // the elected lane
+      if (__all_sync(0xffffffffu, ok)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
-            const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
-            umma_bf16(tmem_base, da + 2 * k, db + 2 * k, IDESC, acc);
-            if (NA == 2) umma_bf16(tmem_base + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
+        for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
+          const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
+          if (elect_one()) umma_bf16(tmem_base, da + 2 * k, db + 2 * k, IDESC, acc);
+          if (NA == 2) {
+            if (elect_one()) umma_bf16(tmem_base + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
           }
         }
-        umma_commit(smem_u32(&bar_empty[s]));  // frees the stage when the MMAs above have read it
       }
+      if (elect_one()) umma_commit(smem_u32(&bar_empty[s]));  // frees the stage when the MMAs above have read it
       __syncwarp();
     }
     if (elect_one()) umma_commit(smem_u32(&bar_accum));
