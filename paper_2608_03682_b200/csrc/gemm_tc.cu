@@ -55,7 +55,11 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   constexpr int ALLOC_COLS = COLS <= 32 ? 32 : COLS <= 64 ? 64 : COLS <= 128 ? 128 : COLS <= 256 ? 256 : 512;   // power of two
   // A producer warp's consecutive copies are NPROD / NCOPY k-steps apart; its parity wait on "stage free" is only
   // meaningful while that step does not exceed the ring depth.
-  static_assert((NPROD + NCOPY - 1) / NCOPY <= STAGES, "producer stride exceeds the stage ring");
+  // Copy issuers: the 8 producer warps, plus (single 64-token tile) the first epilogue warps, which are idle during
+  // the main loop.  One warp's bulk copies complete one at a time (measured), so the number of copies in flight is
+  // the number of issuing warps: with 8 issuers a 16-step main loop of 32 copies took 4.9 us whatever was prefetched.
+  constexpr int NISSUE = (NT == 64 && NA == 1) ? (2 * STAGES < 24 ? 2 * STAGES : 24) : NPROD;
+  static_assert((NISSUE + NCOPY - 1) / NCOPY <= STAGES, "producer stride exceeds the stage ring");
   // instruction descriptor: D fp32 (bit 4), A bf16 (bit 7), B bf16 (bit 10), both K-major,
   // N >> 3 at bit 17, M >> 4 at bit 24.
   constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((128u >> 4) << 24);
@@ -109,8 +113,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     return reinterpret_cast<const uint8_t*>(base) + ((size_t)tile * KC + kc_begin) * A_BYTES;
   };
   const int n_early = nk < STAGES ? (nk > 0 ? nk : 0) : STAGES;   // stages whose weight copies are issued before the wait
-  if (warp < NPROD && lane == 0) {
-    for (int id = warp; id < n_early * NCOPY; id += NPROD) {
+  const int issuer = warp < NPROD ? warp : warp - 1;              // producer warps 0..7, then epilogue warps 9.. -> 8..
+  const bool issues = lane == 0 && warp != 8 && issuer < NISSUE;
+  if (issues) {
+    for (int id = issuer; id < n_early * NCOPY; id += NISSUE) {
       const int i = id / NCOPY, c = id % NCOPY;
       if (c >= NA) continue;
       const uint32_t full = smem_u32(&bar_full[i]);
@@ -124,8 +130,8 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   if (skip_flag) {
     // the weight copies already issued must land before this CTA's shared memory is released: complete their
     // barriers with empty arrivals in place of the activation copies, then wait for them
-    if (warp < NPROD && lane == 0) {
-      for (int id = warp; id < n_early * NCOPY; id += NPROD)
+    if (issues) {
+      for (int id = issuer; id < n_early * NCOPY; id += NISSUE)
         if (id % NCOPY >= NA) mbar_expect_tx(smem_u32(&bar_full[id / NCOPY]), 0);
     }
     __syncthreads();
@@ -139,12 +145,12 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     return;
   }
 
-  if (warp < NPROD) {
-    // ---------------- producers: copy number id = stage * NCOPY + piece goes to warp id % 8 --------------
-    if (lane == 0) {
+  // ---------------- copy issuers: copy number id = k-step * NCOPY + piece goes to issuer id % NISSUE --------------
+  if (issues) {
+    {
       const uint8_t* xsrc =
           reinterpret_cast<const uint8_t*>(g.X) + ((size_t)kc_begin * g.rows_pad + (size_t)tt * NT) * 128;
-      for (int id = warp; id < nk * NCOPY; id += NPROD) {
+      for (int id = issuer; id < nk * NCOPY; id += NISSUE) {
         const int i = id / NCOPY, c = id % NCOPY;
         if (i < n_early && c < NA) continue;                          // issued before the dependency wait
         const int s = i % STAGES;
@@ -163,13 +169,19 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         }
       }
     }
+  }
+  __syncwarp();
+  if (warp < NPROD) {
+    // (producer warps have nothing else to do)
   } else if (warp == 8) {
     // ---------------- MMA issuer (whole warp in the loop, one elected lane issues) ---------------------
     for (int i = 0; i < nk; ++i) {
       const int s = i % STAGES;
       const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
       const bool ok = mbar_wait(smem_u32(&bar_full[s]), ph, wc);
-      tc_fence_after();
+      // (no tcgen05 fence here: the operands were written by the bulk-copy engine and made visible by the mbarrier;
+      // tcgen05.fence::after_thread_sync orders tensor-memory accesses, and it was measured to hold the next MMAs
+      // back until the previous stage's MMAs had drained)
       const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
       const uint64_t da = make_desc(a0);
       const uint64_t da2 = make_desc(a0 + A_BYTES);
@@ -506,7 +518,7 @@ cudaError_t setup_one() {
 
 cudaError_t tc_gemm_setup() {
   cudaError_t e;
-  if ((e = setup_one<64, 1, 6>()) != cudaSuccess) return e;
+  if ((e = setup_one<64, 1, 9>()) != cudaSuccess) return e;
   if ((e = setup_one<64, 2, 4>()) != cudaSuccess) return e;
   if ((e = setup_one<128, 1, 5>()) != cudaSuccess) return e;
   if ((e = setup_one<128, 2, 4>()) != cudaSuccess) return e;
@@ -524,7 +536,7 @@ cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st
   // a plain store epilogue cannot split K: when two-tile CTAs would leave more than half of the SMs idle, take one
   // channel tile per CTA instead
   if (g.epi == TC_BIAS_ROWMAP && nt == 256 && (g.N / 256) * ((g.M + 255) / 256) <= 74) two = false;
-  if (nt == 64) return two ? launch_one<64, 2, 4>(status, g, st) : launch_one<64, 1, 6>(status, g, st);
+  if (nt == 64) return two ? launch_one<64, 2, 4>(status, g, st) : launch_one<64, 1, 9>(status, g, st);
   if (nt == 128) return two ? launch_one<128, 2, 4>(status, g, st) : launch_one<128, 1, 5>(status, g, st);
   // 192-token tiles (two channel tiles per CTA only): for token counts where they fill the SMs better
   if (nt == 192 && g.epi != TC_GEGLU && g.N % 256 == 0) return launch_one<192, 2, 4>(status, g, st);
