@@ -139,10 +139,6 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
     // Programmatic dependent launch: the request block and the prefix K/V were complete before this grid could
     // start, so the first key tile is already on its way; q / k / v of the suffix come from the kernel before.
     pdl_wait();
-    if (status_set(a.status)) {   // same answer in every CTA of the cluster (all earlier kernels have completed)
-      cp_async_wait<0>();
-      return;
-    }
   }
 
   if (a.qr) {
@@ -156,6 +152,14 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       cp_async16(Qs + swz(hl * QROWS + i, c, ROWB), src, ok ? 16u : 0u);
     }
     cp_async_commit();
+  }
+  if constexpr (CLUSTER) {
+    // The status word is read after the Q copies have been requested (their addresses do not depend on the request),
+    // so that its round trip to the L2 overlaps theirs.
+    if (status_set(a.status)) {   // same answer in every CTA of the cluster (all earlier kernels have completed)
+      cp_async_wait<0>();
+      return;
+    }
   }
   // ---- Q: rotate, scale by dh^-1/2, round to bf16, into shared memory (4 column pairs per thread)
   const float qscale = rsqrtf((float)DH);

@@ -125,16 +125,24 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     }
   }
   pdl_wait();
-  if (threadIdx.x == 0) skip_flag = status_set(status) || nk <= 0;
+  // The activation copies of the prefetched stages go out before the status word is known (their addresses do not
+  // depend on the request, and the skip path below waits for them): the status read, a round trip to the L2, then
+  // overlaps their latency.  It is made by the MMA warp, which issues no copies.
+  const uint8_t* xsrc = reinterpret_cast<const uint8_t*>(g.X) + ((size_t)kc_begin * g.rows_pad + (size_t)tt * NT) * 128;
+  auto issue_x = [&](int i, int pc, uint32_t s_idx) {
+    const uint32_t full = smem_u32(&bar_full[s_idx]);
+    mbar_expect_tx(full, B_PIECE);
+    bulk_g2s(tiles + s_idx * STAGE_BYTES + NA * A_BYTES + pc * B_PIECE, xsrc + (size_t)i * g.rows_pad * 128 + (size_t)pc * B_PIECE,
+             B_PIECE, full);
+  };
+  if (issues) {
+    for (int id = issuer; id < n_early * NCOPY; id += NISSUE)
+      if (id % NCOPY >= NA) issue_x(id / NCOPY, id % NCOPY - NA, (uint32_t)(id / NCOPY));
+  }
+  if (threadIdx.x == NPROD * 32) skip_flag = status_set(status) || nk <= 0;
   __syncthreads();
   if (skip_flag) {
-    // the weight copies already issued must land before this CTA's shared memory is released: complete their
-    // barriers with empty arrivals in place of the activation copies, then wait for them
-    if (issues) {
-      for (int id = issuer; id < n_early * NCOPY; id += NISSUE)
-        if (id % NCOPY >= NA) mbar_expect_tx(smem_u32(&bar_full[id / NCOPY]), 0);
-    }
-    __syncthreads();
+    // every copy issued so far must land before this CTA's shared memory is released
     if (threadIdx.x == 0)
       for (int i = 0; i < n_early; ++i) mbar_wait(smem_u32(&bar_full[i]), 0u, wc);
     __syncthreads();
@@ -147,26 +155,17 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
 
   // ---------------- copy issuers: copy number id = k-step * NCOPY + piece goes to issuer id % NISSUE --------------
   if (issues) {
-    {
-      const uint8_t* xsrc =
-          reinterpret_cast<const uint8_t*>(g.X) + ((size_t)kc_begin * g.rows_pad + (size_t)tt * NT) * 128;
-      for (int id = issuer; id < nk * NCOPY; id += NISSUE) {
-        const int i = id / NCOPY, c = id % NCOPY;
-        if (i < n_early && c < NA) continue;                          // issued before the dependency wait
-        const int s = i % STAGES;
-        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc)) break;  // stop issuing copies once aborted
+    for (int id = issuer + (n_early * NCOPY - issuer + NISSUE - 1) / NISSUE * NISSUE; id < nk * NCOPY; id += NISSUE) {
+      const int i = id / NCOPY, c = id % NCOPY;
+      const int s = i % STAGES;
+      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+      if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc)) break;  // stop issuing copies once aborted
+      if (c < NA) {
         const uint32_t full = smem_u32(&bar_full[s]);
-        const uint32_t dst = tiles + (uint32_t)s * STAGE_BYTES;
-        if (c < NA) {
-          mbar_expect_tx(full, A_BYTES);
-          bulk_g2s(dst + c * A_BYTES, wtile(c) + (size_t)i * A_BYTES, A_BYTES, full);
-        } else {
-          const int pc = c - NA;
-          mbar_expect_tx(full, B_PIECE);
-          bulk_g2s(dst + NA * A_BYTES + pc * B_PIECE, xsrc + (size_t)i * g.rows_pad * 128 + (size_t)pc * B_PIECE, B_PIECE,
-                   full);
-        }
+        mbar_expect_tx(full, A_BYTES);
+        bulk_g2s(tiles + (uint32_t)s * STAGE_BYTES + c * A_BYTES, wtile(c) + (size_t)i * A_BYTES, A_BYTES, full);
+      } else {
+        issue_x(i, c - NA, (uint32_t)s);
       }
     }
   }

@@ -446,18 +446,29 @@ __global__ void k_rmsnorm_tiled_reg(const int* status, float* h, const float* ga
 // slab loads of a thread are independent, so they are all in flight together.
 __global__ void __launch_bounds__(512) k_add_slabs_norm(const int* status, float* h, const float* gain, const float* shift,
                                                         __nv_bfloat16* out, int rows_pad, int D, float eps, SlabSum sl) {
-  pdl_enter();
-  if (status_set(status)) return;
+  // Constants (gain, and the shift row of the modulation table, which is complete before the loop starts) are
+  // fetched before the dependency wait; the status word is requested together with the row and its slabs and only
+  // looked at once they are summed, so that the three round trips to the L2 overlap.
+  pdl_launch_dependents();
   __shared__ float red[16];
   const int row = blockIdx.x, t = threadIdx.x, d = t * 4;
+  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), s4 = g;
+  if (out) {
+    g = __ldg(reinterpret_cast<const float4*>(gain + d));
+    if (shift) s4 = __ldg(reinterpret_cast<const float4*>(shift + d));
+  }
+  pdl_wait();
   float* x = h + (size_t)row * D + d;
   float4 v = *reinterpret_cast<const float4*>(x);
+  int stv;
+  asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(stv) : "l"(status) : "memory");
   const float* p = sl.slab + (size_t)row * D + d;
 #pragma unroll 8
   for (int s = 0; s < sl.n; ++s) {
     const float4 q = __ldg(reinterpret_cast<const float4*>(p + (size_t)s * sl.stride));
     v.x += q.x, v.y += q.y, v.z += q.z, v.w += q.w;
   }
+  if (stv != 0) return;
   *reinterpret_cast<float4*>(x) = v;
   if (!out) return;
   float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
@@ -466,12 +477,8 @@ __global__ void __launch_bounds__(512) k_add_slabs_norm(const int* status, float
   float tot = 0.f;
   for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];   // same order in every thread
   const float r = 1.0f / sqrtf(tot / (float)D + eps);
-  const float4 g = __ldg(reinterpret_cast<const float4*>(gain + d));
   float4 o = make_float4(v.x * r * g.x, v.y * r * g.y, v.z * r * g.z, v.w * r * g.w);
-  if (shift) {
-    const float4 s4 = __ldg(reinterpret_cast<const float4*>(shift + d));
-    o.x += s4.x, o.y += s4.y, o.z += s4.z, o.w += s4.w;
-  }
+  if (shift) o.x += s4.x, o.y += s4.y, o.z += s4.z, o.w += s4.w;
   __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
   uint2 pk;
   pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
