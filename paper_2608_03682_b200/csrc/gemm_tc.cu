@@ -222,6 +222,50 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         tok_tab[idx] = e;
       }
     }
+    // per-channel constants of the plain epilogues (weight scale, residual gate, bias) are fetched while the main
+    // loop runs, not after the accumulator is ready
+    float e_sc[NA], e_gt[NA], e_bs[NA], e_il = 1.0f;
+    if (!geglu && g.epi != TC_QKV_ROT && g.epi != TC_GEGLU_IL) {
+#pragma unroll
+      for (int a = 0; a < NA; ++a) {
+        const int n = (nt_idx * NA + a) * 128 + ch;
+        e_sc[a] = g.scale ? g.scale[n] : 1.0f;
+        e_gt[a] = (g.epi == TC_RESID && g.gate) ? g.gate[n] : 1.0f;
+        e_bs[a] = (g.epi == TC_BIAS_ROWMAP && g.bias) ? g.bias[n] : 0.0f;
+      }
+    } else {
+#pragma unroll
+      for (int a = 0; a < NA; ++a) e_sc[a] = e_gt[a] = 1.0f, e_bs[a] = 0.0f;
+      if (g.epi == TC_GEGLU_IL) {
+        const int f = nt_idx * 64 + (ch & 63);
+        const float* sp = q >= 2 ? g.scale2 : g.scale;
+        if (sp) e_il = sp[f];
+      }
+    }
+    // rotary epilogue: the weight scale and the table rows of this thread's first item of accumulator 0 are on
+    // their way before the accumulator is ready (the later ones are requested one item ahead)
+    float4 cs_pre[4];
+    int2 e_pre = make_int2(0, 0);
+    float sc_pre = 1.0f;
+    bool pre = false;
+    if (g.epi == TC_QKV_ROT) {
+      epi_sync();                                   // tok_tab complete
+      const int n0 = nt_idx * NA * 128;
+      if (g.scale) sc_pre = g.scale[n0 + ch];
+      const int rows = min(NT, g.M - tok_base);
+      const int Nq = g.Hq * g.dh, Nk = g.Hkv * g.dh;
+      if (n0 < Nq + Nk && et < rows * 8) {
+        const int nn = n0 < Nq ? n0 : n0 - Nq;
+        const int t = (nn % g.dh) >> 7;
+        e_pre = tok_tab[et >> 3];
+        pre = true;
+        if (g.rope) {
+          const float4* cs = reinterpret_cast<const float4*>(g.rope + (size_t)e_pre.x * (g.dh >> 1) + t * 64 + (et & 7) * 8);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) cs_pre[u] = __ldg(cs + u);
+        }
+      }
+    }
     const bool ok = mbar_wait(smem_u32(&bar_accum), 0, wc);
     tc_fence_after();
     constexpr int HALF = NT / 4;   // token columns per epilogue warp
@@ -231,10 +275,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
 #pragma unroll
       for (int a = 0; a < NA; ++a) {
         const int n = (nt_idx * NA + a) * 128 + ch;   // packed output channel
-        const float sc = g.scale ? g.scale[n] : 1.0f;
+        const float sc = e_sc[a];
         const int n_out = (g.perm_dh && n < g.perm_end) ? qkv_packed_to_channel(n, g.perm_dh) : n;
-        const float gt = (g.epi == TC_RESID && g.gate) ? g.gate[n] : 1.0f;
-        const float bs = (g.epi == TC_BIAS_ROWMAP && g.bias) ? g.bias[n] : 0.0f;
+        const float gt = e_gt[a];
+        const float bs = e_bs[a];
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;  // warp-uniform
           float v[16];
@@ -281,7 +325,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       __nv_bfloat16* img = reinterpret_cast<__nv_bfloat16*>(stage + (size_t)NT * 64);      // [NT][64] bf16, swizzled
       const int c64 = ch & 63, f = nt_idx * 64 + c64;
       if (ok && q >= 2) {
-        const float su = g.scale2 ? g.scale2[f] : 1.0f;
+        const float su = e_il;
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;
           float v[16];
@@ -292,7 +336,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       }
       epi_sync();
       if (ok && q < 2) {
-        const float sg = g.scale ? g.scale[f] : 1.0f;
+        const float sg = e_il;
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;
           float v[16];
@@ -324,7 +368,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       for (int a = 0; a < NA; ++a) {
         const int n0 = (nt_idx * NA + a) * 128;
         if (ok) {
-          const float sc = (g.scale ? g.scale[n0 + ch] : 1.0f) * (g.gate ? g.gate[n0 + ch] : 1.0f);
+          const float sc = e_sc[a] * e_gt[a];
           for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
             if (tok_base + c0 >= g.M) break;          // warp-uniform
             float v[16];
@@ -365,7 +409,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       for (int a = 0; a < NA; ++a) {
         const int n0 = (nt_idx * NA + a) * 128;       // first packed row of this accumulator
         if (ok) {
-          const float sc = g.scale ? g.scale[n0 + ch] : 1.0f;
+          const float sc = a == 0 ? sc_pre : (g.scale ? g.scale[n0 + ch] : 1.0f);
           for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
             if (tok_base + c0 >= g.M) break;          // warp-uniform
             float v[16];
@@ -394,7 +438,13 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
                 for (int u = 0; u < 4; ++u) cs_next[u] = __ldg(cs + u);
               }
             };
-            if (et < rows * 8) fetch(et);
+            if (a == 0 && pre) {
+              e_next = e_pre;
+#pragma unroll
+              for (int u = 0; u < 4; ++u) cs_next[u] = cs_pre[u];
+            } else if (et < rows * 8) {
+              fetch(et);
+            }
             for (int it = et; it < rows * 8; it += NEPI) {
               const int tl = it >> 3, j0 = (it & 7) * 8;
               const int2 e = e_next;
