@@ -198,7 +198,9 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
  * programmatic dependent launch they measured faster than the persistent kernel.  key "use_tc_attention": 1 (default) lets large
  * batches use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "use_cluster_attention": 1 (default) lets calls with few
  * requests merge their key-split attention partials through distributed shared memory (clusters of 8 CTAs), 0
- * keeps the split kernel + merge kernel.  key "use_pair_gemm": 1 runs the
+ * keeps the split kernel + merge kernel.  key "use_fused_oproj": 1 (default) lets that cluster kernel also apply the
+ * attention output projection of its head (head_dim 256, model width 1024, one token tile; one partial per head,
+ * summed in head order by the next kernel), 0 keeps the separate projection.  key "use_pair_gemm": 1 runs the
  * GEMMs of batches above 1024 tokens on CTA pairs (tcgen05 cta_group::2, persistent, overlapped epilogue), 0
  * (default) keeps the single-CTA kernel, which measured faster on the batch-64 shapes.
  * key "slab_splits": 1..16 (default 8), the most k-ranges a residual projection of a single-token-tile call is split into

@@ -81,41 +81,49 @@ constexpr size_t attn_cluster_smem() {   // Q / K / V buffers + the receive area
   return attn_smem<DH, 1, KTT>() + (size_t)8 * 8 * (DH + 4) * 4 + 512;
 }
 
-template <int DH, int KTT>
+template <int DH, int KTT, bool OPROJ = false>
 cudaError_t launch_attn_cluster(const AttnArgs& a, int batch, cudaStream_t st) {
   static bool configured = false;
+  const size_t smem = attn_cluster_smem<DH, KTT>() + (OPROJ ? 1024 : 0);
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_attn_cluster<DH, KTT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)attn_cluster_smem<DH, KTT>());
+    cudaError_t e = cudaFuncSetAttribute(k_attn_cluster<DH, KTT, OPROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(8, a.d.Hq, batch), cfg.blockDim = dim3(128), cfg.dynamicSmemBytes = attn_cluster_smem<DH, KTT>(), cfg.stream = st;
+  cfg.gridDim = dim3(8, a.d.Hq, batch), cfg.blockDim = dim3(128), cfg.dynamicSmemBytes = smem, cfg.stream = st;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 8, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
   at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at, cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, k_attn_cluster<DH, KTT>, a);
+  return cudaLaunchKernelEx(&cfg, k_attn_cluster<DH, KTT, OPROJ>, a);
 }
 
 }  // namespace
 
 // Key-split attention whose partials are merged through distributed shared memory (clusters of 8 CTAs).
+// With `op` set, the output projection of each head follows in the same kernel (see attention_oproj_supported).
 cudaError_t launch_attention_cluster(const Request* rq, int* status, const float* qkv, const float2* rope,
                                      const __nv_bfloat16* qr, const __nv_bfloat16* kr, const __nv_bfloat16* vr, int layer,
                                      __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, const AttnOproj* op) {
   AttnArgs a{};
   a.rq = rq, a.status = status, a.qkv = qkv, a.rope = rope, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
   a.qr = qr, a.kr = kr, a.vr = vr;   // when set: rotated bf16 operands instead of the fp32 QKV output
   a.num_splits = 8, a.d = d, a.wait_limit = wait_limit;
+  if (op) {
+    a.wo = op->wo, a.o_scale = op->scale, a.o_gate = op->gate, a.slab = op->slab, a.slab_stride = op->slab_stride, a.D = d.D;
+    return launch_attn_cluster<256, 64, true>(a, batch, st);
+  }
   if (d.dh == 256) return launch_attn_cluster<256, 64>(a, batch, st);
   if (d.dh == 128) return launch_attn_cluster<128, 64>(a, batch, st);
   return launch_attn_cluster<64, 64>(a, batch, st);
 }
+// The fused projection covers: head_dim 256, 8 out-channel tiles of 128 (one per CTA of the cluster), a suffix of at
+// most 56 rows (the activation tile is packed at 56 rows per k-chunk), rotated bf16 operands.
+bool attention_oproj_supported(const Dims& d) { return d.dh == 256 && d.D == 1024 && d.S <= 56 && d.Hq <= 16; }
 
 bool attention_mma_supported(const Dims& d) {
   return (d.dh == 64 || d.dh == 128 || d.dh == 256) && d.S <= QROWS;

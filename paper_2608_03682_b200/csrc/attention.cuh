@@ -4,6 +4,7 @@
 
 #include "kernels.h"
 #include "ptx.cuh"
+#include "tc.cuh"
 
 namespace phyai {
 namespace {
@@ -53,6 +54,18 @@ struct AttnArgs {
   Dims d;
   unsigned wait_limit;
   const int* order;      // optional: request index of each grid row (batch entries)
+  // fused output projection (cluster variant): CTA r of head h's cluster multiplies the merged head output by the
+  // packed weight blocks (out-channel tile r, k-chunks of head h) and stores slab h of the split-K residual sum
+  const __nv_bfloat16* wo;   // packed [D/128][Nq/64] blocks of 128 x 64
+  const float* o_scale;      // per out channel, or null
+  const float* o_gate;       // per out channel, or null
+  float* slab;               // [Hq][rows][D]
+  size_t slab_stride;        // rows * D
+  int D;
+};
+// shared-memory barriers and tensor-memory base of the fused output projection
+struct OprojCtx {
+  uint32_t x_bar, w_bar, mma_bar, tmem;
 };
 
 // Shared-memory tiles are rows of DH bf16 with no padding; the 16-byte chunk c of row r sits at
@@ -85,9 +98,10 @@ __device__ __forceinline__ void group_sync() {
 // the rows of its partial (O, max, sum) into the shared memory of the CTA that owns them (bulk copies over
 // distributed shared memory, counted on the owner's mbarrier) and every CTA merges its own 8 of the 64 rows: no
 // partials in global memory, no merge kernel.  Needs 8 * 8 * (DH + 4) * 4 + 512 bytes of shared memory beyond the Q / K / V buffers.
-template <int DH, int HPC, int NBUF, int BAR, int KTT, bool CLUSTER = false>
+template <int DH, int HPC, int NBUF, int BAR, int KTT, bool CLUSTER = false, bool OPROJ = false>
 __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp, int b, uint32_t smem_base, int tid,
-                                          uint32_t mrg_bar = 0, volatile int* abort_flag = nullptr) {
+                                          uint32_t mrg_bar = 0, volatile int* abort_flag = nullptr,
+                                          OprojCtx oc = OprojCtx{}) {
   constexpr int ROWB = DH * 2;                // bytes per row
   constexpr int CH = DH / 8;                  // 16-byte chunks per row
   constexpr int NTHREADS = HPC * 128;
@@ -360,7 +374,22 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
     // finished with: the tile loop ends with a barrier), grouped by owner, then sent with one bulk copy per owner
     // (distributed shared memory, completion counted on the owner's mbarrier): remote stores from the threads
     // themselves measured ~3 us for the 64 KB.
-    const uint32_t stg = Ks, stg_ml = Ks + 8u * OWN_BYTES;
+    // (with the fused projection the staging area starts at the Q buffer instead, which is dead as well: the V
+    // buffers then take the projection's weight blocks and the tail of the K buffers its activation tile)
+    const uint32_t stg = OPROJ ? Qs : Ks, stg_ml = stg + 8u * OWN_BYTES;
+    constexpr uint32_t XK = 7u * 1024u;                                     // k-chunk pitch of the activation tile: 56 rows
+    const uint32_t xt = smem_base + ((8u * OWN_BYTES + 512u + 1023u) & ~1023u);   // [4][56 rows][128 B], swizzled
+    if constexpr (OPROJ) {
+      static_assert(DH == 256 && KTT == 64 && HPC == 1 && NBUF == 2, "fused projection: head_dim 256 only");
+      if (tid == 0) {
+        // the four 128 x 64 weight blocks of (out-channel tile = my rank, k-chunks of my head): 64 KB, contiguous
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const uint8_t* wsrc = reinterpret_cast<const uint8_t*>(a.wo) + ((size_t)split * (a.d.Nq / 64) + (size_t)head * 4) * 16384;
+        mbar_expect_tx(oc.w_bar, 65536u);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) bulk_g2s(Vs + (uint32_t)c * 16384u, wsrc + (size_t)c * 16384, 16384u, oc.w_bar);
+      }
+    }
 #pragma unroll
     for (int n = 0; n < DH / 8; ++n) {
       const uint32_t col = (uint32_t)(n * 8 + qd * 2) * 4;
@@ -418,10 +447,86 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
         }
       }
       const float inv = 1.0f / ll;
+      if constexpr (OPROJ) {
+        // my 16 columns of row r, as two 16-byte groups of k-chunk (tid & 15) / 4 of the projection's activation tile
+        const uint32_t base = xt + (uint32_t)((tid & 15) >> 2) * XK + (uint32_t)r * 128u;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const uint32_t grp = (uint32_t)((tid & 3) * 2 + u) ^ (uint32_t)(r & 7);
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(base + grp * 16u),
+                       "r"(pack_bf16(acc[8 * u] * inv, acc[8 * u + 1] * inv)), "r"(pack_bf16(acc[8 * u + 2] * inv, acc[8 * u + 3] * inv)),
+                       "r"(pack_bf16(acc[8 * u + 4] * inv, acc[8 * u + 5] * inv)), "r"(pack_bf16(acc[8 * u + 6] * inv, acc[8 * u + 7] * inv))
+                       : "memory");
+        }
+      } else {
 #pragma unroll
       for (int u = 0; u < CPT / 4; ++u)     // 4 consecutive columns = 8 bytes, inside one 16-byte chunk of the tiled layout
         *reinterpret_cast<uint2*>(a.out + out_index(b * S + r, head * DH + c0 + 4 * u, a.rows_pad, d.Nq)) =
             make_uint2(pack_bf16(acc[4 * u] * inv, acc[4 * u + 1] * inv), pack_bf16(acc[4 * u + 2] * inv, acc[4 * u + 3] * inv));
+      }
+    }
+    if constexpr (OPROJ) {
+      const WaitCtx wc{a.status, abort_flag, a.wait_limit};
+      // ---- all-gather of the merged rows: my rows go from my activation tile into the same place of every peer's
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      group_sync<BAR, NTHREADS>();
+      const int nr = max(0, min(8, S - split * 8));            // rows I own
+      if (tid < 32 && (tid & 7) != split && nr > 0) {
+        const uint32_t peer = (uint32_t)tid & 7u, kc = (uint32_t)tid >> 3;
+        const uint32_t loc = xt + kc * XK + (uint32_t)split * 1024u;
+        uint32_t dst, bar;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(loc), "r"(peer));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(oc.x_bar), "r"(peer));
+        asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                     "r"(loc), "r"((uint32_t)nr * 128u), "r"(bar)
+                     : "memory");
+      }
+      // ---- D[128 out channels][64 tokens] = W[128][256] X^T: 16 MMAs issued by warp 0
+      constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+      if (warp == 0) {
+        const bool okx = mbar_wait(oc.x_bar, 0u, wc);
+        const bool okw = mbar_wait(oc.w_bar, 0u, wc);
+        tc_fence_after();
+        if (__all_sync(0xffffffffu, okx && okw)) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint64_t da = make_desc(Vs + (uint32_t)c * 16384u), db = make_desc(xt + (uint32_t)c * XK);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (elect_one()) umma_bf16(oc.tmem, da + 2 * k, db + 2 * k, IDESC, (c | k) ? 1u : 0u);
+          }
+        }
+        if (elect_one()) umma_commit(oc.mma_bar);
+        __syncwarp();
+      }
+      // ---- epilogue: accumulator -> fp32 [token][128 + 4] in the (now idle) receive area -> slab `head`
+      const int ch = warp * 32 + lane;                       // TMEM lane = out channel within the tile
+      const int n = split * 128 + ch;
+      const float sc = (a.o_scale ? a.o_scale[n] : 1.0f) * (a.o_gate ? a.o_gate[n] : 1.0f);
+      const bool okm = mbar_wait(oc.mma_bar, 0u, wc);
+      tc_fence_after();
+      constexpr int PITCH = 132;
+      if (okm) {
+        for (int c0 = 0; c0 < S; c0 += 16) {
+          float v[16];
+          tmem_ld16(oc.tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(recv + (uint32_t)((c0 + j) * PITCH + ch) * 4u), "f"(v[j] * sc) : "memory");
+        }
+      }
+      tc_fence_before();
+      group_sync<BAR, NTHREADS>();
+      if (okm) {
+        float* dst = a.slab + (size_t)head * a.slab_stride + (size_t)(b * S) * a.D + split * 128;
+        for (int it = tid; it < S * 32; it += NTHREADS) {
+          const int tl = it >> 5, j0 = (it & 31) * 4;
+          float4 x;
+          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w)
+                       : "r"(recv + (uint32_t)(tl * PITCH + j0) * 4u) : "memory");
+          *reinterpret_cast<float4*>(dst + (size_t)tl * a.D + j0) = x;
+        }
+      }
     }
     // every CTA has received everything by now, i.e. every outgoing copy has finished reading its source: only
     // then may a CTA leave and release its shared memory
@@ -464,23 +569,55 @@ __global__ void __launch_bounds__(HPC * 128, 1) k_attn_mma(const AttnArgs a) {
   attn_role<DH, HPC, 2, 0, KTT>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x);
 }
 
-// Cluster variant: grid (8, heads, requests), cluster (8, 1, 1); see attn_role.
-template <int DH, int KTT>
+// Cluster variant: grid (8, heads, requests), cluster (8, 1, 1); see attn_role.  OPROJ: the output projection of
+// the head follows in the same kernel (tcgen05, accumulator in tensor memory) and leaves as slab `head` of the
+// split-K residual sum, so the merged attention output never goes to global memory.
+template <int DH, int KTT, bool OPROJ = false>
 __global__ void __launch_bounds__(128, 1) k_attn_cluster(const AttnArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t mrg_bar;
+  __shared__ __align__(8) uint64_t op_bar[3];
+  __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   pdl_launch_dependents();            // (the dependency wait and the status check are inside the role)
   if (threadIdx.x == 0) {
     abort_flag = 0;
     mbar_init(smem_u32(&mrg_bar), 1);
     mbar_expect_tx(smem_u32(&mrg_bar), 8u * (8u * (DH + 4) * 4u + 64u));   // eight sources: 8 rows of O and of (max, sum)
+    if (OPROJ) {
+      for (int i = 0; i < 3; ++i) mbar_init(smem_u32(&op_bar[i]), 1);
+      // merged rows of the seven peers: every row of the suffix but my own, four 128-byte pieces each
+      const int mine = max(0, min(8, a.d.S - (int)blockIdx.x * 8));
+      mbar_expect_tx(smem_u32(&op_bar[0]), (uint32_t)(a.d.S - mine) * 512u);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // every CTA's merge barrier exists before any peer can send to it (this runs before the dependency wait)
+  OprojCtx oc{};
+  if (OPROJ) {
+    if (threadIdx.x < 32) {
+      tmem_alloc(smem_u32(&tmem_slot), 64);
+      tc_fence_before();
+    }
+  }
+  // every CTA's barriers exist before any peer can send to them (this runs before the dependency wait)
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-  attn_role<DH, 1, 2, 0, KTT, true>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_u32(smem_raw), threadIdx.x,
-                                    smem_u32(&mrg_bar), &abort_flag);
+  if (OPROJ) {
+    __syncthreads();
+    tc_fence_after();
+    oc.x_bar = smem_u32(&op_bar[0]), oc.w_bar = smem_u32(&op_bar[1]), oc.mma_bar = smem_u32(&op_bar[2]);
+    oc.tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  }
+  // (the projection's operands need 1024-byte aligned tiles: the launch adds 1 KB of slack for this)
+  const uint32_t smem_base = OPROJ ? ((smem_u32(smem_raw) + 1023u) & ~1023u) : smem_u32(smem_raw);
+  attn_role<DH, 1, 2, 0, KTT, true, OPROJ>(a, blockIdx.x, blockIdx.y, blockIdx.z, smem_base, threadIdx.x,
+                                           smem_u32(&mrg_bar), &abort_flag, oc);
+  if (OPROJ) {
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      tc_fence_after();
+      tmem_dealloc(oc.tmem, 64);
+    }
+  }
 }
 
 }  // namespace

@@ -87,6 +87,7 @@ struct phyai_expert {
   int use_mega = 0;   // the captured per-operator loop measured faster (10.0 vs 12.6 ms on the pi0-shaped expert): opt-in
   int use_tc_attention = 1;
   int use_cluster_attention = 1;
+  int use_fused_oproj = 1;     // cluster attention also does the output projection of its head (one request, head_dim 256)
   int use_pair_gemm = 0;   // measured slower than the single-CTA kernel on the batch-64 shapes: opt-in
   int n_sm = 0;
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
@@ -380,6 +381,10 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
                            batch * (d.Hq / 2) >= ATTN_TC_MIN_CTAS;
       const bool attn_cluster = !attn_tc && h->attn_mma && h->use_cluster_attention && batch * d.Hq * 8 <= 2 * h->n_sm;
       const bool attn_rot = h->qr_big && (attn_tc || attn_cluster);   // q / k / v leave the QKV epilogue rotated, bf16
+      // one token tile: the cluster attention kernel multiplies each head's output by its slice of Wo itself and
+      // writes one slab per head, which the next norm sums like the k-range partials of a split-K GEMM
+      const bool fuse_o = attn_cluster && attn_rot && h->tc && h->use_fused_oproj && h->slab && M <= 64 &&
+                          d.Hq <= MAX_SLABS && attention_oproj_supported(d);
       if (h->tc) {
         TcGemm g{};
         g.W = h->p_qkv[l], g.X = h->xn_t, g.N = d.Nqkv, g.K = D, g.epi = TC_STORE, g.scale = h->s_qkv[l];
@@ -404,10 +409,13 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         ++cnt;
       } else if (attn_cluster) {
         // few requests: 8 key ranges per head in a cluster of 8 CTAs, merged through distributed shared memory
+        const AttnOproj op{h->p_o[l], h->s_o[l], gate, h->slab, (size_t)M * D};
         cudaError_t e = launch_attention_cluster(h->rq, h->status, h->qkv, h->rope, attn_rot ? h->qr_big : nullptr, h->kr_big,
-                                                 h->vr_big, l, h->attn_t, h->Mpad, d, batch, h->wait_limit, st);
+                                                 h->vr_big, l, h->attn_t, h->Mpad, d, batch, h->wait_limit, st,
+                                                 fuse_o ? &op : nullptr);
         if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
         ++cnt;
+        if (fuse_o) pending_slabs = d.Hq;
       } else if (h->attn_mma) {
         const int splits = attention_pick_splits(d, batch, (int)h->cfg.max_prefix_len);
         cudaError_t e = launch_attention_mma(h->rq, h->status, h->qkv, h->rope, l, h->attn_t, h->Mpad, splits,
@@ -419,7 +427,9 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
                               h->Mpad, d, batch, st);
         ++cnt;
       }
-      if (h->tc) {
+      if (fuse_o) {
+        // (projected inside the attention kernel)
+      } else if (h->tc) {
         TcGemm g{};
         g.W = h->p_o[l], g.X = h->attn_t, g.N = D, g.K = d.Nq, g.epi = TC_RESID, g.scale = h->s_o[l], g.gate = gate;
         g.out_f32 = h->h, g.ldo = D, g.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.Nq / 64);
@@ -947,6 +957,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   if (!strcmp(key, "slab_splits")) {
     if (value < 1 || value > MAX_SLABS) return fail(PHYAI_ERR_INVALID_ARG, "slab_splits out of range");
     h->slab_splits = (int)value;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_fused_oproj")) {
+    h->use_fused_oproj = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

@@ -113,10 +113,20 @@ cudaError_t launch_attention_mma(const Request* rq, int* status, const float* qk
 
 // ---- tcgen05 attention (large batches: two heads per CTA, whole key range, no split) ------------------
 bool attention_tc_supported(const Dims& d);
+// Output projection fused into the cluster attention kernel: packed weight blocks of the layer, optional per-channel
+// weight scale and residual gate, and the slab array [Hq][rows][D] that receives one partial per head.
+struct AttnOproj {
+  const __nv_bfloat16* wo;
+  const float* scale;
+  const float* gate;
+  float* slab;
+  size_t slab_stride;
+};
+bool attention_oproj_supported(const Dims& d);
 cudaError_t launch_attention_cluster(const Request* rq, int* status, const float* qkv, const float2* rope,
                                      const __nv_bfloat16* qr, const __nv_bfloat16* kr, const __nv_bfloat16* vr, int layer,
                                      __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
-                                     cudaStream_t st);
+                                     cudaStream_t st, const AttnOproj* op = nullptr);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
                                 int batch, const int* order, unsigned wait_limit, cudaStream_t st);

@@ -81,15 +81,17 @@ def test_small_bf16_other_head_sizes_through_every_batch1_path(head_dim, n_q, n_
 @pytest.mark.parametrize("name", ["C2", "C3"])
 def test_pi_shaped_bf16_batch1_matches_oracle(name):
     """Full-size batch-1 configurations through the default path (captured per-operator loop: rotary QKV epilogue,
-    cluster-merged attention, interleaved GeGLU tiles), through the same loop with the split attention + merge
-    kernels, and through the persistent kernel."""
+    cluster-merged attention with the output projection fused in, interleaved GeGLU tiles), through the same loop
+    with a separate output projection, with the split attention + merge kernels, and through the persistent
+    kernel."""
     wl = synth.WORKLOADS[name]
     cfg = synth.pi0_config() if name == "C2" else synth.pi05_config()
     W = synth.make_weights(cfg, wl["cfg_id"])
     kv, state, noise = _inputs(cfg, wl["cfg_id"], wl["prefix"])
     ref = O.denoise(cfg, W, kv, wl["prefix"], state, noise, wl["n_steps"])
     with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
-        for label, opts in (("default", {}), ("split attention", {"use_cluster_attention": 0}),
+        for label, opts in (("default", {}), ("separate output projection", {"use_fused_oproj": 0}),
+                            ("split attention", {"use_fused_oproj": 1, "use_cluster_attention": 0}),
                             ("persistent", {"use_cluster_attention": 1, "use_persistent": 1})):
             for k, v in opts.items():
                 ex.set_option(k, v)
