@@ -499,34 +499,24 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
         if (elect_one()) umma_commit(oc.mma_bar);
         __syncwarp();
       }
-      // ---- epilogue: accumulator -> fp32 [token][128 + 4] in the (now idle) receive area -> slab `head`
+      // ---- epilogue: accumulator -> slab `head`.  A warp holds 32 consecutive out channels of every token, so
+      // its stores are whole 128-byte lines without a transpose.
       const int ch = warp * 32 + lane;                       // TMEM lane = out channel within the tile
       const int n = split * 128 + ch;
       const float sc = (a.o_scale ? a.o_scale[n] : 1.0f) * (a.o_gate ? a.o_gate[n] : 1.0f);
       const bool okm = mbar_wait(oc.mma_bar, 0u, wc);
       tc_fence_after();
-      constexpr int PITCH = 132;
       if (okm) {
+        float* dst = a.slab + (size_t)head * a.slab_stride + (size_t)(b * S) * a.D + n;
         for (int c0 = 0; c0 < S; c0 += 16) {
           float v[16];
           tmem_ld16(oc.tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
 #pragma unroll
           for (int j = 0; j < 16; ++j)
-            asm volatile("st.shared.f32 [%0], %1;" ::"r"(recv + (uint32_t)((c0 + j) * PITCH + ch) * 4u), "f"(v[j] * sc) : "memory");
+            if (c0 + j < S) dst[(size_t)(c0 + j) * a.D] = v[j] * sc;
         }
       }
       tc_fence_before();
-      group_sync<BAR, NTHREADS>();
-      if (okm) {
-        float* dst = a.slab + (size_t)head * a.slab_stride + (size_t)(b * S) * a.D + split * 128;
-        for (int it = tid; it < S * 32; it += NTHREADS) {
-          const int tl = it >> 5, j0 = (it & 31) * 4;
-          float4 x;
-          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w)
-                       : "r"(recv + (uint32_t)(tl * PITCH + j0) * 4u) : "memory");
-          *reinterpret_cast<float4*>(dst + (size_t)tl * a.D + j0) = x;
-        }
-      }
     }
     // every CTA has received everything by now, i.e. every outgoing copy has finished reading its source: only
     // then may a CTA leave and release its shared memory
