@@ -51,7 +51,12 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   constexpr int B_PIECE = B_BYTES / NB;
   constexpr int NCOPY = NA + NB;
   constexpr int STAGE_BYTES = A_BYTES * NA + B_BYTES;
-  constexpr int COLS = NA * NT;
+  // Single 64-token tile: two warps issue MMAs, one the even k-steps, one the odd ones, each into an accumulator of
+  // its own (the epilogue adds the two).  The issue sequence of a k-step (four N = 64 MMAs of ~55 clocks each)
+  // takes one thread ~350 clocks plus the wait for the next stage, so a single issuer, not the tensor pipe, set
+  // the pace of these launches.
+  constexpr bool DUAL = NT == 64 && NA == 1;
+  constexpr int COLS = NA * NT * (DUAL ? 2 : 1);
   constexpr int ALLOC_COLS = COLS <= 32 ? 32 : COLS <= 64 ? 64 : COLS <= 128 ? 128 : COLS <= 256 ? 256 : 512;   // power of two
   // A producer warp's consecutive copies are NPROD / NCOPY k-steps apart; its parity wait on "stage free" is only
   // meaningful while that step does not exceed the ring depth.
@@ -71,9 +76,14 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int skip_flag;
+  __shared__ int epi_ok;
   __shared__ int2 tok_tab[NT];   // TC_QKV_ROT: per token of the tile (position, request * 64 + suffix row)
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // The warp index and the tensor-memory base are broadcast from lane 0: the compiler then knows that they are the
+  // same in every lane, keeps the role branches and the MMA operands (descriptors, addresses) in the uniform
+  // datapath, and the issue sequence of one k-step shrinks (measured in a stand-alone model of this main loop:
+  // 530 -> 410 clocks per k-step of four N = 64 MMAs).
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int nt_idx = blockIdx.x, tt = blockIdx.y;
   const bool geglu = g.epi == TC_GEGLU;
   const int KC = g.K >> 6;
@@ -93,7 +103,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       mbar_init(smem_u32(&bar_full[s]), NCOPY);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
-    mbar_init(smem_u32(&bar_accum), 1);
+    mbar_init(smem_u32(&bar_accum), DUAL ? 2 : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 8) {
@@ -102,7 +112,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   }
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *reinterpret_cast<volatile uint32_t*>(&tmem_slot), 0);
   const WaitCtx wc{status, &abort_flag, g.wait_limit};
 
   // weight tile of accumulator a: GeGLU pairs the gate and up tiles of the same channels, otherwise
@@ -113,8 +123,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     return reinterpret_cast<const uint8_t*>(base) + ((size_t)tile * KC + kc_begin) * A_BYTES;
   };
   const int n_early = nk < STAGES ? (nk > 0 ? nk : 0) : STAGES;   // stages whose weight copies are issued before the wait
-  const int issuer = warp < NPROD ? warp : warp - 1;              // producer warps 0..7, then epilogue warps 9.. -> 8..
-  const bool issues = lane == 0 && warp != 8 && issuer < NISSUE;
+  // copy issuers: producer warps 0..7, then the epilogue warps that are idle during the main loop (with two MMA
+  // warps the first epilogue warp is not)
+  const int issuer = warp < NPROD ? warp : warp - (DUAL ? 2 : 1);
+  const bool issues = lane == 0 && warp != 8 && !(DUAL && warp == 9) && issuer < NISSUE;
   if (issues) {
     for (int id = issuer; id < n_early * NCOPY; id += NISSUE) {
       const int i = id / NCOPY, c = id % NCOPY;
@@ -170,11 +182,11 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     }
   }
   __syncwarp();
-  if (warp < NPROD) {
-    // (producer warps have nothing else to do)
-  } else if (warp == 8) {
-    // ---------------- MMA issuer (whole warp in the loop, one elected lane issues) ---------------------
-    for (int i = 0; i < nk; ++i) {
+  if (warp == 8 || (DUAL && warp == 9)) {
+    // ---------------- MMA issuer(s) (whole warp in the loop, one elected lane issues) ---------------------
+    const int first = DUAL ? warp - 8 : 0, step = DUAL ? 2 : 1;
+    const uint32_t tacc = tmem_base + (DUAL ? (uint32_t)(warp - 8) * NT : 0u);
+    for (int i = first; i < nk; i += step) {
       const int s = i % STAGES;
       const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
       const bool ok = mbar_wait(smem_u32(&bar_full[s]), ph, wc);
@@ -190,18 +202,23 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       if (__all_sync(0xffffffffu, ok)) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
-          const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
-          if (elect_one()) umma_bf16(tmem_base, da + 2 * k, db + 2 * k, IDESC, acc);
+          const uint32_t acc = (i > first || k > 0) ? 1u : 0u;   // the warp's first MMA initialises its accumulator
+          if (elect_one()) umma_bf16(tacc, da + 2 * k, db + 2 * k, IDESC, acc);
           if (NA == 2) {
-            if (elect_one()) umma_bf16(tmem_base + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
+            if (elect_one()) umma_bf16(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
           }
         }
       }
-      if (elect_one()) umma_commit(smem_u32(&bar_empty[s]));  // frees the stage when the MMAs above have read it
+      // frees the stage when the MMAs above have read it -- only if a later k-step will reuse the stage (a commit
+      // that nobody waits for still costs the issuing thread time)
+      if (i + STAGES < nk && elect_one()) umma_commit(smem_u32(&bar_empty[s]));
       __syncwarp();
     }
     if (elect_one()) umma_commit(smem_u32(&bar_accum));
     __syncwarp();
+  }
+  if (warp <= 8) {
+    // (producer warps and the first MMA warp have nothing else to do)
   } else {
     // ---------------- epilogue: TMEM -> registers -> global --------------------------------------
     const int ew = warp - 9;                      // 0..15
@@ -209,6 +226,16 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     const int et = ew * 32 + lane;                // 0..511
     const int ch = q * 32 + lane;                 // row of the 128-row tile
     const int tok_base = tt * NT;
+    // 16 accumulator columns of this thread's TMEM lane (two MMA warps: the sum of their accumulators)
+    auto ld_acc = [&](uint32_t col, float* v) {
+      tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + col, v);
+      if (DUAL && nk > 1) {
+        float w[16];
+        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)NT + col, w);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] += w[j];
+      }
+    };
     if (g.epi == TC_QKV_ROT) {
       // while the main loop runs: where each token of the tile sits (request, suffix row, rotary position)
       for (int idx = et; idx < NT; idx += NEPI) {
@@ -266,7 +293,14 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         }
       }
     }
-    const bool ok = mbar_wait(smem_u32(&bar_accum), 0, wc);
+    // one epilogue warp polls the accumulator barrier; the other fifteen wait for it at the named barrier (in
+    // hardware), so that the main loop's shared-memory port is not shared with 512 polling threads
+    if (ew == 0) {
+      const bool okw = mbar_wait(smem_u32(&bar_accum), 0, wc);
+      if (lane == 0) epi_ok = okw ? 1 : 0;
+    }
+    epi_sync();
+    const bool ok = *reinterpret_cast<volatile int*>(&epi_ok) != 0;
     tc_fence_after();
     constexpr int HALF = NT / 4;   // token columns per epilogue warp
     const int c_begin = hf * HALF;
@@ -282,7 +316,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;  // warp-uniform
           float v[16];
-          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NT + c0), v);
+          ld_acc((uint32_t)(a * NT + c0), v);
           if (g.epi == TC_RESID && gridDim.z == 1) {
             // single owner per element: plain read-modify-write, with the 16 loads issued before any is used
             float old[16];
@@ -329,7 +363,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;
           float v[16];
-          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+          ld_acc((uint32_t)c0, v);
 #pragma unroll
           for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * 64 + c64] = v[j] * su;
         }
@@ -340,7 +374,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;
           float v[16];
-          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+          ld_acc((uint32_t)c0, v);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int t = c0 + j;
@@ -372,7 +406,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
           for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
             if (tok_base + c0 >= g.M) break;          // warp-uniform
             float v[16];
-            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NT + c0), v);
+            ld_acc((uint32_t)(a * NT + c0), v);
 #pragma unroll
             for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * PITCH + ch] = v[j] * sc;
           }
@@ -413,7 +447,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
           for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
             if (tok_base + c0 >= g.M) break;          // warp-uniform
             float v[16];
-            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NT + c0), v);
+            ld_acc((uint32_t)(a * NT + c0), v);
 #pragma unroll
             for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * PITCH + ch] = v[j] * sc;
           }
