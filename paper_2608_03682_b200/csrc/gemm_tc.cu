@@ -357,28 +357,34 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       // the bf16 result as the swizzled image of k-chunk `tile` of the down projection's input.
       float* stage = reinterpret_cast<float*>(tiles_ptr);                                  // [NT][64] up values
       __nv_bfloat16* img = reinterpret_cast<__nv_bfloat16*>(stage + (size_t)NT * 64);      // [NT][64] bf16, swizzled
-      const int c64 = ch & 63, f = nt_idx * 64 + c64;
-      if (ok && q >= 2) {
-        const float su = e_il;
-        for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
+      const int c64 = ch & 63;
+      float gel[HALF / 16][16];   // gate half: gelu(gate), computed while the up half is on its way through shared memory
+      if (ok) {
+#pragma unroll
+        for (int u = 0; u < HALF / 16; ++u) {
+          const int c0 = c_begin + u * 16;
           if (tok_base + c0 >= g.M) break;
           float v[16];
           ld_acc((uint32_t)c0, v);
+          if (q >= 2) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * 64 + c64] = v[j] * su;
+            for (int j = 0; j < 16; ++j) stage[(size_t)(c0 + j) * 64 + c64] = v[j] * e_il;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) gel[u][j] = gelu_fast(v[j] * e_il, g.gelu_exact);
+          }
         }
       }
       epi_sync();
       if (ok && q < 2) {
-        const float sg = e_il;
-        for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
+#pragma unroll
+        for (int u = 0; u < HALF / 16; ++u) {
+          const int c0 = c_begin + u * 16;
           if (tok_base + c0 >= g.M) break;
-          float v[16];
-          ld_acc((uint32_t)c0, v);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int t = c0 + j;
-            const float m = gelu_fast(v[j] * sg, g.gelu_exact) * stage[(size_t)t * 64 + c64];
+            const float m = gel[u][j] * stage[(size_t)t * 64 + c64];
             img[(size_t)t * 64 + (((c64 >> 3) ^ (t & 7)) << 3) + (c64 & 7)] = __float2bfloat16_rn(m);
           }
         }
