@@ -35,7 +35,7 @@ METRIC_BATCHED = "chunks/sec at batch %d"
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (bench.py cannot run ncu itself)
-NCU_TRAFFIC = {"C2": (6.406718e9 + 0.137829e9, "profiles/per_operator_loop_c2_batch1.md")}
+NCU_TRAFFIC = {"C2": (6.406537e9 + 0.148150e9, "profiles/per_operator_loop_c2_batch1.md")}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 
 
