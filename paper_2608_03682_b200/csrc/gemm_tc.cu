@@ -148,8 +148,17 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
              B_PIECE, full);
   };
   if (issues) {
-    for (int id = issuer; id < n_early * NCOPY; id += NISSUE)
-      if (id % NCOPY >= NA) issue_x(id / NCOPY, id % NCOPY - NA, (uint32_t)(id / NCOPY));
+    if constexpr (NT == 64 && NA == 1) {
+      // Concurrent copies share the SM's ingest rate, so with one issuer per stage all activation tiles would land
+      // together, late; XW issuers taking the stages round robin (a warp's copies complete in order) bring the
+      // first stages in first.
+      constexpr int XW = 3;   // 1 / 2 / 3 / 5 / 9 issuers measured 7.26 / 7.23 / 7.19 / 7.18 / 7.20 ms per batch-1 chunk
+      if (issuer < XW)
+        for (int i = issuer; i < n_early; i += XW) issue_x(i, 0, (uint32_t)i);
+    } else {
+      for (int id = issuer; id < n_early * NCOPY; id += NISSUE)
+        if (id % NCOPY >= NA) issue_x(id / NCOPY, id % NCOPY - NA, (uint32_t)(id / NCOPY));
+    }
   }
   if (threadIdx.x == NPROD * 32) skip_flag = status_set(status) || nk <= 0;
   __syncthreads();
