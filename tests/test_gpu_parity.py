@@ -101,6 +101,29 @@ def test_pi_shaped_bf16_batch1_matches_oracle(name):
             assert err <= BAR["bf16"], (label, err)
 
 
+@pytest.mark.parametrize("cond,horizon,block_causal", [("pi0", 50, False), ("pi0", 7, True), ("pi05", 55, False),
+                                                       ("pi05", 16, False)])
+def test_full_width_two_layer_expert_through_the_fused_attention_projection(cond, horizon, block_causal):
+    """Width 1024, 8 heads of 256: the shapes for which the cluster attention kernel also applies the output
+    projection.  Two layers keep the oracle fast; prefix lengths cover no prefix at all, key ranges without tiles,
+    a ragged last tile and the maximum; suffix lengths cover owners without rows (8 rows), a full 8-row owner
+    boundary (16 / 56 rows) and the usual 51.  Each case also runs with the separate projection kernel."""
+    cfg = synth.ExpertConfig(n_layers=2, width=1024, mlp_dim=4096, n_q_heads=8, n_kv_heads=1, head_dim=256,
+                             state_dim=32, action_dim=32, horizon=horizon, has_state_token=(cond == "pi0"),
+                             max_prefix_len=968, max_batch=1, cond=cond, dtype="bf16",
+                             suffix_block_causal=block_causal)
+    W = synth.make_weights(cfg, 21)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        for P in (0, 5, 130, 816, 968):
+            kv, state, noise = _inputs(cfg, 21, P)
+            ref = O.denoise(cfg, W, kv, P, state, noise, 3)
+            for fused in (1, 0):
+                ex.set_option("use_fused_oproj", fused)
+                got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
+                err = rel_err(got, ref)
+                assert err <= BAR["bf16"], (P, fused, err)
+
+
 # ------------------------------------------------------------------------------------------ batched, ragged
 def _batched_case(cfg, cfg_id, lens, n_steps, check, engine="auto", std=0.05):
     W = synth.make_weights(cfg, cfg_id, std=std)
