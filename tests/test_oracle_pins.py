@@ -17,7 +17,9 @@ torch.set_num_threads(4)
 
 
 def small_cfg(cond="pi0", D=16, dh=4, Hq=2, Hkv=1, Fm=32, L=2, H=3, ns=True, A=3, Ds=5, P=6, rope=10000.0,
-              gelu_exact=False):
+              gelu_exact=False, heads=None):
+    if heads is not None:
+        Hq, Hkv = heads
     if cond == "pi05":
         ns = False
     return synth.ExpertConfig(n_layers=L, width=D, mlp_dim=Fm, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=dh,
@@ -37,7 +39,8 @@ def rand_inputs(cfg, P, seed=0, std=0.3):
 cfg_strategy = st.builds(
     small_cfg,
     cond=st.sampled_from(["pi0", "pi05"]), D=st.sampled_from([8, 16, 32]), dh=st.sampled_from([2, 4, 8]),
-    Hq=st.sampled_from([1, 2, 4]), Hkv=st.just(1), Fm=st.sampled_from([16, 32]), L=st.integers(1, 3),
+    heads=st.sampled_from([(1, 1), (2, 1), (2, 2), (4, 1), (4, 2)]),   # (query heads, kv heads): grouped-query maps a // G
+    Fm=st.sampled_from([16, 32]), L=st.integers(1, 3),
     H=st.integers(1, 5), ns=st.booleans(), A=st.integers(1, 7), Ds=st.integers(1, 8), P=st.integers(0, 9),
     rope=st.sampled_from([0.0, 10000.0]), gelu_exact=st.booleans())
 fast = settings(max_examples=12, deadline=None, suppress_health_check=list(HealthCheck))
