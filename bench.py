@@ -183,6 +183,8 @@ def main():
     ap.add_argument("--impl", default="phyai", choices=["phyai", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--opt", action="append", default=[], metavar="KEY=VALUE",
+                    help="library option set on the handle before timing (phyai_set_option), may repeat")
     args = ap.parse_args()
     K, Wm = args.steps, max(args.warmup, 3)
 
@@ -229,6 +231,9 @@ def main():
     ex = binding.Expert(cfg, binding.weights_to_device(W))
     if args.no_graph:
         ex.set_option("use_graph", 0)
+    for kv_ in args.opt:
+        key, _, val = kv_.partition("=")
+        ex.set_option(key, int(val))
     del W
     kvs = [synth.make_prefix_kv(cfg, cfg_id, p, b) for b, p in enumerate(lens)]
     kv_h, cu = synth.pack_prefix_kv(kvs)

@@ -191,35 +191,35 @@ phyai_status_t phyai_denoise_batched_host(phyai_expert_t *h, uint32_t batch, con
  */
 phyai_status_t phyai_poll_status(phyai_expert_t *h);
 
-/* Options. key "use_graph": 0 launches the kernels directly, 1 (default) replays a captured CUDA
- * graph per (batch, n_steps).  key "use_persistent": 1 runs calls with batch * suffix_len <= 64
- * tokens as one persistent cooperative kernel (the whole n-step loop, no kernel boundaries; bit-reproducible run
- * to run), 0 (default) uses the per-operator kernels, captured as one CUDA graph, for every batch: with
- * programmatic dependent launch they measured faster than the persistent kernel.  key "use_tc_attention": 1 (default) lets large
- * batches use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "use_cluster_attention": 1 (default) lets calls with few
- * requests merge their key-split attention partials through distributed shared memory (clusters of 8 CTAs), 0
- * keeps the split kernel + merge kernel.  key "use_fused_oproj": 1 (default) lets that cluster kernel also apply the
- * attention output projection of its head (head_dim 256, model width 1024, one token tile; one partial per head,
- * summed in head order by the next kernel), 0 keeps the separate projection.  key "use_pair_gemm": 1 runs the
- * GEMMs of batches above 1024 tokens on CTA pairs (tcgen05 cta_group::2, persistent, overlapped epilogue), 0
- * (default) keeps the single-CTA kernel, which measured faster on the batch-64 shapes.
- * key "slab_splits": 1..16 (default 8), the most k-ranges a residual projection of a single-token-tile call is split into
- * (its partial sums are written as slabs and added in slab order by the next kernel: bit-reproducible).
- * key "wait_limit": iteration bound of
- * device-side waits (testing).  Unknown key -> INVALID_ARG. */
+/* Options (testing and measurement aids).  key "use_graph": 0 launches the kernels directly, 1 (default)
+ * replays a captured CUDA graph per (batch, n_steps).  key "use_tc_attention": 1 (default) lets large batches
+ * use the tcgen05 attention kernel, 0 keeps the mma.sync kernel.  key "use_cluster_attention": 1 (default) lets
+ * calls with few requests merge their key-split attention partials through distributed shared memory (clusters
+ * of 8 CTAs), 0 keeps the split kernel + merge kernel.  key "use_fused_oproj": 1 lets that cluster kernel also
+ * apply the attention output projection of its head (head_dim 256, model width 1024, one token tile).
+ * key "use_cluster_gemm": 1 (default) runs the projections of calls with at most 64 suffix tokens on the
+ * cluster split-K kernel (k-ranges of a channel tile reduce over distributed shared memory; the norms are
+ * folded into the neighbouring projections), 0 keeps the general kernel + norm kernels.
+ * key "slab_splits": 1..16 (default 8), the most k-ranges a residual projection of a single-token-tile call is
+ * split into on the general kernel (partial sums are written as slabs and added in slab order: bit-reproducible).
+ * key "b1_c_qkv" / "b1_c_o" / "b1_c_gu" / "b1_c_d": cluster size (k-ranges per channel tile, 1..8; 0 = choose) of
+ * the four projections on the cluster split-K kernel.  key "trace": see phyai_read_trace.
+ * key "wait_limit": iteration bound of the device-side waits on other agents' progress (testing).
+ * Unknown key -> INVALID_ARG. */
 phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t value);
 
 /*
- * Tracing aid (the paper times phases with GPU-side profiler scopes; Sec. "Results", measurement
- * protocol).  With option "trace" = step * 1000 + layer the persistent kernel records, for that
- * step and layer, four device-global-timer stamps (ns) per CTA and phase: inputs ready (for a
- * GEMM role: accumulator complete), role done, and for GEMM roles first activations in shared memory and
- * last MMA issued.  After the stream is synchronised phyai_read_trace copies them to `out` (HOST
- * memory, capacity >= 148 * 11 * 4 entries) as [cta][phase][4]; unused slots are 0.  Phases in order: norm1,
- * qkv, attention, merge, o-proj, norm2, gate/up, down, embed, embed-gemm, final.  "trace" = -1 turns it off.
+ * Tracing aid (the paper times phases with GPU-side profiler scopes; Sec. "Results", measurement protocol).
+ * With option "trace" = 1, one CTA of every cluster-GEMM and cluster-attention launch of a call writes
+ * device-global-timer stamps (ns) into slot `launch index` (position of the launch within the call, from 0) of a
+ * 4096 x 8 buffer: [0] kernel start, [1] set-up done, [2] dependency resolved (for attention: Q acquired),
+ * [3] MMAs / key tiles complete, [4] partials of the cluster received, [5] results stored, [6] cluster released,
+ * [7] (GEMM) the SM the CTA ran on.  After the stream is synchronised phyai_read_trace copies the buffer to `out`
+ * (HOST memory, capacity >= 4096 * 8 entries); slots of launches that are not traced stay 0.  The stamps cost
+ * a few hundred ns each: a traced call is slower.  "trace" = 0 turns it off.
  */
-phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_ctas,
-                                uint32_t *n_phases);
+phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_slots,
+                                uint32_t *n_stamps);
 
 /* Number of kernel launches (graph nodes) one denoise call with this batch / n_steps issues;
  * 0 if unknown.  Reporting aid for benchmarks. */
@@ -235,13 +235,15 @@ uint64_t phyai_launches_per_call(phyai_expert_t *h, uint32_t batch, uint32_t n_s
  *   qkv             device float32 [batch*suffix_len][(Hq + 2 Hkv) * head_dim] = (q | k | v) rows of
  *                   the suffix tokens, NOT yet rotated
  *   prefix_kv       device bfloat16 [n_layers][2][kv_tokens][Hkv][head_dim]; planes of `layer` are read
- *   cu_prefix_lens  device int32 [batch+1]
+ *   cu_prefix_lens  device int32 [batch+1], non-decreasing, cu[0] >= 0, cu[batch] <= kv_tokens (checked on the
+ *                   device: a violation sets *status_word to PHYAI_ERR_INVALID_ARG and nothing is written);
+ *                   batch <= 65535
  *   rope_cos_sin    device float32 [positions][head_dim/2][2] = (cos, sin) of position * theta^(-2j/dh)
  *                   for every position < max prefix_len + suffix_len, or NULL for no rotation;
  *                   suffix token i of a request sits at position prefix_len + i
  *   out             device bfloat16 (as uint16) row-major [batch*suffix_len][Hq*head_dim]
- *   status_word     device int32, zeroed by the caller; stays 0 on success, becomes
- *                   PHYAI_ERR_TIMEOUT if a bounded wait inside the kernel expired
+ *   status_word     device int32, zeroed by the caller; stays 0 on success, becomes PHYAI_ERR_INVALID_ARG
+ *                   (cu_prefix_lens) or PHYAI_ERR_TIMEOUT (a bounded wait inside the kernel expired)
  *
  * Split-KV partial results need scratch memory: this entry point takes it from the stream-ordered
  * allocator (cudaMallocAsync / cudaFreeAsync on `stream`).  Only enqueues work.  Errors: INVALID_ARG,

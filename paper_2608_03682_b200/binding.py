@@ -90,9 +90,9 @@ def load_library() -> C.CDLL:
     lib.phyai_denoise_batched_host.argtypes = batched
     lib.phyai_poll_status.argtypes = [_VP]
     lib.phyai_set_option.argtypes = [_VP, C.c_char_p, C.c_int64]
+    lib.phyai_read_trace.argtypes = [_VP, _VP, C.c_size_t, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
     lib.phyai_launches_per_call.argtypes = [_VP, C.c_uint32, C.c_uint32]
     lib.phyai_launches_per_call.restype = C.c_uint64
-    lib.phyai_read_trace.argtypes = [_VP, _VP, C.c_size_t, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
     lib.phyai_op_last_error.restype = C.c_char_p
     lib.phyai_suffix_attention_scratch_bytes.restype = C.c_size_t
     lib.phyai_suffix_attention_scratch_bytes.argtypes = [C.POINTER(AttentionDesc), C.c_uint32]
@@ -248,12 +248,12 @@ class Expert:
         _check(self.lib.phyai_set_option(self._handle, key.encode(), int(value)))
 
     def read_trace(self) -> np.ndarray:
-        """Per-CTA, per-phase device timestamps in ns: array [ctas, phases, 4]."""
-        buf = np.zeros(148 * 11 * 4, dtype=np.uint64)
-        n_ctas, n_ph = C.c_uint32(), C.c_uint32()
-        _check(self.lib.phyai_read_trace(self._handle, buf.ctypes.data_as(_VP), buf.size, C.byref(n_ctas),
-                                         C.byref(n_ph)))
-        return buf.reshape(n_ctas.value, n_ph.value, 4)
+        """Timer stamps (ns) of the traced launches of the last call: array [slots, 8] (option "trace" = 1)."""
+        buf = np.zeros(4096 * 8, dtype=np.uint64)
+        n_slots, n_st = C.c_uint32(), C.c_uint32()
+        _check(self.lib.phyai_read_trace(self._handle, buf.ctypes.data_as(_VP), buf.size, C.byref(n_slots),
+                                         C.byref(n_st)))
+        return buf.reshape(n_slots.value, n_st.value)
 
     def launches_per_call(self, batch: int, n_steps: int) -> int:
         return int(self.lib.phyai_launches_per_call(self._handle, batch, n_steps))

@@ -59,12 +59,12 @@ constexpr size_t attn_smem() {
 
 template <int DH, int HPC, int KTT>
 cudaError_t launch_attn(const AttnArgs& a, int batch, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce once;
+  if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(k_attn_mma<DH, HPC, KTT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)attn_smem<DH, HPC, KTT>());
     if (e != cudaSuccess) return e;
-    configured = true;
+    once.done();
   }
   dim3 grid(a.num_splits, a.d.Hq / HPC, batch);
   cudaError_t e = launch_pdl(k_attn_mma<DH, HPC, KTT>, grid, dim3(HPC * 128), attn_smem<DH, HPC, KTT>(), st, a);
@@ -83,12 +83,12 @@ constexpr size_t attn_cluster_smem() {   // Q / K / V buffers + the receive area
 
 template <int DH, int KTT, bool OPROJ = false>
 cudaError_t launch_attn_cluster(const AttnArgs& a, int batch, cudaStream_t st) {
-  static bool configured = false;
+  static PerDeviceOnce once;
   const size_t smem = attn_cluster_smem<DH, KTT>() + (OPROJ ? 1024 : 0);
-  if (!configured) {
+  if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(k_attn_cluster<DH, KTT, OPROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    once.done();
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(8, a.d.Hq, batch), cfg.blockDim = dim3(128), cfg.dynamicSmemBytes = smem, cfg.stream = st;
@@ -108,8 +108,9 @@ cudaError_t launch_attn_cluster(const AttnArgs& a, int batch, cudaStream_t st) {
 cudaError_t launch_attention_cluster(const Request* rq, int* status, const float* qkv, const float2* rope,
                                      const __nv_bfloat16* qr, const __nv_bfloat16* kr, const __nv_bfloat16* vr, int layer,
                                      __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
-                                     cudaStream_t st, const AttnOproj* op) {
+                                     cudaStream_t st, const AttnOproj* op, unsigned long long* trace) {
   AttnArgs a{};
+  a.trace = trace;
   a.rq = rq, a.status = status, a.qkv = qkv, a.rope = rope, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
   a.qr = qr, a.kr = kr, a.vr = vr;   // when set: rotated bf16 operands instead of the fp32 QKV output
   a.num_splits = 8, a.d = d, a.wait_limit = wait_limit;
@@ -184,7 +185,8 @@ phyai_status_t attention_op(const phyai_attention_desc_t* desc, uint32_t batch, 
     return bad("prefix_kv must be 16-byte aligned and out 4-byte aligned");
   if (!desc->n_q_heads || !desc->n_kv_heads || desc->n_q_heads % desc->n_kv_heads || desc->layer >= desc->n_layers)
     return bad("head counts or layer index out of range");
-  if (kv_tokens > (uint64_t)INT32_MAX || batch > (1u << 16)) return bad("kv_tokens or batch too large");
+  if (kv_tokens > (uint64_t)INT32_MAX || batch > 65535u) return bad("kv_tokens exceeds the int32 range or batch exceeds 65535");
+  if (!desc->suffix_len) return bad("suffix_len is 0");
   Dims d{};
   d.L = (int)desc->n_layers, d.Hq = (int)desc->n_q_heads, d.Hkv = (int)desc->n_kv_heads, d.dh = (int)desc->head_dim;
   d.S = (int)desc->suffix_len, d.H = d.S, d.Nq = d.Hq * d.dh, d.Nqkv = (d.Hq + 2 * d.Hkv) * d.dh;
@@ -205,6 +207,9 @@ phyai_status_t attention_op(const phyai_attention_desc_t* desc, uint32_t batch, 
   r.prefix_kv = prefix_kv, r.kv_tokens = kv_tokens, r.cu_lens = cu, r.batch = (int)batch;
   Request* rq = reinterpret_cast<Request*>(scratch);
   launch_set_request(rq, r, nullptr, st);
+  // cu_prefix_lens is checked on the device like in the denoise calls: a violation raises the caller's status word
+  // (INVALID_ARG) and turns the attention kernels into no-ops
+  launch_validate(rq, status_word, (int)kv_tokens, nullptr, st);
   float* partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(scratch) + 256);
   cudaError_t e = launch_attention_mma(rq, status_word, qkv, reinterpret_cast<const float2*>(rope), (int)desc->layer,
                                        reinterpret_cast<__nv_bfloat16*>(out), 0, splits, splits > 1 ? partials : nullptr,

@@ -62,6 +62,8 @@ struct AttnArgs {
   float* slab;               // [Hq][rows][D]
   size_t slab_stride;        // rows * D
   int D;
+  unsigned long long* trace; // cluster kernel: 8-entry slot or null: start, set-up done, Q acquired, tiles done, partials
+                             // received, output written, cluster released
 };
 // shared-memory barriers and tensor-memory base of the fused output projection
 struct OprojCtx {
@@ -234,6 +236,7 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
     if (CLUSTER && t == t_begin) {
       if (!acquire_q()) return;
       acquired = true;
+      if (tid == 0 && split == 0 && hgrp == 0 && b == 0) trace_stamp(a.trace, 2);
 #pragma unroll
       for (int n = 0; n < DH / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
       m0 = m1 = -INFINITY, l0 = l1 = 0.f;
@@ -383,6 +386,7 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
     }
   }
   cp_async_wait<0>();
+  if (CLUSTER && tid == 0 && split == 0 && hgrp == 0 && b == 0) trace_stamp(a.trace, 3);
   if constexpr (CLUSTER) {
     if (!acquired) {   // no key tile for this CTA: it still takes part in the merge, with an empty partial
       if (!acquire_q()) return;
@@ -452,8 +456,9 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
     }
     {
       const WaitCtx wc{a.status, abort_flag, a.wait_limit};
-      mbar_wait(mrg_bar, 0u, wc);     // all eight partials of my rows have landed in `recv`
+      mbar_wait_drain(mrg_bar, 0u, wc);     // all eight partials of my rows have landed in `recv`
     }
+    if (tid == 0 && split == 0 && hgrp == 0 && b == 0) trace_stamp(a.trace, 4);
     constexpr int CPT = DH / 16;                                  // columns per thread: 16 threads cover a row
     const int rl = tid >> 4, r = split * 8 + rl, c0 = (tid & 15) * CPT;
     if (r < S) {
@@ -520,8 +525,8 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       // ---- D[128 out channels][64 tokens] = W[128][256] X^T: 16 MMAs issued by warp 0
       constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
       if (warp == 0) {
-        const bool okx = mbar_wait(oc.x_bar, 0u, wc);
-        const bool okw = mbar_wait(oc.w_bar, 0u, wc);
+        const bool okx = mbar_wait_drain(oc.x_bar, 0u, wc) > 0;
+        const bool okw = mbar_wait_drain(oc.w_bar, 0u, wc) > 0;
         tc_fence_after();
         if (__all_sync(0xffffffffu, okx && okw)) {
 #pragma unroll
@@ -540,7 +545,7 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       const int ch = warp * 32 + lane;                       // TMEM lane = out channel within the tile
       const int n = split * 128 + ch;
       const float sc = (a.o_scale ? a.o_scale[n] : 1.0f) * (a.o_gate ? a.o_gate[n] : 1.0f);
-      const bool okm = mbar_wait(oc.mma_bar, 0u, wc);
+      const bool okm = mbar_wait_drain(oc.mma_bar, 0u, wc) > 0;
       tc_fence_after();
       if (okm) {
         float* dst = a.slab + (size_t)head * a.slab_stride + (size_t)(b * S) * a.D + n;
@@ -554,9 +559,11 @@ __device__ __forceinline__ void attn_role(const AttnArgs& a, int split, int hgrp
       }
       tc_fence_before();
     }
+    if (tid == 0 && split == 0 && hgrp == 0 && b == 0) trace_stamp(a.trace, 5);
     // every CTA has received everything by now, i.e. every outgoing copy has finished reading its source: only
     // then may a CTA leave and release its shared memory
     asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (tid == 0 && split == 0 && hgrp == 0 && b == 0) trace_stamp(a.trace, 6);
   } else if (a.num_splits == 1) {
     const float i0 = 1.0f / l0, i1 = 1.0f / l1;
 #pragma unroll
@@ -606,6 +613,8 @@ __global__ void __launch_bounds__(128, 1) k_attn_cluster(const AttnArgs a) {
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   pdl_launch_dependents();            // (the dependency wait and the status check are inside the role)
+  const bool tracer = threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
+  if (tracer) trace_stamp(a.trace, 0);
   if (threadIdx.x == 0) {
     abort_flag = 0;
     mbar_init(smem_u32(&mrg_bar), 1);
@@ -627,6 +636,7 @@ __global__ void __launch_bounds__(128, 1) k_attn_cluster(const AttnArgs a) {
   }
   // every CTA's barriers exist before any peer can send to them (this runs before the dependency wait)
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (tracer) trace_stamp(a.trace, 1);
   if (OPROJ) {
     __syncthreads();
     tc_fence_after();

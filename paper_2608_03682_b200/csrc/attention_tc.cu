@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((128u >> 4) << 24);
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full[NKV], v_full[NKV], p_full[2], pv_done[2], s_full[2], q_full;
+  __shared__ __align__(8) uint64_t k_full[NKV], v_full[NKV], p_full[2], pv_done[2], s_full[2], q_full, fin_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, skip_flag;
 
@@ -116,6 +116,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       mbar_init(smem_u32(&v_full[i]), 1);
     }
     mbar_init(smem_u32(&q_full), 1);
+    mbar_init(smem_u32(&fin_bar), 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&p_full[i]), 1);
       mbar_init(smem_u32(&pv_done[i]), 1);
@@ -243,6 +244,13 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       if (elect_one()) umma_commit(smem_u32(&pv_done[buf]));
       __syncwarp();
       if (t + 2 < T) issue_s(t + 2);
+    }
+    if (*reinterpret_cast<volatile int*>(&abort_flag)) {
+      // a wait was given up: the softmax warps no longer wait for the tensor core, so make sure here that every MMA
+      // issued above has completed before tensor memory is released below
+      if (elect_one()) umma_commit(smem_u32(&fin_bar));
+      __syncwarp();
+      for (uint32_t it = 0; it < DRAIN_LIMIT && !mbar_test(smem_u32(&fin_bar), 0u); ++it) __nanosleep(64);
     }
   } else {
     // =========================== softmax / correction / output =====================================
@@ -375,12 +383,12 @@ bool attention_tc_supported(const Dims& d) {
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
                                 int batch, const int* order, unsigned wait_limit, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce once;
+  if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(k_attn_tc<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)attn_tc_smem<256>());
     if (e != cudaSuccess) return e;
-    configured = true;
+    once.done();
   }
   AttnArgs a{};
   a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;

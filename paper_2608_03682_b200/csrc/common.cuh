@@ -33,6 +33,19 @@ __device__ __forceinline__ void pdl_enter() {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Tracing aid (the paper times phases with GPU-side profiler scopes): with tracing switched on, one CTA of each
+// traced launch writes device-global-timer stamps (ns) into its 8-entry slot of a trace buffer.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void trace_stamp(unsigned long long* slot, int i) {
+  if (slot) slot[i] = global_ns();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Request block: written by a tiny kernel right before each denoise call, read by every kernel
 // of the loop.  Keeping the per-request pointers and lengths here (not in kernel arguments) lets
 // one captured CUDA graph serve every request of the same (batch, n_steps).

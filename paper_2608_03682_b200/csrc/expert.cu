@@ -10,7 +10,6 @@
 
 #include "../../include/phyai.h"
 #include "kernels.h"
-#include "mega.h"
 
 using namespace phyai;
 
@@ -39,6 +38,8 @@ struct Tables {             // per n_steps
   float* tb = nullptr;      // pi0:  [n][D]  time bias of the folded action MLP
   float* cvec = nullptr;    // pi05: [n][D]
   float* mod = nullptr;     // pi05: [n][sites][3D]  (1+scale | shift | gate)
+  float* shw_qkv = nullptr; // pi05, cluster GEMM path: [n][L][Nqkv] shift . W_qkv in packed row order
+  float* shw_gu = nullptr;  // pi05, cluster GEMM path: [n][L][2F]   shift . W_gate/up, interleaved row order
 };
 
 inline int kind_of(uint32_t dtype) { return dtype == PHYAI_F32 ? 0 : 1; }
@@ -82,26 +83,22 @@ struct phyai_expert {
   float* attn_scratch = nullptr;  // split-KV partials of the tensor-core attention
   bool attn_mma = false;
 
-  // persistent loop kernel (batch * suffix_len <= 64)
-  bool mega_ok = false;
-  int use_mega = 0;   // the captured per-operator loop measured faster (10.0 vs 12.6 ms on the pi0-shaped expert): opt-in
+  bool il_ok = false;          // gate / up also packed interleaved (single-token-tile calls)
+  bool b1_ok = false;          // the cluster split-K GEMM path covers this expert's shapes
+  int use_cluster_gemm = 1;
+  int b1_c[4] = {0, 0, 0, 0};  // cluster sizes of the QKV / O / gate-up / down projections (0 = choose)
+  float *ss_a = nullptr, *ss_b = nullptr;   // [D/128][64] partial sums of squares of h (after O / after down)
+  unsigned long long* trace_buf = nullptr;
+  unsigned long long* trace = nullptr;      // [TRACE_SLOTS][8] timer stamps of the traced launches of one call, or null
   int use_tc_attention = 1;
   int use_cluster_attention = 1;
-  int use_fused_oproj = 1;     // cluster attention also does the output projection of its head (one request, head_dim 256)
-  int use_pair_gemm = 0;   // measured slower than the single-CTA kernel on the batch-64 shapes: opt-in
+  int use_fused_oproj = 1;     // cluster attention also does the output projection of its head (general GEMM path only)
   int n_sm = 0;
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
   __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
   __nv_bfloat16 *qr_big = nullptr, *kr_big = nullptr, *vr_big = nullptr;   // rotated bf16 q / k / v of large batches
-  float* mega_scratch = nullptr;
-  float* mega_slab = nullptr;
-  unsigned* mega_counters = nullptr;
-  unsigned long long* mega_trace = nullptr;   // [148][MP_COUNT][2] when tracing is on
-  int trace_step = 0, trace_layer = 0;
-  struct MegaBatch { MegaCtaPlan* plans = nullptr; int n_cta[MP_COUNT]; int splits = 1; };
-  std::map<int, MegaBatch> mega_batches;
 
   Request* rq = nullptr;
   int* cu_internal = nullptr;
@@ -206,6 +203,20 @@ phyai_status_t build_tables(phyai_expert* h, int n, cudaStream_t st, Tables** ou
       launch_rows_gemm(t.cvec, D, reinterpret_cast<const uint8_t*>(h->wmod) + s * wsite, h->wmod_kind, 0, 3 * D, D,
                        h->bmod + (size_t)s * 3 * D, nullptr, 0, t.mod + (size_t)s * 3 * D, h->sites * 3 * D, n, st);
     launch_mod_finish(t.mod, n * h->sites, D, st);
+    if (h->b1_ok) {
+      // the shift of a folded norm enters the projection after it as a per-channel constant shift . W
+      const int L = h->d.L, Nqkv = h->d.Nqkv, F2 = 2 * h->d.F;
+      ST(h->alloc(&t.shw_qkv, (size_t)n * L * Nqkv));
+      ST(h->alloc(&t.shw_gu, (size_t)n * L * F2));
+      for (int k = 0; k < n; ++k)
+        for (int l = 0; l < L; ++l) {
+          const float* sh1 = t.mod + ((size_t)k * h->sites + 2 * l) * 3 * D + D;
+          const float* sh2 = t.mod + ((size_t)k * h->sites + 2 * l + 1) * 3 * D + D;
+          launch_shift_rows(sh1, h->p_qkv[l], h->s_qkv[l], nullptr, 0, t.shw_qkv + ((size_t)k * L + l) * Nqkv, Nqkv, D, st);
+          launch_shift_rows(sh2, h->p_gu_all + (size_t)l * D * F2, h->s_g[l], h->s_u[l], 1,
+                            t.shw_gu + ((size_t)k * L + l) * F2, F2, D, st);
+        }
+    }
   }
   CU(cudaGetLastError());
   auto ins = h->tables.emplace(n, t);
@@ -220,6 +231,7 @@ phyai_status_t build_tables(phyai_expert* h, int n, cudaStream_t st, Tables** ou
 // merge pass): from this many CTAs on it beats the split mma.sync kernel + merge.
 constexpr int ATTN_TC_MIN_CTAS = 8;
 constexpr int MAX_SLABS = 16;
+constexpr int TRACE_SLOTS = 4096;
 
 int pick_nt(int M) { return M <= 64 ? 64 : (M <= 1024 ? 128 : 256); }
 
@@ -250,56 +262,8 @@ int pick_splits(int n_tiles, int tok_tiles, int KC) {
   return s;
 }
 
-// Per-batch role plan of the persistent kernel (built outside any stream capture: it allocates).
-phyai_status_t mega_prepare(phyai_expert* h, int batch) {
-  const Dims& d = h->d;
-  const int ncta = h->n_sm < 148 ? h->n_sm : 148;
-  if (h->mega_batches.find(batch) == h->mega_batches.end()) {
-    phyai_expert::MegaBatch mb;
-    mb.splits = mega_attention_splits(d, batch, (int)h->cfg.max_prefix_len, ncta);
-    std::vector<MegaCtaPlan> plans(ncta);
-    if (!mega_plan(d, batch, h->ada ? 1 : 0, mb.splits, ncta, plans.data(), mb.n_cta))
-      return fail(PHYAI_ERR_UNSUPPORTED, "persistent kernel cannot plan this shape");
-    ST(h->alloc(&mb.plans, (size_t)ncta));
-    CU(cudaMemcpy(mb.plans, plans.data(), sizeof(MegaCtaPlan) * ncta, cudaMemcpyHostToDevice));
-    h->mega_batches.emplace(batch, mb);
-  }
-  return PHYAI_OK;
-}
-
-// Small batches: the whole loop as one persistent cooperative kernel.
-phyai_status_t enqueue_mega(phyai_expert* h, int batch, int n, const Tables& t, cudaStream_t st) {
-  const Dims& d = h->d;
-  const int ncta = h->n_sm < 148 ? h->n_sm : 148;
-  const phyai_expert::MegaBatch& mb = h->mega_batches.at(batch);
-  MegaParams p{};
-  p.d = d, p.batch = batch, p.M = batch * d.S, p.n_steps = n, p.ada = h->ada ? 1 : 0, p.sites = h->sites;
-  p.attn_splits = mb.splits, p.hpc = 2, p.dt = -1.0f / (float)n, p.wait_limit = h->wait_limit;
-  p.rq = h->rq, p.status = h->status, p.counters = h->mega_counters, p.plans = mb.plans;
-  for (int i = 0; i < MP_COUNT; ++i) p.n_cta[i] = mb.n_cta[i];
-  p.w_qkv = h->p_qkv[0], p.w_o = h->p_o[0], p.w_gu = h->p_gu_all, p.w_d = h->p_d[0], p.w_embed = h->W2p;
-  p.stride_qkv = (size_t)d.D * d.Nqkv * 2, p.stride_o = (size_t)d.Nq * d.D * 2;
-  p.stride_gu = (size_t)d.D * 2 * d.F * 2, p.stride_d = (size_t)d.F * d.D * 2;
-  p.s_qkv = h->s_qkv_all, p.s_o = h->s_o_all, p.s_g = h->s_g_all, p.s_u = h->s_u_all, p.s_d = h->s_d_all;
-  p.Wc = h->Wc, p.bcfold = h->bcfold, p.b2 = h->b2, p.state_tok = h->state_tok, p.Wout = h->Wout, p.bout = h->bout;
-  p.gains = h->gains, p.mod = t.mod, p.tb = t.tb, p.rope = h->rope;
-  p.h = h->h, p.qkv = h->qkv, p.xn64 = h->xn64, p.attn64 = h->attn64, p.m64 = h->m64, p.u64 = h->u64;
-  p.qr = h->qr64, p.kr = h->kr64, p.vr = h->vr64;
-  p.attn_scratch = h->mega_scratch;
-  p.slab = h->mega_slab, p.o_splits = (d.Nq / 64 + 7) / 8, p.d_splits = (d.F / 64 + 7) / 8;
-  p.trace = h->mega_trace, p.trace_step = h->trace_step < n ? h->trace_step : n - 1;
-  p.trace_layer = h->trace_layer < d.L ? h->trace_layer : d.L - 1;
-  launch_begin(h->rq, h->status, h->state_w, h->state_b, h->state_tok, d, batch, st);
-  CU(cudaMemsetAsync(h->mega_counters, 0, sizeof(unsigned) * MP_COUNT, st));
-  cudaError_t e = launch_mega(p, ncta, st);
-  if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "persistent kernel launch failed: %s", cudaGetErrorString(e));
-  h->counting = 2;
-  return PHYAI_OK;
-}
-
 phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, cudaStream_t st) {
   const Dims& d = h->d;
-  if (h->mega_ok && h->use_mega && mega_supported(d, batch)) return enqueue_mega(h, batch, n, t, st);
   const int M = batch * d.S, D = d.D;
   const int nt = pick_nt(M);
   const int tok_tiles = (M + nt - 1) / nt;
@@ -327,11 +291,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       if (g.splits > h->slab_splits) g.splits = h->slab_splits;
       g.slab = h->slab, pending_slabs = g.splits;
     }
-    cudaError_t e;
-    TcGemm gp = g;
-    gp.splits = 1;   // the CTA-pair kernel never splits K
-    if (h->use_pair_gemm && nt == 256 && g.M == M && tc_gemm_pair_supported(gp)) e = launch_tc_gemm_pair(h->status, gp, h->n_sm, st);
-    else e = launch_tc_gemm(h->status, g, g.nt_override ? g.nt_override : nt, st);
+    cudaError_t e = launch_tc_gemm(h->status, g, g.nt_override ? g.nt_override : nt, st);
     if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tensor GEMM launch failed: %s", cudaGetErrorString(e));
     ++cnt;
     return PHYAI_OK;
@@ -341,6 +301,24 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     g.gelu_exact = d.gelu_exact;
     launch_simt_gemm(h->status, g, st);
     ++cnt;
+  };
+
+  // A single 64-token tile: the projections run on the cluster split-K kernel with the norms folded in (five
+  // kernels per layer: QKV, attention, O, gate/up, down).
+  const bool b1_attn_tc = h->attn_mma && h->use_tc_attention && h->qr_big && attention_tc_supported(d) &&
+                          batch * (d.Hq / 2) >= ATTN_TC_MIN_CTAS;
+  const bool b1_attn_cluster = !b1_attn_tc && h->attn_mma && h->use_cluster_attention && batch * d.Hq * 8 <= 2 * h->n_sm;
+  const bool b1 = h->b1_ok && h->use_cluster_gemm && M <= 64 && (b1_attn_tc || b1_attn_cluster);
+  const int ss_n = D / 128;
+  auto b1_gemm = [&](B1Gemm g, int which) -> phyai_status_t {
+    g.M = M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact, g.inv_D = 1.0f / (float)D, g.eps = d.eps;
+    g.trace = (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * 8 : nullptr;
+    int C = b1_pick_cluster(g.N / 128, g.K / 64, h->n_sm);
+    if (h->b1_c[which] > 0 && b1_gemm_supported(g.N, g.K, h->b1_c[which], h->n_sm, which == 0)) C = h->b1_c[which];
+    cudaError_t e = launch_b1_gemm(h->status, g, C, st);
+    if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "cluster GEMM launch failed: %s", cudaGetErrorString(e));
+    ++cnt;
+    return PHYAI_OK;
   };
 
   launch_begin(h->rq, h->status, h->state_w, h->state_b, h->state_tok, d, batch, st);
@@ -375,6 +353,59 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     for (int l = 0; l < d.L; ++l) {
       const float *gain, *shift, *gate;
       site(k, 2 * l, &gain, &shift, &gate);
+      if (b1) {
+        // ---- QKV: layer 0 of a step reads a normalised tile; later layers read bf16(h * gain) and the partial sums of
+        // squares left by the previous layer's down projection
+        if (l == 0) {
+          launch_rmsnorm(h->status, h->h, gain, shift, nullptr, h->xn64, 64, M, D, d.eps, st);
+          ++cnt;
+        }
+        B1Gemm q{};
+        q.W = h->p_qkv[l], q.X = h->xn64, q.N = d.Nqkv, q.K = D, q.epi = B1_QKV, q.wscale = h->s_qkv[l];
+        if (l > 0) {
+          q.ss_part = h->ss_b, q.ss_n = ss_n;
+          q.shift_row = h->ada ? t.shw_qkv + ((size_t)k * d.L + l) * d.Nqkv : nullptr;
+        }
+        q.rq = h->rq, q.rope = h->rope, q.qr = h->qr_big, q.kr = h->kr_big, q.vr = h->vr_big;
+        q.S = d.S, q.Hq = d.Hq, q.Hkv = d.Hkv, q.dh = d.dh;
+        ST(b1_gemm(q, 0));
+        // ---- attention -> bf16 tile of the output projection
+        cudaError_t e;
+        if (b1_attn_tc)
+          e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d, batch, h->order,
+                                  h->wait_limit, st);
+        else
+          e = launch_attention_cluster(h->rq, h->status, h->qkv, h->rope, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d,
+                                       batch, h->wait_limit, st, nullptr,
+                                       (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * 8 : nullptr);
+        if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
+        ++cnt;
+        // ---- O projection + residual; leaves the operands of the second norm
+        const float *gain2, *shift2, *gate2;
+        site(k, 2 * l + 1, &gain2, &shift2, &gate2);
+        B1Gemm o{};
+        o.W = h->p_o[l], o.X = h->attn64, o.N = D, o.K = d.Nq, o.epi = B1_RESID, o.wscale = h->s_o[l];
+        o.h = h->h, o.ldh = D, o.gate = gate, o.gain_next = gain2, o.xn_out = h->xn64, o.ss_out = h->ss_a;
+        ST(b1_gemm(o, 1));
+        // ---- gate / up + GeGLU
+        B1Gemm gu{};
+        gu.W = h->p_gu_all + (size_t)l * D * 2 * d.F, gu.X = h->xn64, gu.N = 2 * d.F, gu.K = D, gu.epi = B1_GEGLU;
+        gu.wscale = h->s_g[l], gu.wscale2 = h->s_u[l], gu.ss_part = h->ss_a, gu.ss_n = ss_n;
+        gu.shift_row = h->ada ? t.shw_gu + ((size_t)k * d.L + l) * 2 * d.F : nullptr;
+        gu.out_tiled = h->m64;
+        ST(b1_gemm(gu, 2));
+        // ---- down projection + residual; leaves the operands of the next layer's first norm
+        B1Gemm dn{};
+        dn.W = h->p_d[l], dn.X = h->m64, dn.N = D, dn.K = d.F, dn.epi = B1_RESID, dn.wscale = h->s_d[l];
+        dn.h = h->h, dn.ldh = D, dn.gate = gate2;
+        if (l + 1 < d.L) {
+          const float *gain3, *shift3, *gate3;
+          site(k, 2 * l + 2, &gain3, &shift3, &gate3);
+          dn.gain_next = gain3, dn.xn_out = h->xn64, dn.ss_out = h->ss_b;
+        }
+        ST(b1_gemm(dn, 3));
+        continue;
+      }
       launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs());
       ++cnt;
       const bool attn_tc = h->attn_mma && h->use_tc_attention && h->qr_big && attention_tc_supported(d) &&
@@ -488,8 +519,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
 phyai_status_t run(phyai_expert* h, const Request& r, int n, cudaStream_t st) {
   Tables* t = nullptr;
   ST(build_tables(h, n, st, &t));
-  if (h->mega_ok && h->use_mega && mega_supported(h->d, r.batch)) ST(mega_prepare(h, r.batch));
-  launch_set_request(h->rq, r, h->cu_internal, st);
+  launch_set_request(h->rq, r, h->cu_internal, st, h->order);
   if (r.cu_lens != nullptr) launch_validate(h->rq, h->status, (int)h->cfg.max_prefix_len, h->order, st);
   const auto key = std::make_pair(r.batch, n);
   if (!h->use_graph) {
@@ -603,7 +633,6 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
 
   auto body = [&]() -> phyai_status_t {
     if (tc) CU(tc_gemm_setup());
-    if (tc) CU(tc_gemm_pair_setup());
     {
       int dev = 0;
       CU(cudaGetDevice(&dev));
@@ -690,8 +719,8 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       ST(h->alloc(&pq_all, (size_t)L * D * Nqkv)); ST(h->alloc(&po_all, (size_t)L * Nq * D));
       ST(h->alloc(&pg_all, (size_t)L * D * F)); ST(h->alloc(&pu_all, (size_t)L * D * F));
       ST(h->alloc(&pd_all, (size_t)L * F * D));
-      h->mega_ok = mega_supported(d, 1);
-      if (h->mega_ok) ST(h->alloc(&h->p_gu_all, (size_t)L * D * 2 * F));
+      h->il_ok = F % 64 == 0;
+      if (h->il_ok) ST(h->alloc(&h->p_gu_all, (size_t)L * D * 2 * F));
       if (w8) {
         ST(h->alloc(&h->s_qkv_all, (size_t)L * Nqkv)); ST(h->alloc(&h->s_o_all, (size_t)L * D));
         ST(h->alloc(&h->s_g_all, (size_t)L * F)); ST(h->alloc(&h->s_u_all, (size_t)L * F));
@@ -706,7 +735,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       if (tc) {
         __nv_bfloat16 *pq = pq_all + (size_t)l * D * Nqkv, *po = po_all + (size_t)l * Nq * D;
         __nv_bfloat16 *pg = pg_all + (size_t)l * D * F, *pu = pu_all + (size_t)l * D * F, *pd = pd_all + (size_t)l * F * D;
-        if (h->mega_ok) {
+        if (h->il_ok) {
           __nv_bfloat16* pgu = h->p_gu_all + (size_t)l * D * 2 * F;
           launch_pack_tiled(w->wgate[l], big_kind, pgu, D, F, 0, st, 64, 0);
           launch_pack_tiled(w->wup[l], big_kind, pgu, D, F, 0, st, 64, 1);
@@ -771,28 +800,18 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         }
         if (need) ST(h->alloc(&h->attn_scratch, need, true));
       }
-      if (h->mega_ok) {
-        CU(cudaDeviceGetAttribute(&h->n_sm, cudaDevAttrMultiProcessorCount, 0));
-        int dev = 0;
-        CU(cudaGetDevice(&dev));
-        CU(cudaDeviceGetAttribute(&h->n_sm, cudaDevAttrMultiProcessorCount, dev));
-        int coop = 0;
-        CU(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
-        if (!coop || h->n_sm < 8) h->mega_ok = false;
-      }
-      if (h->mega_ok) {
-        CU(mega_setup(d.dh));
+      // cluster split-K path (one 64-token tile): compact 64-row activation tiles and the norm partials
+      auto fits = [&](int N, int K, bool qkv) {
+        return b1_gemm_supported(N, K, b1_pick_cluster(N / 128, K / 64, h->n_sm), h->n_sm, qkv);
+      };
+      h->b1_ok = h->il_ok && h->qr_big && D % 128 == 0 && F % 64 == 0 && d.S <= 64 && fits(Nqkv, D, true) &&
+                 fits(D, Nq, false) && fits(2 * F, D, false) && fits(D, F, false);
+      if (h->b1_ok) {
         ST(h->alloc(&h->xn64, (size_t)64 * D, true));
         ST(h->alloc(&h->attn64, (size_t)64 * Nq, true));
         ST(h->alloc(&h->m64, (size_t)64 * F, true));
-        ST(h->alloc(&h->u64, (size_t)64 * D, true));
-        ST(h->alloc(&h->qr64, (size_t)64 * Nq, true));
-        ST(h->alloc(&h->kr64, (size_t)64 * Nkv, true));
-        ST(h->alloc(&h->vr64, (size_t)64 * Nkv, true));
-        ST(h->alloc(&h->mega_scratch, mega_scratch_floats(d, 64 / d.S > 0 ? 64 / d.S : 1, 16), true));
-        ST(h->alloc(&h->mega_counters, (size_t)MP_COUNT, true));
-        const int so = (d.Nq / 64 + 7) / 8, sd = (d.F / 64 + 7) / 8;
-        ST(h->alloc(&h->mega_slab, (size_t)(so > sd ? so : sd) * 64 * D, true));
+        ST(h->alloc(&h->ss_a, (size_t)(D / 128) * 64, true));
+        ST(h->alloc(&h->ss_b, (size_t)(D / 128) * 64, true));
       }
       ST(h->alloc(&h->xn_t, Mp * D, true));
       ST(h->alloc(&h->attn_t, Mp * Nq, true));
@@ -935,19 +954,6 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     h->use_graph = value != 0;
     return PHYAI_OK;
   }
-  if (!strcmp(key, "trace")) {   // value = step * 1000 + layer to trace; negative = off
-    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
-    h->graphs.clear();
-    if (value < 0) {
-      h->mega_trace = nullptr;
-      return PHYAI_OK;
-    }
-    if (!h->mega_ok) return fail(PHYAI_ERR_UNSUPPORTED, "tracing needs the persistent kernel");
-    unsigned long long* buf = nullptr;
-    ST(h->alloc(&buf, (size_t)148 * MP_COUNT * 4, true));
-    h->mega_trace = buf, h->trace_step = (int)(value / 1000), h->trace_layer = (int)(value % 1000);
-    return PHYAI_OK;
-  }
   if (!strcmp(key, "use_tc_attention")) {
     h->use_tc_attention = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
@@ -973,16 +979,27 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     h->graphs.clear();
     return PHYAI_OK;
   }
-  if (!strcmp(key, "use_pair_gemm")) {
-    h->use_pair_gemm = value != 0;
+  if (!strcmp(key, "use_cluster_gemm") || !strcmp(key, "b1_c_qkv") || !strcmp(key, "b1_c_o") || !strcmp(key, "b1_c_gu") ||
+      !strcmp(key, "b1_c_d")) {
+    if (!strcmp(key, "use_cluster_gemm")) {
+      h->use_cluster_gemm = value != 0;
+    } else {
+      if (value < 0 || value > 8) return fail(PHYAI_ERR_INVALID_ARG, "cluster size out of range 0..8");
+      h->b1_c[!strcmp(key, "b1_c_qkv") ? 0 : !strcmp(key, "b1_c_o") ? 1 : !strcmp(key, "b1_c_gu") ? 2 : 3] = (int)value;
+    }
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;
   }
-  if (!strcmp(key, "use_persistent")) {
-    h->use_mega = value != 0;
+  if (!strcmp(key, "trace")) {
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
+    if (value == 0) {
+      h->trace = nullptr;      // (the buffer stays allocated until destroy)
+      return PHYAI_OK;
+    }
+    if (!h->trace_buf) ST(h->alloc(&h->trace_buf, (size_t)TRACE_SLOTS * 8, true));
+    h->trace = h->trace_buf;
     return PHYAI_OK;
   }
   if (!strcmp(key, "wait_limit")) {
@@ -995,14 +1012,13 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   return fail(PHYAI_ERR_INVALID_ARG, "unknown option '%s'", key);
 }
 
-phyai_status_t phyai_read_trace(phyai_expert_t* h, uint64_t* out, size_t capacity, uint32_t* n_ctas,
-                                uint32_t* n_phases) {
-  if (!h || !out || !n_ctas || !n_phases) return fail(PHYAI_ERR_INVALID_ARG, "NULL argument");
-  if (!h->mega_trace) return fail(PHYAI_ERR_INVALID_ARG, "tracing is off (phyai_set_option(h, \"trace\", ...))");
-  const size_t n = (size_t)148 * MP_COUNT * 4;
+phyai_status_t phyai_read_trace(phyai_expert_t* h, uint64_t* out, size_t capacity, uint32_t* n_slots, uint32_t* n_stamps) {
+  if (!h || !out || !n_slots || !n_stamps) return fail(PHYAI_ERR_INVALID_ARG, "NULL argument");
+  if (!h->trace) return fail(PHYAI_ERR_INVALID_ARG, "tracing is off (phyai_set_option(h, \"trace\", 1))");
+  const size_t n = (size_t)TRACE_SLOTS * 8;
   if (capacity < n) return fail(PHYAI_ERR_INVALID_ARG, "capacity %zu < %zu entries", capacity, n);
-  CU(cudaMemcpy(out, h->mega_trace, n * sizeof(uint64_t), cudaMemcpyDeviceToHost));
-  *n_ctas = 148, *n_phases = MP_COUNT;
+  CU(cudaMemcpy(out, h->trace, n * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+  *n_slots = TRACE_SLOTS, *n_stamps = 8;
   return PHYAI_OK;
 }
 

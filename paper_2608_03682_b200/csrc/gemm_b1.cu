@@ -1,0 +1,429 @@
+// Cluster split-K GEMM for calls with a single 64-token tile (one request, or a few short ones).
+//
+// At this size every projection of a layer is a latency chain, not a throughput problem: 51 tokens against a
+// 1024 x 2560 ... 4096 x 1024 weight matrix.  What costs time is (1) the number of dependent kernels per layer and
+// (2) inside a kernel, the length of the k-loop of one CTA (each 64-wide k-step needs 8 KB of activations through
+// the SM's L2 port and four N = 64 MMAs issued by one thread, ~0.18 us) and the epilogue of a whole 128 x 64 tile by
+// one CTA.  So the work is cut the other way round:
+//
+//   * grid = (C k-ranges, N / 128 channel tiles); the C CTAs of a channel tile form a thread-block cluster.  A CTA
+//     multiplies its 128 channels by its K / C slice: its weights (contiguous in the packed layout) are requested
+//     before the programmatic dependency wait, its activations (contiguous in the 64-row tiled layout) right after,
+//     all stages resident, no ring.
+//   * the partial accumulators are reduced over distributed shared memory: every CTA stages its [token][128] fp32
+//     partial in its own shared memory and pushes, with one bulk copy per peer, the token rows that peer owns;
+//     owner c then holds C partials of its ~M / C tokens, adds them in rank order (bit-reproducible) and runs the
+//     epilogue for those tokens only.  The epilogue is thereby spread over the cluster as well.
+//   * the RMSNorm between two projections is folded into them: a residual projection's epilogue writes
+//     h (fp32), bf16(h * gain_next) as the next projection's activation tile, and per (channel tile, token) the
+//     partial sum of squares; the next projection multiplies its accumulator columns by
+//     rsqrt(sum of the partials / D + eps) (the contraction is linear in that per-token factor) and adds, for
+//     adaptive norms, the row shift . W from a per-step table.  No norm kernel, no slab-sum kernel.
+//
+// Epilogues: rotary QKV (rotated, scaled bf16 q / k / v in the attention layout), interleaved GeGLU (64 gate + 64
+// up channels per tile), gated residual with the next norm's operands.  Waits: see mbar_wait_drain -- a given-up
+// wait suppresses the global stores but never the copy / reduce protocol, so peers are not left waiting and
+// nothing is in flight at exit.
+#include "kernels.h"
+#include "ptx.cuh"
+#include "tc.cuh"
+
+namespace phyai {
+namespace {
+
+constexpr int W_BYTES = 128 * 128;     // one weight block: 128 out channels x 64 k (bf16)
+constexpr int X_BYTES = 64 * 128;      // one activation block: 64 tokens x 64 k
+constexpr int STAGE = W_BYTES + X_BYTES;
+constexpr int MAXK = 8;                // k-steps per CTA, all resident (8 x 24 KB + the 32 KB receive area fit one SM)
+constexpr int ROWB = 128 * 4;          // one token row of a partial: 128 channels fp32
+constexpr size_t B1_SMEM_MAX = 227 * 1024 - 2048;   // dynamic shared memory limit: the opt-in maximum less the static part
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ float4 lds4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[MAXK];
+  __shared__ __align__(8) uint64_t bar_accum, bar_recv;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag, suppress, acc_ok, recv_ok;
+  __shared__ float rstd_tab[64], sc_tab[128], sh_tab[128];
+  __shared__ int2 tok_tab[64];     // QKV: (rotary position, request * 64 + suffix row) of every token
+
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int C = (int)gridDim.x, rank = (int)cluster_rank(), tile = blockIdx.y;
+  const int KC = g.K >> 6;
+  const int kc_begin = (KC * rank) / C, nk = (KC * (rank + 1)) / C - kc_begin;
+  const int M = g.M;
+  const int tok_lo = (M * rank) / C, ntok = (M * (rank + 1)) / C - tok_lo;   // token rows this CTA reduces and finishes
+  const int tpc_max = (64 + C - 1) / C;
+  const uint32_t slot = (uint32_t)tpc_max * ROWB;
+
+  pdl_launch_dependents();
+  unsigned long long* tr = (g.trace && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) ? g.trace : nullptr;
+  trace_stamp(tr, 0);
+  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t region = (uint32_t)max(g.nk_max * STAGE, 64 * ROWB);
+  const uint32_t stage = tiles;                        // [64 tokens][128] fp32 partial, over the consumed operand stages
+  const uint32_t recv = tiles + region;                // [C sources][tpc_max][128] fp32
+  const uint32_t rope_s = recv + (uint32_t)C * slot;   // QKV: [tpc_max tokens][64] (cos, sin) of this tile's channel pairs
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < MAXK; ++s) mbar_init(smem_u32(&bar_full[s]), 2);
+    mbar_init(smem_u32(&bar_accum), 1);
+    mbar_init(smem_u32(&bar_recv), 1);
+    if (C > 1 && ntok > 0) mbar_expect_tx(smem_u32(&bar_recv), (uint32_t)(C - 1) * (uint32_t)ntok * ROWB);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_slot), 64);
+    tc_fence_before();
+  }
+  // every CTA's barriers exist before a peer can send to them (this is before the dependency wait)
+  cluster_sync_all();
+  trace_stamp(tr, 1);
+  tc_fence_after();
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *reinterpret_cast<volatile uint32_t*>(&tmem_slot), 0);
+  const WaitCtx wc{status, &abort_flag, g.wait_limit};
+
+  // ---- before the dependency wait: weights (constants) and per-channel constants ------------------------------
+  if (lane == 0) {
+    for (int s = warp; s < nk; s += 8) {
+      const uint32_t full = smem_u32(&bar_full[s]);
+      mbar_expect_tx(full, W_BYTES);
+      bulk_g2s(tiles + (uint32_t)s * STAGE, reinterpret_cast<const uint8_t*>(g.W) + ((size_t)tile * KC + kc_begin + s) * W_BYTES,
+               W_BYTES, full);
+    }
+  }
+  if (tid < 128) {
+    const int n = tile * 128 + tid;
+    float sc = 1.0f;
+    if (EPI == B1_GEGLU) {
+      const float* sp = tid >= 64 ? g.wscale2 : g.wscale;
+      if (sp) sc = sp[tile * 64 + (tid & 63)];
+    } else if (g.wscale) {
+      sc = g.wscale[n];
+    }
+    sc_tab[tid] = sc;
+    sh_tab[tid] = g.shift_row ? g.shift_row[n] : 0.0f;
+  }
+  float4 gate4 = make_float4(1.f, 1.f, 1.f, 1.f), gain4 = gate4;
+  if (EPI == B1_RESID) {
+    const int n = tile * 128 + lane * 4;
+    if (g.gate) gate4 = __ldg(reinterpret_cast<const float4*>(g.gate + n));
+    if (g.gain_next) gain4 = __ldg(reinterpret_cast<const float4*>(g.gain_next + n));
+  }
+  pdl_wait();
+  trace_stamp(tr, 2);
+  // ---- after it: activations, the status word, per-token factors --------------------------------------------------
+  if (lane == 0) {
+    for (int s = (warp + 4) & 7; s < nk; s += 8) {
+      const uint32_t full = smem_u32(&bar_full[s]);
+      mbar_expect_tx(full, X_BYTES);
+      bulk_g2s(tiles + (uint32_t)s * STAGE + W_BYTES, reinterpret_cast<const uint8_t*>(g.X) + (size_t)(kc_begin + s) * X_BYTES,
+               X_BYTES, full);
+    }
+  }
+  if (tid == 255) suppress = status_set(status) ? 1 : 0;
+  if (tid < 64) {
+    float r = 1.0f;
+    if (g.ss_part && tid < M) {
+      float ss = 0.f;
+      for (int i = 0; i < g.ss_n; ++i) ss += g.ss_part[i * 64 + tid];
+      r = 1.0f / sqrtf(ss * g.inv_D + g.eps);
+    }
+    rstd_tab[tid] = r;
+    if (EPI == B1_QKV) {
+      int2 e = make_int2(0, 0);
+      if (tid < M) {
+        const int b = tid / g.S, i = tid - b * g.S;
+        const int* cu = g.rq->cu_lens;
+        e = make_int2(cu[b + 1] - cu[b] + i, b * 64 + i);
+      }
+      tok_tab[tid] = e;
+    }
+  }
+  float4 hpre[2];
+  if (EPI == B1_RESID) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int tl = warp + 8 * u;
+      hpre[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (tl < ntok) hpre[u] = *reinterpret_cast<const float4*>(g.h + (size_t)(tok_lo + tl) * g.ldh + tile * 128 + lane * 4);
+    }
+  }
+  __syncthreads();
+  const int n0 = tile * 128;
+  const int Nq = g.Hq * g.dh, Nk = g.Hkv * g.dh;
+  const bool rot_tile = EPI == B1_QKV && n0 < Nq + Nk;
+  if (EPI == B1_QKV && rot_tile && g.rope) {
+    // the rotary rows of this CTA's tokens for the 64 channel pairs of this tile, while the MMAs run
+    const int nn = n0 < Nq ? n0 : n0 - Nq;
+    const int t64 = (nn % g.dh) >> 7;
+    for (int idx = tid; idx < ntok * 32; idx += 256) {
+      const int tl = idx >> 5, c = idx & 31;
+      const int pos = tok_tab[tok_lo + tl].x;
+      const float4 v = __ldg(reinterpret_cast<const float4*>(g.rope + (size_t)pos * (g.dh >> 1) + t64 * 64) + c);
+      asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(rope_s + (uint32_t)(tl * 32 + c) * 16), "f"(v.x), "f"(v.y),
+                   "f"(v.z), "f"(v.w)
+                   : "memory");
+    }
+  }
+
+  // ---- MMAs: one warp, whole warp in the loop, one elected lane issues -----------------------------------------
+  if (warp == 1) {
+    bool all_ok = true;
+    for (int s = 0; s < nk; ++s) {
+      const bool ok = mbar_wait_drain(smem_u32(&bar_full[s]), 0u, wc) > 0;
+      all_ok = all_ok && ok;
+      const uint32_t a0 = tiles + (uint32_t)s * STAGE;
+      const uint64_t da = make_desc(a0), db = make_desc(a0 + W_BYTES);
+      if (__all_sync(0xffffffffu, ok)) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (elect_one()) umma_bf16(tmem_base, da + 2 * k, db + 2 * k, IDESC, (s > 0 || k > 0) ? 1u : 0u);
+      }
+      __syncwarp();
+    }
+    if (elect_one()) umma_commit(smem_u32(&bar_accum));
+    __syncwarp();
+    const bool okc = mbar_wait_drain(smem_u32(&bar_accum), 0u, wc) > 0;
+    if (lane == 0) acc_ok = (all_ok && okc && nk > 0) ? 1 : 0;
+  }
+  __syncthreads();
+  tc_fence_after();
+  trace_stamp(tr, 3);
+
+  // ---- accumulator -> staging [token][channel] (the operand stages are free: every MMA has completed) -------------
+  {
+    const int q = warp & 3, hf = warp >> 2;
+    if (hf * 32 < M) {
+      float v[32];
+      if (nk > 0) {
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(hf * 32), v);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = 0.f;
+      }
+      const uint32_t dst = stage + (uint32_t)(hf * 32) * ROWB + (uint32_t)(q * 32 + lane) * 4;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst + (uint32_t)j * ROWB), "f"(v[j]) : "memory");
+    }
+  }
+  tc_fence_before();
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the bulk-copy engine
+  __syncthreads();
+  // ---- reduce-scatter over the cluster: every peer gets its token rows of my partial -----------------------------
+  if (tid < C && tid != rank) {
+    const int lo = (M * tid) / C, n = (M * (tid + 1)) / C - lo;
+    if (n > 0) {
+      uint32_t dst, bar;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(recv + (uint32_t)rank * slot), "r"(tid));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(&bar_recv)), "r"(tid));
+      asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                   "r"(stage + (uint32_t)lo * ROWB), "r"((uint32_t)n * ROWB), "r"(bar)
+                   : "memory");
+    }
+  }
+  if (warp == 0) {
+    bool ok = true;
+    if (C > 1 && ntok > 0) ok = mbar_wait_drain(smem_u32(&bar_recv), 0u, wc) > 0;
+    if (lane == 0) recv_ok = ok ? 1 : 0;
+  }
+  __syncthreads();
+  trace_stamp(tr, 4);
+  const bool store = !suppress && acc_ok && recv_ok && !*reinterpret_cast<volatile int*>(&abort_flag);
+
+  // four consecutive channels of one of my tokens: the C partials added in rank order
+  auto sum4 = [&](int tl, int ch) -> float4 {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = 0; c < C; ++c) {
+      const uint32_t p = (c == rank) ? stage + (uint32_t)(tok_lo + tl) * ROWB : recv + (uint32_t)c * slot + (uint32_t)tl * ROWB;
+      const float4 v = lds4(p + (uint32_t)ch * 4);
+      a.x += v.x, a.y += v.y, a.z += v.z, a.w += v.w;
+    }
+    return a;
+  };
+  // accumulator value -> projection output: weight scale, the folded norm's per-token factor, the folded shift row
+  auto fin = [&](float a, int ch, float r) -> float { return fmaf(a * sc_tab[ch], r, sh_tab[ch]); };
+
+  if (store) {
+    if (EPI == B1_QKV) {
+      if (rot_tile) {
+        const bool isq = n0 < Nq;
+        const int nn = isq ? n0 : n0 - Nq;
+        const int head = nn / g.dh, t64 = (nn - head * g.dh) >> 7, half = g.dh >> 1;
+        __nv_bfloat16* base = isq ? g.qr : g.kr;
+        const int H = isq ? g.Hq : g.Hkv;
+        const float osc = isq ? rsqrtf((float)g.dh) : 1.0f;
+        for (int it = tid; it < ntok * 8; it += 256) {
+          const int tl = it >> 3, j0 = (it & 7) * 8;
+          const int2 e = tok_tab[tok_lo + tl];
+          const float r = rstd_tab[tok_lo + tl];
+          float lo[8], hi[8];
+          *reinterpret_cast<float4*>(lo) = sum4(tl, j0), *reinterpret_cast<float4*>(lo + 4) = sum4(tl, j0 + 4);
+          *reinterpret_cast<float4*>(hi) = sum4(tl, 64 + j0), *reinterpret_cast<float4*>(hi + 4) = sum4(tl, 64 + j0 + 4);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) lo[u] = fin(lo[u], j0 + u, r), hi[u] = fin(hi[u], 64 + j0 + u, r);
+          if (g.rope) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const float4 c = lds4(rope_s + (uint32_t)(tl * 64 + j0 + 2 * u) * 8);   // (cos, sin) of channels 2u, 2u + 1
+              const float l0 = lo[2 * u], h0 = hi[2 * u], l1 = lo[2 * u + 1], h1 = hi[2 * u + 1];
+              lo[2 * u] = l0 * c.x - h0 * c.y, hi[2 * u] = h0 * c.x + l0 * c.y;
+              lo[2 * u + 1] = l1 * c.z - h1 * c.w, hi[2 * u + 1] = h1 * c.z + l1 * c.w;
+            }
+          }
+          const int b = e.y >> 6, i = e.y & 63;
+          __nv_bfloat16* dst = base + ((size_t)(b * H + head) * g.S + i) * g.dh + t64 * 64 + j0;
+          *reinterpret_cast<uint4*>(dst) = make_uint4(pack2(lo[0] * osc, lo[1] * osc), pack2(lo[2] * osc, lo[3] * osc),
+                                                      pack2(lo[4] * osc, lo[5] * osc), pack2(lo[6] * osc, lo[7] * osc));
+          *reinterpret_cast<uint4*>(dst + half) = make_uint4(pack2(hi[0] * osc, hi[1] * osc), pack2(hi[2] * osc, hi[3] * osc),
+                                                             pack2(hi[4] * osc, hi[5] * osc), pack2(hi[6] * osc, hi[7] * osc));
+        }
+      } else {
+        const int nn = n0 - Nq - Nk;
+        const int head = nn / g.dh, coff = nn - head * g.dh;       // 128 consecutive v channels
+        for (int it = tid; it < ntok * 16; it += 256) {
+          const int tl = it >> 4, j0 = (it & 15) * 8;
+          const int2 e = tok_tab[tok_lo + tl];
+          const float r = rstd_tab[tok_lo + tl];
+          float x[8];
+          *reinterpret_cast<float4*>(x) = sum4(tl, j0), *reinterpret_cast<float4*>(x + 4) = sum4(tl, j0 + 4);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) x[u] = fin(x[u], j0 + u, r);
+          const int b = e.y >> 6, i = e.y & 63;
+          *reinterpret_cast<uint4*>(g.vr + ((size_t)(b * g.Hkv + head) * g.S + i) * g.dh + coff + j0) =
+              make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
+        }
+      }
+    } else if (EPI == B1_GEGLU) {
+      // rows 0..63 = gate channels f0 .. f0 + 63, rows 64..127 = the matching up channels; the result is one 64-wide
+      // k-chunk (`tile`) of the down projection's activation tile, written as its swizzled 16-byte groups
+      for (int it = tid; it < ntok * 8; it += 256) {
+        const int tl = it >> 3, c8 = it & 7, j0 = c8 * 8, tok = tok_lo + tl;
+        const float r = rstd_tab[tok];
+        float gt[8], up[8];
+        *reinterpret_cast<float4*>(gt) = sum4(tl, j0), *reinterpret_cast<float4*>(gt + 4) = sum4(tl, j0 + 4);
+        *reinterpret_cast<float4*>(up) = sum4(tl, 64 + j0), *reinterpret_cast<float4*>(up + 4) = sum4(tl, 64 + j0 + 4);
+        float m[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) m[u] = gelu_fast(fin(gt[u], j0 + u, r), g.gelu_exact) * fin(up[u], 64 + j0 + u, r);
+        *reinterpret_cast<uint4*>(g.out_tiled + ((size_t)tile * 64 + tok) * 64 + ((c8 ^ (tok & 7)) << 3)) =
+            make_uint4(pack2(m[0], m[1]), pack2(m[2], m[3]), pack2(m[4], m[5]), pack2(m[6], m[7]));
+      }
+    } else {
+      // gated residual: one warp per token, a lane takes four channels.  h stays fp32; the next projection's
+      // activation tile is bf16(h * gain) (its 1 / rms factor follows in that projection's epilogue from the
+      // partial sums of squares written here)
+      auto token = [&](int tl, bool have_old, float4 old) {
+        const int tok = tok_lo + tl, n = n0 + lane * 4;
+        float* hp = g.h + (size_t)tok * g.ldh + n;
+        if (!have_old) old = *reinterpret_cast<const float4*>(hp);
+        const float4 a = sum4(tl, lane * 4);
+        float4 hv;
+        hv.x = old.x + gate4.x * (a.x * sc_tab[lane * 4]), hv.y = old.y + gate4.y * (a.y * sc_tab[lane * 4 + 1]);
+        hv.z = old.z + gate4.z * (a.z * sc_tab[lane * 4 + 2]), hv.w = old.w + gate4.w * (a.w * sc_tab[lane * 4 + 3]);
+        *reinterpret_cast<float4*>(hp) = hv;
+        if (g.xn_out) {
+          *reinterpret_cast<uint2*>(g.xn_out + tiled_index(tok, n, 64)) =
+              make_uint2(pack2(hv.x * gain4.x, hv.y * gain4.y), pack2(hv.z * gain4.z, hv.w * gain4.w));
+          const float ss = warp_sum(hv.x * hv.x + hv.y * hv.y + hv.z * hv.z + hv.w * hv.w);
+          if (lane == 0) g.ss_out[tile * 64 + tok] = ss;
+        }
+      };
+      if (warp < ntok) token(warp, true, hpre[0]);           // (the first two rows of a warp were requested early)
+      if (warp + 8 < ntok) token(warp + 8, true, hpre[1]);
+      for (int tl = warp + 16; tl < ntok; tl += 8) token(tl, false, make_float4(0.f, 0.f, 0.f, 0.f));
+    }
+  }
+  trace_stamp(tr, 5);
+  // every peer has received everything, i.e. every outgoing copy has finished reading its source, before any CTA
+  // leaves and releases its shared memory
+  cluster_sync_all();
+  trace_stamp(tr, 6);
+  if (tr) {
+    unsigned sm;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+    tr[7] = sm;
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 64);
+  }
+}
+
+size_t b1_smem(int nk_max, int C, bool rope_rows) {
+  const int tpc = (64 + C - 1) / C;
+  const size_t region = (size_t)(nk_max * STAGE > 64 * ROWB ? nk_max * STAGE : 64 * ROWB);
+  return 1024 + region + (size_t)C * tpc * ROWB + (rope_rows ? (size_t)tpc * 512 : 0);
+}
+
+template <int EPI>
+cudaError_t launch_one(int* status, const B1Gemm& g, int C, cudaStream_t st) {
+  static PerDeviceOnce once;
+  if (once.needed()) {
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_b1<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1_SMEM_MAX);
+    if (e != cudaSuccess) return e;
+    once.done();
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(C, g.N / 128, 1), cfg.blockDim = dim3(256), cfg.dynamicSmemBytes = b1_smem(g.nk_max, C, g.epi == B1_QKV), cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = C, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at, cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, k_gemm_b1<EPI>, status, g);
+}
+
+}  // namespace
+
+// Largest cluster size (k-ranges per channel tile) for a projection with `tiles` channel tiles and KC k-chunks:
+// at most 8 (portable cluster size), at most one CTA per SM in total, at most one k-chunk per CTA.
+int b1_pick_cluster(int tiles, int KC, int n_sm) {
+  int C = n_sm / tiles;
+  if (C > 8) C = 8;
+  if (C > KC) C = KC;
+  if (C < 1) C = 1;
+  return C;
+}
+// A projection fits when its k-steps per CTA stay resident (<= MAXK) and the cluster has at most one CTA per SM.
+bool b1_gemm_supported(int N, int K, int C, int n_sm, bool qkv) {
+  if (N % 128 || K % 64 || C < 1 || C > 8 || C > K / 64) return false;
+  if ((N / 128) * C > n_sm) return false;
+  const int nk = (K / 64 + C - 1) / C;
+  return nk <= MAXK && b1_smem(nk, C, qkv) <= B1_SMEM_MAX;
+}
+
+cudaError_t launch_b1_gemm(int* status, const B1Gemm& g_in, int C, cudaStream_t st) {
+  B1Gemm g = g_in;
+  const int KC = g.K / 64;
+  g.nk_max = (KC + C - 1) / C;
+  if (b1_smem(g.nk_max, C, g.epi == B1_QKV) > B1_SMEM_MAX) return cudaErrorInvalidConfiguration;
+  if (g.epi == B1_QKV) return launch_one<B1_QKV>(status, g, C, st);
+  if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU>(status, g, C, st);
+  return launch_one<B1_RESID>(status, g, C, st);
+}
+
+}  // namespace phyai

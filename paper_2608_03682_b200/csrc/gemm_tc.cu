@@ -28,8 +28,9 @@
 // and the rotary epilogue of the fused QKV projection (rotated, scaled bf16 q / k / v in the attention layout).
 // The kernel is launched with programmatic stream serialization: barriers, TMEM and the weight halves of the first
 // STAGES stages are set up before griddepcontrol.wait, i.e. while the kernel producing the activations still runs.
-// Every wait is bounded: on expiry the CTA raises the status word, stops issuing copies, and
-// drains to its normal exit (TMEM is always released).
+// Every wait is bounded: on expiry of the caller's limit the CTA raises the status word and skips its MMAs and
+// stores, but keeps the copy / commit pipeline running under a generous limit of its own, so that every copy
+// into its shared memory has landed before it exits (TMEM is always released).
 #include "kernels.h"
 #include "ptx.cuh"
 #include "tc.cuh"
@@ -163,9 +164,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   if (threadIdx.x == NPROD * 32) skip_flag = status_set(status) || nk <= 0;
   __syncthreads();
   if (skip_flag) {
-    // every copy issued so far must land before this CTA's shared memory is released
+    // every copy issued so far must land before this CTA's shared memory is released (a wait on this CTA's own
+    // copies: bounded by the drain limit, not by the caller's)
     if (threadIdx.x == 0)
-      for (int i = 0; i < n_early; ++i) mbar_wait(smem_u32(&bar_full[i]), 0u, wc);
+      for (int i = 0; i < n_early; ++i) mbar_wait_drain(smem_u32(&bar_full[i]), 0u, wc);
     __syncthreads();
     if (warp == 8) {
       tc_fence_after();
@@ -180,7 +182,9 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       const int i = id / NCOPY, c = id % NCOPY;
       const int s = i % STAGES;
       const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-      if (!mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc)) break;  // stop issuing copies once aborted
+      // (after a give-up the pipeline keeps running -- copies, commits and barriers as usual, MMAs and stores
+      // skipped -- so that nothing is in flight when the CTA exits)
+      if (mbar_wait_drain(smem_u32(&bar_empty[s]), ph ^ 1u, wc) < 0) break;
       if (c < NA) {
         const uint32_t full = smem_u32(&bar_full[s]);
         mbar_expect_tx(full, A_BYTES);
@@ -198,7 +202,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     for (int i = first; i < nk; i += step) {
       const int s = i % STAGES;
       const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-      const bool ok = mbar_wait(smem_u32(&bar_full[s]), ph, wc);
+      const bool ok = mbar_wait_drain(smem_u32(&bar_full[s]), ph, wc) > 0;
       // (no tcgen05 fence here: the operands were written by the bulk-copy engine and made visible by the mbarrier;
       // tcgen05.fence::after_thread_sync orders tensor-memory accesses, and it was measured to hold the next MMAs
       // back until the previous stage's MMAs had drained)
@@ -305,7 +309,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     // one epilogue warp polls the accumulator barrier; the other fifteen wait for it at the named barrier (in
     // hardware), so that the main loop's shared-memory port is not shared with 512 polling threads
     if (ew == 0) {
-      const bool okw = mbar_wait(smem_u32(&bar_accum), 0, wc);
+      const bool okw = mbar_wait_drain(smem_u32(&bar_accum), 0, wc) > 0;
       if (lane == 0) epi_ok = okw ? 1 : 0;
     }
     epi_sync();
@@ -585,10 +589,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   }
 
   __syncthreads();
-  if (abort_flag) {
-    // give any bulk copy still in flight time to land before shared memory is released
-    for (int i = 0; i < 64; ++i) __nanosleep(1000);
-  }
+  // (every copy has landed by now, also after a give-up: the MMA warps waited for every stage)
   if (warp == 8) {
     tc_fence_after();
     tmem_dealloc(tmem_base, ALLOC_COLS);

@@ -3,9 +3,28 @@
 
 #include "common.cuh"
 
+#include <atomic>
 #include <utility>
 
 namespace phyai {
+
+// cudaFuncSetAttribute acts on the current device, so "already configured" is remembered per device (bit d of the
+// mask = device d; devices beyond 63 are configured on every launch).  Concurrent first launches may both
+// configure, which is harmless.
+struct PerDeviceOnce {
+  std::atomic<unsigned long long> mask{0};
+  int dev = -1;
+  bool needed() {
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev > 63) {
+      dev = -1;
+      return true;
+    }
+    return !((mask.load(std::memory_order_acquire) >> dev) & 1ull);
+  }
+  void done() {
+    if (dev >= 0) mask.fetch_or(1ull << dev, std::memory_order_release);
+  }
+};
 
 // Launch with programmatic stream serialization (see pdl_enter in common.cuh): only for kernels that call
 // pdl_enter() before touching global memory.
@@ -27,7 +46,7 @@ struct Dims {
 };
 
 // ---- request block ---------------------------------------------------------------------------
-void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st);
+void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st, int* order = nullptr);
 void launch_validate(const Request* rq, int* status, int max_prefix, int* order, cudaStream_t st);
 
 // ---- one-off table / packing kernels (CUDA cores, fp64 accumulation where cheap) ---------------
@@ -126,7 +145,7 @@ bool attention_oproj_supported(const Dims& d);
 cudaError_t launch_attention_cluster(const Request* rq, int* status, const float* qkv, const float2* rope,
                                      const __nv_bfloat16* qr, const __nv_bfloat16* kr, const __nv_bfloat16* vr, int layer,
                                      __nv_bfloat16* out_tiled, int rows_pad, const Dims& d, int batch, unsigned wait_limit,
-                                     cudaStream_t st, const AttnOproj* op = nullptr);
+                                     cudaStream_t st, const AttnOproj* op = nullptr, unsigned long long* trace = nullptr);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
                                 int batch, const int* order, unsigned wait_limit, cudaStream_t st);
@@ -166,10 +185,50 @@ struct TcGemm {
 // Returns cudaSuccess or the launch error; `nt` is the token-tile width (64, 128 or 256).
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st);
 cudaError_t tc_gemm_setup();  // one-time attribute setup (dynamic shared memory opt-in)
-// Large-batch variant on CTA pairs (256-token x 256-channel tiles, persistent, overlapped epilogue).
-// Covers TC_STORE, TC_RESID and TC_GEGLU without split-K; rows_pad must be a multiple of 256.
-bool tc_gemm_pair_supported(const TcGemm& g);
-cudaError_t launch_tc_gemm_pair(int* status, const TcGemm& g, int n_sm, cudaStream_t st);
-cudaError_t tc_gemm_pair_setup();
+// ---- cluster split-K GEMM for a single 64-token tile (gemm_b1.cu) --------------------------------------------
+enum : int { B1_QKV = 0, B1_GEGLU = 1, B1_RESID = 2 };
+struct B1Gemm {
+  const __nv_bfloat16* W;    // packed blocks [N/128][K/64][128x64]
+  const __nv_bfloat16* X;    // tiled activations [K/64][64][64] (64-row tiles, back to back)
+  int N, K, M;               // packed rows, contraction length, valid tokens (<= 64)
+  int epi;
+  int nk_max;                // (set by the launcher) most k-steps of one CTA
+  const float* wscale;       // per packed row dequant scale or null (B1_GEGLU: per gate channel f)
+  const float* wscale2;      // B1_GEGLU: per up channel f
+  // norm folded into this projection: X holds bf16(h * gain); the accumulator columns are multiplied by
+  // rsqrt(sum_i ss_part[i][token] * inv_D + eps) and shift_row (per packed row: shift . W) is added.  ss_part == null:
+  // X is already normalised.
+  const float* ss_part;
+  int ss_n;
+  float inv_D, eps;
+  const float* shift_row;
+  // B1_QKV: see TcGemm (TC_QKV_ROT)
+  const Request* rq;
+  const float2* rope;
+  __nv_bfloat16 *qr, *kr, *vr;
+  int S, Hq, Hkv, dh;
+  // B1_GEGLU: W holds gate and up interleaved in groups of 64 channels; output [N/128][64][64] tiled
+  __nv_bfloat16* out_tiled;
+  int gelu_exact;
+  // B1_RESID: h[token][n] += gate[n] * scale[n] * acc; then, when xn_out is set, the operands of the norm that
+  // follows: xn_out = bf16(h * gain_next) in the tiled layout and ss_out[N/128][64] partial sums of squares
+  float* h;
+  int ldh;
+  const float* gate;
+  const float* gain_next;
+  __nv_bfloat16* xn_out;
+  float* ss_out;
+  unsigned wait_limit;
+  unsigned long long* trace;   // 8-entry slot of this launch or null: start, set-up done, dependency resolved, MMAs
+                               // complete, partials received, epilogue done, cluster released, (SM id)
+};
+int b1_pick_cluster(int tiles, int KC, int n_sm);
+bool b1_gemm_supported(int N, int K, int C, int n_sm, bool qkv);
+cudaError_t launch_b1_gemm(int* status, const B1Gemm& g, int C, cudaStream_t st);
+// out[n] = scale(n) * sum_k shift[k] * W[n][k] for the packed rows n < N of a packed matrix with K / 64 chunks.
+// interleaved = 1: the rows are gate / up channels interleaved in groups of 64 (scale per gate channel f = wscale[f],
+// per up channel wscale2[f]); otherwise scale(n) = wscale[n].  Null scales mean 1.
+void launch_shift_rows(const float* shift, const __nv_bfloat16* Wp, const float* wscale, const float* wscale2,
+                       int interleaved, float* out, int N, int K, cudaStream_t st);
 
 }  // namespace phyai

@@ -45,6 +45,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
   return false;
 }
 
+// Wait on a barrier behind which asynchronous copies into this CTA's shared memory (or tensor-core reads of it) are
+// outstanding.  The caller's limit decides when the call is given up (status word raised, side effects suppressed);
+// the shared memory, however, may only be released once those copies have landed, so the wait then continues under a
+// generous bound of its own.  Returns 1 = completed in time, 0 = given up but the barrier did complete, -1 = not even
+// within the drain bound.  Kernels keep their copy / MMA / commit protocol going after a 0, so every barrier of the
+// pipeline still completes; only global stores are skipped.
+constexpr uint32_t DRAIN_LIMIT = 1u << 22;
+__device__ __forceinline__ int mbar_wait_drain(uint32_t bar, uint32_t parity, const WaitCtx& c) {
+  if (mbar_wait(bar, parity, c)) return 1;
+  for (uint32_t it = 0; it < DRAIN_LIMIT; ++it) {
+    if (mbar_test(bar, parity)) return 0;
+    __nanosleep(64);
+  }
+  return -1;
+}
+
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)

@@ -10,18 +10,21 @@ namespace phyai {
 // =============================================================================================
 // request block
 // =============================================================================================
-__global__ void k_set_request(Request* dst, Request src, int* cu_internal) {
+__global__ void k_set_request(Request* dst, Request src, int* cu_internal, int* order) {
   if (threadIdx.x == 0) {
     if (src.cu_lens == nullptr) {  // single-request entry point: build cu = {0, prefix_len}
       cu_internal[0] = 0;
       cu_internal[1] = src.single_len;
       src.cu_lens = cu_internal;
+      // the walk order of the request-per-CTA kernels: a batched call on the same handle may have left another
+      // request index in entry 0
+      if (order) order[0] = 0;
     }
     *dst = src;
   }
 }
-void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st) {
-  k_set_request<<<1, 32, 0, st>>>(dst, src, cu_internal);
+void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st, int* order) {
+  k_set_request<<<1, 32, 0, st>>>(dst, src, cu_internal, order);
 }
 
 // cu_prefix_lens must be non-decreasing, start >= 0, end <= kv_tokens, differences <= max_prefix.
@@ -113,6 +116,38 @@ void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int
   const size_t chunks = (size_t)N * (K >> 3);
   const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
   k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off, il_group, il_second, perm_dh);
+}
+
+// Row of an adaptive norm's shift through a packed weight matrix: out[n] = scale(n) * sum_k shift[k] * W[n][k].
+// One warp per packed row; a lane reads pairs of k out of the swizzled 128 x 64 blocks.
+__global__ void k_shift_rows(const float* shift, const __nv_bfloat16* Wp, const float* wscale, const float* wscale2,
+                             int interleaved, float* out, int N, int K) {
+  const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (n >= N) return;
+  const int KC = K >> 6, tile = n >> 7, r = n & 127;
+  float acc = 0.f;
+  for (int k2 = lane * 2; k2 < K; k2 += 64) {
+    const int kc = k2 >> 6, w = k2 & 63, c = w >> 3;
+    const size_t idx = (((size_t)tile * KC + kc) * 128 + r) * 64 + (size_t)((c ^ (r & 7)) << 3) + (w & 7);
+    const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162*>(Wp + idx);
+    acc = fmaf(shift[k2], __low2float(p), acc);
+    acc = fmaf(shift[k2 + 1], __high2float(p), acc);
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) {
+    float sc = 1.0f;
+    if (interleaved) {
+      const float* sp = r >= 64 ? wscale2 : wscale;
+      if (sp) sc = sp[tile * 64 + (r & 63)];
+    } else if (wscale) {
+      sc = wscale[n];
+    }
+    out[n] = acc * sc;
+  }
+}
+void launch_shift_rows(const float* shift, const __nv_bfloat16* Wp, const float* wscale, const float* wscale2,
+                       int interleaved, float* out, int N, int K, cudaStream_t st) {
+  k_shift_rows<<<(N + 7) / 8, 256, 0, st>>>(shift, Wp, wscale, wscale2, interleaved, out, N, K);
 }
 
 // dst[n_off + packed(c)] = src[c]: per-channel scales in the packed row order of the fused QKV matrix
@@ -598,11 +633,11 @@ __global__ void __launch_bounds__(256) k_final(const Request* rq, const int* sta
 void launch_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
                   const float* Wout, const float* bout, float dt, const Dims& d, int batch, cudaStream_t st) {
   const int rows = batch * d.H;
-  static bool configured = false;
-  if (!configured) {
+  static PerDeviceOnce once;
+  if (once.needed()) {
     cudaFuncSetAttribute(k_final<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
     cudaFuncSetAttribute(k_final<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    configured = true;
+    once.done();
   }
   // few rows (one request): two rows per block so that the work spreads over more SMs
   if (rows <= 256)

@@ -61,16 +61,17 @@ def test_small_bf16_expert_matches_oracle(cond, engine):
 @pytest.mark.parametrize("head_dim,n_q,n_kv", [(64, 4, 2), (256, 2, 1)])
 def test_small_bf16_other_head_sizes_through_every_batch1_path(head_dim, n_q, n_kv):
     """head_dim 64 takes the fp32 QKV output (no rotary epilogue) into the cluster-merged attention, head_dim 256 the
-    rotated bf16 operands; each also through the split attention + merge kernels and the persistent kernel where it
-    covers the shape.  Prefix lengths: empty, shorter than one key tile, several tiles."""
+    rotated bf16 operands (and, by default, the cluster split-K projections with folded norms); each also through
+    the general GEMM kernel and through the split attention + merge kernels.  Prefix lengths: empty, shorter than
+    one key tile, several tiles."""
     cfg = small_bf16_config("pi0", head_dim=head_dim, n_q_heads=n_q, n_kv_heads=n_kv, max_prefix_len=700)
     W = synth.make_weights(cfg, 18, std=0.05)
     with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
         for P in (0, 41, 700):
             kv, state, noise = _inputs(cfg, 18, P)
             ref = O.denoise(cfg, W, kv, P, state, noise, 3)
-            for opts in ({"use_cluster_attention": 1, "use_persistent": 0}, {"use_cluster_attention": 0},
-                         {"use_persistent": 1}):
+            for opts in ({"use_cluster_attention": 1, "use_cluster_gemm": 1}, {"use_cluster_gemm": 0},
+                         {"use_cluster_attention": 0}):
                 for k, v in opts.items():
                     ex.set_option(k, v)
                 got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
@@ -80,19 +81,19 @@ def test_small_bf16_other_head_sizes_through_every_batch1_path(head_dim, n_q, n_
 # ------------------------------------------------------------------------------------------ C2 / C3
 @pytest.mark.parametrize("name", ["C2", "C3"])
 def test_pi_shaped_bf16_batch1_matches_oracle(name):
-    """Full-size batch-1 configurations through the default path (captured per-operator loop: rotary QKV epilogue,
-    cluster-merged attention with the output projection fused in, interleaved GeGLU tiles), through the same loop
-    with a separate output projection, with the split attention + merge kernels, and through the persistent
-    kernel."""
+    """Full-size batch-1 configurations through the default path (captured loop of cluster split-K projections with
+    folded norms and cluster-merged attention), through the general GEMM kernel + norm kernels (attention with the
+    output projection fused in, then with a separate output projection), and with the split attention + merge
+    kernels."""
     wl = synth.WORKLOADS[name]
     cfg = synth.pi0_config() if name == "C2" else synth.pi05_config()
     W = synth.make_weights(cfg, wl["cfg_id"])
     kv, state, noise = _inputs(cfg, wl["cfg_id"], wl["prefix"])
     ref = O.denoise(cfg, W, kv, wl["prefix"], state, noise, wl["n_steps"])
     with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
-        for label, opts in (("default", {}), ("separate output projection", {"use_fused_oproj": 0}),
-                            ("split attention", {"use_fused_oproj": 1, "use_cluster_attention": 0}),
-                            ("persistent", {"use_cluster_attention": 1, "use_persistent": 1})):
+        for label, opts in (("default", {}), ("general GEMM kernel", {"use_cluster_gemm": 0}),
+                            ("separate output projection", {"use_fused_oproj": 0}),
+                            ("split attention", {"use_fused_oproj": 1, "use_cluster_attention": 0})):
             for k, v in opts.items():
                 ex.set_option(k, v)
             got = gpu_single(cfg, W, kv, wl["prefix"], state, noise, wl["n_steps"], expert=ex)
@@ -107,7 +108,8 @@ def test_full_width_two_layer_expert_through_the_fused_attention_projection(cond
     """Width 1024, 8 heads of 256: the shapes for which the cluster attention kernel also applies the output
     projection.  Two layers keep the oracle fast; prefix lengths cover no prefix at all, key ranges without tiles,
     a ragged last tile and the maximum; suffix lengths cover owners without rows (8 rows), a full 8-row owner
-    boundary (16 / 56 rows) and the usual 51.  Each case also runs with the separate projection kernel."""
+    boundary (16 / 56 rows) and the usual 51.  Each case runs through the cluster split-K projections (default) and
+    through the general GEMM kernel with the fused and with the separate output projection."""
     cfg = synth.ExpertConfig(n_layers=2, width=1024, mlp_dim=4096, n_q_heads=8, n_kv_heads=1, head_dim=256,
                              state_dim=32, action_dim=32, horizon=horizon, has_state_token=(cond == "pi0"),
                              max_prefix_len=968, max_batch=1, cond=cond, dtype="bf16",
@@ -117,11 +119,12 @@ def test_full_width_two_layer_expert_through_the_fused_attention_projection(cond
         for P in (0, 5, 130, 816, 968):
             kv, state, noise = _inputs(cfg, 21, P)
             ref = O.denoise(cfg, W, kv, P, state, noise, 3)
-            for fused in (1, 0):
+            for cluster_gemm, fused in ((1, 0), (0, 1), (0, 0)):
+                ex.set_option("use_cluster_gemm", cluster_gemm)
                 ex.set_option("use_fused_oproj", fused)
                 got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
                 err = rel_err(got, ref)
-                assert err <= BAR["bf16"], (P, fused, err)
+                assert err <= BAR["bf16"], (P, cluster_gemm, fused, err)
 
 
 # ------------------------------------------------------------------------------------------ batched, ragged
@@ -148,7 +151,7 @@ def _batched_case(cfg, cfg_id, lens, n_steps, check, engine="auto", std=0.05):
     for b in check:
         ref = O.denoise(cfg, Wf, kvs[b], int(lens[b]), None if states is None else states[b], noise[b], n_steps)
         assert rel_err(out[b], ref) <= bar, (b, rel_err(out[b], ref))
-        # the batched call (per-operator kernels beyond 64 tokens) and the single-request call (persistent
+        # the batched call (general GEMM kernel beyond 64 tokens) and the single-request call (cluster split-K
         # kernel) round differently, so they agree with each other only to the same bar as with the oracle
         assert rel_err(out[b], singles[b]) <= bar, (b, rel_err(out[b], singles[b]))
     assert np.isfinite(out).all()
@@ -193,9 +196,10 @@ def test_bad_cu_prefix_lens_is_reported_and_nothing_is_written():
 
 # ------------------------------------------------------------------------------------------ kernel families
 @pytest.mark.parametrize("cond", ["pi0", "pi05"])
-def test_persistent_kernel_and_per_operator_kernels_agree(cond):
-    """Small batches run as one persistent kernel; the same request through the per-operator kernels
-    (option use_persistent = 0) must match the oracle too, and both must be reproducible run to run."""
+def test_cluster_gemm_path_and_general_path_agree_and_are_reproducible(cond):
+    """Calls of at most 64 suffix tokens run their projections on the cluster split-K kernel (norms folded in);
+    the same requests through the general GEMM kernel + norm kernels (option use_cluster_gemm = 0) must match the
+    oracle too, and both must give the same bits run to run (partial sums are added in a fixed order)."""
     cfg = small_bf16_config(cond, max_batch=4)
     W = synth.make_weights(cfg, 16, std=0.05)
     lens = [150, 0, 64, 33]
@@ -209,17 +213,40 @@ def test_persistent_kernel_and_per_operator_kernels_agree(cond):
         args = (packed.cuda(), torch.from_numpy(cu).cuda(), None if states is None else states.cuda(), noise.cuda(), 3)
         outs = {}
         for mode in (1, 0):
-            ex.set_option("use_persistent", mode)
+            ex.set_option("use_cluster_gemm", mode)
             a = ex.denoise_batched(*args).clone()
             b2 = ex.denoise_batched(*args).clone()
             torch.cuda.synchronize()
             assert ex.poll_status() == 0
-            if mode == 1:
-                assert torch.equal(a, b2)      # the persistent kernel sums split-K partials in a fixed order
+            assert torch.equal(a, b2)
             outs[mode] = a.double().cpu().numpy()
         for b in range(4):
             for mode in (1, 0):
                 assert rel_err(outs[mode][b], refs[b]) <= BAR["bf16"], (mode, b, rel_err(outs[mode][b], refs[b]))
+
+
+def test_single_request_after_a_ragged_batch_with_many_heads():
+    """16 query heads of 256 select the request-per-CTA tcgen05 attention kernel even for one request; it walks the
+    requests in an order that the batched call writes.  A single-request call on the same handle must reset it."""
+    cfg = small_bf16_config("pi0", head_dim=256, n_q_heads=16, n_kv_heads=2, max_batch=3, max_prefix_len=150)
+    W = synth.make_weights(cfg, 19, std=0.05)
+    lens = [20, 150, 77]
+    kvs = [synth.make_prefix_kv(cfg, 19, p, b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    states = torch.stack([synth.make_state(cfg, 19, b) for b in range(3)])
+    noise = torch.stack([synth.make_noise(cfg, 19, b) for b in range(3)])
+    Wf = O.Weights(W)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        out = ex.denoise_batched(packed.cuda(), torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), 2)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        batched = out.double().cpu().numpy()
+        single = gpu_single(cfg, W, kvs[2], lens[2], states[2], noise[2], 2, expert=ex)
+    for b in range(3):
+        ref = O.denoise(cfg, Wf, kvs[b], lens[b], states[b], noise[b], 2)
+        assert rel_err(batched[b], ref) <= BAR["bf16"], (b, rel_err(batched[b], ref))
+    ref = O.denoise(cfg, Wf, kvs[2], lens[2], states[2], noise[2], 2)
+    assert rel_err(single, ref) <= BAR["bf16"], rel_err(single, ref)
 
 
 def test_large_batch_tcgen05_attention_matches_oracle_and_the_mma_sync_kernel():
@@ -242,19 +269,10 @@ def test_large_batch_tcgen05_attention_matches_oracle_and_the_mma_sync_kernel():
         legacy = ex.denoise_batched(*args).double().cpu().numpy()
         torch.cuda.synchronize()
         assert ex.poll_status() == 0
-        # the same GEMMs on CTA pairs (cta_group::2): 1456 tokens = 5 full 256-token tiles and a ragged one
-        ex.set_option("use_tc_attention", 1)
-        ex.set_option("use_pair_gemm", 1)
-        pair = ex.denoise_batched(*args).double().cpu().numpy()
-        torch.cuda.synchronize()
-        assert ex.poll_status() == 0
     assert np.isfinite(tc).all()
     Wf = O.Weights(W)
     for b in (0, 1, 2, 3, 4, 5, 50, 103):
         ref = O.denoise(cfg, Wf, kvs[b], int(lens[b]), states[b], noise[b], 2)
         assert rel_err(tc[b], ref) <= BAR["bf16"], (b, rel_err(tc[b], ref))
         assert rel_err(legacy[b], ref) <= BAR["bf16"], (b, rel_err(legacy[b], ref))
-        assert rel_err(pair[b], ref) <= BAR["bf16"], (b, rel_err(pair[b], ref))
-    # the two GEMM kernels differ only in where split-K residual adds happen; bf16 re-rounding downstream
-    # amplifies that to a few 1e-3
-    assert rel_err(pair, tc) <= BAR["bf16"]
+
