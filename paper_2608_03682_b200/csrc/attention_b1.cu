@@ -1,0 +1,416 @@
+// Suffix -> (prefix U suffix) attention for calls with very few requests (batch 1): tcgen05 tensor cores, the key
+// range of a request split over a thread-block cluster, partial results merged over distributed shared memory.
+//
+// Work split.  Few queries, one long shared K / V stream: the limiter is how fast the prefix K / V (and Q) get into
+// the SMs, so the keys of a request are divided among the 8 CTAs of a cluster (about (P + S) / 8 <= 128 keys each:
+// ONE 128-key tile per CTA for prefixes up to ~970 tokens, hence no online-softmax loop in the common case), and two
+// query heads that share a kv head are stacked on the M axis (2 x 64 padded rows = the 128 rows of one MMA), so a
+// K / V tile is fetched once per head pair.  Grid = (8 key ranges, Hq / 2 head pairs, requests).
+//   S = Q K^T   tcgen05.mma M = 128, N = 128 keys, K = head_dim; Q in tensor memory (A operand), K tile in shared memory
+//   softmax     one thread per row straight from tensor memory (no shuffles); P (bf16) written back to tensor memory
+//   O = P V     tcgen05.mma M = 128, N = head_dim, K = 128 keys; P is the tensor-memory A operand, V an MN-major B
+//               operand (K and V tiles share one shared-memory layout and loader code)
+// The prefix rows of a CTA's tile are constants of the call and are requested before the programmatic dependency
+// wait; Q and the request's own (suffix) keys come from the QKV projection's epilogue right after it.
+//
+// Merge.  Every CTA holds an un-normalised partial (O, row max, row sum) of all 2 x S rows.  Row i of both heads is
+// owned by CTA i / 8: each CTA writes its partial, rounded to bf16 and grouped by owner, into its own shared memory
+// and sends every owner one bulk copy over distributed shared memory (counted on the owner's mbarrier); the owner
+// combines the 8 partials of its rows in rank order and stores the normalised bf16 rows as the activation tile of
+// the output projection.  No partials in global memory, no merge kernel.
+//
+// Warps: 0-1 load K, 2-3 load V (16-byte cp.async into the swizzled block layout), 4 issues the MMAs, 5-8 Q into
+// tensor memory, softmax, partial out; all nine merge.  Waits are bounded (see mbar_wait_drain); after a give-up the
+// protocol still runs to its end so that no peer is left waiting, only the global stores are skipped.
+#include "attention.cuh"
+#include "tc.cuh"
+
+namespace phyai {
+namespace {
+
+constexpr int KB = 128;            // keys per tile
+constexpr int BAR_K = 1, BAR_V = 2, BAR_SOFT = 3;
+
+template <int DH>
+struct B1Layout {
+  static constexpr int BLOCK = KB * 128;                     // one 64-channel block of a K / V tile: 128 keys x 128 bytes
+  static constexpr int TILE = (DH / 64) * BLOCK;             // a K or V tile
+  static constexpr int PITCH = DH * 2 + 16;                  // bf16 partial row, padded against bank conflicts
+  static constexpr int SLOT = 2 * 8 * (PITCH + 8);           // one owner's block: 2 heads x 8 rows of (O row | max, sum)
+  static constexpr size_t SMEM = 1024 + 2 * (size_t)TILE + 8 * (size_t)SLOT;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
+  using L = B1Layout<DH>;
+  constexpr int COLS = 512;                   // S / P at columns [0, 128), O at [128, 128 + DH), Q at [384, 384 + DH / 2)
+  constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KB >> 3) << 17) | ((128u >> 4) << 24);
+  constexpr uint32_t IDESC_PV =
+      (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((128u >> 4) << 24);
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t k_full, v_full, q_full, s_full, p_full, pv_done, mrg_bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag, suppress, mrg_ok;
+  __shared__ float wtab[16][8];               // merge: weight of partial s for each of my (up to 2 x 8) rows
+
+  const Dims& d = a.d;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rank = blockIdx.x, hp = blockIdx.y, b = blockIdx.z;
+  const int head0 = hp * 2;
+  const int hk = head0 / (d.Hq / d.Hkv);
+  const int S = d.S;
+  const bool tracer = tid == 0 && rank == 0 && hp == 0 && b == 0;
+
+  pdl_launch_dependents();
+  if (tracer) trace_stamp(a.trace, 0);
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t Ks = base, Vs = base + L::TILE;
+  const uint32_t stg = base;                              // partial, grouped by owner: over the K / V tiles once they are dead
+  const uint32_t recv = base + 2 * L::TILE;               // [8 sources][SLOT]
+  const int n_me = max(0, min(8, S - rank * 8));          // suffix rows (per head) this CTA owns in the merge
+  const uint32_t my_bytes = (uint32_t)(2 * n_me * (L::PITCH + 8));
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&k_full), 1), mbar_init(smem_u32(&v_full), 1), mbar_init(smem_u32(&q_full), 1);
+    mbar_init(smem_u32(&s_full), 1), mbar_init(smem_u32(&p_full), 1), mbar_init(smem_u32(&pv_done), 1);
+    mbar_init(smem_u32(&mrg_bar), 1);
+    if (n_me > 0) mbar_expect_tx(smem_u32(&mrg_bar), 7u * my_bytes);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {
+    tmem_alloc(smem_u32(&tmem_slot), COLS);
+    tc_fence_before();
+  }
+  // every CTA's barriers exist before a peer can send to them (this is before the dependency wait)
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  tc_fence_after();
+  if (tracer) trace_stamp(a.trace, 1);
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + KB, tmem_q = tmem_base + 384;
+  const WaitCtx wc{a.status, &abort_flag, a.wait_limit};
+
+  // (the request block is written before the captured loop starts: safe to read ahead of the dependency wait)
+  const Request r = *a.rq;
+  const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
+  const int Kt = P + S;                                   // keys of this request: prefix, then its own suffix
+  const int key_lo = (int)(((long long)Kt * rank) / 8), key_hi = (int)(((long long)Kt * (rank + 1)) / 8);
+  const int T = (key_hi - key_lo + KB - 1) / KB;          // tiles of this CTA (1 unless P + S > 1024; 0 for an empty range)
+
+  if (warp < 4) {
+    // =========================== loaders: warps 0-1 the K tile, warps 2-3 the V tile ============================
+    const bool is_v = warp >= 2;
+    const int lt2 = tid & 63;
+    constexpr int CHUNKS = DH / 8, RSTEP = 64 / CHUNKS;   // 16-byte chunks per row; rows covered by the 64 threads at once
+    const int lc = lt2 % CHUNKS, r0 = lt2 / CHUNKS;       // 16-byte chunk column; rows r0, r0 + RSTEP, ...
+    const size_t kv_stride = (size_t)d.Hkv * DH * 2;
+    const uint8_t* Gp = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
+                        (((size_t)(a.layer * 2 + (is_v ? 1 : 0)) * r.kv_tokens + p0) * d.Hkv + hk) * (DH * 2) + (size_t)lc * 16;
+    const uint8_t* Gs = reinterpret_cast<const uint8_t*>(is_v ? a.vr : a.kr) + ((size_t)(b * d.Hkv + hk) * S) * (DH * 2) +
+                        (size_t)lc * 16;
+    const uint32_t tile_base = (is_v ? Vs : Ks) + (uint32_t)(lc >> 3) * L::BLOCK;
+    // rows of tile t: prefix rows when `prefix` is set, otherwise the suffix rows and the zero fill past the range
+    auto issue = [&](int t, bool prefix) {
+      const int k0 = key_lo + t * KB;
+#pragma unroll 8
+      for (int row = r0; row < KB; row += RSTEP) {
+        const int kidx = k0 + row;
+        const bool is_p = kidx < P && kidx < key_hi;
+        if (is_p != prefix) continue;
+        const bool ok = kidx < key_hi;
+        const uint8_t* src = is_p ? Gp + (size_t)kidx * kv_stride : Gs + (size_t)(ok ? kidx - P : 0) * (DH * 2);
+        cp_async16(tile_base + (uint32_t)row * 128 + (uint32_t)(((lc & 7) ^ (row & 7)) << 4), src, ok ? 16u : 0u);
+      }
+    };
+    if (T > 0) issue(0, true);
+    cp_async_commit();
+    pdl_wait();
+    for (int t = 0; t < T; ++t) {
+      if (t > 0) {
+        // single K / V buffers: tile t may be fetched once P V of tile t - 1 has completed (rare: P + S > 1024)
+        mbar_wait_drain(smem_u32(&pv_done), (uint32_t)(t - 1) & 1u, wc);
+        issue(t, true);
+      }
+      issue(t, false);
+      cp_async_commit();
+      cp_async_wait<0>();
+      fence_async_smem();                    // generic-proxy writes, read next by the tensor core
+      if (is_v) group_sync<BAR_V, 64>(); else group_sync<BAR_K, 64>();
+      if (lt2 == 0) mbar_arrive_local(smem_u32(is_v ? &v_full : &k_full));
+    }
+    if (T == 0) cp_async_wait<0>();
+  } else if (warp == 4) {
+    // =========================== MMA issuer ======================================================================
+    pdl_wait();
+    if (lane == 0) suppress = status_set(a.status) ? 1 : 0;
+    if (T > 0) {
+      mbar_wait_drain(smem_u32(&q_full), 0u, wc);        // Q is in tensor memory
+      tc_fence_after();
+    }
+    for (int t = 0; t < T; ++t) {
+      const uint32_t ph = (uint32_t)t & 1u;
+      bool ok = mbar_wait_drain(smem_u32(&k_full), ph, wc) > 0;
+      tc_fence_after();
+      if (__all_sync(0xffffffffu, ok)) {
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint64_t db = make_desc(Ks + (uint32_t)(kk >> 2) * L::BLOCK + (uint32_t)(kk & 3) * 32);
+          if (elect_one()) umma_bf16_ts(tmem_s, tmem_q + (uint32_t)kk * 8, db, IDESC_S, kk > 0 ? 1u : 0u);
+        }
+      }
+      if (elect_one()) umma_commit(smem_u32(&s_full));
+      __syncwarp();
+      ok = mbar_wait_drain(smem_u32(&v_full), ph, wc) > 0;
+      ok = (mbar_wait_drain(smem_u32(&p_full), ph, wc) > 0) && ok;
+      tc_fence_after();
+      if (__all_sync(0xffffffffu, ok)) {
+#pragma unroll
+        for (int kj = 0; kj < KB / 16; ++kj) {
+          // A = P of this tile: bf16 pairs in the first 64 columns of the S buffer
+          const uint64_t db = make_desc_mn(Vs + (uint32_t)kj * (16 * 128), L::BLOCK, 1024);
+          if (elect_one()) umma_bf16_ts(tmem_o, tmem_s + (uint32_t)kj * 8, db, IDESC_PV, (t > 0 || kj > 0) ? 1u : 0u);
+        }
+      }
+      if (elect_one()) umma_commit(smem_u32(&pv_done));
+      __syncwarp();
+    }
+  } else {
+    // =========================== Q, softmax, partial out (one thread per row) ====================================
+    const int st = tid - 160;                 // 0..127
+    const int q = warp & 3;
+    const int row = q * 32 + lane;            // accumulator row = TMEM lane
+    const int hl = row >> 6, i = row & 63;
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    float m = -INFINITY, l = 0.f;             // running maximum (log2 units) and sum
+    pdl_wait();
+    if (T > 0) {
+      // Q (already rotated, scaled bf16) goes from global memory straight into tensor memory, one row per thread
+      const uint4* qsrc = reinterpret_cast<const uint4*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S + (i < S ? i : 0)) * DH);
+      const uint32_t qdst = tmem_q + lane_addr;
+      uint4 v[DH / 8];                                            // the whole row: every load in flight at once
+#pragma unroll
+      for (int u = 0; u < DH / 8; ++u) v[u] = i < S ? __ldg(qsrc + u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int u = 0; u < DH / 32; ++u) tmem_st16u(qdst + (uint32_t)(16 * u), reinterpret_cast<const uint32_t*>(v + 4 * u));
+      tmem_st_wait();
+      tc_fence_before();
+      group_sync<BAR_SOFT, 128>();
+      if (st == 0) mbar_arrive_local(smem_u32(&q_full));
+    }
+    const bool tr2 = st == 0 && rank == 0 && hp == 0 && b == 0;
+    if (tr2) trace_stamp(a.trace, 2);
+    const bool causal_row = d.block_causal && d.ns && i == 0;
+    for (int t = 0; t < T; ++t) {
+      const uint32_t ph = (uint32_t)t & 1u;
+      mbar_wait_drain(smem_u32(&s_full), ph, wc);
+      tc_fence_after();
+      const int k0 = key_lo + t * KB;
+      // the visible key columns of this row form a prefix of the tile: the keys that exist, and for the state-token row
+      // under the block-causal mask only up to its own key (key P)
+      int nvis = min(KB, key_hi - k0);
+      if (causal_row) nvis = min(nvis, max(0, P + 1 - k0));
+      float s[KB];
+      tmem_ld64(tmem_s + lane_addr, s);
+      tmem_ld64(tmem_s + lane_addr + 64u, s + 64);
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < KB; ++c) {
+        s[c] = c < nvis ? s[c] : -INFINITY;
+        mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * LOG2E;
+      const float m_new = fmaxf(m, mx);
+      const float corr = (m == -INFINITY) ? 1.0f : exp2f(m - m_new);
+      const float nsub = m_new == -INFINITY ? 0.f : -m_new;
+      // P = exp2(S log2e - m) as bf16 pairs over the first 64 columns of the S buffer (masked columns: exp2(-inf) = 0)
+      float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c16 = 0; c16 < KB / 32; ++c16) {
+        uint32_t w[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int c = c16 * 32 + 2 * e;
+          const float e0 = ex2_fast(fmaf(s[c], LOG2E, nsub)), e1 = ex2_fast(fmaf(s[c + 1], LOG2E, nsub));
+          rs4[e & 3] += e0 + e1;
+          w[e] = pack_bf16(e0, e1);
+        }
+        tmem_st16u(tmem_s + lane_addr + (uint32_t)(c16 * 16), w);
+      }
+      const float rs = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+      l = l * corr + rs;
+      m = m_new;
+      if (t > 0) {
+        // (rare path) the accumulator holds tiles 0..t-1 relative to the old maximum; P V of tile t - 1 has completed
+        // (the tensor pipe runs in order and S of this tile was issued after it)
+#pragma unroll 1
+        for (int c = 0; c < DH; c += 16) {
+          float o[16];
+          tmem_ld16(tmem_o + lane_addr + (uint32_t)c, o);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) o[e] *= corr;
+          tmem_st16(tmem_o + lane_addr + (uint32_t)c, o);
+        }
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      group_sync<BAR_SOFT, 128>();
+      if (st == 0) mbar_arrive_local(smem_u32(&p_full));
+      if (tr2) trace_stamp(a.trace, 7);
+    }
+    // ---- partial out: O row -> bf16 into the owner's block of the staging area, with (max, sum) --------------------
+    if (T > 0) mbar_wait_drain(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, wc);
+    tc_fence_after();
+    if (tr2) trace_stamp(a.trace, 3);
+    {
+      const int c = i >> 3, il = i & 7, n_c = max(0, min(8, S - c * 8));
+      const bool wr = i < S;
+      const uint32_t blk = stg + (uint32_t)c * L::SLOT;
+      const uint32_t rowp = blk + (uint32_t)(hl * n_c + il) * L::PITCH;
+#pragma unroll 1
+      for (int c0 = 0; c0 < DH; c0 += 64) {
+        float o[64];
+        if (T > 0) {
+          tmem_ld64(tmem_o + lane_addr + (uint32_t)c0, o);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 64; ++e) o[e] = 0.f;
+        }
+        if (wr) {
+#pragma unroll
+          for (int e = 0; e < 64; e += 8)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(rowp + (uint32_t)(c0 + e) * 2), "r"(pack_bf16(o[e], o[e + 1])),
+                         "r"(pack_bf16(o[e + 2], o[e + 3])), "r"(pack_bf16(o[e + 4], o[e + 5])), "r"(pack_bf16(o[e + 6], o[e + 7]))
+                         : "memory");
+        }
+      }
+      if (wr)
+        asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(blk + (uint32_t)(2 * n_c) * L::PITCH + (uint32_t)(hl * n_c + il) * 8),
+                     "f"(m), "f"(l)
+                     : "memory");
+    }
+    tc_fence_before();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the bulk-copy engine
+    group_sync<BAR_SOFT, 128>();
+    // ---- every owner gets its block of my partial: one bulk copy over distributed shared memory -------------------
+    if (st < 8 && st != rank) {
+      const int n_c = max(0, min(8, S - st * 8));
+      if (n_c > 0) {
+        uint32_t dst, bar;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(recv + (uint32_t)rank * L::SLOT), "r"(st));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(&mrg_bar)), "r"(st));
+        asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                     "r"(stg + (uint32_t)st * L::SLOT), "r"((uint32_t)(2 * n_c * (L::PITCH + 8))), "r"(bar)
+                     : "memory");
+      }
+    }
+    if (warp == 5) {
+      bool ok = true;
+      if (n_me > 0) ok = mbar_wait_drain(smem_u32(&mrg_bar), 0u, wc) > 0;
+      if (lane == 0) mrg_ok = ok ? 1 : 0;
+    }
+  }
+  __syncthreads();
+  // From here on this CTA no longer needs its peers (what they sent has landed); it may leave once every peer says the
+  // same, i.e. once every copy out of its own staging area has completed.  Arriving now and waiting at the very end
+  // hides the skew between the CTAs behind the merge.
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  if (tracer) trace_stamp(a.trace, 4);
+
+  // ---- merge my rows: the 8 partials in rank order, normalise, store as the output projection's activation tile ----
+  const bool store = !*reinterpret_cast<volatile int*>(&suppress) && !*reinterpret_cast<volatile int*>(&abort_flag) &&
+                     (n_me == 0 || *reinterpret_cast<volatile int*>(&mrg_ok));
+  // per row: weight of every partial, already divided by the combined sum
+  if (tid < 2 * n_me) {
+    float ms[8], ls[8], mm = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const uint32_t blk = (s == rank) ? stg + (uint32_t)rank * L::SLOT : recv + (uint32_t)s * L::SLOT;
+      asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(ms[s]), "=f"(ls[s]) : "r"(blk + (uint32_t)(2 * n_me) * L::PITCH + (uint32_t)tid * 8) : "memory");
+      mm = fmaxf(mm, ms[s]);
+    }
+    float w[8], ll = 0.f;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      w[s] = ms[s] == -INFINITY ? 0.f : exp2f(ms[s] - mm);
+      ll = fmaf(w[s], ls[s], ll);
+    }
+    const float inv = 1.0f / ll;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) wtab[tid][s] = w[s] * inv;
+  }
+  __syncthreads();
+  if (store) {
+    constexpr int CH = DH / 8;                // 16-byte chunks (8 columns) per row
+    for (int idx = tid; idx < 2 * n_me * CH; idx += 288) {
+      const int rr = idx / CH, ch = idx - rr * CH;       // rr = hl * n_me + il
+      const int hl = rr >= n_me ? 1 : 0, il = rr - hl * n_me;
+      float acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        const float w = wtab[rr][s];
+        const uint32_t blk = (s == rank) ? stg + (uint32_t)rank * L::SLOT : recv + (uint32_t)s * L::SLOT;
+        uint32_t u0, u1, u2, u3;
+        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3) : "r"(blk + (uint32_t)rr * L::PITCH + (uint32_t)ch * 16) : "memory");
+        const uint32_t uu[4] = {u0, u1, u2, u3};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162*>(&uu[e]);
+          acc[2 * e] = fmaf(w, __low2float(p), acc[2 * e]);
+          acc[2 * e + 1] = fmaf(w, __high2float(p), acc[2 * e + 1]);
+        }
+      }
+      const int orow = b * S + rank * 8 + il, col = (head0 + hl) * DH + ch * 8;
+      *reinterpret_cast<uint4*>(a.out + out_index(orow, col, a.rows_pad, d.Nq)) =
+          make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]), pack_bf16(acc[6], acc[7]));
+    }
+  }
+  if (tracer) trace_stamp(a.trace, 5);
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (tracer) trace_stamp(a.trace, 6);
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, COLS);
+  }
+  (void)base_ptr;
+}
+
+template <int DH>
+cudaError_t launch_one(const AttnArgs& a, int batch, cudaStream_t st) {
+  static PerDeviceOnce once;
+  if (once.needed()) {
+    cudaError_t e = cudaFuncSetAttribute(k_attn_b1<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1Layout<DH>::SMEM);
+    if (e != cudaSuccess) return e;
+    once.done();
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(8, a.d.Hq / 2, batch), cfg.blockDim = dim3(288), cfg.dynamicSmemBytes = B1Layout<DH>::SMEM, cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 8, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at, cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, k_attn_b1<DH>, a);
+}
+
+}  // namespace
+
+// Two query heads per CTA must share a kv head; rotated bf16 operands only.
+bool attention_b1_supported(const Dims& d) {
+  return (d.dh == 256 || d.dh == 128) && d.S <= 64 && d.Hq % 2 == 0 && (d.Hq / d.Hkv) % 2 == 0;
+}
+
+cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
+                                const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
+                                int batch, unsigned wait_limit, cudaStream_t st, unsigned long long* trace) {
+  AttnArgs a{};
+  a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
+  a.num_splits = 8, a.d = d, a.wait_limit = wait_limit, a.trace = trace;
+  return d.dh == 256 ? launch_one<256>(a, batch, st) : launch_one<128>(a, batch, st);
+}
+
+}  // namespace phyai

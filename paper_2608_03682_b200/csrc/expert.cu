@@ -86,6 +86,7 @@ struct phyai_expert {
   bool il_ok = false;          // gate / up also packed interleaved (single-token-tile calls)
   bool b1_ok = false;          // the cluster split-K GEMM path covers this expert's shapes
   int use_cluster_gemm = 1;
+  int use_b1_attention = 1;    // tcgen05 attention with the key range split over a cluster (few requests)
   int b1_c[4] = {0, 0, 0, 0};  // cluster sizes of the QKV / O / gate-up / down projections (0 = choose)
   float *ss_a = nullptr, *ss_b = nullptr;   // [D/128][64] partial sums of squares of h (after O / after down)
   unsigned long long* trace_buf = nullptr;
@@ -371,7 +372,10 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         ST(b1_gemm(q, 0));
         // ---- attention -> bf16 tile of the output projection
         cudaError_t e;
-        if (b1_attn_tc)
+        if (!b1_attn_tc && h->use_b1_attention && attention_b1_supported(d) && batch * (d.Hq / 2) * 8 <= h->n_sm)
+          e = launch_attention_b1(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d, batch, h->wait_limit,
+                                  st, (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * 8 : nullptr);
+        else if (b1_attn_tc)
           e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d, batch, h->order,
                                   h->wait_limit, st);
         else
@@ -975,6 +979,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   }
   if (!strcmp(key, "use_cluster_attention")) {
     h->use_cluster_attention = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_b1_attention")) {
+    h->use_b1_attention = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

@@ -250,6 +250,10 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     if (lane == 0) recv_ok = ok ? 1 : 0;
   }
   __syncthreads();
+  // From here on this CTA no longer needs its peers: what they sent has landed.  It may leave once every peer says the
+  // same (then every copy out of its own staging area has completed): arrive now, wait at the very end, so that the
+  // skew between the CTAs hides behind the epilogue.
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   trace_stamp(tr, 4);
   const bool store = !suppress && acc_ok && recv_ok && !*reinterpret_cast<volatile int*>(&abort_flag);
 
@@ -357,9 +361,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     }
   }
   trace_stamp(tr, 5);
-  // every peer has received everything, i.e. every outgoing copy has finished reading its source, before any CTA
-  // leaves and releases its shared memory
-  cluster_sync_all();
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   trace_stamp(tr, 6);
   if (tr) {
     unsigned sm;
