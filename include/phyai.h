@@ -212,10 +212,11 @@ phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t valu
  * Tracing aid (the paper times phases with GPU-side profiler scopes; Sec. "Results", measurement protocol).
  * With option "trace" = 1, one CTA of every cluster-GEMM and cluster-attention launch of a call writes
  * device-global-timer stamps (ns) into slot `launch index` (position of the launch within the call, from 0) of a
- * 4096 x 8 buffer: [0] kernel start, [1] set-up done, [2] dependency resolved (for attention: Q acquired),
+ * 4096 x 16 buffer: [0] kernel start, [1] set-up done, [2] dependency resolved (for attention: Q acquired),
  * [3] MMAs / key tiles complete, [4] partials of the cluster received, [5] results stored, [6] cluster released,
- * [7] (GEMM) the SM the CTA ran on, (attention) probabilities written.  After the stream is synchronised phyai_read_trace copies the buffer to `out`
- * (HOST memory, capacity >= 4096 * 8 entries); slots of launches that are not traced stay 0.  The stamps cost
+ * [7] (GEMM) the SM the CTA ran on, (attention) probabilities written; [8..15] further stamps of the attention
+ * kernel (Q copied, Q in tensor memory, logits ready, partial staged, ...).  After the stream is synchronised phyai_read_trace copies the buffer to `out`
+ * (HOST memory, capacity >= 4096 * 16 entries); slots of launches that are not traced stay 0.  The stamps cost
  * a few hundred ns each: a traced call is slower.  "trace" = 0 turns it off.
  */
 phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_slots,

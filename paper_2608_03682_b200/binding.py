@@ -248,8 +248,8 @@ class Expert:
         _check(self.lib.phyai_set_option(self._handle, key.encode(), int(value)))
 
     def read_trace(self) -> np.ndarray:
-        """Timer stamps (ns) of the traced launches of the last call: array [slots, 8] (option "trace" = 1)."""
-        buf = np.zeros(4096 * 8, dtype=np.uint64)
+        """Timer stamps (ns) of the traced launches of the last call: array [slots, 16] (option "trace" = 1)."""
+        buf = np.zeros(4096 * 16, dtype=np.uint64)
         n_slots, n_st = C.c_uint32(), C.c_uint32()
         _check(self.lib.phyai_read_trace(self._handle, buf.ctypes.data_as(_VP), buf.size, C.byref(n_slots),
                                          C.byref(n_st)))

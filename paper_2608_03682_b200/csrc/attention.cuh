@@ -62,7 +62,7 @@ struct AttnArgs {
   float* slab;               // [Hq][rows][D]
   size_t slab_stride;        // rows * D
   int D;
-  unsigned long long* trace; // cluster kernel: 8-entry slot or null: start, set-up done, Q acquired, tiles done, partials
+  unsigned long long* trace; // cluster kernel: 16-entry slot or null: start, set-up done, Q acquired, tiles done, partials
                              // received, output written, cluster released
 };
 // shared-memory barriers and tensor-memory base of the fused output projection

@@ -6,7 +6,7 @@
 // ONE 128-key tile per CTA for prefixes up to ~970 tokens, hence no online-softmax loop in the common case), and two
 // query heads that share a kv head are stacked on the M axis (2 x 64 padded rows = the 128 rows of one MMA), so a
 // K / V tile is fetched once per head pair.  Grid = (8 key ranges, Hq / 2 head pairs, requests).
-//   S = Q K^T   tcgen05.mma M = 128, N = 128 keys, K = head_dim; Q in tensor memory (A operand), K tile in shared memory
+//   S = Q K^T   tcgen05.mma M = 128, N = 128 keys, K = head_dim; Q and the K tile in shared memory
 //   softmax     one thread per row straight from tensor memory (no shuffles); P (bf16) written back to tensor memory
 //   O = P V     tcgen05.mma M = 128, N = head_dim, K = 128 keys; P is the tensor-memory A operand, V an MN-major B
 //               operand (K and V tiles share one shared-memory layout and loader code)
@@ -19,8 +19,9 @@
 // combines the 8 partials of its rows in rank order and stores the normalised bf16 rows as the activation tile of
 // the output projection.  No partials in global memory, no merge kernel.
 //
-// Warps: 0-1 load K, 2-3 load V (16-byte cp.async into the swizzled block layout), 4 issues the MMAs, 5-8 Q into
-// tensor memory, softmax, partial out; all nine merge.  Waits are bounded (see mbar_wait_drain); after a give-up the
+// Warps: 4 issues the MMAs; the other eight are two threads per accumulator row (each half of the columns): Q copies,
+// softmax, partial out; warps 0-1 also load K, 2-3 V (16-byte cp.async into the swizzled block
+// layout); all nine merge.  Waits are bounded (see mbar_wait_drain); after a give-up the
 // protocol still runs to its end so that no peer is left waiting, only the global stores are skipped.
 #include "attention.cuh"
 #include "tc.cuh"
@@ -29,7 +30,14 @@ namespace phyai {
 namespace {
 
 constexpr int KB = 128;            // keys per tile
-constexpr int BAR_K = 1, BAR_V = 2, BAR_SOFT = 3;
+// Named barriers: the eight row warps among themselves; row warps -> MMA warp "operands of the tile are in shared
+// memory" and "P is in tensor memory" (the 256 row threads arrive without waiting, the MMA warp waits: a hardware
+// wake-up instead of a polled mbarrier, which measured 0.75 us from arrival to the MMA warp's next instruction).
+constexpr int BAR_ROWS = 1, BAR_QK = 2, BAR_P = 3;
+template <int BAR, int NT>
+__device__ __forceinline__ void named_arrive() {
+  asm volatile("bar.arrive %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
 
 template <int DH>
 struct B1Layout {
@@ -43,16 +51,17 @@ struct B1Layout {
 template <int DH>
 __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   using L = B1Layout<DH>;
-  constexpr int COLS = 512;                   // S / P at columns [0, 128), O at [128, 128 + DH), Q at [384, 384 + DH / 2)
+  constexpr int COLS = 512;                   // S / P at columns [0, 128), O at [128, 128 + DH)
   constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KB >> 3) << 17) | ((128u >> 4) << 24);
   constexpr uint32_t IDESC_PV =
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((128u >> 4) << 24);
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t k_full, v_full, q_full, s_full, p_full, pv_done, mrg_bar;
+  __shared__ __align__(8) uint64_t s_full, pv_done, mrg_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, suppress, mrg_ok;
   __shared__ float wtab[16][8];               // merge: weight of partial s for each of my (up to 2 x 8) rows
+  __shared__ float xch[2][128], xsum[2][128]; // softmax: the two half-row threads exchange their maximum and sum
 
   const Dims& d = a.d;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -69,13 +78,13 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   const uint32_t Ks = base, Vs = base + L::TILE;
   const uint32_t stg = base;                              // partial, grouped by owner: over the K / V tiles once they are dead
   const uint32_t recv = base + 2 * L::TILE;               // [8 sources][SLOT]
+  const uint32_t Qs = recv;                               // Q tile (2 heads x 64 rows), until the logits exist
   const int n_me = max(0, min(8, S - rank * 8));          // suffix rows (per head) this CTA owns in the merge
   const uint32_t my_bytes = (uint32_t)(2 * n_me * (L::PITCH + 8));
 
   if (tid == 0) {
     abort_flag = 0;
-    mbar_init(smem_u32(&k_full), 1), mbar_init(smem_u32(&v_full), 1), mbar_init(smem_u32(&q_full), 1);
-    mbar_init(smem_u32(&s_full), 1), mbar_init(smem_u32(&p_full), 1), mbar_init(smem_u32(&pv_done), 1);
+    mbar_init(smem_u32(&s_full), 1), mbar_init(smem_u32(&pv_done), 1);
     mbar_init(smem_u32(&mrg_bar), 1);
     if (n_me > 0) mbar_expect_tx(smem_u32(&mrg_bar), 7u * my_bytes);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -87,9 +96,8 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   // every CTA's barriers exist before a peer can send to them (this is before the dependency wait)
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   tc_fence_after();
-  if (tracer) trace_stamp(a.trace, 1);
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + KB, tmem_q = tmem_base + 384;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + KB;
   const WaitCtx wc{a.status, &abort_flag, a.wait_limit};
 
   // (the request block is written before the captured loop starts: safe to read ahead of the dependency wait)
@@ -99,8 +107,52 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   const int key_lo = (int)(((long long)Kt * rank) / 8), key_hi = (int)(((long long)Kt * (rank + 1)) / 8);
   const int T = (key_hi - key_lo + KB - 1) / KB;          // tiles of this CTA (1 unless P + S > 1024; 0 for an empty range)
 
-  if (warp < 4) {
-    // =========================== loaders: warps 0-1 the K tile, warps 2-3 the V tile ============================
+  if (warp == 4) {
+    // =========================== MMA issuer ======================================================================
+    pdl_wait();
+    // (this warp never touches the receive area: its part in the cluster barrier that guards it, see the row warps)
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    if (lane == 0) suppress = status_set(a.status) ? 1 : 0;
+    for (int t = 0; t < T; ++t) {
+      const bool trm = lane == 0 && rank == 0 && hp == 0 && b == 0 && t == 0;
+      group_sync<BAR_QK, 288>();              // the K / V tile (and Q) are in shared memory
+      tc_fence_after();
+      if (trm) trace_stamp(a.trace, 14);
+#pragma unroll
+      for (int kk = 0; kk < DH / 16; ++kk) {
+        const uint64_t db = make_desc(Ks + (uint32_t)(kk >> 2) * L::BLOCK + (uint32_t)(kk & 3) * 32);
+        const uint64_t da = make_desc(Qs + (uint32_t)(kk >> 2) * L::BLOCK + (uint32_t)(kk & 3) * 32);
+        if (elect_one()) umma_bf16(tmem_s, da, db, IDESC_S, kk > 0 ? 1u : 0u);
+      }
+      if (elect_one()) umma_commit(smem_u32(&s_full));
+      __syncwarp();
+      if (trm) trace_stamp(a.trace, 15);
+      group_sync<BAR_P, 288>();               // P is in tensor memory
+      tc_fence_after();
+#pragma unroll
+      for (int kj = 0; kj < KB / 16; ++kj) {
+        // A = P of this tile: bf16 pairs in the first 64 columns of the S buffer
+        const uint64_t db = make_desc_mn(Vs + (uint32_t)kj * (16 * 128), L::BLOCK, 1024);
+        if (elect_one()) umma_bf16_ts(tmem_o, tmem_s + (uint32_t)kj * 8, db, IDESC_PV, (t > 0 || kj > 0) ? 1u : 0u);
+      }
+      if (elect_one()) umma_commit(smem_u32(&pv_done));
+      __syncwarp();
+    }
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  } else {
+    // =========================== the eight row warps ==============================================================
+    // Two threads per accumulator row (same TMEM lane quarter = warp % 4): group 0 (warps 5-8) takes the first half of
+    // a row's columns, group 1 (warps 0-3) the second half -- of Q on its way into tensor memory, of the logits in the
+    // softmax, of O on its way out.  Group 1 also loads the tiles: warps 0-1 K, warps 2-3 V.
+    const int g = warp < 4 ? 1 : 0;
+    const int q = warp & 3;
+    const int row = q * 32 + lane;            // accumulator row = TMEM lane
+    const int hl = row >> 6, i = row & 63;
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    const bool lead = warp == 5 && lane == 0;
+    const bool tr2 = lead && rank == 0 && hp == 0 && b == 0;
+    float m = -INFINITY, l = 0.f;             // running maximum (log2 units) and sum
+    // ---- loader state (group 1) ----
     const bool is_v = warp >= 2;
     const int lt2 = tid & 63;
     constexpr int CHUNKS = DH / 8, RSTEP = 64 / CHUNKS;   // 16-byte chunks per row; rows covered by the 64 threads at once
@@ -111,123 +163,106 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     const uint8_t* Gs = reinterpret_cast<const uint8_t*>(is_v ? a.vr : a.kr) + ((size_t)(b * d.Hkv + hk) * S) * (DH * 2) +
                         (size_t)lc * 16;
     const uint32_t tile_base = (is_v ? Vs : Ks) + (uint32_t)(lc >> 3) * L::BLOCK;
-    // rows of tile t: prefix rows when `prefix` is set, otherwise the suffix rows and the zero fill past the range
+    // rows of tile t: the prefix rows when `prefix` is set, otherwise the request's own (suffix) rows and, for V, zeros
+    // in the rows past the range (their probabilities are 0, but 0 x stale shared memory must stay 0; K rows past the
+    // range only produce logits that the softmax masks).  The loops walk exactly the rows they copy.
     auto issue = [&](int t, bool prefix) {
       const int k0 = key_lo + t * KB;
-#pragma unroll 8
-      for (int row = r0; row < KB; row += RSTEP) {
-        const int kidx = k0 + row;
-        const bool is_p = kidx < P && kidx < key_hi;
-        if (is_p != prefix) continue;
-        const bool ok = kidx < key_hi;
-        const uint8_t* src = is_p ? Gp + (size_t)kidx * kv_stride : Gs + (size_t)(ok ? kidx - P : 0) * (DH * 2);
-        cp_async16(tile_base + (uint32_t)row * 128 + (uint32_t)(((lc & 7) ^ (row & 7)) << 4), src, ok ? 16u : 0u);
+      const int np = max(0, min(KB, min(P, key_hi) - k0));   // prefix rows of the tile
+      const int nv = max(0, min(KB, key_hi - k0));           // rows that exist
+      if (prefix) {
+        const uint8_t* src = Gp + (size_t)(k0 + r0) * kv_stride;
+        for (int row2 = r0; row2 < np; row2 += RSTEP, src += (size_t)RSTEP * kv_stride)
+          cp_async16(tile_base + (uint32_t)row2 * 128 + (uint32_t)(((lc & 7) ^ (row2 & 7)) << 4), src, 16u);
+      } else {
+        for (int row2 = np + r0; row2 < nv; row2 += RSTEP)
+          cp_async16(tile_base + (uint32_t)row2 * 128 + (uint32_t)(((lc & 7) ^ (row2 & 7)) << 4),
+                     Gs + (size_t)(k0 + row2 - P) * (DH * 2), 16u);
+        if (is_v)
+          for (int row2 = nv + r0; row2 < KB; row2 += RSTEP)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(tile_base + (uint32_t)row2 * 128 + (uint32_t)(((lc & 7) ^ (row2 & 7)) << 4)),
+                         "r"(0u)
+                         : "memory");
       }
     };
-    if (T > 0) issue(0, true);
-    cp_async_commit();
+    if (g == 1 && T > 0) issue(0, true);      // constants of the call: ahead of the dependency wait
+    if (g == 1) cp_async_commit();
     pdl_wait();
-    for (int t = 0; t < T; ++t) {
-      if (t > 0) {
-        // single K / V buffers: tile t may be fetched once P V of tile t - 1 has completed (rare: P + S > 1024)
-        mbar_wait_drain(smem_u32(&pv_done), (uint32_t)(t - 1) & 1u, wc);
-        issue(t, true);
+    if (tr2) trace_stamp(a.trace, 1);
+    if (T > 0) {
+      if (g == 1) {
+        issue(0, false);
+        cp_async_commit();
       }
-      issue(t, false);
+      // Q (already rotated, scaled bf16): coalesced 16-byte copies into the swizzled K-major block layout of an MMA A
+      // operand, in the receive area of the merge (idle until the peers push).  (One thread per row straight from
+      // global memory into tensor memory measured 3.3 us -- every load instruction of a warp touches 32 lines --,
+      // and via shared memory and tcgen05.st still 2.9 us.)
+      const uint8_t* qg = reinterpret_cast<const uint8_t*>(a.qr);
+      const int rt = warp < 4 ? tid : tid - 32;                    // 0..255 over the eight row warps
+#pragma unroll 4
+      for (int idx = rt; idx < 128 * CHUNKS; idx += 256) {
+        const int rw = idx / CHUNKS, cc = idx % CHUNKS, h2 = rw >> 6, i2 = rw & 63;
+        const bool ok = i2 < S;
+        cp_async16(Qs + (uint32_t)(cc >> 3) * L::BLOCK + (uint32_t)rw * 128 + (uint32_t)(((cc & 7) ^ (rw & 7)) << 4),
+                   qg + ((size_t)(b * d.Hq + head0 + h2) * S + (ok ? i2 : 0)) * (DH * 2) + (size_t)cc * 16, ok ? 16u : 0u);
+      }
       cp_async_commit();
-      cp_async_wait<0>();
-      fence_async_smem();                    // generic-proxy writes, read next by the tensor core
-      if (is_v) group_sync<BAR_V, 64>(); else group_sync<BAR_K, 64>();
-      if (lt2 == 0) mbar_arrive_local(smem_u32(is_v ? &v_full : &k_full));
+      cp_async_wait<0>();                                          // (group 1: its tile rows as well)
+      fence_async_smem();                                          // generic-proxy writes, read next by the tensor core
+      if (tr2) trace_stamp(a.trace, 10);
+      named_arrive<BAR_QK, 288>();
     }
-    if (T == 0) cp_async_wait<0>();
-  } else if (warp == 4) {
-    // =========================== MMA issuer ======================================================================
-    pdl_wait();
-    if (lane == 0) suppress = status_set(a.status) ? 1 : 0;
-    if (T > 0) {
-      mbar_wait_drain(smem_u32(&q_full), 0u, wc);        // Q is in tensor memory
-      tc_fence_after();
-    }
-    for (int t = 0; t < T; ++t) {
-      const uint32_t ph = (uint32_t)t & 1u;
-      bool ok = mbar_wait_drain(smem_u32(&k_full), ph, wc) > 0;
-      tc_fence_after();
-      if (__all_sync(0xffffffffu, ok)) {
-#pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint64_t db = make_desc(Ks + (uint32_t)(kk >> 2) * L::BLOCK + (uint32_t)(kk & 3) * 32);
-          if (elect_one()) umma_bf16_ts(tmem_s, tmem_q + (uint32_t)kk * 8, db, IDESC_S, kk > 0 ? 1u : 0u);
-        }
-      }
-      if (elect_one()) umma_commit(smem_u32(&s_full));
-      __syncwarp();
-      ok = mbar_wait_drain(smem_u32(&v_full), ph, wc) > 0;
-      ok = (mbar_wait_drain(smem_u32(&p_full), ph, wc) > 0) && ok;
-      tc_fence_after();
-      if (__all_sync(0xffffffffu, ok)) {
-#pragma unroll
-        for (int kj = 0; kj < KB / 16; ++kj) {
-          // A = P of this tile: bf16 pairs in the first 64 columns of the S buffer
-          const uint64_t db = make_desc_mn(Vs + (uint32_t)kj * (16 * 128), L::BLOCK, 1024);
-          if (elect_one()) umma_bf16_ts(tmem_o, tmem_s + (uint32_t)kj * 8, db, IDESC_PV, (t > 0 || kj > 0) ? 1u : 0u);
-        }
-      }
-      if (elect_one()) umma_commit(smem_u32(&pv_done));
-      __syncwarp();
-    }
-  } else {
-    // =========================== Q, softmax, partial out (one thread per row) ====================================
-    const int st = tid - 160;                 // 0..127
-    const int q = warp & 3;
-    const int row = q * 32 + lane;            // accumulator row = TMEM lane
-    const int hl = row >> 6, i = row & 63;
-    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    float m = -INFINITY, l = 0.f;             // running maximum (log2 units) and sum
-    pdl_wait();
-    if (T > 0) {
-      // Q (already rotated, scaled bf16) goes from global memory straight into tensor memory, one row per thread
-      const uint4* qsrc = reinterpret_cast<const uint4*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S + (i < S ? i : 0)) * DH);
-      const uint32_t qdst = tmem_q + lane_addr;
-      uint4 v[DH / 8];                                            // the whole row: every load in flight at once
-#pragma unroll
-      for (int u = 0; u < DH / 8; ++u) v[u] = i < S ? __ldg(qsrc + u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-      for (int u = 0; u < DH / 32; ++u) tmem_st16u(qdst + (uint32_t)(16 * u), reinterpret_cast<const uint32_t*>(v + 4 * u));
-      tmem_st_wait();
-      tc_fence_before();
-      group_sync<BAR_SOFT, 128>();
-      if (st == 0) mbar_arrive_local(smem_u32(&q_full));
-    }
-    const bool tr2 = st == 0 && rank == 0 && hp == 0 && b == 0;
+
     if (tr2) trace_stamp(a.trace, 2);
     const bool causal_row = d.block_causal && d.ns && i == 0;
     for (int t = 0; t < T; ++t) {
       const uint32_t ph = (uint32_t)t & 1u;
-      mbar_wait_drain(smem_u32(&s_full), ph, wc);
+      if (t > 0) {
+        // single K / V buffers: tile t may be fetched once P V of tile t - 1 has completed (rare: P + S > 1024)
+        if (warp == 5) mbar_wait_drain(smem_u32(&pv_done), (uint32_t)(t - 1) & 1u, wc);
+        group_sync<BAR_ROWS, 256>();
+        if (g == 1) {
+          issue(t, true);
+          issue(t, false);
+          cp_async_commit();
+          cp_async_wait<0>();
+          fence_async_smem();
+        }
+        named_arrive<BAR_QK, 288>();
+      }
+      // one warp polls the barrier, the other seven wait for it at the named barrier (in hardware): 256 polling threads
+      // would share the shared-memory port with the operand reads of the MMAs they are waiting for
+      if (warp == 5) mbar_wait_drain(smem_u32(&s_full), ph, wc);
+      group_sync<BAR_ROWS, 256>();
       tc_fence_after();
+      // (the last logits exist: the Q tile is dead and the receive area free -- see the cluster barrier ahead of the push)
+      if (t == T - 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+      if (tr2) trace_stamp(a.trace, 11);
       const int k0 = key_lo + t * KB;
       // the visible key columns of this row form a prefix of the tile: the keys that exist, and for the state-token row
       // under the block-causal mask only up to its own key (key P)
       int nvis = min(KB, key_hi - k0);
       if (causal_row) nvis = min(nvis, max(0, P + 1 - k0));
-      float s[KB];
-      tmem_ld64(tmem_s + lane_addr, s);
-      tmem_ld64(tmem_s + lane_addr + 64u, s + 64);
+      nvis -= g * 64;                         // relative to this thread's 64 columns
+      float s[64];
+      tmem_ld64(tmem_s + lane_addr + (uint32_t)(g * 64), s);
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < KB; ++c) {
+      for (int c = 0; c < 64; ++c) {
         s[c] = c < nvis ? s[c] : -INFINITY;
         mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
       }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * LOG2E;
+      xch[g][row] = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      group_sync<BAR_ROWS, 256>();            // (also: both halves of every S row have been read -> P may overwrite them)
+      const float mx = fmaxf(xch[0][row], xch[1][row]) * LOG2E;
       const float m_new = fmaxf(m, mx);
       const float corr = (m == -INFINITY) ? 1.0f : exp2f(m - m_new);
       const float nsub = m_new == -INFINITY ? 0.f : -m_new;
       // P = exp2(S log2e - m) as bf16 pairs over the first 64 columns of the S buffer (masked columns: exp2(-inf) = 0)
       float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c16 = 0; c16 < KB / 32; ++c16) {
+      for (int c16 = 0; c16 < 2; ++c16) {
         uint32_t w[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
@@ -236,16 +271,14 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
           rs4[e & 3] += e0 + e1;
           w[e] = pack_bf16(e0, e1);
         }
-        tmem_st16u(tmem_s + lane_addr + (uint32_t)(c16 * 16), w);
+        tmem_st16u(tmem_s + lane_addr + (uint32_t)(g * 32 + c16 * 16), w);
       }
-      const float rs = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
-      l = l * corr + rs;
-      m = m_new;
+      xsum[g][row] = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
       if (t > 0) {
         // (rare path) the accumulator holds tiles 0..t-1 relative to the old maximum; P V of tile t - 1 has completed
-        // (the tensor pipe runs in order and S of this tile was issued after it)
+        // (the tensor pipe runs in order and S of this tile was issued after it); each thread rescales its half row
 #pragma unroll 1
-        for (int c = 0; c < DH; c += 16) {
+        for (int c = g * (DH / 2); c < (g + 1) * (DH / 2); c += 16) {
           float o[16];
           tmem_ld16(tmem_o + lane_addr + (uint32_t)c, o);
 #pragma unroll
@@ -255,12 +288,19 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
       }
       tmem_st_wait();
       tc_fence_before();
-      group_sync<BAR_SOFT, 128>();
-      if (st == 0) mbar_arrive_local(smem_u32(&p_full));
+      named_arrive<BAR_P, 288>();
+      group_sync<BAR_ROWS, 256>();            // (the other half row's sum is visible)
+      l = l * corr + (xsum[0][row] + xsum[1][row]);
+      m = m_new;
       if (tr2) trace_stamp(a.trace, 7);
     }
-    // ---- partial out: O row -> bf16 into the owner's block of the staging area, with (max, sum) --------------------
-    if (T > 0) mbar_wait_drain(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, wc);
+    if (T == 0) {
+      if (g == 1) cp_async_wait<0>();
+      asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    }
+    // ---- partial out: half an O row -> bf16 into the owner's block of the staging area; group 0 adds (max, sum) ------
+    if (T > 0 && warp == 5) mbar_wait_drain(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, wc);
+    group_sync<BAR_ROWS, 256>();
     tc_fence_after();
     if (tr2) trace_stamp(a.trace, 3);
     {
@@ -269,7 +309,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
       const uint32_t blk = stg + (uint32_t)c * L::SLOT;
       const uint32_t rowp = blk + (uint32_t)(hl * n_c + il) * L::PITCH;
 #pragma unroll 1
-      for (int c0 = 0; c0 < DH; c0 += 64) {
+      for (int c0 = g * (DH / 2); c0 < (g + 1) * (DH / 2); c0 += 64) {
         float o[64];
         if (T > 0) {
           tmem_ld64(tmem_o + lane_addr + (uint32_t)c0, o);
@@ -285,23 +325,28 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
                          : "memory");
         }
       }
-      if (wr)
+      if (wr && g == 0)
         asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(blk + (uint32_t)(2 * n_c) * L::PITCH + (uint32_t)(hl * n_c + il) * 8),
                      "f"(m), "f"(l)
                      : "memory");
     }
     tc_fence_before();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the bulk-copy engine
-    group_sync<BAR_SOFT, 128>();
+    if (tr2) trace_stamp(a.trace, 12);
+    group_sync<BAR_ROWS, 256>();
     // ---- every owner gets its block of my partial: one bulk copy over distributed shared memory -------------------
-    if (st < 8 && st != rank) {
-      const int n_c = max(0, min(8, S - st * 8));
+    // (first: every peer has moved its Q out of its receive area; all of them arrived long ago)
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    // (one copy per warp: the bulk copies issued by one warp complete one after the other)
+    const int peer = warp < 4 ? warp : warp - 1;
+    if (lane == 0 && peer != rank) {
+      const int n_c = max(0, min(8, S - peer * 8));
       if (n_c > 0) {
         uint32_t dst, bar;
-        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(recv + (uint32_t)rank * L::SLOT), "r"(st));
-        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(&mrg_bar)), "r"(st));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(recv + (uint32_t)rank * L::SLOT), "r"(peer));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(&mrg_bar)), "r"(peer));
         asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                     "r"(stg + (uint32_t)st * L::SLOT), "r"((uint32_t)(2 * n_c * (L::PITCH + 8))), "r"(bar)
+                     "r"(stg + (uint32_t)peer * L::SLOT), "r"((uint32_t)(2 * n_c * (L::PITCH + 8))), "r"(bar)
                      : "memory");
       }
     }

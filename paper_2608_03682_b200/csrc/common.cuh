@@ -34,7 +34,7 @@ __device__ __forceinline__ void pdl_enter() {
 
 // ---------------------------------------------------------------------------------------------
 // Tracing aid (the paper times phases with GPU-side profiler scopes): with tracing switched on, one CTA of each
-// traced launch writes device-global-timer stamps (ns) into its 8-entry slot of a trace buffer.
+// traced launch writes device-global-timer stamps (ns) into its 16-entry slot of a trace buffer.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;

@@ -232,7 +232,7 @@ phyai_status_t build_tables(phyai_expert* h, int n, cudaStream_t st, Tables** ou
 // merge pass): from this many CTAs on it beats the split mma.sync kernel + merge.
 constexpr int ATTN_TC_MIN_CTAS = 8;
 constexpr int MAX_SLABS = 16;
-constexpr int TRACE_SLOTS = 4096;
+constexpr int TRACE_SLOTS = 4096, TRACE_STAMPS = 16;
 
 int pick_nt(int M) { return M <= 64 ? 64 : (M <= 1024 ? 128 : 256); }
 
@@ -313,7 +313,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
   const int ss_n = D / 128;
   auto b1_gemm = [&](B1Gemm g, int which) -> phyai_status_t {
     g.M = M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact, g.inv_D = 1.0f / (float)D, g.eps = d.eps;
-    g.trace = (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * 8 : nullptr;
+    g.trace = (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr;
     int C = b1_pick_cluster(g.N / 128, g.K / 64, h->n_sm);
     if (h->b1_c[which] > 0 && b1_gemm_supported(g.N, g.K, h->b1_c[which], h->n_sm, which == 0)) C = h->b1_c[which];
     cudaError_t e = launch_b1_gemm(h->status, g, C, st);
@@ -374,14 +374,14 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         cudaError_t e;
         if (!b1_attn_tc && h->use_b1_attention && attention_b1_supported(d) && batch * (d.Hq / 2) * 8 <= h->n_sm)
           e = launch_attention_b1(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d, batch, h->wait_limit,
-                                  st, (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * 8 : nullptr);
+                                  st, (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
         else if (b1_attn_tc)
           e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d, batch, h->order,
                                   h->wait_limit, st);
         else
           e = launch_attention_cluster(h->rq, h->status, h->qkv, h->rope, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d,
                                        batch, h->wait_limit, st, nullptr,
-                                       (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * 8 : nullptr);
+                                       (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
         if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
         ++cnt;
         // ---- O projection + residual; leaves the operands of the second norm
@@ -1008,7 +1008,7 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
       h->trace = nullptr;      // (the buffer stays allocated until destroy)
       return PHYAI_OK;
     }
-    if (!h->trace_buf) ST(h->alloc(&h->trace_buf, (size_t)TRACE_SLOTS * 8, true));
+    if (!h->trace_buf) ST(h->alloc(&h->trace_buf, (size_t)TRACE_SLOTS * TRACE_STAMPS, true));
     h->trace = h->trace_buf;
     return PHYAI_OK;
   }
@@ -1025,10 +1025,10 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
 phyai_status_t phyai_read_trace(phyai_expert_t* h, uint64_t* out, size_t capacity, uint32_t* n_slots, uint32_t* n_stamps) {
   if (!h || !out || !n_slots || !n_stamps) return fail(PHYAI_ERR_INVALID_ARG, "NULL argument");
   if (!h->trace) return fail(PHYAI_ERR_INVALID_ARG, "tracing is off (phyai_set_option(h, \"trace\", 1))");
-  const size_t n = (size_t)TRACE_SLOTS * 8;
+  const size_t n = (size_t)TRACE_SLOTS * TRACE_STAMPS;
   if (capacity < n) return fail(PHYAI_ERR_INVALID_ARG, "capacity %zu < %zu entries", capacity, n);
   CU(cudaMemcpy(out, h->trace, n * sizeof(uint64_t), cudaMemcpyDeviceToHost));
-  *n_slots = TRACE_SLOTS, *n_stamps = 8;
+  *n_slots = TRACE_SLOTS, *n_stamps = TRACE_STAMPS;
   return PHYAI_OK;
 }
 

@@ -131,27 +131,13 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     if (g.gate) gate4 = __ldg(reinterpret_cast<const float4*>(g.gate + n));
     if (g.gain_next) gain4 = __ldg(reinterpret_cast<const float4*>(g.gain_next + n));
   }
-  pdl_wait();
-  trace_stamp(tr, 2);
-  // ---- after it: activations, the status word, per-token factors --------------------------------------------------
-  if (lane == 0) {
-    for (int s = (warp + 4) & 7; s < nk; s += 8) {
-      const uint32_t full = smem_u32(&bar_full[s]);
-      mbar_expect_tx(full, X_BYTES);
-      bulk_g2s(tiles + (uint32_t)s * STAGE + W_BYTES, reinterpret_cast<const uint8_t*>(g.X) + (size_t)(kc_begin + s) * X_BYTES,
-               X_BYTES, full);
-    }
-  }
-  if (tid == 255) suppress = status_set(status) ? 1 : 0;
-  if (tid < 64) {
-    float r = 1.0f;
-    if (g.ss_part && tid < M) {
-      float ss = 0.f;
-      for (int i = 0; i < g.ss_n; ++i) ss += g.ss_part[i * 64 + tid];
-      r = 1.0f / sqrtf(ss * g.inv_D + g.eps);
-    }
-    rstd_tab[tid] = r;
-    if (EPI == B1_QKV) {
+  const int n0 = tile * 128;
+  const int Nq = g.Hq * g.dh, Nk = g.Hkv * g.dh;
+  const bool rot_tile = EPI == B1_QKV && n0 < Nq + Nk;
+  if (EPI == B1_QKV) {
+    // where every token sits (the request block is written before the captured loop starts: safe to read ahead of
+    // the dependency wait), then the rotary rows of this CTA's tokens for the 64 channel pairs of this tile
+    if (tid < 64) {
       int2 e = make_int2(0, 0);
       if (tid < M) {
         const int b = tid / g.S, i = tid - b * g.S;
@@ -160,31 +146,51 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
       }
       tok_tab[tid] = e;
     }
+    __syncthreads();
+    if (rot_tile && g.rope) {
+      const int nn = n0 < Nq ? n0 : n0 - Nq;
+      const int t64 = (nn % g.dh) >> 7;
+      for (int idx = tid; idx < ntok * 32; idx += 256) {
+        const int tl = idx >> 5, c = idx & 31;
+        const int pos = tok_tab[tok_lo + tl].x;
+        const float4 v = __ldg(reinterpret_cast<const float4*>(g.rope + (size_t)pos * (g.dh >> 1) + t64 * 64) + c);
+        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(rope_s + (uint32_t)(tl * 32 + c) * 16), "f"(v.x), "f"(v.y),
+                     "f"(v.z), "f"(v.w)
+                     : "memory");
+      }
+    }
+  }
+  pdl_wait();
+  trace_stamp(tr, 2);
+  // ---- after it: activations, the status word, per-token factors (nothing the MMA warp has to wait for) -----------
+  if (lane == 0) {
+    for (int s = (warp + 4) & 7; s < nk; s += 8) {
+      const uint32_t full = smem_u32(&bar_full[s]);
+      mbar_expect_tx(full, X_BYTES);
+      bulk_g2s(tiles + (uint32_t)s * STAGE + W_BYTES, reinterpret_cast<const uint8_t*>(g.X) + (size_t)(kc_begin + s) * X_BYTES,
+               X_BYTES, full);
+    }
   }
   float4 hpre[2];
+  if (warp != 1) {
+    if (tid == 255) suppress = status_set(status) ? 1 : 0;
+    if (tid >= 64 && tid < 128) {
+      const int t = tid - 64;
+      float r = 1.0f;
+      if (g.ss_part && t < M) {
+        float ss = 0.f;
+        for (int i = 0; i < g.ss_n; ++i) ss += g.ss_part[i * 64 + t];
+        r = 1.0f / sqrtf(ss * g.inv_D + g.eps);
+      }
+      rstd_tab[t] = r;
+    }
+  }
   if (EPI == B1_RESID) {
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const int tl = warp + 8 * u;
       hpre[u] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (tl < ntok) hpre[u] = *reinterpret_cast<const float4*>(g.h + (size_t)(tok_lo + tl) * g.ldh + tile * 128 + lane * 4);
-    }
-  }
-  __syncthreads();
-  const int n0 = tile * 128;
-  const int Nq = g.Hq * g.dh, Nk = g.Hkv * g.dh;
-  const bool rot_tile = EPI == B1_QKV && n0 < Nq + Nk;
-  if (EPI == B1_QKV && rot_tile && g.rope) {
-    // the rotary rows of this CTA's tokens for the 64 channel pairs of this tile, while the MMAs run
-    const int nn = n0 < Nq ? n0 : n0 - Nq;
-    const int t64 = (nn % g.dh) >> 7;
-    for (int idx = tid; idx < ntok * 32; idx += 256) {
-      const int tl = idx >> 5, c = idx & 31;
-      const int pos = tok_tab[tok_lo + tl].x;
-      const float4 v = __ldg(reinterpret_cast<const float4*>(g.rope + (size_t)pos * (g.dh >> 1) + t64 * 64) + c);
-      asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(rope_s + (uint32_t)(tl * 32 + c) * 16), "f"(v.x), "f"(v.y),
-                   "f"(v.z), "f"(v.w)
-                   : "memory");
     }
   }
 
@@ -233,12 +239,13 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the bulk-copy engine
   __syncthreads();
   // ---- reduce-scatter over the cluster: every peer gets its token rows of my partial -----------------------------
-  if (tid < C && tid != rank) {
-    const int lo = (M * tid) / C, n = (M * (tid + 1)) / C - lo;
+  // (one copy per warp: the bulk copies issued by one warp complete one after the other)
+  if (lane == 0 && warp < C && warp != rank) {
+    const int lo = (M * warp) / C, n = (M * (warp + 1)) / C - lo;
     if (n > 0) {
       uint32_t dst, bar;
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(recv + (uint32_t)rank * slot), "r"(tid));
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(&bar_recv)), "r"(tid));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(recv + (uint32_t)rank * slot), "r"(warp));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(&bar_recv)), "r"(warp));
       asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                    "r"(stage + (uint32_t)lo * ROWB), "r"((uint32_t)n * ROWB), "r"(bar)
                    : "memory");

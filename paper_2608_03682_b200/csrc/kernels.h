@@ -224,7 +224,7 @@ struct B1Gemm {
   __nv_bfloat16* xn_out;
   float* ss_out;
   unsigned wait_limit;
-  unsigned long long* trace;   // 8-entry slot of this launch or null: start, set-up done, dependency resolved, MMAs
+  unsigned long long* trace;   // 16-entry slot of this launch or null: start, set-up done, dependency resolved, MMAs
                                // complete, partials received, epilogue done, cluster released, (SM id)
 };
 int b1_pick_cluster(int tiles, int KC, int n_sm);

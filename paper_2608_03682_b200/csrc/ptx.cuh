@@ -38,7 +38,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
   if (*c.abort_flag) return false;
   for (uint32_t it = 0; it < c.limit; ++it) {
     if (mbar_test(bar, parity)) return true;
-    if (it > 128) __nanosleep(32);
+    // Back off only when the wait is clearly not a pipeline wait of a few microseconds: a warp that sleeps wakes up
+    // late (measured: 0.75 us from an arrival to the waiting warp's next instruction with a 32 ns sleep in the loop,
+    // which every hand-over inside the batch-1 kernels paid).
+    if (it > 8192) __nanosleep(64);
   }
   *c.abort_flag = 1;
   atomicExch(c.status, ST_TIMEOUT);
