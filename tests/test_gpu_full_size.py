@@ -6,7 +6,7 @@ import torch
 
 from oracle import expert_oracle as O
 from paper_2608_03682_b200 import binding, synth
-from tests.helpers import BAR, rel_err
+from tests.helpers import BAR, elem_rel_err, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -28,6 +28,7 @@ def _run_batched(cfg, cfg_id, W, lens, n_steps, check):
     for b in check:
         ref = O.denoise(cfg, Wf, kvs[b], int(lens[b]), states[b], noise[b], n_steps)
         errs[b] = rel_err(out[b], ref)
+        print(f"request {b}: max rel err {errs[b]:.2e}, element-wise (floored) {elem_rel_err(out[b], ref):.2e}")
     return errs
 
 
@@ -41,11 +42,14 @@ def test_batch64_ragged_rollout_matches_oracle_on_sampled_requests():
     assert max(errs.values()) <= BAR["bf16"], errs
 
 
-@pytest.mark.parametrize("batch", [1, 8])
+@pytest.mark.parametrize("batch", [1, 8, 64, 256])
 def test_e4m3_weight_expert_matches_oracle(batch):
+    """Every batch size of the e4m3-weight sweep: 1 (cluster split-K kernels), 8 (general kernel, 128-token tiles,
+    split-K with per-channel scales), 64 and 256 (192 / 256-token tiles, rotary epilogue with scales, tcgen05
+    attention); up to three sampled requests per batch against the oracle."""
     cfg = synth.pi0_config(max_batch=batch, dtype="w8e4m3", max_prefix_len=816)
     W = synth.make_weights(cfg, 5)
-    check = [0] if batch == 1 else [0, batch - 1]
+    check = [0] if batch == 1 else ([0, batch - 1] if batch == 8 else [0, batch // 2, batch - 1])
     errs = _run_batched(cfg, 5, W, [816] * batch, 10, check)
     print(f"C5 batch {batch} max rel err:", {b: f"{e:.2e}" for b, e in errs.items()})
     assert max(errs.values()) <= BAR["w8e4m3"], errs

@@ -6,7 +6,7 @@ import torch
 
 from oracle import expert_oracle as O
 from paper_2608_03682_b200 import binding, synth
-from tests.helpers import BAR, gpu_single, rel_err, small_bf16_config
+from tests.helpers import BAR, elem_rel_err, gpu_single, rel_err, small_bf16_config
 
 pytestmark = pytest.mark.gpu
 
@@ -98,7 +98,8 @@ def test_pi_shaped_bf16_batch1_matches_oracle(name):
                 ex.set_option(k, v)
             got = gpu_single(cfg, W, kv, wl["prefix"], state, noise, wl["n_steps"], expert=ex)
             err = rel_err(got, ref)
-            print(f"{name} [{label}]: max rel err {err:.3e}, ||ref||inf {np.abs(ref).max():.3f}")
+            print(f"{name} [{label}]: max rel err {err:.3e}, element-wise (floored) {elem_rel_err(got, ref):.3e}, "
+                  f"||ref||inf {np.abs(ref).max():.3f}")
             assert err <= BAR["bf16"], (label, err)
 
 

@@ -1,0 +1,49 @@
+"""A device-side wait that gives up: with the iteration bound of the kernels' waits lowered to 1, a pipeline wait
+(a weight or activation copy that has not landed at the first poll) expires, the status word reports TIMEOUT, the
+kernels still run to their end (nothing hangs, nothing is left in flight), and after the bound is restored the same
+handle gives the correct result again.  Nothing here faults or hangs the device: the waited-for data does arrive."""
+import pytest
+import torch
+
+from oracle import expert_oracle as O
+from paper_2608_03682_b200 import binding, synth
+from tests.helpers import BAR, rel_err, small_bf16_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("cluster_gemm", [1, 0])
+@pytest.mark.parametrize("batch", [1, 40])
+def test_expired_wait_is_reported_and_the_handle_recovers(cluster_gemm, batch):
+    cfg = small_bf16_config("pi0", max_batch=batch, max_prefix_len=150)
+    W = synth.make_weights(cfg, 31, std=0.05)
+    lens = [150 - (7 * b) % 90 for b in range(batch)]
+    kvs = [synth.make_prefix_kv(cfg, 31, p, b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    states = torch.stack([synth.make_state(cfg, 31, b) for b in range(batch)])
+    noise = torch.stack([synth.make_noise(cfg, 31, b) for b in range(batch)])
+    args = (packed.cuda(), torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), 3)
+    ref0 = O.denoise(cfg, W, kvs[0], lens[0], states[0], noise[0], 3)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        ex.set_option("use_cluster_gemm", cluster_gemm)
+        good = ex.denoise_batched(*args).clone()
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        assert rel_err(good[0].double().cpu().numpy(), ref0) <= BAR["bf16"]
+
+        ex.set_option("wait_limit", 1)
+        out = torch.full_like(noise, 7.0).cuda()
+        ex.denoise_batched(*args, out=out)
+        torch.cuda.synchronize()                      # returns: every wait is bounded
+        assert ex.poll_status() == binding.ERR_TIMEOUT
+        assert ex.poll_status() == 0                  # reading the status word clears it
+        # the result of a timed-out call is invalid by contract (stores after the give-up are suppressed, earlier
+        # ones are not undone); it is only required to be there, i.e. the call ran to its end
+
+        ex.set_option("wait_limit", 1 << 22)
+        again = ex.denoise_batched(*args).clone()
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        # (beyond 64 tokens the split-K residual adds are atomic, so two runs agree to rounding, not to the bit)
+        assert rel_err(again[0].double().cpu().numpy(), ref0) <= BAR["bf16"]
+        assert rel_err(again.double().cpu().numpy(), good.double().cpu().numpy()) <= BAR["bf16"]
