@@ -174,12 +174,159 @@ def time_oracle(cfg, cfg_id, lens, n_steps, budget_s: float, repeats: int = 1, w
 
 
 # ------------------------------------------------------------------------------------------------
+# one workload on the CUDA path
+# ------------------------------------------------------------------------------------------------
+def percentiles(ms):
+    a = np.sort(np.asarray(ms, dtype=np.float64))
+    return {"mean": float(a.mean()), "p50": float(np.percentile(a, 50)), "p99": float(np.percentile(a, 99)),
+            "min": float(a[0]), "max": float(a[-1])}
+
+
+def roofline_of(name, cfg, lens, n_steps, batch, ms_per_step, peaks):
+    alg_bytes, alg_flops = algorithmic_cost(cfg, lens, n_steps)
+    secs = ms_per_step / 1e3
+    if batch < 8:
+        achieved = alg_bytes / secs / 1e9
+        traffic = NCU_TRAFFIC.get(name, (None, None))
+        return {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": traffic[0], "traffic_source": traffic[1],
+                "kernel": "whole captured loop (one graph launch = one chunk: all Euler steps and layers)",
+                "peak_source": f"{peaks['source']} copy bandwidth", "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_launch": alg_bytes}
+    achieved = alg_flops / secs / 1e12
+    return {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+            "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
+            "kernel": "whole captured loop (one graph launch = one batch of chunks)",
+            "peak_source": f"{peaks['source']} sustained bf16 GEMM (the loop runs for tens of ms under the power cap)",
+            "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+            "algorithmic_flops_per_launch": alg_flops}
+
+
+class Inputs:
+    """Host-side synthetic inputs of one workload; requests are generated once and shared by the batch sizes of a
+    sweep (request b has the same seed whatever the batch)."""
+
+    def __init__(self, cfg, cfg_id, lens):
+        import torch
+
+        self.kvs = [synth.make_prefix_kv(cfg, cfg_id, int(p), b) for b, p in enumerate(lens)]
+        self.states = ([synth.make_state(cfg, cfg_id, b) for b in range(len(lens))] if cfg.has_state_token else None)
+        self.noise = [synth.make_noise(cfg, cfg_id, b) for b in range(len(lens))]
+        self.torch = torch
+
+    def batch(self, n):
+        torch = self.torch
+        kv_h, cu = synth.pack_prefix_kv(self.kvs[:n])
+        states = None if self.states is None else torch.stack(self.states[:n])
+        return kv_h, torch.from_numpy(cu), states, torch.stack(self.noise[:n])
+
+
+def run_workload(name, ex, cfg, lens, n_steps, inputs, K, Wm, world, rank, local_rank, e2e=True, sample_clocks=False):
+    """Times one workload on an existing handle: K calls bracketed by one event pair (``ms_per_step``), one event pair
+    per call as well (mean / p50 / p99 / min), then the same through the host-buffer entry point."""
+    import torch
+
+    from paper_2608_03682_b200 import replicas
+
+    batch = len(lens)
+    batched = batch > 1
+    kv_h, cu_h, states_h, noise_h = inputs.batch(batch)
+    kv_d, noise_d, cu_d = kv_h.cuda(), noise_h.cuda(), cu_h.cuda()
+    states_d = None if states_h is None else states_h.cuda()
+    out_d = torch.empty_like(noise_d)
+    stream = torch.cuda.current_stream()
+
+    def call_device():
+        if batched:
+            ex.denoise_batched(kv_d, cu_d, states_d, noise_d, n_steps, out=out_d, stream=stream)
+        else:
+            ex.denoise(kv_d, lens[0], None if states_d is None else states_d[0], noise_d[0], n_steps, out=out_d[0],
+                       stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        replicas.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, iters):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+        barrier()
+        ev[0].record(stream)
+        for i in range(iters):
+            fn()
+            ev[i + 1].record(stream)
+        barrier()
+        total = replicas.max_over_ranks(ev[0].elapsed_time(ev[iters]), device="cuda")
+        return total, [ev[i].elapsed_time(ev[i + 1]) for i in range(iters)]
+
+    for _ in range(Wm):
+        call_device()
+    torch.cuda.synchronize()
+    status = ex.poll_status()
+    if status != 0:
+        raise SystemExit(f"{name}: device status {status} after warm-up")
+    sampler = ClockSampler(local_rank) if (sample_clocks and rank == 0) else None
+    total_ms, per_call = timed(call_device, K)
+    clocks = sampler.stop() if sampler else None
+    ms_per_step = total_ms / K
+    res = {"ms_per_step": ms_per_step, "per_call_ms": percentiles(per_call), "chunks_per_s": world * batch / (ms_per_step / 1e3),
+           "clocks": clocks, "launches_per_step": int(ex.launches_per_call(batch, n_steps)), "batch": batch}
+    ok = bool(torch.isfinite(out_d).all().item())
+    if e2e:
+        pin = lambda t: None if t is None else t.pin_memory()
+        kv_p, noise_p, states_p, cu_p = pin(kv_h), pin(noise_h), pin(states_h), pin(cu_h)
+        out_p = torch.empty_like(noise_h).pin_memory()
+
+        def call_host():
+            if batched:
+                ex.denoise_batched_host(kv_p, cu_p, states_p, noise_p, n_steps, out_p, stream=stream)
+            else:
+                ex.denoise_host(kv_p, lens[0], None if states_p is None else states_p[0], noise_p[0], n_steps, out_p[0],
+                                stream=stream)
+
+        for _ in range(3):
+            call_host()
+        e2e_total, _ = timed(call_host, K)
+        e2e_ms = e2e_total / K
+        h2d = kv_h.numel() * kv_h.element_size() + noise_h.numel() * 4 + (0 if states_h is None else states_h.numel() * 4)
+        if batched:
+            h2d += cu_h.numel() * 4
+        res["e2e"] = {"ms_per_step": e2e_ms, "chunks_per_s": world * batch / (e2e_ms / 1e3), "h2d_bytes_per_step": int(h2d),
+                      "d2h_bytes_per_step": int(noise_h.numel() * 4)}
+        ok = ok and bool(torch.isfinite(out_p).all().item())
+    status = ex.poll_status()
+    if status != 0:
+        raise SystemExit(f"{name}: device status {status} after the timed region")
+    res["finite"] = ok
+    del kv_d, noise_d, cu_d, states_d, out_d
+    return res
+
+
+def free_port():
+    import socket
+
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def respawn_replicas(n: int) -> int:
+    """``--gpus N`` outside torchrun: start N replica processes of this script (one per GPU, rendezvous on the loopback
+    address) and hand their output through.  Rank 0 of the children prints the JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+# ------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--workload", default=None,
+                    help="time one workload only (C1, C2, C3, C4, C5b1, C5b8, C5b64, C5b256); default: C2 as the headline "
+                         "plus every other configuration of the metric in the line's `workloads` map")
     ap.add_argument("--impl", default="phyai", choices=["phyai", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
@@ -188,16 +335,23 @@ def main():
     args = ap.parse_args()
     K, Wm = args.steps, max(args.warmup, 3)
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(respawn_replicas(args.gpus))
+
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    cfg, cfg_id, batch, lens, n_steps = workload(args.workload)
+    head = args.workload or "C2"
+    cfg, cfg_id, batch, lens, n_steps = workload(head)
     batched = batch > 1
     metric = (METRIC_BATCHED % batch) if batched else METRIC
     unit = "chunks/s" if batched else "ms"
-    config = {"workload": f"{args.workload}: {cfg.cond}-shaped expert, {cfg.dtype}, batch {batch}, "
-                          f"prefix {min(lens)}..{max(lens)}, {cfg.suffix_len} suffix tokens, {n_steps} Euler steps",
-              "batch": batch, "n_steps": n_steps, "replicas": world,
+
+    def describe(name, cfg, batch, lens, n_steps):
+        return (f"{name}: {cfg.cond}-shaped expert, {cfg.dtype}, batch {batch}, prefix {min(lens)}..{max(lens)}, "
+                f"{cfg.suffix_len} suffix tokens, {n_steps} Euler steps")
+
+    config = {"workload": describe(head, cfg, batch, lens, n_steps), "batch": batch, "n_steps": n_steps, "replicas": world,
               "l2": "inputs larger than L2 (weights streamed per step exceed 126 MB); no flush"}
 
     # -------------------------------------------------------------------------- reference arm
@@ -226,127 +380,82 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks = measured_peaks()
 
-    W = synth.make_weights(cfg, cfg_id)
-    ex = binding.Expert(cfg, binding.weights_to_device(W))
-    if args.no_graph:
-        ex.set_option("use_graph", 0)
-    for kv_ in args.opt:
-        key, _, val = kv_.partition("=")
-        ex.set_option(key, int(val))
-    del W
-    kvs = [synth.make_prefix_kv(cfg, cfg_id, p, b) for b, p in enumerate(lens)]
-    kv_h, cu = synth.pack_prefix_kv(kvs)
-    del kvs
-    states_h = torch.stack([synth.make_state(cfg, cfg_id, b) for b in range(batch)]) if cfg.has_state_token else None
-    noise_h = torch.stack([synth.make_noise(cfg, cfg_id, b) for b in range(batch)])
-    cu_h = torch.from_numpy(cu)
-    kv_d, noise_d, cu_d = kv_h.cuda(), noise_h.cuda(), cu_h.cuda()
-    states_d = None if states_h is None else states_h.cuda()
-    out_d = torch.empty_like(noise_d)
-    stream = torch.cuda.current_stream()
+    def make_expert(cfg, cfg_id):
+        W = synth.make_weights(cfg, cfg_id)
+        ex = binding.Expert(cfg, binding.weights_to_device(W))
+        del W
+        if args.no_graph:
+            ex.set_option("use_graph", 0)
+        for kv_ in args.opt:
+            key, _, val = kv_.partition("=")
+            ex.set_option(key, int(val))
+        return ex
 
-    def call_device():
-        if batched:
-            ex.denoise_batched(kv_d, cu_d, states_d, noise_d, n_steps, out=out_d, stream=stream)
-        else:
-            ex.denoise(kv_d, lens[0], None if states_d is None else states_d[0], noise_d[0], n_steps, out=out_d[0],
-                       stream=stream)
+    ex = make_expert(cfg, cfg_id)
+    inputs = Inputs(cfg, cfg_id, lens)
+    res = run_workload(head, ex, cfg, lens, n_steps, inputs, K, Wm, world, rank, local_rank, sample_clocks=True)
+    ex.close()
+    del inputs
+    torch.cuda.empty_cache()
 
-    pin = lambda t: None if t is None else t.pin_memory()
-    kv_p, noise_p, states_p, cu_p = pin(kv_h), pin(noise_h), pin(states_h), pin(cu_h)
-    out_p = torch.empty_like(noise_h).pin_memory()
+    # every other configuration the metric names, on fewer calls: batch 64 (C4), the adaRMS expert (C3), the e4m3 sweep
+    others = {}
+    if args.workload is None and world == 1:
+        Ko, Wo = min(K, 10), 3
+        for name in ("C3", "C4"):
+            c2, id2, b2, l2, n2 = workload(name)
+            e2 = make_expert(c2, id2)
+            r2 = run_workload(name, e2, c2, l2, n2, Inputs(c2, id2, l2), Ko, Wo, world, rank, local_rank)
+            e2.close()
+            torch.cuda.empty_cache()
+            r2["workload"], r2["steps"], r2["warmup"] = describe(name, c2, b2, l2, n2), Ko, Wo
+            r2["roofline"] = roofline_of(name, c2, l2, n2, b2, r2["ms_per_step"], peaks)
+            others[name] = r2
+        c5, id5, _, l5, n5 = workload("C5b256")
+        e5 = make_expert(c5, id5)                       # one handle (max_batch 256) serves the whole sweep
+        in5 = Inputs(c5, id5, l5)
+        for b5 in (1, 8, 64, 256):
+            name = f"C5b{b5}"
+            r5 = run_workload(name, e5, c5, l5[:b5], n5, in5, Ko if b5 < 256 else min(Ko, 5), Wo, world, rank, local_rank,
+                              e2e=(b5 <= 64))
+            r5["workload"], r5["steps"], r5["warmup"] = describe(name, c5, b5, l5[:b5], n5), Ko, Wo
+            r5["roofline"] = roofline_of(name, c5, l5[:b5], n5, b5, r5["ms_per_step"], peaks)
+            others[name] = r5
+        e5.close()
+        del in5
+        torch.cuda.empty_cache()
 
-    def call_host():
-        if batched:
-            ex.denoise_batched_host(kv_p, cu_p, states_p, noise_p, n_steps, out_p, stream=stream)
-        else:
-            ex.denoise_host(kv_p, lens[0], None if states_p is None else states_p[0], noise_p[0], n_steps, out_p[0],
-                            stream=stream)
-
-    from paper_2608_03682_b200 import replicas
-
-    def barrier():
-        torch.cuda.synchronize()
-        replicas.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, iters):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record(stream)
-        for _ in range(iters):
-            fn()
-        e1.record(stream)
-        barrier()
-        return replicas.max_over_ranks(e0.elapsed_time(e1), device="cuda")
-
-    for _ in range(Wm):
-        call_device()
-    torch.cuda.synchronize()
-    status = ex.poll_status()
-    if status != 0:
-        raise SystemExit(f"device status {status} after warm-up")
-
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    total_ms = timed(call_device, K)
-    clocks = sampler.stop() if sampler else None
-    ms_per_step = total_ms / K
-
-    for _ in range(3):
-        call_host()
-    e2e_ms = timed(call_host, K) / K
-    status = ex.poll_status()
-    if status != 0:
-        raise SystemExit(f"device status {status} after the timed region")
-    result_ok = bool(torch.isfinite(out_d).all().item()) and bool(torch.isfinite(out_p).all().item())
-
-    launches = ex.launches_per_call(batch, n_steps)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    peaks = measured_peaks()
-    alg_bytes, alg_flops = algorithmic_cost(cfg, lens, n_steps)
-    secs = ms_per_step / 1e3
-    hbm_bound = not batched or batch < 8
-    traffic = NCU_TRAFFIC.get(args.workload, (None, None))
-    if hbm_bound:
-        achieved = alg_bytes / secs / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": traffic[0], "traffic_source": traffic[1],
-                    "kernel": "whole captured loop (one graph launch = one chunk: all Euler steps and layers)",
-                    "peak_source": f"{peaks['source']} copy bandwidth", "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
-                    "algorithmic_bytes_per_launch": alg_bytes}
-    else:
-        achieved = alg_flops / secs / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
-                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
-                    "kernel": "whole captured loop (one graph launch = one batch of chunks)",
-                    "peak_source": f"{peaks['source']} sustained bf16 GEMM",
-                    "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS, "algorithmic_flops_per_launch": alg_flops}
-
-    value = world * batch / secs if batched else ms_per_step
-    e2e_value = world * batch / (e2e_ms / 1e3) if batched else e2e_ms
-    h2d = kv_h.numel() * kv_h.element_size() + noise_h.numel() * 4 + (0 if states_h is None else states_h.numel() * 4)
-    if batched:
-        h2d += cu_h.numel() * 4
+    ms_per_step = res["ms_per_step"]
+    roofline = roofline_of(head, cfg, lens, n_steps, batch, ms_per_step, peaks)
+    value = res["chunks_per_s"] if batched else ms_per_step
+    e2e_value = res["e2e"]["chunks_per_s"] if batched else res["e2e"]["ms_per_step"]
+    launches = res["launches_per_step"]
     line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": K, "warmup": Wm,
-            "ms_per_step": ms_per_step, "higher_is_better": batched, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if cfg.dtype != "f32" else "f32", "data": "synthetic", "config": config,
-            "chunks_per_s": world * batch / secs, "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": int(h2d),
-                    "d2h_bytes_per_step": int(noise_h.numel() * 4), "ms_per_step": e2e_ms},
-            "gpu_launches": int(launches * K), "launches_per_step": int(launches), "finite": result_ok,
+            "ms_per_step": ms_per_step, "per_call_ms": res["per_call_ms"], "higher_is_better": batched, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if cfg.dtype != "f32" else "f32", "data": "synthetic", "config": config,
+            "chunks_per_s": res["chunks_per_s"], "clocks": res["clocks"],
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": res["e2e"]["h2d_bytes_per_step"],
+                    "d2h_bytes_per_step": res["e2e"]["d2h_bytes_per_step"], "ms_per_step": res["e2e"]["ms_per_step"]},
+            "gpu_launches": int(launches * K), "launches_per_step": int(launches), "finite": res["finite"],
             "roofline": roofline}
+    if others:
+        line["workloads"] = others
+        if "C4" in others:
+            line["chunks_per_s_batch64"] = others["C4"]["chunks_per_s"]
+            line["tensor_frac_batch64"] = others["C4"]["roofline"]["frac"]
 
     if not args.no_cpu_baseline and world == 1:
         ms, sample, cores = time_oracle(cfg, cfg_id, lens, n_steps, budget_s=15.0, repeats=1)
         line["cpu_baseline"] = {"value": batch / (ms / 1e3) if batched else ms, "unit": unit, "cores": cores,
                                 "kind": "oracle", "sample": sample}
     print(json.dumps(line))
-    ex.close()
     if dist is not None:
         dist.destroy_process_group()
 
