@@ -72,6 +72,7 @@ struct phyai_expert {
   std::vector<float*> f_qkv, f_o, f_g, f_u, f_d;                 // SIMT fp32 row-major
   std::vector<__nv_bfloat16*> p_qkv, p_o, p_g, p_u, p_d;         // TC packed
   std::vector<float*> s_qkv, s_o, s_g, s_u, s_d;                 // TC per-channel scales (or null)
+  std::vector<uint8_t*> b_qkv, b_o, b_gu, b_d;                   // e4m3 byte blocks for the cluster GEMM (W8 experts)
 
   float2* rope = nullptr;
 
@@ -86,7 +87,8 @@ struct phyai_expert {
   bool il_ok = false;          // gate / up also packed interleaved (single-token-tile calls)
   bool b1_ok = false;          // the cluster split-K GEMM path covers this expert's shapes
   int use_cluster_gemm = 1;
-  int use_b1_attention = 1;    // tcgen05 attention with the key range split over a cluster (few requests)
+  int use_b1_attention = 1;
+  int use_w8_inkernel = 1;     // e4m3 experts: the cluster GEMM decodes byte blocks itself (0: bf16 images made at create)    // tcgen05 attention with the key range split over a cluster (few requests)
   int b1_c[4] = {0, 0, 0, 0};  // cluster sizes of the QKV / O / gate-up / down projections (0 = choose)
   float *ss_a = nullptr, *ss_b = nullptr;   // [D/128][64] partial sums of squares of h (after O / after down)
   unsigned long long* trace_buf = nullptr;
@@ -312,6 +314,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
   const bool b1 = h->b1_ok && h->use_cluster_gemm && M <= 64 && (b1_attn_tc || b1_attn_cluster);
   const bool b1_attn_b1 = !b1_attn_tc && h->use_b1_attention && attention_b1_supported(d) && batch * (d.Hq / 2) * 8 <= h->n_sm;
   const int ss_n = D / 128;
+  const bool use_w8 = h->use_w8_inkernel && !h->b_qkv.empty();
   auto b1_gemm = [&](B1Gemm g, int which) -> phyai_status_t {
     g.M = M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact, g.inv_D = 1.0f / (float)D, g.eps = d.eps;
     g.trace = (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr;
@@ -367,7 +370,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
           ++cnt;
         }
         B1Gemm q{};
-        q.W = h->p_qkv[l], q.X = h->xn64, q.N = d.Nqkv, q.K = D, q.epi = B1_QKV, q.wscale = h->s_qkv[l];
+        q.W = h->p_qkv[l], q.W8 = use_w8 ? h->b_qkv[l] : nullptr, q.X = h->xn64, q.N = d.Nqkv, q.K = D, q.epi = B1_QKV, q.wscale = h->s_qkv[l];
         if (l > 0) {
           q.ss_part = h->ss_b, q.ss_n = ss_n;
           q.shift_row = h->ada ? t.shw_qkv + ((size_t)k * d.L + l) * d.Nqkv : nullptr;
@@ -393,19 +396,19 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         const float *gain2, *shift2, *gate2;
         site(k, 2 * l + 1, &gain2, &shift2, &gate2);
         B1Gemm o{};
-        o.W = h->p_o[l], o.X = h->attn64, o.N = D, o.K = d.Nq, o.epi = B1_RESID, o.wscale = h->s_o[l];
+        o.W = h->p_o[l], o.W8 = use_w8 ? h->b_o[l] : nullptr, o.X = h->attn64, o.N = D, o.K = d.Nq, o.epi = B1_RESID, o.wscale = h->s_o[l];
         o.h = h->h, o.ldh = D, o.gate = gate, o.gain_next = gain2, o.xn_out = h->xn64, o.ss_out = h->ss_a;
         ST(b1_gemm(o, 1));
         // ---- gate / up + GeGLU
         B1Gemm gu{};
-        gu.W = h->p_gu_all + (size_t)l * D * 2 * d.F, gu.X = h->xn64, gu.N = 2 * d.F, gu.K = D, gu.epi = B1_GEGLU;
+        gu.W = h->p_gu_all + (size_t)l * D * 2 * d.F, gu.W8 = use_w8 ? h->b_gu[l] : nullptr, gu.X = h->xn64, gu.N = 2 * d.F, gu.K = D, gu.epi = B1_GEGLU;
         gu.wscale = h->s_g[l], gu.wscale2 = h->s_u[l], gu.ss_part = h->ss_a, gu.ss_n = ss_n;
         gu.shift_row = h->ada ? t.shw_gu + ((size_t)k * d.L + l) * 2 * d.F : nullptr;
         gu.out_tiled = h->m64;
         ST(b1_gemm(gu, 2));
         // ---- down projection + residual; leaves the operands of the next layer's first norm
         B1Gemm dn{};
-        dn.W = h->p_d[l], dn.X = h->m64, dn.N = D, dn.K = d.F, dn.epi = B1_RESID, dn.wscale = h->s_d[l];
+        dn.W = h->p_d[l], dn.W8 = use_w8 ? h->b_d[l] : nullptr, dn.X = h->m64, dn.N = D, dn.K = d.F, dn.epi = B1_RESID, dn.wscale = h->s_d[l];
         dn.h = h->h, dn.ldh = D, dn.gate = gate2;
         if (l + 1 < d.L) {
           const float *gain3, *shift3, *gate3;
@@ -730,6 +733,12 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       ST(h->alloc(&pd_all, (size_t)L * F * D));
       h->il_ok = F % 64 == 0;
       if (h->il_ok) ST(h->alloc(&h->p_gu_all, (size_t)L * D * 2 * F));
+      // cluster split-K path (one 64-token tile): every projection must fit the kernel's resident stages
+      auto fits = [&](int N, int K, bool qkv) {
+        return b1_gemm_supported(N, K, b1_pick_cluster(N / 128, K / 64, h->n_sm), h->n_sm, qkv);
+      };
+      h->b1_ok = h->il_ok && (d.dh == 128 || d.dh == 256) && D % 128 == 0 && d.S <= 64 && fits(Nqkv, D, true) &&
+                 fits(D, Nq, false) && fits(2 * F, D, false) && fits(D, F, false);
       if (w8) {
         ST(h->alloc(&h->s_qkv_all, (size_t)L * Nqkv)); ST(h->alloc(&h->s_o_all, (size_t)L * D));
         ST(h->alloc(&h->s_g_all, (size_t)L * F)); ST(h->alloc(&h->s_u_all, (size_t)L * F));
@@ -757,6 +766,22 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         launch_pack_tiled(w->wup[l], big_kind, pu, D, F, 0, st);
         launch_pack_tiled(w->wdown[l], big_kind, pd, F, D, 0, st);
         h->p_qkv.push_back(pq), h->p_o.push_back(po), h->p_g.push_back(pg), h->p_u.push_back(pu), h->p_d.push_back(pd);
+        if (w8 && h->b1_ok) {
+          // one byte per weight for the single-tile (HBM-bound) path; larger batches are tensor-bound and keep using
+          // the bf16 images above
+          uint8_t *bq, *bo, *bgu, *bd;
+          ST(h->alloc(&bq, (size_t)D * Nqkv)); ST(h->alloc(&bo, (size_t)Nq * D));
+          ST(h->alloc(&bgu, (size_t)D * 2 * F)); ST(h->alloc(&bd, (size_t)F * D));
+          const uint8_t* cq = reinterpret_cast<const uint8_t*>(w->wq[l]);
+          launch_pack_bytes(cq, bq, D, Nq, 0, st, 0, 0, d.dh);
+          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wk[l]), bq, D, Nkv, Nq, st, 0, 0, d.dh);
+          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wv[l]), bq, D, Nkv, Nq + Nkv, st);
+          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wo[l]), bo, Nq, D, 0, st);
+          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wgate[l]), bgu, D, F, 0, st, 64, 0);
+          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wup[l]), bgu, D, F, 0, st, 64, 1);
+          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wdown[l]), bd, F, D, 0, st);
+          h->b_qkv.push_back(bq), h->b_o.push_back(bo), h->b_gu.push_back(bgu), h->b_d.push_back(bd);
+        }
         float *cq = nullptr, *co = nullptr, *cg = nullptr, *cu = nullptr, *cd = nullptr;
         if (w8) {
           cq = h->s_qkv_all + (size_t)l * Nqkv, co = h->s_o_all + (size_t)l * D, cg = h->s_g_all + (size_t)l * F;
@@ -810,11 +835,6 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         if (need) ST(h->alloc(&h->attn_scratch, need, true));
       }
       // cluster split-K path (one 64-token tile): compact 64-row activation tiles and the norm partials
-      auto fits = [&](int N, int K, bool qkv) {
-        return b1_gemm_supported(N, K, b1_pick_cluster(N / 128, K / 64, h->n_sm), h->n_sm, qkv);
-      };
-      h->b1_ok = h->il_ok && h->qr_big && D % 128 == 0 && F % 64 == 0 && d.S <= 64 && fits(Nqkv, D, true) &&
-                 fits(D, Nq, false) && fits(2 * F, D, false) && fits(D, F, false);
       if (h->b1_ok) {
         ST(h->alloc(&h->xn64, (size_t)64 * D, true));
         ST(h->alloc(&h->attn64, (size_t)64 * Nq, true));
@@ -984,6 +1004,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   }
   if (!strcmp(key, "use_cluster_attention")) {
     h->use_cluster_attention = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_w8_inkernel")) {
+    h->use_w8_inkernel = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

@@ -57,10 +57,29 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int EPI>
+// Four e4m3 codes (one 32-bit word) -> two bf16 pairs, exactly, without the (slow-rate) conversion instructions.
+// A code is S EEEE MMM (bias 7).  Its byte goes to the high byte of a 16-bit half (byte permute): the sign is then
+// in place; the magnitude, moved down by four bits, puts EEEE into the low bits of bf16's exponent field and MMM
+// at the top of its mantissa, i.e. the bf16 number 2^(E - 127) (1 + M/8) -- for E = 0 the bf16 subnormal
+// 2^-126 (M/8).  One exact bf16x2 multiplication by 2^120 restores the bias: 2^(E - 7)(1 + M/8), and for E = 0
+// 2^-6 (M/8), which is the value of e4m3's subnormals; zero stays zero.  (bf16 multiplication has no flush-to-zero
+// mode: subnormal inputs are honoured.)  Five full-rate instructions per pair.
+__device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  uint32_t x0, x1;
+  asm("prmt.b32 %0, %1, 0, 0x1404;" : "=r"(x0) : "r"(w));   // [b1 0 b0 0]
+  asm("prmt.b32 %0, %1, 0, 0x3424;" : "=r"(x1) : "r"(w));   // [b3 0 b2 0]
+  const uint32_t t0 = (x0 & 0x80008000u) | ((x0 >> 4) & 0x07F007F0u);
+  const uint32_t t1 = (x1 & 0x80008000u) | ((x1 >> 4) & 0x07F007F0u);
+  const uint32_t c = 0x7B807B80u;   // (2^120, 2^120)
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(lo) : "r"(t0), "r"(c));
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(hi) : "r"(t1), "r"(c));
+}
+
+template <int EPI, bool W8>
 __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[MAXK];
+  __shared__ __align__(8) uint64_t bar_w8[MAXK];       // e4m3 weights: the byte blocks have landed
   __shared__ __align__(8) uint64_t bar_accum, bar_recv;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, suppress, acc_ok, recv_ok;
@@ -87,7 +106,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
 
   if (tid == 0) {
     abort_flag = 0;
-    for (int s = 0; s < MAXK; ++s) mbar_init(smem_u32(&bar_full[s]), 2);
+    for (int s = 0; s < MAXK; ++s) mbar_init(smem_u32(&bar_full[s]), W8 ? 1 : 2), mbar_init(smem_u32(&bar_w8[s]), 1);
     mbar_init(smem_u32(&bar_accum), 1);
     mbar_init(smem_u32(&bar_recv), 1);
     if (C > 1 && ntok > 0) mbar_expect_tx(smem_u32(&bar_recv), (uint32_t)(C - 1) * (uint32_t)ntok * ROWB);
@@ -107,10 +126,18 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
   // ---- before the dependency wait: weights (constants) and per-channel constants ------------------------------
   if (lane == 0) {
     for (int s = warp; s < nk; s += 8) {
-      const uint32_t full = smem_u32(&bar_full[s]);
-      mbar_expect_tx(full, W_BYTES);
-      bulk_g2s(tiles + (uint32_t)s * STAGE, reinterpret_cast<const uint8_t*>(g.W) + ((size_t)tile * KC + kc_begin + s) * W_BYTES,
-               W_BYTES, full);
+      if (W8) {
+        // one byte per weight: the 8 KB block lands in the upper half of the stage's 16 KB operand slot
+        const uint32_t full = smem_u32(&bar_w8[s]);
+        mbar_expect_tx(full, W_BYTES / 2);
+        bulk_g2s(tiles + (uint32_t)s * STAGE + W_BYTES / 2,
+                 reinterpret_cast<const uint8_t*>(g.W8) + ((size_t)tile * KC + kc_begin + s) * (W_BYTES / 2), W_BYTES / 2, full);
+      } else {
+        const uint32_t full = smem_u32(&bar_full[s]);
+        mbar_expect_tx(full, W_BYTES);
+        bulk_g2s(tiles + (uint32_t)s * STAGE, reinterpret_cast<const uint8_t*>(g.W) + ((size_t)tile * KC + kc_begin + s) * W_BYTES,
+                 W_BYTES, full);
+      }
     }
   }
   if (tid < 128) {
@@ -159,6 +186,42 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
                      : "memory");
       }
     }
+  }
+  if (W8) {
+    // e4m3 -> bf16 in place, ahead of the dependency wait where the weights arrive early (they are constants): every
+    // thread first takes its 32 bytes of every stage into registers (row = tid / 2, four 8-byte chunks), then, after
+    // a barrier, writes them back as 64 bytes of the swizzled K-major bf16 image the MMA reads.  The per-channel
+    // scale stays in the epilogue.
+    if (warp == 0)
+      for (int s = 0; s < nk; ++s) mbar_wait_drain(smem_u32(&bar_w8[s]), 0u, wc);
+    __syncthreads();
+    trace_stamp(tr, 9);
+    uint4 raw[MAXK][2];
+    const int r = tid >> 1, hc = (tid & 1) * 4;
+#pragma unroll
+    for (int s = 0; s < MAXK; ++s)
+      if (s < nk) {
+        const uint32_t src = tiles + (uint32_t)s * STAGE + W_BYTES / 2 + (uint32_t)r * 64 + (uint32_t)hc * 8;
+        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(raw[s][0].x), "=r"(raw[s][0].y), "=r"(raw[s][0].z), "=r"(raw[s][0].w) : "r"(src) : "memory");
+        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(raw[s][1].x), "=r"(raw[s][1].y), "=r"(raw[s][1].z), "=r"(raw[s][1].w) : "r"(src + 16) : "memory");
+      }
+    __syncthreads();
+#pragma unroll
+    for (int s = 0; s < MAXK; ++s)
+      if (s < nk) {
+        const uint32_t words[8] = {raw[s][0].x, raw[s][0].y, raw[s][0].z, raw[s][0].w, raw[s][1].x, raw[s][1].y, raw[s][1].z, raw[s][1].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {       // chunk hc + c: 8 codes = words[2c], words[2c + 1]
+          uint32_t o0, o1, o2, o3;
+          e4m3x4_to_bf16x4(words[2 * c], o0, o1);
+          e4m3x4_to_bf16x4(words[2 * c + 1], o2, o3);
+          const uint32_t dst = tiles + (uint32_t)s * STAGE + (uint32_t)r * 128 + (uint32_t)((((hc + c) ^ (r & 7))) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+        }
+      }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the tensor core's reads
+    __syncthreads();
+    trace_stamp(tr, 10);
   }
   pdl_wait();
   trace_stamp(tr, 2);
@@ -387,11 +450,11 @@ size_t b1_smem(int nk_max, int C, bool rope_rows) {
   return 1024 + region + (size_t)C * tpc * ROWB + (rope_rows ? (size_t)tpc * 512 : 0);
 }
 
-template <int EPI>
+template <int EPI, bool W8>
 cudaError_t launch_one(int* status, const B1Gemm& g, int C, cudaStream_t st) {
   static PerDeviceOnce once;
   if (once.needed()) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_b1<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1_SMEM_MAX);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_b1<EPI, W8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1_SMEM_MAX);
     if (e != cudaSuccess) return e;
     once.done();
   }
@@ -403,7 +466,7 @@ cudaError_t launch_one(int* status, const B1Gemm& g, int C, cudaStream_t st) {
   at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at, cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, k_gemm_b1<EPI>, status, g);
+  return cudaLaunchKernelEx(&cfg, k_gemm_b1<EPI, W8>, status, g);
 }
 
 }  // namespace
@@ -430,9 +493,14 @@ cudaError_t launch_b1_gemm(int* status, const B1Gemm& g_in, int C, cudaStream_t 
   const int KC = g.K / 64;
   g.nk_max = (KC + C - 1) / C;
   if (b1_smem(g.nk_max, C, g.epi == B1_QKV) > B1_SMEM_MAX) return cudaErrorInvalidConfiguration;
-  if (g.epi == B1_QKV) return launch_one<B1_QKV>(status, g, C, st);
-  if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU>(status, g, C, st);
-  return launch_one<B1_RESID>(status, g, C, st);
+  if (g.W8) {
+    if (g.epi == B1_QKV) return launch_one<B1_QKV, true>(status, g, C, st);
+    if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU, true>(status, g, C, st);
+    return launch_one<B1_RESID, true>(status, g, C, st);
+  }
+  if (g.epi == B1_QKV) return launch_one<B1_QKV, false>(status, g, C, st);
+  if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU, false>(status, g, C, st);
+  return launch_one<B1_RESID, false>(status, g, C, st);
 }
 
 }  // namespace phyai

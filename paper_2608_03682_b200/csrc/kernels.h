@@ -63,6 +63,9 @@ void launch_copy_cols(const void* src, int src_kind, const float* scale, float* 
 // (qkv_channel_to_packed).
 void launch_pack_tiled(const void* src, int src_kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st,
                        int il_group = 0, int il_second = 0, int perm_dh = 0);
+// e4m3 codes [in=K][out=N] -> byte blocks [N/128][K/64][128][64] in the packed row order of launch_pack_tiled
+void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group = 0,
+                       int il_second = 0, int perm_dh = 0);
 void launch_permute_scales(const float* src, float* dst, int N, int n_off, int perm_dh, cudaStream_t st);
 // Y[r][n] = act( sum_d X[r][d] * W[(w_row_off + d)][n] + bias[n] + add[n] ), r < R
 void launch_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K, const float* bias,
@@ -194,6 +197,8 @@ cudaError_t tc_gemm_setup();  // one-time attribute setup (dynamic shared memory
 enum : int { B1_QKV = 0, B1_GEGLU = 1, B1_RESID = 2 };
 struct B1Gemm {
   const __nv_bfloat16* W;    // packed blocks [N/128][K/64][128x64]
+  const uint8_t* W8;         // or: e4m3 codes, blocks [N/128][K/64][128 rows][64 bytes] in the same row order, decoded
+                             // to bf16 inside the kernel (one byte per weight crosses HBM); scales as below
   const __nv_bfloat16* X;    // tiled activations [K/64][64][64] (64-row tiles, back to back)
   int N, K, M;               // packed rows, contraction length, valid tokens (<= 64)
   int epi;

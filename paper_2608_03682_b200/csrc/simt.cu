@@ -118,6 +118,31 @@ void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int
   k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off, il_group, il_second, perm_dh);
 }
 
+// e4m3 codes [K][N] -> byte blocks of 128 out channels x 64 k (row order as in k_pack_tiled, no swizzle: the kernel
+// that decodes them writes the swizzled bf16 image itself).  One thread per 8 consecutive k of one out channel.
+__global__ void k_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, int il_group, int il_second,
+                             int perm_dh) {
+  const int KC = K >> 6;
+  const size_t chunks = (size_t)N * (K >> 3);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
+    const int n = (int)(i % N), k0 = (int)(i / N) << 3;
+    const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
+                            : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
+    const int kc = k0 >> 6, c = (k0 & 63) >> 3;
+    __align__(8) uint8_t v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = src[(size_t)(k0 + j) * N + n];
+    *reinterpret_cast<uint2*>(dst + (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 64 + (size_t)c * 8) =
+        *reinterpret_cast<const uint2*>(v);
+  }
+}
+void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group,
+                       int il_second, int perm_dh) {
+  const size_t chunks = (size_t)N * (K >> 3);
+  const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
+  k_pack_bytes<<<blocks, 256, 0, st>>>(src, dst, K, N, n_off, il_group, il_second, perm_dh);
+}
+
 // Row of an adaptive norm's shift through a packed weight matrix: out[n] = scale(n) * sum_k shift[k] * W[n][k].
 // One warp per packed row; a lane reads pairs of k out of the swizzled 128 x 64 blocks.
 __global__ void k_shift_rows(const float* shift, const __nv_bfloat16* Wp, const float* wscale, const float* wscale2,

@@ -226,6 +226,25 @@ def test_cluster_gemm_path_and_general_path_agree_and_are_reproducible(cond):
                 assert rel_err(outs[mode][b], refs[b]) <= BAR["bf16"], (mode, b, rel_err(outs[mode][b], refs[b]))
 
 
+@pytest.mark.parametrize("cond", ["pi0", "pi05"])
+def test_small_e4m3_expert_decoded_in_the_kernel_matches_oracle_and_the_expanded_weights(cond):
+    """e4m3 weights on the cluster split-K path are streamed as bytes and decoded to bf16 inside the kernel; the decode
+    is exact, so the result must equal, bit for bit, the one obtained from the bf16 images made at create time."""
+    cfg = small_bf16_config(cond, dtype="w8e4m3", max_prefix_len=300)
+    W = synth.make_weights(cfg, 22, std=0.05)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        for P in (0, 130, 300):
+            kv, state, noise = _inputs(cfg, 22, P)
+            ref = O.denoise(cfg, W, kv, P, state, noise, 3)
+            outs = []
+            for mode in (1, 0):
+                ex.set_option("use_w8_inkernel", mode)
+                got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
+                assert rel_err(got, ref) <= BAR["w8e4m3"], (P, mode, rel_err(got, ref))
+                outs.append(got)
+            assert np.array_equal(outs[0], outs[1]), P
+
+
 def test_single_request_after_a_ragged_batch_with_many_heads():
     """16 query heads of 256 select the request-per-CTA tcgen05 attention kernel even for one request; it walks the
     requests in an order that the batched call writes.  A single-request call on the same handle must reset it."""
