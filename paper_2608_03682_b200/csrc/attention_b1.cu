@@ -68,7 +68,9 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   const int rank = blockIdx.x, hp = blockIdx.y, b = blockIdx.z;
   const int head0 = hp * 2;
   const int hk = head0 / (d.Hq / d.Hkv);
-  const int S = d.S;
+  const int S = d.S;                                      // query rows per head
+  const int Sk = d.Sk > 0 ? d.Sk : d.S;                   // the request's own (suffix) keys that exist ...
+  const int Sk_stride = d.Sk_stride > 0 ? d.Sk_stride : d.S;   // ... and their row pitch per kv head
   const bool tracer = tid == 0 && rank == 0 && hp == 0 && b == 0;
 
   pdl_launch_dependents();
@@ -103,7 +105,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   // (the request block is written before the captured loop starts: safe to read ahead of the dependency wait)
   const Request r = *a.rq;
   const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
-  const int Kt = P + S;                                   // keys of this request: prefix, then its own suffix
+  const int Kt = P + Sk;                                  // keys of this request: prefix, then its own suffix
   const int key_lo = (int)(((long long)Kt * rank) / 8), key_hi = (int)(((long long)Kt * (rank + 1)) / 8);
   const int T = (key_hi - key_lo + KB - 1) / KB;          // tiles of this CTA (1 unless P + S > 1024; 0 for an empty range)
 
@@ -160,7 +162,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     const size_t kv_stride = (size_t)d.Hkv * DH * 2;
     const uint8_t* Gp = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
                         (((size_t)(a.layer * 2 + (is_v ? 1 : 0)) * r.kv_tokens + p0) * d.Hkv + hk) * (DH * 2) + (size_t)lc * 16;
-    const uint8_t* Gs = reinterpret_cast<const uint8_t*>(is_v ? a.vr : a.kr) + ((size_t)(b * d.Hkv + hk) * S) * (DH * 2) +
+    const uint8_t* Gs = reinterpret_cast<const uint8_t*>(is_v ? a.vr : a.kr) + ((size_t)(b * d.Hkv + hk) * Sk_stride) * (DH * 2) +
                         (size_t)lc * 16;
     const uint32_t tile_base = (is_v ? Vs : Ks) + (uint32_t)(lc >> 3) * L::BLOCK;
     // rows of tile t: the prefix rows when `prefix` is set, otherwise the request's own (suffix) rows and, for V, zeros

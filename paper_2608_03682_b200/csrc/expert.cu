@@ -88,6 +88,8 @@ struct phyai_expert {
   bool b1_ok = false;          // the cluster split-K GEMM path covers this expert's shapes
   int use_cluster_gemm = 1;
   int use_b1_attention = 1;
+  int use_state_cache = 1;     // block-causal experts: state token computed once per call (single-tile calls)
+  __nv_bfloat16 *kr_st = nullptr, *vr_st = nullptr;   // [L][max 64 tokens worth of requests][Hkv][S][dh] suffix K / V per layer
   int use_w8_inkernel = 1;     // e4m3 experts: the cluster GEMM decodes byte blocks itself (0: bf16 images made at create)    // tcgen05 attention with the key range split over a cluster (few requests)
   int b1_c[4] = {0, 0, 0, 0};  // cluster sizes of the QKV / O / gate-up / down projections (0 = choose)
   float *ss_a = nullptr, *ss_b = nullptr;   // [D/128][64] partial sums of squares of h (after O / after down)
@@ -266,7 +268,21 @@ int pick_splits(int n_tiles, int tok_tiles, int KC) {
 }
 
 phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, cudaStream_t st) {
-  const Dims& d = h->d;
+  const Dims& d0 = h->d;
+  // State-token caching (block-causal suffix mask, plain norms): the state token sees the prefix and itself only, so
+  // its hidden states and its rotated key / value of every layer depend neither on x nor on t.  They are computed
+  // once per call by a pass over the state tokens alone and kept as key row 0 of every layer's suffix K / V; the
+  // loop then runs on the action tokens only (query row i = key row 1 + i).  Single-tile calls on the cluster path.
+  // A single 64-token tile: the projections run on the cluster split-K kernel with the norms folded in (five
+  // kernels per layer: QKV, attention, O, gate/up, down).
+  const bool b1_attn_tc = h->attn_mma && h->use_tc_attention && h->qr_big && attention_tc_supported(d0) &&
+                          batch * (d0.Hq / 2) >= ATTN_TC_MIN_CTAS;
+  const bool b1_attn_cluster = !b1_attn_tc && h->attn_mma && h->use_cluster_attention && batch * d0.Hq * 8 <= 2 * h->n_sm;
+  const bool b1 = h->b1_ok && h->use_cluster_gemm && batch * d0.S <= 64 && (b1_attn_tc || b1_attn_cluster);
+  const bool b1_attn_b1 = !b1_attn_tc && h->use_b1_attention && attention_b1_supported(d0) && batch * (d0.Hq / 2) * 8 <= h->n_sm;
+  const bool cache_state = b1 && b1_attn_b1 && h->kr_st && h->use_state_cache;
+  Dims d = d0;
+  if (cache_state) d.ns = 0, d.S = d0.H, d.block_causal = 0, d.Sk = d0.S, d.Sk_stride = d0.S, d.koff = 1;
   const int M = batch * d.S, D = d.D;
   const int nt = pick_nt(M);
   const int tok_tiles = (M + nt - 1) / nt;
@@ -306,17 +322,10 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     ++cnt;
   };
 
-  // A single 64-token tile: the projections run on the cluster split-K kernel with the norms folded in (five
-  // kernels per layer: QKV, attention, O, gate/up, down).
-  const bool b1_attn_tc = h->attn_mma && h->use_tc_attention && h->qr_big && attention_tc_supported(d) &&
-                          batch * (d.Hq / 2) >= ATTN_TC_MIN_CTAS;
-  const bool b1_attn_cluster = !b1_attn_tc && h->attn_mma && h->use_cluster_attention && batch * d.Hq * 8 <= 2 * h->n_sm;
-  const bool b1 = h->b1_ok && h->use_cluster_gemm && M <= 64 && (b1_attn_tc || b1_attn_cluster);
-  const bool b1_attn_b1 = !b1_attn_tc && h->use_b1_attention && attention_b1_supported(d) && batch * (d.Hq / 2) * 8 <= h->n_sm;
   const int ss_n = D / 128;
   const bool use_w8 = h->use_w8_inkernel && !h->b_qkv.empty();
-  auto b1_gemm = [&](B1Gemm g, int which) -> phyai_status_t {
-    g.M = M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact, g.inv_D = 1.0f / (float)D, g.eps = d.eps;
+  auto b1_gemm = [&](B1Gemm g, int which, int Mloc) -> phyai_status_t {
+    g.M = Mloc, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact, g.inv_D = 1.0f / (float)D, g.eps = d.eps;
     g.trace = (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr;
     // The QKV projection leaves the SMs of the attention kernel free: that kernel then starts (and fetches its prefix
     // tiles) while the projection still runs.  Measured on the pi0-shaped expert: 7.6 ms per chunk with 140 CTAs,
@@ -330,8 +339,78 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     return PHYAI_OK;
   };
 
-  launch_begin(h->rq, h->status, h->state_w, h->state_b, h->state_tok, d, batch, st);
+  // One layer on the cluster path: QKV, attention, O, gate/up, down (five kernels; the norms are folded in).
+  // `kv_only`: stop after the QKV projection (the state pass needs nothing but the last layer's key / value).
+  const size_t kv_layer = (size_t)batch * d0.Hkv * d0.S * d0.dh;   // per-layer stride of the cached suffix K / V
+  auto b1_layer = [&](const Dims& dd, int Mloc, int k, int l, bool kv_only, __nv_bfloat16* kr, __nv_bfloat16* vr) -> phyai_status_t {
+    const float *gain, *shift, *gate;
+    site(k, 2 * l, &gain, &shift, &gate);
+    // ---- QKV: layer 0 reads a normalised tile; later layers read bf16(h * gain) and the partial sums of squares left
+    // by the previous layer's down projection
+    if (l == 0) {
+      launch_rmsnorm(h->status, h->h, gain, shift, nullptr, h->xn64, 64, Mloc, D, dd.eps, st);
+      ++cnt;
+    }
+    B1Gemm q{};
+    q.W = h->p_qkv[l], q.W8 = use_w8 ? h->b_qkv[l] : nullptr, q.X = h->xn64, q.N = dd.Nqkv, q.K = D, q.epi = B1_QKV, q.wscale = h->s_qkv[l];
+    if (l > 0) {
+      q.ss_part = h->ss_b, q.ss_n = ss_n;
+      q.shift_row = h->ada ? t.shw_qkv + ((size_t)k * dd.L + l) * dd.Nqkv : nullptr;
+    }
+    q.rq = h->rq, q.rope = h->rope, q.qr = h->qr_big, q.kr = kr, q.vr = vr;
+    q.S = dd.S, q.Hq = dd.Hq, q.Hkv = dd.Hkv, q.dh = dd.dh, q.Sk_stride = suffix_key_stride(dd), q.koff = dd.koff;
+    ST(b1_gemm(q, 0, Mloc));
+    if (kv_only) return PHYAI_OK;
+    // ---- attention -> bf16 tile of the output projection
+    cudaError_t e;
+    if (b1_attn_b1)
+      e = launch_attention_b1(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->wait_limit, st,
+                              (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
+    else if (b1_attn_tc)
+      e = launch_attention_tc(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->order, h->wait_limit, st);
+    else
+      e = launch_attention_cluster(h->rq, h->status, h->qkv, h->rope, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch,
+                                   h->wait_limit, st, nullptr,
+                                   (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
+    if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
+    ++cnt;
+    // ---- O projection + residual; leaves the operands of the second norm
+    const float *gain2, *shift2, *gate2;
+    site(k, 2 * l + 1, &gain2, &shift2, &gate2);
+    B1Gemm o{};
+    o.W = h->p_o[l], o.W8 = use_w8 ? h->b_o[l] : nullptr, o.X = h->attn64, o.N = D, o.K = dd.Nq, o.epi = B1_RESID, o.wscale = h->s_o[l];
+    o.h = h->h, o.ldh = D, o.gate = gate, o.gain_next = gain2, o.xn_out = h->xn64, o.ss_out = h->ss_a;
+    ST(b1_gemm(o, 1, Mloc));
+    // ---- gate / up + GeGLU
+    B1Gemm gu{};
+    gu.W = h->p_gu_all + (size_t)l * D * 2 * dd.F, gu.W8 = use_w8 ? h->b_gu[l] : nullptr, gu.X = h->xn64, gu.N = 2 * dd.F, gu.K = D, gu.epi = B1_GEGLU;
+    gu.wscale = h->s_g[l], gu.wscale2 = h->s_u[l], gu.ss_part = h->ss_a, gu.ss_n = ss_n;
+    gu.shift_row = h->ada ? t.shw_gu + ((size_t)k * dd.L + l) * 2 * dd.F : nullptr;
+    gu.out_tiled = h->m64;
+    ST(b1_gemm(gu, 2, Mloc));
+    // ---- down projection + residual; leaves the operands of the next layer's first norm
+    B1Gemm dn{};
+    dn.W = h->p_d[l], dn.W8 = use_w8 ? h->b_d[l] : nullptr, dn.X = h->m64, dn.N = D, dn.K = dd.F, dn.epi = B1_RESID, dn.wscale = h->s_d[l];
+    dn.h = h->h, dn.ldh = D, dn.gate = gate2;
+    if (l + 1 < dd.L) {
+      const float *gain3, *shift3, *gate3;
+      site(k, 2 * l + 2, &gain3, &shift3, &gate3);
+      dn.gain_next = gain3, dn.xn_out = h->xn64, dn.ss_out = h->ss_b;
+    }
+    ST(b1_gemm(dn, 3, Mloc));
+    return PHYAI_OK;
+  };
+
+  launch_begin(h->rq, h->status, h->state_w, h->state_b, h->state_tok, d0, batch, st);
   ++cnt;
+  if (cache_state) {
+    // the state tokens alone through every layer: row b of h = request b's state token
+    Dims dp = d0;
+    dp.S = 1, dp.Sk = 1, dp.Sk_stride = d0.S, dp.koff = 0;
+    CU(cudaMemcpyAsync(h->h, h->state_tok, (size_t)batch * D * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    for (int l = 0; l < d0.L; ++l)
+      ST(b1_layer(dp, batch, 0, l, l + 1 == d0.L, h->kr_st + (size_t)l * kv_layer, h->vr_st + (size_t)l * kv_layer));
+  }
   for (int k = 0; k < n; ++k) {
     // ---- suffix embedding ----
     if (!h->ada) {
@@ -363,59 +442,8 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       const float *gain, *shift, *gate;
       site(k, 2 * l, &gain, &shift, &gate);
       if (b1) {
-        // ---- QKV: layer 0 of a step reads a normalised tile; later layers read bf16(h * gain) and the partial sums of
-        // squares left by the previous layer's down projection
-        if (l == 0) {
-          launch_rmsnorm(h->status, h->h, gain, shift, nullptr, h->xn64, 64, M, D, d.eps, st);
-          ++cnt;
-        }
-        B1Gemm q{};
-        q.W = h->p_qkv[l], q.W8 = use_w8 ? h->b_qkv[l] : nullptr, q.X = h->xn64, q.N = d.Nqkv, q.K = D, q.epi = B1_QKV, q.wscale = h->s_qkv[l];
-        if (l > 0) {
-          q.ss_part = h->ss_b, q.ss_n = ss_n;
-          q.shift_row = h->ada ? t.shw_qkv + ((size_t)k * d.L + l) * d.Nqkv : nullptr;
-        }
-        q.rq = h->rq, q.rope = h->rope, q.qr = h->qr_big, q.kr = h->kr_big, q.vr = h->vr_big;
-        q.S = d.S, q.Hq = d.Hq, q.Hkv = d.Hkv, q.dh = d.dh;
-        ST(b1_gemm(q, 0));
-        // ---- attention -> bf16 tile of the output projection
-        cudaError_t e;
-        if (b1_attn_b1)
-          e = launch_attention_b1(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d, batch, h->wait_limit,
-                                  st, (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
-        else if (b1_attn_tc)
-          e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d, batch, h->order,
-                                  h->wait_limit, st);
-        else
-          e = launch_attention_cluster(h->rq, h->status, h->qkv, h->rope, h->qr_big, h->kr_big, h->vr_big, l, h->attn64, 64, d,
-                                       batch, h->wait_limit, st, nullptr,
-                                       (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
-        if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
-        ++cnt;
-        // ---- O projection + residual; leaves the operands of the second norm
-        const float *gain2, *shift2, *gate2;
-        site(k, 2 * l + 1, &gain2, &shift2, &gate2);
-        B1Gemm o{};
-        o.W = h->p_o[l], o.W8 = use_w8 ? h->b_o[l] : nullptr, o.X = h->attn64, o.N = D, o.K = d.Nq, o.epi = B1_RESID, o.wscale = h->s_o[l];
-        o.h = h->h, o.ldh = D, o.gate = gate, o.gain_next = gain2, o.xn_out = h->xn64, o.ss_out = h->ss_a;
-        ST(b1_gemm(o, 1));
-        // ---- gate / up + GeGLU
-        B1Gemm gu{};
-        gu.W = h->p_gu_all + (size_t)l * D * 2 * d.F, gu.W8 = use_w8 ? h->b_gu[l] : nullptr, gu.X = h->xn64, gu.N = 2 * d.F, gu.K = D, gu.epi = B1_GEGLU;
-        gu.wscale = h->s_g[l], gu.wscale2 = h->s_u[l], gu.ss_part = h->ss_a, gu.ss_n = ss_n;
-        gu.shift_row = h->ada ? t.shw_gu + ((size_t)k * d.L + l) * 2 * d.F : nullptr;
-        gu.out_tiled = h->m64;
-        ST(b1_gemm(gu, 2));
-        // ---- down projection + residual; leaves the operands of the next layer's first norm
-        B1Gemm dn{};
-        dn.W = h->p_d[l], dn.W8 = use_w8 ? h->b_d[l] : nullptr, dn.X = h->m64, dn.N = D, dn.K = d.F, dn.epi = B1_RESID, dn.wscale = h->s_d[l];
-        dn.h = h->h, dn.ldh = D, dn.gate = gate2;
-        if (l + 1 < d.L) {
-          const float *gain3, *shift3, *gate3;
-          site(k, 2 * l + 2, &gain3, &shift3, &gate3);
-          dn.gain_next = gain3, dn.xn_out = h->xn64, dn.ss_out = h->ss_b;
-        }
-        ST(b1_gemm(dn, 3));
+        ST(b1_layer(d, M, k, l, false, cache_state ? h->kr_st + (size_t)l * kv_layer : h->kr_big,
+                    cache_state ? h->vr_st + (size_t)l * kv_layer : h->vr_big));
         continue;
       }
       launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs());
@@ -841,6 +869,12 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         ST(h->alloc(&h->m64, (size_t)64 * F, true));
         ST(h->alloc(&h->ss_a, (size_t)(D / 128) * 64, true));
         ST(h->alloc(&h->ss_b, (size_t)(D / 128) * 64, true));
+        if (d.block_causal && d.ns && !ada) {
+          // per-layer suffix K / V (key row 0 = the cached state token) for as many requests as fit one 64-token tile
+          const size_t per_layer = (size_t)(64 / d.S > 0 ? 64 / d.S : 1) * d.Hkv * d.S * d.dh;
+          ST(h->alloc(&h->kr_st, (size_t)L * per_layer, true));
+          ST(h->alloc(&h->vr_st, (size_t)L * per_layer, true));
+        }
       }
       ST(h->alloc(&h->xn_t, Mp * D, true));
       ST(h->alloc(&h->attn_t, Mp * Nq, true));
@@ -1004,6 +1038,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   }
   if (!strcmp(key, "use_cluster_attention")) {
     h->use_cluster_attention = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_state_cache")) {
+    h->use_state_cache = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
       if (tid < M) {
         const int b = tid / g.S, i = tid - b * g.S;
         const int* cu = g.rq->cu_lens;
-        e = make_int2(cu[b + 1] - cu[b] + i, b * 64 + i);
+        e = make_int2(cu[b + 1] - cu[b] + g.koff + i, b * 64 + i);
       }
       tok_tab[tid] = e;
     }
@@ -368,7 +368,9 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
             }
           }
           const int b = e.y >> 6, i = e.y & 63;
-          __nv_bfloat16* dst = base + ((size_t)(b * H + head) * g.S + i) * g.dh + t64 * 64 + j0;
+          // (q: one row per query token; k: the request's key rows, query row i at key row koff + i)
+          __nv_bfloat16* dst = base + (isq ? ((size_t)(b * H + head) * g.S + i) : ((size_t)(b * H + head) * g.Sk_stride + g.koff + i)) * g.dh +
+                               t64 * 64 + j0;
           *reinterpret_cast<uint4*>(dst) = make_uint4(pack2(lo[0] * osc, lo[1] * osc), pack2(lo[2] * osc, lo[3] * osc),
                                                       pack2(lo[4] * osc, lo[5] * osc), pack2(lo[6] * osc, lo[7] * osc));
           *reinterpret_cast<uint4*>(dst + half) = make_uint4(pack2(hi[0] * osc, hi[1] * osc), pack2(hi[2] * osc, hi[3] * osc),
@@ -386,7 +388,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
 #pragma unroll
           for (int u = 0; u < 8; ++u) x[u] = fin(x[u], j0 + u, r);
           const int b = e.y >> 6, i = e.y & 63;
-          *reinterpret_cast<uint4*>(g.vr + ((size_t)(b * g.Hkv + head) * g.S + i) * g.dh + coff + j0) =
+          *reinterpret_cast<uint4*>(g.vr + ((size_t)(b * g.Hkv + head) * g.Sk_stride + g.koff + i) * g.dh + coff + j0) =
               make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
         }
       }

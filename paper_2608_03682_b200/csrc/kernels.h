@@ -43,7 +43,13 @@ struct Dims {
   int L, D, F, Hq, Hkv, dh, Ds, A, H, ns, S, Nqkv, Nq;
   float eps;
   int gelu_exact, block_causal;
+  // Suffix keys of the cluster kernels when they differ from the query rows (state-token caching): a request's
+  // rotated suffix K / V rows are Sk_stride rows apart per kv head, the first Sk of them exist, and query row i is
+  // key row koff + i (position prefix_len + koff + i).  All zero = "same as the queries" (Sk = Sk_stride = S, koff = 0).
+  int Sk, Sk_stride, koff;
 };
+inline int suffix_keys(const Dims& d) { return d.Sk > 0 ? d.Sk : d.S; }
+inline int suffix_key_stride(const Dims& d) { return d.Sk_stride > 0 ? d.Sk_stride : d.S; }
 
 // ---- request block ---------------------------------------------------------------------------
 void launch_set_request(Request* dst, const Request& src, int* cu_internal, cudaStream_t st, int* order = nullptr);
@@ -217,6 +223,7 @@ struct B1Gemm {
   const float2* rope;
   __nv_bfloat16 *qr, *kr, *vr;
   int S, Hq, Hkv, dh;
+  int Sk_stride, koff;       // key rows per (request, kv head) in kr / vr and the key row of query row 0 (see Dims)
   // B1_GEGLU: W holds gate and up interleaved in groups of 64 channels; output [N/128][64][64] tiled
   __nv_bfloat16* out_tiled;
   int gelu_exact;

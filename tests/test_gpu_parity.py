@@ -296,3 +296,41 @@ def test_large_batch_tcgen05_attention_matches_oracle_and_the_mma_sync_kernel():
         assert rel_err(tc[b], ref) <= BAR["bf16"], (b, rel_err(tc[b], ref))
         assert rel_err(legacy[b], ref) <= BAR["bf16"], (b, rel_err(legacy[b], ref))
 
+
+
+# ------------------------------------------------------------------------------------------ state-token caching
+@pytest.mark.parametrize("shape", ["small", "full_width"])
+def test_block_causal_state_token_is_cached_once_per_call(shape):
+    """With the block-causal suffix mask the state token's per-layer key and value do not depend on x or t; single-tile
+    calls compute them once per call (a pass over the state tokens alone) and run the loop on the action tokens.
+    Same mathematics as the masked network: compared with the oracle, and with the uncached GPU path."""
+    if shape == "small":
+        cfg = small_bf16_config("pi0", suffix_block_causal=True, max_batch=3, max_prefix_len=300)
+        cases, n = [[300], [0], [41, 0, 222]], 4
+    else:
+        cfg = synth.ExpertConfig(n_layers=2, width=1024, mlp_dim=4096, n_q_heads=8, n_kv_heads=1, head_dim=256,
+                                 state_dim=32, action_dim=32, horizon=50, has_state_token=True, max_prefix_len=968,
+                                 max_batch=1, cond="pi0", dtype="bf16", suffix_block_causal=True)
+        cases, n = [[816], [968], [5]], 3
+    W = synth.make_weights(cfg, 23, std=0.05 if shape == "small" else 0.02)
+    Wf = O.Weights(W)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        for lens in cases:
+            B = len(lens)
+            kvs = [synth.make_prefix_kv(cfg, 23, p, b) for b, p in enumerate(lens)]
+            packed, cu = synth.pack_prefix_kv(kvs)
+            states = torch.stack([synth.make_state(cfg, 23, b) for b in range(B)])
+            noise = torch.stack([synth.make_noise(cfg, 23, b) for b in range(B)])
+            args = (packed.cuda(), torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), n)
+            outs = {}
+            for cached in (1, 0):
+                ex.set_option("use_state_cache", cached)
+                outs[cached] = ex.denoise_batched(*args).double().cpu().numpy()
+                torch.cuda.synchronize()
+                assert ex.poll_status() == 0
+            assert ex.launches_per_call(B, n) > 0
+            for b in range(B):
+                ref = O.denoise(cfg, Wf, kvs[b], lens[b], states[b], noise[b], n)
+                for cached in (1, 0):
+                    assert rel_err(outs[cached][b], ref) <= BAR["bf16"], (lens, b, cached, rel_err(outs[cached][b], ref))
+            assert rel_err(outs[1], outs[0]) <= BAR["bf16"]
