@@ -35,7 +35,8 @@ METRIC_BATCHED = "chunks/sec at batch %d"
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (bench.py cannot run ncu itself)
-NCU_TRAFFIC = {"C2": (6.406537e9 + 0.148150e9, "profiles/per_operator_loop_c2_batch1.md")}
+NCU_TRAFFIC = {"C2": (180 * 37.47e6 + 10 * 5.0e6, "profiles/cluster_loop_c2_c5_batch1.md"),
+               "C5b1": (180 * 20.29e6 + 10 * 5.0e6, "profiles/cluster_loop_c2_c5_batch1.md")}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 
 
@@ -48,6 +49,8 @@ def workload(name: str):
         return synth.tiny_config(), 1, 1, [64], 4
     if name == "C2":
         return synth.pi0_config(), 2, 1, [816], 10
+    if name == "C2m":   # C2 with the block-causal suffix mask (state token cached once per call)
+        return synth.pi0_config().with_(suffix_block_causal=True), 2, 1, [816], 10
     if name == "C3":
         return synth.pi05_config(), 3, 1, [968], 10
     if name == "C4":
@@ -413,6 +416,18 @@ def main():
             r2["workload"], r2["steps"], r2["warmup"] = describe(name, c2, b2, l2, n2), Ko, Wo
             r2["roofline"] = roofline_of(name, c2, l2, n2, b2, r2["ms_per_step"], peaks)
             others[name] = r2
+        # the block-causal variant of C2: state token cached once per call, and the same handle without the cache
+        cm, idm, bm, lm, nm = workload("C2m")
+        em = make_expert(cm, idm)
+        inm = Inputs(cm, idm, lm)
+        rm = run_workload("C2m", em, cm, lm, nm, inm, Ko, Wo, world, rank, local_rank, e2e=False)
+        em.set_option("use_state_cache", 0)
+        rm["ms_per_step_without_state_cache"] = run_workload("C2m", em, cm, lm, nm, inm, Ko, Wo, world, rank, local_rank,
+                                                             e2e=False)["ms_per_step"]
+        em.close()
+        rm["workload"], rm["steps"], rm["warmup"] = describe("C2m", cm, bm, lm, nm) + ", block-causal suffix mask", Ko, Wo
+        rm["roofline"] = roofline_of("C2m", cm, lm, nm, bm, rm["ms_per_step"], peaks)
+        others["C2m"] = rm
         c5, id5, _, l5, n5 = workload("C5b256")
         e5 = make_expert(c5, id5)                       # one handle (max_batch 256) serves the whole sweep
         in5 = Inputs(c5, id5, l5)
@@ -420,6 +435,11 @@ def main():
             name = f"C5b{b5}"
             r5 = run_workload(name, e5, c5, l5[:b5], n5, in5, Ko if b5 < 256 else min(Ko, 5), Wo, world, rank, local_rank,
                               e2e=(b5 <= 64))
+            if b5 == 1:   # the single-tile path streams the e4m3 bytes; for comparison: the bf16 images made at create
+                e5.set_option("use_w8_inkernel", 0)
+                r5["ms_per_step_bf16_images"] = run_workload(name, e5, c5, l5[:b5], n5, in5, Ko, Wo, world, rank, local_rank,
+                                                             e2e=False)["ms_per_step"]
+                e5.set_option("use_w8_inkernel", 1)
             r5["workload"], r5["steps"], r5["warmup"] = describe(name, c5, b5, l5[:b5], n5), Ko, Wo
             r5["roofline"] = roofline_of(name, c5, l5[:b5], n5, b5, r5["ms_per_step"], peaks)
             others[name] = r5

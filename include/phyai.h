@@ -293,6 +293,49 @@ phyai_status_t phyai_suffix_attention_static(const phyai_attention_desc_t *desc,
                                              int32_t *status_word, void *stream);
 size_t phyai_suffix_attention_static_capacity(void);
 
+/*
+ * The steps either side of the loop that belong to the model adapter (Sec. "Architecture": the adapter owns
+ * preprocessing, cache validity and action conversion).
+ *
+ * phyai_pack_prefix_kv: a backbone's padded K / V of every layer -> the library's ragged prefix-KV layout.
+ *   desc            n_layers, n_kv_heads, head_dim, elem_bytes (2 = bfloat16, 4 = float32), batch, p_max
+ *   k, v            device, [n_layers][batch][p_max][n_kv_heads][head_dim], K already rotated; rows >= lens[b] are
+ *                   padding and are never read; 16-byte aligned
+ *   lens            device int32 [batch], 0 <= lens[b] <= p_max
+ *   prefix_kv       device, receives [n_layers][2][kv_tokens][n_kv_heads][head_dim]: request b at rows
+ *                   cu[b] .. cu[b] + lens[b] - 1, no padding rows; rows >= cu[batch] are left untouched
+ *   cu_prefix_lens  device int32 [batch + 1], written: the exclusive prefix sum of lens
+ *   status_word     device int32, zeroed by the caller; a length outside 0..p_max or sum(lens) > kv_tokens sets it to
+ *                   PHYAI_ERR_INVALID_ARG and nothing is copied (cu_prefix_lens is still written)
+ * Bit-exact copy.  Only enqueues work on `stream`.  Errors: INVALID_ARG (NULL, zero size, misalignment, a row that
+ * is not a multiple of 16 bytes), CUDA; message in phyai_adapter_last_error().
+ */
+typedef struct {
+  uint32_t struct_size;
+  uint32_t n_layers, n_kv_heads, head_dim, elem_bytes, batch, p_max;
+} phyai_kv_pack_desc_t;
+
+phyai_status_t phyai_pack_prefix_kv(const phyai_kv_pack_desc_t *desc, const void *k, const void *v, const int32_t *lens,
+                                    void *prefix_kv, uint64_t kv_tokens, int32_t *cu_prefix_lens, int32_t *status_word,
+                                    void *stream);
+
+/*
+ * phyai_postprocess_actions: the raw chunk x at t = 0 -> robot actions (appendices on the pi0 / pi0.5 reproductions:
+ * actions are clipped to [-1, 1] in normalised space and un-normalised with the checkpoint's q01 / q99 quantile
+ * statistics; the controller uses the first out_horizon steps and out_dim action dimensions).
+ *   out[b][h][a] = (clip(x[b][h][a], clip_lo, clip_hi) + 1) / 2 * (q99[a] - q01[a]) + q01[a],  h < out_horizon, a < out_dim
+ *   x     device float32 [batch][horizon][action_dim];  out  device float32 [batch][out_horizon][out_dim]
+ *   q01, q99   device float32 [>= out_dim], or both NULL (no un-normalisation: q01 = -1, q99 = 1)
+ *   clip_lo >= clip_hi disables the clip.
+ * Only enqueues work.  Errors: INVALID_ARG, CUDA.
+ */
+phyai_status_t phyai_postprocess_actions(const float *x, uint32_t batch, uint32_t horizon, uint32_t action_dim,
+                                         const float *q01, const float *q99, float clip_lo, float clip_hi,
+                                         uint32_t out_horizon, uint32_t out_dim, float *out, void *stream);
+
+/* Thread-local description of the last error of an adapter entry point. */
+const char *phyai_adapter_last_error(void);
+
 /* Thread-local description of the last error of an operator entry point. */
 const char *phyai_op_last_error(void);
 

@@ -28,7 +28,8 @@ EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes
            "phyai_denoise_batched", "phyai_denoise_host", "phyai_denoise_batched_host", "phyai_poll_status",
            "phyai_set_option", "phyai_launches_per_call", "phyai_last_error", "phyai_version",
            "phyai_suffix_attention", "phyai_suffix_attention_scratch_bytes", "phyai_op_last_error",
-           "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity", "phyai_read_trace")
+           "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity", "phyai_read_trace",
+           "phyai_pack_prefix_kv", "phyai_postprocess_actions", "phyai_adapter_last_error")
 
 
 class PhyaiError(RuntimeError):
@@ -52,6 +53,11 @@ _VPP = C.POINTER(C.c_void_p)
 class AttentionDesc(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("struct_size", "n_q_heads", "n_kv_heads", "head_dim", "suffix_len",
                                           "n_layers", "layer", "state_token_block_causal", "num_splits")]
+
+
+class KvPackDesc(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("struct_size", "n_layers", "n_kv_heads", "head_dim", "elem_bytes", "batch",
+                                          "p_max")]
 
 
 class WeightsStruct(C.Structure):
@@ -100,6 +106,10 @@ def load_library() -> C.CDLL:
                                            _VP, _VP]
     lib.phyai_suffix_attention_static.argtypes = lib.phyai_suffix_attention.argtypes
     lib.phyai_suffix_attention_static_capacity.restype = C.c_size_t
+    lib.phyai_pack_prefix_kv.argtypes = [C.POINTER(KvPackDesc), _VP, _VP, _VP, _VP, C.c_uint64, _VP, _VP, _VP]
+    lib.phyai_postprocess_actions.argtypes = [_VP, C.c_uint32, C.c_uint32, C.c_uint32, _VP, _VP, C.c_float, C.c_float,
+                                              C.c_uint32, C.c_uint32, _VP, _VP]
+    lib.phyai_adapter_last_error.restype = C.c_char_p
     _lib = lib
     return lib
 
@@ -288,3 +298,38 @@ def suffix_attention(desc: AttentionDesc, qkv: torch.Tensor, prefix_kv: torch.Te
     if st != OK:
         raise PhyaiError(st, lib.phyai_op_last_error().decode())
     return out, status
+
+
+def pack_prefix_kv(k: torch.Tensor, v: torch.Tensor, lens: torch.Tensor, kv_tokens: Optional[int] = None, stream=None):
+    """Padded backbone K / V ``[L, B, p_max, Hkv, dh]`` + ``lens`` (int32 ``[B]``, device) -> the library's ragged
+    layout.  Returns (prefix_kv ``[L, 2, kv_tokens, Hkv, dh]``, cu_prefix_lens int32 ``[B + 1]``, status word)."""
+    lib = load_library()
+    L, B, p_max, Hkv, dh = k.shape
+    if kv_tokens is None:
+        kv_tokens = B * p_max
+    desc = KvPackDesc()
+    desc.struct_size = C.sizeof(KvPackDesc)
+    desc.n_layers, desc.n_kv_heads, desc.head_dim, desc.elem_bytes, desc.batch, desc.p_max = L, Hkv, dh, k.element_size(), B, p_max
+    out = torch.zeros(L, 2, kv_tokens, Hkv, dh, dtype=k.dtype, device=k.device)
+    cu = torch.empty(B + 1, dtype=torch.int32, device=k.device)
+    status = torch.zeros(1, dtype=torch.int32, device=k.device)
+    st = lib.phyai_pack_prefix_kv(C.byref(desc), _ptr(k), _ptr(v), _ptr(lens), _ptr(out), int(kv_tokens), _ptr(cu), _ptr(status),
+                                  _stream_ptr(stream))
+    if st != OK:
+        raise PhyaiError(st, lib.phyai_adapter_last_error().decode())
+    return out, cu, status
+
+
+def postprocess_actions(x: torch.Tensor, q01: Optional[torch.Tensor], q99: Optional[torch.Tensor], clip=(-1.0, 1.0),
+                        out_horizon: Optional[int] = None, out_dim: Optional[int] = None, stream=None) -> torch.Tensor:
+    """Raw chunk ``[B, H, A]`` -> clipped, un-normalised actions ``[B, out_horizon, out_dim]``."""
+    lib = load_library()
+    B, H, A = x.shape
+    out_horizon, out_dim = out_horizon or H, out_dim or A
+    out = torch.empty(B, out_horizon, out_dim, dtype=torch.float32, device=x.device)
+    lo, hi = (clip if clip is not None else (0.0, 0.0))
+    st = lib.phyai_postprocess_actions(_ptr(x), B, H, A, _ptr(q01), _ptr(q99), float(lo), float(hi), out_horizon, out_dim,
+                                       _ptr(out), _stream_ptr(stream))
+    if st != OK:
+        raise PhyaiError(st, lib.phyai_adapter_last_error().decode())
+    return out

@@ -1,0 +1,125 @@
+// The two small steps either side of the denoising loop that belong to the model adapter (paper, Sec. "Architecture":
+// the adapter owns preprocessing, cache layout and action conversion): packing a backbone's padded per-layer K / V
+// into the library's ragged prefix-KV layout, and converting the raw action chunk (x at t = 0) into robot actions.
+// Both are pure data movement / element-wise work: coalesced 16-byte copies, one thread per output element.
+#include <cstdio>
+
+#include "../../include/phyai.h"
+#include "kernels.h"
+
+namespace phyai {
+namespace {
+
+thread_local char g_ad_err[256] = "";
+
+// cu[0] = 0, cu[b + 1] = cu[b] + lens[b]; a length outside 0..p_max or a total beyond kv_tokens raises the status word
+// (INVALID_ARG) and the pack kernel then copies nothing.
+__global__ void k_kv_scan(const int* lens, int batch, int p_max, unsigned long long kv_tokens, int* cu, int* status) {
+  if (threadIdx.x != 0) return;
+  long long acc = 0;
+  bool bad = false;
+  cu[0] = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int n = lens[b];
+    if (n < 0 || n > p_max) bad = true;
+    acc += n < 0 ? 0 : n;
+    cu[b + 1] = (int)(acc > 0x7fffffffLL ? 0x7fffffffLL : acc);
+  }
+  if ((unsigned long long)acc > kv_tokens) bad = true;
+  if (bad) atomicExch(status, ST_INVALID_ARG);
+}
+
+// src [L][B][p_max][row_bytes], dst [L][2][kv_tokens][row_bytes]: plane (l, kv) of request b, rows p < lens[b], go to
+// rows cu[b] + p.  One thread per 16 bytes; grid.y = layer * 2 + (0 = K, 1 = V).
+__global__ void k_kv_pack(const uint4* k, const uint4* v, const int* lens, const int* cu, const int* status, uint4* dst,
+                          int batch, int p_max, unsigned long long kv_tokens, int row_chunks) {
+  if (status_set(status)) return;
+  const int layer = blockIdx.y >> 1, is_v = blockIdx.y & 1;
+  const uint4* src = (is_v ? v : k) + (size_t)layer * batch * p_max * row_chunks;
+  uint4* out = dst + ((size_t)layer * 2 + is_v) * kv_tokens * row_chunks;
+  const size_t total = (size_t)batch * p_max * row_chunks;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % row_chunks);
+    const size_t row = i / row_chunks;
+    const int p = (int)(row % p_max), b = (int)(row / p_max);
+    if (p < lens[b]) out[((size_t)cu[b] + p) * row_chunks + c] = src[i];
+  }
+}
+
+// out[b][h][a] = (clip(x[b][h][a]) + 1) / 2 * (q99[a] - q01[a]) + q01[a] for h < H_out, a < A_out
+__global__ void k_postprocess(const float* x, const float* q01, const float* q99, float* out, int batch, int H, int A,
+                              int H_out, int A_out, float lo, float hi, int do_clip) {
+  const size_t total = (size_t)batch * H_out * A_out;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int a = (int)(i % A_out), hh = (int)((i / A_out) % H_out), b = (int)(i / ((size_t)A_out * H_out));
+    float v = x[((size_t)b * H + hh) * A + a];
+    if (do_clip) v = fminf(fmaxf(v, lo), hi);
+    const float lo_q = q01 ? q01[a] : -1.0f, hi_q = q99 ? q99[a] : 1.0f;
+    out[i] = (v + 1.0f) * 0.5f * (hi_q - lo_q) + lo_q;
+  }
+}
+
+}  // namespace
+}  // namespace phyai
+
+extern "C" {
+
+const char* phyai_adapter_last_error(void) { return phyai::g_ad_err; }
+
+phyai_status_t phyai_pack_prefix_kv(const phyai_kv_pack_desc_t* desc, const void* k, const void* v, const int32_t* lens,
+                                    void* prefix_kv, uint64_t kv_tokens, int32_t* cu_prefix_lens, int32_t* status_word,
+                                    void* stream) {
+  using namespace phyai;
+  auto bad = [](const char* m) {
+    snprintf(g_ad_err, sizeof(g_ad_err), "%s", m);
+    return PHYAI_ERR_INVALID_ARG;
+  };
+  if (!desc || desc->struct_size != sizeof(phyai_kv_pack_desc_t)) return bad("desc is NULL or has a wrong struct_size");
+  if (!k || !v || !lens || !prefix_kv || !cu_prefix_lens || !status_word) return bad("a pointer argument is NULL");
+  if (!desc->n_layers || !desc->n_kv_heads || !desc->head_dim || !desc->batch || !desc->p_max)
+    return bad("a size in desc is zero");
+  if (desc->elem_bytes != 2 && desc->elem_bytes != 4) return bad("elem_bytes must be 2 (bfloat16) or 4 (float32)");
+  const size_t row_bytes = (size_t)desc->n_kv_heads * desc->head_dim * desc->elem_bytes;
+  if (row_bytes % 16) return bad("n_kv_heads * head_dim * elem_bytes must be a multiple of 16");
+  if ((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(prefix_kv)) & 15u)
+    return bad("k, v and prefix_kv must be 16-byte aligned");
+  if (kv_tokens > 0x7fffffffull || desc->batch > 65535u || desc->n_layers > 32767u) return bad("kv_tokens, batch or n_layers too large");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int chunks = (int)(row_bytes / 16);
+  k_kv_scan<<<1, 32, 0, st>>>(lens, (int)desc->batch, (int)desc->p_max, kv_tokens, cu_prefix_lens, status_word);
+  const size_t total = (size_t)desc->batch * desc->p_max * chunks;
+  const int blocks = (int)((total + 255) / 256 < 2048 ? (total + 255) / 256 : 2048);
+  k_kv_pack<<<dim3(blocks, desc->n_layers * 2), 256, 0, st>>>(reinterpret_cast<const uint4*>(k), reinterpret_cast<const uint4*>(v), lens,
+                                                             cu_prefix_lens, status_word, reinterpret_cast<uint4*>(prefix_kv),
+                                                             (int)desc->batch, (int)desc->p_max, kv_tokens, chunks);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    snprintf(g_ad_err, sizeof(g_ad_err), "kernel launch failed: %s", cudaGetErrorString(e));
+    return PHYAI_ERR_CUDA;
+  }
+  return PHYAI_OK;
+}
+
+phyai_status_t phyai_postprocess_actions(const float* x, uint32_t batch, uint32_t horizon, uint32_t action_dim,
+                                         const float* q01, const float* q99, float clip_lo, float clip_hi,
+                                         uint32_t out_horizon, uint32_t out_dim, float* out, void* stream) {
+  using namespace phyai;
+  if (!x || !out || !batch || !horizon || !action_dim || !out_horizon || !out_dim || out_horizon > horizon ||
+      out_dim > action_dim || ((q01 == nullptr) != (q99 == nullptr))) {
+    snprintf(g_ad_err, sizeof(g_ad_err), "NULL pointer, zero size, out_horizon > horizon, out_dim > action_dim, or only one of q01 / q99 given");
+    return PHYAI_ERR_INVALID_ARG;
+  }
+  const size_t total = (size_t)batch * out_horizon * out_dim;
+  const int blocks = (int)((total + 255) / 256 < 1024 ? (total + 255) / 256 : 1024);
+  k_postprocess<<<blocks, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(x, q01, q99, out, (int)batch, (int)horizon,
+                                                                           (int)action_dim, (int)out_horizon, (int)out_dim,
+                                                                           clip_lo, clip_hi, clip_lo < clip_hi ? 1 : 0);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    snprintf(g_ad_err, sizeof(g_ad_err), "kernel launch failed: %s", cudaGetErrorString(e));
+    return PHYAI_ERR_CUDA;
+  }
+  return PHYAI_OK;
+}
+
+}  // extern "C"

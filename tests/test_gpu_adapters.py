@@ -1,0 +1,81 @@
+"""The adapter-side entry points on the GPU against their oracle: the KV-layout writer is a bit-exact gather, the
+action post-processing float32 arithmetic (one fused multiply-add per element: 1e-6 relative)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import adapter_oracle as A
+from paper_2608_03682_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("dtype,L,B,p_max,Hkv,dh", [(torch.bfloat16, 3, 5, 70, 1, 256), (torch.float32, 2, 4, 33, 2, 24),
+                                                      (torch.bfloat16, 18, 8, 968, 1, 256)])
+def test_kv_layout_writer_is_a_bit_exact_ragged_gather(dtype, L, B, p_max, Hkv, dh):
+    g = torch.Generator().manual_seed(7)
+    k = torch.randn(L, B, p_max, Hkv, dh, generator=g).to(dtype)
+    v = torch.randn(L, B, p_max, Hkv, dh, generator=g).to(dtype)
+    lens = synth.make_ragged_lengths(41, B, 0, p_max)
+    lens[0], lens[-1] = 0, p_max                                    # an empty request and a full one
+    as_bits = (lambda t: t.view(torch.int16).numpy()) if dtype == torch.bfloat16 else (lambda t: t.numpy())
+    ref, cu_ref = A.pack_prefix_kv(as_bits(k), as_bits(v), lens)
+    total = int(cu_ref[-1])
+    out, cu, status = binding.pack_prefix_kv(k.cuda(), v.cuda(), torch.from_numpy(lens).cuda(), kv_tokens=total + 3)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert cu.cpu().numpy().tolist() == cu_ref.tolist()
+    got = as_bits(out.cpu())
+    assert np.array_equal(got[:, :, :total], ref)
+    assert not got[:, :, total:].any()                              # rows past the last request stay untouched
+
+
+def test_kv_layout_writer_feeds_the_denoising_call():
+    """Packed by the writer, the prefix KV gives the same actions as the host-side packing of the synthetic inputs."""
+    from tests.helpers import small_bf16_config
+    cfg = small_bf16_config("pi0", max_batch=3, max_prefix_len=90)
+    W = synth.make_weights(cfg, 24, std=0.05)
+    lens = np.array([90, 0, 37], dtype=np.int32)
+    kvs = [synth.make_prefix_kv(cfg, 24, int(p), b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    padded = torch.zeros(cfg.n_layers, 2, 3, 90, cfg.n_kv_heads, cfg.head_dim, dtype=torch.bfloat16)
+    for b, kv in enumerate(kvs):
+        padded[:, :, b, : kv.shape[2]] = kv
+    out, cu_d, status = binding.pack_prefix_kv(padded[:, 0].contiguous().cuda(), padded[:, 1].contiguous().cuda(),
+                                               torch.from_numpy(lens).cuda(), kv_tokens=int(cu[-1]))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(out.cpu(), packed)
+    states = torch.stack([synth.make_state(cfg, 24, b) for b in range(3)]).cuda()
+    noise = torch.stack([synth.make_noise(cfg, 24, b) for b in range(3)]).cuda()
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        a = ex.denoise_batched(out, cu_d, states, noise, 3).clone()
+        b2 = ex.denoise_batched(packed.cuda(), torch.from_numpy(cu).cuda(), states, noise, 3).clone()
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0 and torch.equal(a, b2)
+
+
+def test_kv_layout_writer_reports_bad_lengths_on_the_device():
+    k = torch.zeros(1, 2, 8, 1, 64, dtype=torch.bfloat16).cuda()
+    for lens in ([3, 9], [-1, 2]):
+        out, cu, status = binding.pack_prefix_kv(k, k, torch.tensor(lens, dtype=torch.int32).cuda(), kv_tokens=16)
+        torch.cuda.synchronize()
+        assert int(status.item()) == binding.ERR_INVALID_ARG and not out.any()
+    out, cu, status = binding.pack_prefix_kv(k, k, torch.tensor([8, 8], dtype=torch.int32).cuda(), kv_tokens=15)
+    torch.cuda.synchronize()
+    assert int(status.item()) == binding.ERR_INVALID_ARG            # does not fit the output buffer
+    with pytest.raises(binding.PhyaiError):
+        binding.pack_prefix_kv(torch.zeros(1, 1, 4, 1, 4, dtype=torch.bfloat16).cuda(),   # 8-byte rows
+                               torch.zeros(1, 1, 4, 1, 4, dtype=torch.bfloat16).cuda(), torch.tensor([1], dtype=torch.int32).cuda())
+
+
+def test_action_postprocessing_matches_oracle():
+    g = torch.Generator().manual_seed(9)
+    x = torch.randn(6, 50, 32, generator=g) * 1.3
+    q01, q99 = -torch.rand(32, generator=g) * 3 - 0.1, torch.rand(32, generator=g) * 3 + 0.1
+    for kw in (dict(), dict(out_horizon=32, out_dim=14), dict(clip=None)):
+        ref = A.postprocess_actions(x.numpy(), q01.numpy(), q99.numpy(), **kw)
+        got = binding.postprocess_actions(x.cuda(), q01.cuda(), q99.cuda(), **kw).cpu().numpy()
+        assert got.shape == ref.shape
+        np.testing.assert_allclose(got, ref, rtol=1e-6, atol=1e-6)
+    got = binding.postprocess_actions(x.cuda(), None, None, clip=(-1.0, 1.0)).cpu().numpy()
+    np.testing.assert_allclose(got, np.clip(x.numpy(), -1, 1), rtol=0, atol=1e-7)
