@@ -336,6 +336,35 @@ phyai_status_t phyai_postprocess_actions(const float *x, uint32_t batch, uint32_
 /* Thread-local description of the last error of an adapter entry point. */
 const char *phyai_adapter_last_error(void);
 
+/*
+ * Data-parallel serving front-end, host side (Sec. "Parallel Execution": data-parallel runners exchange no state;
+ * appendix on eight-GPU serving: rank 0 collects at most 32 pending observations, waits up to 20 ms for a batch to
+ * fill, gives every worker a fixed local batch -- the shape its CUDA graph was captured for --, pads the local
+ * inputs to that shape and drops the padded outputs after the gather).  No device work; thread-safe.
+ *
+ *   config   max_batch (most requests of one batch), n_workers x local_batch >= max_batch, window_ms >= 0
+ *   submit   any thread: queue a request (an opaque 64-bit id chosen by the caller)
+ *   next     the serving loop: blocks until a batch is due -- max_batch requests pending, or window_ms passed since
+ *            the OLDEST pending request arrived -- or until timeout_ms have passed (then *n = 0).  ids: HOST array of
+ *            max_batch entries, filled in arrival order.
+ *   plan     pure function: slots[w * local_batch + j] = index into the batch (request for worker w, slot j) or -1
+ *            (padding); requests fill the workers in order.  *active_workers = workers that hold a request.
+ * Errors: INVALID_ARG (NULL, zero sizes, n_workers * local_batch < max_batch, n > max_batch), OOM.
+ */
+typedef struct phyai_batcher phyai_batcher_t;
+typedef struct {
+  uint32_t struct_size;
+  uint32_t max_batch, n_workers, local_batch;
+  double window_ms;
+} phyai_batcher_config_t;
+
+phyai_status_t phyai_batcher_create(const phyai_batcher_config_t *cfg, phyai_batcher_t **out);
+void phyai_batcher_destroy(phyai_batcher_t *b);
+phyai_status_t phyai_batcher_submit(phyai_batcher_t *b, uint64_t request_id);
+phyai_status_t phyai_batcher_next(phyai_batcher_t *b, double timeout_ms, uint64_t *ids, uint32_t *n);
+uint32_t phyai_batcher_pending(phyai_batcher_t *b);
+phyai_status_t phyai_batcher_plan(const phyai_batcher_config_t *cfg, uint32_t n, int32_t *slots, uint32_t *active_workers);
+
 /* Thread-local description of the last error of an operator entry point. */
 const char *phyai_op_last_error(void);
 

@@ -29,7 +29,9 @@ EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes
            "phyai_set_option", "phyai_launches_per_call", "phyai_last_error", "phyai_version",
            "phyai_suffix_attention", "phyai_suffix_attention_scratch_bytes", "phyai_op_last_error",
            "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity", "phyai_read_trace",
-           "phyai_pack_prefix_kv", "phyai_postprocess_actions", "phyai_adapter_last_error")
+           "phyai_pack_prefix_kv", "phyai_postprocess_actions", "phyai_adapter_last_error", "phyai_batcher_create",
+           "phyai_batcher_destroy", "phyai_batcher_submit", "phyai_batcher_next", "phyai_batcher_pending",
+           "phyai_batcher_plan")
 
 
 class PhyaiError(RuntimeError):
@@ -58,6 +60,10 @@ class AttentionDesc(C.Structure):
 class KvPackDesc(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("struct_size", "n_layers", "n_kv_heads", "head_dim", "elem_bytes", "batch",
                                           "p_max")]
+
+
+class BatcherConfig(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("struct_size", "max_batch", "n_workers", "local_batch")] + [("window_ms", C.c_double)]
 
 
 class WeightsStruct(C.Structure):
@@ -110,6 +116,14 @@ def load_library() -> C.CDLL:
     lib.phyai_postprocess_actions.argtypes = [_VP, C.c_uint32, C.c_uint32, C.c_uint32, _VP, _VP, C.c_float, C.c_float,
                                               C.c_uint32, C.c_uint32, _VP, _VP]
     lib.phyai_adapter_last_error.restype = C.c_char_p
+    lib.phyai_batcher_create.argtypes = [C.POINTER(BatcherConfig), C.POINTER(_VP)]
+    lib.phyai_batcher_destroy.argtypes = [_VP]
+    lib.phyai_batcher_destroy.restype = None
+    lib.phyai_batcher_submit.argtypes = [_VP, C.c_uint64]
+    lib.phyai_batcher_next.argtypes = [_VP, C.c_double, C.POINTER(C.c_uint64), C.POINTER(C.c_uint32)]
+    lib.phyai_batcher_pending.argtypes = [_VP]
+    lib.phyai_batcher_pending.restype = C.c_uint32
+    lib.phyai_batcher_plan.argtypes = [C.POINTER(BatcherConfig), C.c_uint32, C.POINTER(C.c_int32), C.POINTER(C.c_uint32)]
     _lib = lib
     return lib
 
@@ -333,3 +347,53 @@ def postprocess_actions(x: torch.Tensor, q01: Optional[torch.Tensor], q99: Optio
     if st != OK:
         raise PhyaiError(st, lib.phyai_adapter_last_error().decode())
     return out
+
+
+class Batcher:
+    """Batching window of the data-parallel front-end (``phyai_batcher_*``): thread-safe queue; ``next`` returns the ids
+    of the batch that is due (possibly empty after ``timeout_ms``)."""
+
+    def __init__(self, max_batch: int, n_workers: int, local_batch: int, window_ms: float):
+        self.lib = load_library()
+        self.cfg = BatcherConfig(C.sizeof(BatcherConfig), max_batch, n_workers, local_batch, float(window_ms))
+        h = _VP()
+        st = self.lib.phyai_batcher_create(C.byref(self.cfg), C.byref(h))
+        if st != OK:
+            raise PhyaiError(st, "bad batcher configuration")
+        self._h = h
+
+    def submit(self, request_id: int):
+        self.lib.phyai_batcher_submit(self._h, int(request_id))
+
+    def pending(self) -> int:
+        return int(self.lib.phyai_batcher_pending(self._h))
+
+    def next(self, timeout_ms: float):
+        ids = (C.c_uint64 * self.cfg.max_batch)()
+        n = C.c_uint32()
+        st = self.lib.phyai_batcher_next(self._h, float(timeout_ms), ids, C.byref(n))
+        if st != OK:
+            raise PhyaiError(st, "phyai_batcher_next failed")
+        return [int(ids[i]) for i in range(n.value)]
+
+    def plan(self, n: int):
+        """(slots as a list of n_workers lists of local_batch indices, -1 = padding; number of workers with a request)"""
+        total = self.cfg.n_workers * self.cfg.local_batch
+        slots = (C.c_int32 * total)()
+        act = C.c_uint32()
+        st = self.lib.phyai_batcher_plan(C.byref(self.cfg), int(n), slots, C.byref(act))
+        if st != OK:
+            raise PhyaiError(st, "phyai_batcher_plan: n exceeds max_batch")
+        L = self.cfg.local_batch
+        return [[int(slots[w * L + j]) for j in range(L)] for w in range(self.cfg.n_workers)], int(act.value)
+
+    def close(self):
+        if self._h:
+            self.lib.phyai_batcher_destroy(self._h)
+            self._h = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()

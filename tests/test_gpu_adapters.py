@@ -79,3 +79,25 @@ def test_action_postprocessing_matches_oracle():
         np.testing.assert_allclose(got, ref, rtol=1e-6, atol=1e-6)
     got = binding.postprocess_actions(x.cuda(), None, None, clip=(-1.0, 1.0)).cpu().numpy()
     np.testing.assert_allclose(got, np.clip(x.numpy(), -1, 1), rtol=0, atol=1e-7)
+
+
+def test_frontend_worker_pads_the_local_batch_to_its_fixed_shape():
+    """One rank: three requests into a fixed local batch of four.  The padded slot runs as a request with an empty
+    prefix, its output is dropped; every real request matches the oracle."""
+    from oracle import expert_oracle as O
+    from paper_2608_03682_b200.frontend import DPFrontend, ExpertWorker
+    from tests.helpers import BAR, rel_err, small_bf16_config
+    cfg = small_bf16_config("pi0", max_batch=4, max_prefix_len=120)
+    W = synth.make_weights(cfg, 25, std=0.05)
+    reqs = [dict(prefix_kv=synth.make_prefix_kv(cfg, 25, p, b), state=synth.make_state(cfg, 25, b),
+                 noise=synth.make_noise(cfg, 25, b), n_steps=3) for b, p in enumerate([120, 0, 57])]
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        fe = DPFrontend(ExpertWorker(ex, cfg, 3), local_batch=4, window_ms=5.0)
+        ids = [fe.submit(r) for r in reqs]
+        out = fe.serve_round(timeout_ms=500.0)
+        assert sorted(out) == ids and fe.serve_round(timeout_ms=10.0) == {}
+        fe.close()
+    Wf = O.Weights(W)
+    for rid, r in zip(ids, reqs):
+        ref = O.denoise(cfg, Wf, r["prefix_kv"], r["prefix_kv"].shape[2], r["state"], r["noise"], 3)
+        assert rel_err(out[rid], ref) <= BAR["bf16"], (rid, rel_err(out[rid], ref))
