@@ -203,7 +203,14 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
  * key "slab_splits": 1..16 (default 8), the most k-ranges a residual projection of a single-token-tile call is
  * split into on the general kernel (partial sums are written as slabs and added in slab order: bit-reproducible).
  * key "b1_c_qkv" / "b1_c_o" / "b1_c_gu" / "b1_c_d": cluster size (k-ranges per channel tile, 1..8; 0 = choose) of
- * the four projections on the cluster split-K kernel.  key "trace": see phyai_read_trace.
+ * the four projections on the cluster split-K kernel.  key "use_b1_attention": 1 (default) lets those calls use
+ * the cluster tcgen05 attention kernel (head_dim 128 / 256, even head and group counts), 0 keeps the mma.sync
+ * cluster kernel.  key "use_w8_inkernel": 1 (default) streams PHYAI_DTYPE_FP8_E4M3 weights as bytes and decodes
+ * them inside the cluster GEMM, 0 reads the bf16 images made at create (bit-identical results, twice the bytes).
+ * key "use_state_cache": 1 (default) lets a block-causal expert (Sec. "adapters"; the state tokens see only the
+ * prefix and themselves, so their keys and values do not change over the steps) run its state tokens once per
+ * call and the loop on the action tokens only, 0 runs every suffix token in every step.
+ * key "trace": see phyai_read_trace.
  * key "wait_limit": iteration bound of the device-side waits on other agents' progress (testing).
  * Unknown key -> INVALID_ARG. */
 phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t value);
