@@ -88,12 +88,14 @@ struct phyai_expert {
   bool b1_ok = false;          // the cluster split-K GEMM path covers this expert's shapes
   int use_cluster_gemm = 1;
   int use_b1_attention = 1;
+  int use_b1_step = 1;         // single-tile calls: velocity head + Euler update + next embedding as one cluster kernel
   int use_state_cache = 1;     // block-causal experts: state token computed once per call (single-tile calls)
   __nv_bfloat16 *kr_st = nullptr, *vr_st = nullptr;   // [L][max 64 tokens worth of requests][Hkv][S][dh] suffix K / V per layer
   int use_w8_inkernel = 1;     // e4m3 experts: the cluster GEMM decodes byte blocks itself (0: bf16 images made at create)    // tcgen05 attention with the key range split over a cluster (few requests)
   int b1_c[4] = {0, 0, 0, 0};  // cluster sizes of the QKV / O / gate-up / down projections (0 = choose)
   float *ss_a = nullptr, *ss_b = nullptr;   // [D/128][64] partial sums of squares of h (after O / after down)
   unsigned long long* trace_buf = nullptr;
+  int trace_all_from = 0;                   // > 0: launches [from, from + 5) of a call trace every CTA
   unsigned long long* trace = nullptr;      // [TRACE_SLOTS][8] timer stamps of the traced launches of one call, or null
   int use_tc_attention = 1;
   int use_cluster_attention = 1;
@@ -323,6 +325,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
   };
 
   const int ss_n = D / 128;
+  int trace_cursor = 0;
   const bool use_w8 = h->use_w8_inkernel && !h->b_qkv.empty();
   auto b1_gemm = [&](B1Gemm g, int which, int Mloc) -> phyai_status_t {
     g.M = Mloc, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact, g.inv_D = 1.0f / (float)D, g.eps = d.eps;
@@ -332,7 +335,23 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     // 6.6 ms with 80 - 120.
     const int reserve = (which == 0 && b1_attn_b1) ? 8 * (d.Hq / 2) * batch : 0;
     int C = b1_pick_cluster(g.N / 128, g.K / 64, h->n_sm - reserve);
+    if (which == 0) {
+      // Fewer, longer k-ranges for the QKV projection (about six k-chunks per CTA): all of its CTAs then find a free SM
+      // while the previous layer's down projection still runs, and the reduce has fewer partials.  Measured on the
+      // pi0-shaped expert: 6.31 ms per chunk with 5 k-ranges (100 CTAs), 6.23 ms with 3 (60 CTAs).
+      const int c6 = (g.K / 64 + 5) / 6;
+      if (c6 >= 1 && c6 < C && b1_gemm_supported(g.N, g.K, c6, h->n_sm, true)) C = c6;
+    }
     if (h->b1_c[which] > 0 && b1_gemm_supported(g.N, g.K, h->b1_c[which], h->n_sm, which == 0)) C = h->b1_c[which];
+    if (h->trace && h->trace_all_from > 0) {
+      // every CTA of five consecutive launches stamps, one slot per CTA in launch order
+      g.trace = nullptr;
+      const int n_cta = C * (g.N / 128);
+      if (cnt >= h->trace_all_from && cnt < h->trace_all_from + 5 && trace_cursor + n_cta <= TRACE_SLOTS) {
+        g.trace = h->trace + (size_t)trace_cursor * TRACE_STAMPS, g.trace_all = 1;
+        trace_cursor += n_cta;
+      }
+    }
     cudaError_t e = launch_b1_gemm(h->status, g, C, st);
     if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "cluster GEMM launch failed: %s", cudaGetErrorString(e));
     ++cnt;
@@ -342,18 +361,19 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
   // One layer on the cluster path: QKV, attention, O, gate/up, down (five kernels; the norms are folded in).
   // `kv_only`: stop after the QKV projection (the state pass needs nothing but the last layer's key / value).
   const size_t kv_layer = (size_t)batch * d0.Hkv * d0.S * d0.dh;   // per-layer stride of the cached suffix K / V
-  auto b1_layer = [&](const Dims& dd, int Mloc, int k, int l, bool kv_only, __nv_bfloat16* kr, __nv_bfloat16* vr) -> phyai_status_t {
+  auto b1_layer = [&](const Dims& dd, int Mloc, int k, int l, bool kv_only, __nv_bfloat16* kr, __nv_bfloat16* vr,
+                      bool folded_first = false) -> phyai_status_t {
     const float *gain, *shift, *gate;
     site(k, 2 * l, &gain, &shift, &gate);
-    // ---- QKV: layer 0 reads a normalised tile; later layers read bf16(h * gain) and the partial sums of squares left
-    // by the previous layer's down projection
-    if (l == 0) {
+    // ---- QKV: layer 0 reads a normalised tile (or, `folded_first`, what the embedding kernels left); later layers
+    // read bf16(h * gain) and the partial sums of squares left by the previous layer's down projection
+    if (l == 0 && !folded_first) {
       launch_rmsnorm(h->status, h->h, gain, shift, nullptr, h->xn64, 64, Mloc, D, dd.eps, st);
       ++cnt;
     }
     B1Gemm q{};
     q.W = h->p_qkv[l], q.W8 = use_w8 ? h->b_qkv[l] : nullptr, q.X = h->xn64, q.N = dd.Nqkv, q.K = D, q.epi = B1_QKV, q.wscale = h->s_qkv[l];
-    if (l > 0) {
+    if (l > 0 || folded_first) {
       q.ss_part = h->ss_b, q.ss_n = ss_n;
       q.shift_row = h->ada ? t.shw_qkv + ((size_t)k * dd.L + l) * dd.Nqkv : nullptr;
     }
@@ -365,13 +385,13 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     cudaError_t e;
     if (b1_attn_b1)
       e = launch_attention_b1(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->wait_limit, st,
-                              (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
+                              (h->trace && !h->trace_all_from && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
     else if (b1_attn_tc)
       e = launch_attention_tc(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->order, h->wait_limit, st);
     else
       e = launch_attention_cluster(h->rq, h->status, h->qkv, h->rope, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch,
                                    h->wait_limit, st, nullptr,
-                                   (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
+                                   (h->trace && !h->trace_all_from && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
     if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
     ++cnt;
     // ---- O projection + residual; leaves the operands of the second norm
@@ -411,9 +431,47 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     for (int l = 0; l < d0.L; ++l)
       ST(b1_layer(dp, batch, 0, l, l + 1 == d0.L, h->kr_st + (size_t)l * kv_layer, h->vr_st + (size_t)l * kv_layer));
   }
+  // Single-tile calls: one cluster kernel per step boundary (velocity head and Euler update of step k - 1, embedding
+  // of step k), then for pi0 the MLP's second layer on the cluster GEMM, whose epilogue leaves layer 0's norm operands.
+  const bool b1_step = b1 && h->use_b1_step && h->tc && step_b1_supported(d, batch) && (h->ada || h->W2p);
+  auto step_kernel = [&](int k, bool first, bool last) -> phyai_status_t {
+    StepB1 p{};
+    p.rq = h->rq, p.batch = batch, p.S = d.S, p.H = d.H, p.ns = d.ns, p.A = d.A, p.D = D, p.M = M, p.eps = d.eps;
+    p.wait_limit = h->wait_limit, p.first = first, p.last = last, p.h_in = h->h, p.Wout = h->Wout, p.bout = h->bout, p.dt = dt;
+    if (!first) {
+      const float* gate_unused;
+      site(k - 1, 2 * d.L, &p.gain_f, &p.shift_f, &gate_unused);
+    }
+    p.ada = h->ada ? 1 : 0, p.Wc = h->Wc, p.state_tok = h->state_tok;
+    if (!last) {
+      if (h->ada) {
+        const float *shift0, *gate0;
+        site(k, 0, &p.gain_next, &shift0, &gate0);
+        p.bias = h->bcfold, p.h_out = h->h, p.xn_out = h->xn64, p.ss_out = h->ss_b;
+      } else {
+        p.bias = t.tb + (size_t)k * D, p.u = h->m64;
+      }
+    }
+    p.trace = (h->trace && !h->trace_all_from && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr;
+    cudaError_t e = launch_step_b1(h->status, p, st);
+    if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "step kernel launch failed: %s", cudaGetErrorString(e));
+    ++cnt;
+    return PHYAI_OK;
+  };
   for (int k = 0; k < n; ++k) {
     // ---- suffix embedding ----
-    if (!h->ada) {
+    if (b1_step) {
+      ST(step_kernel(k, k == 0, false));
+      if (!h->ada) {
+        B1Gemm e{};
+        e.W = h->W2p, e.X = h->m64, e.N = D, e.K = D, e.epi = B1_RESID, e.h = h->h, e.ldh = D;
+        e.bias = h->b2, e.state_tok = h->state_tok, e.ns = d.ns, e.S = d.S;
+        const float *shift0, *gate0;
+        site(k, 0, &e.gain_next, &shift0, &gate0);
+        e.xn_out = h->xn64, e.ss_out = h->ss_b;
+        ST(b1_gemm(e, 1, M));
+      }
+    } else if (!h->ada) {
       launch_embed_pi0(h->rq, h->status, h->Wc, t.tb + (size_t)k * D, h->state_tok, h->h, h->u_f, h->u_t, h->Mpad, d,
                        batch, st);
       ++cnt;
@@ -443,7 +501,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       site(k, 2 * l, &gain, &shift, &gate);
       if (b1) {
         ST(b1_layer(d, M, k, l, false, cache_state ? h->kr_st + (size_t)l * kv_layer : h->kr_big,
-                    cache_state ? h->vr_st + (size_t)l * kv_layer : h->vr_big));
+                    cache_state ? h->vr_st + (size_t)l * kv_layer : h->vr_big, b1_step));
         continue;
       }
       launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs());
@@ -541,6 +599,10 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       }
     }
     // ---- final norm, velocity head, Euler update ----
+    if (b1_step) {
+      if (k + 1 == n) ST(step_kernel(n, false, true));
+      continue;
+    }
     const float *gain, *shift, *gate;
     site(k, 2 * d.L, &gain, &shift, &gate);
     if (pending_slabs) {
@@ -1042,6 +1104,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     h->graphs.clear();
     return PHYAI_OK;
   }
+  if (!strcmp(key, "use_b1_step")) {
+    h->use_b1_step = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
   if (!strcmp(key, "use_state_cache")) {
     h->use_state_cache = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
@@ -1081,6 +1149,14 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     }
     if (!h->trace_buf) ST(h->alloc(&h->trace_buf, (size_t)TRACE_SLOTS * TRACE_STAMPS, true));
     h->trace = h->trace_buf;
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "trace_all_from")) {
+    if (value < 0 || value >= TRACE_SLOTS) return fail(PHYAI_ERR_INVALID_ARG, "trace_all_from out of range");
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    h->trace_all_from = (int)value;
+    if (h->trace_buf) CU(cudaMemset(h->trace_buf, 0, (size_t)TRACE_SLOTS * TRACE_STAMPS * sizeof(unsigned long long)));
     return PHYAI_OK;
   }
   if (!strcmp(key, "wait_limit")) {

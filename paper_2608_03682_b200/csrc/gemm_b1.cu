@@ -96,7 +96,11 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
   const uint32_t slot = (uint32_t)tpc_max * ROWB;
 
   pdl_launch_dependents();
-  unsigned long long* tr = (g.trace && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) ? g.trace : nullptr;
+  unsigned long long* tr = nullptr;
+  if (g.trace && tid == 0) {
+    if (g.trace_all) tr = g.trace + (size_t)(blockIdx.y * gridDim.x + blockIdx.x) * 16;   // every CTA, one slot each
+    else if (blockIdx.x == 0 && blockIdx.y == 0) tr = g.trace;
+  }
   trace_stamp(tr, 0);
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t region = (uint32_t)max(g.nk_max * STAGE, 64 * ROWB);
@@ -235,6 +239,18 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     }
   }
   float4 hpre[2];
+  // B1_RESID: what the projection output is added to -- the residual stream, or (MLP second layer) the bias / the state
+  // token's embedding
+  auto is_state_row = [&](int tok) -> bool { return g.bias && (tok % g.S) < g.ns; };
+  auto old_of = [&](int tok) -> float4 {
+    const int n = tile * 128 + lane * 4;
+    if (g.bias) {
+      const int b = tok / g.S;
+      return (tok - b * g.S) < g.ns ? __ldg(reinterpret_cast<const float4*>(g.state_tok + (size_t)b * g.N + n))
+                                    : __ldg(reinterpret_cast<const float4*>(g.bias + n));
+    }
+    return *reinterpret_cast<const float4*>(g.h + (size_t)tok * g.ldh + n);
+  };
   if (warp != 1) {
     if (tid == 255) suppress = status_set(status) ? 1 : 0;
     if (tid >= 64 && tid < 128) {
@@ -253,7 +269,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     for (int u = 0; u < 2; ++u) {
       const int tl = warp + 8 * u;
       hpre[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (tl < ntok) hpre[u] = *reinterpret_cast<const float4*>(g.h + (size_t)(tok_lo + tl) * g.ldh + tile * 128 + lane * 4);
+      if (tl < ntok) hpre[u] = old_of(tok_lo + tl);
     }
   }
 
@@ -414,8 +430,9 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
       auto token = [&](int tl, bool have_old, float4 old) {
         const int tok = tok_lo + tl, n = n0 + lane * 4;
         float* hp = g.h + (size_t)tok * g.ldh + n;
-        if (!have_old) old = *reinterpret_cast<const float4*>(hp);
-        const float4 a = sum4(tl, lane * 4);
+        if (!have_old) old = old_of(tok);
+        float4 a = sum4(tl, lane * 4);
+        if (is_state_row(tok)) a = make_float4(0.f, 0.f, 0.f, 0.f);
         float4 hv;
         hv.x = old.x + gate4.x * (a.x * sc_tab[lane * 4]), hv.y = old.y + gate4.y * (a.y * sc_tab[lane * 4 + 1]);
         hv.z = old.z + gate4.z * (a.z * sc_tab[lane * 4 + 2]), hv.w = old.w + gate4.w * (a.w * sc_tab[lane * 4 + 3]);
@@ -485,7 +502,7 @@ int b1_pick_cluster(int tiles, int KC, int n_sm) {
 // A projection fits when its k-steps per CTA stay resident (<= MAXK) and the cluster has at most one CTA per SM.
 bool b1_gemm_supported(int N, int K, int C, int n_sm, bool qkv) {
   if (N % 128 || K % 64 || C < 1 || C > 8 || C > K / 64) return false;
-  if ((N / 128) * C > n_sm) return false;
+  if ((N / 128) * C > 2 * n_sm) return false;
   const int nk = (K / 64 + C - 1) / C;
   return nk <= MAXK && b1_smem(nk, C, qkv) <= B1_SMEM_MAX;
 }

@@ -235,10 +235,45 @@ struct B1Gemm {
   const float* gain_next;
   __nv_bfloat16* xn_out;
   float* ss_out;
+  // B1_RESID as the second layer of the pi0 action / time MLP: with `bias` set, h is written, not updated --
+  // h[token][n] = bias[n] + scale[n] * acc for action rows, h = state_tok[request][n] for the first `ns` rows of every
+  // request's S suffix rows (the state tokens, whose embedding does not pass through the MLP)
+  const float* bias;
+  const float* state_tok;
+  int ns;
   unsigned wait_limit;
+  int trace_all;               // every CTA stamps, into slot (linear CTA index) of `trace`
   unsigned long long* trace;   // 16-entry slot of this launch or null: start, set-up done, dependency resolved, MMAs
                                // complete, partials received, epilogue done, cluster released, (SM id)
 };
+// ---- step boundary of the single-tile loop (step_b1.cu): velocity head + Euler update of step k - 1, suffix embedding
+// of step k, one cluster of D / 128 CTAs -----------------------------------------------------------------------------
+struct StepB1 {
+  const Request* rq;
+  int batch, S, H, ns, A, D, M;   // M = batch * S token rows (<= 64)
+  float eps;
+  int first, last;                // first: no head (the actions are the noise); last: no embedding
+  const float* h_in;              // [M][D] residual stream after the last layer
+  const float* gain_f;            // final norm: gain (1 + gamma or 1 + scale) and shift or null
+  const float* shift_f;
+  const float* Wout;              // [D][A]
+  const float* bout;              // [A]
+  float dt;
+  int ada;                        // 0: pi0 (u = swish(x Wc + bias) -> bf16 tile), 1: pi0.5 (h = x Wc + bias, + norm operands)
+  const float* Wc;                // [A][D]
+  const float* bias;              // [D]
+  const float* state_tok;         // [batch][D]
+  __nv_bfloat16* u;               // pi0: tiled [D/64][64][64], row = token row
+  float* h_out;                   // pi0.5: [M][D]
+  const float* gain_next;         // pi0.5: gain of the first norm of layer 0
+  __nv_bfloat16* xn_out;          // pi0.5: bf16(h * gain_next), tiled
+  float* ss_out;                  // pi0.5: [D/128][64] partial sums of squares
+  unsigned wait_limit;
+  unsigned long long* trace;      // 16-entry slot or null: start, constants fetched, dependency resolved, slice
+                                  // staged, partial formed, partials received, embedding stored
+};
+bool step_b1_supported(const Dims& d, int batch);
+cudaError_t launch_step_b1(int* status, const StepB1& p, cudaStream_t st);
 int b1_pick_cluster(int tiles, int KC, int n_sm);
 bool b1_gemm_supported(int N, int K, int C, int n_sm, bool qkv);
 cudaError_t launch_b1_gemm(int* status, const B1Gemm& g, int C, cudaStream_t st);
