@@ -62,6 +62,7 @@ struct AttnArgs {
   float* slab;               // [Hq][rows][D]
   size_t slab_stride;        // rows * D
   int D;
+  int trace_all;             // every CTA stamps, into slot (linear CTA index) of `trace`
   unsigned long long* trace; // cluster kernel: 16-entry slot or null: start, set-up done, Q acquired, tiles done, partials
                              // received, output written, cluster released
 };

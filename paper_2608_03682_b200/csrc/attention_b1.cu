@@ -71,10 +71,13 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   const int S = d.S;                                      // query rows per head
   const int Sk = d.Sk > 0 ? d.Sk : d.S;                   // the request's own (suffix) keys that exist ...
   const int Sk_stride = d.Sk_stride > 0 ? d.Sk_stride : d.S;   // ... and their row pitch per kv head
-  const bool tracer = tid == 0 && rank == 0 && hp == 0 && b == 0;
+  // tracing: one CTA of the launch, or (trace_all) every CTA into the slot of its linear index
+  const bool tcta = a.trace && (a.trace_all || (rank == 0 && hp == 0 && b == 0));
+  unsigned long long* const trp = a.trace_all ? a.trace + (size_t)((b * gridDim.y + hp) * gridDim.x + rank) * 16 : a.trace;
+  const bool tracer = tid == 0 && tcta;
 
   pdl_launch_dependents();
-  if (tracer) trace_stamp(a.trace, 0);
+  if (tracer) trace_stamp(trp, 0);
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t Ks = base, Vs = base + L::TILE;
@@ -116,10 +119,10 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     if (lane == 0) suppress = status_set(a.status) ? 1 : 0;
     for (int t = 0; t < T; ++t) {
-      const bool trm = lane == 0 && rank == 0 && hp == 0 && b == 0 && t == 0;
+      const bool trm = lane == 0 && tcta && t == 0;
       group_sync<BAR_QK, 288>();              // the K / V tile (and Q) are in shared memory
       tc_fence_after();
-      if (trm) trace_stamp(a.trace, 14);
+      if (trm) trace_stamp(trp, 14);
 #pragma unroll
       for (int kk = 0; kk < DH / 16; ++kk) {
         const uint64_t db = make_desc(Ks + (uint32_t)(kk >> 2) * L::BLOCK + (uint32_t)(kk & 3) * 32);
@@ -128,7 +131,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
       }
       if (elect_one()) umma_commit(smem_u32(&s_full));
       __syncwarp();
-      if (trm) trace_stamp(a.trace, 15);
+      if (trm) trace_stamp(trp, 15);
       group_sync<BAR_P, 288>();               // P is in tensor memory
       tc_fence_after();
 #pragma unroll
@@ -152,7 +155,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     const int hl = row >> 6, i = row & 63;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     const bool lead = warp == 5 && lane == 0;
-    const bool tr2 = lead && rank == 0 && hp == 0 && b == 0;
+    const bool tr2 = lead && tcta;
     float m = -INFINITY, l = 0.f;             // running maximum (log2 units) and sum
     // ---- loader state (group 1) ----
     const bool is_v = warp >= 2;
@@ -190,7 +193,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     if (g == 1 && T > 0) issue(0, true);      // constants of the call: ahead of the dependency wait
     if (g == 1) cp_async_commit();
     pdl_wait();
-    if (tr2) trace_stamp(a.trace, 1);
+    if (tr2) trace_stamp(trp, 1);
     if (T > 0) {
       if (g == 1) {
         issue(0, false);
@@ -212,11 +215,11 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
       cp_async_commit();
       cp_async_wait<0>();                                          // (group 1: its tile rows as well)
       fence_async_smem();                                          // generic-proxy writes, read next by the tensor core
-      if (tr2) trace_stamp(a.trace, 10);
+      if (tr2) trace_stamp(trp, 10);
       named_arrive<BAR_QK, 288>();
     }
 
-    if (tr2) trace_stamp(a.trace, 2);
+    if (tr2) trace_stamp(trp, 2);
     const bool causal_row = d.block_causal && d.ns && i == 0;
     for (int t = 0; t < T; ++t) {
       const uint32_t ph = (uint32_t)t & 1u;
@@ -240,7 +243,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
       tc_fence_after();
       // (the last logits exist: the Q tile is dead and the receive area free -- see the cluster barrier ahead of the push)
       if (t == T - 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-      if (tr2) trace_stamp(a.trace, 11);
+      if (tr2) trace_stamp(trp, 11);
       const int k0 = key_lo + t * KB;
       // the visible key columns of this row form a prefix of the tile: the keys that exist, and for the state-token row
       // under the block-causal mask only up to its own key (key P)
@@ -294,7 +297,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
       group_sync<BAR_ROWS, 256>();            // (the other half row's sum is visible)
       l = l * corr + (xsum[0][row] + xsum[1][row]);
       m = m_new;
-      if (tr2) trace_stamp(a.trace, 7);
+      if (tr2) trace_stamp(trp, 7);
     }
     if (T == 0) {
       if (g == 1) cp_async_wait<0>();
@@ -304,7 +307,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     if (T > 0 && warp == 5) mbar_wait_drain(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, wc);
     group_sync<BAR_ROWS, 256>();
     tc_fence_after();
-    if (tr2) trace_stamp(a.trace, 3);
+    if (tr2) trace_stamp(trp, 3);
     {
       const int c = i >> 3, il = i & 7, n_c = max(0, min(8, S - c * 8));
       const bool wr = i < S;
@@ -334,7 +337,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     }
     tc_fence_before();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the bulk-copy engine
-    if (tr2) trace_stamp(a.trace, 12);
+    if (tr2) trace_stamp(trp, 12);
     group_sync<BAR_ROWS, 256>();
     // ---- every owner gets its block of my partial: one bulk copy over distributed shared memory -------------------
     // (first: every peer has moved its Q out of its receive area; all of them arrived long ago)
@@ -363,7 +366,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   // same, i.e. once every copy out of its own staging area has completed.  Arriving now and waiting at the very end
   // hides the skew between the CTAs behind the merge.
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  if (tracer) trace_stamp(a.trace, 4);
+  if (tracer) trace_stamp(trp, 4);
 
   // ---- merge my rows: the 8 partials in rank order, normalise, store as the output projection's activation tile ----
   const bool store = !*reinterpret_cast<volatile int*>(&suppress) && !*reinterpret_cast<volatile int*>(&abort_flag) &&
@@ -415,9 +418,9 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
           make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]), pack_bf16(acc[6], acc[7]));
     }
   }
-  if (tracer) trace_stamp(a.trace, 5);
+  if (tracer) trace_stamp(trp, 5);
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-  if (tracer) trace_stamp(a.trace, 6);
+  if (tracer) trace_stamp(trp, 6);
   if (warp == 4) {
     tc_fence_after();
     tmem_dealloc(tmem_base, COLS);
@@ -453,10 +456,10 @@ bool attention_b1_supported(const Dims& d) {
 
 cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, unsigned wait_limit, cudaStream_t st, unsigned long long* trace) {
+                                int batch, unsigned wait_limit, cudaStream_t st, unsigned long long* trace, int trace_all) {
   AttnArgs a{};
   a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
-  a.num_splits = 8, a.d = d, a.wait_limit = wait_limit, a.trace = trace;
+  a.num_splits = 8, a.d = d, a.wait_limit = wait_limit, a.trace = trace, a.trace_all = trace_all;
   return d.dh == 256 ? launch_one<256>(a, batch, st) : launch_one<128>(a, batch, st);
 }
 

@@ -383,9 +383,17 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     if (kv_only) return PHYAI_OK;
     // ---- attention -> bf16 tile of the output projection
     cudaError_t e;
-    if (b1_attn_b1)
-      e = launch_attention_b1(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->wait_limit, st,
-                              (h->trace && !h->trace_all_from && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr);
+    if (b1_attn_b1) {
+      unsigned long long* atr = (h->trace && !h->trace_all_from && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr;
+      int all = 0;
+      const int n_cta = 8 * (dd.Hq / 2) * batch;
+      if (h->trace && h->trace_all_from > 0 && cnt >= h->trace_all_from && cnt < h->trace_all_from + 5 &&
+          trace_cursor + n_cta <= TRACE_SLOTS) {
+        atr = h->trace + (size_t)trace_cursor * TRACE_STAMPS, all = 1;
+        trace_cursor += n_cta;
+      }
+      e = launch_attention_b1(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->wait_limit, st, atr, all);
+    }
     else if (b1_attn_tc)
       e = launch_attention_tc(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->order, h->wait_limit, st);
     else

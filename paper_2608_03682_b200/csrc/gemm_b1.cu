@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
   __shared__ __align__(8) uint64_t bar_accum, bar_recv;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, suppress, acc_ok, recv_ok;
-  __shared__ float rstd_tab[64], sc_tab[128], sh_tab[128];
+  __shared__ __align__(16) float rstd_tab[64], sc_tab[128], sh_tab[128];
   __shared__ int2 tok_tab[64];     // QKV: (rotary position, request * 64 + suffix row) of every token
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31, tid = threadIdx.x;
@@ -354,7 +354,15 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     return a;
   };
   // accumulator value -> projection output: weight scale, the folded norm's per-token factor, the folded shift row
-  auto fin = [&](float a, int ch, float r) -> float { return fmaf(a * sc_tab[ch], r, sh_tab[ch]); };
+  // (eight consecutive channels at a time: the tables are read as 16-byte vectors; no shift table without a shift)
+  const bool has_shift = g.shift_row != nullptr;
+  auto fin8 = [&](float (&x)[8], int ch, float r) {
+    const float4 s0 = *reinterpret_cast<const float4*>(sc_tab + ch), s1 = *reinterpret_cast<const float4*>(sc_tab + ch + 4);
+    float4 h0 = make_float4(0.f, 0.f, 0.f, 0.f), h1 = h0;
+    if (has_shift) h0 = *reinterpret_cast<const float4*>(sh_tab + ch), h1 = *reinterpret_cast<const float4*>(sh_tab + ch + 4);
+    x[0] = fmaf(x[0] * s0.x, r, h0.x), x[1] = fmaf(x[1] * s0.y, r, h0.y), x[2] = fmaf(x[2] * s0.z, r, h0.z), x[3] = fmaf(x[3] * s0.w, r, h0.w);
+    x[4] = fmaf(x[4] * s1.x, r, h1.x), x[5] = fmaf(x[5] * s1.y, r, h1.y), x[6] = fmaf(x[6] * s1.z, r, h1.z), x[7] = fmaf(x[7] * s1.w, r, h1.w);
+  };
 
   if (store) {
     if (EPI == B1_QKV) {
@@ -372,8 +380,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
           float lo[8], hi[8];
           *reinterpret_cast<float4*>(lo) = sum4(tl, j0), *reinterpret_cast<float4*>(lo + 4) = sum4(tl, j0 + 4);
           *reinterpret_cast<float4*>(hi) = sum4(tl, 64 + j0), *reinterpret_cast<float4*>(hi + 4) = sum4(tl, 64 + j0 + 4);
-#pragma unroll
-          for (int u = 0; u < 8; ++u) lo[u] = fin(lo[u], j0 + u, r), hi[u] = fin(hi[u], 64 + j0 + u, r);
+          fin8(lo, j0, r), fin8(hi, 64 + j0, r);
           if (g.rope) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -401,8 +408,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
           const float r = rstd_tab[tok_lo + tl];
           float x[8];
           *reinterpret_cast<float4*>(x) = sum4(tl, j0), *reinterpret_cast<float4*>(x + 4) = sum4(tl, j0 + 4);
-#pragma unroll
-          for (int u = 0; u < 8; ++u) x[u] = fin(x[u], j0 + u, r);
+          fin8(x, j0, r);
           const int b = e.y >> 6, i = e.y & 63;
           *reinterpret_cast<uint4*>(g.vr + ((size_t)(b * g.Hkv + head) * g.Sk_stride + g.koff + i) * g.dh + coff + j0) =
               make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
@@ -417,9 +423,10 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
         float gt[8], up[8];
         *reinterpret_cast<float4*>(gt) = sum4(tl, j0), *reinterpret_cast<float4*>(gt + 4) = sum4(tl, j0 + 4);
         *reinterpret_cast<float4*>(up) = sum4(tl, 64 + j0), *reinterpret_cast<float4*>(up + 4) = sum4(tl, 64 + j0 + 4);
+        fin8(gt, j0, r), fin8(up, 64 + j0, r);
         float m[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) m[u] = gelu_fast(fin(gt[u], j0 + u, r), g.gelu_exact) * fin(up[u], 64 + j0 + u, r);
+        for (int u = 0; u < 8; ++u) m[u] = gelu_fast(gt[u], g.gelu_exact) * up[u];
         *reinterpret_cast<uint4*>(g.out_tiled + ((size_t)tile * 64 + tok) * 64 + ((c8 ^ (tok & 7)) << 3)) =
             make_uint4(pack2(m[0], m[1]), pack2(m[2], m[3]), pack2(m[4], m[5]), pack2(m[6], m[7]));
       }
@@ -434,8 +441,9 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
         float4 a = sum4(tl, lane * 4);
         if (is_state_row(tok)) a = make_float4(0.f, 0.f, 0.f, 0.f);
         float4 hv;
-        hv.x = old.x + gate4.x * (a.x * sc_tab[lane * 4]), hv.y = old.y + gate4.y * (a.y * sc_tab[lane * 4 + 1]);
-        hv.z = old.z + gate4.z * (a.z * sc_tab[lane * 4 + 2]), hv.w = old.w + gate4.w * (a.w * sc_tab[lane * 4 + 3]);
+        const float4 sc = *reinterpret_cast<const float4*>(sc_tab + lane * 4);
+        hv.x = old.x + gate4.x * (a.x * sc.x), hv.y = old.y + gate4.y * (a.y * sc.y);
+        hv.z = old.z + gate4.z * (a.z * sc.z), hv.w = old.w + gate4.w * (a.w * sc.w);
         *reinterpret_cast<float4*>(hp) = hv;
         if (g.xn_out) {
           *reinterpret_cast<uint2*>(g.xn_out + tiled_index(tok, n, 64)) =

@@ -159,7 +159,8 @@ cudaError_t launch_attention_cluster(const Request* rq, int* status, const float
 bool attention_b1_supported(const Dims& d);
 cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, unsigned wait_limit, cudaStream_t st, unsigned long long* trace = nullptr);
+                                int batch, unsigned wait_limit, cudaStream_t st, unsigned long long* trace = nullptr,
+                                int trace_all = 0);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
                                 int batch, const int* order, unsigned wait_limit, cudaStream_t st);
