@@ -35,6 +35,8 @@ constexpr int W_BYTES = 128 * 128;     // one weight block: 128 out channels x 6
 constexpr int X_BYTES = 64 * 128;      // one activation block: 64 tokens x 64 k
 constexpr int STAGE = W_BYTES + X_BYTES;
 constexpr int MAXK = 8;                // k-steps per CTA, all resident (8 x 24 KB + the 32 KB receive area fit one SM)
+constexpr int NT = 512, NW = NT / 32;   // threads / warps of a CTA: the epilogues are chains of dependent instructions per
+                                        // thread, so more threads with less work each finish sooner
 constexpr int ROWB = 128 * 4;          // one token row of a partial: 128 channels fp32
 constexpr size_t B1_SMEM_MAX = 227 * 1024 - 2048;   // dynamic shared memory limit: the opt-in maximum less the static part
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
@@ -76,7 +78,7 @@ __device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t& lo, uint3
 }
 
 template <int EPI, bool W8>
-__global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g) {
+__global__ void __launch_bounds__(NT, 1) k_gemm_b1(int* status, const B1Gemm g) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[MAXK];
   __shared__ __align__(8) uint64_t bar_w8[MAXK];       // e4m3 weights: the byte blocks have landed
@@ -129,7 +131,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
 
   // ---- before the dependency wait: weights (constants) and per-channel constants ------------------------------
   if (lane == 0) {
-    for (int s = warp; s < nk; s += 8) {
+    for (int s = warp; s < nk; s += NW) {
       if (W8) {
         // one byte per weight: the 8 KB block lands in the upper half of the stage's 16 KB operand slot
         const uint32_t full = smem_u32(&bar_w8[s]);
@@ -181,7 +183,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     if (rot_tile && g.rope) {
       const int nn = n0 < Nq ? n0 : n0 - Nq;
       const int t64 = (nn % g.dh) >> 7;
-      for (int idx = tid; idx < ntok * 32; idx += 256) {
+      for (int idx = tid; idx < ntok * 32; idx += NT) {
         const int tl = idx >> 5, c = idx & 31;
         const int pos = tok_tab[tok_lo + tl].x;
         const float4 v = __ldg(reinterpret_cast<const float4*>(g.rope + (size_t)pos * (g.dh >> 1) + t64 * 64) + c);
@@ -193,29 +195,28 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
   }
   if (W8) {
     // e4m3 -> bf16 in place, ahead of the dependency wait where the weights arrive early (they are constants): every
-    // thread first takes its 32 bytes of every stage into registers (row = tid / 2, four 8-byte chunks), then, after
-    // a barrier, writes them back as 64 bytes of the swizzled K-major bf16 image the MMA reads.  The per-channel
+    // thread first takes its 16 bytes of every stage into registers (row = tid / 4, two 8-byte chunks), then, after
+    // a barrier, writes them back as 32 bytes of the swizzled K-major bf16 image the MMA reads.  The per-channel
     // scale stays in the epilogue.
     if (warp == 0)
       for (int s = 0; s < nk; ++s) mbar_wait_drain(smem_u32(&bar_w8[s]), 0u, wc);
     __syncthreads();
     trace_stamp(tr, 9);
-    uint4 raw[MAXK][2];
-    const int r = tid >> 1, hc = (tid & 1) * 4;
+    uint4 raw[MAXK];
+    const int r = tid >> 2, hc = (tid & 3) * 2;       // row, first of my two 8-code chunks
 #pragma unroll
     for (int s = 0; s < MAXK; ++s)
       if (s < nk) {
         const uint32_t src = tiles + (uint32_t)s * STAGE + W_BYTES / 2 + (uint32_t)r * 64 + (uint32_t)hc * 8;
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(raw[s][0].x), "=r"(raw[s][0].y), "=r"(raw[s][0].z), "=r"(raw[s][0].w) : "r"(src) : "memory");
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(raw[s][1].x), "=r"(raw[s][1].y), "=r"(raw[s][1].z), "=r"(raw[s][1].w) : "r"(src + 16) : "memory");
+        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(raw[s].x), "=r"(raw[s].y), "=r"(raw[s].z), "=r"(raw[s].w) : "r"(src) : "memory");
       }
     __syncthreads();
 #pragma unroll
     for (int s = 0; s < MAXK; ++s)
       if (s < nk) {
-        const uint32_t words[8] = {raw[s][0].x, raw[s][0].y, raw[s][0].z, raw[s][0].w, raw[s][1].x, raw[s][1].y, raw[s][1].z, raw[s][1].w};
+        const uint32_t words[4] = {raw[s].x, raw[s].y, raw[s].z, raw[s].w};
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {       // chunk hc + c: 8 codes = words[2c], words[2c + 1]
+        for (int c = 0; c < 2; ++c) {       // chunk hc + c: 8 codes = words[2c], words[2c + 1]
           uint32_t o0, o1, o2, o3;
           e4m3x4_to_bf16x4(words[2 * c], o0, o1);
           e4m3x4_to_bf16x4(words[2 * c + 1], o2, o3);
@@ -231,7 +232,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
   trace_stamp(tr, 2);
   // ---- after it: activations, the status word, per-token factors (nothing the MMA warp has to wait for) -----------
   if (lane == 0) {
-    for (int s = (warp + 4) & 7; s < nk; s += 8) {
+    for (int s = (warp + 4) & (NW - 1); s < nk; s += NW) {
       const uint32_t full = smem_u32(&bar_full[s]);
       mbar_expect_tx(full, X_BYTES);
       bulk_g2s(tiles + (uint32_t)s * STAGE + W_BYTES, reinterpret_cast<const uint8_t*>(g.X) + (size_t)(kc_begin + s) * X_BYTES,
@@ -252,7 +253,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     return *reinterpret_cast<const float4*>(g.h + (size_t)tok * g.ldh + n);
   };
   if (warp != 1) {
-    if (tid == 255) suppress = status_set(status) ? 1 : 0;
+    if (tid == NT - 1) suppress = status_set(status) ? 1 : 0;
     if (tid >= 64 && tid < 128) {
       const int t = tid - 64;
       float r = 1.0f;
@@ -267,7 +268,7 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
   if (EPI == B1_RESID) {
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
-      const int tl = warp + 8 * u;
+      const int tl = warp + NW * u;
       hpre[u] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (tl < ntok) hpre[u] = old_of(tok_lo + tl);
     }
@@ -299,18 +300,19 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
 
   // ---- accumulator -> staging [token][channel] (the operand stages are free: every MMA has completed) -------------
   {
-    const int q = warp & 3, hf = warp >> 2;
-    if (hf * 32 < M) {
-      float v[32];
+    // warp (q, cg): TMEM lanes 32 q .. + 31 (channels), columns 16 cg .. + 15 (tokens)
+    const int q = warp & 3, cg = warp >> 2;
+    if (cg * 16 < M) {
+      float v[16];
       if (nk > 0) {
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(hf * 32), v);
+        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cg * 16), v);
       } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = 0.f;
+        for (int j = 0; j < 16; ++j) v[j] = 0.f;
       }
-      const uint32_t dst = stage + (uint32_t)(hf * 32) * ROWB + (uint32_t)(q * 32 + lane) * 4;
+      const uint32_t dst = stage + (uint32_t)(cg * 16) * ROWB + (uint32_t)(q * 32 + lane) * 4;
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
+      for (int j = 0; j < 16; ++j)
         asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst + (uint32_t)j * ROWB), "f"(v[j]) : "memory");
     }
   }
@@ -354,14 +356,13 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
     return a;
   };
   // accumulator value -> projection output: weight scale, the folded norm's per-token factor, the folded shift row
-  // (eight consecutive channels at a time: the tables are read as 16-byte vectors; no shift table without a shift)
+  // (four consecutive channels at a time: the tables are read as 16-byte vectors; no shift table without a shift)
   const bool has_shift = g.shift_row != nullptr;
-  auto fin8 = [&](float (&x)[8], int ch, float r) {
-    const float4 s0 = *reinterpret_cast<const float4*>(sc_tab + ch), s1 = *reinterpret_cast<const float4*>(sc_tab + ch + 4);
-    float4 h0 = make_float4(0.f, 0.f, 0.f, 0.f), h1 = h0;
-    if (has_shift) h0 = *reinterpret_cast<const float4*>(sh_tab + ch), h1 = *reinterpret_cast<const float4*>(sh_tab + ch + 4);
-    x[0] = fmaf(x[0] * s0.x, r, h0.x), x[1] = fmaf(x[1] * s0.y, r, h0.y), x[2] = fmaf(x[2] * s0.z, r, h0.z), x[3] = fmaf(x[3] * s0.w, r, h0.w);
-    x[4] = fmaf(x[4] * s1.x, r, h1.x), x[5] = fmaf(x[5] * s1.y, r, h1.y), x[6] = fmaf(x[6] * s1.z, r, h1.z), x[7] = fmaf(x[7] * s1.w, r, h1.w);
+  auto fin4 = [&](float4 x, int ch, float r) -> float4 {
+    const float4 s0 = *reinterpret_cast<const float4*>(sc_tab + ch);
+    float4 h0 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (has_shift) h0 = *reinterpret_cast<const float4*>(sh_tab + ch);
+    return make_float4(fmaf(x.x * s0.x, r, h0.x), fmaf(x.y * s0.y, r, h0.y), fmaf(x.z * s0.z, r, h0.z), fmaf(x.w * s0.w, r, h0.w));
   };
 
   if (store) {
@@ -373,62 +374,51 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
         __nv_bfloat16* base = isq ? g.qr : g.kr;
         const int H = isq ? g.Hq : g.Hkv;
         const float osc = isq ? rsqrtf((float)g.dh) : 1.0f;
-        for (int it = tid; it < ntok * 8; it += 256) {
-          const int tl = it >> 3, j0 = (it & 7) * 8;
+        // an item: four channels of the head's first half and their four rotary partners, of one token
+        for (int it = tid; it < ntok * 16; it += NT) {
+          const int tl = it >> 4, j0 = (it & 15) * 4;
           const int2 e = tok_tab[tok_lo + tl];
           const float r = rstd_tab[tok_lo + tl];
-          float lo[8], hi[8];
-          *reinterpret_cast<float4*>(lo) = sum4(tl, j0), *reinterpret_cast<float4*>(lo + 4) = sum4(tl, j0 + 4);
-          *reinterpret_cast<float4*>(hi) = sum4(tl, 64 + j0), *reinterpret_cast<float4*>(hi + 4) = sum4(tl, 64 + j0 + 4);
-          fin8(lo, j0, r), fin8(hi, 64 + j0, r);
+          float4 lo = fin4(sum4(tl, j0), j0, r), hi = fin4(sum4(tl, 64 + j0), 64 + j0, r);
           if (g.rope) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const float4 c = lds4(rope_s + (uint32_t)(tl * 64 + j0 + 2 * u) * 8);   // (cos, sin) of channels 2u, 2u + 1
-              const float l0 = lo[2 * u], h0 = hi[2 * u], l1 = lo[2 * u + 1], h1 = hi[2 * u + 1];
-              lo[2 * u] = l0 * c.x - h0 * c.y, hi[2 * u] = h0 * c.x + l0 * c.y;
-              lo[2 * u + 1] = l1 * c.z - h1 * c.w, hi[2 * u + 1] = h1 * c.z + l1 * c.w;
-            }
+            const float4 c0 = lds4(rope_s + (uint32_t)(tl * 64 + j0) * 8);       // (cos, sin) of channels j0, j0 + 1
+            const float4 c1 = lds4(rope_s + (uint32_t)(tl * 64 + j0 + 2) * 8);   // ... j0 + 2, j0 + 3
+            const float4 l = lo, h = hi;
+            lo.x = l.x * c0.x - h.x * c0.y, hi.x = h.x * c0.x + l.x * c0.y;
+            lo.y = l.y * c0.z - h.y * c0.w, hi.y = h.y * c0.z + l.y * c0.w;
+            lo.z = l.z * c1.x - h.z * c1.y, hi.z = h.z * c1.x + l.z * c1.y;
+            lo.w = l.w * c1.z - h.w * c1.w, hi.w = h.w * c1.z + l.w * c1.w;
           }
           const int b = e.y >> 6, i = e.y & 63;
           // (q: one row per query token; k: the request's key rows, query row i at key row koff + i)
           __nv_bfloat16* dst = base + (isq ? ((size_t)(b * H + head) * g.S + i) : ((size_t)(b * H + head) * g.Sk_stride + g.koff + i)) * g.dh +
                                t64 * 64 + j0;
-          *reinterpret_cast<uint4*>(dst) = make_uint4(pack2(lo[0] * osc, lo[1] * osc), pack2(lo[2] * osc, lo[3] * osc),
-                                                      pack2(lo[4] * osc, lo[5] * osc), pack2(lo[6] * osc, lo[7] * osc));
-          *reinterpret_cast<uint4*>(dst + half) = make_uint4(pack2(hi[0] * osc, hi[1] * osc), pack2(hi[2] * osc, hi[3] * osc),
-                                                             pack2(hi[4] * osc, hi[5] * osc), pack2(hi[6] * osc, hi[7] * osc));
+          *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(lo.x * osc, lo.y * osc), pack2(lo.z * osc, lo.w * osc));
+          *reinterpret_cast<uint2*>(dst + half) = make_uint2(pack2(hi.x * osc, hi.y * osc), pack2(hi.z * osc, hi.w * osc));
         }
       } else {
         const int nn = n0 - Nq - Nk;
         const int head = nn / g.dh, coff = nn - head * g.dh;       // 128 consecutive v channels
-        for (int it = tid; it < ntok * 16; it += 256) {
-          const int tl = it >> 4, j0 = (it & 15) * 8;
+        for (int it = tid; it < ntok * 32; it += NT) {
+          const int tl = it >> 5, j0 = (it & 31) * 4;
           const int2 e = tok_tab[tok_lo + tl];
-          const float r = rstd_tab[tok_lo + tl];
-          float x[8];
-          *reinterpret_cast<float4*>(x) = sum4(tl, j0), *reinterpret_cast<float4*>(x + 4) = sum4(tl, j0 + 4);
-          fin8(x, j0, r);
+          const float4 x = fin4(sum4(tl, j0), j0, rstd_tab[tok_lo + tl]);
           const int b = e.y >> 6, i = e.y & 63;
-          *reinterpret_cast<uint4*>(g.vr + ((size_t)(b * g.Hkv + head) * g.Sk_stride + g.koff + i) * g.dh + coff + j0) =
-              make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
+          *reinterpret_cast<uint2*>(g.vr + ((size_t)(b * g.Hkv + head) * g.Sk_stride + g.koff + i) * g.dh + coff + j0) =
+              make_uint2(pack2(x.x, x.y), pack2(x.z, x.w));
         }
       }
     } else if (EPI == B1_GEGLU) {
       // rows 0..63 = gate channels f0 .. f0 + 63, rows 64..127 = the matching up channels; the result is one 64-wide
-      // k-chunk (`tile`) of the down projection's activation tile, written as its swizzled 16-byte groups
-      for (int it = tid; it < ntok * 8; it += 256) {
-        const int tl = it >> 3, c8 = it & 7, j0 = c8 * 8, tok = tok_lo + tl;
+      // k-chunk (`tile`) of the down projection's activation tile, written as halves of its swizzled 16-byte groups
+      for (int it = tid; it < ntok * 16; it += NT) {
+        const int tl = it >> 4, c4 = it & 15, j0 = c4 * 4, tok = tok_lo + tl;
         const float r = rstd_tab[tok];
-        float gt[8], up[8];
-        *reinterpret_cast<float4*>(gt) = sum4(tl, j0), *reinterpret_cast<float4*>(gt + 4) = sum4(tl, j0 + 4);
-        *reinterpret_cast<float4*>(up) = sum4(tl, 64 + j0), *reinterpret_cast<float4*>(up + 4) = sum4(tl, 64 + j0 + 4);
-        fin8(gt, j0, r), fin8(up, 64 + j0, r);
-        float m[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) m[u] = gelu_fast(gt[u], g.gelu_exact) * up[u];
-        *reinterpret_cast<uint4*>(g.out_tiled + ((size_t)tile * 64 + tok) * 64 + ((c8 ^ (tok & 7)) << 3)) =
-            make_uint4(pack2(m[0], m[1]), pack2(m[2], m[3]), pack2(m[4], m[5]), pack2(m[6], m[7]));
+        const float4 gt = fin4(sum4(tl, j0), j0, r), up = fin4(sum4(tl, 64 + j0), 64 + j0, r);
+        const float m0 = gelu_fast(gt.x, g.gelu_exact) * up.x, m1 = gelu_fast(gt.y, g.gelu_exact) * up.y;
+        const float m2 = gelu_fast(gt.z, g.gelu_exact) * up.z, m3 = gelu_fast(gt.w, g.gelu_exact) * up.w;
+        *reinterpret_cast<uint2*>(g.out_tiled + ((size_t)tile * 64 + tok) * 64 + (((c4 >> 1) ^ (tok & 7)) << 3) + (c4 & 1) * 4) =
+            make_uint2(pack2(m0, m1), pack2(m2, m3));
       }
     } else {
       // gated residual: one warp per token, a lane takes four channels.  h stays fp32; the next projection's
@@ -453,8 +443,8 @@ __global__ void __launch_bounds__(256, 1) k_gemm_b1(int* status, const B1Gemm g)
         }
       };
       if (warp < ntok) token(warp, true, hpre[0]);           // (the first two rows of a warp were requested early)
-      if (warp + 8 < ntok) token(warp + 8, true, hpre[1]);
-      for (int tl = warp + 16; tl < ntok; tl += 8) token(tl, false, make_float4(0.f, 0.f, 0.f, 0.f));
+      if (warp + NW < ntok) token(warp + NW, true, hpre[1]);
+      for (int tl = warp + 2 * NW; tl < ntok; tl += NW) token(tl, false, make_float4(0.f, 0.f, 0.f, 0.f));
     }
   }
   trace_stamp(tr, 5);
@@ -486,7 +476,7 @@ cudaError_t launch_one(int* status, const B1Gemm& g, int C, cudaStream_t st) {
     once.done();
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(C, g.N / 128, 1), cfg.blockDim = dim3(256), cfg.dynamicSmemBytes = b1_smem(g.nk_max, C, g.epi == B1_QKV), cfg.stream = st;
+  cfg.gridDim = dim3(C, g.N / 128, 1), cfg.blockDim = dim3(NT), cfg.dynamicSmemBytes = b1_smem(g.nk_max, C, g.epi == B1_QKV), cfg.stream = st;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = C, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
