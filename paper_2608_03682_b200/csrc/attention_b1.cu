@@ -39,25 +39,28 @@ __device__ __forceinline__ void named_arrive() {
   asm volatile("bar.arrive %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
 }
 
-template <int DH>
+template <int DH, int HPC>
 struct B1Layout {
   static constexpr int BLOCK = KB * 128;                     // one 64-channel block of a K / V tile: 128 keys x 128 bytes
   static constexpr int TILE = (DH / 64) * BLOCK;             // a K or V tile
   static constexpr int PITCH = DH * 2 + 16;                  // bf16 partial row, padded against bank conflicts
-  static constexpr int SLOT = 2 * 8 * (PITCH + 8);           // one owner's block: 2 heads x 8 rows of (O row | max, sum)
-  static constexpr size_t SMEM = 1024 + 2 * (size_t)TILE + 8 * (size_t)SLOT;
+  static constexpr int SLOT = HPC * 8 * (PITCH + 16);        // one owner's block: HPC heads x 8 rows of O, then their (max, sum)
+                                                             // in 16-byte entries (a bulk copy moves multiples of 16 bytes)
+  static constexpr int QTILE = 128 * DH * 2;                 // the Q operand (128 rows; with one head the upper 64 idle)
+  static constexpr int RECV = 8 * SLOT > QTILE ? 8 * SLOT : QTILE;   // receive area of the merge; first holds Q
+  static constexpr size_t SMEM = 1024 + 2 * (size_t)TILE + (size_t)RECV;
 };
 
-template <int DH>
+template <int DH, int HPC>
 __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
-  using L = B1Layout<DH>;
+  using L = B1Layout<DH, HPC>;
   constexpr int COLS = 512;                   // S / P at columns [0, 128), O at [128, 128 + DH)
   constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KB >> 3) << 17) | ((128u >> 4) << 24);
   constexpr uint32_t IDESC_PV =
       (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((128u >> 4) << 24);
 
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t s_full, pv_done, mrg_bar;
+  __shared__ __align__(8) uint64_t s_full, pv_done, mrg_bar, q_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, suppress, mrg_ok;
   __shared__ float wtab[16][8];               // merge: weight of partial s for each of my (up to 2 x 8) rows
@@ -66,7 +69,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   const Dims& d = a.d;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rank = blockIdx.x, hp = blockIdx.y, b = blockIdx.z;
-  const int head0 = hp * 2;
+  const int head0 = hp * HPC;
   const int hk = head0 / (d.Hq / d.Hkv);
   const int S = d.S;                                      // query rows per head
   const int Sk = d.Sk > 0 ? d.Sk : d.S;                   // the request's own (suffix) keys that exist ...
@@ -85,12 +88,13 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   const uint32_t recv = base + 2 * L::TILE;               // [8 sources][SLOT]
   const uint32_t Qs = recv;                               // Q tile (2 heads x 64 rows), until the logits exist
   const int n_me = max(0, min(8, S - rank * 8));          // suffix rows (per head) this CTA owns in the merge
-  const uint32_t my_bytes = (uint32_t)(2 * n_me * (L::PITCH + 8));
+  const uint32_t my_bytes = (uint32_t)(HPC * n_me * (L::PITCH + 16));
 
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(smem_u32(&s_full), 1), mbar_init(smem_u32(&pv_done), 1);
     mbar_init(smem_u32(&mrg_bar), 1);
+    mbar_init(smem_u32(&q_bar), 8);
     if (n_me > 0) mbar_expect_tx(smem_u32(&mrg_bar), 7u * my_bytes);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -108,9 +112,12 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   // (the request block is written before the captured loop starts: safe to read ahead of the dependency wait)
   const Request r = *a.rq;
   const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
-  const int Kt = P + Sk;                                  // keys of this request: prefix, then its own suffix
-  const int key_lo = (int)(((long long)Kt * rank) / 8), key_hi = (int)(((long long)Kt * (rank + 1)) / 8);
-  const int T = (key_hi - key_lo + KB - 1) / KB;          // tiles of this CTA (1 unless P + S > 1024; 0 for an empty range)
+  // Keys of this CTA: an eighth of the prefix keys followed by an eighth of the request's own (suffix) keys -- the
+  // suffix rows only exist after the dependency wait, so every CTA fetches its share of them then, not one CTA all.
+  const int pre_lo = (int)(((long long)P * rank) / 8), n_pre = (int)(((long long)P * (rank + 1)) / 8) - pre_lo;
+  const int suf_lo = (Sk * rank) / 8, n_suf = (Sk * (rank + 1)) / 8 - suf_lo;
+  const int n_keys = n_pre + n_suf;
+  const int T = (n_keys + KB - 1) / KB;                   // tiles of this CTA (1 unless P + S > 1024; 0 for an empty range)
 
   if (warp == 4) {
     // =========================== MMA issuer ======================================================================
@@ -120,7 +127,8 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     if (lane == 0) suppress = status_set(a.status) ? 1 : 0;
     for (int t = 0; t < T; ++t) {
       const bool trm = lane == 0 && tcta && t == 0;
-      group_sync<BAR_QK, 288>();              // the K / V tile (and Q) are in shared memory
+      group_sync<BAR_QK, 288>();              // the K / V tile is in shared memory
+      if (t == 0) mbar_wait_drain(smem_u32(&q_bar), 0u, wc);    // ... and the Q tile (one bulk copy)
       tc_fence_after();
       if (trm) trace_stamp(trp, 14);
 #pragma unroll
@@ -172,17 +180,16 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     // in the rows past the range (their probabilities are 0, but 0 x stale shared memory must stay 0; K rows past the
     // range only produce logits that the softmax masks).  The loops walk exactly the rows they copy.
     auto issue = [&](int t, bool prefix) {
-      const int k0 = key_lo + t * KB;
-      const int np = max(0, min(KB, min(P, key_hi) - k0));   // prefix rows of the tile
-      const int nv = max(0, min(KB, key_hi - k0));           // rows that exist
+      const int np = max(0, min(KB, n_pre - t * KB));        // prefix rows of the tile
+      const int nv = max(0, min(KB, n_keys - t * KB));       // rows that exist
       if (prefix) {
-        const uint8_t* src = Gp + (size_t)(k0 + r0) * kv_stride;
+        const uint8_t* src = Gp + (size_t)(pre_lo + t * KB + r0) * kv_stride;
         for (int row2 = r0; row2 < np; row2 += RSTEP, src += (size_t)RSTEP * kv_stride)
           cp_async16(tile_base + (uint32_t)row2 * 128 + (uint32_t)(((lc & 7) ^ (row2 & 7)) << 4), src, 16u);
       } else {
         for (int row2 = np + r0; row2 < nv; row2 += RSTEP)
           cp_async16(tile_base + (uint32_t)row2 * 128 + (uint32_t)(((lc & 7) ^ (row2 & 7)) << 4),
-                     Gs + (size_t)(k0 + row2 - P) * (DH * 2), 16u);
+                     Gs + (size_t)(suf_lo + t * KB + row2 - n_pre) * (DH * 2), 16u);
         if (is_v)
           for (int row2 = nv + r0; row2 < KB; row2 += RSTEP)
             asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(tile_base + (uint32_t)row2 * 128 + (uint32_t)(((lc & 7) ^ (row2 & 7)) << 4)),
@@ -199,20 +206,27 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
         issue(0, false);
         cp_async_commit();
       }
-      // Q (already rotated, scaled bf16): coalesced 16-byte copies into the swizzled K-major block layout of an MMA A
-      // operand, in the receive area of the merge (idle until the peers push).  (One thread per row straight from
-      // global memory into tensor memory measured 3.3 us -- every load instruction of a warp touches 32 lines --,
-      // and via shared memory and tcgen05.st still 2.9 us.)
-      const uint8_t* qg = reinterpret_cast<const uint8_t*>(a.qr);
-      const int rt = warp < 4 ? tid : tid - 32;                    // 0..255 over the eight row warps
-#pragma unroll 4
-      for (int idx = rt; idx < 128 * CHUNKS; idx += 256) {
-        const int rw = idx / CHUNKS, cc = idx % CHUNKS, h2 = rw >> 6, i2 = rw & 63;
-        const bool ok = i2 < S;
-        cp_async16(Qs + (uint32_t)(cc >> 3) * L::BLOCK + (uint32_t)rw * 128 + (uint32_t)(((cc & 7) ^ (rw & 7)) << 4),
-                   qg + ((size_t)(b * d.Hq + head0 + h2) * S + (ok ? i2 : 0)) * (DH * 2) + (size_t)cc * 16, ok ? 16u : 0u);
+      // Q (rotated, scaled bf16) was written by the QKV projection as this kernel's operand tile: one bulk copy into the
+      // receive area of the merge (idle until the peers push).  (16-byte asynchronous copies by all row threads took
+      // 1.5 us for the 64 KB; one thread per row straight into tensor memory 3.3 us.)
+      // (an eighth per row warp: the copies of one warp complete one after the other, those of different warps overlap)
+      if (lane == 0) {
+        constexpr uint32_t QBYTES = 128u * DH * 2u;
+        const int part = warp < 4 ? warp : warp - 1;
+        const uint8_t* qt = reinterpret_cast<const uint8_t*>(a.qr) + (size_t)(b * (d.Hq >> 1) + (head0 >> 1)) * QBYTES;
+        if (HPC == 2) {
+          constexpr uint32_t QPART = QBYTES / 8;
+          mbar_expect_tx(smem_u32(&q_bar), QPART);
+          bulk_g2s(Qs + (uint32_t)part * QPART, qt + (size_t)part * QPART, QPART, smem_u32(&q_bar));
+        } else {
+          // one head: its 64 rows of every 64-channel block of the pair's tile (the other 64 rows of the MMA idle)
+          constexpr uint32_t PARTS = 8 / (DH / 64), QPART = 8192u / PARTS;      // pieces per block, bytes per piece
+          const uint32_t kb = (uint32_t)part / PARTS, pc = (uint32_t)part % PARTS;
+          mbar_expect_tx(smem_u32(&q_bar), QPART);
+          bulk_g2s(Qs + kb * (uint32_t)L::BLOCK + pc * QPART, qt + (size_t)kb * L::BLOCK + (size_t)(head0 & 1) * 8192 + pc * QPART, QPART,
+                   smem_u32(&q_bar));
+        }
       }
-      cp_async_commit();
       cp_async_wait<0>();                                          // (group 1: its tile rows as well)
       fence_async_smem();                                          // generic-proxy writes, read next by the tensor core
       if (tr2) trace_stamp(trp, 10);
@@ -244,11 +258,10 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
       // (the last logits exist: the Q tile is dead and the receive area free -- see the cluster barrier ahead of the push)
       if (t == T - 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
       if (tr2) trace_stamp(trp, 11);
-      const int k0 = key_lo + t * KB;
       // the visible key columns of this row form a prefix of the tile: the keys that exist, and for the state-token row
-      // under the block-causal mask only up to its own key (key P)
-      int nvis = min(KB, key_hi - k0);
-      if (causal_row) nvis = min(nvis, max(0, P + 1 - k0));
+      // under the block-causal mask only the prefix keys and its own key (suffix key 0, in the first CTA's range)
+      int nvis = min(KB, n_keys - t * KB);
+      if (causal_row) nvis = min(nvis, max(0, n_pre + (suf_lo == 0 && n_suf > 0 ? 1 : 0) - t * KB));
       nvis -= g * 64;                         // relative to this thread's 64 columns
       float s[64];
       tmem_ld64(tmem_s + lane_addr + (uint32_t)(g * 64), s);
@@ -310,7 +323,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
     if (tr2) trace_stamp(trp, 3);
     {
       const int c = i >> 3, il = i & 7, n_c = max(0, min(8, S - c * 8));
-      const bool wr = i < S;
+      const bool wr = hl < HPC && i < S;
       const uint32_t blk = stg + (uint32_t)c * L::SLOT;
       const uint32_t rowp = blk + (uint32_t)(hl * n_c + il) * L::PITCH;
 #pragma unroll 1
@@ -331,7 +344,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
         }
       }
       if (wr && g == 0)
-        asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(blk + (uint32_t)(2 * n_c) * L::PITCH + (uint32_t)(hl * n_c + il) * 8),
+        asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(blk + (uint32_t)(HPC * n_c) * L::PITCH + (uint32_t)(hl * n_c + il) * 16),
                      "f"(m), "f"(l)
                      : "memory");
     }
@@ -351,7 +364,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
         asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(recv + (uint32_t)rank * L::SLOT), "r"(peer));
         asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(&mrg_bar)), "r"(peer));
         asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                     "r"(stg + (uint32_t)peer * L::SLOT), "r"((uint32_t)(2 * n_c * (L::PITCH + 8))), "r"(bar)
+                     "r"(stg + (uint32_t)peer * L::SLOT), "r"((uint32_t)(HPC * n_c * (L::PITCH + 16))), "r"(bar)
                      : "memory");
       }
     }
@@ -372,12 +385,12 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   const bool store = !*reinterpret_cast<volatile int*>(&suppress) && !*reinterpret_cast<volatile int*>(&abort_flag) &&
                      (n_me == 0 || *reinterpret_cast<volatile int*>(&mrg_ok));
   // per row: weight of every partial, already divided by the combined sum
-  if (tid < 2 * n_me) {
+  if (tid < HPC * n_me) {
     float ms[8], ls[8], mm = -INFINITY;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
       const uint32_t blk = (s == rank) ? stg + (uint32_t)rank * L::SLOT : recv + (uint32_t)s * L::SLOT;
-      asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(ms[s]), "=f"(ls[s]) : "r"(blk + (uint32_t)(2 * n_me) * L::PITCH + (uint32_t)tid * 8) : "memory");
+      asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(ms[s]), "=f"(ls[s]) : "r"(blk + (uint32_t)(HPC * n_me) * L::PITCH + (uint32_t)tid * 16) : "memory");
       mm = fmaxf(mm, ms[s]);
     }
     float w[8], ll = 0.f;
@@ -393,7 +406,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   __syncthreads();
   if (store) {
     constexpr int CH = DH / 8;                // 16-byte chunks (8 columns) per row
-    for (int idx = tid; idx < 2 * n_me * CH; idx += 288) {
+    for (int idx = tid; idx < HPC * n_me * CH; idx += 288) {
       const int rr = idx / CH, ch = idx - rr * CH;       // rr = hl * n_me + il
       const int hl = rr >= n_me ? 1 : 0, il = rr - hl * n_me;
       float acc[8];
@@ -428,23 +441,23 @@ __global__ void __launch_bounds__(288, 1) k_attn_b1(const AttnArgs a) {
   (void)base_ptr;
 }
 
-template <int DH>
+template <int DH, int HPC>
 cudaError_t launch_one(const AttnArgs& a, int batch, cudaStream_t st) {
   static PerDeviceOnce once;
   if (once.needed()) {
-    cudaError_t e = cudaFuncSetAttribute(k_attn_b1<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1Layout<DH>::SMEM);
+    cudaError_t e = cudaFuncSetAttribute(k_attn_b1<DH, HPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1Layout<DH, HPC>::SMEM);
     if (e != cudaSuccess) return e;
     once.done();
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(8, a.d.Hq / 2, batch), cfg.blockDim = dim3(288), cfg.dynamicSmemBytes = B1Layout<DH>::SMEM, cfg.stream = st;
+  cfg.gridDim = dim3(8, a.d.Hq / HPC, batch), cfg.blockDim = dim3(288), cfg.dynamicSmemBytes = B1Layout<DH, HPC>::SMEM, cfg.stream = st;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 8, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
   at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at, cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, k_attn_b1<DH>, a);
+  return cudaLaunchKernelEx(&cfg, k_attn_b1<DH, HPC>, a);
 }
 
 }  // namespace
@@ -454,13 +467,17 @@ bool attention_b1_supported(const Dims& d) {
   return (d.dh == 256 || d.dh == 128) && d.S <= 64 && d.Hq % 2 == 0 && (d.Hq / d.Hkv) % 2 == 0;
 }
 
-cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
+// CTAs of one launch with `hpc` (1 or 2) query heads per CTA
+int attention_b1_ctas(const Dims& d, int batch, int hpc) { return 8 * (d.Hq / hpc) * batch; }
+
+cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloat16* q_tiles, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, unsigned wait_limit, cudaStream_t st, unsigned long long* trace, int trace_all) {
+                                int batch, int hpc, unsigned wait_limit, cudaStream_t st, unsigned long long* trace, int trace_all) {
   AttnArgs a{};
-  a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
+  a.rq = rq, a.status = status, a.qr = q_tiles, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
   a.num_splits = 8, a.d = d, a.wait_limit = wait_limit, a.trace = trace, a.trace_all = trace_all;
-  return d.dh == 256 ? launch_one<256>(a, batch, st) : launch_one<128>(a, batch, st);
+  if (hpc == 1) return d.dh == 256 ? launch_one<256, 1>(a, batch, st) : launch_one<128, 1>(a, batch, st);
+  return d.dh == 256 ? launch_one<256, 2>(a, batch, st) : launch_one<128, 2>(a, batch, st);
 }
 
 }  // namespace phyai

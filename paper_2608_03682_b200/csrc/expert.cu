@@ -88,6 +88,7 @@ struct phyai_expert {
   bool b1_ok = false;          // the cluster split-K GEMM path covers this expert's shapes
   int use_cluster_gemm = 1;
   int use_b1_attention = 1;
+  int b1_attn_hpc = 0;         // query heads per CTA of the cluster attention kernel (0 = choose)
   int use_b1_step = 1;         // single-tile calls: velocity head + Euler update + next embedding as one cluster kernel
   int use_state_cache = 1;     // block-causal experts: state token computed once per call (single-tile calls)
   __nv_bfloat16 *kr_st = nullptr, *vr_st = nullptr;   // [L][max 64 tokens worth of requests][Hkv][S][dh] suffix K / V per layer
@@ -105,6 +106,7 @@ struct phyai_expert {
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
   __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
+  __nv_bfloat16* q_tiles = nullptr;   // cluster attention: q as [request][head pair][dh / 64][128 rows][64] swizzled tiles
   __nv_bfloat16 *qr_big = nullptr, *kr_big = nullptr, *vr_big = nullptr;   // rotated bf16 q / k / v of large batches
 
   Request* rq = nullptr;
@@ -281,7 +283,11 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
                           batch * (d0.Hq / 2) >= ATTN_TC_MIN_CTAS;
   const bool b1_attn_cluster = !b1_attn_tc && h->attn_mma && h->use_cluster_attention && batch * d0.Hq * 8 <= 2 * h->n_sm;
   const bool b1 = h->b1_ok && h->use_cluster_gemm && batch * d0.S <= 64 && (b1_attn_tc || b1_attn_cluster);
-  const bool b1_attn_b1 = !b1_attn_tc && h->use_b1_attention && attention_b1_supported(d0) && batch * (d0.Hq / 2) * 8 <= h->n_sm;
+  const bool b1_attn_b1 = !b1_attn_tc && h->use_b1_attention && h->q_tiles && attention_b1_supported(d0) && batch * (d0.Hq / 2) * 8 <= h->n_sm;
+  // one query head per CTA while the attention kernel then still leaves the QKV projection room beside it (the partial
+  // results that cross the cluster, the softmax rows and the Q tile of a CTA halve), else two heads per CTA
+  const int b1_hpc = (h->b1_attn_hpc == 1 || h->b1_attn_hpc == 2) ? h->b1_attn_hpc
+                                                                 : (attention_b1_ctas(d0, batch, 1) <= h->n_sm / 2 ? 1 : 2);
   const bool cache_state = b1 && b1_attn_b1 && h->kr_st && h->use_state_cache;
   Dims d = d0;
   if (cache_state) d.ns = 0, d.S = d0.H, d.block_causal = 0, d.Sk = d0.S, d.Sk_stride = d0.S, d.koff = 1;
@@ -333,7 +339,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     // The QKV projection leaves the SMs of the attention kernel free: that kernel then starts (and fetches its prefix
     // tiles) while the projection still runs.  Measured on the pi0-shaped expert: 7.6 ms per chunk with 140 CTAs,
     // 6.6 ms with 80 - 120.
-    const int reserve = (which == 0 && b1_attn_b1) ? 8 * (d.Hq / 2) * batch : 0;
+    const int reserve = (which == 0 && b1_attn_b1) ? attention_b1_ctas(d, batch, b1_hpc) : 0;
     int C = b1_pick_cluster(g.N / 128, g.K / 64, h->n_sm - reserve);
     if (which == 0) {
       // Fewer, longer k-ranges for the QKV projection (about six k-chunks per CTA): all of its CTAs then find a free SM
@@ -378,6 +384,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       q.shift_row = h->ada ? t.shw_qkv + ((size_t)k * dd.L + l) * dd.Nqkv : nullptr;
     }
     q.rq = h->rq, q.rope = h->rope, q.qr = h->qr_big, q.kr = kr, q.vr = vr;
+    q.q_tiles = b1_attn_b1 ? h->q_tiles : nullptr;
     q.S = dd.S, q.Hq = dd.Hq, q.Hkv = dd.Hkv, q.dh = dd.dh, q.Sk_stride = suffix_key_stride(dd), q.koff = dd.koff;
     ST(b1_gemm(q, 0, Mloc));
     if (kv_only) return PHYAI_OK;
@@ -386,13 +393,13 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     if (b1_attn_b1) {
       unsigned long long* atr = (h->trace && !h->trace_all_from && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr;
       int all = 0;
-      const int n_cta = 8 * (dd.Hq / 2) * batch;
+      const int n_cta = attention_b1_ctas(dd, batch, b1_hpc);
       if (h->trace && h->trace_all_from > 0 && cnt >= h->trace_all_from && cnt < h->trace_all_from + 5 &&
           trace_cursor + n_cta <= TRACE_SLOTS) {
         atr = h->trace + (size_t)trace_cursor * TRACE_STAMPS, all = 1;
         trace_cursor += n_cta;
       }
-      e = launch_attention_b1(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->wait_limit, st, atr, all);
+      e = launch_attention_b1(h->rq, h->status, h->q_tiles, kr, vr, l, h->attn64, 64, dd, batch, b1_hpc, h->wait_limit, st, atr, all);
     }
     else if (b1_attn_tc)
       e = launch_attention_tc(h->rq, h->status, h->qr_big, kr, vr, l, h->attn64, 64, dd, batch, h->order, h->wait_limit, st);
@@ -939,6 +946,8 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         ST(h->alloc(&h->m64, (size_t)64 * F, true));
         ST(h->alloc(&h->ss_a, (size_t)(D / 128) * 64, true));
         ST(h->alloc(&h->ss_b, (size_t)(D / 128) * 64, true));
+        if (attention_b1_supported(d) && d.Hq >= 2)   // q as operand tiles of the cluster attention kernel: up to 64 query rows
+          ST(h->alloc(&h->q_tiles, (size_t)64 * (d.Hq / 2) * 128 * d.dh, true));
         if (d.block_causal && d.ns && !ada) {
           // per-layer suffix K / V (key row 0 = the cached state token) for as many requests as fit one 64-token tile
           const size_t per_layer = (size_t)(64 / d.S > 0 ? 64 / d.S : 1) * d.Hkv * d.S * d.dh;
@@ -1108,6 +1117,13 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
   }
   if (!strcmp(key, "use_cluster_attention")) {
     h->use_cluster_attention = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "b1_attn_hpc")) {
+    if (value < 0 || value > 2) return fail(PHYAI_ERR_INVALID_ARG, "b1_attn_hpc is 0 (choose), 1 or 2");
+    h->b1_attn_hpc = (int)value;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

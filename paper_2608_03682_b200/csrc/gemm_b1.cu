@@ -390,11 +390,22 @@ __global__ void __launch_bounds__(NT, 1) k_gemm_b1(int* status, const B1Gemm g) 
             lo.w = l.w * c1.z - h.w * c1.w, hi.w = h.w * c1.z + l.w * c1.w;
           }
           const int b = e.y >> 6, i = e.y & 63;
-          // (q: one row per query token; k: the request's key rows, query row i at key row koff + i)
-          __nv_bfloat16* dst = base + (isq ? ((size_t)(b * H + head) * g.S + i) : ((size_t)(b * H + head) * g.Sk_stride + g.koff + i)) * g.dh +
-                               t64 * 64 + j0;
-          *reinterpret_cast<uint2*>(dst) = make_uint2(pack2(lo.x * osc, lo.y * osc), pack2(lo.z * osc, lo.w * osc));
-          *reinterpret_cast<uint2*>(dst + half) = make_uint2(pack2(hi.x * osc, hi.y * osc), pack2(hi.z * osc, hi.w * osc));
+          const uint2 vlo = make_uint2(pack2(lo.x * osc, lo.y * osc), pack2(lo.z * osc, lo.w * osc));
+          const uint2 vhi = make_uint2(pack2(hi.x * osc, hi.y * osc), pack2(hi.z * osc, hi.w * osc));
+          if (isq && g.q_tiles) {
+            // q as the attention kernel's operand tiles: per (request, head pair) dh / 64 blocks of [128 rows][64
+            // channels], row = 64 * (head & 1) + token, the 16-byte chunks of a 128-byte row XOR-swizzled by row & 7
+            const int rw = (head & 1) * 64 + i, c_lo = t64 * 64 + j0, c_hi = c_lo + half;
+            __nv_bfloat16* tb = g.q_tiles + (size_t)(b * (g.Hq >> 1) + (head >> 1)) * (size_t)(128 * g.dh);
+            *reinterpret_cast<uint2*>(tb + (size_t)(c_lo >> 6) * 8192 + rw * 64 + ((((c_lo & 63) >> 3) ^ (rw & 7)) << 3) + (c_lo & 7)) = vlo;
+            *reinterpret_cast<uint2*>(tb + (size_t)(c_hi >> 6) * 8192 + rw * 64 + ((((c_hi & 63) >> 3) ^ (rw & 7)) << 3) + (c_hi & 7)) = vhi;
+          } else {
+            // (q: one row per query token; k: the request's key rows, query row i at key row koff + i)
+            __nv_bfloat16* dst = base + (isq ? ((size_t)(b * H + head) * g.S + i) : ((size_t)(b * H + head) * g.Sk_stride + g.koff + i)) * g.dh +
+                                 t64 * 64 + j0;
+            *reinterpret_cast<uint2*>(dst) = vlo;
+            *reinterpret_cast<uint2*>(dst + half) = vhi;
+          }
         }
       } else {
         const int nn = n0 - Nq - Nk;

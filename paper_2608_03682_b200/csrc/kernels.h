@@ -157,10 +157,12 @@ cudaError_t launch_attention_cluster(const Request* rq, int* status, const float
                                      cudaStream_t st, const AttnOproj* op = nullptr, unsigned long long* trace = nullptr);
 // ---- tcgen05 attention for very few requests: key range split over a cluster of 8, two heads per CTA (attention_b1.cu)
 bool attention_b1_supported(const Dims& d);
-cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
+cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloat16* q_tiles, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, unsigned wait_limit, cudaStream_t st, unsigned long long* trace = nullptr,
+                                int batch, int hpc, unsigned wait_limit, cudaStream_t st, unsigned long long* trace = nullptr,
                                 int trace_all = 0);
+// CTAs of one launch with `hpc` (1 or 2) query heads per CTA
+int attention_b1_ctas(const Dims& d, int batch, int hpc);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
                                 int batch, const int* order, unsigned wait_limit, cudaStream_t st);
@@ -223,6 +225,7 @@ struct B1Gemm {
   const Request* rq;
   const float2* rope;
   __nv_bfloat16 *qr, *kr, *vr;
+  __nv_bfloat16* q_tiles;    // set: q goes out as the cluster attention kernel's operand tiles instead of rows (qr)
   int S, Hq, Hkv, dh;
   int Sk_stride, koff;       // key rows per (request, kv head) in kr / vr and the key row of query row 0 (see Dims)
   // B1_GEGLU: W holds gate and up interleaved in groups of 64 channels; output [N/128][64][64] tiled
