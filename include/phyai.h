@@ -207,9 +207,12 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
  * the cluster tcgen05 attention kernel (head_dim 128 / 256, even head and group counts), 0 keeps the mma.sync
  * cluster kernel.  key "use_w8_inkernel": 1 (default) streams PHYAI_DTYPE_FP8_E4M3 weights as bytes and decodes
  * them inside the cluster GEMM, 0 reads the bf16 images made at create (bit-identical results, twice the bytes).
- * key "use_state_cache": 1 (default) lets a block-causal expert (Sec. "adapters"; the state tokens see only the
- * prefix and themselves, so their keys and values do not change over the steps) run its state tokens once per
- * call and the loop on the action tokens only, 0 runs every suffix token in every step.
+ * key "use_state_cache": 1 lets a block-causal expert (Sec. "adapters"; the state tokens see only the prefix and
+ * themselves, so their keys and values do not change over the steps) run its state tokens once per call and the
+ * loop on the action tokens only; 0 (default) runs every suffix token in every step, which is faster as long as the
+ * state token does not cost a token tile of its own.
+ * key "b1_attn_hpc": query heads per CTA (1 or 2; 0 = choose) of the cluster attention kernel.  key "use_b1_step":
+ * 1 (default) runs the step boundary of those calls (velocity head, Euler update, next embedding) as one cluster kernel.
  * key "trace": see phyai_read_trace.
  * key "wait_limit": iteration bound of the device-side waits on other agents' progress (testing).
  * Unknown key -> INVALID_ARG. */

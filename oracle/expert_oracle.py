@@ -23,7 +23,9 @@ Pins (tests/test_oracle_*.py): zero velocity head returns the noise bit-exactly;
 closed form; brute-force attention in pure-Python loops; torch float64 library routines for
 rms_norm / gelu / silu / scaled_dot_product_attention; prefix permutation; NaN tail beyond
 prefix_len; sinusoid special values; RoPE relative-position property; hand-computed network
-with identity blocks; exhaustive e4m3 decode against ml_dtypes.
+with identity blocks; exhaustive e4m3 decode against ml_dtypes; e4m3 rounding against torch's
+float8_e4m3fn cast, all codes as fixed points, ties and saturation by hand; the W8A8 projection on
+inputs that are already on the e4m3 grid.
 Whole-network values: **parity unpinned** by any number printed in the paper (it prints none);
 they are covered by the composition of the pins above and by a second, differently structured
 transcription in the tests.
@@ -57,7 +59,7 @@ def decode_e4m3(codes: np.ndarray) -> np.ndarray:
 
 def to_f64(t) -> np.ndarray:
     """Stored tensor -> float64 array, exactly.  Accepts numpy arrays, torch tensors (f32/bf16)
-    and ``(codes_uint8[in,out], scales_f32[out])`` pairs of the W8A16 mode, which decode to
+    and ``(codes_uint8[in,out], scales_f32[out])`` pairs of the W8A16 / W8A8 modes, which decode to
     ``decode(code) * scale`` per output channel (column)."""
     if isinstance(t, tuple):
         codes, scales = t
@@ -68,6 +70,43 @@ def to_f64(t) -> np.ndarray:
     import torch  # storage container only
 
     return t.detach().to(torch.float64).cpu().numpy()
+
+
+def round_e4m3(y: np.ndarray) -> np.ndarray:
+    """Nearest OCP e4m3 "fn" value of every element, ties to the even mantissa, saturating at the
+    largest finite value 448 (the format has no infinities): the round-to-nearest of the quantization
+    paragraph applied to a value that is already divided by its scale.  Normal numbers 2^e (1 + m/8),
+    e in [-6, 8]; below 2^-6 the grid is uniform with step 2^-9 (subnormals)."""
+    y = np.asarray(y, dtype=F64)
+    a = np.minimum(np.abs(y), 448.0)
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.clip(e, -6.0, 8.0)
+    step = np.exp2(e - 3.0)                      # spacing of the grid in the binade of a
+    q = np.rint(a / step) * step                 # numpy.rint rounds halves to even
+    return np.sign(y) * np.minimum(q, 448.0)
+
+
+def quantize_rows_e4m3(x: np.ndarray):
+    """W8A8 activation quantization (quantization paragraph: the paper lists W8A8 among its
+    round-to-nearest modes; granularity and scale rule are a reading): every row (token) gets the scale
+    s = max|x| / 448 (1 for an all-zero row) and its elements become round_e4m3(x / s).  The decision is
+    taken in float32 -- the precision the device takes it in -- on the float32 rounding of x.  Returns
+    (codes' values as float64, scales as float64): the projection then computes (values @ Wq) * s."""
+    x32 = np.asarray(x, dtype=np.float32)
+    amax = np.max(np.abs(x32), axis=-1, keepdims=True)
+    s = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+    y = (x32 / s).astype(np.float32)
+    return round_e4m3(y.astype(F64)), s.astype(F64)
+
+
+def project(cfg, x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """x @ w for one of the seven large per-layer matrices; in the W8A8 mode through the per-token
+    e4m3 quantization of x (the weights are already the decoded e4m3 values times their scales)."""
+    if getattr(cfg, "dtype", "") == "w8a8e4m3":
+        q, s = quantize_rows_e4m3(x)
+        return (q @ w) * s
+    return x @ w
 
 
 # ----------------------------------------------------------------------------------------------
@@ -229,21 +268,21 @@ def velocity(cfg, W: Weights, prefix_kv: np.ndarray, prefix_len: int, state, x: 
             n1, g1 = norm_ada(h, c, W.layer("norm1", l), W.layer("norm1_b", l), cfg.rms_eps)
         else:
             n1, g1 = norm_plain(h, W.layer("norm1", l), cfg.rms_eps), 1.0
-        q = (n1 @ W.layer("wq", l)).reshape(S, Hq, dh)
-        ks = (n1 @ W.layer("wk", l)).reshape(S, Hkv, dh)
-        vs = (n1 @ W.layer("wv", l)).reshape(S, Hkv, dh)
+        q = project(cfg, n1, W.layer("wq", l)).reshape(S, Hq, dh)
+        ks = project(cfg, n1, W.layer("wk", l)).reshape(S, Hkv, dh)
+        vs = project(cfg, n1, W.layer("wv", l)).reshape(S, Hkv, dh)
         q = rope(q, pos, cfg.rope_theta)
         ks = rope(ks, pos, cfg.rope_theta)
         # attention over prefix (as given, K already rotated) and suffix
         o = attention(q, prefix_kv[l, 0, :P], prefix_kv[l, 1, :P], ks, vs, mask, Hq // Hkv)
-        h = h + g1 * (o.reshape(S, Hq * dh) @ W.layer("wo", l))
+        h = h + g1 * project(cfg, o.reshape(S, Hq * dh), W.layer("wo", l))
         # norm -> gate/up -> GeGLU -> down
         if ada:
             n2, g2 = norm_ada(h, c, W.layer("norm2", l), W.layer("norm2_b", l), cfg.rms_eps)
         else:
             n2, g2 = norm_plain(h, W.layer("norm2", l), cfg.rms_eps), 1.0
-        m = gelu(n2 @ W.layer("wgate", l), cfg.gelu_exact) * (n2 @ W.layer("wup", l))
-        h = h + g2 * (m @ W.layer("wdown", l))
+        m = gelu(project(cfg, n2, W.layer("wgate", l)), cfg.gelu_exact) * project(cfg, n2, W.layer("wup", l))
+        h = h + g2 * project(cfg, m, W.layer("wdown", l))
 
     if ada:
         nf, _ = norm_ada(h, c, W["final_norm"], W["final_norm_b"], cfg.rms_eps)

@@ -90,7 +90,8 @@ struct phyai_expert {
   int use_b1_attention = 1;
   int b1_attn_hpc = 0;         // query heads per CTA of the cluster attention kernel (0 = choose)
   int use_b1_step = 1;         // single-tile calls: velocity head + Euler update + next embedding as one cluster kernel
-  int use_state_cache = 1;     // block-causal experts: state token computed once per call (single-tile calls)
+  int use_state_cache = 0;     // block-causal experts: state token computed once per call (single-tile calls); exact, but at
+                               // one request the 18-layer state pass costs more than the 51st row it saves (measured)
   __nv_bfloat16 *kr_st = nullptr, *vr_st = nullptr;   // [L][max 64 tokens worth of requests][Hkv][S][dh] suffix K / V per layer
   int use_w8_inkernel = 1;     // e4m3 experts: the cluster GEMM decodes byte blocks itself (0: bf16 images made at create)    // tcgen05 attention with the key range split over a cluster (few requests)
   int b1_c[4] = {0, 0, 0, 0};  // cluster sizes of the QKV / O / gate-up / down projections (0 = choose)

@@ -44,7 +44,8 @@ class ExpertConfig:
     max_prefix_len: int
     max_batch: int = 1
     cond: str = "pi0"            # "pi0": time concatenated into the action MLP; "pi05": adaRMSNorm
-    dtype: str = "bf16"          # "f32" | "bf16" | "w8e4m3" (storage of weights and prefix KV)
+    dtype: str = "bf16"          # "f32" | "bf16" | "w8e4m3" | "w8a8e4m3" (storage of weights and prefix KV; the last
+                                 # also names the arithmetic of the seven large projections: e4m3 x e4m3)
     rms_eps: float = 1e-6
     rope_theta: float = 10000.0  # 0 disables RoPE
     time_min_period: float = 4e-3
@@ -172,14 +173,14 @@ def quantize_e4m3_columns(w: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
 def make_weights(cfg: ExpertConfig, cfg_id: int, std: float = 0.02) -> Dict[str, object]:
     """All weights of one expert, ~N(0, std) in float32, cast to the configuration's storage.
 
-    For ``dtype == "w8e4m3"`` the seven large per-layer matrices become ``(codes, scales)``
+    For ``dtype == "w8e4m3"`` / ``"w8a8e4m3"`` the seven large per-layer matrices become ``(codes, scales)``
     tuples and everything else is bfloat16."""
     rng = _rng(cfg_id, STREAM_WEIGHTS)
     W: Dict[str, object] = {}
     for name, shape in weight_shapes(cfg):
         master = _normal(rng, shape, std)
         base = name.split(".")[0]
-        if cfg.dtype == "w8e4m3" and base in BIG_MATS:
+        if cfg.dtype in ("w8e4m3", "w8a8e4m3") and base in BIG_MATS:
             W[name] = quantize_e4m3_columns(master)
         else:
             W[name] = _store(master, "f32" if cfg.dtype == "f32" else "bf16")
