@@ -59,6 +59,9 @@ def workload(name: str):
     if name.startswith("C5b"):
         b = int(name[3:])
         return synth.pi0_config(max_batch=b, dtype="w8e4m3", max_prefix_len=816), 5, b, [816] * b, 10
+    if name.startswith("C6b"):   # the C5 expert in the W8A8 mode: per-token e4m3 activations, FP8 tensor path
+        b = int(name[3:])
+        return synth.pi0_config(max_batch=b, dtype="w8a8e4m3", max_prefix_len=816), 5, b, [816] * b, 10
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -66,7 +69,7 @@ def algorithmic_cost(cfg, lens, n_steps):
     """Bytes that must cross HBM and FLOPs per chunk: every big weight once per Euler step, each
     request's prefix KV once per layer per step; activations and tables are cache resident."""
     D, F, L, S = cfg.width, cfg.mlp_dim, cfg.n_layers, cfg.suffix_len
-    wbytes = 1 if cfg.dtype == "w8e4m3" else (4 if cfg.dtype == "f32" else 2)
+    wbytes = 1 if cfg.dtype in ("w8e4m3", "w8a8e4m3") else (4 if cfg.dtype == "f32" else 2)
     ebytes = 4 if cfg.dtype == "f32" else 2
     nqkv = cfg.q_dim + 2 * cfg.kv_dim
     per_layer_params = D * nqkv + cfg.q_dim * D + 2 * D * F + F * D
@@ -197,6 +200,15 @@ def roofline_of(name, cfg, lens, n_steps, batch, ms_per_step, peaks):
                 "peak_source": f"{peaks['source']} copy bandwidth", "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": alg_bytes}
     achieved = alg_flops / secs / 1e12
+    if cfg.dtype == "w8a8e4m3":
+        # the linear layers (5/6 of the FLOPs) run on the FP8 tensor path: measured bf16 rate x the nominal FP8 : bf16
+        # ratio of 2; attention stays bf16, so this peak is an upper bound of what the loop can reach
+        pk = 2.0 * peaks["bf16_tflops_sustained"]
+        return {"bound": "tensor", "achieved": achieved, "peak": pk, "unit": "TFLOP/s", "frac": achieved / pk, "traffic": None,
+                "kernel": "whole captured loop (one graph launch = one batch of chunks)",
+                "peak_source": f"2 x {peaks['source']} sustained bf16 GEMM (nominal FP8 : bf16 ratio)",
+                "frac_of_bf16_sustained": achieved / peaks["bf16_tflops_sustained"],
+                "frac_of_nominal": achieved / (2.0 * NOMINAL_BF16_TFLOPS), "algorithmic_flops_per_launch": alg_flops}
     return {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
             "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
             "kernel": "whole captured loop (one graph launch = one batch of chunks)",
@@ -328,7 +340,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default=None,
-                    help="time one workload only (C1, C2, C3, C4, C5b1, C5b8, C5b64, C5b256); default: C2 as the headline "
+                    help="time one workload only (C1, C2, C3, C4, C5b1, C5b8, C5b64, C5b256, C6b8 ... C6b256: W8A8); default: C2 as the headline "
                          "plus every other configuration of the metric in the line's `workloads` map")
     ap.add_argument("--impl", default="phyai", choices=["phyai", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -444,6 +456,18 @@ def main():
             r5["roofline"] = roofline_of(name, c5, l5[:b5], n5, b5, r5["ms_per_step"], peaks)
             others[name] = r5
         e5.close()
+        torch.cuda.empty_cache()
+        # the same expert and requests in the W8A8 mode (FP8 tensor path)
+        c6, id6, _, l6, n6 = workload("C6b256")
+        e6 = make_expert(c6, id6)
+        for b6 in (8, 64, 256):
+            name = f"C6b{b6}"
+            r6 = run_workload(name, e6, c6, l6[:b6], n6, in5, Ko if b6 < 256 else min(Ko, 5), Wo, world, rank, local_rank,
+                              e2e=False)
+            r6["workload"], r6["steps"], r6["warmup"] = describe(name, c6, b6, l6[:b6], n6), Ko, Wo
+            r6["roofline"] = roofline_of(name, c6, l6[:b6], n6, b6, r6["ms_per_step"], peaks)
+            others[name] = r6
+        e6.close()
         del in5
         torch.cuda.empty_cache()
 

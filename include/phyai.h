@@ -50,9 +50,14 @@ typedef enum {
 typedef enum {
   PHYAI_F32 = 0,       /* everything float32; arithmetic in true fp32 (no TF32)                       */
   PHYAI_BF16 = 1,      /* weights and prefix KV bfloat16; bf16 tensor-core operands, fp32 accumulate   */
-  PHYAI_W8E4M3_A16 = 2 /* the seven large per-layer matrices as e4m3 bytes with one fp32 scale per
+  PHYAI_W8E4M3_A16 = 2, /* the seven large per-layer matrices as e4m3 bytes with one fp32 scale per
                           output channel (offline round-to-nearest, quantization paragraph); all other
                           tensors and the prefix KV bfloat16; activations bf16                        */
+  PHYAI_W8A8_E4M3 = 3  /* storage as PHYAI_W8E4M3_A16; in addition the input of each of the four large
+                          projections of a layer (fused QKV, attention output, gate / up, down) is
+                          quantised per token to e4m3 -- scale = max|x| / 448, codes round-to-nearest-even,
+                          saturating -- and the products run on the FP8 tensor path (quantization
+                          paragraph: W8A8).  Tensor path only; kernels of the general (any batch) family */
 } phyai_dtype_t;
 
 /* How the time t_k conditions the expert. */
@@ -345,6 +350,25 @@ phyai_status_t phyai_postprocess_actions(const float *x, uint32_t batch, uint32_
 
 /* Thread-local description of the last error of an adapter entry point. */
 const char *phyai_adapter_last_error(void);
+
+/*
+ * Stand-alone W8A8 projection (quantization paragraph: W8A8, round-to-nearest): the activation quantization kernel
+ * and the FP8 tensor-core GEMM that the PHYAI_W8A8_E4M3 loop uses, on one activation matrix.
+ *   s[m]    = max_k |x[m][k]| / 448   (1 for an all-zero row), float32
+ *   q[m][k] = e4m3 code nearest to x[m][k] / s[m] (ties to the even mantissa, saturating at +-448)
+ *   y[m][n] = s[m] * w_scales[n] * sum_k value(q[m][k]) * value(w_codes[k][n]),  fp32 accumulation
+ *   x_bf16        device bfloat16 [M][K] row-major (16-byte aligned)
+ *   w_codes       device uint8 (e4m3) [K][N] row-major;  w_scales device float32 [N]
+ *   y             device float32 [M][N]
+ *   x_codes_out   device uint8 [M][K] or NULL: the activation codes;  x_scales_out device float32 [M] or NULL
+ * 1 <= M <= 65536; K a multiple of 128, at most 4096; N a multiple of 128, at most 65536.  Allocates its temporaries,
+ * runs on `stream` and synchronises it before returning (a verification entry point, not part of a serving loop).
+ * Errors: INVALID_ARG, OOM, CUDA, TIMEOUT; message in phyai_w8a8_last_error().
+ */
+phyai_status_t phyai_w8a8_project(const void *x_bf16, const uint8_t *w_codes, const float *w_scales, uint32_t M,
+                                  uint32_t K, uint32_t N, float *y, uint8_t *x_codes_out, float *x_scales_out,
+                                  void *stream);
+const char *phyai_w8a8_last_error(void);
 
 /*
  * Data-parallel serving front-end, host side (Sec. "Parallel Execution": data-parallel runners exchange no state;

@@ -87,16 +87,25 @@ def round_e4m3(y: np.ndarray) -> np.ndarray:
     return np.sign(y) * np.minimum(q, 448.0)
 
 
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """float32 -> nearest bfloat16 (ties to even), returned as float32: the upper 16 bits of the float32 pattern after
+    adding half an ulp (0x7FFF plus the lowest kept bit)."""
+    u = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000).astype(np.uint32)
+    return r.view(np.float32)
+
+
 def quantize_rows_e4m3(x: np.ndarray):
     """W8A8 activation quantization (quantization paragraph: the paper lists W8A8 among its
-    round-to-nearest modes; granularity and scale rule are a reading): every row (token) gets the scale
+    round-to-nearest modes; granularity and scale rule are a reading).  The activation that enters a
+    projection is a bfloat16 tensor, as in the W8A16 mode; every row (token) of it gets the scale
     s = max|x| / 448 (1 for an all-zero row) and its elements become round_e4m3(x / s).  The decision is
-    taken in float32 -- the precision the device takes it in -- on the float32 rounding of x.  Returns
-    (codes' values as float64, scales as float64): the projection then computes (values @ Wq) * s."""
-    x32 = np.asarray(x, dtype=np.float32)
-    amax = np.max(np.abs(x32), axis=-1, keepdims=True)
+    taken the way the device takes it: on the bfloat16 rounding of x, with scale and quotient in float32.
+    Returns (codes' values as float64, scales as float64): the projection then computes (values @ Wq) * s."""
+    xb = round_bf16(np.asarray(x, dtype=np.float32))
+    amax = np.max(np.abs(xb), axis=-1, keepdims=True)
     s = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
-    y = (x32 / s).astype(np.float32)
+    y = (xb / s).astype(np.float32)
     return round_e4m3(y.astype(F64)), s.astype(F64)
 
 

@@ -31,7 +31,7 @@ EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes
            "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity", "phyai_read_trace",
            "phyai_pack_prefix_kv", "phyai_postprocess_actions", "phyai_adapter_last_error", "phyai_batcher_create",
            "phyai_batcher_destroy", "phyai_batcher_submit", "phyai_batcher_next", "phyai_batcher_pending",
-           "phyai_batcher_plan")
+           "phyai_batcher_plan", "phyai_w8a8_project", "phyai_w8a8_last_error")
 
 
 class PhyaiError(RuntimeError):
@@ -116,6 +116,8 @@ def load_library() -> C.CDLL:
     lib.phyai_postprocess_actions.argtypes = [_VP, C.c_uint32, C.c_uint32, C.c_uint32, _VP, _VP, C.c_float, C.c_float,
                                               C.c_uint32, C.c_uint32, _VP, _VP]
     lib.phyai_adapter_last_error.restype = C.c_char_p
+    lib.phyai_w8a8_project.argtypes = [_VP, _VP, _VP, C.c_uint32, C.c_uint32, C.c_uint32, _VP, _VP, _VP, _VP]
+    lib.phyai_w8a8_last_error.restype = C.c_char_p
     lib.phyai_batcher_create.argtypes = [C.POINTER(BatcherConfig), C.POINTER(_VP)]
     lib.phyai_batcher_destroy.argtypes = [_VP]
     lib.phyai_batcher_destroy.restype = None
@@ -347,6 +349,22 @@ def postprocess_actions(x: torch.Tensor, q01: Optional[torch.Tensor], q99: Optio
     if st != OK:
         raise PhyaiError(st, lib.phyai_adapter_last_error().decode())
     return out
+
+
+def w8a8_project(x: torch.Tensor, w_codes: torch.Tensor, w_scales: torch.Tensor, return_codes: bool = False, stream=None):
+    """Stand-alone W8A8 projection (``phyai_w8a8_project``): ``x`` bf16 ``[M, K]``, ``w_codes`` uint8 ``[K, N]``,
+    ``w_scales`` float32 ``[N]`` -> float32 ``[M, N]`` (and, on request, the activation codes and scales)."""
+    lib = load_library()
+    M, K = x.shape
+    N = w_codes.shape[1]
+    y = torch.empty(M, N, dtype=torch.float32, device=x.device)
+    codes = torch.empty(M, K, dtype=torch.uint8, device=x.device) if return_codes else None
+    scales = torch.empty(M, dtype=torch.float32, device=x.device) if return_codes else None
+    st = lib.phyai_w8a8_project(_ptr(x), _ptr(w_codes), _ptr(w_scales), M, K, N, _ptr(y), _ptr(codes), _ptr(scales),
+                                _stream_ptr(stream))
+    if st != OK:
+        raise PhyaiError(st, lib.phyai_w8a8_last_error().decode())
+    return (y, codes, scales) if return_codes else y
 
 
 class Batcher:

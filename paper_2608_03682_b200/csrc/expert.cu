@@ -2,6 +2,7 @@
 // sequence of one denoising loop, CUDA-graph capture and replay.
 #include <cstdarg>
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
 #include <map>
 #include <new>
@@ -42,7 +43,7 @@ struct Tables {             // per n_steps
   float* shw_gu = nullptr;  // pi05, cluster GEMM path: [n][L][2F]   shift . W_gate/up, interleaved row order
 };
 
-inline int kind_of(uint32_t dtype) { return dtype == PHYAI_F32 ? 0 : 1; }
+inline int kind_of(uint32_t dtype) { return dtype == PHYAI_F32 ? 0 : 1; }   // storage of everything but the big matrices
 
 }  // namespace
 
@@ -51,6 +52,7 @@ struct phyai_expert {
   Dims d{};
   bool tc = false;       // tensor-core engine
   bool ada = false;
+  bool a8 = false;       // W8A8: e4m3 activations, FP8 tensor path (general kernels only)
   int sites = 0;
   int Mpad = 0;
   std::vector<void*> allocs;
@@ -107,6 +109,8 @@ struct phyai_expert {
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
   __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
+  uint8_t* xq = nullptr;     // W8A8: tiled e4m3 image of the current projection input [K/128][Mpad][128]
+  float* xs = nullptr;       // W8A8: its per-token scales [Mpad]
   __nv_bfloat16* q_tiles = nullptr;   // cluster attention: q as [request][head pair][dh / 64][128 rows][64] swizzled tiles
   __nv_bfloat16 *qr_big = nullptr, *kr_big = nullptr, *vr_big = nullptr;   // rotated bf16 q / k / v of large batches
 
@@ -168,7 +172,7 @@ phyai_status_t check_config(const phyai_expert_config_t* c) {
     return fail(PHYAI_ERR_INVALID_ARG, "has_state_token / state_dim inconsistent");
   if (c->n_q_heads % c->n_kv_heads) return fail(PHYAI_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
   if ((c->head_dim & 1) || (c->width & 1)) return fail(PHYAI_ERR_INVALID_ARG, "head_dim and width must be even");
-  if (c->cond > PHYAI_COND_PI05_ADARMS || c->dtype > PHYAI_W8E4M3_A16 || c->engine > PHYAI_ENGINE_SIMT)
+  if (c->cond > PHYAI_COND_PI05_ADARMS || c->dtype > PHYAI_W8A8_E4M3 || c->engine > PHYAI_ENGINE_SIMT)
     return fail(PHYAI_ERR_INVALID_ARG, "unknown cond / dtype / engine value");
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta >= 0.f) || !(c->time_min_period > 0.f) || !(c->time_max_period > 0.f))
     return fail(PHYAI_ERR_INVALID_ARG, "rms_eps / rope_theta / time periods out of range");
@@ -313,8 +317,17 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     pending_slabs = 0;
     return sl;
   };
-  auto tc_gemm = [&](TcGemm g) -> phyai_status_t {
+  const bool norm_q8 = h->a8 && rmsnorm_quantizes(D);   // W8A8: the norms write their e4m3 quantization themselves
+  auto tc_gemm = [&](TcGemm g, bool prequantized = false) -> phyai_status_t {
     g.rows_pad = h->Mpad, g.M = g.M ? g.M : M, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact;
+    if (h->a8) {
+      // W8A8: the projection input goes through the per-token e4m3 quantization, the product onto the FP8 tensor path
+      if (!prequantized) {
+        launch_quant_rows(h->status, g.X, h->xq, h->xs, h->Mpad, g.M, g.K, st);
+        ++cnt;
+      }
+      g.X = reinterpret_cast<const __nv_bfloat16*>(h->xq), g.fp8 = 1, g.xscale = h->xs;
+    }
     if (g.epi == TC_RESID && g.splits > 1 && nt == 64 && h->slab && D <= 2048) {
       if (g.splits > h->slab_splits) g.splits = h->slab_splits;
       g.slab = h->slab, pending_slabs = g.splits;
@@ -331,6 +344,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
     ++cnt;
   };
 
+  const int kcb = h->a8 ? 128 : 64;   // contraction elements per 128-byte operand row (k-chunk of the tile GEMM)
   const int ss_n = D / 128;
   int trace_cursor = 0;
   const bool use_w8 = h->use_w8_inkernel && !h->b_qkv.empty();
@@ -520,7 +534,8 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
                     cache_state ? h->vr_st + (size_t)l * kv_layer : h->vr_big, b1_step));
         continue;
       }
-      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs());
+      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs(),
+                     norm_q8 ? h->xq : nullptr, norm_q8 ? h->xs : nullptr);
       ++cnt;
       const bool attn_tc = h->attn_mma && h->use_tc_attention && h->qr_big && attention_tc_supported(d) &&
                            batch * (d.Hq / 2) >= ATTN_TC_MIN_CTAS;
@@ -528,7 +543,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       const bool attn_rot = h->qr_big && (attn_tc || attn_cluster);   // q / k / v leave the QKV epilogue rotated, bf16
       // one token tile: the cluster attention kernel multiplies each head's output by its slice of Wo itself and
       // writes one slab per head, which the next norm sums like the k-range partials of a split-K GEMM
-      const bool fuse_o = attn_cluster && attn_rot && h->tc && h->use_fused_oproj && h->slab && M <= 64 &&
+      const bool fuse_o = attn_cluster && attn_rot && h->tc && !h->a8 && h->use_fused_oproj && h->slab && M <= 64 &&
                           d.Hq <= MAX_SLABS && attention_oproj_supported(d);
       if (h->tc) {
         TcGemm g{};
@@ -540,7 +555,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
           g.epi = TC_QKV_ROT, g.rq = h->rq, g.rope = h->rope, g.qr = h->qr_big, g.kr = h->kr_big, g.vr = h->vr_big;
           g.S = d.S, g.Hq = d.Hq, g.Hkv = d.Hkv, g.dh = d.dh;
         }
-        ST(tc_gemm(g));
+        ST(tc_gemm(g, norm_q8));
       } else {
         SimtGemm g{};
         g.A = h->xn_f, g.lda = D, g.B = h->f_qkv[l], g.M = M, g.N = d.Nqkv, g.K = D, g.epi = EPI_STORE;
@@ -577,8 +592,8 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       } else if (h->tc) {
         TcGemm g{};
         g.W = h->p_o[l], g.X = h->attn_t, g.N = D, g.K = d.Nq, g.epi = TC_RESID, g.scale = h->s_o[l], g.gate = gate;
-        g.out_f32 = h->h, g.ldo = D, g.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.Nq / 64);
-        if (nt == 256 && D % 256 == 0) pick_resid_tiling(M, h->Mpad, D, d.Nq / 64, h->n_sm, &g.nt_override, &g.splits);
+        g.out_f32 = h->h, g.ldo = D, g.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.Nq / kcb);
+        if (nt == 256 && D % 256 == 0) pick_resid_tiling(M, h->Mpad, D, d.Nq / kcb, h->n_sm, &g.nt_override, &g.splits);
         ST(tc_gemm(g));
       } else {
         SimtGemm g{};
@@ -587,7 +602,8 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         simt_gemm(g);
       }
       site(k, 2 * l + 1, &gain, &shift, &gate);
-      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs());
+      launch_rmsnorm(h->status, h->h, gain, shift, h->xn_f, h->xn_t, h->Mpad, M, D, d.eps, st, take_slabs(),
+                     norm_q8 ? h->xq : nullptr, norm_q8 ? h->xs : nullptr);
       ++cnt;
       if (h->tc) {
         TcGemm g{};
@@ -597,11 +613,11 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
           // a single token tile: interleaved gate / up tiles put the weight stream on twice as many SMs
           g.W = h->p_gu_all + (size_t)l * D * 2 * d.F, g.W2 = nullptr, g.N = 2 * d.F, g.epi = TC_GEGLU_IL;
         }
-        ST(tc_gemm(g));
+        ST(tc_gemm(g, norm_q8));
         TcGemm g2{};
         g2.W = h->p_d[l], g2.X = h->m_t, g2.N = D, g2.K = d.F, g2.epi = TC_RESID, g2.scale = h->s_d[l], g2.gate = gate;
-        g2.out_f32 = h->h, g2.ldo = D, g2.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.F / 64);
-        if (nt == 256 && D % 256 == 0) pick_resid_tiling(M, h->Mpad, D, d.F / 64, h->n_sm, &g2.nt_override, &g2.splits);
+        g2.out_f32 = h->h, g2.ldo = D, g2.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.F / kcb);
+        if (nt == 256 && D % 256 == 0) pick_resid_tiling(M, h->Mpad, D, d.F / kcb, h->n_sm, &g2.nt_override, &g2.splits);
         ST(tc_gemm(g2));
       } else {
         SimtGemm g{};
@@ -726,7 +742,12 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
     if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->wgate[l] || !w->wup[l] || !w->wdown[l] || !w->norm1[l] ||
         !w->norm2[l] || (ada && (!w->norm1_b[l] || !w->norm2_b[l])))
       return fail(PHYAI_ERR_INVALID_ARG, "a per-layer weight pointer is NULL (layer %u)", l);
-  const bool w8 = cfg->dtype == PHYAI_W8E4M3_A16;
+  const bool a8 = cfg->dtype == PHYAI_W8A8_E4M3;     // e4m3 activations as well: the FP8 tensor path
+  const bool w8 = cfg->dtype == PHYAI_W8E4M3_A16 || a8;
+  if (a8 && !tc) return fail(PHYAI_ERR_UNSUPPORTED, "PHYAI_W8A8_E4M3 runs on the tensor path only (engine AUTO)");
+  if (a8 && (cfg->width % 128 || cfg->mlp_dim % 128 || (cfg->n_q_heads * cfg->head_dim) % 128 || cfg->mlp_dim > 4096 ||
+             cfg->width > 4096 || cfg->n_q_heads * cfg->head_dim > 4096))
+    return fail(PHYAI_ERR_UNSUPPORTED, "PHYAI_W8A8_E4M3 needs contraction lengths that are multiples of 128 and at most 4096");
   if (w8)
     for (int m = 0; m < 7; ++m) {
       if (!w->scales[m]) return fail(PHYAI_ERR_INVALID_ARG, "scales[%d] is NULL", m);
@@ -737,7 +758,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
   phyai_expert* h = new (std::nothrow) phyai_expert();
   if (!h) return fail(PHYAI_ERR_OOM, "host allocation failed");
   h->cfg = *cfg;
-  h->tc = tc, h->ada = ada;
+  h->tc = tc, h->ada = ada, h->a8 = a8;
   Dims& d = h->d;
   d.L = cfg->n_layers, d.D = cfg->width, d.F = cfg->mlp_dim, d.Hq = cfg->n_q_heads, d.Hkv = cfg->n_kv_heads;
   d.dh = cfg->head_dim, d.Ds = cfg->state_dim, d.A = cfg->action_dim, d.H = cfg->horizon, d.ns = cfg->has_state_token;
@@ -837,7 +858,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       ST(h->alloc(&pq_all, (size_t)L * D * Nqkv)); ST(h->alloc(&po_all, (size_t)L * Nq * D));
       ST(h->alloc(&pg_all, (size_t)L * D * F)); ST(h->alloc(&pu_all, (size_t)L * D * F));
       ST(h->alloc(&pd_all, (size_t)L * F * D));
-      h->il_ok = F % 64 == 0;
+      h->il_ok = F % 64 == 0 && !a8;   // (W8A8 keeps to the general kernels: no interleaved image, no cluster path)
       if (h->il_ok) ST(h->alloc(&h->p_gu_all, (size_t)L * D * 2 * F));
       // cluster split-K path (one 64-token tile): every projection must fit the kernel's resident stages
       auto fits = [&](int N, int K, bool qkv) {
@@ -864,13 +885,27 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
           launch_pack_tiled(w->wgate[l], big_kind, pgu, D, F, 0, st, 64, 0);
           launch_pack_tiled(w->wup[l], big_kind, pgu, D, F, 0, st, 64, 1);
         }
-        launch_pack_tiled(w->wq[l], big_kind, pq, D, Nq, 0, st, 0, 0, d.dh);
-        launch_pack_tiled(w->wk[l], big_kind, pq, D, Nkv, Nq, st, 0, 0, d.dh);
-        launch_pack_tiled(w->wv[l], big_kind, pq, D, Nkv, Nq + Nkv, st);
-        launch_pack_tiled(w->wo[l], big_kind, po, Nq, D, 0, st);
-        launch_pack_tiled(w->wgate[l], big_kind, pg, D, F, 0, st);
-        launch_pack_tiled(w->wup[l], big_kind, pu, D, F, 0, st);
-        launch_pack_tiled(w->wdown[l], big_kind, pd, F, D, 0, st);
+        if (a8) {
+          // the e4m3 codes themselves as operand images: blocks of 128 channels x 128 k (the allocations are sized
+          // for bf16 images: half of each is used)
+          auto u8 = [](const void* p) { return reinterpret_cast<const uint8_t*>(p); };
+          auto o8 = [](__nv_bfloat16* p) { return reinterpret_cast<uint8_t*>(p); };
+          launch_pack_bytes(u8(w->wq[l]), o8(pq), D, Nq, 0, st, 0, 0, d.dh, 1);
+          launch_pack_bytes(u8(w->wk[l]), o8(pq), D, Nkv, Nq, st, 0, 0, d.dh, 1);
+          launch_pack_bytes(u8(w->wv[l]), o8(pq), D, Nkv, Nq + Nkv, st, 0, 0, 0, 1);
+          launch_pack_bytes(u8(w->wo[l]), o8(po), Nq, D, 0, st, 0, 0, 0, 1);
+          launch_pack_bytes(u8(w->wgate[l]), o8(pg), D, F, 0, st, 0, 0, 0, 1);
+          launch_pack_bytes(u8(w->wup[l]), o8(pu), D, F, 0, st, 0, 0, 0, 1);
+          launch_pack_bytes(u8(w->wdown[l]), o8(pd), F, D, 0, st, 0, 0, 0, 1);
+        } else {
+          launch_pack_tiled(w->wq[l], big_kind, pq, D, Nq, 0, st, 0, 0, d.dh);
+          launch_pack_tiled(w->wk[l], big_kind, pq, D, Nkv, Nq, st, 0, 0, d.dh);
+          launch_pack_tiled(w->wv[l], big_kind, pq, D, Nkv, Nq + Nkv, st);
+          launch_pack_tiled(w->wo[l], big_kind, po, Nq, D, 0, st);
+          launch_pack_tiled(w->wgate[l], big_kind, pg, D, F, 0, st);
+          launch_pack_tiled(w->wup[l], big_kind, pu, D, F, 0, st);
+          launch_pack_tiled(w->wdown[l], big_kind, pd, F, D, 0, st);
+        }
         h->p_qkv.push_back(pq), h->p_o.push_back(po), h->p_g.push_back(pg), h->p_u.push_back(pu), h->p_d.push_back(pd);
         if (w8 && h->b1_ok) {
           // one byte per weight for the single-tile (HBM-bound) path; larger batches are tensor-bound and keep using
@@ -930,6 +965,11 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       ST(h->alloc(&h->vr_big, Mp * (size_t)(d.Hkv * d.dh), true));
     }
     ST(h->alloc(&h->state_tok, (size_t)cfg->max_batch * D, true));
+    if (a8) {   // tiled e4m3 activations of the widest projection input, and the per-token scales
+      const size_t kmax = (size_t)std::max(std::max(D, d.Nq), d.F);
+      ST(h->alloc(&h->xq, Mp * kmax, true));
+      ST(h->alloc(&h->xs, Mp, true));
+    }
     if (tc) {
       h->attn_mma = attention_mma_supported(d);
       if (h->attn_mma) {

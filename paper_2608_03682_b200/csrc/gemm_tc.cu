@@ -69,6 +69,8 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   // instruction descriptor: D fp32 (bit 4), A bf16 (bit 7), B bf16 (bit 10), both K-major,
   // N >> 3 at bit 17, M >> 4 at bit 24.
   constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((128u >> 4) << 24);
+  // e4m3 x e4m3 (kind::f8f6f4): format fields 0, fp32 accumulation
+  constexpr uint32_t IDESC_F8 = (1u << 4) | ((uint32_t)(NT >> 3) << 17) | ((128u >> 4) << 24);
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[STAGES];
@@ -87,7 +89,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int nt_idx = blockIdx.x, tt = blockIdx.y;
   const bool geglu = g.epi == TC_GEGLU;
-  const int KC = g.K >> 6;
+  const int KC = g.fp8 ? g.K >> 7 : g.K >> 6;   // k-chunks of 128 bytes per operand row
   const int kc_begin = (int)(((long long)KC * blockIdx.z) / gridDim.z);
   const int kc_end = (int)(((long long)KC * (blockIdx.z + 1)) / gridDim.z);
   const int nk = kc_end - kc_begin;
@@ -216,9 +218,16 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
 #pragma unroll
         for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
           const uint32_t acc = (i > first || k > 0) ? 1u : 0u;   // the warp's first MMA initialises its accumulator
-          if (elect_one()) umma_bf16(tacc, da + 2 * k, db + 2 * k, IDESC, acc);
-          if (NA == 2) {
-            if (elect_one()) umma_bf16(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
+          if (g.fp8) {
+            if (elect_one()) umma_f8(tacc, da + 2 * k, db + 2 * k, IDESC_F8, acc);
+            if (NA == 2) {
+              if (elect_one()) umma_f8(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC_F8, acc);
+            }
+          } else {
+            if (elect_one()) umma_bf16(tacc, da + 2 * k, db + 2 * k, IDESC, acc);
+            if (NA == 2) {
+              if (elect_one()) umma_bf16(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
+            }
           }
         }
       }
@@ -240,6 +249,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     const int ch = q * 32 + lane;                 // row of the 128-row tile
     const int tok_base = tt * NT;
     // 16 accumulator columns of this thread's TMEM lane (two MMA warps: the sum of their accumulators)
+    // W8A8: activation scale of every token of the tile.  The table sits at the end of the operand stages, which are
+    // free once the accumulator is complete; the values are fetched into registers while the main loop still runs.
+    float* xs_tab = reinterpret_cast<float*>(tiles_ptr + (size_t)STAGES * STAGE_BYTES) - NT;
+    // (W8A8: times the activation scale of each column's token)
     auto ld_acc = [&](uint32_t col, float* v) {
       tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + col, v);
       if (DUAL && nk > 1) {
@@ -248,7 +261,14 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] += w[j];
       }
+      if (g.xscale) {
+        const float* xs = xs_tab + (col % (uint32_t)NT);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] *= xs[j];
+      }
     };
+    float xs_reg = 0.f;
+    if (g.xscale && et < NT && tok_base + et < g.M) xs_reg = g.xscale[tok_base + et];
     if (g.epi == TC_QKV_ROT) {
       // while the main loop runs: where each token of the tile sits (request, suffix row, rotary position)
       for (int idx = et; idx < NT; idx += NEPI) {
@@ -315,6 +335,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     epi_sync();
     const bool ok = *reinterpret_cast<volatile int*>(&epi_ok) != 0;
     tc_fence_after();
+    if (g.xscale) {
+      if (et < NT) xs_tab[et] = xs_reg;
+      epi_sync();
+    }
     constexpr int HALF = NT / 4;   // token columns per epilogue warp
     const int c_begin = hf * HALF;
     const bool resid_red = g.epi == TC_RESID && gridDim.z > 1;   // split-K: vector reductions, see below
@@ -567,6 +591,10 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
           float vg[16], vu[16];
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, vg);
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(NT + c0), vu);
+          if (g.xscale) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) vg[j] *= xs_tab[c0 + j], vu[j] *= xs_tab[c0 + j];
+          }
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int t = c0 + j;   // token within the tile

@@ -71,7 +71,14 @@ void launch_pack_tiled(const void* src, int src_kind, __nv_bfloat16* dst, int K,
                        int il_group = 0, int il_second = 0, int perm_dh = 0);
 // e4m3 codes [in=K][out=N] -> byte blocks [N/128][K/64][128][64] in the packed row order of launch_pack_tiled
 void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group = 0,
-                       int il_second = 0, int perm_dh = 0);
+                       int il_second = 0, int perm_dh = 0, int wide = 0);
+// (wide: blocks [N/128][K/128][128][128] instead, the 16-byte chunks of a row XOR-swizzled by row & 7: the e4m3
+// operand image of the FP8 tensor path)
+// Per-token e4m3 quantization of a tiled bf16 activation matrix [K/64][rows_pad][64] (W8A8): scale[r] = max|x_r| / 448
+// (1 for a zero row), codes = round-to-nearest-even e4m3 of x / scale, saturating, written as the tiled e4m3 matrix
+// [K/128][rows_pad][128] with the same 16-byte chunk swizzle.  Rows >= M are left alone.
+void launch_quant_rows(const int* status, const __nv_bfloat16* x, uint8_t* out, float* scale, int rows_pad, int M, int K,
+                       cudaStream_t st);
 void launch_permute_scales(const float* src, float* dst, int N, int n_off, int perm_dh, cudaStream_t st);
 // Y[r][n] = act( sum_d X[r][d] * W[(w_row_off + d)][n] + bias[n] + add[n] ), r < R
 void launch_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K, const float* bias,
@@ -102,9 +109,12 @@ struct SlabSum {
   int n;
   size_t stride;
 };
+// (W8A8, widths for which rmsnorm_quantizes() holds: with out8 / xscale set the row leaves as its per-token e4m3
+// quantization, codes in the tiled e4m3 layout, instead of as bf16)
+bool rmsnorm_quantizes(int D);
 void launch_rmsnorm(const int* status, float* h, const float* gain, const float* shift, float* out_f32,
                     __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st,
-                    SlabSum slabs = SlabSum{nullptr, 0, 0});
+                    SlabSum slabs = SlabSum{nullptr, 0, 0}, uint8_t* out8 = nullptr, float* xscale = nullptr);
 // final norm -> out-proj -> Euler update x += dt * (v + bout)
 void launch_final(const Request* rq, const int* status, const float* h, const float* gain, const float* shift,
                   const float* Wout, const float* bout, float dt, const Dims& d, int batch, cudaStream_t st);
@@ -176,6 +186,10 @@ struct TcGemm {
   int rows_pad, M, N, K;
   int epi;
   const float* scale;  // per-out-channel dequant scale or null
+  // W8A8: W and X hold e4m3 codes (128-byte rows = 128 k per block / tile chunk), the product runs on the FP8 tensor
+  // path and every accumulator column is multiplied by its token's activation scale
+  int fp8;
+  const float* xscale;   // [rows] per-token activation scale (fp8 only)
   const float* scale2;
   const float* bias;   // TC_BIAS_ROWMAP
   const float* gate;   // TC_RESID (null = 1)

@@ -121,26 +121,97 @@ void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int
 // e4m3 codes [K][N] -> byte blocks of 128 out channels x 64 k (row order as in k_pack_tiled, no swizzle: the kernel
 // that decodes them writes the swizzled bf16 image itself).  One thread per 8 consecutive k of one out channel.
 __global__ void k_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, int il_group, int il_second,
-                             int perm_dh) {
-  const int KC = K >> 6;
+                             int perm_dh, int wide) {
+  const int KC = wide ? K >> 7 : K >> 6;
   const size_t chunks = (size_t)N * (K >> 3);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
     const int n = (int)(i % N), k0 = (int)(i / N) << 3;
     const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
                             : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
-    const int kc = k0 >> 6, c = (k0 & 63) >> 3;
     __align__(8) uint8_t v[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) v[j] = src[(size_t)(k0 + j) * N + n];
-    *reinterpret_cast<uint2*>(dst + (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 64 + (size_t)c * 8) =
-        *reinterpret_cast<const uint2*>(v);
+    size_t off;
+    if (wide) {
+      // 128-byte rows: 16-byte chunk ((k0 % 128) / 16) XOR (row % 8), then the 8-byte half inside it
+      const int kc = k0 >> 7, w = k0 & 127, r = np & 127;
+      off = (((size_t)(np >> 7) * KC + kc) * 128 + r) * 128 + (size_t)(((w >> 4) ^ (r & 7)) << 4) + (size_t)(w & 8);
+    } else {
+      const int kc = k0 >> 6, c = (k0 & 63) >> 3;
+      off = (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 64 + (size_t)c * 8;
+    }
+    *reinterpret_cast<uint2*>(dst + off) = *reinterpret_cast<const uint2*>(v);
   }
 }
 void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group,
-                       int il_second, int perm_dh) {
+                       int il_second, int perm_dh, int wide) {
   const size_t chunks = (size_t)N * (K >> 3);
   const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
-  k_pack_bytes<<<blocks, 256, 0, st>>>(src, dst, K, N, n_off, il_group, il_second, perm_dh);
+  k_pack_bytes<<<blocks, 256, 0, st>>>(src, dst, K, N, n_off, il_group, il_second, perm_dh, wide);
+}
+
+// W8A8 activation quantization: one warp per token row.  A lane takes the 16-column groups lane, lane + 32, ... of
+// the row (two 16-byte chunks of the bf16 tile -> one 16-byte chunk of the e4m3 tile); the row stays in registers
+// between the maximum and the rounding.  The division by the scale is the IEEE one, so that the rounding decision
+// depends on nothing but the stored activations.
+constexpr int QR_MAXG = 8;    // 16-column groups per lane: K <= 32 * 8 * 16 = 4096
+__global__ void __launch_bounds__(256) k_quant_rows(const int* status, const __nv_bfloat16* x, uint8_t* out, float* scale,
+                                                    int rows_pad, int M, int K) {
+  pdl_enter();
+  if (status_set(status)) return;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const int groups = K >> 4;
+  uint4 v[QR_MAXG][2];
+  float amax = 0.f;
+#pragma unroll
+  for (int j = 0; j < QR_MAXG; ++j) {
+    const int gi = lane + 32 * j;
+    if (gi < groups) {
+      const int col = gi << 4, kc = col >> 6, c = (col & 63) >> 3;           // two consecutive 8-column chunks c, c + 1
+      const __nv_bfloat16* base = x + ((size_t)kc * rows_pad + row) * 64;
+      v[j][0] = *reinterpret_cast<const uint4*>(base + ((c ^ (row & 7)) << 3));
+      v[j][1] = *reinterpret_cast<const uint4*>(base + (((c + 1) ^ (row & 7)) << 3));
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t w[4] = {v[j][h].x, v[j][h].y, v[j][h].z, v[j][h].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
+          amax = fmaxf(amax, fmaxf(fabsf(__low2float(p)), fabsf(__high2float(p))));
+        }
+      }
+    }
+  }
+  amax = warp_max(amax);
+  const float s = amax > 0.f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+  if (lane == 0) scale[row] = s;
+#pragma unroll
+  for (int j = 0; j < QR_MAXG; ++j) {
+    const int gi = lane + 32 * j;
+    if (gi < groups) {
+      uint32_t o[4];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t w[4] = {v[j][h].x, v[j][h].y, v[j][h].z, v[j][h].w};
+#pragma unroll
+        for (int e = 0; e < 4; e += 2) {
+          const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
+          const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&w[e + 1]);
+          uint16_t lo, hi;    // cvt packs its first source into the upper byte
+          asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(__high2float(p0), s)), "f"(__fdiv_rn(__low2float(p0), s)));
+          asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(__high2float(p1), s)), "f"(__fdiv_rn(__low2float(p1), s)));
+          o[h * 2 + (e >> 1)] = (uint32_t)lo | ((uint32_t)hi << 16);
+        }
+      }
+      const int col = gi << 4, kc = col >> 7, c16 = (col & 127) >> 4;
+      *reinterpret_cast<uint4*>(out + ((size_t)kc * rows_pad + row) * 128 + ((c16 ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+}
+void launch_quant_rows(const int* status, const __nv_bfloat16* x, uint8_t* out, float* scale, int rows_pad, int M, int K,
+                       cudaStream_t st) {
+  launch_pdl(k_quant_rows, dim3((M + 7) / 8), dim3(256), 0, st, status, x, out, scale, rows_pad, M, K);
 }
 
 // Row of an adaptive norm's shift through a packed weight matrix: out[n] = scale(n) * sum_k shift[k] * W[n][k].
@@ -455,9 +526,12 @@ __global__ void k_rmsnorm_tiled4(const int* status, float* h, const float* gain,
 
 // Same, with the whole row held in registers (D = NV * 128): every load of the row is in flight at once and the
 // row is read once.
+// With out8 set (W8A8) the normalised row leaves as its per-token e4m3 quantization instead (codes in the tiled e4m3
+// layout, scale in xscale[row]): the bf16 rounding of every element is what gets quantized, as in k_quant_rows.
 template <int NV>
 __global__ void k_rmsnorm_tiled_reg(const int* status, float* h, const float* gain, const float* shift,
-                                    __nv_bfloat16* out, int rows_pad, int M, float eps, SlabSum sl) {
+                                    __nv_bfloat16* out, int rows_pad, int M, float eps, SlabSum sl, uint8_t* out8,
+                                    float* xscale) {
   pdl_enter();
   if (status_set(status)) return;
   constexpr int D = NV * 128;
@@ -495,9 +569,30 @@ __global__ void k_rmsnorm_tiled_reg(const int* status, float* h, const float* ga
       o.x += s4.x, o.y += s4.y, o.z += s4.z, o.w += s4.w;
     }
     __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+    if (out8) {   // keep the bf16-rounded values for the quantization below
+      v[k] = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+      continue;
+    }
     uint2 pk;
     pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
     *reinterpret_cast<uint2*>(out + tiled_index(row, d, rows_pad)) = pk;
+  }
+  if (out8) {
+    float amax = 0.f;
+#pragma unroll
+    for (int k = 0; k < NV; ++k) amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[k].x), fabsf(v[k].y)), fmaxf(fabsf(v[k].z), fabsf(v[k].w))));
+    amax = warp_max(amax);
+    const float s = amax > 0.f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+    if (lane == 0) xscale[row] = s;
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      uint16_t lo, hi;    // cvt packs its first source into the upper byte
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(v[k].y, s)), "f"(__fdiv_rn(v[k].x, s)));
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(v[k].w, s)), "f"(__fdiv_rn(v[k].z, s)));
+      // channels k * 128 + 4 lane .. + 3: k-chunk k of the e4m3 tile, 16-byte chunk lane / 4, bytes 4 (lane % 4) ..
+      *reinterpret_cast<uint32_t*>(out8 + ((size_t)k * rows_pad + row) * 128 + ((((lane >> 2) ^ (row & 7))) << 4) + (lane & 3) * 4) =
+          (uint32_t)lo | ((uint32_t)hi << 16);
+    }
   }
 }
 
@@ -551,9 +646,12 @@ void launch_add_slabs(const int* status, float* h, int M, int D, cudaStream_t st
              (__nv_bfloat16*)nullptr, 0, D, 0.0f, sl);
 }
 
+bool rmsnorm_quantizes(int D) { return D == 1024 || D == 2048; }
+
 void launch_rmsnorm(const int* status, float* h, const float* gain, const float* shift, float* out_f32,
-                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st, SlabSum sl) {
-  if (sl.n && out_tiled && D % 128 == 0 && D <= 2048) {
+                    __nv_bfloat16* out_tiled, int rows_pad, int M, int D, float eps, cudaStream_t st, SlabSum sl,
+                    uint8_t* out8, float* xscale) {
+  if (sl.n && !out8 && out_tiled && D % 128 == 0 && D <= 2048) {
     launch_pdl(k_add_slabs_norm, dim3(M), dim3(D / 4), 0, st, status, h, gain, shift, out_tiled, rows_pad, D, eps, sl);
     return;
   }
@@ -561,11 +659,13 @@ void launch_rmsnorm(const int* status, float* h, const float* gain, const float*
   const int wpb = sl.n ? 1 : 4;
   const int blocks = (M + wpb - 1) / wpb;
   if (out_tiled && D == 1024) {
-    launch_pdl(k_rmsnorm_tiled_reg<8>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl);
+    launch_pdl(k_rmsnorm_tiled_reg<8>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl, out8,
+               xscale);
     return;
   }
   if (out_tiled && D == 2048) {
-    launch_pdl(k_rmsnorm_tiled_reg<16>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl);
+    launch_pdl(k_rmsnorm_tiled_reg<16>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl, out8,
+               xscale);
     return;
   }
   if (out_tiled && D % 128 == 0) {

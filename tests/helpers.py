@@ -44,3 +44,17 @@ def elem_rel_err(got, ref):
     got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
     floor = 1e-3 * np.max(np.abs(ref))
     return float(np.max(np.abs(got - ref) / np.maximum(np.abs(ref), floor)))
+
+
+def w8a8_bar(cfg, W, kv, P, state, noise, n_steps, ref_w8a8):
+    """Tolerance of a whole-network W8A8 comparison.  The activation quantizer is a step function with steps of
+    1/16 .. 1/8 of an element: the bf16-level differences between the device's activations and the oracle's move a few
+    per cent of the elements across a step, and each such element then differs by a whole step -- noise of the same
+    kind, and nearly the same size, as the quantization noise of the mode itself.  That size is measured on the
+    case at hand as the distance d_q between the oracle's W8A8 and W8A16 results; the device result must lie within
+    2.5 d_q of the W8A8 oracle (and within 15 % in any case).  The arithmetic of the mode itself -- codes, scales,
+    FP8 product -- is checked exactly in test_gpu_w8a8.py."""
+    import dataclasses
+    cfg16 = dataclasses.replace(cfg, dtype="w8e4m3")
+    d_q = O.max_rel_err(O.denoise(cfg16, W, kv, P, state, noise, n_steps), ref_w8a8)
+    return min(0.15, 2.5 * d_q), d_q

@@ -20,7 +20,7 @@ def lib():
 
 def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "phyai.h")).read()
-    declared = set(re.findall(r"\b(phyai_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(phyai_[a-z0-9_]+)\s*\(", header))
     assert declared == set(binding.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), name

@@ -6,7 +6,7 @@ import torch
 
 from oracle import expert_oracle as O
 from paper_2608_03682_b200 import binding, synth
-from tests.helpers import BAR, elem_rel_err, rel_err
+from tests.helpers import BAR, elem_rel_err, rel_err, w8a8_bar
 
 pytestmark = pytest.mark.gpu
 
@@ -53,3 +53,20 @@ def test_e4m3_weight_expert_matches_oracle(batch):
     errs = _run_batched(cfg, 5, W, [816] * batch, 10, check)
     print(f"C5 batch {batch} max rel err:", {b: f"{e:.2e}" for b, e in errs.items()})
     assert max(errs.values()) <= BAR["w8e4m3"], errs
+
+
+@pytest.mark.parametrize("batch", [1, 8, 64])
+def test_w8a8_expert_matches_oracle(batch):
+    """The pi0-shaped expert with e4m3 weights and per-token e4m3 activations (FP8 tensor path) against the oracle's
+    W8A8 mode on sampled requests, within the tolerance that the mode's own quantization noise sets (see w8a8_bar)."""
+    cfg = synth.pi0_config(max_batch=batch, dtype="w8a8e4m3", max_prefix_len=816)
+    W = synth.make_weights(cfg, 5)
+    check = [0] if batch == 1 else [0, batch - 1]
+    errs = _run_batched(cfg, 5, W, [816] * batch, 10, check)
+    Wf = O.Weights(W)
+    for b in check:
+        kv, st, nz = synth.make_prefix_kv(cfg, 5, 816, b), synth.make_state(cfg, 5, b), synth.make_noise(cfg, 5, b)
+        ref = O.denoise(cfg, Wf, kv, 816, st, nz, 10)
+        bar, d_q = w8a8_bar(cfg, Wf, kv, 816, st, nz, 10, ref)
+        print(f"W8A8 batch {batch} request {b}: max rel err {errs[b]:.2e}, quantization noise of the mode {d_q:.2e}, bar {bar:.2e}")
+        assert errs[b] <= bar, (b, errs[b], bar)

@@ -6,7 +6,7 @@ import torch
 
 from oracle import expert_oracle as O
 from paper_2608_03682_b200 import binding, synth
-from tests.helpers import BAR, elem_rel_err, gpu_single, rel_err, small_bf16_config
+from tests.helpers import BAR, elem_rel_err, gpu_single, rel_err, small_bf16_config, w8a8_bar
 
 pytestmark = pytest.mark.gpu
 
@@ -243,6 +243,37 @@ def test_small_e4m3_expert_decoded_in_the_kernel_matches_oracle_and_the_expanded
                 assert rel_err(got, ref) <= BAR["w8e4m3"], (P, mode, rel_err(got, ref))
                 outs.append(got)
             assert np.array_equal(outs[0], outs[1]), P
+
+
+@pytest.mark.parametrize("cond", ["pi0", "pi05"])
+def test_small_w8a8_expert_matches_oracle_single_and_batched(cond):
+    """W8A8: per-token e4m3 activations and e4m3 weights on the FP8 tensor path (general kernels at every batch size);
+    the oracle applies the same quantization rule ahead of the seven large projections."""
+    cfg = small_bf16_config(cond, dtype="w8a8e4m3", max_prefix_len=300, max_batch=5)
+    W = synth.make_weights(cfg, 23, std=0.05)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        for P in (0, 1, 130, 300):
+            kv, state, noise = _inputs(cfg, 23, P)
+            ref = O.denoise(cfg, W, kv, P, state, noise, 3)
+            got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
+            bar, d_q = w8a8_bar(cfg, W, kv, P, state, noise, 3, ref)
+            print(f"w8a8 {cond} P={P}: {rel_err(got, ref):.2e} (quantization noise of the mode {d_q:.2e}, bar {bar:.2e})")
+            assert rel_err(got, ref) <= bar, (P, rel_err(got, ref), bar)
+        lens = [300, 0, 17, 129, 64]
+        kvs = [synth.make_prefix_kv(cfg, 23, p, b) if p else synth.make_prefix_kv(cfg, 23, 1, b)[:, :, :0] for b, p in enumerate(lens)]
+        packed, cu = synth.pack_prefix_kv(kvs)
+        states = torch.stack([synth.make_state(cfg, 23, b) for b in range(5)]) if cfg.has_state_token else None
+        noise = torch.stack([synth.make_noise(cfg, 23, b) for b in range(5)])
+        out = ex.denoise_batched(packed.cuda(), torch.from_numpy(cu).cuda(), None if states is None else states.cuda(),
+                                 noise.cuda(), 3)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        out = out.double().cpu().numpy()
+        for b in range(5):
+            ref = O.denoise(cfg, W, kvs[b], lens[b], None if states is None else states[b], noise[b], 3)
+            bar, d_q = w8a8_bar(cfg, W, kvs[b], lens[b], None if states is None else states[b], noise[b], 3, ref)
+            print(f"w8a8 {cond} batched request {b}: {rel_err(out[b], ref):.2e} (noise {d_q:.2e}, bar {bar:.2e})")
+            assert rel_err(out[b], ref) <= bar, (b, rel_err(out[b], ref), bar)
 
 
 def test_single_request_after_a_ragged_batch_with_many_heads():

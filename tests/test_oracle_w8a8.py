@@ -45,6 +45,17 @@ def test_ties_go_to_the_even_mantissa_and_large_values_saturate():
     assert np.array_equal(O.round_e4m3(np.array([448.0, 460.0, 1e9, -1e9])), np.array([448.0, 448.0, 448.0, -448.0]))
 
 
+def test_bf16_rounding_agrees_with_the_library_cast():
+    rng = np.random.default_rng(11)
+    x = np.concatenate([rng.standard_normal(50000) * np.exp(rng.uniform(-20, 20, 50000)),
+                        np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8), 0.0, 2.0 ** -130])]).astype(np.float32)
+    lib = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(O.round_bf16(x), lib)
+    # ties to even by hand: 1 + 2^-8 is halfway between 1 and 1 + 2^-7 -> 1; 1 + 3 * 2^-8 -> 1 + 2^-6
+    assert O.round_bf16(np.float32(1.0 + 2.0 ** -8)) == np.float32(1.0)
+    assert O.round_bf16(np.float32(1.0 + 3 * 2.0 ** -8)) == np.float32(1.0 + 2.0 ** -6)
+
+
 def test_row_scale_rule_by_hand():
     x = np.array([[0.5, -3.5, 1.0, 0.0], [0.0, 0.0, 0.0, 0.0], [448.0, 1.0, -2.0, 3.0]])
     q, s = O.quantize_rows_e4m3(x)
@@ -82,8 +93,9 @@ def test_quantization_error_of_a_projection_is_within_the_format_bound():
     rng = np.random.default_rng(5)
     x = rng.standard_normal((7, 256)) * np.exp(rng.standard_normal((7, 1)))
     q, s = O.quantize_rows_e4m3(x)
-    err = np.abs(x.astype(np.float32).astype(np.float64) - q * s)
-    assert np.all(err <= np.abs(x) / 16.0 + s * 2.0 ** -10 + 1e-12)
+    xb = O.round_bf16(x.astype(np.float32)).astype(np.float64)
+    err = np.abs(xb - q * s)
+    assert np.all(err <= np.abs(xb) / 16.0 + s * 2.0 ** -10 + 1e-12)
 
 
 @pytest.mark.parametrize("cond", ["pi0", "pi05"])
