@@ -2,24 +2,27 @@
 // range of a request split over a thread-block cluster, partial results merged over distributed shared memory.
 //
 // Work split.  Few queries, one long shared K / V stream: the limiter is how fast the prefix K / V (and Q) get into
-// the SMs, so the keys of a request are divided among the 8 CTAs of a cluster (about (P + S) / 8 <= 128 keys each:
-// ONE 128-key tile per CTA for prefixes up to ~970 tokens, hence no online-softmax loop in the common case), and two
-// query heads that share a kv head are stacked on the M axis (2 x 64 padded rows = the 128 rows of one MMA), so a
-// K / V tile is fetched once per head pair.  Grid = (8 key ranges, Hq / 2 head pairs, requests).
+// the SMs, so the keys of a request are divided among the 8 CTAs of a cluster (an eighth of the prefix keys plus an
+// eighth of the request's own suffix keys each, <= 128 keys: ONE 128-key tile per CTA for prefixes up to ~970 tokens,
+// hence no online-softmax loop in the common case).  A CTA takes HPC query heads: one (rows 0..63 of the 128-row MMA;
+// the Q tile, the partials that cross the cluster and the merge are then half as large, and the call runs on 8 Hq
+// CTAs) or, when the SMs do not allow that many CTAs, two heads that share a kv head stacked on the M axis.
+// Grid = (8 key ranges, Hq / HPC, requests).
 //   S = Q K^T   tcgen05.mma M = 128, N = 128 keys, K = head_dim; Q and the K tile in shared memory
 //   softmax     one thread per row straight from tensor memory (no shuffles); P (bf16) written back to tensor memory
 //   O = P V     tcgen05.mma M = 128, N = head_dim, K = 128 keys; P is the tensor-memory A operand, V an MN-major B
 //               operand (K and V tiles share one shared-memory layout and loader code)
 // The prefix rows of a CTA's tile are constants of the call and are requested before the programmatic dependency
-// wait; Q and the request's own (suffix) keys come from the QKV projection's epilogue right after it.
+// wait; Q (written by the QKV projection's epilogue as this kernel's swizzled operand tile: eight bulk copies) and the
+// CTA's share of the request's own (suffix) keys come right after it.
 //
-// Merge.  Every CTA holds an un-normalised partial (O, row max, row sum) of all 2 x S rows.  Row i of both heads is
+// Merge.  Every CTA holds an un-normalised partial (O, row max, row sum) of all HPC x S rows.  Row i of every head is
 // owned by CTA i / 8: each CTA writes its partial, rounded to bf16 and grouped by owner, into its own shared memory
 // and sends every owner one bulk copy over distributed shared memory (counted on the owner's mbarrier); the owner
 // combines the 8 partials of its rows in rank order and stores the normalised bf16 rows as the activation tile of
 // the output projection.  No partials in global memory, no merge kernel.
 //
-// Warps: 4 issues the MMAs; the other eight are two threads per accumulator row (each half of the columns): Q copies,
+// Warps: 4 issues the MMAs; the other eight are two threads per accumulator row (each half of the columns): the
 // softmax, partial out; warps 0-1 also load K, 2-3 V (16-byte cp.async into the swizzled block
 // layout); all nine merge.  Waits are bounded (see mbar_wait_drain); after a give-up the
 // protocol still runs to its end so that no peer is left waiting, only the global stores are skipped.

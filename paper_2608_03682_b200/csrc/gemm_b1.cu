@@ -20,8 +20,11 @@
 //     rsqrt(sum of the partials / D + eps) (the contraction is linear in that per-token factor) and adds, for
 //     adaptive norms, the row shift . W from a per-step table.  No norm kernel, no slab-sum kernel.
 //
-// Epilogues: rotary QKV (rotated, scaled bf16 q / k / v in the attention layout), interleaved GeGLU (64 gate + 64
-// up channels per tile), gated residual with the next norm's operands.  Waits: see mbar_wait_drain -- a given-up
+// Epilogues: rotary QKV (rotated, scaled bf16 k / v rows, q as rows or as the cluster attention kernel's swizzled
+// operand tiles), interleaved GeGLU (64 gate + 64 up channels per tile), gated residual with the next norm's
+// operands (also: the second layer of the pi0 action / time MLP, bias and state-token rows instead of the residual).
+// 512 threads: an epilogue is a chain of dependent instructions per thread, so items are small (four channels of a
+// token) and the per-channel tables are read as 16-byte vectors.  Waits: see mbar_wait_drain -- a given-up
 // wait suppresses the global stores but never the copy / reduce protocol, so peers are not left waiting and
 // nothing is in flight at exit.
 #include "kernels.h"
