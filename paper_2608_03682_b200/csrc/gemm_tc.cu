@@ -31,6 +31,8 @@
 // Every wait is bounded: on expiry of the caller's limit the CTA raises the status word and skips its MMAs and
 // stores, but keeps the copy / commit pipeline running under a generous limit of its own, so that every copy
 // into its shared memory has landed before it exits (TMEM is always released).
+#include <type_traits>
+
 #include "kernels.h"
 #include "ptx.cuh"
 #include "tc.cuh"
@@ -201,41 +203,47 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     // ---------------- MMA issuer(s) (whole warp in the loop, one elected lane issues) ---------------------
     const int first = DUAL ? warp - 8 : 0, step = DUAL ? 2 : 1;
     const uint32_t tacc = tmem_base + (DUAL ? (uint32_t)(warp - 8) * NT : 0u);
-    for (int i = first; i < nk; i += step) {
-      const int s = i % STAGES;
-      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-      const bool ok = mbar_wait_drain(smem_u32(&bar_full[s]), ph, wc) > 0;
-      // (no tcgen05 fence here: the operands were written by the bulk-copy engine and made visible by the mbarrier;
-      // tcgen05.fence::after_thread_sync orders tensor-memory accesses, and it was measured to hold the next MMAs
-      // back until the previous stage's MMAs had drained)
-      const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
-      const uint64_t da = make_desc(a0);
-      const uint64_t da2 = make_desc(a0 + A_BYTES);
-      const uint64_t db = make_desc(a0 + A_BYTES * NA);
-      // control flow and descriptors stay warp-uniform; only the tcgen05 instructions themselves are predicated on
-      // the elected lane
-      if (__all_sync(0xffffffffu, ok)) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
-          const uint32_t acc = (i > first || k > 0) ? 1u : 0u;   // the warp's first MMA initialises its accumulator
-          if (g.fp8) {
-            if (elect_one()) umma_f8(tacc, da + 2 * k, db + 2 * k, IDESC_F8, acc);
-            if (NA == 2) {
-              if (elect_one()) umma_f8(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC_F8, acc);
-            }
-          } else {
-            if (elect_one()) umma_bf16(tacc, da + 2 * k, db + 2 * k, IDESC, acc);
-            if (NA == 2) {
-              if (elect_one()) umma_bf16(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
+    // (the operand kind is fixed per launch: the loop exists once per kind, so that the issue sequence of a k-step,
+    // which paces small tiles, carries no test of it)
+    auto main_loop = [&](auto f8) {
+      for (int i = first; i < nk; i += step) {
+        const int s = i % STAGES;
+        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        const bool ok = mbar_wait_drain(smem_u32(&bar_full[s]), ph, wc) > 0;
+        // (no tcgen05 fence here: the operands were written by the bulk-copy engine and made visible by the mbarrier;
+        // tcgen05.fence::after_thread_sync orders tensor-memory accesses, and it was measured to hold the next MMAs
+        // back until the previous stage's MMAs had drained)
+        const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
+        const uint64_t da = make_desc(a0);
+        const uint64_t da2 = make_desc(a0 + A_BYTES);
+        const uint64_t db = make_desc(a0 + A_BYTES * NA);
+        // control flow and descriptors stay warp-uniform; only the tcgen05 instructions themselves are predicated on
+        // the elected lane
+        if (__all_sync(0xffffffffu, ok)) {
+  #pragma unroll
+          for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
+            const uint32_t acc = (i > first || k > 0) ? 1u : 0u;   // the warp's first MMA initialises its accumulator
+            if constexpr (decltype(f8)::value) {
+              if (elect_one()) umma_f8(tacc, da + 2 * k, db + 2 * k, IDESC_F8, acc);
+              if (NA == 2) {
+                if (elect_one()) umma_f8(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC_F8, acc);
+              }
+            } else {
+              if (elect_one()) umma_bf16(tacc, da + 2 * k, db + 2 * k, IDESC, acc);
+              if (NA == 2) {
+                if (elect_one()) umma_bf16(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
+              }
             }
           }
         }
+        // frees the stage when the MMAs above have read it -- only if a later k-step will reuse the stage (a commit
+        // that nobody waits for still costs the issuing thread time)
+        if (i + STAGES < nk && elect_one()) umma_commit(smem_u32(&bar_empty[s]));
+        __syncwarp();
       }
-      // frees the stage when the MMAs above have read it -- only if a later k-step will reuse the stage (a commit
-      // that nobody waits for still costs the issuing thread time)
-      if (i + STAGES < nk && elect_one()) umma_commit(smem_u32(&bar_empty[s]));
-      __syncwarp();
-    }
+    };
+    if (g.fp8) main_loop(std::true_type{});
+    else main_loop(std::false_type{});
     if (elect_one()) umma_commit(smem_u32(&bar_accum));
     __syncwarp();
   }
