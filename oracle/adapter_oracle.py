@@ -12,8 +12,14 @@ quantile statistics, the controller uses a slice of the chunk):
 * ``postprocess_actions``: ``(clip(x, lo, hi) + 1) / 2 * (q99 - q01) + q01`` on the first ``out_horizon`` steps and
   ``out_dim`` action dimensions, float64.  Reading: the clip acts in normalised space, before un-normalisation.
 
+* ``project_features_kv``: the request-local K / V projections of a feature-handoff head (results section, phase
+  list of the GR00T profile: the action head contains "request-local cross-attention K/V projections"; the paper gives
+  no equations -- reading: per layer ``K_l = F Wk_l``, ``V_l = F Wv_l`` of the fixed vision-language features ``F``,
+  computed once per request, no rotary embedding on features) -> ``[L, 2, P, Hkv, dh]``, float64 matmul.
+
 Pins (tests/test_adapter_oracle.py): a hand-written ragged example with distinct integers; endpoints and midpoint of
-the quantile map (x = -1 -> q01, x = +1 -> q99, x = 0 -> the mean of the two), saturation outside [-1, 1], the slice.
+the quantile map (x = -1 -> q01, x = +1 -> q99, x = 0 -> the mean of the two), saturation outside [-1, 1], the slice;
+the projection with one-hot weights (a column selection), with small integers by hand, and its layer / plane order.
 """
 from __future__ import annotations
 
@@ -46,3 +52,14 @@ def postprocess_actions(x, q01, q99, clip=(-1.0, 1.0), out_horizon=None, out_dim
     lo = -np.ones(out_dim) if q01 is None else np.asarray(q01, dtype=np.float64)[:out_dim]
     hi = np.ones(out_dim) if q99 is None else np.asarray(q99, dtype=np.float64)[:out_dim]
     return (y + 1.0) / 2.0 * (hi - lo) + lo
+
+
+def project_features_kv(features, wk, wv, n_kv_heads: int, head_dim: int) -> np.ndarray:
+    """features ``[P, Dv]``; wk, wv: per-layer lists of ``[Dv, Hkv * dh]``.  Returns ``[L, 2, P, Hkv, dh]`` float64."""
+    F = np.asarray(features, dtype=np.float64)
+    L = len(wk)
+    out = np.zeros((L, 2, F.shape[0], n_kv_heads, head_dim), dtype=np.float64)
+    for l in range(L):
+        out[l, 0] = (F @ np.asarray(wk[l], dtype=np.float64)).reshape(F.shape[0], n_kv_heads, head_dim)
+        out[l, 1] = (F @ np.asarray(wv[l], dtype=np.float64)).reshape(F.shape[0], n_kv_heads, head_dim)
+    return out

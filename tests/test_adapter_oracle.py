@@ -38,3 +38,25 @@ def test_postprocess_quantile_map_endpoints_midpoint_saturation_and_slice():
     z = A.postprocess_actions(x, q01, q99, out_horizon=2, out_dim=2)
     assert z.shape == (1, 2, 2) and z[0, 1].tolist() == [2.0, 1.0]
     assert A.postprocess_actions(x, None, None, clip=None)[0, 3].tolist() == [1.5, -7.0, 0.5]
+
+
+def test_feature_projection_by_hand_and_with_one_hot_weights():
+    # two tokens, three feature channels, one kv head of two channels, two layers, small integers
+    F = np.array([[1.0, 2.0, 3.0], [0.0, -1.0, 4.0]])
+    wk = [np.array([[1.0, 0.0], [0.0, 1.0], [1.0, 1.0]]), np.array([[2.0, 0.0], [0.0, 0.0], [0.0, -1.0]])]
+    wv = [np.array([[0.0, 1.0], [1.0, 0.0], [0.0, 0.0]]), np.array([[1.0, 1.0], [1.0, 1.0], [1.0, 1.0]])]
+    out = A.project_features_kv(F, wk, wv, 1, 2)
+    assert out.shape == (2, 2, 2, 1, 2)
+    assert np.array_equal(out[0, 0, :, 0], [[4.0, 5.0], [4.0, 3.0]])      # K, layer 0: (f0 + f2, f1 + f2)
+    assert np.array_equal(out[0, 1, :, 0], [[2.0, 1.0], [-1.0, 0.0]])     # V, layer 0: (f1, f0)
+    assert np.array_equal(out[1, 0, :, 0], [[2.0, -3.0], [0.0, -4.0]])    # K, layer 1: (2 f0, -f2)
+    assert np.array_equal(out[1, 1, :, 0], [[6.0, 6.0], [3.0, 3.0]])      # V, layer 1: sums
+    # one-hot weights select feature columns, head-major then channel
+    rng = np.random.default_rng(0)
+    F = rng.standard_normal((5, 8))
+    sel = np.zeros((8, 4))
+    for c, f in enumerate([7, 0, 3, 3]):
+        sel[f, c] = 1.0
+    out = A.project_features_kv(F, [sel], [sel[:, ::-1]], 2, 2)
+    assert np.array_equal(out[0, 0].reshape(5, 4), F[:, [7, 0, 3, 3]])
+    assert np.array_equal(out[0, 1].reshape(5, 4), F[:, [3, 3, 0, 7]])
