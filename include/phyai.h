@@ -348,6 +348,28 @@ phyai_status_t phyai_postprocess_actions(const float *x, uint32_t batch, uint32_
                                          const float *q01, const float *q99, float clip_lo, float clip_hi,
                                          uint32_t out_horizon, uint32_t out_dim, float *out, void *stream);
 
+/*
+ * phyai_project_features_kv: the request-local K / V projections of a feature-handoff action head (results section,
+ * GR00T phase list: the action head contains "request-local cross-attention K/V projections"; the vision-language
+ * features are fixed over the denoising steps, so their per-layer keys and values are computed once per request and
+ * then serve as the loop's prefix KV; no rotary embedding on features).  K_l = F Wk_l, V_l = F Wv_l on the tensor cores.
+ *   desc        n_layers, n_kv_heads, head_dim, feat_dim (a multiple of 64; 2 * n_kv_heads * head_dim a multiple of 128)
+ *   features    device bfloat16 [tokens][feat_dim] row-major: the requests' feature rows, concatenated in the order
+ *               of their prefix rows (cu_prefix_lens of the later denoise call)
+ *   wk, wv      HOST arrays of n_layers DEVICE pointers, bfloat16 [feat_dim][n_kv_heads * head_dim] ([in, out])
+ *   prefix_kv   device bfloat16 [n_layers][2][kv_tokens][n_kv_heads][head_dim]; rows [0, tokens) of every plane are
+ *               written
+ * Allocates its temporaries, runs on `stream` and synchronises it before returning (once per request batch, outside
+ * the captured loop).  Errors: INVALID_ARG, OOM, CUDA, TIMEOUT.
+ */
+typedef struct {
+  uint32_t struct_size;
+  uint32_t n_layers, n_kv_heads, head_dim, feat_dim;
+} phyai_kv_proj_desc_t;
+phyai_status_t phyai_project_features_kv(const phyai_kv_proj_desc_t *desc, const void *features, const void *const *wk,
+                                         const void *const *wv, uint64_t tokens, uint64_t kv_tokens, void *prefix_kv,
+                                         void *stream);
+
 /* Thread-local description of the last error of an adapter entry point. */
 const char *phyai_adapter_last_error(void);
 

@@ -31,7 +31,7 @@ EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes
            "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity", "phyai_read_trace",
            "phyai_pack_prefix_kv", "phyai_postprocess_actions", "phyai_adapter_last_error", "phyai_batcher_create",
            "phyai_batcher_destroy", "phyai_batcher_submit", "phyai_batcher_next", "phyai_batcher_pending",
-           "phyai_batcher_plan", "phyai_w8a8_project", "phyai_w8a8_last_error")
+           "phyai_batcher_plan", "phyai_w8a8_project", "phyai_w8a8_last_error", "phyai_project_features_kv")
 
 
 class PhyaiError(RuntimeError):
@@ -118,6 +118,7 @@ def load_library() -> C.CDLL:
     lib.phyai_adapter_last_error.restype = C.c_char_p
     lib.phyai_w8a8_project.argtypes = [_VP, _VP, _VP, C.c_uint32, C.c_uint32, C.c_uint32, _VP, _VP, _VP, _VP]
     lib.phyai_w8a8_last_error.restype = C.c_char_p
+    lib.phyai_project_features_kv.argtypes = [_VP, _VP, _VP, _VP, C.c_uint64, C.c_uint64, _VP, _VP]
     lib.phyai_batcher_create.argtypes = [C.POINTER(BatcherConfig), C.POINTER(_VP)]
     lib.phyai_batcher_destroy.argtypes = [_VP]
     lib.phyai_batcher_destroy.restype = None
@@ -345,6 +346,31 @@ def postprocess_actions(x: torch.Tensor, q01: Optional[torch.Tensor], q99: Optio
     out = torch.empty(B, out_horizon, out_dim, dtype=torch.float32, device=x.device)
     lo, hi = (clip if clip is not None else (0.0, 0.0))
     st = lib.phyai_postprocess_actions(_ptr(x), B, H, A, _ptr(q01), _ptr(q99), float(lo), float(hi), out_horizon, out_dim,
+                                       _ptr(out), _stream_ptr(stream))
+    if st != OK:
+        raise PhyaiError(st, lib.phyai_adapter_last_error().decode())
+    return out
+
+
+class KvProjDesc(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("n_layers", C.c_uint32), ("n_kv_heads", C.c_uint32), ("head_dim", C.c_uint32),
+                ("feat_dim", C.c_uint32)]
+
+
+def project_features_kv(features: torch.Tensor, wk, wv, n_kv_heads: int, head_dim: int, kv_tokens: Optional[int] = None,
+                        stream=None) -> torch.Tensor:
+    """Request-local K / V projections of a feature-handoff head (``phyai_project_features_kv``): ``features`` bf16
+    ``[tokens, Dv]``, ``wk`` / ``wv`` lists of bf16 ``[Dv, Hkv * dh]`` -> prefix KV bf16 ``[L, 2, kv_tokens, Hkv, dh]``."""
+    lib = load_library()
+    tokens, Dv = features.shape
+    L = len(wk)
+    kv_tokens = kv_tokens or tokens
+    out = torch.zeros(L, 2, kv_tokens, n_kv_heads, head_dim, dtype=torch.bfloat16, device=features.device)
+    desc = KvProjDesc(C.sizeof(KvProjDesc), L, n_kv_heads, head_dim, Dv)
+    ak, av = (_VP * L)(), (_VP * L)()
+    for l in range(L):
+        ak[l], av[l] = wk[l].data_ptr(), wv[l].data_ptr()
+    st = lib.phyai_project_features_kv(C.byref(desc), _ptr(features), C.cast(ak, _VP), C.cast(av, _VP), tokens, kv_tokens,
                                        _ptr(out), _stream_ptr(stream))
     if st != OK:
         raise PhyaiError(st, lib.phyai_adapter_last_error().decode())

@@ -59,6 +59,23 @@ __global__ void k_postprocess(const float* x, const float* q01, const float* q99
   }
 }
 
+
+// fp32 [tokens][2 * nkv] (K channels, then V channels) -> bf16 rows of the K plane and the V plane of one layer
+__global__ void k_kv_planes(const float* src, __nv_bfloat16* kplane, __nv_bfloat16* vplane, int tokens, int nkv) {
+  const size_t n = (size_t)tokens * (nkv >> 2) * 2;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int per_row = (nkv >> 2) * 2;
+    const int t = (int)(i / per_row), c4 = (int)(i % per_row);
+    const float4 v = *reinterpret_cast<const float4*>(src + (size_t)t * 2 * nkv + c4 * 4);
+    const int col = c4 * 4;
+    __nv_bfloat16* dst = col < nkv ? kplane + (size_t)t * nkv + col : vplane + (size_t)t * nkv + (col - nkv);
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst) = pk;
+  }
+}
+
 }  // namespace
 }  // namespace phyai
 
@@ -123,3 +140,60 @@ phyai_status_t phyai_postprocess_actions(const float* x, uint32_t batch, uint32_
 }
 
 }  // extern "C"
+
+// Request-local K / V projections of a feature-handoff head: per layer one tcgen05 GEMM of the (tiled) feature rows
+// against [Wk | Wv], fp32 out, then the bf16 rows of the two planes.  Runs once per request batch, ahead of the loop.
+extern "C" phyai_status_t phyai_project_features_kv(const phyai_kv_proj_desc_t* desc, const void* features,
+                                                    const void* const* wk, const void* const* wv, uint64_t tokens,
+                                                    uint64_t kv_tokens, void* prefix_kv, void* stream) {
+  using namespace phyai;
+  g_ad_err[0] = 0;
+  auto fail = [](phyai_status_t st, const char* msg, cudaError_t e = cudaSuccess) {
+    if (e != cudaSuccess) snprintf(g_ad_err, sizeof(g_ad_err), "%s: %s", msg, cudaGetErrorString(e));
+    else snprintf(g_ad_err, sizeof(g_ad_err), "%s", msg);
+    return st;
+  };
+  if (!desc || desc->struct_size != sizeof(phyai_kv_proj_desc_t) || !features || !wk || !wv || !prefix_kv)
+    return fail(PHYAI_ERR_INVALID_ARG, "NULL argument or wrong struct_size");
+  const int L = (int)desc->n_layers, nkv = (int)(desc->n_kv_heads * desc->head_dim), Dv = (int)desc->feat_dim;
+  if (L <= 0 || nkv <= 0 || Dv <= 0 || Dv % 64 || (2 * nkv) % 128 || tokens == 0 || tokens > kv_tokens || tokens > (1u << 22))
+    return fail(PHYAI_ERR_INVALID_ARG, "need feat_dim a multiple of 64, 2 * n_kv_heads * head_dim a multiple of 128, 1 <= tokens <= kv_tokens");
+  for (int l = 0; l < L; ++l)
+    if (!wk[l] || !wv[l]) return fail(PHYAI_ERR_INVALID_ARG, "a per-layer weight pointer is NULL");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cudaError_t e = tc_gemm_setup();
+  if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tc_gemm_setup", e);
+  const int M = (int)tokens, rows_pad = (M + 255) / 256 * 256, N = 2 * nkv;
+  __nv_bfloat16 *xt = nullptr, *wp = nullptr;
+  float* y = nullptr;
+  int* status = nullptr;
+  auto cleanup = [&]() { cudaFree(xt), cudaFree(wp), cudaFree(y), cudaFree(status); };
+  if ((e = cudaMalloc(&xt, (size_t)rows_pad * Dv * 2)) != cudaSuccess || (e = cudaMalloc(&wp, (size_t)Dv * N * 2)) != cudaSuccess ||
+      (e = cudaMalloc(&y, (size_t)M * N * 4)) != cudaSuccess || (e = cudaMalloc(&status, 4)) != cudaSuccess) {
+    cleanup();
+    return fail(PHYAI_ERR_OOM, "cudaMalloc", e);
+  }
+  cudaMemsetAsync(xt, 0, (size_t)rows_pad * Dv * 2, st);
+  cudaMemsetAsync(status, 0, 4, st);
+  launch_rows_to_tiled(reinterpret_cast<const __nv_bfloat16*>(features), xt, M, Dv, rows_pad, st);
+  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(prefix_kv);
+  for (int l = 0; l < L && e == cudaSuccess; ++l) {
+    launch_pack_tiled(wk[l], 1, wp, Dv, nkv, 0, st);
+    launch_pack_tiled(wv[l], 1, wp, Dv, nkv, nkv, st);
+    TcGemm g{};
+    g.W = wp, g.X = xt, g.M = M, g.N = N, g.K = Dv, g.epi = TC_STORE, g.out_f32 = y, g.ldo = N, g.splits = 1;
+    g.rows_pad = rows_pad, g.wait_limit = 1u << 28;
+    e = launch_tc_gemm(status, g, M <= 64 ? 64 : (M <= 1024 ? 128 : 256), st);
+    if (e != cudaSuccess) break;
+    const size_t n = (size_t)M * (nkv >> 2) * 2;
+    k_kv_planes<<<(int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096), 256, 0, st>>>(
+        y, out + ((size_t)l * 2) * kv_tokens * nkv, out + ((size_t)l * 2 + 1) * kv_tokens * nkv, M, nkv);
+  }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  int hs = 0;
+  if (e == cudaSuccess) e = cudaMemcpy(&hs, status, 4, cudaMemcpyDeviceToHost);
+  cleanup();
+  if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "feature K/V projection", e);
+  if (hs != 0) return fail(PHYAI_ERR_TIMEOUT, "a bounded device-side wait expired");
+  return PHYAI_OK;
+}

@@ -74,6 +74,8 @@ void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off
                        int il_second = 0, int perm_dh = 0, int wide = 0);
 // (wide: blocks [N/128][K/128][128][128] instead, the 16-byte chunks of a row XOR-swizzled by row & 7: the e4m3
 // operand image of the FP8 tensor path)
+// row-major bf16 [M][K] (K a multiple of 8, 16-byte aligned rows) -> the tiled bf16 layout of the GEMM inputs
+void launch_rows_to_tiled(const __nv_bfloat16* x, __nv_bfloat16* tiled, int M, int K, int rows_pad, cudaStream_t st);
 // Per-token e4m3 quantization of a tiled bf16 activation matrix [K/64][rows_pad][64] (W8A8): scale[r] = max|x_r| / 448
 // (1 for a zero row), codes = round-to-nearest-even e4m3 of x / scale, saturating, written as the tiled e4m3 matrix
 // [K/128][rows_pad][128] with the same 16-byte chunk swizzle.  Rows >= M are left alone.

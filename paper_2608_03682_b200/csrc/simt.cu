@@ -150,6 +150,20 @@ void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off
   k_pack_bytes<<<blocks, 256, 0, st>>>(src, dst, K, N, n_off, il_group, il_second, perm_dh, wide);
 }
 
+// row-major bf16 [M][K] -> tiled bf16 [K/64][rows_pad][64] (16-byte chunks XOR-swizzled by row & 7)
+__global__ void k_rows_to_tiled(const __nv_bfloat16* x, __nv_bfloat16* t, int M, int K, int rows_pad) {
+  const size_t n = (size_t)M * (K >> 3);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int row = (int)(i / (K >> 3)), c8 = (int)(i % (K >> 3));
+    const uint4 v = *reinterpret_cast<const uint4*>(x + (size_t)row * K + c8 * 8);
+    *reinterpret_cast<uint4*>(t + tiled_index(row, c8 * 8, rows_pad)) = v;
+  }
+}
+void launch_rows_to_tiled(const __nv_bfloat16* x, __nv_bfloat16* tiled, int M, int K, int rows_pad, cudaStream_t st) {
+  const size_t n = (size_t)M * (K >> 3);
+  k_rows_to_tiled<<<(int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096), 256, 0, st>>>(x, tiled, M, K, rows_pad);
+}
+
 // W8A8 activation quantization: one warp per token row.  A lane takes the 16-column groups lane, lane + 32, ... of
 // the row (two 16-byte chunks of the bf16 tile -> one 16-byte chunk of the e4m3 tile); the row stays in registers
 // between the maximum and the rounding.  The division by the scale is the IEEE one, so that the rounding decision

@@ -11,15 +11,6 @@
 namespace phyai {
 namespace {
 
-// row-major bf16 [M][K] -> tiled bf16 [K/64][rows_pad][64] (16-byte chunks XOR-swizzled by row & 7)
-__global__ void k_rows_to_tiled(const __nv_bfloat16* x, __nv_bfloat16* t, int M, int K, int rows_pad) {
-  const size_t n = (size_t)M * (K >> 3);
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-    const int row = (int)(i / (K >> 3)), c8 = (int)(i % (K >> 3));
-    const uint4 v = *reinterpret_cast<const uint4*>(x + (size_t)row * K + c8 * 8);
-    *reinterpret_cast<uint4*>(t + tiled_index(row, c8 * 8, rows_pad)) = v;
-  }
-}
 // tiled e4m3 [K/128][rows_pad][128] -> row-major codes [M][K]
 __global__ void k_codes_to_rows(const uint8_t* t, uint8_t* out, int M, int K, int rows_pad) {
   const size_t n = (size_t)M * (K >> 4);
@@ -71,7 +62,7 @@ extern "C" phyai_status_t phyai_w8a8_project(const void* x_bf16, const uint8_t* 
   cudaMemsetAsync(xq, 0, (size_t)rows_pad * K, st);
   cudaMemsetAsync(xs, 0, (size_t)rows_pad * 4, st);
   cudaMemsetAsync(status, 0, 4, st);
-  k_rows_to_tiled<<<256, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x_bf16), xt, (int)M, (int)K, rows_pad);
+  launch_rows_to_tiled(reinterpret_cast<const __nv_bfloat16*>(x_bf16), xt, (int)M, (int)K, rows_pad, st);
   launch_quant_rows(status, xt, xq, xs, rows_pad, (int)M, (int)K, st);
   launch_pack_bytes(w_codes, wp, (int)K, (int)N, 0, st, 0, 0, 0, 1);
   TcGemm g{};

@@ -202,6 +202,33 @@ def make_noise(cfg: ExpertConfig, cfg_id: int, request: int = 0) -> torch.Tensor
     return _normal(_rng(cfg_id, STREAM_NOISE, request), (cfg.horizon, cfg.action_dim), 1.0)
 
 
+STREAM_FEATURES, STREAM_KV_PROJ = 6, 7
+
+
+def make_features(cfg_id: int, tokens: int, feat_dim: int, request: int = 0) -> torch.Tensor:
+    """Vision-language feature rows of one request for a feature-handoff head, ``[tokens, feat_dim]`` ~N(0,1), bf16."""
+    return _normal(_rng(cfg_id, STREAM_FEATURES, request), (tokens, feat_dim), 1.0).to(torch.bfloat16)
+
+
+def make_kv_projections(cfg: ExpertConfig, cfg_id: int, feat_dim: int):
+    """Per-layer request-local K / V projection matrices ``[feat_dim, Hkv * dh]`` ~N(0, feat_dim^-1/2), bf16: the
+    projected keys and values then have unit scale like the synthetic prefix KV of the other workloads."""
+    rng = _rng(cfg_id, STREAM_KV_PROJ)
+    std = float(feat_dim) ** -0.5
+    wk = [_normal(rng, (feat_dim, cfg.kv_dim), std).to(torch.bfloat16) for _ in range(cfg.n_layers)]
+    wv = [_normal(rng, (feat_dim, cfg.kv_dim), std).to(torch.bfloat16) for _ in range(cfg.n_layers)]
+    return wk, wv
+
+
+def groot_like_config(max_batch: int = 1, n_layers: int = 16, max_prefix_len: int = 640) -> ExpertConfig:
+    """A feature-handoff action head of the shape the paper's GR00T profile names (action chunk 40 x 132, four
+    flow-matching steps); the paper gives no widths for it, so the transformer dimensions are this repository's
+    choice: width 1024, MLP 4096, 8 query heads on 2 kv heads of 128, no rotary embedding on the feature keys."""
+    return ExpertConfig(n_layers=n_layers, width=1024, mlp_dim=4096, n_q_heads=8, n_kv_heads=2, head_dim=128, state_dim=64,
+                        action_dim=132, horizon=40, has_state_token=True, max_prefix_len=max_prefix_len, max_batch=max_batch,
+                        cond="pi0", dtype="bf16", rope_theta=0.0)
+
+
 def make_ragged_lengths(cfg_id: int, batch: int, lo: int, hi: int) -> np.ndarray:
     """``batch`` prefix lengths, integers uniform on [lo, hi] inclusive."""
     return _rng(cfg_id, STREAM_LENS).integers(lo, hi + 1, size=batch).astype(np.int32)

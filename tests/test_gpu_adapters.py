@@ -5,6 +5,7 @@ import pytest
 import torch
 
 from oracle import adapter_oracle as A
+from oracle import expert_oracle as O
 from paper_2608_03682_b200 import binding, synth
 
 pytestmark = pytest.mark.gpu
@@ -101,3 +102,52 @@ def test_frontend_worker_pads_the_local_batch_to_its_fixed_shape():
     for rid, r in zip(ids, reqs):
         ref = O.denoise(cfg, Wf, r["prefix_kv"], r["prefix_kv"].shape[2], r["state"], r["noise"], 3)
         assert rel_err(out[rid], ref) <= BAR["bf16"], (rid, rel_err(out[rid], ref))
+
+
+# ------------------------------------------------------------------ feature-handoff head: request-local K / V projections
+@pytest.mark.parametrize("tokens,feat_dim,n_kv,dh,layers", [(300, 512, 2, 128, 3), (37, 1024, 1, 256, 2), (1500, 256, 2, 64, 2)])
+def test_feature_projection_matches_oracle(tokens, feat_dim, n_kv, dh, layers):
+    cfg = synth.ExpertConfig(n_layers=layers, width=256, mlp_dim=512, n_q_heads=2 * n_kv, n_kv_heads=n_kv, head_dim=dh,
+                             state_dim=4, action_dim=4, horizon=4, has_state_token=True, max_prefix_len=tokens, max_batch=1,
+                             cond="pi0", dtype="bf16")
+    F = synth.make_features(41, tokens, feat_dim)
+    wk, wv = synth.make_kv_projections(cfg, 41, feat_dim)
+    got = binding.project_features_kv(F.cuda(), [w.cuda() for w in wk], [w.cuda() for w in wv], n_kv, dh, kv_tokens=tokens + 5)
+    torch.cuda.synchronize()
+    ref = A.project_features_kv(F.double().numpy(), [w.double().numpy() for w in wk], [w.double().numpy() for w in wv], n_kv, dh)
+    g = got.double().cpu().numpy()
+    assert np.all(g[:, :, tokens:] == 0)                      # rows past `tokens` are left alone
+    err = np.abs(g[:, :, :tokens] - ref)
+    # bf16 storage of an fp32-accumulated product: half an ulp (2^-9 relative) plus accumulation noise
+    assert np.all(err <= np.abs(ref) * 2.0 ** -8 + 1e-4), float(err.max())
+
+
+@pytest.mark.parametrize("batch", [1, 3])
+def test_feature_handoff_head_end_to_end(batch):
+    """Projected features as the loop's prefix KV: the device projects and denoises (four steps, 40 x 132 chunk); the
+    oracle projects in float64, stores bf16 and denoises.  Reduced depth so that the oracle stays fast."""
+    cfg = synth.groot_like_config(max_batch=batch, n_layers=4, max_prefix_len=400)
+    W = synth.make_weights(cfg, 42)
+    feat_dim = 768
+    wk, wv = synth.make_kv_projections(cfg, 42, feat_dim)
+    lens = [400, 123, 256][:batch]
+    feats = [synth.make_features(42, n, feat_dim, b) for b, n in enumerate(lens)]
+    states = torch.stack([synth.make_state(cfg, 42, b) for b in range(batch)])
+    noise = torch.stack([synth.make_noise(cfg, 42, b) for b in range(batch)])
+    cu = np.zeros(batch + 1, dtype=np.int32)
+    cu[1:] = np.cumsum(lens)
+    kv = binding.project_features_kv(torch.cat(feats).cuda(), [w.cuda() for w in wk], [w.cuda() for w in wv], cfg.n_kv_heads,
+                                     cfg.head_dim)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        out = ex.denoise_batched(kv, torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), 4)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        out = out.double().cpu().numpy()
+    for b in range(batch):
+        kv_ref = A.project_features_kv(feats[b].double().numpy(), [w.double().numpy() for w in wk],
+                                       [w.double().numpy() for w in wv], cfg.n_kv_heads, cfg.head_dim)
+        kv_ref = torch.from_numpy(kv_ref).to(torch.bfloat16)          # the layout stores bf16
+        ref = O.denoise(cfg, W, kv_ref, lens[b], states[b], noise[b], 4)
+        err = O.max_rel_err(out[b], ref)
+        print(f"feature-handoff head, request {b}: max rel err {err:.2e}")
+        assert err <= 2e-2, (b, err)
