@@ -128,6 +128,40 @@ def test_full_width_two_layer_expert_through_the_fused_attention_projection(cond
                 assert err <= BAR["bf16"], (P, cluster_gemm, fused, err)
 
 
+@pytest.mark.parametrize("cond", ["pi0", "pi05"])
+@pytest.mark.parametrize("block_causal", [False, True])
+def test_full_width_several_short_requests_share_the_single_tile_path(cond, block_causal):
+    """Width 1024 with several requests whose suffix tokens together fit one 64-token tile: the cluster kernels, the
+    step-boundary kernel (token row -> request, action row) and the cluster attention kernel (two heads per CTA, since
+    8 x heads x requests CTAs do not fit) all see more than one request; ragged prefixes including an empty one."""
+    if block_causal and cond == "pi05":
+        pytest.skip("the block-causal mask concerns the state token, which pi0.5 has not")
+    cfg = synth.ExpertConfig(n_layers=2, width=1024, mlp_dim=4096, n_q_heads=8, n_kv_heads=1, head_dim=256,
+                             state_dim=32, action_dim=32, horizon=11, has_state_token=(cond == "pi0"),
+                             max_prefix_len=400, max_batch=4, cond=cond, dtype="bf16", suffix_block_causal=block_causal)
+    lens = [400, 0, 33, 257]
+    W = synth.make_weights(cfg, 24)
+    kvs = [synth.make_prefix_kv(cfg, 24, p, b) if p else synth.make_prefix_kv(cfg, 24, 1, b)[:, :, :0] for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    states = torch.stack([synth.make_state(cfg, 24, b) for b in range(4)]) if cfg.has_state_token else None
+    noise = torch.stack([synth.make_noise(cfg, 24, b) for b in range(4)])
+    Wf = O.Weights(W)
+    refs = [O.denoise(cfg, Wf, kvs[b], lens[b], None if states is None else states[b], noise[b], 3) for b in range(4)]
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        for opts in ({}, {"use_state_cache": 1}, {"use_b1_step": 0}, {"b1_attn_hpc": 2}):
+            for k, v in opts.items():
+                ex.set_option(k, v)
+            out = ex.denoise_batched(packed.cuda(), torch.from_numpy(cu).cuda(), None if states is None else states.cuda(),
+                                     noise.cuda(), 3)
+            torch.cuda.synchronize()
+            assert ex.poll_status() == 0
+            out = out.double().cpu().numpy()
+            for b in range(4):
+                assert rel_err(out[b], refs[b]) <= BAR["bf16"], (opts, b, rel_err(out[b], refs[b]))
+            for k in opts:
+                ex.set_option(k, 1 if k == "use_b1_step" else 0)
+
+
 # ------------------------------------------------------------------------------------------ batched, ragged
 def _batched_case(cfg, cfg_id, lens, n_steps, check, engine="auto", std=0.05):
     W = synth.make_weights(cfg, cfg_id, std=std)
