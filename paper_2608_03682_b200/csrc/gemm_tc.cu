@@ -31,8 +31,6 @@
 // Every wait is bounded: on expiry of the caller's limit the CTA raises the status word and skips its MMAs and
 // stores, but keeps the copy / commit pipeline running under a generous limit of its own, so that every copy
 // into its shared memory has landed before it exits (TMEM is always released).
-#include <type_traits>
-
 #include "kernels.h"
 #include "ptx.cuh"
 #include "tc.cuh"
@@ -47,7 +45,9 @@ constexpr int BAR_EPI = 1;
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync %0, %1;" ::"n"(BAR_EPI), "n"(NEPI) : "memory"); }
 
-template <int NT, int NA, int STAGES>
+// F8: e4m3 operands (kind::f8f6f4) and per-token activation scales, a kernel of its own so that the bf16 kernel carries
+// none of it.
+template <int NT, int NA, int STAGES, bool F8 = false>
 __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g) {
   constexpr int B_BYTES = NT * 128;
   constexpr int NB = NT > 128 ? NT / 128 : 1;          // the activation tile is copied in pieces of <= 16 KB
@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int nt_idx = blockIdx.x, tt = blockIdx.y;
   const bool geglu = g.epi == TC_GEGLU;
-  const int KC = g.fp8 ? g.K >> 7 : g.K >> 6;   // k-chunks of 128 bytes per operand row
+  const int KC = F8 ? g.K >> 7 : g.K >> 6;   // k-chunks of 128 bytes per operand row
   const int kc_begin = (int)(((long long)KC * blockIdx.z) / gridDim.z);
   const int kc_end = (int)(((long long)KC * (blockIdx.z + 1)) / gridDim.z);
   const int nk = kc_end - kc_begin;
@@ -203,47 +203,41 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     // ---------------- MMA issuer(s) (whole warp in the loop, one elected lane issues) ---------------------
     const int first = DUAL ? warp - 8 : 0, step = DUAL ? 2 : 1;
     const uint32_t tacc = tmem_base + (DUAL ? (uint32_t)(warp - 8) * NT : 0u);
-    // (the operand kind is fixed per launch: the loop exists once per kind, so that the issue sequence of a k-step,
-    // which paces small tiles, carries no test of it)
-    auto main_loop = [&](auto f8) {
-      for (int i = first; i < nk; i += step) {
-        const int s = i % STAGES;
-        const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        const bool ok = mbar_wait_drain(smem_u32(&bar_full[s]), ph, wc) > 0;
-        // (no tcgen05 fence here: the operands were written by the bulk-copy engine and made visible by the mbarrier;
-        // tcgen05.fence::after_thread_sync orders tensor-memory accesses, and it was measured to hold the next MMAs
-        // back until the previous stage's MMAs had drained)
-        const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
-        const uint64_t da = make_desc(a0);
-        const uint64_t da2 = make_desc(a0 + A_BYTES);
-        const uint64_t db = make_desc(a0 + A_BYTES * NA);
-        // control flow and descriptors stay warp-uniform; only the tcgen05 instructions themselves are predicated on
-        // the elected lane
-        if (__all_sync(0xffffffffu, ok)) {
-  #pragma unroll
-          for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
-            const uint32_t acc = (i > first || k > 0) ? 1u : 0u;   // the warp's first MMA initialises its accumulator
-            if constexpr (decltype(f8)::value) {
-              if (elect_one()) umma_f8(tacc, da + 2 * k, db + 2 * k, IDESC_F8, acc);
-              if (NA == 2) {
-                if (elect_one()) umma_f8(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC_F8, acc);
-              }
-            } else {
-              if (elect_one()) umma_bf16(tacc, da + 2 * k, db + 2 * k, IDESC, acc);
-              if (NA == 2) {
-                if (elect_one()) umma_bf16(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
-              }
+    for (int i = first; i < nk; i += step) {
+      const int s = i % STAGES;
+      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+      const bool ok = mbar_wait_drain(smem_u32(&bar_full[s]), ph, wc) > 0;
+      // (no tcgen05 fence here: the operands were written by the bulk-copy engine and made visible by the mbarrier;
+      // tcgen05.fence::after_thread_sync orders tensor-memory accesses, and it was measured to hold the next MMAs
+      // back until the previous stage's MMAs had drained)
+      const uint32_t a0 = tiles + (uint32_t)s * STAGE_BYTES;
+      const uint64_t da = make_desc(a0);
+      const uint64_t da2 = make_desc(a0 + A_BYTES);
+      const uint64_t db = make_desc(a0 + A_BYTES * NA);
+      // control flow and descriptors stay warp-uniform; only the tcgen05 instructions themselves are predicated on
+      // the elected lane
+      if (__all_sync(0xffffffffu, ok)) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {  // 4 x (K = 16) per 64-wide chunk: +32 bytes = +2 descriptor units
+          const uint32_t acc = (i > first || k > 0) ? 1u : 0u;   // the warp's first MMA initialises its accumulator
+          if constexpr (F8) {
+            if (elect_one()) umma_f8(tacc, da + 2 * k, db + 2 * k, IDESC_F8, acc);
+            if (NA == 2) {
+              if (elect_one()) umma_f8(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC_F8, acc);
+            }
+          } else {
+            if (elect_one()) umma_bf16(tacc, da + 2 * k, db + 2 * k, IDESC, acc);
+            if (NA == 2) {
+              if (elect_one()) umma_bf16(tacc + NT, da2 + 2 * k, db + 2 * k, IDESC, acc);
             }
           }
         }
-        // frees the stage when the MMAs above have read it -- only if a later k-step will reuse the stage (a commit
-        // that nobody waits for still costs the issuing thread time)
-        if (i + STAGES < nk && elect_one()) umma_commit(smem_u32(&bar_empty[s]));
-        __syncwarp();
       }
-    };
-    if (g.fp8) main_loop(std::true_type{});
-    else main_loop(std::false_type{});
+      // frees the stage when the MMAs above have read it -- only if a later k-step will reuse the stage (a commit
+      // that nobody waits for still costs the issuing thread time)
+      if (i + STAGES < nk && elect_one()) umma_commit(smem_u32(&bar_empty[s]));
+      __syncwarp();
+    }
     if (elect_one()) umma_commit(smem_u32(&bar_accum));
     __syncwarp();
   }
@@ -269,14 +263,14 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] += w[j];
       }
-      if (g.xscale) {
+      if constexpr (F8) {
         const float* xs = xs_tab + (col % (uint32_t)NT);
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] *= xs[j];
       }
     };
     float xs_reg = 0.f;
-    if (g.xscale && et < NT && tok_base + et < g.M) xs_reg = g.xscale[tok_base + et];
+    if (F8 && et < NT && tok_base + et < g.M) xs_reg = g.xscale[tok_base + et];
     if (g.epi == TC_QKV_ROT) {
       // while the main loop runs: where each token of the tile sits (request, suffix row, rotary position)
       for (int idx = et; idx < NT; idx += NEPI) {
@@ -343,7 +337,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     epi_sync();
     const bool ok = *reinterpret_cast<volatile int*>(&epi_ok) != 0;
     tc_fence_after();
-    if (g.xscale) {
+    if constexpr (F8) {
       if (et < NT) xs_tab[et] = xs_reg;
       epi_sync();
     }
@@ -599,7 +593,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
           float vg[16], vu[16];
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, vg);
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(NT + c0), vu);
-          if (g.xscale) {
+          if constexpr (F8) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) vg[j] *= xs_tab[c0 + j], vu[j] *= xs_tab[c0 + j];
           }
@@ -640,12 +634,19 @@ constexpr size_t smem_bytes() {
 template <int NT, int NA, int STAGES>
 cudaError_t launch_one(int* status, const TcGemm& g, cudaStream_t st) {
   dim3 grid(g.N / 128 / (g.epi == TC_GEGLU ? 1 : NA), (g.M + NT - 1) / NT, g.splits > 0 ? g.splits : 1);
-  return launch_pdl(k_gemm_tc<NT, NA, STAGES>, grid, dim3(800), smem_bytes<NT, NA, STAGES>(), st, status, g);
+  if (g.fp8) {
+    if (!g.xscale) return cudaErrorInvalidValue;
+    return launch_pdl(k_gemm_tc<NT, NA, STAGES, true>, grid, dim3(800), smem_bytes<NT, NA, STAGES>(), st, status, g);
+  }
+  return launch_pdl(k_gemm_tc<NT, NA, STAGES, false>, grid, dim3(800), smem_bytes<NT, NA, STAGES>(), st, status, g);
 }
 
 template <int NT, int NA, int STAGES>
 cudaError_t setup_one() {
-  return cudaFuncSetAttribute(k_gemm_tc<NT, NA, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<NT, NA, STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem_bytes<NT, NA, STAGES>());
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_gemm_tc<NT, NA, STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)smem_bytes<NT, NA, STAGES>());
 }
 

@@ -542,7 +542,7 @@ __global__ void k_rmsnorm_tiled4(const int* status, float* h, const float* gain,
 // row is read once.
 // With out8 set (W8A8) the normalised row leaves as its per-token e4m3 quantization instead (codes in the tiled e4m3
 // layout, scale in xscale[row]): the bf16 rounding of every element is what gets quantized, as in k_quant_rows.
-template <int NV>
+template <int NV, bool Q8>
 __global__ void k_rmsnorm_tiled_reg(const int* status, float* h, const float* gain, const float* shift,
                                     __nv_bfloat16* out, int rows_pad, int M, float eps, SlabSum sl, uint8_t* out8,
                                     float* xscale) {
@@ -583,7 +583,7 @@ __global__ void k_rmsnorm_tiled_reg(const int* status, float* h, const float* ga
       o.x += s4.x, o.y += s4.y, o.z += s4.z, o.w += s4.w;
     }
     __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
-    if (out8) {   // keep the bf16-rounded values for the quantization below
+    if constexpr (Q8) {   // keep the bf16-rounded values for the quantization below
       v[k] = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
       continue;
     }
@@ -591,7 +591,7 @@ __global__ void k_rmsnorm_tiled_reg(const int* status, float* h, const float* ga
     pk.x = *reinterpret_cast<uint32_t*>(&lo), pk.y = *reinterpret_cast<uint32_t*>(&hi);
     *reinterpret_cast<uint2*>(out + tiled_index(row, d, rows_pad)) = pk;
   }
-  if (out8) {
+  if constexpr (Q8) {
     float amax = 0.f;
 #pragma unroll
     for (int k = 0; k < NV; ++k) amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v[k].x), fabsf(v[k].y)), fmaxf(fabsf(v[k].z), fabsf(v[k].w))));
@@ -673,13 +673,21 @@ void launch_rmsnorm(const int* status, float* h, const float* gain, const float*
   const int wpb = sl.n ? 1 : 4;
   const int blocks = (M + wpb - 1) / wpb;
   if (out_tiled && D == 1024) {
-    launch_pdl(k_rmsnorm_tiled_reg<8>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl, out8,
-               xscale);
+    if (out8)
+      launch_pdl(k_rmsnorm_tiled_reg<8, true>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps,
+                 sl, out8, xscale);
+    else
+      launch_pdl(k_rmsnorm_tiled_reg<8, false>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps,
+                 sl, out8, xscale);
     return;
   }
   if (out_tiled && D == 2048) {
-    launch_pdl(k_rmsnorm_tiled_reg<16>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps, sl, out8,
-               xscale);
+    if (out8)
+      launch_pdl(k_rmsnorm_tiled_reg<16, true>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps,
+                 sl, out8, xscale);
+    else
+      launch_pdl(k_rmsnorm_tiled_reg<16, false>, dim3(blocks), dim3(32 * wpb), 0, st, status, h, gain, shift, out_tiled, rows_pad, M, eps,
+                 sl, out8, xscale);
     return;
   }
   if (out_tiled && D % 128 == 0) {
