@@ -57,10 +57,25 @@ def decode_e4m3(codes: np.ndarray) -> np.ndarray:
     return (sign * val).astype(F64)
 
 
+def decode_int4(packed) -> np.ndarray:
+    """W4A16 storage (quantization paragraph: W4A16, round-to-nearest; the format is a reading): a byte holds the
+    codes of two neighbouring output channels of one input row, the even channel in the low nibble; a code c in 0..15
+    stands for the integer c - 8.  ``[in, out / 2]`` bytes -> ``[in, out]`` float64 integers in [-8, 7]."""
+    b = packed.numpy() if hasattr(packed, "numpy") else np.asarray(packed)
+    b = b.astype(np.int64)
+    out = np.empty((b.shape[0], 2 * b.shape[1]), dtype=F64)
+    out[:, 0::2] = (b & 15) - 8
+    out[:, 1::2] = (b >> 4) - 8
+    return out
+
+
 def to_f64(t) -> np.ndarray:
     """Stored tensor -> float64 array, exactly.  Accepts numpy arrays, torch tensors (f32/bf16)
-    and ``(codes_uint8[in,out], scales_f32[out])`` pairs of the W8A16 / W8A8 modes, which decode to
+    and ``(codes_uint8[in,out], scales_f32[out])`` pairs of the W8A16 / W8A8 modes (and ``(packed, scales, "int4")``
+    triples of the W4A16 mode), which decode to
     ``decode(code) * scale`` per output channel (column)."""
+    if isinstance(t, tuple) and len(t) == 3 and t[2] == "int4":
+        return decode_int4(t[0]) * to_f64(t[1])[None, :]
     if isinstance(t, tuple):
         codes, scales = t
         codes = codes.numpy() if hasattr(codes, "numpy") else np.asarray(codes)

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libphyai.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(6)
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "OOM", 4: "CUDA", 5: "TIMEOUT"}
-DTYPES = {"f32": 0, "bf16": 1, "w8e4m3": 2, "w8a8e4m3": 3}
+DTYPES = {"f32": 0, "bf16": 1, "w8e4m3": 2, "w8a8e4m3": 3, "w4a16": 4}
 CONDS = {"pi0": 0, "pi05": 1}
 ENGINES = {"auto": 0, "simt": 1}
 BIG = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
@@ -205,7 +205,7 @@ class Expert:
                     arr[l] = dev(w)
             keep.append(arr)
             setattr(ws, n, C.cast(arr, _VPP))
-        if cfg.dtype in ("w8e4m3", "w8a8e4m3"):
+        if cfg.dtype in ("w8e4m3", "w8a8e4m3", "w4a16"):
             for i, m in enumerate(BIG):
                 keep.append(scale_arrays[m])
                 ws.scales[i] = C.cast(scale_arrays[m], _VPP)

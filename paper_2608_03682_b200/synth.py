@@ -4,7 +4,8 @@ This module only *describes shapes* and *draws random numbers*.  It contains non
 method's arithmetic (no norm, attention, embedding or solver code), so both the CPU oracle's
 tests and the CUDA path's tests can take their inputs from here without sharing any
 computation.  The only numeric transformations are storage casts done by library routines:
-round-to-nearest-even float32 -> bfloat16 and float32 -> float8_e4m3fn (PyTorch casts).
+round-to-nearest-even float32 -> bfloat16, float32 -> float8_e4m3fn (PyTorch casts) and float32 -> 4-bit integers
+(``torch.round`` and a clamp) with one scale per output channel.
 
 Shapes follow the paper's pi0 / pi0.5 serving workloads (three camera views, a 50-action
 chunk, ten Euler steps, bf16; Sec. "Results", batch sweep) with random-initialised weights:
@@ -44,8 +45,8 @@ class ExpertConfig:
     max_prefix_len: int
     max_batch: int = 1
     cond: str = "pi0"            # "pi0": time concatenated into the action MLP; "pi05": adaRMSNorm
-    dtype: str = "bf16"          # "f32" | "bf16" | "w8e4m3" | "w8a8e4m3" (storage of weights and prefix KV; the last
-                                 # also names the arithmetic of the seven large projections: e4m3 x e4m3)
+    dtype: str = "bf16"          # "f32" | "bf16" | "w8e4m3" | "w8a8e4m3" | "w4a16" (storage of weights and prefix KV; the last
+                                 # "w8a8e4m3" also names the arithmetic of the seven large projections: e4m3 x e4m3)
     rms_eps: float = 1e-6
     rope_theta: float = 10000.0  # 0 disables RoPE
     time_min_period: float = 4e-3
@@ -170,6 +171,19 @@ def quantize_e4m3_columns(w: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
     return q.view(torch.uint8).contiguous(), scale.contiguous()
 
 
+def quantize_int4_columns(w: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor, str]:
+    """Round-to-nearest per-output-channel symmetric int4 storage of a float32 ``[in, out]`` matrix (``out`` even).
+
+    Returns (packed uint8 ``[in, out / 2]``, float32 scales ``[out]``, the tag ``"int4"``): ``scale = max|column| / 7``
+    (1 for an all-zero column), integer ``q = clamp(round_half_even(w / scale), -8, 7)``, stored as the code ``q + 8``;
+    a byte holds two neighbouring output channels of one input row, the even channel in the low nibble."""
+    amax = w.abs().amax(dim=0)
+    scale = torch.where(amax > 0, amax / 7.0, torch.ones_like(amax)).to(torch.float32)
+    q = torch.round(w / scale).clamp_(-8, 7).to(torch.int16) + 8          # torch.round: half to even
+    packed = (q[:, 0::2] | (q[:, 1::2] << 4)).to(torch.uint8)
+    return packed.contiguous(), scale.contiguous(), "int4"
+
+
 def make_weights(cfg: ExpertConfig, cfg_id: int, std: float = 0.02) -> Dict[str, object]:
     """All weights of one expert, ~N(0, std) in float32, cast to the configuration's storage.
 
@@ -182,6 +196,8 @@ def make_weights(cfg: ExpertConfig, cfg_id: int, std: float = 0.02) -> Dict[str,
         base = name.split(".")[0]
         if cfg.dtype in ("w8e4m3", "w8a8e4m3") and base in BIG_MATS:
             W[name] = quantize_e4m3_columns(master)
+        elif cfg.dtype == "w4a16" and base in BIG_MATS:
+            W[name] = quantize_int4_columns(master)
         else:
             W[name] = _store(master, "f32" if cfg.dtype == "f32" else "bf16")
     return W

@@ -114,3 +114,35 @@ def test_w8a8_network_stays_close_to_the_w8a16_network(cond):
     b = O.denoise(cfg16, W, kv, 9, state, noise, 3)
     d = O.max_rel_err(a, b)
     assert 0.0 < d < 0.2, d
+
+
+# ------------------------------------------------------------------------------------------------ W4A16 storage
+def test_int4_decode_every_code_and_the_nibble_order_by_hand():
+    # byte 0x1F: low nibble 15 -> +7 (even channel), high nibble 1 -> -7 (odd channel); 0x80: (0 -> -8, 8 -> 0)
+    packed = np.array([[0x1F, 0x80], [0x98, 0x07]], dtype=np.uint8)
+    assert np.array_equal(O.decode_int4(packed), [[7.0, -7.0, -8.0, 0.0], [0.0, 1.0, -1.0, -8.0]])
+    allc = np.array([[(hi << 4) | lo for lo in range(16)] for hi in range(16)], dtype=np.uint8)
+    dec = O.decode_int4(allc)
+    assert np.array_equal(dec[:, 0::2], np.tile(np.arange(16) - 8.0, (16, 1)))
+    assert np.array_equal(dec[:, 1::2], np.tile((np.arange(16) - 8.0)[:, None], (1, 16)))
+
+
+def test_int4_column_quantizer_is_round_to_nearest_within_half_a_step():
+    rng = np.random.default_rng(9)
+    w = torch.from_numpy(rng.standard_normal((64, 10)).astype(np.float32))
+    w[:, 3] = 0.0                                                   # an all-zero column: scale 1, codes 8
+    w[0, 4], w[1, 4], w[2, 4], w[3, 4] = 7.0, 0.5, 1.5, -7.6        # column maximum 7.6... see below
+    packed, scales, tag = synth.quantize_int4_columns(w)
+    assert tag == "int4" and packed.shape == (64, 5) and packed.dtype == torch.uint8
+    deq = O.to_f64((packed, scales, tag))
+    s = scales.double().numpy()
+    assert s[3] == 1.0 and np.all(deq[:, 3] == 0.0)
+    assert np.allclose(s, np.maximum(w.abs().amax(dim=0).double().numpy(), 0) / 7.0 + (s == 1.0) * 1.0, rtol=1e-6)
+    assert np.all(np.abs(deq - w.double().numpy()) <= s[None, :] / 2 * (1 + 1e-6))
+    ints = deq / s[None, :]
+    assert np.all(np.abs(ints - np.rint(ints)) < 1e-9) and ints.min() >= -8 and ints.max() <= 7
+    # ties go to the even integer: with scale 1 (column maximum 7) 0.5 -> 0, 1.5 -> 2, 2.5 -> 2, -0.5 -> 0
+    t = torch.tensor([[7.0], [0.5], [1.5], [2.5], [-0.5], [-7.0]])
+    t = torch.cat([t, torch.zeros_like(t)], dim=1)
+    p2, s2, _ = synth.quantize_int4_columns(t)
+    assert np.array_equal(O.to_f64((p2, s2, "int4"))[:, 0], [7.0, 0.0, 2.0, 2.0, 0.0, -7.0])
