@@ -53,11 +53,17 @@ typedef enum {
   PHYAI_W8E4M3_A16 = 2, /* the seven large per-layer matrices as e4m3 bytes with one fp32 scale per
                           output channel (offline round-to-nearest, quantization paragraph); all other
                           tensors and the prefix KV bfloat16; activations bf16                        */
-  PHYAI_W8A8_E4M3 = 3  /* storage as PHYAI_W8E4M3_A16; in addition the input of each of the four large
+  PHYAI_W8A8_E4M3 = 3, /* storage as PHYAI_W8E4M3_A16; in addition the input of each of the four large
                           projections of a layer (fused QKV, attention output, gate / up, down) is
                           quantised per token to e4m3 -- scale = max|x| / 448, codes round-to-nearest-even,
                           saturating -- and the products run on the FP8 tensor path (quantization
                           paragraph: W8A8).  Tensor path only; kernels of the general (any batch) family */
+  PHYAI_W4A16 = 4      /* the seven large per-layer matrices as symmetric 4-bit integers with one fp32 scale per
+                          output channel (quantization paragraph: W4A16, round-to-nearest): a byte of the
+                          [in][out / 2] array holds the codes of output channels 2j (low nibble) and 2j + 1
+                          (high nibble) of one input row, code c = integer c - 8 in [-8, 7], weight = integer x
+                          scale; everything else as PHYAI_W8E4M3_A16.  The integers are expanded to bf16 operand
+                          images at create (exact), the scales enter in the epilogues                        */
 } phyai_dtype_t;
 
 /* How the time t_k conditions the expert. */

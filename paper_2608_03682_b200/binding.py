@@ -290,7 +290,10 @@ def weights_to_device(weights: Dict[str, object], device="cuda") -> Dict[str, ob
     """Copy a generated weight dictionary to the device (tuples element-wise)."""
     out = {}
     for k, v in weights.items():
-        out[k] = tuple(t.to(device).contiguous() for t in v) if isinstance(v, tuple) else v.to(device).contiguous()
+        if isinstance(v, tuple):   # (codes, scales) or (packed codes, scales, format tag)
+            out[k] = tuple(t.to(device).contiguous() if hasattr(t, "to") else t for t in v)
+        else:
+            out[k] = v.to(device).contiguous()
     return out
 
 

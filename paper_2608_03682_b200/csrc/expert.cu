@@ -172,7 +172,7 @@ phyai_status_t check_config(const phyai_expert_config_t* c) {
     return fail(PHYAI_ERR_INVALID_ARG, "has_state_token / state_dim inconsistent");
   if (c->n_q_heads % c->n_kv_heads) return fail(PHYAI_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
   if ((c->head_dim & 1) || (c->width & 1)) return fail(PHYAI_ERR_INVALID_ARG, "head_dim and width must be even");
-  if (c->cond > PHYAI_COND_PI05_ADARMS || c->dtype > PHYAI_W8A8_E4M3 || c->engine > PHYAI_ENGINE_SIMT)
+  if (c->cond > PHYAI_COND_PI05_ADARMS || c->dtype > PHYAI_W4A16 || c->engine > PHYAI_ENGINE_SIMT)
     return fail(PHYAI_ERR_INVALID_ARG, "unknown cond / dtype / engine value");
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta >= 0.f) || !(c->time_min_period > 0.f) || !(c->time_max_period > 0.f))
     return fail(PHYAI_ERR_INVALID_ARG, "rms_eps / rope_theta / time periods out of range");
@@ -743,7 +743,10 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         !w->norm2[l] || (ada && (!w->norm1_b[l] || !w->norm2_b[l])))
       return fail(PHYAI_ERR_INVALID_ARG, "a per-layer weight pointer is NULL (layer %u)", l);
   const bool a8 = cfg->dtype == PHYAI_W8A8_E4M3;     // e4m3 activations as well: the FP8 tensor path
-  const bool w8 = cfg->dtype == PHYAI_W8E4M3_A16 || a8;
+  const bool w4 = cfg->dtype == PHYAI_W4A16;        // int4 codes + scales, expanded to bf16 images at create
+  if (w4 && ((cfg->n_q_heads * cfg->head_dim) % 2 || (cfg->n_kv_heads * cfg->head_dim) % 2 || cfg->width % 2 || cfg->mlp_dim % 2))
+    return fail(PHYAI_ERR_INVALID_ARG, "PHYAI_W4A16 stores two output channels per byte: output widths must be even");
+  const bool w8 = cfg->dtype == PHYAI_W8E4M3_A16 || a8 || w4;   // per-output-channel scales
   if (a8 && !tc) return fail(PHYAI_ERR_UNSUPPORTED, "PHYAI_W8A8_E4M3 runs on the tensor path only (engine AUTO)");
   if (a8 && (cfg->width % 128 || cfg->mlp_dim % 128 || (cfg->n_q_heads * cfg->head_dim) % 128 || cfg->mlp_dim > 4096 ||
              cfg->width > 4096 || cfg->n_q_heads * cfg->head_dim > 4096))
@@ -767,7 +770,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
   h->sites = 2 * d.L + 1;
   h->Mpad = (int)(((size_t)cfg->max_batch * d.S + 255) / 256 * 256);
   const int D = d.D, L = d.L, kind = kind_of(cfg->dtype);     // storage of non-quantised tensors
-  const int big_kind = w8 ? 2 : kind;                         // storage of the seven big matrices
+  const int big_kind = w4 ? 3 : (w8 ? 2 : kind);              // storage of the seven big matrices
   const size_t Mp = h->Mpad;
 
   auto body = [&]() -> phyai_status_t {
@@ -907,7 +910,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
           launch_pack_tiled(w->wdown[l], big_kind, pd, F, D, 0, st);
         }
         h->p_qkv.push_back(pq), h->p_o.push_back(po), h->p_g.push_back(pg), h->p_u.push_back(pu), h->p_d.push_back(pd);
-        if (w8 && h->b1_ok) {
+        if (w8 && !w4 && h->b1_ok) {
           // one byte per weight for the single-tile (HBM-bound) path; larger batches are tensor-bound and keep using
           // the bf16 images above
           uint8_t *bq, *bo, *bgu, *bd;

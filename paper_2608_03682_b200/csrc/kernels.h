@@ -56,7 +56,8 @@ void launch_set_request(Request* dst, const Request& src, int* cu_internal, cuda
 void launch_validate(const Request* rq, int* status, int max_prefix, int* order, cudaStream_t st);
 
 // ---- one-off table / packing kernels (CUDA cores, fp64 accumulation where cheap) ---------------
-// src_kind: 0 = float32, 1 = bfloat16, 2 = e4m3 byte codes
+// src_kind: 0 = float32, 1 = bfloat16, 2 = e4m3 byte codes, 3 = int4 codes (two neighbouring elements of a row per
+// byte, the even one in the low nibble; rows of even length)
 void launch_to_f32(const void* src, int src_kind, float* dst, size_t n, cudaStream_t st);
 // dst[r][col_off + c] = src[r][c] * (scale ? scale[c] : 1)
 void launch_copy_cols(const void* src, int src_kind, const float* scale, float* dst, int rows, int cols, int ld_dst,

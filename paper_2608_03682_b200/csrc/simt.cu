@@ -59,6 +59,10 @@ void launch_validate(const Request* rq, int* status, int max_prefix, int* order,
 __device__ __forceinline__ float load_src(const void* src, int kind, size_t i) {
   if (kind == 0) return reinterpret_cast<const float*>(src)[i];
   if (kind == 1) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(src)[i]);
+  if (kind == 3) {   // int4: two neighbouring elements per byte, the even one in the low nibble; code c = integer c - 8
+    const uint8_t b = reinterpret_cast<const uint8_t*>(src)[i >> 1];
+    return (float)((int)((i & 1) ? (b >> 4) : (b & 15)) - 8);
+  }
   const __half_raw hr = __nv_cvt_fp8_to_halfraw(reinterpret_cast<const __nv_fp8_storage_t*>(src)[i], __NV_E4M3);
   return __half2float(__half(hr));
 }

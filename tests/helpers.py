@@ -5,7 +5,7 @@ import torch
 from oracle import expert_oracle as O
 from paper_2608_03682_b200 import binding, synth
 
-BAR = {"f32": 1e-4, "bf16": 2e-2, "w8e4m3": 2e-2}   # max relative error on the final action chunk
+BAR = {"f32": 1e-4, "bf16": 2e-2, "w8e4m3": 2e-2, "w4a16": 2e-2}   # max relative error on the final action chunk
 
 
 def gpu_single(cfg, W, kv, P, state, noise, n_steps, engine="auto", use_graph=True, expert=None):

@@ -70,3 +70,14 @@ def test_w8a8_expert_matches_oracle(batch):
         bar, d_q = w8a8_bar(cfg, Wf, kv, 816, st, nz, 10, ref)
         print(f"W8A8 batch {batch} request {b}: max rel err {errs[b]:.2e}, quantization noise of the mode {d_q:.2e}, bar {bar:.2e}")
         assert errs[b] <= bar, (b, errs[b], bar)
+
+
+@pytest.mark.parametrize("batch", [1, 64])
+def test_w4a16_expert_matches_oracle(batch):
+    """The pi0-shaped expert with 4-bit integer weights against the oracle on sampled requests."""
+    cfg = synth.pi0_config(max_batch=batch, dtype="w4a16", max_prefix_len=816)
+    W = synth.make_weights(cfg, 5)
+    check = [0] if batch == 1 else [0, batch - 1]
+    errs = _run_batched(cfg, 5, W, [816] * batch, 10, check)
+    print(f"W4A16 batch {batch} max rel err:", {b: f"{e:.2e}" for b, e in errs.items()})
+    assert max(errs.values()) <= BAR["w4a16"], errs

@@ -310,6 +310,35 @@ def test_small_w8a8_expert_matches_oracle_single_and_batched(cond):
             assert rel_err(out[b], ref) <= bar, (b, rel_err(out[b], ref), bar)
 
 
+@pytest.mark.parametrize("cond", ["pi0", "pi05"])
+@pytest.mark.parametrize("engine", ["auto", "simt"])
+def test_small_w4a16_expert_matches_oracle_single_and_batched(cond, engine):
+    """W4A16: the seven large matrices as 4-bit integers (two output channels per byte) with per-channel scales;
+    single requests (cluster split-K kernels), a ragged batch (general kernels) and the CUDA-core engine."""
+    cfg = small_bf16_config(cond, dtype="w4a16", max_prefix_len=300, max_batch=5)
+    W = synth.make_weights(cfg, 25, std=0.05)
+    bar = BAR["f32"] if engine == "simt" else BAR["w4a16"]
+    with binding.Expert(cfg, binding.weights_to_device(W), engine=engine) as ex:
+        for P in (0, 130, 300):
+            kv, state, noise = _inputs(cfg, 25, P)
+            ref = O.denoise(cfg, W, kv, P, state, noise, 3)
+            got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
+            assert rel_err(got, ref) <= bar, (P, rel_err(got, ref))
+        lens = [300, 0, 17, 129, 64]
+        kvs = [synth.make_prefix_kv(cfg, 25, p, b) if p else synth.make_prefix_kv(cfg, 25, 1, b)[:, :, :0] for b, p in enumerate(lens)]
+        packed, cu = synth.pack_prefix_kv(kvs)
+        states = torch.stack([synth.make_state(cfg, 25, b) for b in range(5)]) if cfg.has_state_token else None
+        noise = torch.stack([synth.make_noise(cfg, 25, b) for b in range(5)])
+        out = ex.denoise_batched(packed.cuda(), torch.from_numpy(cu).cuda(), None if states is None else states.cuda(),
+                                 noise.cuda(), 3)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        out = out.double().cpu().numpy()
+        for b in range(5):
+            ref = O.denoise(cfg, W, kvs[b], lens[b], None if states is None else states[b], noise[b], 3)
+            assert rel_err(out[b], ref) <= bar, (b, rel_err(out[b], ref))
+
+
 def test_single_request_after_a_ragged_batch_with_many_heads():
     """16 query heads of 256 select the request-per-CTA tcgen05 attention kernel even for one request; it walks the
     requests in an order that the batched call writes.  A single-request call on the same handle must reset it."""
