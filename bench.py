@@ -59,6 +59,9 @@ def workload(name: str):
     if name.startswith("C5b"):
         b = int(name[3:])
         return synth.pi0_config(max_batch=b, dtype="w8e4m3", max_prefix_len=816), 5, b, [816] * b, 10
+    if name.startswith("C7b"):   # the C5 expert with 4-bit integer weights (W4A16)
+        b = int(name[3:])
+        return synth.pi0_config(max_batch=b, dtype="w4a16", max_prefix_len=816), 5, b, [816] * b, 10
     if name.startswith("C6b"):   # the C5 expert in the W8A8 mode: per-token e4m3 activations, FP8 tensor path
         b = int(name[3:])
         return synth.pi0_config(max_batch=b, dtype="w8a8e4m3", max_prefix_len=816), 5, b, [816] * b, 10
@@ -69,7 +72,7 @@ def algorithmic_cost(cfg, lens, n_steps):
     """Bytes that must cross HBM and FLOPs per chunk: every big weight once per Euler step, each
     request's prefix KV once per layer per step; activations and tables are cache resident."""
     D, F, L, S = cfg.width, cfg.mlp_dim, cfg.n_layers, cfg.suffix_len
-    wbytes = 1 if cfg.dtype in ("w8e4m3", "w8a8e4m3") else (4 if cfg.dtype == "f32" else 2)
+    wbytes = 0.5 if cfg.dtype == "w4a16" else (1 if cfg.dtype in ("w8e4m3", "w8a8e4m3") else (4 if cfg.dtype == "f32" else 2))
     ebytes = 4 if cfg.dtype == "f32" else 2
     nqkv = cfg.q_dim + 2 * cfg.kv_dim
     per_layer_params = D * nqkv + cfg.q_dim * D + 2 * D * F + F * D
@@ -469,6 +472,20 @@ def main():
             others[name] = r6
         e6.close()
         del in5
+        torch.cuda.empty_cache()
+        # the same expert with 4-bit integer weights at batch 1: the cluster path streams half a byte per weight
+        c7, id7, _, l7, n7 = workload("C7b1")
+        e7 = make_expert(c7, id7)
+        in7 = Inputs(c7, id7, l7)
+        r7 = run_workload("C7b1", e7, c7, l7, n7, in7, Ko, Wo, world, rank, local_rank, e2e=False)
+        e7.set_option("use_w8_inkernel", 0)
+        r7["ms_per_step_bf16_images"] = run_workload("C7b1", e7, c7, l7, n7, in7, Ko, Wo, world, rank, local_rank,
+                                                     e2e=False)["ms_per_step"]
+        r7["workload"], r7["steps"], r7["warmup"] = describe("C7b1", c7, 1, l7, n7), Ko, Wo
+        r7["roofline"] = roofline_of("C7b1", c7, l7, n7, 1, r7["ms_per_step"], peaks)
+        others["C7b1"] = r7
+        e7.close()
+        del in7
         torch.cuda.empty_cache()
         # a feature-handoff head of the shape the paper's GR00T profile names (40 x 132 chunk, four steps): the
         # request-local K / V projections of the features, then the loop on the projected prefix

@@ -350,6 +350,7 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
   const bool use_w8 = h->use_w8_inkernel && !h->b_qkv.empty();
   auto b1_gemm = [&](B1Gemm g, int which, int Mloc) -> phyai_status_t {
     g.M = Mloc, g.wait_limit = h->wait_limit, g.gelu_exact = d.gelu_exact, g.inv_D = 1.0f / (float)D, g.eps = d.eps;
+    g.w_bits = h->cfg.dtype == PHYAI_W4A16 ? 4 : 8;
     g.trace = (h->trace && cnt < TRACE_SLOTS) ? h->trace + cnt * TRACE_STAMPS : nullptr;
     // The QKV projection leaves the SMs of the attention kernel free: that kernel then starts (and fetches its prefix
     // tiles) while the projection still runs.  Measured on the pi0-shaped expert: 7.6 ms per chunk with 140 CTAs,
@@ -910,20 +911,24 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
           launch_pack_tiled(w->wdown[l], big_kind, pd, F, D, 0, st);
         }
         h->p_qkv.push_back(pq), h->p_o.push_back(po), h->p_g.push_back(pg), h->p_u.push_back(pu), h->p_d.push_back(pd);
-        if (w8 && !w4 && h->b1_ok) {
+        if (w8 && !a8 && h->b1_ok) {
           // one byte per weight for the single-tile (HBM-bound) path; larger batches are tensor-bound and keep using
           // the bf16 images above
           uint8_t *bq, *bo, *bgu, *bd;
-          ST(h->alloc(&bq, (size_t)D * Nqkv)); ST(h->alloc(&bo, (size_t)Nq * D));
-          ST(h->alloc(&bgu, (size_t)D * 2 * F)); ST(h->alloc(&bd, (size_t)F * D));
-          const uint8_t* cq = reinterpret_cast<const uint8_t*>(w->wq[l]);
-          launch_pack_bytes(cq, bq, D, Nq, 0, st, 0, 0, d.dh);
-          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wk[l]), bq, D, Nkv, Nq, st, 0, 0, d.dh);
-          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wv[l]), bq, D, Nkv, Nq + Nkv, st);
-          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wo[l]), bo, Nq, D, 0, st);
-          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wgate[l]), bgu, D, F, 0, st, 64, 0);
-          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wup[l]), bgu, D, F, 0, st, 64, 1);
-          launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wdown[l]), bd, F, D, 0, st);
+          const size_t div = w4 ? 2 : 1;     // int4: half a byte per weight
+          ST(h->alloc(&bq, (size_t)D * Nqkv / div)); ST(h->alloc(&bo, (size_t)Nq * D / div));
+          ST(h->alloc(&bgu, (size_t)D * 2 * F / div)); ST(h->alloc(&bd, (size_t)F * D / div));
+          auto pack = [&](const void* src, uint8_t* dst, int K, int N, int n_off, int il = 0, int second = 0, int perm = 0) {
+            if (w4) launch_pack_nibbles(reinterpret_cast<const uint8_t*>(src), dst, K, N, n_off, st, il, second, perm);
+            else launch_pack_bytes(reinterpret_cast<const uint8_t*>(src), dst, K, N, n_off, st, il, second, perm);
+          };
+          pack(w->wq[l], bq, D, Nq, 0, 0, 0, d.dh);
+          pack(w->wk[l], bq, D, Nkv, Nq, 0, 0, d.dh);
+          pack(w->wv[l], bq, D, Nkv, Nq + Nkv);
+          pack(w->wo[l], bo, Nq, D, 0);
+          pack(w->wgate[l], bgu, D, F, 0, 64, 0);
+          pack(w->wup[l], bgu, D, F, 0, 64, 1);
+          pack(w->wdown[l], bd, F, D, 0);
           h->b_qkv.push_back(bq), h->b_o.push_back(bo), h->b_gu.push_back(bgu), h->b_d.push_back(bd);
         }
         float *cq = nullptr, *co = nullptr, *cg = nullptr, *cu = nullptr, *cd = nullptr;

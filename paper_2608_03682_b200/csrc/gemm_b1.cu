@@ -80,8 +80,12 @@ __device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t& lo, uint3
   asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(hi) : "r"(t1), "r"(c));
 }
 
-template <int EPI, bool W8>
+// WB: bits per streamed weight -- 0 = the bf16 operand image itself, 8 = e4m3 codes, 4 = int4 codes; the codes are
+// decoded to the bf16 image in shared memory ahead of the dependency wait.
+template <int EPI, int WB>
 __global__ void __launch_bounds__(NT, 1) k_gemm_b1(int* status, const B1Gemm g) {
+  constexpr bool W8 = WB != 0;          // (weights arrive as codes)
+  constexpr uint32_t CODE_BYTES = WB == 4 ? W_BYTES / 4 : W_BYTES / 2;   // one block of codes
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[MAXK];
   __shared__ __align__(8) uint64_t bar_w8[MAXK];       // e4m3 weights: the byte blocks have landed
@@ -136,11 +140,12 @@ __global__ void __launch_bounds__(NT, 1) k_gemm_b1(int* status, const B1Gemm g) 
   if (lane == 0) {
     for (int s = warp; s < nk; s += NW) {
       if (W8) {
-        // one byte per weight: the 8 KB block lands in the upper half of the stage's 16 KB operand slot
+        // one byte (or half a byte) per weight: the 8 KB (4 KB) block of codes lands at the end of the stage's 16 KB
+        // operand slot
         const uint32_t full = smem_u32(&bar_w8[s]);
-        mbar_expect_tx(full, W_BYTES / 2);
-        bulk_g2s(tiles + (uint32_t)s * STAGE + W_BYTES / 2,
-                 reinterpret_cast<const uint8_t*>(g.W8) + ((size_t)tile * KC + kc_begin + s) * (W_BYTES / 2), W_BYTES / 2, full);
+        mbar_expect_tx(full, CODE_BYTES);
+        bulk_g2s(tiles + (uint32_t)s * STAGE + W_BYTES - CODE_BYTES,
+                 reinterpret_cast<const uint8_t*>(g.W8) + ((size_t)tile * KC + kc_begin + s) * CODE_BYTES, CODE_BYTES, full);
       } else {
         const uint32_t full = smem_u32(&bar_full[s]);
         mbar_expect_tx(full, W_BYTES);
@@ -205,6 +210,7 @@ __global__ void __launch_bounds__(NT, 1) k_gemm_b1(int* status, const B1Gemm g) 
       for (int s = 0; s < nk; ++s) mbar_wait_drain(smem_u32(&bar_w8[s]), 0u, wc);
     __syncthreads();
     trace_stamp(tr, 9);
+    if constexpr (WB == 8) {
     uint4 raw[MAXK];
     const int r = tid >> 2, hc = (tid & 3) * 2;       // row, first of my two 8-code chunks
 #pragma unroll
@@ -227,6 +233,39 @@ __global__ void __launch_bounds__(NT, 1) k_gemm_b1(int* status, const B1Gemm g) 
           asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
         }
       }
+    } else {
+      // int4: a row of the block is 32 bytes = 64 codes, byte j = codes (k = 2j in the low nibble, 2j + 1 in the high
+      // one); a thread takes 8 bytes of its row (row = tid / 4) and writes 16 bf16 = two 16-byte chunks.  A nibble c
+      // becomes the bf16 number 128 + c by bit insertion (0x4300 | c: the unit of the mantissa at 128 is 1), and one
+      // exact bf16x2 subtraction of 136 makes it c - 8.
+      uint2 raw[MAXK];
+      const int r = tid >> 2, qd = tid & 3;
+#pragma unroll
+      for (int s = 0; s < MAXK; ++s)
+        if (s < nk) {
+          const uint32_t src = tiles + (uint32_t)s * STAGE + W_BYTES - CODE_BYTES + (uint32_t)r * 32 + (uint32_t)qd * 8;
+          asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(raw[s].x), "=r"(raw[s].y) : "r"(src) : "memory");
+        }
+      __syncthreads();
+      auto pair = [](uint32_t byte) -> uint32_t {       // one byte -> (bf16(lo - 8), bf16(hi - 8))
+        uint32_t w = 0x43004300u | (byte & 15u) | ((byte & 0xF0u) << 12), o;
+        asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(o) : "r"(w), "r"(0x43084308u));
+        return o;
+      };
+#pragma unroll
+      for (int s = 0; s < MAXK; ++s)
+        if (s < nk) {
+          const uint32_t words[2] = {raw[s].x, raw[s].y};
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {       // 16-byte chunk 2 qd + c: codes of bytes 4c .. 4c + 3 of my 8
+            const uint32_t w4 = words[c];
+            const uint32_t dst = tiles + (uint32_t)s * STAGE + (uint32_t)r * 128 + (uint32_t)((((2 * qd + c) ^ (r & 7))) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(pair(w4 & 0xFFu)), "r"(pair((w4 >> 8) & 0xFFu)),
+                         "r"(pair((w4 >> 16) & 0xFFu)), "r"(pair(w4 >> 24))
+                         : "memory");
+          }
+        }
+    }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the tensor core's reads
     __syncthreads();
     trace_stamp(tr, 10);
@@ -481,11 +520,11 @@ size_t b1_smem(int nk_max, int C, bool rope_rows) {
   return 1024 + region + (size_t)C * tpc * ROWB + (rope_rows ? (size_t)tpc * 512 : 0);
 }
 
-template <int EPI, bool W8>
+template <int EPI, int WB>
 cudaError_t launch_one(int* status, const B1Gemm& g, int C, cudaStream_t st) {
   static PerDeviceOnce once;
   if (once.needed()) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_b1<EPI, W8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1_SMEM_MAX);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_b1<EPI, WB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)B1_SMEM_MAX);
     if (e != cudaSuccess) return e;
     once.done();
   }
@@ -497,7 +536,7 @@ cudaError_t launch_one(int* status, const B1Gemm& g, int C, cudaStream_t st) {
   at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at, cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, k_gemm_b1<EPI, W8>, status, g);
+  return cudaLaunchKernelEx(&cfg, k_gemm_b1<EPI, WB>, status, g);
 }
 
 }  // namespace
@@ -524,14 +563,19 @@ cudaError_t launch_b1_gemm(int* status, const B1Gemm& g_in, int C, cudaStream_t 
   const int KC = g.K / 64;
   g.nk_max = (KC + C - 1) / C;
   if (b1_smem(g.nk_max, C, g.epi == B1_QKV) > B1_SMEM_MAX) return cudaErrorInvalidConfiguration;
-  if (g.W8) {
-    if (g.epi == B1_QKV) return launch_one<B1_QKV, true>(status, g, C, st);
-    if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU, true>(status, g, C, st);
-    return launch_one<B1_RESID, true>(status, g, C, st);
+  if (g.W8 && g.w_bits == 4) {
+    if (g.epi == B1_QKV) return launch_one<B1_QKV, 4>(status, g, C, st);
+    if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU, 4>(status, g, C, st);
+    return launch_one<B1_RESID, 4>(status, g, C, st);
   }
-  if (g.epi == B1_QKV) return launch_one<B1_QKV, false>(status, g, C, st);
-  if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU, false>(status, g, C, st);
-  return launch_one<B1_RESID, false>(status, g, C, st);
+  if (g.W8) {
+    if (g.epi == B1_QKV) return launch_one<B1_QKV, 8>(status, g, C, st);
+    if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU, 8>(status, g, C, st);
+    return launch_one<B1_RESID, 8>(status, g, C, st);
+  }
+  if (g.epi == B1_QKV) return launch_one<B1_QKV, 0>(status, g, C, st);
+  if (g.epi == B1_GEGLU) return launch_one<B1_GEGLU, 0>(status, g, C, st);
+  return launch_one<B1_RESID, 0>(status, g, C, st);
 }
 
 }  // namespace phyai

@@ -82,6 +82,10 @@ void launch_rows_to_tiled(const __nv_bfloat16* x, __nv_bfloat16* tiled, int M, i
 // [K/128][rows_pad][128] with the same 16-byte chunk swizzle.  Rows >= M are left alone.
 void launch_quant_rows(const int* status, const __nv_bfloat16* x, uint8_t* out, float* scale, int rows_pad, int M, int K,
                        cudaStream_t st);
+// int4 codes [K][N/2] (two neighbouring out channels per byte) -> nibble blocks [N/128][K/64][128][32] in the packed
+// row order of launch_pack_tiled, byte j of a row = codes of k = 2j (low nibble) and 2j + 1 (high nibble)
+void launch_pack_nibbles(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group = 0,
+                         int il_second = 0, int perm_dh = 0);
 void launch_permute_scales(const float* src, float* dst, int N, int n_off, int perm_dh, cudaStream_t st);
 // Y[r][n] = act( sum_d X[r][d] * W[(w_row_off + d)][n] + bias[n] + add[n] ), r < R
 void launch_rows_gemm(const float* X, int ldx, const void* W, int w_kind, int w_row_off, int N, int K, const float* bias,
@@ -223,6 +227,8 @@ cudaError_t tc_gemm_setup();  // one-time attribute setup (dynamic shared memory
 enum : int { B1_QKV = 0, B1_GEGLU = 1, B1_RESID = 2 };
 struct B1Gemm {
   const __nv_bfloat16* W;    // packed blocks [N/128][K/64][128x64]
+  int w_bits;                // 8 (e4m3 codes) or 4 (int4 codes: blocks of [128 rows][32 bytes], byte j of a row = codes of
+                             // k = 2j (low nibble) and 2j + 1) when W8 is set
   const uint8_t* W8;         // or: e4m3 codes, blocks [N/128][K/64][128 rows][64 bytes] in the same row order, decoded
                              // to bf16 inside the kernel (one byte per weight crosses HBM); scales as below
   const __nv_bfloat16* X;    // tiled activations [K/64][64][64] (64-row tiles, back to back)

@@ -232,6 +232,35 @@ void launch_quant_rows(const int* status, const __nv_bfloat16* x, uint8_t* out, 
   launch_pdl(k_quant_rows, dim3((M + 7) / 8), dim3(256), 0, st, status, x, out, scale, rows_pad, M, K);
 }
 
+// int4 codes: source [K][N/2] with two neighbouring out channels per byte; destination blocks of 128 out channels x
+// 64 k with two neighbouring k per byte (what a row of the MMA's K-major operand needs).  One thread per 8 k of one
+// out channel (4 destination bytes).
+__global__ void k_pack_nibbles(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, int il_group, int il_second,
+                               int perm_dh) {
+  const int KC = K >> 6;
+  const size_t chunks = (size_t)N * (K >> 3);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
+    const int n = (int)(i % N), k0 = (int)(i / N) << 3;
+    const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
+                            : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
+    uint32_t w = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint8_t b = src[(size_t)(k0 + j) * (N >> 1) + (n >> 1)];
+      const uint32_t c = (n & 1) ? (b >> 4) : (b & 15);
+      w |= c << (4 * j);
+    }
+    const int kc = k0 >> 6;
+    *reinterpret_cast<uint32_t*>(dst + (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 32 + ((k0 & 63) >> 1)) = w;
+  }
+}
+void launch_pack_nibbles(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group,
+                         int il_second, int perm_dh) {
+  const size_t chunks = (size_t)N * (K >> 3);
+  const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
+  k_pack_nibbles<<<blocks, 256, 0, st>>>(src, dst, K, N, n_off, il_group, il_second, perm_dh);
+}
+
 // Row of an adaptive norm's shift through a packed weight matrix: out[n] = scale(n) * sum_k shift[k] * W[n][k].
 // One warp per packed row; a lane reads pairs of k out of the swizzled 128 x 64 blocks.
 __global__ void k_shift_rows(const float* shift, const __nv_bfloat16* Wp, const float* wscale, const float* wscale2,

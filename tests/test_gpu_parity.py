@@ -324,6 +324,13 @@ def test_small_w4a16_expert_matches_oracle_single_and_batched(cond, engine):
             ref = O.denoise(cfg, W, kv, P, state, noise, 3)
             got = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
             assert rel_err(got, ref) <= bar, (P, rel_err(got, ref))
+            if engine == "auto":
+                # the cluster path streams the 4-bit codes and decodes them in the kernel (exactly): bit-equal to the
+                # run on the bf16 images made at create
+                ex.set_option("use_w8_inkernel", 0)
+                again = gpu_single(cfg, W, kv, P, state, noise, 3, expert=ex)
+                ex.set_option("use_w8_inkernel", 1)
+                assert np.array_equal(got, again), P
         lens = [300, 0, 17, 129, 64]
         kvs = [synth.make_prefix_kv(cfg, 25, p, b) if p else synth.make_prefix_kv(cfg, 25, 1, b)[:, :, :0] for b, p in enumerate(lens)]
         packed, cu = synth.pack_prefix_kv(kvs)
