@@ -36,7 +36,8 @@ NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (bench.py cannot run ncu itself)
 NCU_TRAFFIC = {"C2": (180 * 37.41e6 + 10 * 2.8e6, "profiles/cluster_loop_c2_c5_batch1.md"),
-               "C5b1": (180 * 20.39e6 + 10 * 2.8e6, "profiles/cluster_loop_c2_c5_batch1.md")}
+               "C5b1": (180 * 20.39e6 + 10 * 2.8e6, "profiles/cluster_loop_c2_c5_batch1.md"),
+               "C7b1": (180 * 11.70e6 + 10 * 2.8e6, "profiles/cluster_loop_c2_c5_batch1.md")}
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 
 
