@@ -202,69 +202,67 @@ __global__ void __launch_bounds__(NT, 1) k_gemm_b1(int* status, const B1Gemm g) 
     }
   }
   if (W8) {
-    // e4m3 -> bf16 in place, ahead of the dependency wait where the weights arrive early (they are constants): every
-    // thread first takes its 16 bytes of every stage into registers (row = tid / 4, two 8-byte chunks), then, after
-    // a barrier, writes them back as 32 bytes of the swizzled K-major bf16 image the MMA reads.  The per-channel
-    // scale stays in the epilogue.
-    if (warp == 0)
-      for (int s = 0; s < nk; ++s) mbar_wait_drain(smem_u32(&bar_w8[s]), 0u, wc);
-    __syncthreads();
-    trace_stamp(tr, 9);
-    if constexpr (WB == 8) {
-    uint4 raw[MAXK];
-    const int r = tid >> 2, hc = (tid & 3) * 2;       // row, first of my two 8-code chunks
+    // codes -> bf16 in place, ahead of the dependency wait where the weights arrive early (they are constants), stage
+    // by stage as the blocks land: warps 2 s and 2 s + 1 take stage s, 64 rows each (8 x 8 rows; a lane takes 16 codes
+    // of a row and writes them as 32 bytes of the swizzled K-major bf16 image the MMA reads).  The codes sit at the end
+    // of the image they expand into, so both warps of a stage read all their codes into registers, meet at a named
+    // barrier, and only then write.  The per-channel scale stays in the epilogue.
+    const int s = warp >> 1, hf = warp & 1;
+    if (s < nk) {
+      mbar_wait_drain(smem_u32(&bar_w8[s]), 0u, wc);
+      const uint32_t slot0 = tiles + (uint32_t)s * STAGE;
+      const int r0 = hf * 64 + (lane >> 2), cq = lane & 3;       // my row of every group of 8 rows, my quarter of a row
+      if constexpr (WB == 8) {
+        uint4 raw[8];
 #pragma unroll
-    for (int s = 0; s < MAXK; ++s)
-      if (s < nk) {
-        const uint32_t src = tiles + (uint32_t)s * STAGE + W_BYTES / 2 + (uint32_t)r * 64 + (uint32_t)hc * 8;
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(raw[s].x), "=r"(raw[s].y), "=r"(raw[s].z), "=r"(raw[s].w) : "r"(src) : "memory");
-      }
-    __syncthreads();
-#pragma unroll
-    for (int s = 0; s < MAXK; ++s)
-      if (s < nk) {
-        const uint32_t words[4] = {raw[s].x, raw[s].y, raw[s].z, raw[s].w};
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {       // chunk hc + c: 8 codes = words[2c], words[2c + 1]
-          uint32_t o0, o1, o2, o3;
-          e4m3x4_to_bf16x4(words[2 * c], o0, o1);
-          e4m3x4_to_bf16x4(words[2 * c + 1], o2, o3);
-          const uint32_t dst = tiles + (uint32_t)s * STAGE + (uint32_t)r * 128 + (uint32_t)((((hc + c) ^ (r & 7))) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t src = slot0 + W_BYTES - CODE_BYTES + (uint32_t)(r0 + 8 * j) * 64 + (uint32_t)cq * 16;
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(raw[j].x), "=r"(raw[j].y), "=r"(raw[j].z), "=r"(raw[j].w) : "r"(src) : "memory");
         }
-      }
-    } else {
-      // int4: a row of the block is 32 bytes = 64 codes, byte j = codes (k = 2j in the low nibble, 2j + 1 in the high
-      // one); a thread takes 8 bytes of its row (row = tid / 4) and writes 16 bf16 = two 16-byte chunks.  A nibble c
-      // becomes the bf16 number 128 + c by bit insertion (0x4300 | c: the unit of the mantissa at 128 is 1), and one
-      // exact bf16x2 subtraction of 136 makes it c - 8.
-      uint2 raw[MAXK];
-      const int r = tid >> 2, qd = tid & 3;
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
 #pragma unroll
-      for (int s = 0; s < MAXK; ++s)
-        if (s < nk) {
-          const uint32_t src = tiles + (uint32_t)s * STAGE + W_BYTES - CODE_BYTES + (uint32_t)r * 32 + (uint32_t)qd * 8;
-          asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(raw[s].x), "=r"(raw[s].y) : "r"(src) : "memory");
+        for (int j = 0; j < 8; ++j) {
+          const int r = r0 + 8 * j;
+          const uint32_t words[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {       // 16-byte chunk 2 cq + c of the row: 8 codes = words[2c], words[2c + 1]
+            uint32_t o0, o1, o2, o3;
+            e4m3x4_to_bf16x4(words[2 * c], o0, o1);
+            e4m3x4_to_bf16x4(words[2 * c + 1], o2, o3);
+            const uint32_t dst = slot0 + (uint32_t)r * 128 + (uint32_t)((((2 * cq + c) ^ (r & 7))) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+          }
         }
-      __syncthreads();
-      auto pair = [](uint32_t byte) -> uint32_t {       // one byte -> (bf16(lo - 8), bf16(hi - 8))
-        uint32_t w = 0x43004300u | (byte & 15u) | ((byte & 0xF0u) << 12), o;
-        asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(o) : "r"(w), "r"(0x43084308u));
-        return o;
-      };
+      } else {
+        // int4: a row of the block is 32 bytes = 64 codes, byte j = codes (k = 2j in the low nibble, 2j + 1 in the
+        // high one).  A nibble c becomes the bf16 number 128 + c by bit insertion (0x4300 | c: the unit of the mantissa
+        // at 128 is 1), and one exact bf16x2 subtraction of 136 makes it c - 8.
+        uint2 raw[8];
 #pragma unroll
-      for (int s = 0; s < MAXK; ++s)
-        if (s < nk) {
-          const uint32_t words[2] = {raw[s].x, raw[s].y};
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t src = slot0 + W_BYTES - CODE_BYTES + (uint32_t)(r0 + 8 * j) * 32 + (uint32_t)cq * 8;
+          asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(raw[j].x), "=r"(raw[j].y) : "r"(src) : "memory");
+        }
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
+        auto pair = [](uint32_t byte) -> uint32_t {       // one byte -> (bf16(lo - 8), bf16(hi - 8))
+          uint32_t w = 0x43004300u | (byte & 15u) | ((byte & 0xF0u) << 12), o;
+          asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(o) : "r"(w), "r"(0x43084308u));
+          return o;
+        };
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {       // 16-byte chunk 2 qd + c: codes of bytes 4c .. 4c + 3 of my 8
+        for (int j = 0; j < 8; ++j) {
+          const int r = r0 + 8 * j;
+          const uint32_t words[2] = {raw[j].x, raw[j].y};
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {       // 16-byte chunk 2 cq + c: codes of bytes 4c .. 4c + 3 of my 8
             const uint32_t w4 = words[c];
-            const uint32_t dst = tiles + (uint32_t)s * STAGE + (uint32_t)r * 128 + (uint32_t)((((2 * qd + c) ^ (r & 7))) << 4);
+            const uint32_t dst = slot0 + (uint32_t)r * 128 + (uint32_t)((((2 * cq + c) ^ (r & 7))) << 4);
             asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(pair(w4 & 0xFFu)), "r"(pair((w4 >> 8) & 0xFFu)),
                          "r"(pair((w4 >> 16) & 0xFFu)), "r"(pair(w4 >> 24))
                          : "memory");
           }
         }
+      }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the tensor core's reads
     __syncthreads();
