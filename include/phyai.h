@@ -239,6 +239,9 @@ phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t valu
  * kernel (Q copied, Q in tensor memory, logits ready, partial staged, ...).  After the stream is synchronised phyai_read_trace copies the buffer to `out`
  * (HOST memory, capacity >= 4096 * 16 entries); slots of launches that are not traced stay 0.  The stamps cost
  * a few hundred ns each: a traced call is slower.  "trace" = 0 turns it off.
+ * Option "trace_all_from" = i > 0 (with "trace" = 1): instead, EVERY CTA of the cluster-GEMM and cluster-attention
+ * launches with index i .. i + 4 of a call stamps, into consecutive slots (slot = CTAs of the earlier traced launches +
+ * the CTA's linear index in its grid); 0 returns to one CTA per launch.
  */
 phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_slots,
                                 uint32_t *n_stamps);
