@@ -378,6 +378,18 @@ typedef struct {
 phyai_status_t phyai_project_features_kv(const phyai_kv_proj_desc_t *desc, const void *features, const void *const *wk,
                                          const void *const *wv, uint64_t tokens, uint64_t kv_tokens, void *prefix_kv,
                                          void *stream);
+/*
+ * The same with the packed weight images and the workspace held in a handle: create packs the 2 * n_layers matrices
+ * once (synchronises `stream`); run only enqueues kernels on `stream` (no allocation, no synchronisation; one run in
+ * flight per handle) for up to max_tokens feature rows.  A bounded device-side wait that expired leaves rows unwritten;
+ * the one-shot call above reports it, a projector's caller sees non-finite / stale rows downstream.
+ */
+typedef struct phyai_kv_projector phyai_kv_projector_t;
+phyai_status_t phyai_kv_projector_create(const phyai_kv_proj_desc_t *desc, const void *const *wk, const void *const *wv,
+                                         uint64_t max_tokens, void *stream, phyai_kv_projector_t **out);
+phyai_status_t phyai_kv_projector_run(phyai_kv_projector_t *p, const void *features, uint64_t tokens, uint64_t kv_tokens,
+                                      void *prefix_kv, void *stream);
+void phyai_kv_projector_destroy(phyai_kv_projector_t *p);
 
 /* Thread-local description of the last error of an adapter entry point. */
 const char *phyai_adapter_last_error(void);

@@ -31,7 +31,8 @@ EXPORTS = ("phyai_expert_create", "phyai_expert_destroy", "phyai_prefix_kv_bytes
            "phyai_suffix_attention_static", "phyai_suffix_attention_static_capacity", "phyai_read_trace",
            "phyai_pack_prefix_kv", "phyai_postprocess_actions", "phyai_adapter_last_error", "phyai_batcher_create",
            "phyai_batcher_destroy", "phyai_batcher_submit", "phyai_batcher_next", "phyai_batcher_pending",
-           "phyai_batcher_plan", "phyai_w8a8_project", "phyai_w8a8_last_error", "phyai_project_features_kv")
+           "phyai_batcher_plan", "phyai_w8a8_project", "phyai_w8a8_last_error", "phyai_project_features_kv", "phyai_kv_projector_create",
+           "phyai_kv_projector_run", "phyai_kv_projector_destroy")
 
 
 class PhyaiError(RuntimeError):
@@ -119,6 +120,10 @@ def load_library() -> C.CDLL:
     lib.phyai_w8a8_project.argtypes = [_VP, _VP, _VP, C.c_uint32, C.c_uint32, C.c_uint32, _VP, _VP, _VP, _VP]
     lib.phyai_w8a8_last_error.restype = C.c_char_p
     lib.phyai_project_features_kv.argtypes = [_VP, _VP, _VP, _VP, C.c_uint64, C.c_uint64, _VP, _VP]
+    lib.phyai_kv_projector_create.argtypes = [_VP, _VP, _VP, C.c_uint64, _VP, C.POINTER(_VP)]
+    lib.phyai_kv_projector_run.argtypes = [_VP, _VP, C.c_uint64, C.c_uint64, _VP, _VP]
+    lib.phyai_kv_projector_destroy.argtypes = [_VP]
+    lib.phyai_kv_projector_destroy.restype = None
     lib.phyai_batcher_create.argtypes = [C.POINTER(BatcherConfig), C.POINTER(_VP)]
     lib.phyai_batcher_destroy.argtypes = [_VP]
     lib.phyai_batcher_destroy.restype = None
@@ -378,6 +383,49 @@ def project_features_kv(features: torch.Tensor, wk, wv, n_kv_heads: int, head_di
     if st != OK:
         raise PhyaiError(st, lib.phyai_adapter_last_error().decode())
     return out
+
+
+class KvProjector:
+    """Handle form of the feature K / V projection (``phyai_kv_projector_*``): weights packed once, ``run`` only enqueues."""
+
+    def __init__(self, wk, wv, n_kv_heads: int, head_dim: int, max_tokens: int, stream=None):
+        self.lib = load_library()
+        self.L, self.n_kv_heads, self.head_dim = len(wk), n_kv_heads, head_dim
+        desc = KvProjDesc(C.sizeof(KvProjDesc), self.L, n_kv_heads, head_dim, wk[0].shape[0])
+        ak, av = (_VP * self.L)(), (_VP * self.L)()
+        for l in range(self.L):
+            ak[l], av[l] = wk[l].data_ptr(), wv[l].data_ptr()
+        self._h = _VP()
+        st = self.lib.phyai_kv_projector_create(C.byref(desc), C.cast(ak, _VP), C.cast(av, _VP), max_tokens,
+                                                _stream_ptr(stream), C.byref(self._h))
+        if st != OK:
+            raise PhyaiError(st, self.lib.phyai_adapter_last_error().decode())
+
+    def run(self, features: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        tokens = features.shape[0]
+        if out is None:
+            out = torch.zeros(self.L, 2, tokens, self.n_kv_heads, self.head_dim, dtype=torch.bfloat16, device=features.device)
+        st = self.lib.phyai_kv_projector_run(self._h, _ptr(features), tokens, out.shape[2], _ptr(out), _stream_ptr(stream))
+        if st != OK:
+            raise PhyaiError(st, self.lib.phyai_adapter_last_error().decode())
+        return out
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self.lib.phyai_kv_projector_destroy(self._h)
+            self._h = _VP()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def w8a8_project(x: torch.Tensor, w_codes: torch.Tensor, w_scales: torch.Tensor, return_codes: bool = False, stream=None):

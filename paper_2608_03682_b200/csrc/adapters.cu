@@ -3,6 +3,7 @@
 // into the library's ragged prefix-KV layout, and converting the raw action chunk (x at t = 0) into robot actions.
 // Both are pure data movement / element-wise work: coalesced 16-byte copies, one thread per output element.
 #include <cstdio>
+#include <new>
 
 #include "../../include/phyai.h"
 #include "kernels.h"
@@ -142,58 +143,113 @@ phyai_status_t phyai_postprocess_actions(const float* x, uint32_t batch, uint32_
 }  // extern "C"
 
 // Request-local K / V projections of a feature-handoff head: per layer one tcgen05 GEMM of the (tiled) feature rows
-// against [Wk | Wv], fp32 out, then the bf16 rows of the two planes.  Runs once per request batch, ahead of the loop.
+// against [Wk | Wv], fp32 out, then the bf16 rows of the two planes.  The projector handle owns the packed weight
+// images and the workspace, so that a run only enqueues kernels.
+struct phyai_kv_projector {
+  int L = 0, nkv = 0, Dv = 0, max_tokens = 0, rows_pad = 0;
+  __nv_bfloat16* wp = nullptr;    // [L] packed [Wk | Wv] images, Dv x 2 nkv each
+  __nv_bfloat16* xt = nullptr;    // tiled features [Dv / 64][rows_pad][64]
+  float* y = nullptr;             // [max_tokens][2 nkv]
+  int* status = nullptr;
+};
+
+namespace {
+phyai_status_t proj_fail(phyai_status_t st, const char* msg, cudaError_t e = cudaSuccess) {
+  using namespace phyai;
+  if (e != cudaSuccess) snprintf(g_ad_err, sizeof(g_ad_err), "%s: %s", msg, cudaGetErrorString(e));
+  else snprintf(g_ad_err, sizeof(g_ad_err), "%s", msg);
+  return st;
+}
+}  // namespace
+
+extern "C" void phyai_kv_projector_destroy(phyai_kv_projector_t* p) {
+  if (!p) return;
+  cudaFree(p->wp), cudaFree(p->xt), cudaFree(p->y), cudaFree(p->status);
+  delete p;
+}
+
+extern "C" phyai_status_t phyai_kv_projector_create(const phyai_kv_proj_desc_t* desc, const void* const* wk,
+                                                    const void* const* wv, uint64_t max_tokens, void* stream,
+                                                    phyai_kv_projector_t** out) {
+  using namespace phyai;
+  g_ad_err[0] = 0;
+  if (out) *out = nullptr;
+  if (!desc || desc->struct_size != sizeof(phyai_kv_proj_desc_t) || !wk || !wv || !out)
+    return proj_fail(PHYAI_ERR_INVALID_ARG, "NULL argument or wrong struct_size");
+  const int L = (int)desc->n_layers, nkv = (int)(desc->n_kv_heads * desc->head_dim), Dv = (int)desc->feat_dim;
+  if (L <= 0 || nkv <= 0 || Dv <= 0 || Dv % 64 || (2 * nkv) % 128 || max_tokens == 0 || max_tokens > (1u << 22))
+    return proj_fail(PHYAI_ERR_INVALID_ARG,
+                     "need feat_dim a multiple of 64, 2 * n_kv_heads * head_dim a multiple of 128, 1 <= max_tokens <= 2^22");
+  for (int l = 0; l < L; ++l)
+    if (!wk[l] || !wv[l]) return proj_fail(PHYAI_ERR_INVALID_ARG, "a per-layer weight pointer is NULL");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cudaError_t e = tc_gemm_setup();
+  if (e != cudaSuccess) return proj_fail(PHYAI_ERR_CUDA, "tc_gemm_setup", e);
+  phyai_kv_projector* p = new (std::nothrow) phyai_kv_projector();
+  if (!p) return proj_fail(PHYAI_ERR_OOM, "host allocation failed");
+  p->L = L, p->nkv = nkv, p->Dv = Dv, p->max_tokens = (int)max_tokens, p->rows_pad = ((int)max_tokens + 255) / 256 * 256;
+  const size_t N = 2 * (size_t)nkv;
+  if ((e = cudaMalloc(&p->wp, (size_t)L * Dv * N * 2)) != cudaSuccess || (e = cudaMalloc(&p->xt, (size_t)p->rows_pad * Dv * 2)) != cudaSuccess ||
+      (e = cudaMalloc(&p->y, (size_t)max_tokens * N * 4)) != cudaSuccess || (e = cudaMalloc(&p->status, 4)) != cudaSuccess) {
+    phyai_kv_projector_destroy(p);
+    return proj_fail(PHYAI_ERR_OOM, "cudaMalloc", e);
+  }
+  cudaMemsetAsync(p->xt, 0, (size_t)p->rows_pad * Dv * 2, st);
+  cudaMemsetAsync(p->status, 0, 4, st);
+  for (int l = 0; l < L; ++l) {
+    launch_pack_tiled(wk[l], 1, p->wp + (size_t)l * Dv * N, Dv, nkv, 0, st);
+    launch_pack_tiled(wv[l], 1, p->wp + (size_t)l * Dv * N, Dv, nkv, nkv, st);
+  }
+  e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    phyai_kv_projector_destroy(p);
+    return proj_fail(PHYAI_ERR_CUDA, "weight packing", e);
+  }
+  *out = p;
+  return PHYAI_OK;
+}
+
+extern "C" phyai_status_t phyai_kv_projector_run(phyai_kv_projector_t* p, const void* features, uint64_t tokens,
+                                                 uint64_t kv_tokens, void* prefix_kv, void* stream) {
+  using namespace phyai;
+  g_ad_err[0] = 0;
+  if (!p || !features || !prefix_kv) return proj_fail(PHYAI_ERR_INVALID_ARG, "NULL argument");
+  if (tokens == 0 || tokens > (uint64_t)p->max_tokens || tokens > kv_tokens)
+    return proj_fail(PHYAI_ERR_INVALID_ARG, "need 1 <= tokens <= max_tokens and tokens <= kv_tokens");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int M = (int)tokens, N = 2 * p->nkv;
+  launch_rows_to_tiled(reinterpret_cast<const __nv_bfloat16*>(features), p->xt, M, p->Dv, p->rows_pad, st);
+  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(prefix_kv);
+  for (int l = 0; l < p->L; ++l) {
+    TcGemm g{};
+    g.W = p->wp + (size_t)l * p->Dv * N, g.X = p->xt, g.M = M, g.N = N, g.K = p->Dv, g.epi = TC_STORE, g.out_f32 = p->y, g.ldo = N;
+    g.splits = 1, g.rows_pad = p->rows_pad, g.wait_limit = 1u << 28;
+    cudaError_t e = launch_tc_gemm(p->status, g, M <= 64 ? 64 : (M <= 1024 ? 128 : 256), st);
+    if (e != cudaSuccess) return proj_fail(PHYAI_ERR_CUDA, "projection GEMM launch", e);
+    const size_t n = (size_t)M * (p->nkv >> 2) * 2;
+    k_kv_planes<<<(int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096), 256, 0, st>>>(
+        p->y, out + ((size_t)l * 2) * kv_tokens * p->nkv, out + ((size_t)l * 2 + 1) * kv_tokens * p->nkv, M, p->nkv);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return proj_fail(PHYAI_ERR_CUDA, "kernel launch failed", e);
+  return PHYAI_OK;
+}
+
+// One-shot form: create, run, synchronise, destroy.
 extern "C" phyai_status_t phyai_project_features_kv(const phyai_kv_proj_desc_t* desc, const void* features,
                                                     const void* const* wk, const void* const* wv, uint64_t tokens,
                                                     uint64_t kv_tokens, void* prefix_kv, void* stream) {
-  using namespace phyai;
-  g_ad_err[0] = 0;
-  auto fail = [](phyai_status_t st, const char* msg, cudaError_t e = cudaSuccess) {
-    if (e != cudaSuccess) snprintf(g_ad_err, sizeof(g_ad_err), "%s: %s", msg, cudaGetErrorString(e));
-    else snprintf(g_ad_err, sizeof(g_ad_err), "%s", msg);
-    return st;
-  };
-  if (!desc || desc->struct_size != sizeof(phyai_kv_proj_desc_t) || !features || !wk || !wv || !prefix_kv)
-    return fail(PHYAI_ERR_INVALID_ARG, "NULL argument or wrong struct_size");
-  const int L = (int)desc->n_layers, nkv = (int)(desc->n_kv_heads * desc->head_dim), Dv = (int)desc->feat_dim;
-  if (L <= 0 || nkv <= 0 || Dv <= 0 || Dv % 64 || (2 * nkv) % 128 || tokens == 0 || tokens > kv_tokens || tokens > (1u << 22))
-    return fail(PHYAI_ERR_INVALID_ARG, "need feat_dim a multiple of 64, 2 * n_kv_heads * head_dim a multiple of 128, 1 <= tokens <= kv_tokens");
-  for (int l = 0; l < L; ++l)
-    if (!wk[l] || !wv[l]) return fail(PHYAI_ERR_INVALID_ARG, "a per-layer weight pointer is NULL");
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  cudaError_t e = tc_gemm_setup();
-  if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tc_gemm_setup", e);
-  const int M = (int)tokens, rows_pad = (M + 255) / 256 * 256, N = 2 * nkv;
-  __nv_bfloat16 *xt = nullptr, *wp = nullptr;
-  float* y = nullptr;
-  int* status = nullptr;
-  auto cleanup = [&]() { cudaFree(xt), cudaFree(wp), cudaFree(y), cudaFree(status); };
-  if ((e = cudaMalloc(&xt, (size_t)rows_pad * Dv * 2)) != cudaSuccess || (e = cudaMalloc(&wp, (size_t)Dv * N * 2)) != cudaSuccess ||
-      (e = cudaMalloc(&y, (size_t)M * N * 4)) != cudaSuccess || (e = cudaMalloc(&status, 4)) != cudaSuccess) {
-    cleanup();
-    return fail(PHYAI_ERR_OOM, "cudaMalloc", e);
-  }
-  cudaMemsetAsync(xt, 0, (size_t)rows_pad * Dv * 2, st);
-  cudaMemsetAsync(status, 0, 4, st);
-  launch_rows_to_tiled(reinterpret_cast<const __nv_bfloat16*>(features), xt, M, Dv, rows_pad, st);
-  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(prefix_kv);
-  for (int l = 0; l < L && e == cudaSuccess; ++l) {
-    launch_pack_tiled(wk[l], 1, wp, Dv, nkv, 0, st);
-    launch_pack_tiled(wv[l], 1, wp, Dv, nkv, nkv, st);
-    TcGemm g{};
-    g.W = wp, g.X = xt, g.M = M, g.N = N, g.K = Dv, g.epi = TC_STORE, g.out_f32 = y, g.ldo = N, g.splits = 1;
-    g.rows_pad = rows_pad, g.wait_limit = 1u << 28;
-    e = launch_tc_gemm(status, g, M <= 64 ? 64 : (M <= 1024 ? 128 : 256), st);
-    if (e != cudaSuccess) break;
-    const size_t n = (size_t)M * (nkv >> 2) * 2;
-    k_kv_planes<<<(int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096), 256, 0, st>>>(
-        y, out + ((size_t)l * 2) * kv_tokens * nkv, out + ((size_t)l * 2 + 1) * kv_tokens * nkv, M, nkv);
-  }
-  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  phyai_kv_projector_t* p = nullptr;
+  phyai_status_t st = phyai_kv_projector_create(desc, wk, wv, tokens ? tokens : 1, stream, &p);
+  if (st != PHYAI_OK) return st;
+  st = phyai_kv_projector_run(p, features, tokens, kv_tokens, prefix_kv, stream);
+  cudaError_t e = cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream));
   int hs = 0;
-  if (e == cudaSuccess) e = cudaMemcpy(&hs, status, 4, cudaMemcpyDeviceToHost);
-  cleanup();
-  if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "feature K/V projection", e);
-  if (hs != 0) return fail(PHYAI_ERR_TIMEOUT, "a bounded device-side wait expired");
+  if (e == cudaSuccess) e = cudaMemcpy(&hs, p->status, 4, cudaMemcpyDeviceToHost);
+  phyai_kv_projector_destroy(p);
+  if (st != PHYAI_OK) return st;
+  if (e != cudaSuccess) return proj_fail(PHYAI_ERR_CUDA, "feature K/V projection", e);
+  if (hs != 0) return proj_fail(PHYAI_ERR_TIMEOUT, "a bounded device-side wait expired");
   return PHYAI_OK;
 }

@@ -151,3 +151,20 @@ def test_feature_handoff_head_end_to_end(batch):
         err = O.max_rel_err(out[b], ref)
         print(f"feature-handoff head, request {b}: max rel err {err:.2e}")
         assert err <= 2e-2, (b, err)
+
+
+def test_projector_handle_gives_the_one_shot_result_for_every_token_count():
+    cfg = synth.ExpertConfig(n_layers=3, width=256, mlp_dim=512, n_q_heads=4, n_kv_heads=2, head_dim=128, state_dim=4,
+                             action_dim=4, horizon=4, has_state_token=True, max_prefix_len=700, max_batch=1, cond="pi0",
+                             dtype="bf16")
+    wk, wv = synth.make_kv_projections(cfg, 43, 512)
+    wk, wv = [w.cuda() for w in wk], [w.cuda() for w in wv]
+    with binding.KvProjector(wk, wv, 2, 128, max_tokens=700) as proj:
+        for tokens in (700, 1, 64, 333):                      # one handle, shrinking and growing inputs
+            F = synth.make_features(43, tokens, 512, request=tokens).cuda()
+            a = proj.run(F)
+            torch.cuda.synchronize()
+            b = binding.project_features_kv(F, wk, wv, 2, 128)
+            assert torch.equal(a, b), tokens
+        with pytest.raises(binding.PhyaiError):
+            proj.run(synth.make_features(43, 701, 512).cuda())
