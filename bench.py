@@ -11,6 +11,11 @@ events on the launching stream; ``e2e`` goes through the host-buffer entry point
 inputs, host<->device copies inside the timed region).  ``--impl reference`` times the float64 CPU
 oracle on the host cores instead.  Under torchrun every rank runs an independent replica (the
 path shards by request, no collective); rank 0 reports the maximum time over ranks.
+
+Workloads: C2 (pi0-shaped, bf16, batch 1: the headline), C2m (C2 with the block-causal mask), C3 (pi0.5-shaped), C4
+(batch 64, ragged prefixes), C5b1 / b8 / b64 / b256 (e4m3 weights), C6b8 / b64 / b256 (e4m3 weights and per-token e4m3
+activations: W8A8), C7b1 (int4 weights), G1 (a GR00T-shaped feature-handoff head: K / V projections of the features,
+then four steps on a 40 x 132 chunk).  A run without --workload reports C2 on the line and the others in ``workloads``.
 """
 from __future__ import annotations
 
