@@ -47,3 +47,33 @@ def test_expired_wait_is_reported_and_the_handle_recovers(cluster_gemm, batch):
         # (beyond 64 tokens the split-K residual adds are atomic, so two runs agree to rounding, not to the bit)
         assert rel_err(again[0].double().cpu().numpy(), ref0) <= BAR["bf16"]
         assert rel_err(again.double().cpu().numpy(), good.double().cpu().numpy()) <= BAR["bf16"]
+
+
+@pytest.mark.parametrize("cond,dtype", [("pi0", "bf16"), ("pi05", "bf16"), ("pi0", "w8e4m3"), ("pi0", "w4a16")])
+def test_expired_waits_in_the_full_width_single_tile_kernels(cond, dtype):
+    """Width 1024: the step-boundary cluster kernel, the one-head-per-CTA attention kernel with its bulk-copied Q tile
+    and the stage-by-stage weight decode all have waits of their own; lowered to one poll they give up (the data
+    still arrives), the call returns with TIMEOUT, and the handle is good again afterwards."""
+    cfg = synth.ExpertConfig(n_layers=2, width=1024, mlp_dim=4096, n_q_heads=8, n_kv_heads=1, head_dim=256, state_dim=32,
+                             action_dim=32, horizon=50, has_state_token=(cond == "pi0"), max_prefix_len=300, max_batch=1,
+                             cond=cond, dtype=dtype)
+    W = synth.make_weights(cfg, 32)
+    kv = synth.make_prefix_kv(cfg, 32, 300)
+    state = synth.make_state(cfg, 32) if cfg.has_state_token else None
+    noise = synth.make_noise(cfg, 32)
+    ref = O.denoise(cfg, W, kv, 300, state, noise, 3)
+    dev = lambda t: None if t is None else t.cuda()
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        good = ex.denoise(dev(kv), 300, dev(state), dev(noise), 3).clone()
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        assert rel_err(good.double().cpu().numpy(), ref) <= BAR["bf16"]
+        ex.set_option("wait_limit", 1)
+        ex.denoise(dev(kv), 300, dev(state), dev(noise), 3)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == binding.ERR_TIMEOUT
+        ex.set_option("wait_limit", 1 << 22)
+        again = ex.denoise(dev(kv), 300, dev(state), dev(noise), 3)
+        torch.cuda.synchronize()
+        assert ex.poll_status() == 0
+        assert torch.equal(again, good)              # the single-tile path is bit-reproducible
