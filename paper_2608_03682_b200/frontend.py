@@ -26,9 +26,15 @@ class ExpertWorker:
 
     def __init__(self, expert, cfg, n_steps: int, device="cuda"):
         self.ex, self.cfg, self.n_steps, self.device = expert, cfg, n_steps, device
+        self.stream = None      # created on first use (CUDA only)
 
-    def __call__(self, requests: List[Optional[dict]]) -> List[np.ndarray]:
+    def launch(self, requests: List[Optional[dict]]):
+        """Enqueue one local batch on the worker's own stream and return at once (the paper's RTC schedule prepares the
+        next action chunk while the current one is being executed: a caller launches the next request here and
+        collects it when the controller is ready for the hand-over).  One batch in flight per worker."""
         cfg = self.cfg
+        if self.stream is None:
+            self.stream = torch.cuda.Stream(device=self.device)
         kv_dtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
         empty = torch.zeros(cfg.n_layers, 2, 0, cfg.n_kv_heads, cfg.head_dim, dtype=kv_dtype)
         kvs = [empty if r is None else r["prefix_kv"] for r in requests]
@@ -40,14 +46,26 @@ class ExpertWorker:
         noise = torch.stack([torch.zeros(cfg.horizon, cfg.action_dim) if r is None else r["noise"] for r in requests])
         states = None
         if cfg.has_state_token:
-            states = torch.stack([torch.zeros(cfg.state_dim) if r is None else r["state"] for r in requests]).to(self.device)
-        out = self.ex.denoise_batched(packed.to(self.device), torch.from_numpy(cu).to(self.device), states,
-                                      noise.to(self.device), self.n_steps)
-        torch.cuda.synchronize()
+            states = torch.stack([torch.zeros(cfg.state_dim) if r is None else r["state"] for r in requests])
+        host = [packed.pin_memory(), torch.from_numpy(cu).pin_memory(), None if states is None else states.pin_memory(),
+                noise.pin_memory()]
+        with torch.cuda.stream(self.stream):
+            dev = [None if t is None else t.to(self.device, non_blocking=True) for t in host]
+            out = self.ex.denoise_batched(dev[0], dev[1], dev[2], dev[3], self.n_steps, stream=self.stream)
+            done = torch.cuda.Event()
+            done.record(self.stream)
+        return {"out": out, "done": done, "keep": (host, dev)}
+
+    def collect(self, pending) -> List[np.ndarray]:
+        """Wait for a launched batch and return its action chunks."""
+        pending["done"].synchronize()
         status = self.ex.poll_status()
         if status != 0:
             raise RuntimeError(f"device status {status}")
-        return [o.cpu().numpy() for o in out]
+        return [o.cpu().numpy() for o in pending["out"]]
+
+    def __call__(self, requests: List[Optional[dict]]) -> List[np.ndarray]:
+        return self.collect(self.launch(requests))
 
 
 class DPFrontend:

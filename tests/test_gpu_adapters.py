@@ -104,6 +104,26 @@ def test_frontend_worker_pads_the_local_batch_to_its_fixed_shape():
         assert rel_err(out[rid], ref) <= BAR["bf16"], (rid, rel_err(out[rid], ref))
 
 
+def test_two_workers_prepare_the_next_chunk_while_the_first_is_in_flight():
+    """launch / collect: two handles on two streams, both batches enqueued before either is collected (the RTC
+    schedule: the next chunk is prepared during the current execution window); results equal the blocking calls."""
+    from paper_2608_03682_b200.frontend import ExpertWorker
+    from tests.helpers import small_bf16_config
+    cfg = small_bf16_config("pi0", max_batch=2, max_prefix_len=120)
+    W = synth.make_weights(cfg, 26, std=0.05)
+    mk = lambda b, p: dict(prefix_kv=synth.make_prefix_kv(cfg, 26, p, b), state=synth.make_state(cfg, 26, b),
+                           noise=synth.make_noise(cfg, 26, b), n_steps=3)
+    batch_a, batch_b = [mk(0, 120), mk(1, 33)], [mk(2, 77), None]
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex_a, binding.Expert(cfg, binding.weights_to_device(W)) as ex_b:
+        wa, wb = ExpertWorker(ex_a, cfg, 3), ExpertWorker(ex_b, cfg, 3)
+        pa = wa.launch(batch_a)
+        pb = wb.launch(batch_b)                      # enqueued while the first batch is still running
+        out_b, out_a = wb.collect(pb), wa.collect(pa)
+        ref_a, ref_b = wa(batch_a), wb(batch_b)
+    for got, ref in zip(out_a + out_b[:1], ref_a + ref_b[:1]):
+        assert np.array_equal(got, ref)
+
+
 # ------------------------------------------------------------------ feature-handoff head: request-local K / V projections
 @pytest.mark.parametrize("tokens,feat_dim,n_kv,dh,layers", [(300, 512, 2, 128, 3), (37, 1024, 1, 256, 2), (1500, 256, 2, 64, 2)])
 def test_feature_projection_matches_oracle(tokens, feat_dim, n_kv, dh, layers):
