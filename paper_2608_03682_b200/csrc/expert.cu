@@ -106,6 +106,8 @@ struct phyai_expert {
   int use_fused_oproj = 1;     // cluster attention also does the output projection of its head (general GEMM path only)
   int n_sm = 0;
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
+  __nv_bfloat16* p_gu16 = nullptr;          // gate/up interleaved in groups of 16 channels (persistent gate/up kernel)
+  int use_persistent_gu = 1;
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
   __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
@@ -332,6 +334,9 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       if (g.splits > h->slab_splits) g.splits = h->slab_splits;
       g.slab = h->slab, pending_slabs = g.splits;
     }
+    // trace_all_from = n: launch n of the call, if it is a tile GEMM, stamps one slot per CTA
+    const long n_cta = (long)(g.N / 128) * ((g.M + 63) / 64) * (g.splits > 0 ? g.splits : 1);
+    g.trace = (h->trace && h->trace_all_from > 0 && cnt == h->trace_all_from && n_cta <= TRACE_SLOTS) ? h->trace : nullptr;
     cudaError_t e = launch_tc_gemm(h->status, g, g.nt_override ? g.nt_override : nt, st);
     if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "tensor GEMM launch failed: %s", cudaGetErrorString(e));
     ++cnt;
@@ -614,7 +619,24 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
           // a single token tile: interleaved gate / up tiles put the weight stream on twice as many SMs
           g.W = h->p_gu_all + (size_t)l * D * 2 * d.F, g.W2 = nullptr, g.N = 2 * d.F, g.epi = TC_GEGLU_IL;
         }
-        ST(tc_gemm(g, norm_q8));
+        if (nt == 256 && h->p_gu16 && h->use_persistent_gu && gu_gemm_supported(M, d.F, D, h->Mpad, h->a8)) {
+          if (h->a8 && !norm_q8) {
+            launch_quant_rows(h->status, h->xn_t, h->xq, h->xs, h->Mpad, M, D, st);
+            ++cnt;
+          }
+          GuGemm p{};
+          p.W = h->p_gu16 + (size_t)l * D * 2 * d.F / (h->a8 ? 2 : 1);
+          p.X = h->a8 ? reinterpret_cast<const __nv_bfloat16*>(h->xq) : h->xn_t;
+          p.out_tiled = h->m_t, p.scale_g = h->s_g[l], p.scale_u = h->s_u[l], p.xscale = h->a8 ? h->xs : nullptr;
+          p.M = M, p.F = d.F, p.K = D, p.rows_pad = h->Mpad, p.gelu_exact = d.gelu_exact, p.fp8 = h->a8 ? 1 : 0;
+          p.wait_limit = h->wait_limit;
+          p.trace = (h->trace && h->trace_all_from > 0 && cnt == h->trace_all_from) ? h->trace : nullptr;
+          cudaError_t e = launch_gu_gemm(h->status, p, h->n_sm, st);
+          if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "gate/up GEMM launch failed: %s", cudaGetErrorString(e));
+          ++cnt;
+        } else {
+          ST(tc_gemm(g, norm_q8));
+        }
         TcGemm g2{};
         g2.W = h->p_d[l], g2.X = h->m_t, g2.N = D, g2.K = d.F, g2.epi = TC_RESID, g2.scale = h->s_d[l], g2.gate = gate;
         g2.out_f32 = h->h, g2.ldo = D, g2.splits = pick_splits(D / 128 / ((nt == 256 && D % 256 == 0) ? 2 : 1), tok_tiles, d.F / kcb);
@@ -776,6 +798,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
 
   auto body = [&]() -> phyai_status_t {
     if (tc) CU(tc_gemm_setup());
+    if (tc) CU(gu_gemm_setup());
     {
       int dev = 0;
       CU(cudaGetDevice(&dev));
@@ -864,6 +887,9 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       ST(h->alloc(&pd_all, (size_t)L * F * D));
       h->il_ok = F % 64 == 0 && !a8;   // (W8A8 keeps to the general kernels: no interleaved image, no cluster path)
       if (h->il_ok) ST(h->alloc(&h->p_gu_all, (size_t)L * D * 2 * F));
+      // token counts that use 256-token tiles: the persistent gate / up kernel and its weight image
+      if (pick_nt((int)(cfg->max_batch * d.S)) == 256 && gu_gemm_supported((int)(cfg->max_batch * d.S), F, D, h->Mpad, a8))
+        ST(h->alloc(&h->p_gu16, (size_t)L * D * 2 * F / (a8 ? 2 : 1)));
       // cluster split-K path (one 64-token tile): every projection must fit the kernel's resident stages
       auto fits = [&](int N, int K, bool qkv) {
         return b1_gemm_supported(N, K, b1_pick_cluster(N / 128, K / 64, h->n_sm), h->n_sm, qkv);
@@ -884,6 +910,17 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       if (tc) {
         __nv_bfloat16 *pq = pq_all + (size_t)l * D * Nqkv, *po = po_all + (size_t)l * Nq * D;
         __nv_bfloat16 *pg = pg_all + (size_t)l * D * F, *pu = pu_all + (size_t)l * D * F, *pd = pd_all + (size_t)l * F * D;
+        if (h->p_gu16) {
+          // (bf16 image: 2 bytes per weight; W8A8: the e4m3 codes, 1 byte per weight, in the first half of the layer's slot)
+          __nv_bfloat16* p16 = h->p_gu16 + (size_t)l * D * 2 * F / (a8 ? 2 : 1);
+          if (a8) {
+            launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wgate[l]), reinterpret_cast<uint8_t*>(p16), D, F, 0, st, 16, 0, 0, 1);
+            launch_pack_bytes(reinterpret_cast<const uint8_t*>(w->wup[l]), reinterpret_cast<uint8_t*>(p16), D, F, 0, st, 16, 1, 0, 1);
+          } else {
+            launch_pack_tiled(w->wgate[l], big_kind, p16, D, F, 0, st, 16, 0);
+            launch_pack_tiled(w->wup[l], big_kind, p16, D, F, 0, st, 16, 1);
+          }
+        }
         if (h->il_ok) {
           __nv_bfloat16* pgu = h->p_gu_all + (size_t)l * D * 2 * F;
           launch_pack_tiled(w->wgate[l], big_kind, pgu, D, F, 0, st, 64, 0);
@@ -1222,6 +1259,12 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     }
     if (!h->trace_buf) ST(h->alloc(&h->trace_buf, (size_t)TRACE_SLOTS * TRACE_STAMPS, true));
     h->trace = h->trace_buf;
+    return PHYAI_OK;
+  }
+  if (!strcmp(key, "use_persistent_gu")) {
+    h->use_persistent_gu = value != 0;
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
     return PHYAI_OK;
   }
   if (!strcmp(key, "trace_all_from")) {

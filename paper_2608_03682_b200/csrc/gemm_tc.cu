@@ -100,6 +100,9 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   // to pdl_wait() touches only shared / tensor memory and the weights (constants): barriers, TMEM, and the weight
   // halves of the first STAGES stages are in flight before the activations this GEMM depends on exist.
   pdl_launch_dependents();
+  unsigned long long* const trc =
+      g.trace ? g.trace + (size_t)((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 16 : nullptr;
+  if (threadIdx.x == 0) trace_stamp(trc, 0);
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles_ptr = smem_raw + (tiles - smem_u32(smem_raw));
   if (threadIdx.x == 0) {
@@ -117,6 +120,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   }
   __syncthreads();
   tc_fence_after();
+  if (threadIdx.x == 0) trace_stamp(trc, 1);
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, *reinterpret_cast<volatile uint32_t*>(&tmem_slot), 0);
   const WaitCtx wc{status, &abort_flag, g.wait_limit};
 
@@ -142,6 +146,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     }
   }
   pdl_wait();
+  if (threadIdx.x == 0) trace_stamp(trc, 2);
   // The activation copies of the prefetched stages go out before the status word is known (their addresses do not
   // depend on the request, and the skip path below waits for them): the status read, a round trip to the L2, then
   // overlaps their latency.  It is made by the MMA warp, which issues no copies.
@@ -207,6 +212,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
       const int s = i % STAGES;
       const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
       const bool ok = mbar_wait_drain(smem_u32(&bar_full[s]), ph, wc) > 0;
+      if (i == 0 && lane == 0) trace_stamp(trc, 3);
       // (no tcgen05 fence here: the operands were written by the bulk-copy engine and made visible by the mbarrier;
       // tcgen05.fence::after_thread_sync orders tensor-memory accesses, and it was measured to hold the next MMAs
       // back until the previous stage's MMAs had drained)
@@ -240,6 +246,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     }
     if (elect_one()) umma_commit(smem_u32(&bar_accum));
     __syncwarp();
+    if (warp == 8 && lane == 0) trace_stamp(trc, 4);
   }
   if (warp <= 8) {
     // (producer warps and the first MMA warp have nothing else to do)
@@ -337,6 +344,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
     epi_sync();
     const bool ok = *reinterpret_cast<volatile int*>(&epi_ok) != 0;
     tc_fence_after();
+    if (et == 0) trace_stamp(trc, 5);
     if constexpr (F8) {
       if (et < NT) xs_tab[et] = xs_reg;
       epi_sync();
@@ -352,6 +360,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         const int n_out = (g.perm_dh && n < g.perm_end) ? qkv_packed_to_channel(n, g.perm_dh) : n;
         const float gt = e_gt[a];
         const float bs = e_bs[a];
+#pragma unroll 1
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;  // warp-uniform
           float v[16];
@@ -433,6 +442,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         const int rows = min(NT, g.M - tok_base);
         uint4* dst = reinterpret_cast<uint4*>(g.out_tiled + ((size_t)nt_idx * g.rows_pad + tok_base) * 64);
         const uint4* src = reinterpret_cast<const uint4*>(img);
+#pragma unroll 1
         for (int idx = et; idx < rows * 8; idx += NEPI) dst[idx] = src[idx];
       }
     }
@@ -448,6 +458,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         const int n0 = (nt_idx * NA + a) * 128;
         if (ok) {
           const float sc = e_sc[a] * e_gt[a];
+#pragma unroll 1
           for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
             if (tok_base + c0 >= g.M) break;          // warp-uniform
             float v[16];
@@ -458,6 +469,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         }
         epi_sync();
         if (ok) {
+#pragma unroll 1
           for (int it = et; it < rows * 32; it += NEPI) {
             const int tl = it >> 5, j0 = (it & 31) * 4;
             const float4 x = *reinterpret_cast<const float4*>(stage + (size_t)tl * PITCH + j0);
@@ -489,6 +501,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         const int n0 = (nt_idx * NA + a) * 128;       // first packed row of this accumulator
         if (ok) {
           const float sc = a == 0 ? sc_pre : (g.scale ? g.scale[n0 + ch] : 1.0f);
+#pragma unroll 1
           for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
             if (tok_base + c0 >= g.M) break;          // warp-uniform
             float v[16];
@@ -524,6 +537,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
             } else if (et < rows * 8) {
               fetch(et);
             }
+#pragma unroll 1
             for (int it = et; it < rows * 8; it += NEPI) {
               const int tl = it >> 3, j0 = (it & 7) * 8;
               const int2 e = e_next;
@@ -560,6 +574,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
           } else {
             const int nn = n0 - Nq - Nk;
             const int head = nn / g.dh, coff = nn - head * g.dh;       // 128 consecutive v channels
+#pragma unroll 1
             for (int it = et; it < rows * 16; it += NEPI) {
               const int tl = it >> 4, j0 = (it & 15) * 8;
               const int2 e = tok_tab[tl];
@@ -588,6 +603,7 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         const int n = nt_idx * 128 + ch;
         const float sg = g.scale ? g.scale[n] : 1.0f, su = g.scale2 ? g.scale2[n] : 1.0f;
         const int kc_sel = ch >> 6, c64 = ch & 63;
+#pragma unroll 1
         for (int c0 = c_begin; c0 < c_begin + HALF; c0 += 16) {
           if (tok_base + c0 >= g.M) break;
           float vg[16], vu[16];
@@ -611,11 +627,20 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
         for (int kc_sel = 0; kc_sel < 2; ++kc_sel) {
           uint4* dst = reinterpret_cast<uint4*>(g.out_tiled + ((size_t)(nt_idx * 2 + kc_sel) * g.rows_pad + tok_base) * 64);
           const uint4* src = reinterpret_cast<const uint4*>(img + (size_t)kc_sel * NT * 64);
+#pragma unroll 1
           for (int idx = et; idx < rows * 8; idx += NEPI) dst[idx] = src[idx];
         }
       }
     }
     tc_fence_before();
+    if (et == 0 && trc) {
+      // (own stores issued; the timer read is tied to this point by the memory clobber)
+      unsigned long long t;
+      unsigned sm;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+      trc[6] = t, trc[7] = sm;
+    }
   }
 
   __syncthreads();
@@ -623,6 +648,11 @@ __global__ void __launch_bounds__(800, 1) k_gemm_tc(int* status, const TcGemm g)
   if (warp == 8) {
     tc_fence_after();
     tmem_dealloc(tmem_base, ALLOC_COLS);
+    if (lane == 0 && trc) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
+      trc[8] = t;
+    }
   }
 }
 

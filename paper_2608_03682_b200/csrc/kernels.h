@@ -196,6 +196,9 @@ struct TcGemm {
   // W8A8: W and X hold e4m3 codes (128-byte rows = 128 k per block / tile chunk), the product runs on the FP8 tensor
   // path and every accumulator column is multiplied by its token's activation scale
   int fp8;
+  unsigned long long* trace;   // or null: every CTA stamps into slot (linear block index) x 16: start, set-up done,
+                               // dependency resolved, first operands landed, MMAs issued, accumulator complete, stores
+                               // done, (SM id)
   const float* xscale;   // [rows] per-token activation scale (fp8 only)
   const float* scale2;
   const float* bias;   // TC_BIAS_ROWMAP
@@ -223,6 +226,26 @@ struct TcGemm {
 // Returns cudaSuccess or the launch error; `nt` is the token-tile width (64, 128 or 256).
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st);
 cudaError_t tc_gemm_setup();  // one-time attribute setup (dynamic shared memory opt-in)
+
+// Persistent gate / up projection with the GeGLU epilogue (gemm_gu.cu): 128-row weight tiles that hold the gate and
+// up rows of the same 64 channels (rows 32 q + i = gate, 32 q + 16 + i = up of channel 16 q + i of the tile), 256-token
+// tiles, two accumulators in tensor memory so that the epilogue of a tile overlaps the main loop of the next.
+struct GuGemm {
+  const __nv_bfloat16* W;       // interleaved image: (2 F / 128) tiles x KC blocks of 128 rows x 128 bytes (bf16 or e4m3)
+  const __nv_bfloat16* X;       // tiled activations [KC][rows_pad][128 bytes]
+  __nv_bfloat16* out_tiled;     // [F / 64][rows_pad][64] bf16, 16-byte chunks swizzled by row & 7
+  const float* scale_g;         // per-channel weight scales or null
+  const float* scale_u;
+  const float* xscale;          // fp8: per-token activation scales
+  int M, F, K, rows_pad;
+  int gelu_exact, fp8;
+  unsigned wait_limit;
+  unsigned long long* trace;    // or null: CTA b stamps slot b (16 words)
+};
+bool gu_gemm_supported(int M, int F, int K, int rows_pad, bool fp8);
+int gu_gemm_ctas(const GuGemm& g, int n_sm);
+cudaError_t gu_gemm_setup();
+cudaError_t launch_gu_gemm(int* status, const GuGemm& g, int n_sm, cudaStream_t st);
 // ---- cluster split-K GEMM for a single 64-token tile (gemm_b1.cu) --------------------------------------------
 enum : int { B1_QKV = 0, B1_GEGLU = 1, B1_RESID = 2 };
 struct B1Gemm {
