@@ -12,7 +12,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libphyai.so")
-SOURCES = ["expert.cu", "simt.cu", "gemm_tc.cu", "gemm_gu.cu", "gemm_b1.cu", "step_b1.cu", "attention.cu", "attention_tc.cu", "attention_b1.cu", "adapters.cu", "w8a8_op.cu", "frontend.cu"]
+SOURCES = ["expert.cu", "simt.cu", "gemm_tc.cu", "gemm_persist.cu", "gemm_b1.cu", "step_b1.cu", "attention.cu", "attention_tc.cu", "attention_b1.cu", "adapters.cu", "w8a8_op.cu", "frontend.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

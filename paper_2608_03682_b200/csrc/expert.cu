@@ -106,8 +106,9 @@ struct phyai_expert {
   int use_fused_oproj = 1;     // cluster attention also does the output projection of its head (general GEMM path only)
   int n_sm = 0;
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
-  __nv_bfloat16* p_gu16 = nullptr;          // gate/up interleaved in groups of 16 channels (persistent gate/up kernel)
-  int use_persistent_gu = 1;
+  __nv_bfloat16* p_gu16 = nullptr;          // gate/up interleaved in groups of 16 channels (persistent tile GEMM)
+  __nv_bfloat16* p_qkv16 = nullptr;         // q|k|v with the rows of every tile interleaved in groups of 16 (the same kernel)
+  int use_persistent_gu = 1, use_persistent_qkv = 1;
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
   __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
@@ -561,7 +562,26 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
           g.epi = TC_QKV_ROT, g.rq = h->rq, g.rope = h->rope, g.qr = h->qr_big, g.kr = h->kr_big, g.vr = h->vr_big;
           g.S = d.S, g.Hq = d.Hq, g.Hkv = d.Hkv, g.dh = d.dh;
         }
-        ST(tc_gemm(g, norm_q8));
+        if (attn_rot && nt == 256 && h->p_qkv16 && h->use_persistent_qkv && persist_gemm_supported(M, d.Nqkv, D, h->Mpad, h->a8)) {
+          if (h->a8 && !norm_q8) {
+            launch_quant_rows(h->status, h->xn_t, h->xq, h->xs, h->Mpad, M, D, st);
+            ++cnt;
+          }
+          PersistGemm p{};
+          p.W = h->p_qkv16 + (size_t)l * D * d.Nqkv / (h->a8 ? 2 : 1);
+          p.X = h->a8 ? reinterpret_cast<const __nv_bfloat16*>(h->xq) : h->xn_t;
+          p.scale_g = h->s_qkv[l], p.xscale = h->a8 ? h->xs : nullptr;
+          p.M = M, p.N = d.Nqkv, p.K = D, p.rows_pad = h->Mpad, p.fp8 = h->a8 ? 1 : 0, p.qkv = 1;
+          p.wait_limit = h->wait_limit;
+          p.rq = h->rq, p.rope = h->rope, p.qr = h->qr_big, p.kr = h->kr_big, p.vr = h->vr_big;
+          p.S = d.S, p.Hq = d.Hq, p.Hkv = d.Hkv, p.dh = d.dh;
+          p.trace = (h->trace && h->trace_all_from > 0 && cnt == h->trace_all_from) ? h->trace : nullptr;
+          cudaError_t e = launch_persist_gemm(h->status, p, h->n_sm, st);
+          if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "q|k|v GEMM launch failed: %s", cudaGetErrorString(e));
+          ++cnt;
+        } else {
+          ST(tc_gemm(g, norm_q8));
+        }
       } else {
         SimtGemm g{};
         g.A = h->xn_f, g.lda = D, g.B = h->f_qkv[l], g.M = M, g.N = d.Nqkv, g.K = D, g.epi = EPI_STORE;
@@ -619,19 +639,19 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
           // a single token tile: interleaved gate / up tiles put the weight stream on twice as many SMs
           g.W = h->p_gu_all + (size_t)l * D * 2 * d.F, g.W2 = nullptr, g.N = 2 * d.F, g.epi = TC_GEGLU_IL;
         }
-        if (nt == 256 && h->p_gu16 && h->use_persistent_gu && gu_gemm_supported(M, d.F, D, h->Mpad, h->a8)) {
+        if (nt == 256 && h->p_gu16 && h->use_persistent_gu && persist_gemm_supported(M, 2 * d.F, D, h->Mpad, h->a8)) {
           if (h->a8 && !norm_q8) {
             launch_quant_rows(h->status, h->xn_t, h->xq, h->xs, h->Mpad, M, D, st);
             ++cnt;
           }
-          GuGemm p{};
+          PersistGemm p{};
           p.W = h->p_gu16 + (size_t)l * D * 2 * d.F / (h->a8 ? 2 : 1);
           p.X = h->a8 ? reinterpret_cast<const __nv_bfloat16*>(h->xq) : h->xn_t;
           p.out_tiled = h->m_t, p.scale_g = h->s_g[l], p.scale_u = h->s_u[l], p.xscale = h->a8 ? h->xs : nullptr;
-          p.M = M, p.F = d.F, p.K = D, p.rows_pad = h->Mpad, p.gelu_exact = d.gelu_exact, p.fp8 = h->a8 ? 1 : 0;
+          p.M = M, p.N = 2 * d.F, p.K = D, p.rows_pad = h->Mpad, p.gelu_exact = d.gelu_exact, p.fp8 = h->a8 ? 1 : 0;
           p.wait_limit = h->wait_limit;
           p.trace = (h->trace && h->trace_all_from > 0 && cnt == h->trace_all_from) ? h->trace : nullptr;
-          cudaError_t e = launch_gu_gemm(h->status, p, h->n_sm, st);
+          cudaError_t e = launch_persist_gemm(h->status, p, h->n_sm, st);
           if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "gate/up GEMM launch failed: %s", cudaGetErrorString(e));
           ++cnt;
         } else {
@@ -798,7 +818,7 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
 
   auto body = [&]() -> phyai_status_t {
     if (tc) CU(tc_gemm_setup());
-    if (tc) CU(gu_gemm_setup());
+    if (tc) CU(persist_gemm_setup());
     {
       int dev = 0;
       CU(cudaGetDevice(&dev));
@@ -888,8 +908,10 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
       h->il_ok = F % 64 == 0 && !a8;   // (W8A8 keeps to the general kernels: no interleaved image, no cluster path)
       if (h->il_ok) ST(h->alloc(&h->p_gu_all, (size_t)L * D * 2 * F));
       // token counts that use 256-token tiles: the persistent gate / up kernel and its weight image
-      if (pick_nt((int)(cfg->max_batch * d.S)) == 256 && gu_gemm_supported((int)(cfg->max_batch * d.S), F, D, h->Mpad, a8))
+      if (pick_nt((int)(cfg->max_batch * d.S)) == 256 && persist_gemm_supported((int)(cfg->max_batch * d.S), 2 * F, D, h->Mpad, a8)) {
         ST(h->alloc(&h->p_gu16, (size_t)L * D * 2 * F / (a8 ? 2 : 1)));
+        if ((d.dh == 128 || d.dh == 256) && d.S <= 64) ST(h->alloc(&h->p_qkv16, (size_t)L * D * Nqkv / (a8 ? 2 : 1)));
+      }
       // cluster split-K path (one 64-token tile): every projection must fit the kernel's resident stages
       auto fits = [&](int N, int K, bool qkv) {
         return b1_gemm_supported(N, K, b1_pick_cluster(N / 128, K / 64, h->n_sm), h->n_sm, qkv);
@@ -919,6 +941,20 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
           } else {
             launch_pack_tiled(w->wgate[l], big_kind, p16, D, F, 0, st, 16, 0);
             launch_pack_tiled(w->wup[l], big_kind, p16, D, F, 0, st, 16, 1);
+          }
+        }
+        if (h->p_qkv16) {
+          __nv_bfloat16* p16 = h->p_qkv16 + (size_t)l * D * Nqkv / (a8 ? 2 : 1);
+          if (a8) {
+            auto u8 = [](const void* p) { return reinterpret_cast<const uint8_t*>(p); };
+            uint8_t* o8 = reinterpret_cast<uint8_t*>(p16);
+            launch_pack_bytes(u8(w->wq[l]), o8, D, Nq, 0, st, 0, 0, d.dh, 1, 1);
+            launch_pack_bytes(u8(w->wk[l]), o8, D, Nkv, Nq, st, 0, 0, d.dh, 1, 1);
+            launch_pack_bytes(u8(w->wv[l]), o8, D, Nkv, Nq + Nkv, st, 0, 0, 0, 1, 1);
+          } else {
+            launch_pack_tiled(w->wq[l], big_kind, p16, D, Nq, 0, st, 0, 0, d.dh, 1);
+            launch_pack_tiled(w->wk[l], big_kind, p16, D, Nkv, Nq, st, 0, 0, d.dh, 1);
+            launch_pack_tiled(w->wv[l], big_kind, p16, D, Nkv, Nq + Nkv, st, 0, 0, 0, 1);
           }
         }
         if (h->il_ok) {
@@ -1261,8 +1297,8 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     h->trace = h->trace_buf;
     return PHYAI_OK;
   }
-  if (!strcmp(key, "use_persistent_gu")) {
-    h->use_persistent_gu = value != 0;
+  if (!strcmp(key, "use_persistent_gu") || !strcmp(key, "use_persistent_qkv")) {
+    (!strcmp(key, "use_persistent_gu") ? h->use_persistent_gu : h->use_persistent_qkv) = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

@@ -1,19 +1,21 @@
-// Gate / up projection with the GeGLU epilogue for many token tiles (Sec. 3.2: the MLP's first layer,
-// m = gelu(x Wg) * (x Wu)), as a persistent kernel: one CTA per SM walks over output tiles, and the epilogue of one
-// tile runs while the tensor cores work on the next.
+// Persistent tile GEMM for many token tiles: one CTA per SM walks over 128-row x 256-token output tiles, and the
+// epilogue of one tile runs while the tensor cores work on the next.  Two epilogues: the gate / up projection with
+// GeGLU (Sec. 3.2: the MLP's first layer, m = gelu(x Wg) * (x Wu)) and the fused q | k | v projection with the rotary
+// embedding (the attention kernel's operands, bf16).
 //
-// Why a kernel of its own.  With one 256-token x 256-row tile per CTA (gate and up accumulators of 128 channels) the
-// 512 tensor-memory columns are full, so a tile's epilogue (3.5 - 5 us of fp32 work for 65536 accumulator values, 8 us
-// on the first CTA of an SM while the code is fetched) cannot overlap anything: measured per tile 9.9 us of main loop,
-// 5 - 11 us of epilogue, ~2.5 us of launch / set-up / first operands, i.e. the tensor pipe idles half the time.  Here a
-// tile is 128 weight rows x 256 tokens (256 columns), two accumulators alternate, and the weight rows are interleaved
-// so that a tile holds gate AND up of the same 64 channels: rows 32 q + i (i < 16) are the gate rows of channels
-// 16 q + i, rows 32 q + 16 + i the up rows of the same channels.  A channel's gate and up values then sit in the same
-// warp's tensor-memory lanes i and i + 16, meet through one warp shuffle, and the result goes straight to global memory:
-// no shared-memory staging, no barrier among the epilogue warps, and the operand stages stay with the main loop.
+// Why a kernel of its own.  With one 256-token x 256-row tile per CTA (two accumulators of 128 rows) the 512
+// tensor-memory columns are full, so a tile's epilogue (3.5 - 5 us of fp32 work for 65536 accumulator values, 8 - 12 us
+// on the first CTA of an SM while the code is fetched) cannot overlap anything: measured per tile of the gate / up
+// projection 9.9 us of main loop, 5 - 11 us of epilogue, ~2.5 us of launch / set-up / first operands, i.e. the tensor
+// pipe idles half the time.  Here a tile is 128 weight rows x 256 tokens (256 columns), two accumulators alternate, and
+// the weight rows are interleaved so that the two rows which the epilogue combines sit in one warp's tensor-memory
+// lanes i and i + 16: rows 32 q + i (i < 16) are the gate rows (q / k: the first-half channels) of 16 channels, rows
+// 32 q + 16 + i the up rows (the rotary partners) of the same channels.  They meet through one warp shuffle and the
+// result goes straight to global memory: no shared-memory staging, no barrier among the epilogue warps (q | k | v: one
+// per tile, for the token table), and the operand stages stay with the main loop.
 // The price is 48 KB instead of 64 KB of operands per (128 x 256 x 64) MACs x 2, i.e. 1.5 x the bytes per flop: the
-// main loop runs at the SM's ingest rate (measured 62 bytes per clock with all SMs streaming), ~6.4 us per tile, which
-// still beats 17 - 24 us per pair of such tiles.
+// main loop runs at the SM's ingest rate (measured 62 bytes per clock with all SMs streaming), ~6.4 us per tile at
+// K = 1024, which still beats 17 - 24 us per pair of such tiles.
 //
 // Roles (800 threads): warps 0-7 issue bulk copies (one weight block of 16 KB and two activation pieces of 16 KB per
 // k-chunk, four stages), warp 8 issues the MMAs, warps 9-24 are the epilogue (tensor-memory lane quarter = warp % 4,
@@ -27,6 +29,7 @@ namespace phyai {
 namespace {
 
 constexpr int GU_NT = 256;                  // tokens per tile
+constexpr int BAR_PEPI = 1, NPEPI = 512;    // named barrier of the 16 epilogue warps
 constexpr int GU_STAGES = 4;
 constexpr int GU_A_BYTES = 128 * 128;       // weight block: 128 rows x 128 bytes
 constexpr int GU_B_PIECE = 128 * 128;       // activation piece: 128 tokens x 128 bytes
@@ -36,8 +39,8 @@ constexpr int GU_NPROD = 8;
 constexpr size_t GU_SMEM = (size_t)GU_STAGES * GU_STAGE_BYTES + 1024;
 static_assert((GU_NPROD + GU_NCOPY - 1) / GU_NCOPY <= GU_STAGES, "producer stride exceeds the stage ring");
 
-template <bool F8>
-__global__ void __launch_bounds__(800, 1) k_gemm_gu(int* status, const GuGemm g) {
+template <bool F8, bool QKV>
+__global__ void __launch_bounds__(800, 1) k_gemm_persist(int* status, const PersistGemm g) {
   // instruction descriptors: D fp32 (bit 4), A / B bf16 (bits 7, 10) or e4m3 (format fields 0), K-major, N >> 3 at
   // bit 17, M >> 4 at bit 24
   constexpr uint32_t IDESC = F8 ? ((1u << 4) | ((uint32_t)(GU_NT >> 3) << 17) | ((128u >> 4) << 24))
@@ -50,10 +53,11 @@ __global__ void __launch_bounds__(800, 1) k_gemm_gu(int* status, const GuGemm g)
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int skip_flag;
+  __shared__ int2 tok_tab[QKV ? 2 : 1][QKV ? GU_NT : 1];   // q | k | v: per token (position, request * 64 + suffix row)
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int KC = F8 ? g.K >> 7 : g.K >> 6;         // k-chunks of 128 bytes per operand row
-  const int n_n = (2 * g.F) >> 7;                  // weight tiles (64 channels each)
+  const int n_n = g.N >> 7;                        // weight tiles of 128 packed rows
   const int n_t = (g.M + GU_NT - 1) / GU_NT;       // token tiles
   const int n_tiles = n_n * n_t;
   const int n_my = ((int)blockIdx.x < n_tiles) ? (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
@@ -185,26 +189,76 @@ __global__ void __launch_bounds__(800, 1) k_gemm_gu(int* status, const GuGemm g)
     }
     if (lane == 0) trace_stamp(trc, 4);
   } else {
-    // ---------------- epilogue: tensor memory -> registers -> GeGLU -> global ------------------------------------
+    // ---------------- epilogue: tensor memory -> registers -> global ---------------------------------------------
     const int ew = warp - 9;                 // 0..15
     const int q = warp & 3, hf = ew >> 2;    // tensor-memory lane quarter, quarter of the token columns
-    const int hi = lane >> 4;                // 0: this lane holds a gate row, 1: an up row
+    const int hi = lane >> 4;                // 0: this lane holds a gate / first-half row, 1: an up / partner row
     const int cl = 16 * q + (lane & 15);     // channel within the tile's 64
+    const int et = ew * 32 + lane;
+    bool dead = false;
     for (int i = 0; i < n_my; ++i) {
       const int buf = i & 1;
       const int t = (int)blockIdx.x + i * (int)gridDim.x;
       const int nt = t % n_n, tok_base = (t / n_n) * GU_NT;
-      const int f = nt * 64 + cl;
-      // (per-channel weight scales of the tile: requested before the accumulator is complete)
-      const float sg = g.scale_g ? g.scale_g[f] : 1.0f, su = g.scale_u ? g.scale_u[f] : 1.0f;
+      // (per-row weight scales of the tile and, q | k | v, the token table: before the accumulator is complete)
+      float s_lo = 1.0f, s_hi = 1.0f;
+      if constexpr (QKV) {
+        // packed row of this lane's channel and of its partner in the scale vector's (un-interleaved) order
+        if (g.scale_g) s_lo = g.scale_g[nt * 128 + cl], s_hi = g.scale_g[nt * 128 + 64 + cl];
+        if (et < GU_NT) {
+          const int tok = tok_base + et;
+          int2 e = make_int2(0, 0);
+          if (tok < g.M) {
+            const int b = tok / g.S, ii = tok - b * g.S;
+            const int* cu = g.rq->cu_lens;
+            e = make_int2(cu[b + 1] - cu[b] + ii, b * 64 + ii);
+          }
+          tok_tab[buf][et] = e;
+        }
+        // (a warp can be at most one tile ahead of the slowest: it passes this barrier only after every warp has left
+        // the tile before, so the table of the tile before that is free to be overwritten)
+        asm volatile("bar.sync %0, %1;" ::"n"(BAR_PEPI), "n"(NPEPI) : "memory");
+      } else {
+        const int f = nt * 64 + cl;
+        if (g.scale_g) s_lo = g.scale_g[f];
+        if (g.scale_u) s_hi = g.scale_u[f];
+      }
+      // q | k tiles: (cos, sin) of this lane's rotary pair at its 8 tokens of a 16-column chunk, requested one chunk ahead
+      // (the first chunk's before the accumulator is complete)
+      float2 cs_next[8];
+      const bool rot_tile = QKV && nt * 128 < (g.Hq + g.Hkv) * g.dh && g.rope != nullptr;
+      const int pidx_tile = QKV ? ((((nt * 128) % g.dh) >> 7) * 64 + cl) : 0;
+      auto fetch_cs = [&](int c0) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          cs_next[j] = __ldg(g.rope + (size_t)tok_tab[buf][c0 + 8 * hi + j].x * (g.dh >> 1) + pidx_tile);
+      };
+      if constexpr (QKV) {
+        if (rot_tile) fetch_cs(hf * 64);
+      }
+      // (after a wait that did not even end within the drain bound the warp keeps walking its tiles, without waiting
+      // and without stores: the other warps meet it at the table barrier of every tile)
       int r = 0;
-      if (lane == 0) r = mbar_wait_drain(smem_u32(&bar_tfull[buf]), ((uint32_t)i >> 1) & 1u, wc);
-      r = __shfl_sync(0xffffffffu, r, 0);
-      if (r < 0) break;
-      const bool ok = r > 0 && !*reinterpret_cast<volatile int*>(&abort_flag);
+      if (!dead) {
+        if (lane == 0) r = mbar_wait_drain(smem_u32(&bar_tfull[buf]), ((uint32_t)i >> 1) & 1u, wc);
+        r = __shfl_sync(0xffffffffu, r, 0);
+        if (r < 0) dead = true;
+      }
+      const bool ok = !dead && r > 0 && !*reinterpret_cast<volatile int*>(&abort_flag);
       tc_fence_after();
       if (i == 0 && ew == 0 && lane == 0) trace_stamp(trc, 5);
-      __nv_bfloat16* const orow = g.out_tiled + (size_t)nt * g.rows_pad * 64 + (size_t)(cl & 7);
+      // q | k | v: what this tile is
+      const int Nq = g.Hq * g.dh, Nk = g.Hkv * g.dh, n0 = nt * 128;
+      const bool rot = QKV && n0 < Nq + Nk;     // q or k tile: 64 first-half channels and their rotary partners
+      const bool isq = n0 < Nq;
+      const int nn = isq ? n0 : (rot ? n0 - Nq : n0 - Nq - Nk);
+      const int head = QKV ? nn / g.dh : 0;
+      const int coff = nn - head * g.dh;        // v: first of the tile's 128 channels; q / k: 128 x (64-channel slice)
+      const int half = g.dh >> 1;
+      const float osc = (QKV && isq) ? rsqrtf((float)g.dh) : 1.0f;
+      __nv_bfloat16* const obase = !QKV ? g.out_tiled + (size_t)nt * g.rows_pad * 64 + (size_t)(cl & 7)
+                                        : (rot ? (isq ? g.qr : g.kr) : g.vr);
+      const int H = isq ? g.Hq : g.Hkv;
 #pragma unroll 1
       for (int c0 = hf * 64; c0 < hf * 64 + 64; c0 += 16) {
         float v[16];
@@ -214,22 +268,57 @@ __global__ void __launch_bounds__(800, 1) k_gemm_gu(int* status, const GuGemm g)
           tc_fence_before();
           if (lane == 0) mbar_arrive_local(smem_u32(&bar_tempty[buf]));
         }
-        // gate lanes take the tile's token columns c0 .. c0 + 7, up lanes c0 + 8 .. c0 + 15: each sends the other half
-        // to its partner lane (lane ^ 16)
-        const int tok0 = tok_base + c0 + 8 * hi;
+        if (QKV && !rot) {
+          // v tile: lane = channel 64 hi + cl of the tile (the rows are interleaved like those of the q / k tiles), 16
+          // token columns each
+          const float sc = hi ? s_hi : s_lo;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int tl = c0 + j, tok = tok_base + tl;
+            float x = v[j] * sc;
+            if constexpr (F8) x *= tok < g.M ? __ldg(g.xscale + tok) : 0.f;
+            const int2 e = tok_tab[buf][tl];
+            const int b = e.y >> 6, ii = e.y & 63;
+            if (ok && tok < g.M)
+              obase[((size_t)(b * g.Hkv + head) * g.S + ii) * g.dh + coff + 64 * hi + cl] = __float2bfloat16_rn(x);
+          }
+          continue;
+        }
+        // gate (first-half) lanes take the tile's token columns c0 .. c0 + 7, up (partner) lanes c0 + 8 .. c0 + 15: each
+        // sends the other half to its partner lane (lane ^ 16)
+        const int tl0 = c0 + 8 * hi;
+        float2 cs_cur[8];
+        if constexpr (QKV) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) cs_cur[j] = cs_next[j];
+          if (rot_tile && c0 + 16 < hf * 64 + 64) fetch_cs(c0 + 16);
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const float mine = hi ? v[8 + j] : v[j];
           const float send = hi ? v[j] : v[8 + j];
           const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
-          float gate = hi ? recv : mine, up = hi ? mine : recv;
-          const int tok = tok0 + j;
+          float lo = (hi ? recv : mine) * s_lo, up = (hi ? mine : recv) * s_hi;
+          const int tok = tok_base + tl0 + j;
           if constexpr (F8) {
             const float xs = tok < g.M ? __ldg(g.xscale + tok) : 0.f;
-            gate *= xs, up *= xs;
+            lo *= xs, up *= xs;
           }
-          const float val = gelu_fast(gate * sg, g.gelu_exact) * (up * su);
-          if (ok && tok < g.M) orow[(size_t)tok * 64 + (((cl >> 3) ^ (tok & 7)) << 3)] = __float2bfloat16_rn(val);
+          if constexpr (QKV) {
+            const int2 e = tok_tab[buf][tl0 + j];
+            const int pidx = (coff >> 7) * 64 + cl;        // rotary pair: channel pidx and pidx + dh / 2 of the head
+            if (g.rope) {
+              const float2 cs = cs_cur[j];
+              const float l2 = lo * cs.x - up * cs.y, u2 = up * cs.x + lo * cs.y;
+              lo = l2, up = u2;
+            }
+            const int b = e.y >> 6, ii = e.y & 63;
+            __nv_bfloat16* dst = obase + ((size_t)(b * H + head) * g.S + ii) * g.dh + pidx;
+            if (ok && tok < g.M) dst[0] = __float2bfloat16_rn(lo * osc), dst[half] = __float2bfloat16_rn(up * osc);
+          } else {
+            const float val = gelu_fast(lo, g.gelu_exact) * up;
+            if (ok && tok < g.M) obase[(size_t)tok * 64 + (((cl >> 3) ^ (tok & 7)) << 3)] = __float2bfloat16_rn(val);
+          }
         }
       }
     }
@@ -258,28 +347,34 @@ __global__ void __launch_bounds__(800, 1) k_gemm_gu(int* status, const GuGemm g)
 
 }  // namespace
 
-bool gu_gemm_supported(int M, int F, int K, int rows_pad, bool fp8) {
+bool persist_gemm_supported(int M, int N, int K, int rows_pad, bool fp8) {
   const int kb = fp8 ? 128 : 64;
-  return F % 64 == 0 && K % kb == 0 && K >= kb && rows_pad % GU_NT == 0 && (M + GU_NT - 1) / GU_NT * GU_NT <= rows_pad;
+  return N % 128 == 0 && K % kb == 0 && K >= kb && rows_pad % GU_NT == 0 && (M + GU_NT - 1) / GU_NT * GU_NT <= rows_pad;
 }
 
-cudaError_t gu_gemm_setup() {
-  cudaError_t e = cudaFuncSetAttribute(k_gemm_gu<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GU_SMEM);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_gemm_gu<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GU_SMEM);
+cudaError_t persist_gemm_setup() {
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(k_gemm_persist<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GU_SMEM))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_persist<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GU_SMEM))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_persist<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GU_SMEM))) return e;
+  return cudaFuncSetAttribute(k_gemm_persist<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GU_SMEM);
 }
 
-int gu_gemm_ctas(const GuGemm& g, int n_sm) {
-  const int n_tiles = ((2 * g.F) >> 7) * ((g.M + GU_NT - 1) / GU_NT);
+int persist_gemm_ctas(const PersistGemm& g, int n_sm) {
+  const int n_tiles = (g.N >> 7) * ((g.M + GU_NT - 1) / GU_NT);
   return n_tiles < n_sm ? n_tiles : n_sm;
 }
 
-cudaError_t launch_gu_gemm(int* status, const GuGemm& g, int n_sm, cudaStream_t st) {
-  if (!gu_gemm_supported(g.M, g.F, g.K, g.rows_pad, g.fp8 != 0)) return cudaErrorInvalidValue;
+cudaError_t launch_persist_gemm(int* status, const PersistGemm& g, int n_sm, cudaStream_t st) {
+  if (!persist_gemm_supported(g.M, g.N, g.K, g.rows_pad, g.fp8 != 0)) return cudaErrorInvalidValue;
   if (g.fp8 && !g.xscale) return cudaErrorInvalidValue;
-  const dim3 grid(gu_gemm_ctas(g, n_sm));
-  if (g.fp8) return launch_pdl(k_gemm_gu<true>, grid, dim3(800), GU_SMEM, st, status, g);
-  return launch_pdl(k_gemm_gu<false>, grid, dim3(800), GU_SMEM, st, status, g);
+  if (g.qkv && (!g.rq || g.S > 64 || (g.dh != 128 && g.dh != 256) || g.N != (g.Hq + 2 * g.Hkv) * g.dh)) return cudaErrorInvalidValue;
+  const dim3 grid(persist_gemm_ctas(g, n_sm));
+  if (g.fp8)
+    return g.qkv ? launch_pdl(k_gemm_persist<true, true>, grid, dim3(800), GU_SMEM, st, status, g)
+                 : launch_pdl(k_gemm_persist<true, false>, grid, dim3(800), GU_SMEM, st, status, g);
+  return g.qkv ? launch_pdl(k_gemm_persist<false, true>, grid, dim3(800), GU_SMEM, st, status, g)
+               : launch_pdl(k_gemm_persist<false, false>, grid, dim3(800), GU_SMEM, st, status, g);
 }
 
 }  // namespace phyai

@@ -67,12 +67,13 @@ void launch_copy_cols(const void* src, int src_kind, const float* scale, float* 
 // With il_group > 0 the channels of two matrices are interleaved in groups of il_group rows
 // (il_second selects the second matrix): packed row = (n / g) * 2g + n % g + (second ? g : 0).
 // With perm_dh > 0 the channels follow the rotary-pair row order of the fused QKV matrix
-// (qkv_channel_to_packed).
+// (qkv_channel_to_packed).  With pair16 the rows of every 128-row tile are then interleaved in groups of 16: packed
+// row r of the tile goes to row 32 ((r % 64) / 16) + 16 (r / 64) + r % 16 (rows r and r + 64 end up 16 apart).
 void launch_pack_tiled(const void* src, int src_kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st,
-                       int il_group = 0, int il_second = 0, int perm_dh = 0);
+                       int il_group = 0, int il_second = 0, int perm_dh = 0, int pair16 = 0);
 // e4m3 codes [in=K][out=N] -> byte blocks [N/128][K/64][128][64] in the packed row order of launch_pack_tiled
 void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group = 0,
-                       int il_second = 0, int perm_dh = 0, int wide = 0);
+                       int il_second = 0, int perm_dh = 0, int wide = 0, int pair16 = 0);
 // (wide: blocks [N/128][K/128][128][128] instead, the 16-byte chunks of a row XOR-swizzled by row & 7: the e4m3
 // operand image of the FP8 tensor path)
 // row-major bf16 [M][K] (K a multiple of 8, 16-byte aligned rows) -> the tiled bf16 layout of the GEMM inputs
@@ -227,25 +228,34 @@ struct TcGemm {
 cudaError_t launch_tc_gemm(int* status, const TcGemm& g, int nt, cudaStream_t st);
 cudaError_t tc_gemm_setup();  // one-time attribute setup (dynamic shared memory opt-in)
 
-// Persistent gate / up projection with the GeGLU epilogue (gemm_gu.cu): 128-row weight tiles that hold the gate and
-// up rows of the same 64 channels (rows 32 q + i = gate, 32 q + 16 + i = up of channel 16 q + i of the tile), 256-token
-// tiles, two accumulators in tensor memory so that the epilogue of a tile overlaps the main loop of the next.
-struct GuGemm {
-  const __nv_bfloat16* W;       // interleaved image: (2 F / 128) tiles x KC blocks of 128 rows x 128 bytes (bf16 or e4m3)
+// Persistent tile GEMM (gemm_persist.cu): 128-row weight tiles x 256-token tiles, two accumulators in tensor memory so
+// that the epilogue of a tile overlaps the main loop of the next.  The rows of every weight tile are interleaved in
+// groups of 16: rows 32 q + i (i < 16) and 32 q + 16 + i are combined by the epilogue.
+//   gate / up (qkv = 0): the tile holds 64 channels, gate rows at 32 q + i and up rows at 32 q + 16 + i of channel
+//     16 q + i; N = 2 x mlp_dim; out_tiled gets gelu(gate) * up.
+//   q | k | v (qkv = 1): the packing of qkv_channel_to_packed (64 first-half channels of a head, then their rotary
+//     partners; v: 128 channels) with packed row r of a tile moved to row 32 ((r % 64) / 16) + 16 (r / 64) + r % 16;
+//     q rotated and scaled by 1 / sqrt(dh), k rotated, v as is, all bf16, laid out as for TC_QKV_ROT.
+struct PersistGemm {
+  const __nv_bfloat16* W;       // (N / 128) tiles x KC blocks of 128 rows x 128 bytes (bf16 or e4m3)
   const __nv_bfloat16* X;       // tiled activations [KC][rows_pad][128 bytes]
-  __nv_bfloat16* out_tiled;     // [F / 64][rows_pad][64] bf16, 16-byte chunks swizzled by row & 7
-  const float* scale_g;         // per-channel weight scales or null
+  __nv_bfloat16* out_tiled;     // gate / up: [N / 128][rows_pad][64] bf16, 16-byte chunks swizzled by row & 7
+  const float* scale_g;         // per-channel weight scales or null (q | k | v: per packed row, un-interleaved order)
   const float* scale_u;
   const float* xscale;          // fp8: per-token activation scales
-  int M, F, K, rows_pad;
-  int gelu_exact, fp8;
+  int M, N, K, rows_pad;
+  int gelu_exact, fp8, qkv;
   unsigned wait_limit;
   unsigned long long* trace;    // or null: CTA b stamps slot b (16 words)
+  const Request* rq;            // q | k | v
+  const float2* rope;
+  __nv_bfloat16 *qr, *kr, *vr;
+  int S, Hq, Hkv, dh;
 };
-bool gu_gemm_supported(int M, int F, int K, int rows_pad, bool fp8);
-int gu_gemm_ctas(const GuGemm& g, int n_sm);
-cudaError_t gu_gemm_setup();
-cudaError_t launch_gu_gemm(int* status, const GuGemm& g, int n_sm, cudaStream_t st);
+bool persist_gemm_supported(int M, int N, int K, int rows_pad, bool fp8);
+int persist_gemm_ctas(const PersistGemm& g, int n_sm);
+cudaError_t persist_gemm_setup();
+cudaError_t launch_persist_gemm(int* status, const PersistGemm& g, int n_sm, cudaStream_t st);
 // ---- cluster split-K GEMM for a single 64-token tile (gemm_b1.cu) --------------------------------------------
 enum : int { B1_QKV = 0, B1_GEGLU = 1, B1_RESID = 2 };
 struct B1Gemm {

@@ -96,8 +96,12 @@ void launch_copy_cols(const void* src, int kind, const float* scale, float* dst,
 
 // Weight [K][N] -> packed out-channel-major swizzled blocks.  One thread per 16-byte chunk
 // (8 consecutive k of one out channel): reads are strided by N (one-off cost at create).
+__device__ __forceinline__ int pair16_row(int np) {
+  const int r = np & 127;
+  return (np & ~127) | (32 * ((r & 63) >> 4) + 16 * (r >> 6) + (r & 15));
+}
 __global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, int il_group,
-                             int il_second, int perm_dh) {
+                             int il_second, int perm_dh, int pair16) {
   const int KC = K >> 6;
   const size_t chunks = (size_t)N * (K >> 3);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
@@ -105,8 +109,9 @@ __global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int 
     const int k8 = (int)(i / N);        // chunk index along K
     const int k0 = k8 << 3;
     // optional interleave: groups of il_group channels of two matrices alternate in the packed rows
-    const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
-                            : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
+    int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
+                      : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
+    if (pair16) np = pair16_row(np);
     const int kc = k0 >> 6, c = (k0 & 63) >> 3;
     const size_t base = (((size_t)(np >> 7) * KC + kc) * 128 + (np & 127)) * 64 + (size_t)((c ^ (np & 7)) << 3);
     __align__(16) __nv_bfloat16 v[8];
@@ -116,22 +121,23 @@ __global__ void k_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int 
   }
 }
 void launch_pack_tiled(const void* src, int kind, __nv_bfloat16* dst, int K, int N, int n_off, cudaStream_t st,
-                       int il_group, int il_second, int perm_dh) {
+                       int il_group, int il_second, int perm_dh, int pair16) {
   const size_t chunks = (size_t)N * (K >> 3);
   const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
-  k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off, il_group, il_second, perm_dh);
+  k_pack_tiled<<<blocks, 256, 0, st>>>(src, kind, dst, K, N, n_off, il_group, il_second, perm_dh, pair16);
 }
 
 // e4m3 codes [K][N] -> byte blocks of 128 out channels x 64 k (row order as in k_pack_tiled, no swizzle: the kernel
 // that decodes them writes the swizzled bf16 image itself).  One thread per 8 consecutive k of one out channel.
 __global__ void k_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, int il_group, int il_second,
-                             int perm_dh, int wide) {
+                             int perm_dh, int wide, int pair16) {
   const int KC = wide ? K >> 7 : K >> 6;
   const size_t chunks = (size_t)N * (K >> 3);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
     const int n = (int)(i % N), k0 = (int)(i / N) << 3;
-    const int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
-                            : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
+    int np = il_group ? (n / il_group) * (2 * il_group) + (n % il_group) + (il_second ? il_group : 0)
+                      : n_off + (perm_dh ? qkv_channel_to_packed(n, perm_dh) : n);
+    if (pair16) np = pair16_row(np);
     __align__(8) uint8_t v[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) v[j] = src[(size_t)(k0 + j) * N + n];
@@ -148,10 +154,10 @@ __global__ void k_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int
   }
 }
 void launch_pack_bytes(const uint8_t* src, uint8_t* dst, int K, int N, int n_off, cudaStream_t st, int il_group,
-                       int il_second, int perm_dh, int wide) {
+                       int il_second, int perm_dh, int wide, int pair16) {
   const size_t chunks = (size_t)N * (K >> 3);
   const int blocks = (int)((chunks + 255) / 256 < 16384 ? (chunks + 255) / 256 : 16384);
-  k_pack_bytes<<<blocks, 256, 0, st>>>(src, dst, K, N, n_off, il_group, il_second, perm_dh, wide);
+  k_pack_bytes<<<blocks, 256, 0, st>>>(src, dst, K, N, n_off, il_group, il_second, perm_dh, wide, pair16);
 }
 
 // row-major bf16 [M][K] -> tiled bf16 [K/64][rows_pad][64] (16-byte chunks XOR-swizzled by row & 7)

@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("cluster_gemm", [1, 0])
-@pytest.mark.parametrize("batch", [1, 40])
+@pytest.mark.parametrize("batch", [1, 40, 80])   # 80 requests = 1120 tokens: the persistent 256-token-tile kernels
 def test_expired_wait_is_reported_and_the_handle_recovers(cluster_gemm, batch):
     cfg = small_bf16_config("pi0", max_batch=batch, max_prefix_len=150)
     W = synth.make_weights(cfg, 31, std=0.05)
