@@ -224,6 +224,9 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
  * state token does not cost a token tile of its own.
  * key "b1_attn_hpc": query heads per CTA (1 or 2; 0 = choose) of the cluster attention kernel.  key "use_b1_step":
  * 1 (default) runs the step boundary of those calls (velocity head, Euler update, next embedding) as one cluster kernel.
+ * key "use_persistent_gu" / "use_persistent_qkv": 1 (default) runs the gate/up and the q|k|v projection of calls
+ * with more than 1024 suffix tokens on the persistent tile kernel (one CTA per SM, two accumulators, a tile's
+ * epilogue under the next tile's main loop); 0 keeps them on the one-tile-per-CTA kernel.
  * key "trace": see phyai_read_trace.
  * key "wait_limit": iteration bound of the device-side waits on other agents' progress (testing).
  * Unknown key -> INVALID_ARG. */
@@ -242,6 +245,10 @@ phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t valu
  * Option "trace_all_from" = i > 0 (with "trace" = 1): instead, EVERY CTA of the cluster-GEMM and cluster-attention
  * launches with index i .. i + 4 of a call stamps, into consecutive slots (slot = CTAs of the earlier traced launches +
  * the CTA's linear index in its grid); 0 returns to one CTA per launch.
+ * For calls with more than 64 suffix tokens "trace_all_from" = i traces launch i alone, if it is a tile GEMM: slot =
+ * the CTA's linear index, stamps [0] start, [1] set-up done, [2] dependency resolved, [3] first operands landed,
+ * [4] last MMA issued, [5] (first) accumulator complete, [6] epilogue's stores issued, [7] SM, [8] tensor memory
+ * released, [9] tiles walked (persistent kernel).
  */
 phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_slots,
                                 uint32_t *n_stamps);
