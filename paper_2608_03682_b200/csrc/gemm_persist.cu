@@ -53,7 +53,9 @@ __global__ void __launch_bounds__(800, 1) k_gemm_persist(int* status, const Pers
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ int skip_flag;
-  __shared__ int2 tok_tab[QKV ? 2 : 1][QKV ? GU_NT : 1];   // q | k | v: per token (position, request * 64 + suffix row)
+  // q | k | v: per token (position x dh / 2, element offset of its row in q [b][Hq][S][dh] without the head term, the
+  // same for k / v [b][Hkv][S][dh], 1 if the token exists)
+  __shared__ int4 tok_tab[QKV ? 2 : 1][QKV ? GU_NT : 1];
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int KC = F8 ? g.K >> 7 : g.K >> 6;         // k-chunks of 128 bytes per operand row
@@ -207,11 +209,11 @@ __global__ void __launch_bounds__(800, 1) k_gemm_persist(int* status, const Pers
         if (g.scale_g) s_lo = g.scale_g[nt * 128 + cl], s_hi = g.scale_g[nt * 128 + 64 + cl];
         if (et < GU_NT) {
           const int tok = tok_base + et;
-          int2 e = make_int2(0, 0);
+          int4 e = make_int4(0, 0, 0, 0);
           if (tok < g.M) {
             const int b = tok / g.S, ii = tok - b * g.S;
             const int* cu = g.rq->cu_lens;
-            e = make_int2(cu[b + 1] - cu[b] + ii, b * 64 + ii);
+            e = make_int4((cu[b + 1] - cu[b] + ii) * (g.dh >> 1), (b * g.Hq * g.S + ii) * g.dh, (b * g.Hkv * g.S + ii) * g.dh, 1);
           }
           tok_tab[buf][et] = e;
         }
@@ -227,11 +229,11 @@ __global__ void __launch_bounds__(800, 1) k_gemm_persist(int* status, const Pers
       // (the first chunk's before the accumulator is complete)
       float2 cs_next[8];
       const bool rot_tile = QKV && nt * 128 < (g.Hq + g.Hkv) * g.dh && g.rope != nullptr;
-      const int pidx_tile = QKV ? ((((nt * 128) % g.dh) >> 7) * 64 + cl) : 0;
+      const int pidx_tile = QKV ? ((((nt * 128) % g.dh) >> 7) * 64 + cl) : 0;   // rotary pair: channels pidx, pidx + dh / 2
+      const float2* const rope_p = g.rope + pidx_tile;
       auto fetch_cs = [&](int c0) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          cs_next[j] = __ldg(g.rope + (size_t)tok_tab[buf][c0 + 8 * hi + j].x * (g.dh >> 1) + pidx_tile);
+        for (int j = 0; j < 8; ++j) cs_next[j] = __ldg(rope_p + tok_tab[buf][c0 + 8 * hi + j].x);
       };
       if constexpr (QKV) {
         if (rot_tile) fetch_cs(hf * 64);
@@ -255,10 +257,16 @@ __global__ void __launch_bounds__(800, 1) k_gemm_persist(int* status, const Pers
       const int head = QKV ? nn / g.dh : 0;
       const int coff = nn - head * g.dh;        // v: first of the tile's 128 channels; q / k: 128 x (64-channel slice)
       const int half = g.dh >> 1;
-      const float osc = (QKV && isq) ? rsqrtf((float)g.dh) : 1.0f;
-      __nv_bfloat16* const obase = !QKV ? g.out_tiled + (size_t)nt * g.rows_pad * 64 + (size_t)(cl & 7)
-                                        : (rot ? (isq ? g.qr : g.kr) : g.vr);
-      const int H = isq ? g.Hq : g.Hkv;
+      if (QKV && isq) {   // q leaves scaled by 1 / sqrt(dh): folded into the row scales (the rotation is linear)
+        const float osc = rsqrtf((float)g.dh);
+        s_lo *= osc, s_hi *= osc;
+      }
+      // gate / up: the tile's k-chunk of the output image; q / k: this lane's rotary pair in the tile's head; v: this
+      // lane's channel in the tile's head (the token's row offset comes from the table)
+      __nv_bfloat16* const obase =
+          !QKV ? g.out_tiled + (size_t)nt * g.rows_pad * 64 + (size_t)(cl & 7)
+               : (rot ? (isq ? g.qr : g.kr) + (size_t)head * g.S * g.dh + pidx_tile
+                      : g.vr + (size_t)head * g.S * g.dh + coff + 64 * hi + cl);
 #pragma unroll 1
       for (int c0 = hf * 64; c0 < hf * 64 + 64; c0 += 16) {
         float v[16];
@@ -277,10 +285,8 @@ __global__ void __launch_bounds__(800, 1) k_gemm_persist(int* status, const Pers
             const int tl = c0 + j, tok = tok_base + tl;
             float x = v[j] * sc;
             if constexpr (F8) x *= tok < g.M ? __ldg(g.xscale + tok) : 0.f;
-            const int2 e = tok_tab[buf][tl];
-            const int b = e.y >> 6, ii = e.y & 63;
-            if (ok && tok < g.M)
-              obase[((size_t)(b * g.Hkv + head) * g.S + ii) * g.dh + coff + 64 * hi + cl] = __float2bfloat16_rn(x);
+            const int4 e = tok_tab[buf][tl];
+            if (ok && e.w) obase[e.z] = __float2bfloat16_rn(x);
           }
           continue;
         }
@@ -305,16 +311,14 @@ __global__ void __launch_bounds__(800, 1) k_gemm_persist(int* status, const Pers
             lo *= xs, up *= xs;
           }
           if constexpr (QKV) {
-            const int2 e = tok_tab[buf][tl0 + j];
-            const int pidx = (coff >> 7) * 64 + cl;        // rotary pair: channel pidx and pidx + dh / 2 of the head
+            const int4 e = tok_tab[buf][tl0 + j];
             if (g.rope) {
               const float2 cs = cs_cur[j];
               const float l2 = lo * cs.x - up * cs.y, u2 = up * cs.x + lo * cs.y;
               lo = l2, up = u2;
             }
-            const int b = e.y >> 6, ii = e.y & 63;
-            __nv_bfloat16* dst = obase + ((size_t)(b * H + head) * g.S + ii) * g.dh + pidx;
-            if (ok && tok < g.M) dst[0] = __float2bfloat16_rn(lo * osc), dst[half] = __float2bfloat16_rn(up * osc);
+            __nv_bfloat16* dst = obase + (isq ? e.y : e.z);
+            if (ok && e.w) dst[0] = __float2bfloat16_rn(lo), dst[half] = __float2bfloat16_rn(up);
           } else {
             const float val = gelu_fast(lo, g.gelu_exact) * up;
             if (ok && tok < g.M) obase[(size_t)tok * 64 + (((cl >> 3) ^ (tok & 7)) << 3)] = __float2bfloat16_rn(val);
