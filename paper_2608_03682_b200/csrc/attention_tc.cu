@@ -31,6 +31,7 @@ constexpr int KTC = 64;          // keys per tile
 constexpr int NKV = 3;           // K and V tile buffers each
 constexpr int BAR_LOAD = 1;      // named barrier of the 2 K loader warps
 constexpr int BAR_SOFT = 2;      // named barrier of the 4 softmax warps (3 = the V loader warps)
+constexpr int BAR_QSTAGE = 4;    // softmax warps (arrive) -> V loader warps (sync): the Q staging area is free
 constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units
 
 template <int DH>
@@ -58,9 +59,12 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t Ks = base, Vs = Ks + NKV * KV_BYTES;
 
-  pdl_enter();
+  unsigned long long* const trc = a.trace ? a.trace + (size_t)(blockIdx.y * gridDim.x + blockIdx.x) * 16 : nullptr;
+  if (tid == 0) trace_stamp(trc, 0);
+  // Programmatic dependent launch: barriers and tensor memory are set up while the kernel before this one (the q|k|v
+  // projection) still runs; the first access to anything it wrote comes after pdl_wait().
+  pdl_launch_dependents();
   if (tid == 0) {
-    skip_flag = status_set(a.status) ? 1 : 0;
     abort_flag = 0;
     for (int i = 0; i < NKV; ++i) {
       mbar_init(smem_u32(&k_full[i]), 1);
@@ -75,16 +79,24 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  __syncthreads();
-  if (skip_flag) return;
   if (warp == 4) {
     tmem_alloc(smem_u32(&tmem_slot), COLS);
     tc_fence_before();
   }
   const WaitCtx wc{a.status, &abort_flag, a.wait_limit};
-  __syncthreads();                             // the TMEM base address is published
+  __syncthreads();                             // barriers initialised, the TMEM base address published
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  pdl_wait();
+  if (tid == 0) {
+    trace_stamp(trc, 1);
+    skip_flag = status_set(a.status) ? 1 : 0;
+  }
+  __syncthreads();
+  if (skip_flag) {
+    if (warp == 4) tmem_dealloc(tmem_base, COLS);
+    return;
+  }
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * KTC, tmem_q = tmem_base + 2 * KTC + DH;
 
   const Request r = *a.rq;
@@ -139,6 +151,8 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       fence_async_smem();
       if (is_v) group_sync<BAR_LOAD + 2, 64>(); else group_sync<BAR_LOAD, 64>();
       if (lt2 == 0) mbar_arrive_local(smem_u32(&full[0]));
+      // (V buffers 1 and 2 are the staging area of the Q rows until the softmax warps have moved them to tensor memory)
+      if (is_v) asm volatile("bar.sync %0, %1;" ::"n"(BAR_QSTAGE), "n"(192) : "memory");
       if (T > 1) issue(1);
       if (T > 2) issue(2);
     }
@@ -174,8 +188,10 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     {
       mbar_wait(smem_u32(&q_full), 0u, wc);    // Q is in tensor memory
       tc_fence_after();
+      if (lane == 0) trace_stamp(trc, 2);
     }
     issue_s(0);
+    if (lane == 0) trace_stamp(trc, 3);
     if (T > 1) issue_s(1);
     for (int t = 0; t < T; ++t) {
       const int buf = t & 1, vbuf = t % NKV;
@@ -195,7 +211,9 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       if (elect_one()) umma_commit(smem_u32(&pv_done[buf]));
       __syncwarp();
       if (t + 2 < T) issue_s(t + 2);
+      if (t == 0 && lane == 0) trace_stamp(trc, 4);
     }
+    if (lane == 0) trace_stamp(trc, 5);
     if (*reinterpret_cast<volatile int*>(&abort_flag)) {
       // a wait was given up: the softmax warps no longer wait for the tensor core, so make sure here that every MMA
       // issued above has completed before tensor memory is released below
@@ -212,18 +230,46 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     float m = -INFINITY, l = 0.f;             // running maximum (log2 units) and sum
     {
-      // Q (already rotated, scaled bf16) goes from global memory straight into tensor memory, one row per thread,
-      // where it is the A operand of every S = Q K^T (two bf16 per 32-bit column, in memory order)
-      const uint4* qsrc = reinterpret_cast<const uint4*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S + (i < S ? i : 0)) * DH);
+      // Q (already rotated, scaled bf16) -> tensor memory, where it is the A operand of every S = Q K^T (two bf16 per
+      // 32-bit column, in memory order), one row per thread.  A row is 2 DH bytes of global memory: read by its own
+      // thread, one 16-byte load would touch 32 different lines per warp instruction.  Each warp instead copies its 32
+      // rows (contiguous in global memory) with coalesced 16-byte cp.async into a staging block (V buffers 1 and 2,
+      // not needed before the second key tile's P V; 16-byte chunks XOR-swizzled by the row so that both the row-wise
+      // writes and the one-row-per-thread reads are free of bank conflicts), and every thread then reads its row.
+      constexpr int QROW = DH * 2;                                  // bytes per row
+      constexpr int QCH = QROW / 16;                                // 16-byte chunks per row (32)
+      static_assert(4 * 32 * QROW <= 2 * KV_BYTES, "Q staging exceeds two V buffers");
+      const uint32_t qstage = Vs + KV_BYTES + (uint32_t)q * (32 * QROW);
+      const int i0 = (q * 32) & 63;                                 // first token of this warp's 32 rows
+      const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(a.qr + ((size_t)(b * d.Hq + head0 + hl) * S) * DH);
+#pragma unroll 8
+      for (int rr = 0; rr < 32; ++rr) {
+        const bool ok = i0 + rr < S;                                // rows past the suffix are zero-filled
+        for (int c = lane; c < QCH; c += 32)
+          cp_async16(qstage + (uint32_t)rr * QROW + (uint32_t)((c ^ (rr & (QCH - 1))) << 4),
+                     qsrc + (size_t)(ok ? i0 + rr : 0) * QROW + (size_t)c * 16, ok ? 16u : 0u);
+      }
+      cp_async_commit();
+      cp_async_wait<0>();
+      __syncwarp();
+      const uint32_t qrow = qstage + (uint32_t)lane * QROW;
       const uint32_t qdst = tmem_q + lane_addr;
 #pragma unroll 1
-      for (int c = 0; c < DH / 2; c += 64) {                      // 64 columns = 128 bf16 = 16 x 16 bytes per round,
-        uint4 v[16];                                              // all loads of a round in flight together
+      for (int c = 0; c < DH / 2; c += 64) {                      // 64 columns = 128 bf16 = 16 x 16 bytes per round
+        uint4 v[16];
 #pragma unroll
-        for (int u = 0; u < 16; ++u) v[u] = i < S ? __ldg(qsrc + (c >> 2) + u) : make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < 16; ++u) {
+          const int ch = (c >> 2) + u;
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(v[u].x), "=r"(v[u].y), "=r"(v[u].z), "=r"(v[u].w)
+                       : "r"(qrow + (uint32_t)((ch ^ (lane & (QCH - 1))) << 4))
+                       : "memory");
+        }
 #pragma unroll
         for (int u = 0; u < 4; ++u) tmem_st16u(qdst + (uint32_t)(c + 16 * u), reinterpret_cast<const uint32_t*>(v + 4 * u));
       }
+      // the staging area goes back to the V loaders
+      asm volatile("bar.arrive %0, %1;" ::"n"(BAR_QSTAGE), "n"(192) : "memory");
       tmem_st_wait();
       tc_fence_before();
       group_sync<BAR_SOFT, 128>();
@@ -294,7 +340,42 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     const bool okf =
         __all_sync(0xffffffffu, mbar_wait(smem_u32(&pv_done[(T - 1) & 1]), (uint32_t)((T - 1) >> 1) & 1u, wc));
     tc_fence_after();
-    {
+    if (st == 0) trace_stamp(trc, 6);
+    if (a.rows_pad > 0) {
+      // O / l -> bf16 in the tiled layout of the O projection's input.  A thread holds one row; its 128 bytes of a
+      // 64-channel k-chunk go to a staging block of the warp (the K buffers are free: every MMA has completed) at the
+      // position they have in global memory, where the warp's 32 rows of a k-chunk are one contiguous range, and the
+      // warp then copies that range with coalesced 16-byte stores (one row per thread, stored directly, would touch 32
+      // lines per instruction).
+      const float inv = 1.0f / l;
+      const int i0 = (q * 32) & 63;
+      const int orow = b * S + i0 + lane, head = head0 + hl;
+      const int nrow = okf ? max(0, min(32, S - i0)) : 0;        // rows of this warp that exist
+      const uint32_t ostage = Ks + (uint32_t)q * 4096u;
+      const uint32_t orow_s = ostage + (uint32_t)lane * 128u;
+#pragma unroll 1
+      for (int c = 0; c < DH; c += 64) {
+        float o[64];
+        tmem_ld64(tmem_o + lane_addr + (uint32_t)c, o);         // four loads in flight, one wait
+#pragma unroll
+        for (int e = 0; e < 64; e += 8) {
+          const uint32_t w0 = pack_bf16(o[e] * inv, o[e + 1] * inv), w1 = pack_bf16(o[e + 2] * inv, o[e + 3] * inv);
+          const uint32_t w2 = pack_bf16(o[e + 4] * inv, o[e + 5] * inv), w3 = pack_bf16(o[e + 6] * inv, o[e + 7] * inv);
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(orow_s + (uint32_t)((((e >> 3) ^ (orow & 7))) << 4)), "r"(w0),
+                       "r"(w1), "r"(w2), "r"(w3)
+                       : "memory");
+        }
+        __syncwarp();
+        // k-chunk (head * DH + c) / 64 of the output, rows b * S + i0 ..: nrow * 128 contiguous bytes
+        uint4* dst = reinterpret_cast<uint4*>(a.out + ((size_t)((head * DH + c) >> 6) * a.rows_pad + (size_t)(b * S + i0)) * 64);
+        for (int idx = lane; idx < nrow * 8; idx += 32) {
+          uint4 v;
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(ostage + (uint32_t)idx * 16u) : "memory");
+          dst[idx] = v;
+        }
+        __syncwarp();
+      }
+    } else {
       const bool wr = okf && i < S;             // the TMEM loads stay warp-uniform; only the stores are predicated
       const float inv = 1.0f / l;
       const int orow = b * S + (i < S ? i : 0), head = head0 + hl;
@@ -311,6 +392,13 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       }
     }
     tc_fence_before();
+    if (st == 0 && trc) {
+      unsigned long long tt_;
+      unsigned sm;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt_)::"memory");
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+      trc[8] = tt_, trc[7] = sm, trc[9] = (unsigned long long)T;
+    }
   }
 
   __syncthreads();
@@ -333,7 +421,7 @@ bool attention_tc_supported(const Dims& d) {
 
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, const int* order, unsigned wait_limit, cudaStream_t st) {
+                                int batch, const int* order, unsigned wait_limit, cudaStream_t st, unsigned long long* trace) {
   static PerDeviceOnce once;
   if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(k_attn_tc<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -343,7 +431,7 @@ cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloa
   }
   AttnArgs a{};
   a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
-  a.num_splits = 1, a.d = d, a.wait_limit = wait_limit, a.order = order;
+  a.num_splits = 1, a.d = d, a.wait_limit = wait_limit, a.order = order, a.trace = trace;
   dim3 grid(d.Hq / 2, batch);
   return launch_pdl(k_attn_tc<256>, grid, dim3(288), attn_tc_smem<256>(), st, a);
 }

@@ -590,7 +590,8 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
       }
       if (attn_tc) {
         cudaError_t e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn_t, h->Mpad, d,
-                                            batch, h->order, h->wait_limit, st);
+                                            batch, h->order, h->wait_limit, st,
+                                            (h->trace && h->trace_all_from > 0 && cnt == h->trace_all_from && batch * (d.Hq / 2) <= TRACE_SLOTS) ? h->trace : nullptr);
         if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
         ++cnt;
       } else if (attn_cluster) {

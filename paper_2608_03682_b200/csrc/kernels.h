@@ -183,7 +183,7 @@ cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloa
 int attention_b1_ctas(const Dims& d, int batch, int hpc);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, const int* order, unsigned wait_limit, cudaStream_t st);
+                                int batch, const int* order, unsigned wait_limit, cudaStream_t st, unsigned long long* trace = nullptr);
 
 // ---- tcgen05 GEMM ------------------------------------------------------------------------------
 enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3, TC_QKV_ROT = 4, TC_GEGLU_IL = 5 };
