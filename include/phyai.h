@@ -249,6 +249,9 @@ phyai_status_t phyai_set_option(phyai_expert_t *h, const char *key, int64_t valu
  * the CTA's linear index, stamps [0] start, [1] set-up done, [2] dependency resolved, [3] first operands landed,
  * [4] last MMA issued, [5] (first) accumulator complete, [6] epilogue's stores issued, [7] SM, [8] tensor memory
  * released, [9] tiles walked (persistent kernel).
+ * The tcgen05 attention kernel of such calls is traced the same way: [0] start, [1] dependency resolved, [2] Q in
+ * tensor memory, [3] S(0) issued, [4] P V(0) issued, [5] all MMAs issued, [6] last P V complete, [7] SM, [8] output
+ * stored, [9] key tiles, [10] = 1.
  */
 phyai_status_t phyai_read_trace(phyai_expert_t *h, uint64_t *out, size_t capacity, uint32_t *n_slots,
                                 uint32_t *n_stamps);

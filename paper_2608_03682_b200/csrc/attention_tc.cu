@@ -397,7 +397,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
       unsigned sm;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tt_)::"memory");
       asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
-      trc[8] = tt_, trc[7] = sm, trc[9] = (unsigned long long)T;
+      trc[8] = tt_, trc[7] = sm, trc[9] = (unsigned long long)T, trc[10] = 1;   // ([10]: marks an attention slot)
     }
   }
 
