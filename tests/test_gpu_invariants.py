@@ -166,3 +166,40 @@ def test_host_buffer_entry_points_match_the_device_ones():
         torch.cuda.synchronize()
         assert ex.poll_status() == 0
         assert rel_err(single.double().numpy(), dev[2].double().numpy()) <= BAR["bf16"]
+
+
+def test_timer_stamps_of_the_tile_kernels_are_ordered_and_do_not_change_the_result():
+    """Tracing aid at more than 1024 suffix tokens: with "trace_all_from" = i every CTA of launch i (a tile GEMM or the
+    tcgen05 attention kernel) stamps one slot; the stamps of a slot are in order, the number of slots is the launch's
+    grid, and a traced call returns the same action chunk as an untraced one (to the rounding of the atomic split-K
+    adds)."""
+    cfg = small_bf16_config("pi0", max_batch=90, max_prefix_len=96, head_dim=256, n_q_heads=4)
+    W = synth.make_weights(cfg, 41, std=0.05)
+    lens = [96 - (5 * b) % 60 for b in range(90)]
+    kvs = [synth.make_prefix_kv(cfg, 41, p, b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    states = torch.stack([synth.make_state(cfg, 41, b) for b in range(90)])
+    noise = torch.stack([synth.make_noise(cfg, 41, b) for b in range(90)])
+    args = (packed.cuda(), torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), 2)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        plain = ex.denoise_batched(*args).double().cpu().numpy()
+        ex.set_option("trace", 1)
+        traced_launches = 0
+        for launch in range(1, 12):
+            ex.set_option("trace_all_from", launch)
+            out = ex.denoise_batched(*args).double().cpu().numpy()
+            assert ex.poll_status() == 0
+            assert rel_err(out, plain) <= BAR["bf16"]
+            tr = ex.read_trace().astype(np.int64)
+            r = tr[tr[:, 0] != 0]
+            if len(r) == 0:
+                continue
+            traced_launches += 1
+            assert len(r) <= 148 * 4
+            attention = r[:, 10].max() == 1
+            order = (0, 1, 2, 3, 4, 5, 6, 8) if attention else (0, 1, 2, 3, 4)
+            for a, b in zip(order[:-1], order[1:]):
+                assert (r[:, b] >= r[:, a]).all(), (launch, a, b)
+            assert (r[:, 8] >= r[:, 6]).all() and (r[:, 6] >= r[:, 5]).all()
+            assert (r[:, 8] - r[:, 0]).max() < 1e9           # ns: a CTA lives microseconds, not seconds
+        assert traced_launches >= 4                           # q|k|v, attention, O, gate/up, down of the first layer
