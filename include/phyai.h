@@ -227,6 +227,8 @@ phyai_status_t phyai_poll_status(phyai_expert_t *h);
  * key "use_persistent_gu" / "use_persistent_qkv": 1 (default) runs the gate/up and the q|k|v projection of calls
  * with more than 1024 suffix tokens on the persistent tile kernel (one CTA per SM, two accumulators, a tile's
  * epilogue under the next tile's main loop); 0 keeps them on the one-tile-per-CTA kernel.
+ * key "use_attn_splits": 1 (default) lets calls of few requests (at most a quarter of the SMs' worth of head-pair
+ * CTAs) split every request's key tiles over up to 8 CTAs of the tcgen05 attention kernel, merged by a second launch.
  * key "trace": see phyai_read_trace.
  * key "wait_limit": iteration bound of the device-side waits on other agents' progress (testing).
  * Unknown key -> INVALID_ARG. */

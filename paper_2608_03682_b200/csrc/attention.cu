@@ -130,6 +130,14 @@ bool attention_mma_supported(const Dims& d) {
   return (d.dh == 64 || d.dh == 128 || d.dh == 256) && d.S <= QROWS;
 }
 
+cudaError_t launch_attention_merge(int* status, const float* part_o, const float* part_ml, __nv_bfloat16* out, int rows_pad,
+                                   int num_splits, const Dims& d, int batch, cudaStream_t st) {
+  dim3 g2(d.S, d.Hq, batch);
+  if (d.dh == 256) return launch_pdl(k_attn_merge<256>, g2, dim3(128), 0, st, status, part_o, part_ml, out, rows_pad, num_splits, d.S, d.Hq);
+  if (d.dh == 128) return launch_pdl(k_attn_merge<128>, g2, dim3(128), 0, st, status, part_o, part_ml, out, rows_pad, num_splits, d.S, d.Hq);
+  return launch_pdl(k_attn_merge<64>, g2, dim3(128), 0, st, status, part_o, part_ml, out, rows_pad, num_splits, d.S, d.Hq);
+}
+
 int attention_pick_splits(const Dims& d, int batch, int max_prefix) {
   const int ctas = batch * d.Hq;
   int want = (2 * 148 + ctas - 1) / ctas;

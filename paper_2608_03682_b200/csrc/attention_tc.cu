@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t Ks = base, Vs = Ks + NKV * KV_BYTES;
 
-  unsigned long long* const trc = a.trace ? a.trace + (size_t)(blockIdx.y * gridDim.x + blockIdx.x) * 16 : nullptr;
+  unsigned long long* const trc = a.trace ? a.trace + (size_t)((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 16 : nullptr;
   if (tid == 0) trace_stamp(trc, 0);
   // Programmatic dependent launch: barriers and tensor memory are set up while the kernel before this one (the q|k|v
   // projection) still runs; the first access to anything it wrote comes after pdl_wait().
@@ -102,9 +102,28 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
   const Request r = *a.rq;
   const int p0 = r.cu_lens[b], P = r.cu_lens[b + 1] - p0;
   const int Tp = (P + KTC - 1) / KTC;
-  // Tile 0 is the suffix (this request's own <= 64 keys, built below while the first prefix tile is in
-  // flight); tile t >= 1 is prefix keys [(t-1) * 64, t * 64).  Softmax does not care about the order.
-  const int T = Tp + 1;
+  // Key tile 0 is the suffix (this request's own <= 64 keys); key tile g >= 1 is prefix keys [(g-1) * 64, g * 64).
+  // Softmax does not care about the order.  With num_splits > 1 (grids far below one wave: few requests) the CTA takes
+  // key tiles [g_lo, g_lo + T) of the Tp + 1 and leaves its unnormalised result for the merge kernel.
+  const int ns = a.num_splits > 1 ? a.num_splits : 1, split = blockIdx.z;
+  const int g_lo = (int)(((long long)(Tp + 1) * split) / ns);
+  const int T = (int)(((long long)(Tp + 1) * (split + 1)) / ns) - g_lo;
+  if (T <= 0) {
+    // a request with fewer key tiles than splits: this range is empty, the merge kernel skips it
+    if (tid >= 160) {
+      const int row = tid - 160, hl = row >> 6, i = row & 63;
+      if (i < S) {
+        const size_t slab = ((size_t)(b * d.Hq + head0 + hl) * ns + split) * QROWS + i;
+        a.part_ml[slab * 2] = -INFINITY, a.part_ml[slab * 2 + 1] = 0.f;
+      }
+    }
+    __syncthreads();
+    if (warp == 4) {
+      tc_fence_after();
+      tmem_dealloc(tmem_base, COLS);
+    }
+    return;
+  }
 
   // ---- loader state (warps 0-3): warps 0-1 stream K tiles, warps 2-3 stream V tiles -----------------
   const bool is_v = warp >= 2;
@@ -114,10 +133,11 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
   const uint8_t* G = reinterpret_cast<const uint8_t*>(r.prefix_kv) +
                      (((size_t)(a.layer * 2 + (is_v ? 1 : 0)) * r.kv_tokens + p0) * d.Hkv + hk) * (DH * 2) + (size_t)lc * 16;
   const uint32_t tile_base = (is_v ? Vs : Ks) + (uint32_t)(lc >> 3) * KV_BLOCK;
-  auto issue = [&](int t) {                  // t >= 1
+  auto issue = [&](int t) {                  // local tile t of a prefix key tile (g_lo + t >= 1)
+    const int gt = g_lo + t;
     const uint32_t tb = tile_base + (uint32_t)(t % NKV) * KV_BYTES;
-    const int rows = min(KTC, P - (t - 1) * KTC);
-    const uint8_t* g0 = G + (size_t)(t - 1) * KTC * kv_stride;
+    const int rows = min(KTC, P - (gt - 1) * KTC);
+    const uint8_t* g0 = G + (size_t)(gt - 1) * KTC * kv_stride;
 #pragma unroll 8
     for (int row = r0; row < KTC; row += 2) {
       const bool ok = row < rows;            // rows past the prefix are zero-filled
@@ -135,16 +155,20 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     // earlier anyway, and it keeps the waited barrier from running a whole phase ahead of the parity wait.
     uint64_t* full = is_v ? v_full : k_full;
     {
-      // tile 0 = this request's own keys / values (rotated bf16 from the QKV epilogue); rows >= S are zero-filled
-      const uint8_t* src = reinterpret_cast<const uint8_t*>(is_v ? a.vr : a.kr) + ((size_t)(b * d.Hkv + hk) * S) * (DH * 2) +
-                           (size_t)lc * 16;
+      if (g_lo == 0) {
+        // key tile 0 = this request's own keys / values (rotated bf16 from the QKV epilogue); rows >= S are zero-filled
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(is_v ? a.vr : a.kr) + ((size_t)(b * d.Hkv + hk) * S) * (DH * 2) +
+                             (size_t)lc * 16;
 #pragma unroll 8
-      for (int row = r0; row < KTC; row += 2) {
-        const bool ok = row < S;
-        cp_async16(tile_base + (uint32_t)row * 128 + (uint32_t)(((lc & 7) ^ (row & 7)) << 4),
-                   src + (size_t)(ok ? row : 0) * (DH * 2), ok ? 16u : 0u);
+        for (int row = r0; row < KTC; row += 2) {
+          const bool ok = row < S;
+          cp_async16(tile_base + (uint32_t)row * 128 + (uint32_t)(((lc & 7) ^ (row & 7)) << 4),
+                     src + (size_t)(ok ? row : 0) * (DH * 2), ok ? 16u : 0u);
+        }
+        cp_async_commit();
+      } else {
+        issue(0);
       }
-      cp_async_commit();
       // The prefix tiles are requested only after tile 0 has landed: every CTA of the grid starts at the same time,
       // and requests issued together share the SM's ingest bandwidth, which would delay the data needed first.
       cp_async_wait<0>();
@@ -279,14 +303,15 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
     for (int t = 0; t < T; ++t) {
       mbar_wait(smem_u32(&s_full[t & 1]), (uint32_t)(t >> 1) & 1u, wc);
       tc_fence_after();
-      const int valid = t == 0 ? S : min(KTC, P - (t - 1) * KTC);
+      const int gt = g_lo + t;
+      const int valid = gt == 0 ? S : min(KTC, P - (gt - 1) * KTC);
       float s[KTC];
       tmem_ld64(tmem_s + (uint32_t)(t & 1) * KTC + lane_addr, s);
       if (valid < KTC) {
 #pragma unroll
         for (int c = 0; c < KTC; ++c) s[c] = c < valid ? s[c] : -INFINITY;
       }
-      if (causal_row && t == 0) {             // the state token sees, of the suffix, only itself
+      if (causal_row && gt == 0) {            // the state token sees, of the suffix, only itself
 #pragma unroll
         for (int c = 1; c < KTC; ++c) s[c] = -INFINITY;
       }
@@ -341,7 +366,38 @@ __global__ void __launch_bounds__(288, 1) k_attn_tc(const AttnArgs a) {
         __all_sync(0xffffffffu, mbar_wait(smem_u32(&pv_done[(T - 1) & 1]), (uint32_t)((T - 1) >> 1) & 1u, wc));
     tc_fence_after();
     if (st == 0) trace_stamp(trc, 6);
-    if (a.rows_pad > 0) {
+    if (ns > 1) {
+      // Split key range: the unnormalised accumulator rows (fp32) and (running maximum in log2 units, sum) of this
+      // range go to the merge kernel.  A row is 4 DH bytes of global memory: staged per warp (64 columns = 256 bytes
+      // per row at a time, 16-byte chunks XOR-swizzled by the row) and copied out with coalesced 16-byte stores.
+      const int i0 = (q * 32) & 63;
+      const int nrow = okf ? max(0, min(32, S - i0)) : 0;
+      const size_t slab = ((size_t)(b * d.Hq + head0 + hl) * ns + split) * QROWS + i0;   // first row of this warp
+      if (lane < nrow) {
+        a.part_ml[(slab + lane) * 2] = m;
+        a.part_ml[(slab + lane) * 2 + 1] = l;
+      }
+      const uint32_t ostage = Ks + (uint32_t)q * 8192u;
+#pragma unroll 1
+      for (int c = 0; c < DH; c += 64) {
+        float o[64];
+        tmem_ld64(tmem_o + lane_addr + (uint32_t)c, o);
+#pragma unroll
+        for (int e = 0; e < 64; e += 4)
+          asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(ostage + (uint32_t)lane * 256u + (uint32_t)((((e >> 2) ^ (lane & 15))) << 4)),
+                       "f"(o[e]), "f"(o[e + 1]), "f"(o[e + 2]), "f"(o[e + 3])
+                       : "memory");
+        __syncwarp();
+        for (int idx = lane; idx < nrow * 16; idx += 32) {
+          const int rr = idx >> 4, ch = idx & 15;
+          float4 v;
+          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                       : "r"(ostage + (uint32_t)rr * 256u + (uint32_t)((ch ^ (rr & 15)) << 4)) : "memory");
+          *reinterpret_cast<float4*>(a.part_o + (slab + rr) * DH + c + ch * 4) = v;
+        }
+        __syncwarp();
+      }
+    } else if (a.rows_pad > 0) {
       // O / l -> bf16 in the tiled layout of the O projection's input.  A thread holds one row; its 128 bytes of a
       // 64-channel k-chunk go to a staging block of the warp (the K buffers are free: every MMA has completed) at the
       // position they have in global memory, where the warp's 32 rows of a k-chunk are one contiguous range, and the
@@ -415,13 +471,28 @@ constexpr size_t attn_tc_smem() {
 
 }  // namespace
 
+// Key-range splits of the tcgen05 attention kernel: only for grids far below one wave (few requests), at most 8 and
+// at most the key tiles of the longest prefix (a request with fewer key tiles leaves some of its ranges empty).
+int attention_tc_splits(const Dims& d, int batch, int n_sm, int max_prefix) {
+  const int ctas = batch * (d.Hq / 2);
+  int want = n_sm / (ctas > 0 ? ctas : 1);
+  const int tiles = (max_prefix + KTC - 1) / KTC + 1;
+  if (want > tiles) want = tiles;
+  if (want > 8) want = 8;
+  // (measured on the pi0-shaped expert, 816-token prefixes: 4 requests 12.2 -> 11.3 ms per call with 8 ranges,
+  // 8 requests 12.9 -> 12.6 ms with 4, 16 requests 16.8 -> 17.6 ms with 2: the merge kernel and the fp32 partials cost
+  // more than two ranges save)
+  return want < 4 ? 1 : want;
+}
+
 bool attention_tc_supported(const Dims& d) {
   return d.dh == 256 && d.S <= 64 && d.Hq % 2 == 0 && (d.Hq / d.Hkv) % 2 == 0;
 }
 
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, const int* order, unsigned wait_limit, cudaStream_t st, unsigned long long* trace) {
+                                int batch, const int* order, unsigned wait_limit, cudaStream_t st, unsigned long long* trace,
+                                int num_splits, float* scratch) {
   static PerDeviceOnce once;
   if (once.needed()) {
     cudaError_t e = cudaFuncSetAttribute(k_attn_tc<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -431,9 +502,15 @@ cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloa
   }
   AttnArgs a{};
   a.rq = rq, a.status = status, a.qr = qr, a.kr = kr, a.vr = vr, a.layer = layer, a.out = out_tiled, a.rows_pad = rows_pad;
-  a.num_splits = 1, a.d = d, a.wait_limit = wait_limit, a.order = order, a.trace = trace;
-  dim3 grid(d.Hq / 2, batch);
-  return launch_pdl(k_attn_tc<256>, grid, dim3(288), attn_tc_smem<256>(), st, a);
+  if (num_splits > 1 && !scratch) return cudaErrorInvalidValue;
+  a.num_splits = num_splits > 1 ? num_splits : 1, a.d = d, a.wait_limit = wait_limit, a.order = order, a.trace = trace;
+  a.part_o = scratch;
+  a.part_ml = scratch ? scratch + (size_t)batch * d.Hq * a.num_splits * QROWS * d.dh : nullptr;
+  dim3 grid(d.Hq / 2, batch, a.num_splits);
+  cudaError_t e = launch_pdl(k_attn_tc<256>, grid, dim3(288), attn_tc_smem<256>(), st, a);
+  if (e == cudaSuccess && a.num_splits > 1)
+    e = launch_attention_merge(status, a.part_o, a.part_ml, out_tiled, rows_pad, a.num_splits, d, batch, st);
+  return e;
 }
 
 }  // namespace phyai

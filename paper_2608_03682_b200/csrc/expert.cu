@@ -108,7 +108,7 @@ struct phyai_expert {
   __nv_bfloat16* p_gu_all = nullptr;        // gate/up interleaved in groups of 64 channels, all layers
   __nv_bfloat16* p_gu16 = nullptr;          // gate/up interleaved in groups of 16 channels (persistent tile GEMM)
   __nv_bfloat16* p_qkv16 = nullptr;         // q|k|v with the rows of every tile interleaved in groups of 16 (the same kernel)
-  int use_persistent_gu = 1, use_persistent_qkv = 1;
+  int use_persistent_gu = 1, use_persistent_qkv = 1, use_attn_splits = 1;
   float *s_qkv_all = nullptr, *s_o_all = nullptr, *s_g_all = nullptr, *s_u_all = nullptr, *s_d_all = nullptr;
   __nv_bfloat16 *xn64 = nullptr, *attn64 = nullptr, *m64 = nullptr, *u64 = nullptr;
   __nv_bfloat16 *qr64 = nullptr, *kr64 = nullptr, *vr64 = nullptr;
@@ -589,11 +589,13 @@ phyai_status_t enqueue_loop(phyai_expert* h, int batch, int n, const Tables& t, 
         simt_gemm(g);
       }
       if (attn_tc) {
+        const int tsp = (h->use_attn_splits && h->attn_scratch) ? attention_tc_splits(d, batch, h->n_sm, (int)h->cfg.max_prefix_len) : 1;
         cudaError_t e = launch_attention_tc(h->rq, h->status, h->qr_big, h->kr_big, h->vr_big, l, h->attn_t, h->Mpad, d,
                                             batch, h->order, h->wait_limit, st,
-                                            (h->trace && h->trace_all_from > 0 && cnt == h->trace_all_from && batch * (d.Hq / 2) <= TRACE_SLOTS) ? h->trace : nullptr);
+                                            (h->trace && h->trace_all_from > 0 && cnt == h->trace_all_from && batch * (d.Hq / 2) * tsp <= TRACE_SLOTS) ? h->trace : nullptr,
+                                            tsp, h->attn_scratch);
         if (e != cudaSuccess) return fail(PHYAI_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(e));
-        ++cnt;
+        cnt += tsp > 1 ? 2 : 1;
       } else if (attn_cluster) {
         // few requests: 8 key ranges per head in a cluster of 8 CTAs, merged through distributed shared memory
         const AttnOproj op{h->p_o[l], h->s_o[l], gate, h->slab, (size_t)M * D};
@@ -1059,6 +1061,10 @@ phyai_status_t phyai_expert_create(const phyai_expert_config_t* cfg, const phyai
         for (int bb = 1; bb <= (int)cfg->max_batch; ++bb) {
           const size_t n = attention_scratch_floats(d, bb, attention_pick_splits(d, bb, (int)cfg->max_prefix_len));
           need = n > need ? n : need;
+          if (attention_tc_supported(d)) {
+            const size_t n2 = attention_scratch_floats(d, bb, attention_tc_splits(d, bb, h->n_sm, (int)cfg->max_prefix_len));
+            need = n2 > need ? n2 : need;
+          }
         }
         if (need) ST(h->alloc(&h->attn_scratch, need, true));
       }
@@ -1298,8 +1304,8 @@ phyai_status_t phyai_set_option(phyai_expert_t* h, const char* key, int64_t valu
     h->trace = h->trace_buf;
     return PHYAI_OK;
   }
-  if (!strcmp(key, "use_persistent_gu") || !strcmp(key, "use_persistent_qkv")) {
-    (!strcmp(key, "use_persistent_gu") ? h->use_persistent_gu : h->use_persistent_qkv) = value != 0;
+  if (!strcmp(key, "use_persistent_gu") || !strcmp(key, "use_persistent_qkv") || !strcmp(key, "use_attn_splits")) {
+    (!strcmp(key, "use_persistent_gu") ? h->use_persistent_gu : !strcmp(key, "use_attn_splits") ? h->use_attn_splits : h->use_persistent_qkv) = value != 0;
     for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
     h->graphs.clear();
     return PHYAI_OK;

@@ -183,7 +183,13 @@ cudaError_t launch_attention_b1(const Request* rq, int* status, const __nv_bfloa
 int attention_b1_ctas(const Dims& d, int batch, int hpc);
 cudaError_t launch_attention_tc(const Request* rq, int* status, const __nv_bfloat16* qr, const __nv_bfloat16* kr,
                                 const __nv_bfloat16* vr, int layer, __nv_bfloat16* out_tiled, int rows_pad, const Dims& d,
-                                int batch, const int* order, unsigned wait_limit, cudaStream_t st, unsigned long long* trace = nullptr);
+                                int batch, const int* order, unsigned wait_limit, cudaStream_t st, unsigned long long* trace = nullptr,
+                                int num_splits = 1, float* scratch = nullptr);
+// key-range splits for grids far below one wave (1 = none)
+int attention_tc_splits(const Dims& d, int batch, int n_sm, int max_prefix);
+// combines split-KV partials ([b][head][split][64][dh] unnormalised rows, then [..][64][2] (max in log2 units, sum))
+cudaError_t launch_attention_merge(int* status, const float* part_o, const float* part_ml, __nv_bfloat16* out, int rows_pad,
+                                   int num_splits, const Dims& d, int batch, cudaStream_t st);
 
 // ---- tcgen05 GEMM ------------------------------------------------------------------------------
 enum : int { TC_STORE = 0, TC_RESID = 1, TC_GEGLU = 2, TC_BIAS_ROWMAP = 3, TC_QKV_ROT = 4, TC_GEGLU_IL = 5 };

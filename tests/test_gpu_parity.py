@@ -243,6 +243,38 @@ def test_persistent_tile_gemm_with_more_tiles_than_sms(cond, dtype, head_dim, n_
     assert rel_err(out, plain) <= (BAR["bf16"] if dtype != "w8a8e4m3" else 0.15), rel_err(out, plain)
 
 
+@pytest.mark.parametrize("batch", [5, 9, 20])
+def test_tcgen05_attention_with_split_key_ranges_matches_oracle_and_the_unsplit_kernel(batch):
+    """Few requests: the tcgen05 attention kernel splits every request's key tiles over up to 8 CTAs per head pair and a
+    merge kernel combines the partial results.  Ragged prefixes from 0 (a single key tile: all ranges but one are
+    empty) to 200 (four tiles); compared with the oracle per request and with the unsplit kernel."""
+    cfg = small_bf16_config("pi0", max_batch=batch, max_prefix_len=200, head_dim=256, n_q_heads=4)
+    lens = [0, 200, 63, 64, 129, 1, 65, 199, 128][:batch] + [int(x) for x in synth.make_ragged_lengths(17, max(0, batch - 9), 0, 200)]
+    lens = lens[:batch]
+    W = synth.make_weights(cfg, 17, std=0.05)
+    kvs = [synth.make_prefix_kv(cfg, 17, int(p), b) for b, p in enumerate(lens)]
+    packed, cu = synth.pack_prefix_kv(kvs)
+    states = torch.stack([synth.make_state(cfg, 17, b) for b in range(batch)])
+    noise = torch.stack([synth.make_noise(cfg, 17, b) for b in range(batch)])
+    args = (packed.cuda(), torch.from_numpy(cu).cuda(), states.cuda(), noise.cuda(), 3)
+    with binding.Expert(cfg, binding.weights_to_device(W)) as ex:
+        n_split = ex.launches_per_call(batch, 3)
+        out = ex.denoise_batched(*args).double().cpu().numpy()
+        assert ex.poll_status() == 0
+        n_split = ex.launches_per_call(batch, 3)
+        ex.set_option("use_attn_splits", 0)
+        plain = ex.denoise_batched(*args).double().cpu().numpy()
+        assert ex.poll_status() == 0
+        n_plain = ex.launches_per_call(batch, 3)
+    # the split path adds one merge launch per layer and step (3 layers x 3 steps) where it is chosen
+    assert n_split == n_plain + (9 if batch * 2 <= 148 // 4 else 0), (n_split, n_plain)
+    Wf = O.Weights(W)
+    for b in range(min(batch, 9)):
+        ref = O.denoise(cfg, Wf, kvs[b], int(lens[b]), states[b], noise[b], 3)
+        assert rel_err(out[b], ref) <= BAR["bf16"], (b, lens[b], rel_err(out[b], ref))
+    assert rel_err(out, plain) <= BAR["bf16"], rel_err(out, plain)
+
+
 def test_fp32_ragged_batch_matches_oracle_per_request():
     cfg = synth.ExpertConfig(n_layers=2, width=64, mlp_dim=96, n_q_heads=2, n_kv_heads=2, head_dim=16, state_dim=3,
                              action_dim=4, horizon=6, has_state_token=True, max_prefix_len=30, max_batch=4,
