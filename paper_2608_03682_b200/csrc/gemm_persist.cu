@@ -1,6 +1,6 @@
 // Persistent tile GEMM for many token tiles: one CTA per SM walks over 128-row x 256-token output tiles, and the
 // epilogue of one tile runs while the tensor cores work on the next.  Two epilogues: the gate / up projection with
-// GeGLU (Sec. 3.2: the MLP's first layer, m = gelu(x Wg) * (x Wu)) and the fused q | k | v projection with the rotary
+// GeGLU (the expert MLP's first layer, m = gelu(x Wg) * (x Wu)) and the fused q | k | v projection with the rotary
 // embedding (the attention kernel's operands, bf16).
 //
 // Why a kernel of its own.  With one 256-token x 256-row tile per CTA (two accumulators of 128 rows) the 512

@@ -14,8 +14,10 @@
 //
 // A CTA computes NA (1 or 2) 128-channel tiles against one NT-token tile (NT = 64, 128, 192 or 256): with NA = 2
 // and NT = 256 a k-step moves 64 KB for 8 MMAs of 128 clocks, i.e. 64 bytes per clock.  One SM alone ingests that
-// (~126 GB/s measured); with all SMs streaming the measured rate is 38-40 bytes per clock per SM, which makes the
-// main loop crossbar-bound at ~1600 clocks per k-step.  A single 128 x 256 tile would need 96 bytes per clock.
+// (~126 GB/s measured); with all SMs streaming the main loop was measured at ~1180 clocks per k-step (55 bytes per
+// clock per SM, 87 % of the tensor rate).  A single 128 x 256 tile would need 96 bytes per clock.  What a 256 x 256
+// tile loses is its epilogue and set-up: they cannot overlap a next tile because the accumulators fill the tensor
+// memory (see gemm_persist.cu for the projections with more tiles than SMs).
 //
 // Warp roles (800 threads): warps 0..7 = copy producers (the copies of all stages are dealt round
 // robin to the eight warps: one warp's bulk copies complete one at a time, about 0.5 us each whatever
