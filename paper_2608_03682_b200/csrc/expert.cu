@@ -253,8 +253,10 @@ constexpr int TRACE_SLOTS = 4096, TRACE_STAMPS = 16;
 int pick_nt(int M) { return M <= 64 ? 64 : (M <= 1024 ? 128 : 256); }
 
 // Token-tile width and split-K factor of a residual GEMM (N = width, large token counts): the pair that minimises
-// waves x (k-chunks per CTA x clocks per k-chunk + epilogue).  Clocks per k-chunk follow the measured SM ingest of
-// ~39 bytes per clock: 64 KB per k-chunk at 256 tokens, 56 KB at 192.
+// waves x (k-chunks per CTA x clocks per k-chunk + epilogue).  The constants are a fit to launch durations (they
+// put part of the exposed set-up and epilogue into the k-chunk term: the main loop alone runs at ~1180 clocks per
+// 64 KB k-chunk); the choice they make for the pi-shaped expert at 64 requests, 192-token tiles with two k-ranges,
+// is the measured optimum.
 void pick_resid_tiling(int M, int Mpad, int N, int KC, int n_sm, int* nt_out, int* splits_out) {
   const int nts[2] = {256, 192};
   double best = 1e30;
